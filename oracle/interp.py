@@ -1,0 +1,161 @@
+"""Float64 interpreter of an operator DAG (test infrastructure only).
+
+Every node is materialised in float64 and evaluated from the operator's plain
+definition, in the order the spec lists the nodes.  There is no fusion, no
+tiling and no reordering: what the fused GPU kernels must reproduce is exactly
+this composition (fusion changes the schedule, not the mathematics).
+
+Operator classes follow the paper's Table 1: elementwise (add, sub, mul, div,
+sqrt, sin, cos, relu, ...), reduction (sum, mean, softmax, ...) and
+compute-intensive (matmul, conv).
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+from scipy.special import erf as _erf
+
+from .graph import Graph, parse, UNARY, BINARY
+
+
+# ---- elementwise (Table 1, "Elementwise") ---------------------------------------------------
+
+def relu(x):
+    return np.maximum(x, 0.0)
+
+
+def sigmoid(x):
+    return 1.0 / (1.0 + np.exp(-x))
+
+
+def gelu_tanh(x):
+    # 0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))
+    return 0.5 * x * (1.0 + np.tanh(math.sqrt(2.0 / math.pi) * (x + 0.044715 * x * x * x)))
+
+
+def gelu_erf(x):
+    # 0.5 x (1 + erf(x / sqrt 2))
+    return 0.5 * x * (1.0 + _erf(x / math.sqrt(2.0)))
+
+
+_UNARY_FN = {
+    "relu": relu, "gelu_tanh": gelu_tanh, "gelu_erf": gelu_erf, "sigmoid": sigmoid,
+    "exp": np.exp, "tanh": np.tanh, "sqrt": np.sqrt, "sin": np.sin, "cos": np.cos,
+    "neg": np.negative, "abs": np.abs,
+}
+_BINARY_FN = {
+    "add": np.add, "sub": np.subtract, "mul": np.multiply, "div": np.divide,
+    "max": np.maximum, "min": np.minimum,
+}
+
+
+# ---- row reductions (Table 1, "Reduction") --------------------------------------------------
+
+def row_sum(x):
+    return x.sum(axis=1, keepdims=True)
+
+
+def row_mean(x):
+    return x.sum(axis=1, keepdims=True) / x.shape[1]
+
+
+def row_max(x):
+    return x.max(axis=1, keepdims=True)
+
+
+def row_softmax(x):
+    # y_ij = exp(x_ij - m_i) / sum_j exp(x_ij - m_i), m_i the row maximum
+    e = np.exp(x - x.max(axis=1, keepdims=True))
+    return e / e.sum(axis=1, keepdims=True)
+
+
+def row_layernorm(x, gamma, beta, eps):
+    # mu_i = mean_j x_ij ; v_i = mean_j (x_ij - mu_i)^2 (biased) ;
+    # y_ij = (x_ij - mu_i) / sqrt(v_i + eps) * gamma_j + beta_j
+    mu = x.sum(axis=1, keepdims=True) / x.shape[1]
+    d = x - mu
+    v = (d * d).sum(axis=1, keepdims=True) / x.shape[1]
+    return d / np.sqrt(v + eps) * gamma.reshape(1, -1) + beta.reshape(1, -1)
+
+
+# ---- contractions (Table 1, "ComputeIntensive") ---------------------------------------------
+
+def gemm(a, b):
+    # C_ij = sum_k A_ik B_kj for row-major A[M,K], B[K,N]
+    return np.matmul(a, b)
+
+
+def conv2d(x, w, stride, pad):
+    """Y[n,k,h,w] = sum_{c,r,s} X[n,c,h*stride-pad+r, w*stride-pad+s] * Wt[k,c,r,s].
+
+    Cross-correlation over an NCHW input with zeros outside the image, as in
+    the paper's convolution case study (input row h - P + kh, column w - P + kw,
+    taps outside the image contribute nothing; output index ((n*K+k)*H+h)*W+w).
+    For each tap (r, s) the strided window of the zero-padded input is
+    contracted over channels with the tap's [K,C] weight slice.
+    """
+    n, c, h, wd = x.shape
+    k, _, kr, ks = w.shape
+    ho = (h + 2 * pad - kr) // stride + 1
+    wo = (wd + 2 * pad - ks) // stride + 1
+    xp = np.zeros((n, c, h + 2 * pad, wd + 2 * pad), dtype=np.float64)
+    xp[:, :, pad:pad + h, pad:pad + wd] = x
+    y = np.zeros((n, k, ho, wo), dtype=np.float64)
+    for r in range(kr):
+        for s in range(ks):
+            win = xp[:, :, r:r + (ho - 1) * stride + 1:stride, s:s + (wo - 1) * stride + 1:stride]
+            y += np.einsum("nchw,kc->nkhw", win, w[:, :, r, s], optimize=True)
+    return y
+
+
+# ---- interpreter ----------------------------------------------------------------------------
+
+def run_nodes(spec, inputs: dict) -> dict:
+    """Evaluate every node; returns name -> float64 array for all nodes (inputs included).
+
+    ``inputs`` maps input names to arrays already widened to float64 (the
+    stored float32 / bfloat16 values, exactly).
+    """
+    g = spec if isinstance(spec, Graph) else parse(spec)
+    val = {}
+    for name, node in g.nodes.items():
+        if node.op == "input":
+            a = np.asarray(inputs[name], dtype=np.float64)
+            if tuple(a.shape) != tuple(node.shape):
+                raise ValueError(f"input {name}: expected shape {node.shape}, got {a.shape}")
+            val[name] = a
+            continue
+        args = [val[a] if isinstance(a, str) else float(a) for a in node.args]
+        op = node.op
+        if op in UNARY:
+            out = _UNARY_FN[op](args[0])
+        elif op in BINARY:
+            out = _BINARY_FN[op](args[0], args[1])
+            out = np.broadcast_to(out, node.shape)
+        elif op == "row_softmax":
+            out = row_softmax(args[0])
+        elif op == "row_sum":
+            out = row_sum(args[0])
+        elif op == "row_mean":
+            out = row_mean(args[0])
+        elif op == "row_max":
+            out = row_max(args[0])
+        elif op == "row_layernorm":
+            out = row_layernorm(args[0], args[1], args[2], node.attrs["eps"])
+        elif op == "gemm":
+            out = gemm(args[0], args[1])
+        elif op == "conv2d":
+            out = conv2d(args[0], args[1], node.attrs["stride"], node.attrs["pad"])
+        else:  # pragma: no cover - parse() rejects unknown operators
+            raise ValueError(op)
+        assert tuple(out.shape) == tuple(node.shape), (name, out.shape, node.shape)
+        val[name] = np.asarray(out, dtype=np.float64)
+    return val
+
+
+def run(spec, inputs: dict) -> dict:
+    """Evaluate the graph; returns output name -> float64 array (no output rounding)."""
+    g = spec if isinstance(spec, Graph) else parse(spec)
+    val = run_nodes(g, inputs)
+    return {name: val[name] for name, _ in g.outputs}

@@ -1,0 +1,120 @@
+"""The benchmark chains as operator-DAG spec text plus the recipe for their inputs.
+
+Each entry gives the spec, and per input the sampling law, so that the CUDA
+library and the CPU oracle are fed identical seeded tensors.  Input ``i`` of a
+config is drawn from stream ``i`` of the config's seed.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+from .tensors import make_tensor
+
+
+def _n(std=1.0, mean=0.0):
+    return {"kind": "normal", "mean": mean, "std": std}
+
+
+def _u(lo, hi):
+    return {"kind": "uniform", "lo": lo, "hi": hi}
+
+
+def gemm_bias_relu(m=256, k=256, n=256):
+    spec = f"""hct 1
+input a    f32 [{m},{k}]
+input b    f32 [{k},{n}]
+input bias f32 [{n}]
+node  t0 = gemm(a, b)
+node  t1 = add(t0, bias)
+node  t2 = relu(t1)
+output t2 f32
+"""
+    laws = {"a": _u(-1, 1), "b": _u(-1, 1), "bias": _u(-1, 1)}
+    return spec, laws
+
+
+def softmax_layernorm_chain(r=8192, c=4096):
+    spec = f"""hct 1
+input x     f32 [{r},{c}]
+input scale f32 [{c}]
+input shift f32 [{c}]
+input gamma f32 [{c}]
+input beta  f32 [{c}]
+node  t0 = mul(x, scale)
+node  t1 = add(t0, shift)
+node  t2 = gelu_tanh(t1)
+node  t3 = row_softmax(t2)
+node  t4 = row_layernorm(t3, gamma, beta, eps=1e-5)
+output t4 f32
+"""
+    laws = {"x": _n(), "scale": _n(0.1, 1.0), "shift": _n(0.1), "gamma": _n(0.1, 1.0), "beta": _n(0.1)}
+    return spec, laws
+
+
+def gemm_bf16_gelu_residual(m=8192, k=4096, n=4096):
+    spec = f"""hct 1
+input x    bf16 [{m},{k}]
+input w    bf16 [{k},{n}]
+input bias bf16 [{n}]
+input r    bf16 [{m},{n}]
+node  t0 = gemm(x, w)
+node  t1 = add(t0, bias)
+node  t2 = gelu_tanh(t1)
+node  t3 = add(t2, r)
+output t3 bf16
+"""
+    laws = {"x": _n(), "w": _n(1.0 / math.sqrt(k)), "bias": _n(0.1), "r": _n()}
+    return spec, laws
+
+
+def conv_bn_relu(n=32, c=128, h=56, w=56, k=128, ksize=3, stride=1, pad=1):
+    spec = f"""hct 1
+input x     bf16 [{n},{c},{h},{w}]
+input wt    bf16 [{k},{c},{ksize},{ksize}]
+input scale f32  [{k},1,1]
+input shift f32  [{k},1,1]
+node  t0 = conv2d(x, wt, stride={stride}, pad={pad})
+node  t1 = mul(t0, scale)
+node  t2 = add(t1, shift)
+node  t3 = relu(t2)
+output t3 bf16
+"""
+    laws = {"x": _n(), "wt": _n(math.sqrt(2.0 / (c * ksize * ksize))), "scale": _u(0.5, 1.5), "shift": _n(0.1)}
+    return spec, laws
+
+
+CONFIGS = {
+    "c1_gemm_bias_relu_f32": (gemm_bias_relu, {}),
+    "c2_softmax_layernorm_chain": (softmax_layernorm_chain, {}),
+    "c3_gemm_bf16_gelu_residual": (gemm_bf16_gelu_residual, {}),
+    "c4_conv_bn_relu_bf16": (conv_bn_relu, {}),
+}
+
+
+def parse_inputs(spec: str):
+    """(name, dtype, shape) of every ``input`` line, in order.  Text handling only."""
+    out = []
+    for line in spec.splitlines():
+        line = line.split("#", 1)[0].strip()
+        if line.startswith("input"):
+            _, name, dtype, shape = line.split(None, 3)
+            dims = tuple(int(t) for t in shape.strip()[1:-1].split(",") if t.strip())
+            out.append((name, dtype, dims))
+    return out
+
+
+def draw_inputs(spec: str, laws: dict, seed: int = 0) -> dict:
+    """name -> array (float32, or uint16 bfloat16 patterns) for every input of ``spec``."""
+    tensors = {}
+    for stream, (name, dtype, dims) in enumerate(parse_inputs(spec)):
+        tensors[name] = make_tensor(laws[name], dims, dtype, seed, stream)
+    return tensors
+
+
+def get_config(name: str, **overrides):
+    fn, kw = CONFIGS[name]
+    args = dict(kw)
+    args.update(overrides)
+    return fn(**args)
