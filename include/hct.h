@@ -1,0 +1,149 @@
+/*
+ * hct — fused operator-chain execution on one NVIDIA B200 (sm_100a).
+ *
+ * A computation graph is a DAG whose nodes are computations and whose edges
+ * are data flow (paper §3.2).  The operators are the classes of the paper's
+ * Table 1 that dominate fused deep-learning chains: elementwise and
+ * activation, broadcast, row reductions (softmax, layer normalisation, sums),
+ * GEMM and conv2d.  hct_graph_create() reads a text description of such a
+ * graph, checks it (acyclic, operand shapes and dtypes consistent, nothing
+ * dangling — the validity rules of §3.2), partitions it into fused kernels,
+ * generates and compiles them for sm_100a, and returns a handle;
+ * hct_graph_run() launches those kernels on caller-owned device memory.
+ *
+ * There is no CPU execution path: if the device is not compute capability
+ * 10.x, or a kernel cannot be built, the call fails with an error code.
+ *
+ * Spec text (line oriented, '#' starts a comment):
+ *
+ *     hct 1
+ *     input  NAME DTYPE [d0,d1,...]           DTYPE: f32 | bf16, rank 1..4
+ *     node   NAME = OP(arg, ..., key=value)   args: earlier names or (binary ops) a number
+ *     output NAME [DTYPE]                     stored dtype, default f32
+ *
+ *   unary   relu gelu_tanh gelu_erf sigmoid exp tanh sqrt sin cos neg abs
+ *   binary  add sub mul div max min   operands broadcast like numpy; supported
+ *           patterns: equal shapes, [C] against [..,C], [..,1] against [..,C],
+ *           [K,1,1] against [N,K,H,W], a number
+ *   row     row_softmax(x)  row_sum(x)  row_mean(x)  row_max(x)   x: [R,C]; sums give [R,1]
+ *           row_layernorm(x, gamma, beta, eps=1e-5)   biased variance, eps inside the root
+ *   gemm(a, b)            a[M,K] · b[K,N], both row-major, both f32 or both bf16 inputs;
+ *                         bf16 multiplies on tensor cores with fp32 accumulation, f32
+ *                         uses error-compensated TF32 products (or fp32 FMA for shapes
+ *                         the tensor-core path does not take)
+ *   conv2d(x, w, stride=1, pad=0)   x[N,C,H,W], w[K,C,R,S]; cross-correlation, zero padding
+ *
+ * Every computed value is fp32; bf16 inputs are widened exactly; an output
+ * stored as bf16 is rounded to nearest-even once, at the store.
+ *
+ * All tensors are dense, contiguous and row-major (conv2d: NCHW / KCRS).
+ * Pointers passed to hct_graph_run are DEVICE pointers, 16-byte aligned.
+ * Functions return HCT_OK or an error code; the text of the last error on the
+ * calling thread is available from hct_last_error().  No exception crosses
+ * this boundary.
+ */
+#ifndef HCT_H_
+#define HCT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define HCT_API __attribute__((visibility("default")))
+#else
+#define HCT_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hct_graph hct_graph_t; /* opaque; owned by the library until hct_graph_destroy */
+
+typedef enum {
+  HCT_OK = 0,
+  HCT_ERR_INVALID_ARG = 1, /* null pointer, wrong count, misaligned pointer, workspace too small */
+  HCT_ERR_PARSE = 2,       /* spec syntax; message carries the line                         */
+  HCT_ERR_GRAPH = 3,       /* undefined or forward operand (cycle / dangling node), node that
+                              reaches no output, dtype or shape mismatch (paper §3.2)       */
+  HCT_ERR_UNSUPPORTED = 4, /* valid graph outside the supported set; never a CPU fallback   */
+  HCT_ERR_COMPILE = 5,     /* kernel compilation or module load failed                      */
+  HCT_ERR_CUDA = 6,        /* driver error at launch or query; code in the message          */
+  HCT_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired (read by hct_graph_status) */
+  HCT_ERR_ARCH = 8,        /* device is not compute capability 10.x                         */
+  HCT_ERR_OOM = 9
+} hct_status_t;
+
+enum { HCT_F32 = 0, HCT_BF16 = 1 };
+
+/* Device id that asks for planning and kernel compilation only (no CUDA driver
+ * needed); the handle can be queried but not run. */
+#define HCT_DEVICE_NONE (-1)
+
+/*
+ * Build a graph handle from spec text (host memory, spec_len bytes, need not
+ * be NUL-terminated).  Parses and validates the DAG (§3.2), infers shapes,
+ * plans the fused kernels, compiles them for sm_100a and, unless device is
+ * HCT_DEVICE_NONE, loads them on CUDA device `device` (its primary context).
+ * On success *out owns the handle; on failure *out is NULL.
+ * Host-only work plus module loading; no kernel is launched.
+ */
+HCT_API hct_status_t hct_graph_create(const char* spec, size_t spec_len, int device, hct_graph_t** out);
+
+/*
+ * Launch the graph's kernels, in dependency order, on `cuda_stream`
+ * (a cudaStream_t / CUstream; NULL is the default stream).  Does not
+ * synchronise.
+ *   inputs[i]   device pointer to the i-th `input` line's tensor (read only)
+ *   outputs[i]  device pointer to the i-th `output` line's tensor (written)
+ *   workspace   device scratch of at least hct_graph_workspace_bytes() bytes,
+ *               256-byte aligned, caller-owned; may be NULL when that is 0
+ * Outputs must not alias inputs or the workspace.  A handle is used by one
+ * thread at a time.  Errors: HCT_ERR_INVALID_ARG (counts, NULL or misaligned
+ * pointers, small workspace), HCT_ERR_CUDA (launch failure).
+ */
+HCT_API hct_status_t hct_graph_run(hct_graph_t* g, const void* const* inputs, int n_inputs, void* const* outputs,
+                           int n_outputs, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * After the caller has synchronised the stream: reads the handle's device
+ * status word.  HCT_OK, or HCT_ERR_TIMEOUT if a kernel gave up on a bounded
+ * wait (its outputs are then undefined).  Clears the word.
+ */
+HCT_API hct_status_t hct_graph_status(hct_graph_t* g);
+
+/* Release the handle and everything it owns.  NULL is accepted. */
+HCT_API hct_status_t hct_graph_destroy(hct_graph_t* g);
+
+/* ---- queries (host only) ---- */
+HCT_API int hct_graph_num_inputs(const hct_graph_t* g);
+HCT_API int hct_graph_num_outputs(const hct_graph_t* g);
+/* Name (owned by g), dtype (HCT_F32/HCT_BF16), rank and extents of an input (is_output = 0)
+ * or output (is_output = 1) tensor, as inferred from the spec. */
+HCT_API hct_status_t hct_graph_tensor_info(const hct_graph_t* g, int is_output, int idx, const char** name, int* dtype,
+                                   int* rank, int64_t shape[4]);
+HCT_API size_t hct_graph_workspace_bytes(const hct_graph_t* g);
+/* Number of kernel launches one hct_graph_run issues. */
+HCT_API int hct_graph_num_kernels(const hct_graph_t* g);
+/*
+ * Work accounting for roofline figures.  algorithmic_bytes: every graph input
+ * read once and every output written once, plus one write and one read for
+ * each intermediate that no single pass can keep on chip (an edge from a
+ * contraction into a row reduction, or from any node into a contraction).
+ * flops: 2·M·N·K summed over the contractions.
+ */
+HCT_API hct_status_t hct_graph_cost(const hct_graph_t* g, double* algorithmic_bytes, double* flops);
+/* Human-readable fusion plan: one line per kernel with its nodes.  Owned by g. */
+HCT_API const char* hct_graph_plan_text(const hct_graph_t* g);
+/* Generated CUDA source / entry-point name of kernel `idx` (0 <= idx < num_kernels).  Owned by g. */
+HCT_API const char* hct_graph_kernel_source(const hct_graph_t* g, int idx);
+HCT_API const char* hct_graph_kernel_name(const hct_graph_t* g, int idx);
+
+/* Message of the last failing call on this thread ("" if none). */
+HCT_API const char* hct_last_error(void);
+HCT_API const char* hct_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HCT_H_ */

@@ -111,11 +111,13 @@ def conv2d(x, w, stride, pad):
 
 # ---- interpreter ----------------------------------------------------------------------------
 
-def run_nodes(spec, inputs: dict) -> dict:
+def run_nodes(spec, inputs: dict, post=None) -> dict:
     """Evaluate every node; returns name -> float64 array for all nodes (inputs included).
 
     ``inputs`` maps input names to arrays already widened to float64 (the
-    stored float32 / bfloat16 values, exactly).
+    stored float32 / bfloat16 values, exactly).  ``post``, if given, is applied
+    to every computed node (used only to study how a graph reacts to rounding
+    each intermediate, never for expected values).
     """
     g = spec if isinstance(spec, Graph) else parse(spec)
     val = {}
@@ -150,7 +152,8 @@ def run_nodes(spec, inputs: dict) -> dict:
         else:  # pragma: no cover - parse() rejects unknown operators
             raise ValueError(op)
         assert tuple(out.shape) == tuple(node.shape), (name, out.shape, node.shape)
-        val[name] = np.asarray(out, dtype=np.float64)
+        out = np.asarray(out, dtype=np.float64)
+        val[name] = post(out) if post is not None else out
     return val
 
 

@@ -1,0 +1,68 @@
+"""Writes workloads/sweep_specs.json: the 200 random operator DAGs of the graph-augmentation sweep.
+
+    python -m oracle.make_sweep
+
+For seed 0..199 the generator (workloads.random_dag, after the paper's Algorithm 1) is asked
+for a graph; the graph is then checked for data-flow validity in the numerical sense: it is
+evaluated by the oracle on a 4-row proxy twice, once exactly and once with every node rounded
+to float32, and it is rolled back and redrawn (next attempt number) when any value is
+non-finite or above 1e30, or when rounding alone already moves the result by more than 2e-6
+of the row's magnitude, i.e. when no float32 implementation could be compared at 1e-5.
+Calls only workloads/ and oracle/.
+"""
+from __future__ import annotations
+
+import json
+import os
+
+import numpy as np
+
+from oracle import graph as ograph
+from oracle import interp
+from workloads import configs, random_dag, tensors
+
+N_SEEDS = 200
+PROXY_ROWS = 4
+OUT = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "workloads", "sweep_specs.json")
+
+
+def well_conditioned(spec: str, laws: dict, seed: int) -> bool:
+    g = ograph.parse(spec)
+    t = configs.draw_inputs(spec, laws, seed)
+    ins = {n: tensors.as_float64(t[n], d) for n, d, _ in configs.parse_inputs(spec)}
+    with np.errstate(all="ignore"):
+        exact = interp.run_nodes(g, ins)
+        rounded = interp.run_nodes(g, ins, post=lambda a: a.astype(np.float32).astype(np.float64))
+    for name, node in g.nodes.items():
+        v = exact[name]
+        if not np.all(np.isfinite(v)) or np.abs(v).max() > 1e30:
+            return False
+    out = g.outputs[0][0]
+    a, b = exact[out], rounded[out]
+    if not np.all(np.isfinite(b)):
+        return False
+    rho = np.abs(a).max(axis=-1, keepdims=True)
+    return bool(np.all(np.abs(a - b) <= 2e-6 * np.maximum(np.abs(a), rho)))
+
+
+def main():
+    entries = []
+    for seed in range(N_SEEDS):
+        attempt = 0
+        while True:
+            proxy_spec, laws, meta = random_dag.make_dag(seed, attempt, rows=PROXY_ROWS)
+            if well_conditioned(proxy_spec, laws, seed):
+                break
+            attempt += 1
+            assert attempt < 64, f"seed {seed}: no well-conditioned graph in 64 attempts"
+        entries.append({"seed": seed, "attempt": attempt, "rows": meta["rows"], "cols": meta["cols"], "n_ops": meta["n_ops"],
+                        "rollbacks": meta["rollbacks"]})
+    with open(OUT, "w") as f:
+        json.dump({"generator": "workloads.random_dag.make_dag(seed, attempt)", "entries": entries}, f, indent=0)
+        f.write("\n")
+    rej = sum(e["attempt"] for e in entries)
+    print(f"wrote {OUT}: {len(entries)} graphs, {rej} redraws for conditioning")
+
+
+if __name__ == "__main__":
+    main()

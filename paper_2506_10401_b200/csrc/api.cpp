@@ -1,0 +1,301 @@
+// C ABI: graph handle life cycle, launches and queries.
+#include <cstring>
+#include <memory>
+#include <sstream>
+
+#include "../../include/hct.h"
+#include "codegen.h"
+#include "driver.h"
+#include "graph.h"
+#include "plan.h"
+#include "runtime.h"
+
+using namespace hct;
+
+namespace {
+thread_local std::string g_last_error;
+
+hct_status_t set_error(int code, const std::string& msg) {
+  g_last_error = msg;
+  return (hct_status_t)code;
+}
+
+struct LoadedKernel {
+  KernelSpec spec;
+  CUmodule_t module = nullptr;
+  CUfunction_t func = nullptr;
+  unsigned grid[3] = {1, 1, 1};
+};
+
+std::string cu_error(const Driver& d, CUresult_t rc, const char* what) {
+  const char* s = nullptr;
+  d.GetErrorString(rc, &s);
+  std::ostringstream os;
+  os << what << " failed: CUDA error " << rc << " (" << (s ? s : "?") << ")";
+  return os.str();
+}
+}  // namespace
+
+struct hct_graph {
+  Graph graph;
+  Plan plan;
+  std::vector<LoadedKernel> kernels;
+  size_t scratch_bytes = 0;     // kernel-private scratch appended after the planner's intermediates
+  size_t workspace_bytes = 0;
+  int device = HCT_DEVICE_NONE;
+  CUcontext_t ctx = nullptr;
+  CUdevice_t cudev = 0;
+  CUdeviceptr_t status_word = 0;
+  std::string plan_text;
+};
+
+namespace {
+
+struct CtxGuard {
+  const Driver& d;
+  bool pushed = false;
+  CtxGuard(const Driver& drv, CUcontext_t ctx) : d(drv) { pushed = ctx && d.CtxPushCurrent(ctx) == 0; }
+  ~CtxGuard() {
+    CUcontext_t c;
+    if (pushed) d.CtxPopCurrent(&c);
+  }
+};
+
+void* resolve(const hct_graph* g, const BufRef& b, const void* const* inputs, void* const* outputs, char* workspace) {
+  if (b.kind == BufRef::Scratch) return workspace + g->plan.workspace_bytes + b.scratch_off;
+  const Node& n = g->graph.nodes[b.node];
+  if (n.cls == OpClass::Input) return const_cast<void*>(inputs[n.input_index]);
+  if (!b.ws_copy && n.output_index >= 0) return outputs[n.output_index];
+  return workspace + g->plan.ws_offset[b.node];
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* hct_last_error(void) { return g_last_error.c_str(); }
+const char* hct_version(void) { return "hct 0.1 (sm_100a)"; }
+
+hct_status_t hct_graph_create(const char* spec, size_t spec_len, int device, hct_graph_t** out) {
+  if (out) *out = nullptr;
+  if (!spec || !out) return set_error(HCT_ERR_INVALID_ARG, "spec and out must not be NULL");
+  std::unique_ptr<hct_graph> h(new (std::nothrow) hct_graph);
+  if (!h) return set_error(HCT_ERR_OOM, "out of host memory");
+  try {
+    h->graph = parse_spec(std::string(spec, spec_len));
+    h->plan = make_plan(h->graph);
+    Tunables tun = Tunables::from_env();
+    std::vector<KernelSpec> specs;
+    std::vector<int> spec_group;
+    for (size_t gi = 0; gi < h->plan.groups.size(); ++gi) {
+      size_t before = specs.size();
+      if (h->plan.groups[gi].kind == GroupKind::Row)
+        gen_row_kernel(h->graph, h->plan, (int)gi, tun, &specs);
+      else
+        gen_contraction_kernels(h->graph, h->plan, (int)gi, tun, &h->scratch_bytes, &specs);
+      for (size_t k = before; k < specs.size(); ++k) spec_group.push_back((int)gi);
+    }
+    h->workspace_bytes = h->plan.workspace_bytes + h->scratch_bytes;
+    std::ostringstream pt;
+    pt << h->plan.text;
+    for (size_t k = 0; k < specs.size(); ++k) pt << "launch " << k << ": " << specs[k].name << " (" << specs[k].desc << ")\n";
+    h->plan_text = pt.str();
+    h->device = device;
+
+    const Driver* d = nullptr;
+    int sms = 148;
+    if (device != HCT_DEVICE_NONE) {
+      d = &driver();
+      CUresult_t rc = d->DeviceGet(&h->cudev, device);
+      if (rc != 0) throw Error(HCT_ERR_INVALID_ARG, cu_error(*d, rc, "cuDeviceGet"));
+      int major = 0, minor = 0;
+      d->DeviceGetAttribute(&major, kAttrComputeCapabilityMajor, h->cudev);
+      d->DeviceGetAttribute(&minor, kAttrComputeCapabilityMinor, h->cudev);
+      if (major != 10) {
+        std::ostringstream os;
+        os << "device " << device << " has compute capability " << major << "." << minor << "; 10.x is required";
+        throw Error(HCT_ERR_ARCH, os.str());
+      }
+      d->DeviceGetAttribute(&sms, kAttrMultiprocessorCount, h->cudev);
+      rc = d->DevicePrimaryCtxRetain(&h->ctx, h->cudev);
+      if (rc != 0) throw Error(HCT_ERR_CUDA, cu_error(*d, rc, "cuDevicePrimaryCtxRetain"));
+    }
+    for (auto& ks : specs) {
+      LoadedKernel lk;
+      lk.spec = ks;
+      const std::vector<char>& cubin = compile_cubin(ks.source, ks.name);
+      for (int i = 0; i < 3; ++i) lk.grid[i] = ks.grid[i];
+      if (d) {
+        CtxGuard guard(*d, h->ctx);
+        CUresult_t rc = d->ModuleLoadData(&lk.module, cubin.data());
+        if (rc != 0) throw Error(HCT_ERR_COMPILE, cu_error(*d, rc, "cuModuleLoadData"));
+        rc = d->ModuleGetFunction(&lk.func, lk.module, ks.name.c_str());
+        if (rc != 0) throw Error(HCT_ERR_COMPILE, cu_error(*d, rc, "cuModuleGetFunction"));
+        if (ks.smem_bytes > 48 * 1024) {
+          rc = d->FuncSetAttribute(lk.func, kFuncAttrMaxDynamicSharedSizeBytes, (int)ks.smem_bytes);
+          if (rc != 0) throw Error(HCT_ERR_CUDA, cu_error(*d, rc, "cuFuncSetAttribute(max dynamic shared memory)"));
+        }
+        if (ks.persistent) {
+          int per_sm = 1;
+          rc = d->OccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, lk.func, (int)(ks.block[0] * ks.block[1] * ks.block[2]),
+                                                            ks.smem_bytes);
+          if (rc != 0 || per_sm < 1) per_sm = 1;
+          unsigned want = (unsigned)(sms * per_sm);
+          lk.grid[0] = std::max(1u, std::min(want, ks.max_grid));
+        }
+      }
+      h->kernels.push_back(std::move(lk));
+    }
+    if (d) {
+      CtxGuard guard(*d, h->ctx);
+      CUresult_t rc = d->MemAlloc(&h->status_word, 256);
+      if (rc != 0) throw Error(HCT_ERR_OOM, cu_error(*d, rc, "cuMemAlloc(status word)"));
+      d->MemsetD8(h->status_word, 0, 256);
+    }
+  } catch (const Error& e) {
+    hct_graph_destroy(h.release());
+    return set_error(e.code, e.what());
+  } catch (const std::bad_alloc&) {
+    hct_graph_destroy(h.release());
+    return set_error(HCT_ERR_OOM, "out of host memory");
+  } catch (const std::exception& e) {
+    hct_graph_destroy(h.release());
+    return set_error(HCT_ERR_INVALID_ARG, e.what());
+  }
+  *out = h.release();
+  return HCT_OK;
+}
+
+hct_status_t hct_graph_run(hct_graph_t* g, const void* const* inputs, int n_inputs, void* const* outputs, int n_outputs,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!g) return set_error(HCT_ERR_INVALID_ARG, "graph is NULL");
+  if (g->device == HCT_DEVICE_NONE) return set_error(HCT_ERR_INVALID_ARG, "graph was created without a device");
+  if (n_inputs != (int)g->graph.inputs.size() || n_outputs != (int)g->graph.outputs.size())
+    return set_error(HCT_ERR_INVALID_ARG, "wrong number of inputs or outputs");
+  if ((n_inputs && !inputs) || !outputs) return set_error(HCT_ERR_INVALID_ARG, "inputs/outputs array is NULL");
+  for (int i = 0; i < n_inputs; ++i)
+    if (!inputs[i] || ((uintptr_t)inputs[i] & 15)) return set_error(HCT_ERR_INVALID_ARG, "input pointer NULL or not 16-byte aligned");
+  for (int i = 0; i < n_outputs; ++i)
+    if (!outputs[i] || ((uintptr_t)outputs[i] & 15)) return set_error(HCT_ERR_INVALID_ARG, "output pointer NULL or not 16-byte aligned");
+  if (g->workspace_bytes) {
+    if (!workspace || workspace_bytes < g->workspace_bytes) return set_error(HCT_ERR_INVALID_ARG, "workspace missing or too small");
+    if ((uintptr_t)workspace & 255) return set_error(HCT_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+  }
+  try {
+    const Driver& d = driver();
+    CtxGuard guard(d, g->ctx);
+    for (auto& k : g->kernels) {
+      // parameter block: tensor maps first (64-byte aligned), then pointers
+      struct alignas(64) Params {
+        TensorMap tmap[8];
+        void* ptr[32];
+      } params;
+      size_t ntm = k.spec.tmaps.size(), np = k.spec.ptrs.size() + (k.spec.wants_status ? 1 : 0);
+      if (ntm > 8 || np > 32) return set_error(HCT_ERR_UNSUPPORTED, "kernel has too many arguments");
+      void* ptrs[32];
+      for (size_t i = 0; i < k.spec.ptrs.size(); ++i) ptrs[i] = resolve(g, k.spec.ptrs[i], inputs, outputs, (char*)workspace);
+      if (k.spec.wants_status) ptrs[np - 1] = (void*)g->status_word;
+      for (size_t i = 0; i < ntm; ++i) {
+        const TmaDesc& t = k.spec.tmaps[i];
+        void* base = resolve(g, t.buf, inputs, outputs, (char*)workspace);
+        uint32_t estr[5] = {1, 1, 1, 1, 1};
+        int dtype = t.elem_bytes == 2 ? 9 /* bf16 */ : 7 /* fp32 */;
+        CUresult_t rc = d.TensorMapEncodeTiled(&params.tmap[i], dtype, (unsigned)t.rank, base, t.dims, t.strides + 1, t.box, estr,
+                                               0 /* no interleave */, t.swizzle, 2 /* L2 promotion 128B */, 0 /* zero fill */);
+        if (rc != 0) return set_error(HCT_ERR_CUDA, cu_error(d, rc, "cuTensorMapEncodeTiled"));
+      }
+      // the kernel's single by-value argument is either {ptr[]} or {tmap[], ptr[]}
+      alignas(64) char block[sizeof(Params)];
+      size_t off = 0;
+      if (ntm) {
+        std::memcpy(block, params.tmap, ntm * sizeof(TensorMap));
+        off = ntm * sizeof(TensorMap);
+      }
+      std::memcpy(block + off, ptrs, std::max<size_t>(np, 1) * sizeof(void*));
+      void* args[] = {block};
+      CUresult_t rc = d.LaunchKernel(k.func, k.grid[0], k.grid[1], k.grid[2], k.spec.block[0], k.spec.block[1], k.spec.block[2],
+                                     k.spec.smem_bytes, (CUstream_t)cuda_stream, args, nullptr);
+      if (rc != 0) return set_error(HCT_ERR_CUDA, cu_error(d, rc, ("launch of " + k.spec.name).c_str()));
+    }
+  } catch (const Error& e) {
+    return set_error(e.code, e.what());
+  }
+  return HCT_OK;
+}
+
+hct_status_t hct_graph_status(hct_graph_t* g) {
+  if (!g) return set_error(HCT_ERR_INVALID_ARG, "graph is NULL");
+  if (g->device == HCT_DEVICE_NONE) return HCT_OK;
+  try {
+    const Driver& d = driver();
+    CtxGuard guard(d, g->ctx);
+    unsigned word[4] = {0, 0, 0, 0};
+    CUresult_t rc = d.MemcpyDtoH(word, g->status_word, sizeof word);
+    if (rc != 0) return set_error(HCT_ERR_CUDA, cu_error(d, rc, "cuMemcpyDtoH(status word)"));
+    if (word[0] != 0) {
+      d.MemsetD8(g->status_word, 0, 256);
+      std::ostringstream os;
+      os << "a device-side wait expired (code " << word[0] << ", where " << word[1] << ")";
+      return set_error(HCT_ERR_TIMEOUT, os.str());
+    }
+  } catch (const Error& e) {
+    return set_error(e.code, e.what());
+  }
+  return HCT_OK;
+}
+
+hct_status_t hct_graph_destroy(hct_graph_t* g) {
+  if (!g) return HCT_OK;
+  if (g->device != HCT_DEVICE_NONE && g->ctx) {
+    try {
+      const Driver& d = driver();
+      {
+        CtxGuard guard(d, g->ctx);
+        for (auto& k : g->kernels)
+          if (k.module) d.ModuleUnload(k.module);
+        if (g->status_word) d.MemFree(g->status_word);
+      }
+      d.DevicePrimaryCtxRelease(g->cudev);
+    } catch (const Error&) {
+    }
+  }
+  delete g;
+  return HCT_OK;
+}
+
+int hct_graph_num_inputs(const hct_graph_t* g) { return g ? (int)g->graph.inputs.size() : -1; }
+int hct_graph_num_outputs(const hct_graph_t* g) { return g ? (int)g->graph.outputs.size() : -1; }
+
+hct_status_t hct_graph_tensor_info(const hct_graph_t* g, int is_output, int idx, const char** name, int* dtype, int* rank,
+                                   int64_t shape[4]) {
+  if (!g) return set_error(HCT_ERR_INVALID_ARG, "graph is NULL");
+  const std::vector<int>& list = is_output ? g->graph.outputs : g->graph.inputs;
+  if (idx < 0 || idx >= (int)list.size()) return set_error(HCT_ERR_INVALID_ARG, "tensor index out of range");
+  const Node& n = g->graph.nodes[list[idx]];
+  if (name) *name = n.name.c_str();
+  if (dtype) *dtype = is_output ? (int)n.out_dtype : (int)n.dtype;
+  if (rank) *rank = (int)n.shape.size();
+  if (shape)
+    for (size_t i = 0; i < 4; ++i) shape[i] = i < n.shape.size() ? n.shape[i] : 1;
+  return HCT_OK;
+}
+
+size_t hct_graph_workspace_bytes(const hct_graph_t* g) { return g ? g->workspace_bytes : 0; }
+int hct_graph_num_kernels(const hct_graph_t* g) { return g ? (int)g->kernels.size() : -1; }
+
+hct_status_t hct_graph_cost(const hct_graph_t* g, double* algorithmic_bytes, double* flops) {
+  if (!g) return set_error(HCT_ERR_INVALID_ARG, "graph is NULL");
+  if (algorithmic_bytes) *algorithmic_bytes = g->plan.algorithmic_bytes;
+  if (flops) *flops = g->plan.flops;
+  return HCT_OK;
+}
+
+const char* hct_graph_plan_text(const hct_graph_t* g) { return g ? g->plan_text.c_str() : ""; }
+const char* hct_graph_kernel_source(const hct_graph_t* g, int idx) {
+  return (g && idx >= 0 && idx < (int)g->kernels.size()) ? g->kernels[idx].spec.source.c_str() : nullptr;
+}
+const char* hct_graph_kernel_name(const hct_graph_t* g, int idx) {
+  return (g && idx >= 0 && idx < (int)g->kernels.size()) ? g->kernels[idx].spec.name.c_str() : nullptr;
+}
+
+}  // extern "C"

@@ -1,0 +1,59 @@
+// Kernel generators: turn a planned group into specialised CUDA source for sm_100a.
+#pragma once
+#include <string>
+#include <vector>
+
+#include "graph.h"
+#include "plan.h"
+
+namespace hct {
+
+struct BufRef {
+  enum Kind { NodeBuf, Scratch } kind = NodeBuf;
+  int node = -1;          // NodeBuf: graph input, graph output or workspace slot of this node
+  bool ws_copy = false;   // NodeBuf: the fp32 workspace copy rather than the output buffer
+  int64_t scratch_off = 0;  // Scratch: byte offset inside the kernel-private part of the workspace
+};
+
+// One tensor map the runtime must encode before launch (TMA-fed kernels only).
+struct TmaDesc {
+  BufRef buf;
+  int elem_bytes = 2;             // 2: bf16, 4: fp32/tf32
+  int rank = 2;
+  uint64_t dims[5] = {1, 1, 1, 1, 1};     // innermost first
+  uint64_t strides[5] = {0, 0, 0, 0, 0};  // bytes, for dims[1..]; strides[0] unused
+  uint32_t box[5] = {1, 1, 1, 1, 1};
+  int swizzle = 3;                // 0 none, 1 32B, 2 64B, 3 128B
+};
+
+struct KernelSpec {
+  std::string name;    // entry point
+  std::string source;  // full translation unit
+  std::string desc;    // one-line description for the plan text
+  unsigned grid[3] = {1, 1, 1};
+  unsigned block[3] = {1, 1, 1};
+  unsigned smem_bytes = 0;       // dynamic shared memory
+  bool persistent = false;       // grid[0] is scaled to SM count x occupancy at load time
+  unsigned max_grid = 0;         // upper bound for a persistent grid (number of work items)
+  std::vector<BufRef> ptrs;      // pointer arguments in order (params.ptr[i])
+  std::vector<TmaDesc> tmaps;    // tensor maps in order (params.tmap[i])
+  bool wants_status = false;     // last pointer argument is the device status word
+};
+
+struct Tunables {
+  int row_nv = 4;        // vectors per thread in row kernels
+  int row_cta = 256;     // threads per CTA in row kernels
+  bool simt_only = false;  // keep contractions on the fp32 FMA kernels (for debugging tensor-core paths)
+  static Tunables from_env();
+};
+
+// Extra workspace a group's kernels need beyond the planner's intermediates is appended to
+// `scratch_bytes` (byte offsets in BufRef::Scratch are relative to the start of that region).
+void gen_row_kernel(const Graph& g, const Plan& p, int group, const Tunables& t, std::vector<KernelSpec>* out);
+void gen_contraction_kernels(const Graph& g, const Plan& p, int group, const Tunables& t, size_t* scratch_bytes,
+                             std::vector<KernelSpec>* out);
+
+// Source text of a named kernel skeleton (embedded at build time).
+const char* skeleton_source(const char* name);
+
+}  // namespace hct

@@ -1,0 +1,126 @@
+// Generators for contraction groups (gemm / conv2d plus fused epilogue).
+#include <sstream>
+
+#include "../../include/hct.h"
+#include "codegen.h"
+
+namespace hct {
+
+std::string float_lit(double v);
+const char* ctype(DType d);
+
+namespace {
+
+struct EpiGen {
+  const Graph& g;
+  const Plan& p;
+  const Group& grp;
+  int gi;
+  std::vector<BufRef> ptrs;
+
+  int ptr_index(int node, bool ws_copy) {
+    for (size_t i = 0; i < ptrs.size(); ++i)
+      if (ptrs[i].kind == BufRef::NodeBuf && ptrs[i].node == node && ptrs[i].ws_copy == ws_copy) return (int)i;
+    BufRef b;
+    b.node = node;
+    b.ws_copy = ws_copy;
+    ptrs.push_back(b);
+    return (int)ptrs.size() - 1;
+  }
+  DType buf_dtype(int node) const { return g.nodes[node].cls == OpClass::Input ? g.nodes[node].dtype : F32; }
+  bool is_ws(int node) const { return g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0; }
+
+  // Scalar epilogue: value `acc` of element at linear offset `off`, per-row index `ri`
+  // (GEMM row, or n*K+k for NCHW), per-column index `ci` (GEMM column, or channel k).
+  std::string scalar_fn() {
+    std::ostringstream f;
+    f << "__device__ __forceinline__ void hct_epilogue(const HctParams& hct_p, float acc, long long off, long long ri, int ci) {\n";
+    int anchor = grp.nodes[0];
+    f << "  const float e" << anchor << " = acc;\n";
+    auto ref = [&](const Operand& a) -> std::string {
+      if (a.is_literal()) return float_lit(a.literal);
+      if (p.group_of[a.node] == gi) return "e" + std::to_string(a.node);
+      int k = find_ext(grp, a.node);
+      const ExtOperand& e = grp.ext[k];
+      int pi = ptr_index(e.node, is_ws(e.node));
+      std::string ptr = std::string("((const ") + ctype(buf_dtype(e.node)) + "*)hct_p.ptr[" + std::to_string(pi) + "])";
+      switch (e.bcast) {
+        case Bcast::Full: return "hct_ld1(" + ptr + " + off)";
+        case Bcast::RowVec: return "hct_ld1(" + ptr + " + ci)";
+        case Bcast::Scalar: return "hct_ld1(" + ptr + ")";
+        case Bcast::RowIdx: return grp.kind == GroupKind::Conv ? "hct_ld1(" + ptr + " + ci)" : "hct_ld1(" + ptr + " + ri)";
+      }
+      return "";
+    };
+    for (size_t i = 1; i < grp.nodes.size(); ++i) {
+      const Node& nd = g.nodes[grp.nodes[i]];
+      f << "  const float e" << grp.nodes[i] << " = hct_" << nd.op << "(";
+      for (size_t a = 0; a < nd.args.size(); ++a) f << (a ? ", " : "") << ref(nd.args[a]);
+      f << ");  // " << nd.name << "\n";
+    }
+    for (auto& s : grp.stores) {
+      int pi = ptr_index(s.node, !s.to_output);
+      f << "  hct_st1((" << ctype(s.dtype) << "*)hct_p.ptr[" << pi << "] + off, e" << s.node << ");\n";
+    }
+    f << "}\n";
+    return f.str();
+  }
+};
+
+}  // namespace
+
+void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunables& tun, size_t* scratch_bytes,
+                             std::vector<KernelSpec>* out) {
+  (void)tun;
+  (void)scratch_bytes;
+  const Group& grp = p.groups[gi];
+  const Node& anchor = g.nodes[grp.nodes[0]];
+  const Node& a = g.nodes[anchor.args[0].node];
+  const Node& b = g.nodes[anchor.args[1].node];
+  EpiGen eg{g, p, grp, gi, {}};
+  auto operand_buf = [&](int node) {
+    return eg.ptr_index(node, g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0);
+  };
+  int pa = operand_buf(anchor.args[0].node);
+  int pb = operand_buf(anchor.args[1].node);
+  DType ta = eg.buf_dtype(anchor.args[0].node), tb = eg.buf_dtype(anchor.args[1].node);
+  std::string epi = eg.scalar_fn();
+
+  KernelSpec k;
+  std::ostringstream src;
+  if (grp.kind == GroupKind::Gemm) {
+    int64_t M = a.shape[0], K = a.shape[1], N = b.shape[1];
+    k.name = "hct_gemm_simt_g" + std::to_string(gi);
+    src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n";
+    src << "#define HCT_TA " << ctype(ta) << "\n#define HCT_TB " << ctype(tb) << "\n#define HCT_PA " << pa << "\n#define HCT_PB "
+        << pb << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
+    src << skeleton_source("common") << "\nstruct HctParams { void* ptr[" << eg.ptrs.size() << "]; };\n" << epi
+        << skeleton_source("gemm_simt");
+    k.grid[0] = (unsigned)((N + 63) / 64);
+    k.grid[1] = (unsigned)((M + 63) / 64);
+    if ((M + 63) / 64 > 65535) throw Error(HCT_ERR_UNSUPPORTED, "gemm with more than 4M rows is not supported");
+    k.block[0] = 256;
+    k.desc = "gemm fp32-FMA 64x64x16";
+  } else {
+    const auto& xs = a.shape;
+    const auto& ws = b.shape;
+    k.name = "hct_conv_simt_g" + std::to_string(gi);
+    src << "#define HCT_NB " << xs[0] << "\n#define HCT_CI " << xs[1] << "\n#define HCT_H " << xs[2] << "\n#define HCT_W " << xs[3]
+        << "\n#define HCT_KO " << ws[0] << "\n#define HCT_FR " << ws[2] << "\n#define HCT_FS " << ws[3] << "\n#define HCT_STRIDE "
+        << anchor.stride << "\n#define HCT_PAD " << anchor.pad << "\n#define HCT_HO " << anchor.shape[2] << "\n#define HCT_WO "
+        << anchor.shape[3] << "\n";
+    src << "#define HCT_TA " << ctype(ta) << "\n#define HCT_TB " << ctype(tb) << "\n#define HCT_PA " << pa << "\n#define HCT_PB "
+        << pb << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
+    src << skeleton_source("common") << "\nstruct HctParams { void* ptr[" << eg.ptrs.size() << "]; };\n" << epi
+        << skeleton_source("conv_simt");
+    int64_t total = anchor.numel();
+    k.grid[0] = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 64);
+    k.block[0] = 256;
+    k.desc = "conv2d direct fp32-FMA";
+  }
+  k.source = src.str();
+  k.ptrs = eg.ptrs;
+  out->push_back(k);
+}
+
+}  // namespace hct

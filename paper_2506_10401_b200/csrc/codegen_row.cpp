@@ -1,0 +1,222 @@
+// Generator for fused row kernels: elementwise, broadcast and row-reduction chains over one [R,C] space.
+#include <cstdio>
+#include <cstdlib>
+#include <sstream>
+
+#include "../../include/hct.h"
+#include "codegen.h"
+
+namespace hct {
+
+Tunables Tunables::from_env() {
+  Tunables t;
+  if (const char* s = std::getenv("HCT_ROW_NV")) t.row_nv = std::max(1, std::atoi(s));
+  if (const char* s = std::getenv("HCT_ROW_CTA")) t.row_cta = std::max(32, std::atoi(s));
+  if (const char* s = std::getenv("HCT_SIMT_ONLY")) t.simt_only = std::atoi(s) != 0;
+  return t;
+}
+
+std::string float_lit(double v) {
+  char buf[64];
+  float f = (float)v;
+  if (f != f) return "__int_as_float(0x7fc00000)";
+  if (f == 1.0f / 0.0f) return "HCT_INF";
+  if (f == -1.0f / 0.0f) return "(-HCT_INF)";
+  std::snprintf(buf, sizeof buf, "%.9ef", (double)f);
+  return buf;
+}
+
+const char* ctype(DType d) { return d == BF16 ? "hct_bf16_t" : "float"; }
+
+namespace {
+
+struct RowGen {
+  const Graph& g;
+  const Plan& p;
+  const Group& grp;
+  int gi;
+  std::ostringstream body;
+  std::vector<BufRef> ptrs;
+
+  int ptr_index(int node, bool ws_copy) {
+    for (size_t i = 0; i < ptrs.size(); ++i)
+      if (ptrs[i].node == node && ptrs[i].ws_copy == ws_copy) return (int)i;
+    BufRef b;
+    b.node = node;
+    b.ws_copy = ws_copy;
+    ptrs.push_back(b);
+    return (int)ptrs.size() - 1;
+  }
+
+  // storage dtype of a buffer this group reads
+  DType ext_dtype(int node) const { return g.nodes[node].cls == OpClass::Input ? g.nodes[node].dtype : F32; }
+  bool ext_is_ws(int node) const { return g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0; }
+
+  // expression for operand `a` at element index variable `e` (full-width context) or as a row scalar
+  std::string ref(const Operand& a, bool full_ctx) {
+    if (a.is_literal()) return float_lit(a.literal);
+    int n = a.node;
+    if (p.group_of[n] == gi) {
+      if (p.is_colv[n]) return "s" + std::to_string(n);
+      return full_ctx ? "v" + std::to_string(n) + "[e]" : "v" + std::to_string(n) + "[0]";
+    }
+    int k = find_ext(grp, n);
+    switch (grp.ext[k].bcast) {
+      case Bcast::Full: return "x" + std::to_string(k) + "[e]";
+      case Bcast::RowVec: return "x" + std::to_string(k) + "[e]";
+      default: return "c" + std::to_string(k);
+    }
+  }
+};
+
+}  // namespace
+
+void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, std::vector<KernelSpec>* out) {
+  const Group& grp = p.groups[gi];
+  const int64_t R = grp.R, C = grp.C;
+  if (C > (1 << 17)) throw Error(HCT_ERR_UNSUPPORTED, "rows longer than 131072 elements are not supported");
+
+  // vector width from alignment of every full-width buffer: rows start at multiples of C elements
+  int V = (C % 4 == 0) ? 4 : (C % 2 == 0) ? 2 : 1;
+  int64_t nvec = (C + V - 1) / V;
+  int T = 8;
+  while (T < 1024 && (nvec + T - 1) / T > tun.row_nv) T *= 2;
+  int NV = (int)((nvec + T - 1) / T);
+  if (NV * V > 128) throw Error(HCT_ERR_UNSUPPORTED, "row does not fit the register budget of one CTA");
+  int cta = std::max(T, std::min(tun.row_cta, 1024));
+  int G = std::max(1, cta / T);
+  if (G > 15) G = 15;  // one named barrier per row slot
+  if ((int64_t)G > R) G = (int)std::max<int64_t>(1, R);
+  // whole warps only
+  while ((G * T) % 32 != 0) ++G;
+
+  RowGen rg{g, p, grp, gi, {}, {}};
+  std::ostringstream& b = rg.body;
+  std::string name = "hct_row_g" + std::to_string(gi);
+
+  // ---- external operands
+  std::ostringstream pre, loads;
+  for (size_t k = 0; k < grp.ext.size(); ++k) {
+    const ExtOperand& e = grp.ext[k];
+    int pi = rg.ptr_index(e.node, rg.ext_is_ws(e.node));
+    const char* ct = ctype(rg.ext_dtype(e.node));
+    pre << "    const " << ct << "* __restrict__ q" << k << " = (const " << ct << "*)hct_p.ptr[" << pi << "];\n";
+    switch (e.bcast) {
+      case Bcast::Full:
+        loads << "      float x" << k << "[HCT_E]; hct_load_row(q" << k << ", hct_row, hct_t, x" << k << ", false);\n";
+        break;
+      case Bcast::RowVec:
+        loads << "      float x" << k << "[HCT_E]; hct_load_row(q" << k << ", 0, hct_t, x" << k << ", true);\n";
+        break;
+      case Bcast::Scalar:
+        pre << "    const float c" << k << " = hct_ld1(q" << k << ");\n";
+        break;
+      case Bcast::RowIdx: {
+        // index from the row's leading coordinates
+        loads << "      float c" << k << ";\n      {\n        long long r_ = hct_row, i_ = 0;\n";
+        for (int d = (int)grp.full_shape.size() - 2; d >= 0; --d) {
+          int64_t ext = grp.full_shape[d];
+          int64_t st = e.lead_stride[d];
+          if (st != 0) loads << "        i_ += (r_ % " << ext << "LL) * " << st << "LL;\n";
+          loads << "        r_ /= " << ext << "LL;\n";
+        }
+        loads << "        c" << k << " = hct_ld1(q" << k << " + i_);\n      }\n";
+        break;
+      }
+    }
+  }
+
+  // ---- nodes
+  for (int ni : grp.nodes) {
+    const Node& nd = g.nodes[ni];
+    std::string id = std::to_string(ni);
+    b << "      // " << nd.name << " = " << nd.op << "\n";
+    if (nd.cls == OpClass::Unary || nd.cls == OpClass::Binary) {
+      std::string call = "hct_" + nd.op + "(";
+      if (p.is_colv[ni]) {
+        for (size_t a = 0; a < nd.args.size(); ++a) call += (a ? ", " : "") + rg.ref(nd.args[a], false);
+        b << "      const float s" << id << " = " << call << ");\n";
+      } else {
+        for (size_t a = 0; a < nd.args.size(); ++a) call += (a ? ", " : "") + rg.ref(nd.args[a], true);
+        b << "      float v" << id << "[HCT_E];\n"
+          << "      _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) v" << id << "[e] = " << call << ");\n";
+      }
+    } else if (nd.cls == OpClass::RowReduce) {
+      std::string a = rg.ref(nd.args[0], true);
+      bool is_max = nd.op == "row_max";
+      b << "      float s" << id << " = " << (is_max ? "-HCT_INF" : "0.0f") << ";\n"
+        << "      _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) if (HCT_HAS(e)) s" << id << " = "
+        << (is_max ? "fmaxf(s" + id + ", " + a + ")" : "s" + id + " + " + a) << ";\n"
+        << "      s" << id << " = " << (is_max ? "HCT_RMAX" : "HCT_RSUM") << "(s" << id << ");\n";
+      if (nd.op == "row_mean") b << "      s" << id << " = s" << id << " / (float)HCT_C;\n";
+    } else if (nd.cls == OpClass::RowSoftmax) {
+      std::string a = rg.ref(nd.args[0], true);
+      b << "      float v" << id << "[HCT_E];\n"
+        << "      {\n"
+        << "        float m_ = -HCT_INF;\n"
+        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) if (HCT_HAS(e)) m_ = fmaxf(m_, " << a << ");\n"
+        << "        m_ = HCT_RMAX(m_);\n"
+        << "        float d_ = 0.0f;\n"
+        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) { v" << id << "[e] = HCT_HAS(e) ? hct_exp(" << a
+        << " - m_) : 0.0f; d_ += v" << id << "[e]; }\n"
+        << "        d_ = HCT_RSUM(d_);\n"
+        << "        const float inv_ = 1.0f / d_;\n"
+        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) v" << id << "[e] *= inv_;\n"
+        << "      }\n";
+    } else if (nd.cls == OpClass::RowLayernorm) {
+      std::string a = rg.ref(nd.args[0], true);
+      std::string ga = rg.ref(nd.args[1], true), be = rg.ref(nd.args[2], true);
+      b << "      float v" << id << "[HCT_E];\n"
+        << "      {\n"
+        << "        float m_ = 0.0f;\n"
+        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) if (HCT_HAS(e)) m_ += " << a << ";\n"
+        << "        m_ = HCT_RSUM(m_) / (float)HCT_C;\n"
+        << "        float q_ = 0.0f;\n"
+        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) { const float d_ = HCT_HAS(e) ? " << a
+        << " - m_ : 0.0f; v" << id << "[e] = d_; q_ = fmaf(d_, d_, q_); }\n"
+        << "        q_ = HCT_RSUM(q_) / (float)HCT_C;\n"
+        << "        const float r_ = 1.0f / sqrtf(q_ + " << float_lit(nd.eps) << ");\n"
+        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) v" << id << "[e] = fmaf(v" << id << "[e] * r_, " << ga
+        << ", " << be << ");\n"
+        << "      }\n";
+    } else {
+      throw Error(HCT_ERR_UNSUPPORTED, "operator " + nd.op + " cannot be part of a row kernel");
+    }
+  }
+
+  // ---- stores
+  std::ostringstream stores;
+  for (auto& s : grp.stores) {
+    int pi = rg.ptr_index(s.node, !s.to_output);
+    const char* ct = ctype(s.dtype);
+    std::string id = std::to_string(s.node);
+    if (p.is_colv[s.node])
+      stores << "      if (hct_live && hct_t == 0) hct_st1((" << ct << "*)hct_p.ptr[" << pi << "] + hct_row, s" << id << ");\n";
+    else
+      stores << "      if (hct_live) hct_store_row((" << ct << "*)hct_p.ptr[" << pi << "], hct_row, hct_t, v" << id << ");\n";
+  }
+
+  std::ostringstream src;
+  src << "#define HCT_T " << T << "\n#define HCT_G " << G << "\n#define HCT_V " << V << "\n#define HCT_NV " << NV << "\n"
+      << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "\n#define HCT_NPTR " << std::max<size_t>(1, rg.ptrs.size()) << "\n"
+      << skeleton_source("common") << "\n"
+      << skeleton_source("row") << "\n"
+      << "HCT_ROW_KERNEL_BEGIN(" << name << ")\n"
+      << pre.str() << "  HCT_ROW_LOOP_BEGIN\n"
+      << loads.str() << b.str() << stores.str() << "  HCT_ROW_LOOP_END\nHCT_ROW_KERNEL_END\n";
+
+  KernelSpec k;
+  k.name = name;
+  k.source = src.str();
+  k.block[0] = (unsigned)(G * T);
+  k.persistent = true;
+  k.max_grid = (unsigned)std::min<int64_t>((R + G - 1) / G, 0x7fffffff);
+  k.grid[0] = k.max_grid;
+  k.ptrs = rg.ptrs;
+  std::ostringstream d;
+  d << "row kernel T=" << T << " G=" << G << " V=" << V << " NV=" << NV;
+  k.desc = d.str();
+  out->push_back(k);
+}
+
+}  // namespace hct

@@ -1,0 +1,55 @@
+// The few CUDA driver entry points the library uses, resolved from libcuda.so.1 at first use.
+// Types are declared locally so that no CUDA header is needed to build the host code.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+
+namespace hct {
+
+typedef int CUresult_t;
+typedef int CUdevice_t;
+typedef struct CUctx_st* CUcontext_t;
+typedef struct CUmod_st* CUmodule_t;
+typedef struct CUfunc_st* CUfunction_t;
+typedef struct CUstream_st* CUstream_t;
+typedef unsigned long long CUdeviceptr_t;
+
+struct alignas(64) TensorMap {
+  uint64_t opaque[16];
+};
+
+enum {
+  kAttrComputeCapabilityMajor = 75,
+  kAttrComputeCapabilityMinor = 76,
+  kAttrMultiprocessorCount = 16,
+  kAttrMaxSharedMemoryPerBlockOptin = 97,
+  kFuncAttrMaxDynamicSharedSizeBytes = 8,
+};
+
+struct Driver {
+  CUresult_t (*Init)(unsigned);
+  CUresult_t (*GetErrorString)(CUresult_t, const char**);
+  CUresult_t (*DeviceGet)(CUdevice_t*, int);
+  CUresult_t (*DeviceGetAttribute)(int*, int, CUdevice_t);
+  CUresult_t (*DevicePrimaryCtxRetain)(CUcontext_t*, CUdevice_t);
+  CUresult_t (*DevicePrimaryCtxRelease)(CUdevice_t);
+  CUresult_t (*CtxPushCurrent)(CUcontext_t);
+  CUresult_t (*CtxPopCurrent)(CUcontext_t*);
+  CUresult_t (*ModuleLoadData)(CUmodule_t*, const void*);
+  CUresult_t (*ModuleUnload)(CUmodule_t);
+  CUresult_t (*ModuleGetFunction)(CUfunction_t*, CUmodule_t, const char*);
+  CUresult_t (*FuncSetAttribute)(CUfunction_t, int, int);
+  CUresult_t (*OccupancyMaxActiveBlocksPerMultiprocessor)(int*, CUfunction_t, int, size_t);
+  CUresult_t (*LaunchKernel)(CUfunction_t, unsigned, unsigned, unsigned, unsigned, unsigned, unsigned, unsigned, CUstream_t,
+                             void**, void**);
+  CUresult_t (*MemAlloc)(CUdeviceptr_t*, size_t);
+  CUresult_t (*MemFree)(CUdeviceptr_t);
+  CUresult_t (*MemcpyDtoH)(void*, CUdeviceptr_t, size_t);
+  CUresult_t (*MemsetD8)(CUdeviceptr_t, unsigned char, size_t);
+  // CUtensorMap*, dtype, rank, globalAddress, globalDim, globalStrides, boxDim, elementStrides, interleave, swizzle,
+  // l2Promotion, oobFill
+  CUresult_t (*TensorMapEncodeTiled)(TensorMap*, int, unsigned, void*, const uint64_t*, const uint64_t*, const uint32_t*,
+                                     const uint32_t*, int, int, int, int);
+};
+
+}  // namespace hct

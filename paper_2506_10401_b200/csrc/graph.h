@@ -1,0 +1,56 @@
+// Typed operator DAG built from spec text: parsing, validation and shape inference.
+#pragma once
+#include <cstdint>
+#include <stdexcept>
+#include <string>
+#include <vector>
+
+namespace hct {
+
+enum DType { F32 = 0, BF16 = 1 };
+
+enum class OpClass { Input, Unary, Binary, RowSoftmax, RowLayernorm, RowReduce, Gemm, Conv };
+
+struct Error : std::runtime_error {
+  int code;
+  Error(int c, const std::string& m) : std::runtime_error(m), code(c) {}
+};
+
+struct Operand {
+  int node = -1;       // index into Graph::nodes, or -1 for a literal
+  double literal = 0;  // used when node < 0
+  bool is_literal() const { return node < 0; }
+};
+
+struct Node {
+  std::string name;
+  std::string op;  // "input" or the operator name
+  OpClass cls = OpClass::Input;
+  std::vector<Operand> args;
+  std::vector<int64_t> shape;
+  DType dtype = F32;  // storage dtype of an input; computed nodes are fp32 values
+  double eps = 1e-5;
+  int stride = 1, pad = 0;
+  int input_index = -1;   // position among `input` lines
+  int output_index = -1;  // position among `output` lines
+  DType out_dtype = F32;  // storage dtype when the node is a graph output
+  int64_t numel() const {
+    int64_t n = 1;
+    for (auto d : shape) n *= d;
+    return n;
+  }
+};
+
+struct Graph {
+  std::vector<Node> nodes;   // definition order is a topological order
+  std::vector<int> inputs;   // node indices
+  std::vector<int> outputs;  // node indices
+};
+
+// Throws Error(HCT_ERR_PARSE | HCT_ERR_GRAPH | HCT_ERR_UNSUPPORTED).
+Graph parse_spec(const std::string& text);
+
+bool is_unary(const std::string& op);
+bool is_binary(const std::string& op);
+
+}  // namespace hct

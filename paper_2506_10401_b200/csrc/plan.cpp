@@ -1,0 +1,245 @@
+#include "plan.h"
+
+#include <algorithm>
+#include <sstream>
+
+#include "../../include/hct.h"
+
+namespace hct {
+
+namespace {
+
+std::vector<int64_t> col_shape(std::vector<int64_t> s) {
+  s.back() = 1;
+  return s;
+}
+
+bool all_ones(const std::vector<int64_t>& s) {
+  for (auto d : s)
+    if (d != 1) return false;
+  return true;
+}
+
+// Classify operand shape `s` against the group's full shape.  Returns false if the pattern is unsupported.
+bool classify(const std::vector<int64_t>& s, const std::vector<int64_t>& full, Bcast* kind, std::vector<int64_t>* lead_stride) {
+  lead_stride->clear();
+  if (s == full) {
+    *kind = Bcast::Full;
+    return true;
+  }
+  if (all_ones(s)) {
+    *kind = Bcast::Scalar;
+    return true;
+  }
+  if (s.size() > full.size()) return false;
+  // right-align
+  std::vector<int64_t> a(full.size(), 1);
+  for (size_t i = 0; i < s.size(); ++i) a[full.size() - s.size() + i] = s[i];
+  for (size_t i = 0; i < full.size(); ++i)
+    if (a[i] != 1 && a[i] != full[i]) return false;
+  bool lead_ones = true;
+  for (size_t i = 0; i + 1 < a.size(); ++i) lead_ones = lead_ones && a[i] == 1;
+  if (lead_ones && a.back() == full.back()) {
+    *kind = Bcast::RowVec;
+    return true;
+  }
+  if (a.back() == 1) {
+    *kind = Bcast::RowIdx;
+    lead_stride->assign(full.size() - 1, 0);
+    int64_t st = 1;
+    for (int i = (int)a.size() - 2; i >= 0; --i) {
+      if (a[i] != 1) {
+        (*lead_stride)[i] = st;
+        st *= a[i];
+      }
+    }
+    return true;
+  }
+  return false;  // e.g. [R,C] with [H,1,C]: broadcast along a middle axis of a full-width operand
+}
+
+}  // namespace
+
+int find_ext(const Group& grp, int node) {
+  for (size_t i = 0; i < grp.ext.size(); ++i)
+    if (grp.ext[i].node == node) return (int)i;
+  return -1;
+}
+
+Plan make_plan(const Graph& g) {
+  Plan p;
+  const int n = (int)g.nodes.size();
+  p.group_of.assign(n, -1);
+  p.ws_offset.assign(n, -1);
+  p.is_colv.assign(n, 0);
+
+  auto add_ext = [&](Group& grp, int node, int consumer) {
+    if (find_ext(grp, node) >= 0) return;
+    ExtOperand e;
+    e.node = node;
+    if (!classify(g.nodes[node].shape, grp.full_shape, &e.bcast, &e.lead_stride))
+      throw Error(HCT_ERR_UNSUPPORTED, "node '" + g.nodes[consumer].name + "': broadcast pattern of operand '" +
+                                           g.nodes[node].name + "' is not supported");
+    grp.ext.push_back(e);
+  };
+
+  // Can node i (elementwise or row op) live in group gi?
+  auto can_join = [&](int gi, int i) -> bool {
+    const Group& grp = p.groups[gi];
+    const Node& nd = g.nodes[i];
+    bool full = nd.shape == grp.full_shape;
+    bool colv = nd.shape == col_shape(grp.full_shape);
+    if (grp.kind != GroupKind::Row) {
+      if (!(nd.cls == OpClass::Unary || nd.cls == OpClass::Binary) || !full) return false;
+      for (auto& a : nd.args) {
+        if (a.is_literal() || p.group_of[a.node] == gi) continue;
+        Bcast b;
+        std::vector<int64_t> ls;
+        if (!classify(g.nodes[a.node].shape, grp.full_shape, &b, &ls)) return false;
+        if (b == Bcast::RowIdx) {
+          // contraction epilogues index per-row scalars by GEMM row, or by channel for NCHW outputs
+          if (grp.kind == GroupKind::Conv) {
+            const auto& s = g.nodes[a.node].shape;
+            int64_t K = grp.full_shape[1];
+            bool chan = (s.size() == 3 && s[0] == K && s[1] == 1 && s[2] == 1) ||
+                        (s.size() == 4 && s[0] == 1 && s[1] == K && s[2] == 1 && s[3] == 1);
+            if (!chan) return false;
+          }
+        }
+        if (b == Bcast::RowVec && grp.kind == GroupKind::Conv) return false;
+      }
+      return true;
+    }
+    if (!full && !colv) return false;
+    if (nd.cls == OpClass::RowSoftmax || nd.cls == OpClass::RowLayernorm || nd.cls == OpClass::RowReduce) {
+      if (g.nodes[nd.args[0].node].shape != grp.full_shape) return false;
+      if (grp.full_shape.size() != 2) return false;
+    }
+    for (auto& a : nd.args) {
+      if (a.is_literal() || p.group_of[a.node] == gi) continue;
+      Bcast b;
+      std::vector<int64_t> ls;
+      if (!classify(g.nodes[a.node].shape, grp.full_shape, &b, &ls)) return false;
+    }
+    return true;
+  };
+
+  for (int i = 0; i < n; ++i) {
+    const Node& nd = g.nodes[i];
+    if (nd.cls == OpClass::Input) continue;
+    int gi = -1;
+    if (nd.cls == OpClass::Gemm || nd.cls == OpClass::Conv) {
+      Group grp;
+      grp.kind = nd.cls == OpClass::Gemm ? GroupKind::Gemm : GroupKind::Conv;
+      grp.full_shape = nd.shape;
+      p.groups.push_back(grp);
+      gi = (int)p.groups.size() - 1;
+    } else {
+      int cand = -1;
+      for (auto& a : nd.args)
+        if (!a.is_literal()) cand = std::max(cand, p.group_of[a.node]);
+      if (cand >= 0 && can_join(cand, i)) {
+        gi = cand;
+      } else {
+        Group grp;
+        grp.kind = GroupKind::Row;
+        if (nd.cls == OpClass::Unary || nd.cls == OpClass::Binary)
+          grp.full_shape = nd.shape;
+        else
+          grp.full_shape = g.nodes[nd.args[0].node].shape;
+        p.groups.push_back(grp);
+        gi = (int)p.groups.size() - 1;
+      }
+    }
+    Group& grp = p.groups[gi];
+    grp.nodes.push_back(i);
+    p.group_of[i] = gi;
+    if (grp.kind == GroupKind::Row && nd.shape != grp.full_shape) p.is_colv[i] = 1;
+    if (nd.cls == OpClass::RowSoftmax || nd.cls == OpClass::RowLayernorm || nd.cls == OpClass::RowReduce)
+      grp.has_reduction = true;
+  }
+
+  // Iteration spaces, external operands.
+  for (auto& grp : p.groups) {
+    grp.C = grp.full_shape.back();
+    grp.R = 1;
+    for (size_t d = 0; d + 1 < grp.full_shape.size(); ++d) grp.R *= grp.full_shape[d];
+  }
+  for (int i = 0; i < n; ++i) {
+    const Node& nd = g.nodes[i];
+    if (nd.cls == OpClass::Input) continue;
+    Group& grp = p.groups[p.group_of[i]];
+    bool anchor = nd.cls == OpClass::Gemm || nd.cls == OpClass::Conv;
+    for (auto& a : nd.args) {
+      if (a.is_literal() || p.group_of[a.node] == p.group_of[i]) continue;
+      if (anchor) continue;  // contraction operands are bound separately
+      add_ext(grp, a.node, i);
+    }
+  }
+
+  // Stores: a node is written if it is a graph output or read by another group.
+  std::vector<char> cross(n, 0);
+  for (int i = 0; i < n; ++i)
+    for (auto& a : g.nodes[i].args)
+      if (!a.is_literal() && g.nodes[a.node].cls != OpClass::Input && p.group_of[a.node] != p.group_of[i]) cross[a.node] = 1;
+  size_t ws = 0;
+  for (int i = 0; i < n; ++i) {
+    const Node& nd = g.nodes[i];
+    if (nd.cls == OpClass::Input) continue;
+    Group& grp = p.groups[p.group_of[i]];
+    bool out = nd.output_index >= 0;
+    // consumers always read fp32; an output stored as bf16 cannot serve them
+    bool need_ws = cross[i] && !(out && nd.out_dtype == F32);
+    if (out) grp.stores.push_back({i, nd.out_dtype, true});
+    if (need_ws) {
+      p.ws_offset[i] = (int64_t)ws;
+      ws += ((size_t)nd.numel() * 4 + 255) / 256 * 256;
+      grp.stores.push_back({i, F32, false});
+    }
+  }
+  p.workspace_bytes = ws;
+
+  // Work accounting.
+  auto dsize = [](DType d) { return d == BF16 ? 2.0 : 4.0; };
+  for (int i : g.inputs) p.algorithmic_bytes += g.nodes[i].numel() * dsize(g.nodes[i].dtype);
+  for (int i : g.outputs) p.algorithmic_bytes += g.nodes[i].numel() * dsize(g.nodes[i].out_dtype);
+  for (int i = 0; i < n; ++i) {
+    const Node& nd = g.nodes[i];
+    if (nd.cls == OpClass::Gemm) {
+      const auto& a = g.nodes[nd.args[0].node].shape;
+      p.flops += 2.0 * a[0] * a[1] * nd.shape[1];
+    } else if (nd.cls == OpClass::Conv) {
+      const auto& w = g.nodes[nd.args[1].node].shape;
+      p.flops += 2.0 * nd.numel() * w[1] * w[2] * w[3];
+    }
+    if (p.ws_offset[i] < 0) continue;
+    // an intermediate no single pass could keep on chip: contraction -> row group (row wider than one
+    // accumulator tile), or anything -> contraction operand
+    bool unavoidable = false;
+    for (int j = 0; j < n; ++j)
+      for (auto& a : g.nodes[j].args) {
+        if (a.is_literal() || a.node != i || p.group_of[j] == p.group_of[i]) continue;
+        bool into_contraction = g.nodes[j].cls == OpClass::Gemm || g.nodes[j].cls == OpClass::Conv;
+        bool from_contraction = p.groups[p.group_of[i]].kind != GroupKind::Row && p.groups[p.group_of[j]].has_reduction &&
+                                nd.shape.back() > 512;
+        unavoidable = unavoidable || into_contraction || from_contraction;
+      }
+    if (unavoidable) p.algorithmic_bytes += 8.0 * nd.numel();
+  }
+
+  std::ostringstream os;
+  for (size_t gi = 0; gi < p.groups.size(); ++gi) {
+    const Group& grp = p.groups[gi];
+    os << "kernel " << gi << " " << (grp.kind == GroupKind::Row ? "row" : grp.kind == GroupKind::Gemm ? "gemm" : "conv") << " [";
+    for (size_t d = 0; d < grp.full_shape.size(); ++d) os << (d ? "," : "") << grp.full_shape[d];
+    os << "]:";
+    for (int i : grp.nodes) os << " " << g.nodes[i].name << "=" << g.nodes[i].op;
+    os << " | stores:";
+    for (auto& s : grp.stores) os << " " << g.nodes[s.node].name << (s.to_output ? "" : "(ws)");
+    os << "\n";
+  }
+  p.text = os.str();
+  return p;
+}
+
+}  // namespace hct

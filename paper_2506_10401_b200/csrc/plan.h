@@ -1,0 +1,64 @@
+// Fusion planner: partitions the operator DAG into kernels.
+//
+// Two kinds of group exist.  A *row group* is a maximal set of elementwise, broadcast and
+// row-reduction nodes that share one [R,C] iteration space, so a row can stay in registers from
+// the first load to the last store.  A *contraction group* is one gemm or conv2d node together
+// with the elementwise nodes that consume its result (its epilogue).  Values that cross a group
+// boundary are written once to caller-provided workspace (fp32).
+#pragma once
+#include <string>
+#include <vector>
+
+#include "graph.h"
+
+namespace hct {
+
+enum class GroupKind { Row, Gemm, Conv };
+
+// How an operand indexes relative to the group's full shape [.., C].
+enum class Bcast {
+  Full,    // same shape: element (row, col)
+  RowVec,  // [C] / [1,..,C]: indexed by col
+  RowIdx,  // last extent 1: one scalar per row, index = sum of row coordinates times strides
+  Scalar   // a single element
+};
+
+struct ExtOperand {
+  int node;  // producing node (a graph input or a node materialised by an earlier group)
+  Bcast bcast;
+  // RowIdx: index = sum_d coord_d * stride[d] over the leading extents of the full shape
+  std::vector<int64_t> lead_stride;
+};
+
+struct Store {
+  int node;
+  DType dtype;
+  bool to_output;  // graph output buffer, else workspace
+};
+
+struct Group {
+  GroupKind kind = GroupKind::Row;
+  std::vector<int> nodes;           // topological; a contraction group starts with its anchor
+  std::vector<int64_t> full_shape;  // shape of full-size values ([R,C], [M,N] or [N,K,H,W])
+  int64_t R = 0, C = 0;             // rows = product of leading extents, cols = last extent
+  std::vector<ExtOperand> ext;      // deduplicated external operands
+  std::vector<Store> stores;
+  bool has_reduction = false;
+};
+
+struct Plan {
+  std::vector<Group> groups;
+  std::vector<int> group_of;           // per node (-1 for inputs)
+  std::vector<int64_t> ws_offset;      // per node, -1 if not in workspace
+  std::vector<char> is_colv;           // per node: value is one scalar per row of its group
+  size_t workspace_bytes = 0;
+  double algorithmic_bytes = 0, flops = 0;
+  std::string text;
+};
+
+Plan make_plan(const Graph& g);
+
+// Index of `node` in group.ext, or -1.
+int find_ext(const Group& grp, int node);
+
+}  // namespace hct

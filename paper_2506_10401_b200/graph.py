@@ -1,0 +1,80 @@
+"""Convenience wrapper: owns a graph handle and runs it on torch CUDA tensors.
+
+torch is used for device memory and streams only.
+"""
+from __future__ import annotations
+
+from . import binding as B
+
+
+class FusedGraph:
+    def __init__(self, spec: str, device: int = 0):
+        self.handle = B.hct_graph_create(spec, device)
+        self.device = device
+        self.n_in = B.hct_graph_num_inputs(self.handle)
+        self.n_out = B.hct_graph_num_outputs(self.handle)
+        self.inputs = [B.hct_graph_tensor_info(self.handle, False, i) for i in range(self.n_in)]
+        self.outputs = [B.hct_graph_tensor_info(self.handle, True, i) for i in range(self.n_out)]
+        self.workspace_bytes = B.hct_graph_workspace_bytes(self.handle)
+        self._ws = None
+
+    # -- queries
+    @property
+    def plan(self) -> str:
+        return B.hct_graph_plan_text(self.handle)
+
+    @property
+    def num_kernels(self) -> int:
+        return B.hct_graph_num_kernels(self.handle)
+
+    def cost(self):
+        return B.hct_graph_cost(self.handle)
+
+    def kernel_source(self, i: int) -> str:
+        return B.hct_graph_kernel_source(self.handle, i)
+
+    # -- execution on torch tensors
+    def alloc_outputs(self):
+        import torch
+        outs = []
+        for _, dtype, shape in self.outputs:
+            outs.append(torch.empty(shape, dtype=torch.bfloat16 if dtype == B.HCT_BF16 else torch.float32, device=f"cuda:{self.device}"))
+        return outs
+
+    def workspace(self):
+        import torch
+        if self._ws is None and self.workspace_bytes:
+            self._ws = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=f"cuda:{self.device}")
+        return self._ws
+
+    def run(self, inputs, outputs=None, stream=None):
+        """inputs: torch CUDA tensors in spec order.  Returns the output tensors.  Does not synchronise."""
+        import torch
+        if outputs is None:
+            outputs = self.alloc_outputs()
+        for t, (name, dtype, shape) in zip(inputs, self.inputs):
+            want = torch.bfloat16 if dtype == B.HCT_BF16 else torch.float32
+            if tuple(t.shape) != tuple(shape) or t.dtype != want or not t.is_contiguous() or not t.is_cuda:
+                raise ValueError(f"input {name}: expected contiguous CUDA {want} tensor of shape {shape}")
+        ws = self.workspace()
+        ws_ptr = 0
+        if ws is not None:
+            ws_ptr = (ws.data_ptr() + 255) // 256 * 256
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        B.hct_graph_run(self.handle, [t.data_ptr() for t in inputs], [t.data_ptr() for t in outputs], ws_ptr, self.workspace_bytes,
+                        s.cuda_stream)
+        return outputs
+
+    def status(self):
+        B.hct_graph_status(self.handle)
+
+    def close(self):
+        if self.handle is not None:
+            B.hct_graph_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

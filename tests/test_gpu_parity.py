@@ -1,0 +1,198 @@
+"""Parity of the CUDA library against the CPU oracle on identical seeded inputs.  Needs a B200."""
+import numpy as np
+import pytest
+
+from tests import parity
+from workloads import configs, sweep
+
+pytestmark = pytest.mark.gpu
+
+N_ = {"kind": "normal", "mean": 0.0, "std": 1.0}
+POS_ = {"kind": "uniform", "lo": 0.5, "hi": 2.0}
+
+
+def check_f32(spec, laws, seed=0):
+    got, want, g = parity.run_both(spec, laws, seed)
+    worst = max(parity.f32_violation(a, b) for a, b in zip(got, want))
+    assert worst <= 1.0, f"fp32 parity violated by factor {worst:.3g}\n{g.plan}"
+    return g
+
+
+def check_bf16(spec, laws, seed=0):
+    got, want, g = parity.run_both(spec, laws, seed)
+    worst = max(parity.bf16_violation(a, b) for a, b in zip(got, want))
+    assert worst <= 1.0, f"bf16 parity violated by factor {worst:.3g}\n{g.plan}"
+    return g
+
+
+# ------------------------------------------------------------------ memory-bound chains
+
+@pytest.mark.parametrize("r,c", [(300, 4096), (37, 1000), (5, 1023), (64, 130), (3, 2), (1, 4096), (129, 256), (33, 8192), (7, 20000)])
+def test_softmax_layernorm_chain_shapes(r, c):
+    spec, laws = configs.get_config("c2_softmax_layernorm_chain", r=r, c=c)
+    g = check_f32(spec, laws)
+    assert g.num_kernels == 1
+
+
+@pytest.mark.parametrize("op", ["relu", "gelu_tanh", "gelu_erf", "sigmoid", "exp", "tanh", "sqrt", "sin", "cos", "neg", "abs"])
+def test_unary(op):
+    spec = f"hct 1\ninput x f32 [67,200]\nnode y = {op}(x)\noutput y\n"
+    check_f32(spec, {"x": POS_ if op == "sqrt" else N_})
+
+
+@pytest.mark.parametrize("op", ["add", "sub", "mul", "div", "max", "min"])
+def test_binary_broadcast_kinds(op):
+    spec = f"""hct 1
+input x f32 [45,132]
+input full f32 [45,132]
+input rowv f32 [132]
+input colv f32 [45,1]
+input one f32 [1]
+node a = {op}(x, full)
+node b = {op}(a, rowv)
+node c = {op}(colv, b)
+node d = {op}(c, 1.5)
+node e = {op}(0.75, d)
+node f = {op}(e, one)
+output f
+output b
+"""
+    check_f32(spec, {"x": POS_, "full": POS_, "rowv": POS_, "colv": POS_, "one": POS_})
+
+
+def test_row_reductions_and_column_values():
+    spec = """hct 1
+input x f32 [70,777]
+node s = row_sum(x)
+node m = row_mean(x)
+node mx = row_max(x)
+node c = sub(x, m)
+node n = div(c, mx)
+node t = tanh(s)
+node y = mul(n, t)
+output y
+output s
+output m
+output mx
+"""
+    check_f32(spec, {"x": POS_})
+
+
+def test_bf16_input_and_output_rows():
+    spec = "hct 1\ninput x bf16 [50,264]\ninput b bf16 [264]\nnode t = add(x, b)\nnode y = row_softmax(t)\noutput y bf16\n"
+    got, want, g = parity.run_both(spec, {"x": N_, "b": N_})
+    assert parity.bf16_violation(got[0], want[0]) <= 1.0
+
+
+def test_channel_broadcast_rank4():
+    spec = "hct 1\ninput x f32 [3,5,6,20]\ninput s f32 [5,1,1]\ninput t f32 [1,5,1,1]\nnode a = mul(x, s)\nnode y = add(a, t)\noutput y\n"
+    check_f32(spec, {"x": N_, "s": N_, "t": N_})
+
+
+# ------------------------------------------------------------------ contractions
+
+def test_config1_gemm_bias_relu_full_size():
+    spec, laws = configs.get_config("c1_gemm_bias_relu_f32")
+    check_f32(spec, laws)
+
+
+@pytest.mark.parametrize("m,k,n", [(1, 1, 1), (5, 7, 3), (130, 260, 72), (300, 1000, 520), (64, 4096, 128)])
+def test_gemm_f32_shapes(m, k, n):
+    spec, laws = configs.get_config("c1_gemm_bias_relu_f32", m=m, k=k, n=n)
+    check_f32(spec, laws)
+
+
+def test_gemm_f32_integer_inputs_are_exact():
+    spec, _ = configs.get_config("c1_gemm_bias_relu_f32", m=96, k=160, n=136)
+    il = {"kind": "int", "lo": -8, "hi": 8}
+    got, want, _ = parity.run_both(spec, {"a": il, "b": il, "bias": il})
+    np.testing.assert_array_equal(got[0], want[0])
+
+
+@pytest.mark.parametrize("m,k,n", [(300, 264, 520), (128, 64, 256), (1, 8, 8), (257, 4096, 136), (2048, 512, 1024)])
+def test_gemm_bf16_chain_shapes(m, k, n):
+    spec, laws = configs.get_config("c3_gemm_bf16_gelu_residual", m=m, k=k, n=n)
+    check_bf16(spec, laws)
+
+
+def test_gemm_bf16_integer_inputs_are_exact():
+    spec = "hct 1\ninput x bf16 [200,320]\ninput w bf16 [320,264]\nnode y = gemm(x, w)\noutput y f32\n"
+    il = {"kind": "int", "lo": -8, "hi": 8}
+    got, want, _ = parity.run_both(spec, {"x": il, "w": il})
+    np.testing.assert_array_equal(got[0], want[0])
+
+
+@pytest.mark.parametrize("kw", [
+    dict(n=2, c=128, h=14, w=14, k=128),
+    dict(n=1, c=128, h=56, w=56, k=128),
+    dict(n=3, c=64, h=9, w=11, k=32),
+    dict(n=2, c=3, h=8, w=8, k=5, ksize=1, pad=0),
+    dict(n=1, c=8, h=12, w=10, k=4, stride=2, pad=1),
+    dict(n=1, c=4, h=7, w=7, k=4, ksize=3, pad=0),
+])
+def test_conv_chain_shapes(kw):
+    spec, laws = configs.get_config("c4_conv_bn_relu_bf16", **kw)
+    check_bf16(spec, laws)
+
+
+def test_conv_f32_integer_inputs_are_exact():
+    spec = "hct 1\ninput x f32 [2,16,10,12]\ninput w f32 [8,16,3,3]\nnode y = conv2d(x, w, stride=1, pad=1)\noutput y\n"
+    il = {"kind": "int", "lo": -4, "hi": 4}
+    got, want, _ = parity.run_both(spec, {"x": il, "w": il})
+    np.testing.assert_array_equal(got[0], want[0])
+
+
+# ------------------------------------------------------------------ multi-kernel graphs
+
+def test_gemm_between_row_kernels():
+    spec = """hct 1
+input x f32 [96,256]
+input w f32 [256,384]
+input b f32 [384]
+node a = relu(x)
+node s = row_sum(a)
+node c = div(a, s)
+node m = gemm(c, w)
+node d = add(m, b)
+node e = row_softmax(d)
+output e
+output s
+"""
+    g = check_f32(spec, {"x": POS_, "w": N_, "b": N_})
+    assert g.num_kernels >= 3
+
+
+@pytest.mark.parametrize("seed", list(range(0, 200, 5)))
+def test_sweep_graphs_reduced_rows(seed):
+    """Same random graphs as the sweep, 96 rows each so that the oracle stays fast."""
+    spec, laws, _ = sweep.get(seed, rows=96)
+    check_f32(spec, laws, seed)
+
+
+def test_run_twice_is_bitwise_repeatable():
+    import torch
+    import paper_2506_10401_b200 as hct
+    spec, laws = configs.get_config("c2_softmax_layernorm_chain", r=512, c=4096)
+    t = configs.draw_inputs(spec, laws, 0)
+    g = hct.FusedGraph(spec, 0)
+    ins = parity.to_device(spec, t)
+    a = g.run(ins)[0].clone()
+    b = g.run(ins)[0]
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+
+
+def test_bad_pointers_are_rejected_on_the_host():
+    import torch
+    import paper_2506_10401_b200 as hct
+    spec = "hct 1\ninput x f32 [8,64]\nnode y = relu(x)\noutput y\n"
+    g = hct.FusedGraph(spec, 0)
+    x = torch.zeros(8 * 64 + 4, device="cuda")
+    y = torch.zeros(8, 64, device="cuda")
+    with pytest.raises(hct.HctError) as e:
+        hct.hct_graph_run(g.handle, [x.data_ptr() + 4], [y.data_ptr()])
+    assert e.value.code == hct.HCT_ERR_INVALID_ARG
+    with pytest.raises(hct.HctError):
+        hct.hct_graph_run(g.handle, [x.data_ptr()], [])
+    with pytest.raises(hct.HctError):
+        hct.hct_graph_run(g.handle, [0], [y.data_ptr()])

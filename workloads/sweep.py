@@ -1,0 +1,26 @@
+"""The graph-augmentation sweep: 200 random operator DAGs, seeds 0..199.
+
+``sweep_specs.json`` records, per seed, which attempt of the generator was kept (graphs that are
+numerically ill-conditioned are redrawn, see oracle/make_sweep.py); the spec text itself is
+regenerated from (seed, attempt).
+"""
+from __future__ import annotations
+
+import json
+import os
+
+from . import random_dag
+
+_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "sweep_specs.json")
+
+
+def entries():
+    with open(_PATH) as f:
+        return json.load(f)["entries"]
+
+
+def get(seed: int, rows: int | None = None):
+    """(spec, laws, meta) of sweep graph ``seed``; ``rows`` overrides the row count."""
+    e = entries()[seed]
+    assert e["seed"] == seed
+    return random_dag.make_dag(seed, e["attempt"], rows=rows)
