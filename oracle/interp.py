@@ -99,9 +99,9 @@ def conv2d(x, w, stride, pad):
     k, _, kr, ks = w.shape
     ho = (h + 2 * pad - kr) // stride + 1
     wo = (wd + 2 * pad - ks) // stride + 1
-    xp = np.zeros((n, c, h + 2 * pad, wd + 2 * pad), dtype=np.float64)
+    xp = np.zeros((n, c, h + 2 * pad, wd + 2 * pad), dtype=x.dtype)
     xp[:, :, pad:pad + h, pad:pad + wd] = x
-    y = np.zeros((n, k, ho, wo), dtype=np.float64)
+    y = np.zeros((n, k, ho, wo), dtype=x.dtype)
     for r in range(kr):
         for s in range(ks):
             win = xp[:, :, r:r + (ho - 1) * stride + 1:stride, s:s + (wo - 1) * stride + 1:stride]
@@ -111,19 +111,20 @@ def conv2d(x, w, stride, pad):
 
 # ---- interpreter ----------------------------------------------------------------------------
 
-def run_nodes(spec, inputs: dict, post=None) -> dict:
-    """Evaluate every node; returns name -> float64 array for all nodes (inputs included).
+def run_nodes(spec, inputs: dict, dtype=np.float64, gemm_fn=None) -> dict:
+    """Evaluate every node; returns name -> array for all nodes (inputs included).
 
     ``inputs`` maps input names to arrays already widened to float64 (the
-    stored float32 / bfloat16 values, exactly).  ``post``, if given, is applied
-    to every computed node (used only to study how a graph reacts to rounding
-    each intermediate, never for expected values).
+    stored float32 / bfloat16 values, exactly).  ``dtype`` is float64 for every
+    expected value; float32 is accepted only to study how a graph reacts to
+    single-precision evaluation (the sweep's conditioning check), never as a
+    reference; ``gemm_fn`` replaces the matrix product in such a study.
     """
     g = spec if isinstance(spec, Graph) else parse(spec)
     val = {}
     for name, node in g.nodes.items():
         if node.op == "input":
-            a = np.asarray(inputs[name], dtype=np.float64)
+            a = np.asarray(inputs[name], dtype=dtype)
             if tuple(a.shape) != tuple(node.shape):
                 raise ValueError(f"input {name}: expected shape {node.shape}, got {a.shape}")
             val[name] = a
@@ -146,14 +147,13 @@ def run_nodes(spec, inputs: dict, post=None) -> dict:
         elif op == "row_layernorm":
             out = row_layernorm(args[0], args[1], args[2], node.attrs["eps"])
         elif op == "gemm":
-            out = gemm(args[0], args[1])
+            out = (gemm_fn or gemm)(args[0], args[1])
         elif op == "conv2d":
             out = conv2d(args[0], args[1], node.attrs["stride"], node.attrs["pad"])
         else:  # pragma: no cover - parse() rejects unknown operators
             raise ValueError(op)
         assert tuple(out.shape) == tuple(node.shape), (name, out.shape, node.shape)
-        out = np.asarray(out, dtype=np.float64)
-        val[name] = post(out) if post is not None else out
+        val[name] = np.asarray(out, dtype=dtype)
     return val
 
 

@@ -4,10 +4,12 @@
 
 For seed 0..199 the generator (workloads.random_dag, after the paper's Algorithm 1) is asked
 for a graph; the graph is then checked for data-flow validity in the numerical sense: it is
-evaluated by the oracle on a 4-row proxy twice, once exactly and once with every node rounded
-to float32, and it is rolled back and redrawn (next attempt number) when any value is
-non-finite or above 1e30, or when rounding alone already moves the result by more than 2e-6
-of the row's magnitude, i.e. when no float32 implementation could be compared at 1e-5.
+evaluated by the oracle on a 64-row proxy twice, once in float64 and once with the same
+definitions carried out in float32, and it is rolled back and redrawn (next attempt number)
+when any value is non-finite or above 1e30, or when single precision alone already moves the
+result by more than 2e-6 of the row's magnitude, i.e. when the graph is too ill-conditioned
+for any float32 implementation to be compared at 1e-5 (sums that cancel, exponentials of
+large arguments, results that underflow).
 Calls only workloads/ and oracle/.
 """
 from __future__ import annotations
@@ -22,8 +24,25 @@ from oracle import interp
 from workloads import configs, random_dag, tensors
 
 N_SEEDS = 200
-PROXY_ROWS = 4
+PROXY_ROWS = 64
 OUT = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "workloads", "sweep_specs.json")
+
+
+def gemm_f32_sequential(a, b):
+    """Single-precision product accumulated term by term in k order (no blocking, no pairwise
+    summation): the least favourable accumulation a float32 implementation may use."""
+    acc = np.zeros((a.shape[0], b.shape[1]), dtype=np.float32)
+    for k in range(a.shape[1]):
+        acc += a[:, k:k + 1] * b[k:k + 1, :]
+    return acc
+
+
+def column_scale(a):
+    """Magnitude against which an element's error is judged: the largest value of its row, or of
+    the whole tensor when rows have a single element."""
+    if a.shape[-1] == 1:
+        return np.full_like(a, np.abs(a).max())
+    return np.abs(a).max(axis=-1, keepdims=True)
 
 
 def well_conditioned(spec: str, laws: dict, seed: int) -> bool:
@@ -32,16 +51,16 @@ def well_conditioned(spec: str, laws: dict, seed: int) -> bool:
     ins = {n: tensors.as_float64(t[n], d) for n, d, _ in configs.parse_inputs(spec)}
     with np.errstate(all="ignore"):
         exact = interp.run_nodes(g, ins)
-        rounded = interp.run_nodes(g, ins, post=lambda a: a.astype(np.float32).astype(np.float64))
+        single = interp.run_nodes(g, ins, dtype=np.float32, gemm_fn=gemm_f32_sequential)
     for name, node in g.nodes.items():
         v = exact[name]
         if not np.all(np.isfinite(v)) or np.abs(v).max() > 1e30:
             return False
     out = g.outputs[0][0]
-    a, b = exact[out], rounded[out]
+    a, b = exact[out], single[out].astype(np.float64)
     if not np.all(np.isfinite(b)):
         return False
-    rho = np.abs(a).max(axis=-1, keepdims=True)
+    rho = column_scale(a)
     return bool(np.all(np.abs(a - b) <= 2e-6 * np.maximum(np.abs(a), rho)))
 
 
