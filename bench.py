@@ -1,0 +1,266 @@
+#!/usr/bin/env python
+"""Benchmark of fused operator chains on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step = one run of a whole fused chain (every kernel of its plan) on one batch of seeded
+synthetic input.  The headline workload is the memory-bound chain (affine, GELU, row softmax,
+row layer normalisation on an fp32 [8192,4096] tensor); throughput is algorithmic bytes per
+second (inputs read once, outputs written once).  Contraction chains report TFLOP/s.
+With N > 1 every rank runs an independent replica on its own GPU (the chains do not shard
+across devices); the value is the sum over ranks divided by the slowest rank's time.
+Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from workloads import configs  # noqa: E402
+
+WORKLOADS = {
+    "c2_softmax_layernorm_chain": dict(bound="hbm", sample=dict(r=8192)),
+    "c3_gemm_bf16_gelu_residual": dict(bound="tensor", sample=dict(m=2048)),
+    "c4_conv_bn_relu_bf16": dict(bound="tensor", sample=dict(n=8)),
+    "c1_gemm_bias_relu_f32": dict(bound="tensor", sample=dict()),
+}
+HEADLINE = "c2_softmax_layernorm_chain"
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm": p["hbm_gbs"], "tensor": p["bf16_tflops"], "source": "measured"}
+    return {"hbm": 6650.0, "tensor": 1590.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        q = "clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+            "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([t.strip() for t in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], 0.0, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = max(mx, float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx or None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def metric_of(bound, bytes_, flops, seconds):
+    if bound == "hbm":
+        return bytes_ / seconds / 1e9, "GB/s"
+    return flops / seconds / 1e12, "TFLOP/s"
+
+
+def oracle_arm(name, steps, warmup):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload."""
+    import oracle
+    from workloads import tensors
+    info = WORKLOADS[name]
+    spec, laws = configs.get_config(name, **info["sample"])
+    t = configs.draw_inputs(spec, laws, 0)
+    ins = {n: tensors.as_float64(t[n], d) for n, d, _ in configs.parse_inputs(spec)}
+    g = oracle.parse(spec)
+    in_bytes = sum(t[n].nbytes for n in t)
+    out_elems = sum(int(np.prod(g.nodes[o].shape)) for o, _ in g.outputs)
+    out_bytes = sum(int(np.prod(g.nodes[o].shape)) * (2 if d == "bf16" else 4) for o, d in g.outputs)
+    flops = 0.0
+    for node in g.nodes.values():
+        if node.op == "gemm":
+            flops += 2.0 * g.nodes[node.args[0]].shape[0] * g.nodes[node.args[0]].shape[1] * node.shape[1]
+        elif node.op == "conv2d":
+            w = g.nodes[node.args[1]].shape
+            flops += 2.0 * np.prod(node.shape) * w[1] * w[2] * w[3]
+    for _ in range(warmup):
+        oracle.run(g, ins)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.run(g, ins)
+    dt = (time.perf_counter() - t0) / steps
+    value, unit = metric_of(info["bound"], in_bytes + out_bytes, flops, dt)
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    sample = ", ".join(f"{k}={v}" for k, v in info["sample"].items()) or "full size"
+    return dict(value=value, unit=unit, cores=cores, kind="oracle", sample=f"{name} at {sample} ({out_elems} output elements per step)",
+                ms_per_step=dt * 1e3)
+
+
+def run_gpu(name, steps, warmup, rank, world, device):
+    import torch
+    import paper_2506_10401_b200 as hct
+    from tests import parity
+
+    info = WORKLOADS[name]
+    spec, laws = configs.get_config(name)
+    host = configs.draw_inputs(spec, laws, 0)
+    g = hct.FusedGraph(spec, device)
+    ins = parity.to_device(spec, host, f"cuda:{device}")
+    outs = g.alloc_outputs()
+    bytes_, flops = g.cost()
+    stream = torch.cuda.current_stream(device)
+    flush = torch.empty(192 * 1024 * 1024, dtype=torch.uint8, device=f"cuda:{device}")  # larger than the 126 MB L2
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize(device)
+
+    for _ in range(max(warmup, 3)):
+        flush.zero_()
+        g.run(ins, outs, stream)
+    barrier()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    with ClockSampler(device) as clocks:
+        for a, b in ev:
+            flush.zero_()           # evict the previous step's data from L2; not timed
+            a.record(stream)
+            g.run(ins, outs, stream)
+            b.record(stream)
+        barrier()
+    g.status()
+    per_step = [a.elapsed_time(b) * 1e-3 for a, b in ev]
+    dev_s = float(np.sum(per_step))
+
+    # end to end: pinned host inputs -> device, run, result back to the host, every step
+    pinned = [torch.from_numpy(host[n].view(np.int16) if d == "bf16" else host[n]).pin_memory() for n, d, _ in configs.parse_inputs(spec)]
+    dev_in = [torch.empty_like(t, device=f"cuda:{device}") for t in pinned]
+    run_in = [t.view(torch.bfloat16) if d == "bf16" else t for t, (_, d, _) in zip(dev_in, configs.parse_inputs(spec))]
+    host_out = [torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in outs]
+    h2d = sum(t.numel() * t.element_size() for t in pinned)
+    d2h = sum(t.numel() * t.element_size() for t in host_out)
+    e2e_steps = max(2, min(steps, 5))
+
+    def e2e_once():
+        for src, dst in zip(pinned, dev_in):
+            dst.copy_(src, non_blocking=True)
+        g.run(run_in, outs, stream)
+        for src, dst in zip(outs, host_out):
+            dst.copy_(src, non_blocking=True)
+
+    e2e_once()
+    barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(e2e_steps):
+        e2e_once()
+    b.record(stream)
+    barrier()
+    e2e_s = a.elapsed_time(b) * 1e-3 / e2e_steps
+
+    if world > 1:
+        t = torch.tensor([dev_s, e2e_s], device=f"cuda:{device}", dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        dev_s, e2e_s = float(t[0]), float(t[1])
+    value, unit = metric_of(info["bound"], bytes_ * world, flops * world, dev_s / steps)
+    e2e_v, _ = metric_of(info["bound"], bytes_ * world, flops * world, e2e_s)
+    kern_s = float(np.mean(per_step))
+    return dict(value=value, unit=unit, ms_per_step=dev_s / steps * 1e3, bytes=bytes_, flops=flops, kernel_s=kern_s,
+                kernels=g.num_kernels, clocks=clocks.summary(), e2e=dict(value=e2e_v, unit=unit, h2d_bytes_per_step=h2d,
+                                                                         d2h_bytes_per_step=d2h), plan=g.plan)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="hct", choices=["hct", "reference"])
+    ap.add_argument("--workload", default=HEADLINE, choices=list(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    name = args.workload
+    info = WORKLOADS[name]
+    metric = "fused-chain throughput: GB/s (memory-bound) / TFLOP/s (GEMM,conv) and % of B200 roofline"
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        r = oracle_arm(name, max(1, min(args.steps, 5)), min(args.warmup, 1))
+        line = dict(impl="reference", metric=metric, value=r["value"], unit=r["unit"], n_gpus=args.gpus, steps=args.steps,
+                    warmup=args.warmup, ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
+                    dtype="f64", data="synthetic", config={"workload": name, "sample": r["sample"]},
+                    cpu_baseline=dict(value=r["value"], unit=r["unit"], cores=r["cores"], kind="oracle", sample=r["sample"]),
+                    e2e=dict(value=r["value"], unit=r["unit"], h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+        print(json.dumps(line))
+        return
+
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the fused chains have no CPU execution path")
+    if world > 1:
+        torch.cuda.set_device(local)
+        torch.distributed.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    r = run_gpu(name, args.steps, args.warmup, rank, world, local)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        o = oracle_arm(name, 4, 1)
+        cpu = dict(value=o["value"], unit=o["unit"], cores=o["cores"], kind="oracle", sample=o["sample"])
+    if rank == 0:
+        pk = peaks()
+        achieved, unit = metric_of(info["bound"], r["bytes"], r["flops"], r["kernel_s"])
+        peak = pk["hbm"] if info["bound"] == "hbm" else pk["tensor"]
+        line = dict(metric=metric, value=r["value"], unit=r["unit"], n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+                    ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
+                    dtype="bf16" if "bf16" in name else "f32", data="synthetic",
+                    config={"workload": name, "l2": "flushed between steps (192 MB write, untimed)", "kernels_per_step": r["kernels"],
+                            "parallelism": "replicas" if world > 1 else "single"},
+                    clocks=r["clocks"], e2e=r["e2e"], gpu_launches=r["kernels"] * args.steps,
+                    roofline=dict(bound=info["bound"], achieved=achieved, peak=peak, unit=("GB/s" if info["bound"] == "hbm" else "TFLOP/s"),
+                                  frac=achieved / peak, traffic=None, peak_source=pk["source"]),
+                    cpu_baseline=cpu)
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
