@@ -65,6 +65,62 @@ struct EpiGen {
     f << "}\n";
     return f.str();
   }
+
+  // Run epilogue for the tensor-core GEMM: one thread owns 32 consecutive columns of one row.
+  // `ncols` of them exist; vector access is legal when N is a multiple of the vector length.
+  std::string run_fn(int64_t N) {
+    std::ostringstream f;
+    f << "__device__ __forceinline__ void hct_epilogue_run(const HctParams& hct_p, float (&acc)[32], long long row, int col0, int ncols) {\n";
+    int anchor = grp.nodes[0];
+    std::ostringstream loads;
+    auto vec_ok = [&](DType d) { return N % (d == BF16 ? 8 : 4) == 0 ? "true" : "false"; };
+    auto ref = [&](const Operand& a) -> std::string {
+      if (a.is_literal()) return float_lit(a.literal);
+      if (p.group_of[a.node] == gi) return a.node == anchor ? "acc[j]" : "e" + std::to_string(a.node);
+      int k = find_ext(grp, a.node);
+      const ExtOperand& e = grp.ext[k];
+      if (e.bcast == Bcast::Full || e.bcast == Bcast::RowVec) return "x" + std::to_string(k) + "[j]";
+      return "c" + std::to_string(k);
+    };
+    for (size_t k = 0; k < grp.ext.size(); ++k) {
+      const ExtOperand& e = grp.ext[k];
+      int pi = ptr_index(e.node, is_ws(e.node));
+      DType d = buf_dtype(e.node);
+      std::string ptr = std::string("((const ") + ctype(d) + "*)hct_p.ptr[" + std::to_string(pi) + "])";
+      switch (e.bcast) {
+        case Bcast::Full:
+          loads << "  float x" << k << "[32]; hct_ld_run32<" << ctype(d) << ">(" << ptr << " + row * " << N << "LL + col0, x" << k
+                << ", ncols, " << vec_ok(d) << ");\n";
+          break;
+        case Bcast::RowVec:
+          loads << "  float x" << k << "[32]; hct_ld_run32<" << ctype(d) << ">(" << ptr << " + col0, x" << k << ", ncols, " << vec_ok(d)
+                << ");\n";
+          break;
+        case Bcast::Scalar: loads << "  const float c" << k << " = hct_ld1(" << ptr << ");\n"; break;
+        case Bcast::RowIdx: loads << "  const float c" << k << " = hct_ld1(" << ptr << " + row);\n"; break;
+      }
+    }
+    f << loads.str();
+    for (auto& st : grp.stores) f << "  float o" << st.node << "_" << (st.to_output ? 1 : 0) << "[32];\n";
+    f << "  _Pragma(\"unroll\") for (int j = 0; j < 32; ++j) {\n";
+    for (size_t i = 1; i < grp.nodes.size(); ++i) {
+      const Node& nd = g.nodes[grp.nodes[i]];
+      f << "    const float e" << grp.nodes[i] << " = hct_" << nd.op << "(";
+      for (size_t a = 0; a < nd.args.size(); ++a) f << (a ? ", " : "") << ref(nd.args[a]);
+      f << ");  // " << nd.name << "\n";
+    }
+    for (auto& st : grp.stores)
+      f << "    o" << st.node << "_" << (st.to_output ? 1 : 0) << "[j] = " << (st.node == anchor ? "acc[j]" : "e" + std::to_string(st.node))
+        << ";\n";
+    f << "  }\n";
+    for (auto& st : grp.stores) {
+      int pi = ptr_index(st.node, !st.to_output);
+      f << "  hct_st_run32<" << ctype(st.dtype) << ">((" << ctype(st.dtype) << "*)hct_p.ptr[" << pi << "] + row * " << N << "LL + col0, o"
+        << st.node << "_" << (st.to_output ? 1 : 0) << ", ncols, " << vec_ok(st.dtype) << ");\n";
+    }
+    f << "}\n";
+    return f.str();
+  }
 };
 
 }  // namespace
@@ -78,6 +134,55 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
   const Node& a = g.nodes[anchor.args[0].node];
   const Node& b = g.nodes[anchor.args[1].node];
   EpiGen eg{g, p, grp, gi, {}};
+
+  // ---- tensor-core GEMM: bf16 operands straight from their buffers
+  if (grp.kind == GroupKind::Gemm && !tun.simt_only) {
+    int64_t M = a.shape[0], K = a.shape[1], N = b.shape[1];
+    DType da = g.nodes[anchor.args[0].node].cls == OpClass::Input ? a.dtype : F32;
+    DType db = g.nodes[anchor.args[1].node].cls == OpClass::Input ? b.dtype : F32;
+    if (da == BF16 && db == BF16 && K % 8 == 0 && N % 8 == 0 && M <= 0x7fffffff && N <= 0x7fffffff && K <= 0x7fffffff) {
+      int BN = N > 128 ? 256 : N > 64 ? 128 : 64;
+      int stages = BN == 256 ? 4 : 6;
+      std::string epi = eg.run_fn(N);
+      KernelSpec k;
+      k.name = "hct_gemm_tc_bf16_g" + std::to_string(gi);
+      std::ostringstream src;
+      src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n#define HCT_BN " << BN
+          << "\n#define HCT_STAGES " << stages << "\n#define HCT_TF32X3 0\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
+          << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
+      src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[2]; void* ptr["
+          << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source("gemm_tc");
+      k.source = src.str();
+      k.ptrs = eg.ptrs;
+      k.wants_status = true;
+      TmaDesc ta, tb;
+      ta.buf.node = anchor.args[0].node;
+      ta.elem_bytes = 2;
+      ta.rank = 2;
+      ta.dims[0] = (uint64_t)K; ta.dims[1] = (uint64_t)M;
+      ta.strides[1] = (uint64_t)K * 2;
+      ta.box[0] = 64; ta.box[1] = 128;
+      tb.buf.node = anchor.args[1].node;
+      tb.elem_bytes = 2;
+      tb.rank = 2;
+      tb.dims[0] = (uint64_t)N; tb.dims[1] = (uint64_t)K;
+      tb.strides[1] = (uint64_t)N * 2;
+      tb.box[0] = 64; tb.box[1] = 64;
+      k.tmaps = {ta, tb};
+      int64_t tiles = ((M + 127) / 128) * ((N + BN - 1) / BN);
+      k.block[0] = 192;
+      k.smem_bytes = (unsigned)(stages * (128 * 128 + BN * 128) + 1024);
+      k.persistent = true;
+      k.max_grid = (unsigned)std::min<int64_t>(tiles, 0x7fffffff);
+      k.grid[0] = k.max_grid;
+      std::ostringstream d;
+      d << "gemm tcgen05 bf16 128x" << BN << "x64, " << stages << " stages";
+      k.desc = d.str();
+      out->push_back(k);
+      return;
+    }
+  }
+
   auto operand_buf = [&](int node) {
     return eg.ptr_index(node, g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0);
   };

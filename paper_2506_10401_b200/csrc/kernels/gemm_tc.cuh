@@ -1,0 +1,173 @@
+// Persistent tensor-core GEMM with fused epilogue:  D[M,N] = epilogue(A[M,K] * B[K,N]).
+//
+// One CTA per SM walks over 128 x HCT_BN output tiles.  Warp 0 feeds a ring of shared-memory
+// stages with TMA tile loads (A is K-major, B is row-major [K,N], i.e. N-major), warp 1 issues
+// tcgen05.mma from those stages into one of two accumulators in tensor memory, warps 2..5 drain
+// the other accumulator (tcgen05.ld), apply the generated epilogue and store, so the epilogue of
+// tile i overlaps the main loop of tile i+1.  All hand-offs are mbarriers with bounded waits.
+//
+// Defined by the generator: HCT_M, HCT_N, HCT_K, HCT_BN, HCT_STAGES, HCT_TF32X3 (0/1),
+// HCT_NPTR, HCT_STATUS_SLOT, HCT_KERNEL_NAME, HctParams, hct_epilogue_run().
+#define HCT_BM 128
+#if HCT_TF32X3
+#define HCT_BK 32                                  // 32 fp32 = one 128-byte swizzle row
+#define HCT_ELT 4
+#define HCT_UMMA_K 8
+#else
+#define HCT_BK 64                                  // 64 bf16 = one 128-byte swizzle row
+#define HCT_ELT 2
+#define HCT_UMMA_K 16
+#endif
+#define HCT_NBOX (128 / HCT_ELT)                   // B elements along N per 128-byte row
+#define HCT_A_BYTES (HCT_BM * 128)
+#define HCT_B_BYTES (HCT_BN * 128)
+#define HCT_BBOX_BYTES (HCT_NBOX * HCT_BK * HCT_ELT)  // one [BK x NBOX] box of B
+#if HCT_TF32X3
+#define HCT_STAGE_BYTES (2 * HCT_A_BYTES + 2 * HCT_B_BYTES)   // hi and lo parts of both operands
+#else
+#define HCT_STAGE_BYTES (HCT_A_BYTES + HCT_B_BYTES)
+#endif
+#define HCT_KB ((HCT_K + HCT_BK - 1) / HCT_BK)
+#define HCT_MB ((HCT_M + HCT_BM - 1) / HCT_BM)
+#define HCT_NB ((HCT_N + HCT_BN - 1) / HCT_BN)
+#define HCT_TILES ((long long)HCT_MB * HCT_NB)
+#define HCT_TMEM_COLS (2 * HCT_BN < 32 ? 32 : 2 * HCT_BN)
+
+extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __grid_constant__ HctParams hct_p) {
+  extern __shared__ unsigned char hct_smem_raw[];
+  __shared__ unsigned long long bars[2 * HCT_STAGES + 4];
+  __shared__ hct_u32 tmem_holder;
+  __shared__ int failed;
+  const hct_u32 smem_base = (hct_smem_addr(hct_smem_raw) + 1023u) & ~1023u;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  unsigned int* status = (unsigned int*)hct_p.ptr[HCT_STATUS_SLOT];
+  const hct_u32 full0 = hct_smem_addr(&bars[0]), empty0 = hct_smem_addr(&bars[HCT_STAGES]);
+  const hct_u32 tfull0 = hct_smem_addr(&bars[2 * HCT_STAGES]), tempty0 = hct_smem_addr(&bars[2 * HCT_STAGES + 2]);
+
+  if (threadIdx.x == 0) {
+    failed = 0;
+    for (int s = 0; s < HCT_STAGES; ++s) {
+      hct_mbar_init(full0 + 8 * s, 1);
+      hct_mbar_init(empty0 + 8 * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      hct_mbar_init(tfull0 + 8 * a, 1);
+      hct_mbar_init(tempty0 + 8 * a, 128);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    hct_prefetch_tmap(&hct_p.tmap[0]);
+    hct_prefetch_tmap(&hct_p.tmap[1]);
+  }
+  if (warp == 1) hct_tmem_alloc(hct_smem_addr(&tmem_holder), HCT_TMEM_COLS);
+  hct_tc_fence_before();
+  __syncthreads();
+  hct_tc_fence_after();
+  const hct_u32 tmem_base = *(volatile hct_u32*)&tmem_holder;
+
+  if (warp == 0) {
+    // ---------------- TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      hct_u32 phase = 0;
+      for (long long tile = blockIdx.x; tile < HCT_TILES; tile += gridDim.x) {
+        const int nb = (int)(tile % HCT_NB), mb = (int)(tile / HCT_NB);
+        for (int kb = 0; kb < HCT_KB; ++kb) {
+          hct_mbar_wait(empty0 + 8 * stage, phase ^ 1u, &failed, status, 1);
+          const hct_u32 full = full0 + 8 * stage;
+          hct_mbar_expect_tx(full, HCT_STAGE_BYTES);
+          hct_u32 dst = smem_base + stage * HCT_STAGE_BYTES;
+#if HCT_TF32X3
+          hct_tma_load_2d(dst, &hct_p.tmap[0], kb * HCT_BK, mb * HCT_BM, full);                    // A hi
+          hct_tma_load_2d(dst + HCT_A_BYTES, &hct_p.tmap[1], kb * HCT_BK, mb * HCT_BM, full);      // A lo
+          dst += 2 * HCT_A_BYTES;
+          for (int j = 0; j < HCT_BN / HCT_NBOX; ++j) {
+            hct_tma_load_2d(dst + j * HCT_BBOX_BYTES, &hct_p.tmap[2], nb * HCT_BN + j * HCT_NBOX, kb * HCT_BK, full);                 // B hi
+            hct_tma_load_2d(dst + HCT_B_BYTES + j * HCT_BBOX_BYTES, &hct_p.tmap[3], nb * HCT_BN + j * HCT_NBOX, kb * HCT_BK, full);   // B lo
+          }
+#else
+          hct_tma_load_2d(dst, &hct_p.tmap[0], kb * HCT_BK, mb * HCT_BM, full);
+          dst += HCT_A_BYTES;
+          for (int j = 0; j < HCT_BN / HCT_NBOX; ++j)
+            hct_tma_load_2d(dst + j * HCT_BBOX_BYTES, &hct_p.tmap[1], nb * HCT_BN + j * HCT_NBOX, kb * HCT_BK, full);
+#endif
+          if (++stage == HCT_STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      // instruction descriptor: fp32 accumulate, A K-major, B N-major, M = 128, N = HCT_BN
+#if HCT_TF32X3
+      const hct_u32 idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 16) | ((hct_u32)(HCT_BN >> 3) << 17) | ((hct_u32)(HCT_BM >> 4) << 24);
+#else
+      const hct_u32 idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((hct_u32)(HCT_BN >> 3) << 17) | ((hct_u32)(HCT_BM >> 4) << 24);
+#endif
+      int stage = 0, acc = 0;
+      hct_u32 phase = 0, acc_phase = 0;
+      for (long long tile = blockIdx.x; tile < HCT_TILES; tile += gridDim.x) {
+        hct_mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, &failed, status, 2);
+        hct_tc_fence_after();
+        const hct_u32 d_tmem = tmem_base + acc * HCT_BN;
+        for (int kb = 0; kb < HCT_KB; ++kb) {
+          hct_mbar_wait(full0 + 8 * stage, phase, &failed, status, 3);
+          hct_tc_fence_after();
+          const hct_u32 a_addr = smem_base + stage * HCT_STAGE_BYTES;
+#if HCT_TF32X3
+          const hct_u32 b_addr = a_addr + 2 * HCT_A_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < HCT_BK / HCT_UMMA_K; ++kk) {
+            // K-major A: 32 bytes further along the swizzled row; N-major B: one 8-row group (1024 bytes) further
+            const hct_u64 a_hi = hct_smem_desc(a_addr + kk * 32, 16, 1024), a_lo = hct_smem_desc(a_addr + HCT_A_BYTES + kk * 32, 16, 1024);
+            const hct_u64 b_hi = hct_smem_desc(b_addr + kk * 1024, HCT_BBOX_BYTES, 1024);
+            const hct_u64 b_lo = hct_smem_desc(b_addr + HCT_B_BYTES + kk * 1024, HCT_BBOX_BYTES, 1024);
+            // small cross terms first, then the leading product
+            hct_mma_tf32(d_tmem, a_lo, b_hi, idesc, (kb | kk) != 0);
+            hct_mma_tf32(d_tmem, a_hi, b_lo, idesc, 1);
+            hct_mma_tf32(d_tmem, a_hi, b_hi, idesc, 1);
+          }
+#else
+          const hct_u32 b_addr = a_addr + HCT_A_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < HCT_BK / HCT_UMMA_K; ++kk) {
+            const hct_u64 adesc = hct_smem_desc(a_addr + kk * 32, 16, 1024);
+            const hct_u64 bdesc = hct_smem_desc(b_addr + kk * 2048, HCT_BBOX_BYTES, 1024);
+            hct_mma_f16(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0);
+          }
+#endif
+          hct_mma_commit(empty0 + 8 * stage);   // frees the stage once these MMAs have read it
+          if (++stage == HCT_STAGES) { stage = 0; phase ^= 1u; }
+        }
+        hct_mma_commit(tfull0 + 8 * acc);       // accumulator complete
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ---------------- epilogue: warp w may only touch TMEM lanes 32 (w mod 4) .. +31
+    const int q = warp & 3;
+    int acc = 0;
+    hct_u32 acc_phase = 0;
+    for (long long tile = blockIdx.x; tile < HCT_TILES; tile += gridDim.x) {
+      const int nb = (int)(tile % HCT_NB), mb = (int)(tile / HCT_NB);
+      hct_mbar_wait(tfull0 + 8 * acc, acc_phase, &failed, status, 4);
+      hct_tc_fence_after();
+      const long long row = (long long)mb * HCT_BM + q * 32 + lane;
+#pragma unroll 1
+      for (int c = 0; c < HCT_BN / 32; ++c) {
+        float v[32];
+        hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * HCT_BN + c * 32, v);
+        const long long col0 = (long long)nb * HCT_BN + c * 32;
+        const int ncols = (int)(HCT_N - col0 < 32 ? HCT_N - col0 : 32);
+        if (row < HCT_M && ncols > 0) hct_epilogue_run(hct_p, v, row, (int)col0, ncols);
+      }
+      hct_tc_fence_before();
+      hct_mbar_arrive(tempty0 + 8 * acc);
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+  }
+  hct_tc_fence_before();
+  __syncthreads();
+  if (warp == 1) hct_tmem_dealloc(tmem_base, HCT_TMEM_COLS);
+}
