@@ -183,6 +183,87 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     }
   }
 
+  // ---- tensor-core GEMM on fp32 operands: split pre-pass, then three TF32 products per k step
+  if (grp.kind == GroupKind::Gemm && !tun.simt_only) {
+    int64_t M = a.shape[0], K = a.shape[1], N = b.shape[1];
+    DType da = g.nodes[anchor.args[0].node].cls == OpClass::Input ? a.dtype : F32;
+    DType db = g.nodes[anchor.args[1].node].cls == OpClass::Input ? b.dtype : F32;
+    if (da == F32 && db == F32 && K % 4 == 0 && M <= 0x7fffffff && N <= 0x7fffffff && K <= 0x7fffffff) {
+      auto align256 = [](int64_t v) { return (v + 255) / 256 * 256; };
+      const int64_t a_bytes = align256(M * K * 4), b_bytes = align256(K * N * 4);
+      const int64_t off_ahi = 0, off_alo = a_bytes, off_bhi = 2 * a_bytes, off_blo = 2 * a_bytes + b_bytes;
+      *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(2 * a_bytes + 2 * b_bytes));
+      auto scratch = [](int64_t off) {
+        BufRef r;
+        r.kind = BufRef::Scratch;
+        r.scratch_off = off;
+        return r;
+      };
+      auto node_buf = [&](int node) {
+        BufRef r;
+        r.node = node;
+        r.ws_copy = g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0;
+        return r;
+      };
+      {  // split pre-pass
+        KernelSpec k;
+        k.name = "hct_split_tf32_g" + std::to_string(gi);
+        std::ostringstream src;
+        src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n#define HCT_KERNEL_NAME " << k.name << "\n"
+            << skeleton_source("common") << "\nstruct HctParams { void* ptr[6]; };\n" << skeleton_source("split_tf32");
+        k.source = src.str();
+        k.ptrs = {node_buf(anchor.args[0].node), node_buf(anchor.args[1].node), scratch(off_ahi), scratch(off_alo), scratch(off_bhi),
+                  scratch(off_blo)};
+        int64_t blocks = (M * K / 4 + 1023) / 1024 + ((K + 31) / 32) * ((N + 31) / 32);
+        k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(blocks, 148 * 16));
+        k.block[0] = 256;
+        k.desc = "tf32 head/tail split of both gemm operands, B transposed";
+        out->push_back(k);
+      }
+      int BN = N > 64 ? 128 : N > 32 ? 64 : 32;
+      int stages = BN == 128 ? 3 : BN == 64 ? 4 : 5;
+      std::string epi = eg.run_fn(N);
+      KernelSpec k;
+      k.name = "hct_gemm_tc_tf32x3_g" + std::to_string(gi);
+      std::ostringstream src;
+      src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n#define HCT_BN " << BN
+          << "\n#define HCT_STAGES " << stages << "\n#define HCT_TF32X3 1\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
+          << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
+      src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[4]; void* ptr["
+          << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source("gemm_tc");
+      k.source = src.str();
+      k.ptrs = eg.ptrs;
+      k.wants_status = true;
+      for (int i = 0; i < 4; ++i) {
+        TmaDesc t;
+        t.buf = scratch(i == 0 ? off_ahi : i == 1 ? off_alo : i == 2 ? off_bhi : off_blo);
+        t.elem_bytes = 4;
+        t.rank = 2;
+        if (i < 2) {
+          t.dims[0] = (uint64_t)K; t.dims[1] = (uint64_t)M;
+          t.strides[1] = (uint64_t)K * 4;
+          t.box[0] = 32; t.box[1] = 128;
+        } else {  // B transposed to [N,K]
+          t.dims[0] = (uint64_t)K; t.dims[1] = (uint64_t)N;
+          t.strides[1] = (uint64_t)K * 4;
+          t.box[0] = 32; t.box[1] = (uint32_t)BN;
+        }
+        k.tmaps.push_back(t);
+      }
+      int64_t tiles = ((M + 127) / 128) * ((N + BN - 1) / BN);
+      k.block[0] = 192;
+      k.smem_bytes = (unsigned)(stages * (2 * 128 * 128 + 2 * BN * 128) + 1024);
+      k.persistent = true;
+      k.max_grid = (unsigned)std::min<int64_t>(tiles, 0x7fffffff);
+      k.grid[0] = k.max_grid;
+      std::ostringstream d;
+      d << "gemm tcgen05 tf32x3 128x" << BN << "x32, " << stages << " stages";
+      k.desc = d.str();
+      out->push_back(k);
+      return;
+    }
+  }
+
   auto operand_buf = [&](int node) {
     return eg.ptr_index(node, g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0);
   };

@@ -1,7 +1,8 @@
 // Persistent tensor-core GEMM with fused epilogue:  D[M,N] = epilogue(A[M,K] * B[K,N]).
 //
 // One CTA per SM walks over 128 x HCT_BN output tiles.  Warp 0 feeds a ring of shared-memory
-// stages with TMA tile loads (A is K-major, B is row-major [K,N], i.e. N-major), warp 1 issues
+// stages with TMA tile loads (A is K-major; bf16 B is row-major [K,N], i.e. N-major; the TF32
+// variant reads B already transposed to [N,K] by its split pre-pass), warp 1 issues
 // tcgen05.mma from those stages into one of two accumulators in tensor memory, warps 2..5 drain
 // the other accumulator (tcgen05.ld), apply the generated epilogue and store, so the epilogue of
 // tile i overlaps the main loop of tile i+1.  All hand-offs are mbarriers with bounded waits.
@@ -28,6 +29,17 @@
 #define HCT_STAGE_BYTES (HCT_A_BYTES + HCT_B_BYTES)
 #endif
 #define HCT_KB ((HCT_K + HCT_BK - 1) / HCT_BK)
+// The tensor core adds into its fp32 accumulator with truncation, which biases long sums by about
+// 1e-8 per accumulated element.  The TF32 variant therefore accumulates at most HCT_KBC k-blocks
+// (128 elements of K) in tensor memory and sums those partial results in registers, rounding to
+// nearest; the bf16 variant, judged at 2e-2, accumulates the whole K extent in tensor memory.
+#if HCT_TF32X3
+#define HCT_KBC 4
+#else
+#define HCT_KBC HCT_KB
+#endif
+#define HCT_NCH ((HCT_KB + HCT_KBC - 1) / HCT_KBC)
+#define HCT_NCH_IS_ONE (!HCT_TF32X3)
 #define HCT_MB ((HCT_M + HCT_BM - 1) / HCT_BM)
 #define HCT_NB ((HCT_N + HCT_BN - 1) / HCT_BN)
 #define HCT_TILES ((long long)HCT_MB * HCT_NB)
@@ -80,10 +92,8 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
           hct_tma_load_2d(dst, &hct_p.tmap[0], kb * HCT_BK, mb * HCT_BM, full);                    // A hi
           hct_tma_load_2d(dst + HCT_A_BYTES, &hct_p.tmap[1], kb * HCT_BK, mb * HCT_BM, full);      // A lo
           dst += 2 * HCT_A_BYTES;
-          for (int j = 0; j < HCT_BN / HCT_NBOX; ++j) {
-            hct_tma_load_2d(dst + j * HCT_BBOX_BYTES, &hct_p.tmap[2], nb * HCT_BN + j * HCT_NBOX, kb * HCT_BK, full);                 // B hi
-            hct_tma_load_2d(dst + HCT_B_BYTES + j * HCT_BBOX_BYTES, &hct_p.tmap[3], nb * HCT_BN + j * HCT_NBOX, kb * HCT_BK, full);   // B lo
-          }
+          hct_tma_load_2d(dst, &hct_p.tmap[2], kb * HCT_BK, nb * HCT_BN, full);                    // B^T hi
+          hct_tma_load_2d(dst + HCT_B_BYTES, &hct_p.tmap[3], kb * HCT_BK, nb * HCT_BN, full);      // B^T lo
 #else
           hct_tma_load_2d(dst, &hct_p.tmap[0], kb * HCT_BK, mb * HCT_BM, full);
           dst += HCT_A_BYTES;
@@ -97,19 +107,21 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
   } else if (warp == 1) {
     // ---------------- MMA issuer
     if (lane == 0) {
-      // instruction descriptor: fp32 accumulate, A K-major, B N-major, M = 128, N = HCT_BN
+      // instruction descriptor: fp32 accumulate, A K-major, B N-major (bf16) or K-major (TF32), M = 128, N = HCT_BN
 #if HCT_TF32X3
-      const hct_u32 idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 16) | ((hct_u32)(HCT_BN >> 3) << 17) | ((hct_u32)(HCT_BM >> 4) << 24);
+      const hct_u32 idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((hct_u32)(HCT_BN >> 3) << 17) | ((hct_u32)(HCT_BM >> 4) << 24);
 #else
       const hct_u32 idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((hct_u32)(HCT_BN >> 3) << 17) | ((hct_u32)(HCT_BM >> 4) << 24);
 #endif
       int stage = 0, acc = 0;
       hct_u32 phase = 0, acc_phase = 0;
       for (long long tile = blockIdx.x; tile < HCT_TILES; tile += gridDim.x) {
+       for (int ch = 0; ch < HCT_NCH; ++ch) {
         hct_mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, &failed, status, 2);
         hct_tc_fence_after();
         const hct_u32 d_tmem = tmem_base + acc * HCT_BN;
-        for (int kb = 0; kb < HCT_KB; ++kb) {
+        const int kb0 = ch * HCT_KBC, kb1 = kb0 + HCT_KBC < HCT_KB ? kb0 + HCT_KBC : HCT_KB;
+        for (int kb = kb0; kb < kb1; ++kb) {
           hct_mbar_wait(full0 + 8 * stage, phase, &failed, status, 3);
           hct_tc_fence_after();
           const hct_u32 a_addr = smem_base + stage * HCT_STAGE_BYTES;
@@ -117,12 +129,11 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
           const hct_u32 b_addr = a_addr + 2 * HCT_A_BYTES;
 #pragma unroll
           for (int kk = 0; kk < HCT_BK / HCT_UMMA_K; ++kk) {
-            // K-major A: 32 bytes further along the swizzled row; N-major B: one 8-row group (1024 bytes) further
+            // both operands K-major: one MMA step is 32 bytes further along the swizzled rows
             const hct_u64 a_hi = hct_smem_desc(a_addr + kk * 32, 16, 1024), a_lo = hct_smem_desc(a_addr + HCT_A_BYTES + kk * 32, 16, 1024);
-            const hct_u64 b_hi = hct_smem_desc(b_addr + kk * 1024, HCT_BBOX_BYTES, 1024);
-            const hct_u64 b_lo = hct_smem_desc(b_addr + HCT_B_BYTES + kk * 1024, HCT_BBOX_BYTES, 1024);
+            const hct_u64 b_hi = hct_smem_desc(b_addr + kk * 32, 16, 1024), b_lo = hct_smem_desc(b_addr + HCT_B_BYTES + kk * 32, 16, 1024);
             // small cross terms first, then the leading product
-            hct_mma_tf32(d_tmem, a_lo, b_hi, idesc, (kb | kk) != 0);
+            hct_mma_tf32(d_tmem, a_lo, b_hi, idesc, (kb > kb0) || (kk != 0));
             hct_mma_tf32(d_tmem, a_hi, b_lo, idesc, 1);
             hct_mma_tf32(d_tmem, a_hi, b_hi, idesc, 1);
           }
@@ -132,15 +143,16 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
           for (int kk = 0; kk < HCT_BK / HCT_UMMA_K; ++kk) {
             const hct_u64 adesc = hct_smem_desc(a_addr + kk * 32, 16, 1024);
             const hct_u64 bdesc = hct_smem_desc(b_addr + kk * 2048, HCT_BBOX_BYTES, 1024);
-            hct_mma_f16(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0);
+            hct_mma_f16(d_tmem, adesc, bdesc, idesc, (kb > kb0) || (kk != 0));
           }
 #endif
           hct_mma_commit(empty0 + 8 * stage);   // frees the stage once these MMAs have read it
           if (++stage == HCT_STAGES) { stage = 0; phase ^= 1u; }
         }
-        hct_mma_commit(tfull0 + 8 * acc);       // accumulator complete
+        hct_mma_commit(tfull0 + 8 * acc);       // this chunk's accumulator is complete
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
+       }
       }
     }
   } else {
@@ -150,9 +162,10 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
     hct_u32 acc_phase = 0;
     for (long long tile = blockIdx.x; tile < HCT_TILES; tile += gridDim.x) {
       const int nb = (int)(tile % HCT_NB), mb = (int)(tile / HCT_NB);
+      const long long row = (long long)mb * HCT_BM + q * 32 + lane;
+#if HCT_NCH_IS_ONE
       hct_mbar_wait(tfull0 + 8 * acc, acc_phase, &failed, status, 4);
       hct_tc_fence_after();
-      const long long row = (long long)mb * HCT_BM + q * 32 + lane;
 #pragma unroll 1
       for (int c = 0; c < HCT_BN / 32; ++c) {
         float v[32];
@@ -165,6 +178,33 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
       hct_mbar_arrive(tempty0 + 8 * acc);
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
+#else
+      float sum[HCT_BN];
+#pragma unroll
+      for (int j = 0; j < HCT_BN; ++j) sum[j] = 0.0f;
+#pragma unroll 1
+      for (int ch = 0; ch < HCT_NCH; ++ch) {
+        hct_mbar_wait(tfull0 + 8 * acc, acc_phase, &failed, status, 4);
+        hct_tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < HCT_BN / 32; ++c) {
+          float v[32];
+          hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * HCT_BN + c * 32, v);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) sum[c * 32 + j] += v[j];
+        }
+        hct_tc_fence_before();
+        hct_mbar_arrive(tempty0 + 8 * acc);
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+#pragma unroll
+      for (int c = 0; c < HCT_BN / 32; ++c) {
+        const long long col0 = (long long)nb * HCT_BN + c * 32;
+        const int ncols = (int)(HCT_N - col0 < 32 ? HCT_N - col0 : 32);
+        if (row < HCT_M && ncols > 0) hct_epilogue_run(hct_p, *(float(*)[32])(sum + c * 32), row, (int)col0, ncols);
+      }
+#endif
     }
   }
   hct_tc_fence_before();
