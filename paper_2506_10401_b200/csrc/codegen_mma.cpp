@@ -121,6 +121,55 @@ struct EpiGen {
     f << "}\n";
     return f.str();
   }
+
+  // Epilogue of the tensor-core convolution: one thread owns one output pixel (n,h,w) and 32
+  // consecutive output channels k0..k0+31, `nk` of which exist.  NCHW: channel j lies j planes further.
+  std::string conv_fn(int64_t KO, int64_t HO, int64_t WO) {
+    std::ostringstream f;
+    f << "__device__ __forceinline__ void hct_epilogue_conv(const HctParams& hct_p, float (&acc)[32], int n, int h, int w, int k0, int nk) {\n";
+    f << "  const long long plane = " << HO * WO << "LL;\n";
+    f << "  const long long off0 = (((long long)n * " << KO << "LL + k0) * " << HO << "LL + h) * " << WO << "LL + w;\n";
+    int anchor = grp.nodes[0];
+    auto ref = [&](const Operand& a) -> std::string {
+      if (a.is_literal()) return float_lit(a.literal);
+      if (p.group_of[a.node] == gi) return a.node == anchor ? "acc[j]" : "e" + std::to_string(a.node);
+      int k = find_ext(grp, a.node);
+      const ExtOperand& e = grp.ext[k];
+      if (e.bcast == Bcast::Scalar) return "c" + std::to_string(k);
+      return "x" + std::to_string(k) + "[j]";
+    };
+    for (size_t k = 0; k < grp.ext.size(); ++k) {
+      const ExtOperand& e = grp.ext[k];
+      int pi = ptr_index(e.node, is_ws(e.node));
+      DType d = buf_dtype(e.node);
+      std::string ptr = std::string("((const ") + ctype(d) + "*)hct_p.ptr[" + std::to_string(pi) + "])";
+      switch (e.bcast) {
+        case Bcast::RowIdx:  // per-channel operand [K,1,1]
+          f << "  float x" << k << "[32]; hct_ld_run32<" << ctype(d) << ">(" << ptr << " + k0, x" << k << ", nk, true);\n";
+          break;
+        case Bcast::Full:
+          f << "  float x" << k << "[32];\n  _Pragma(\"unroll\") for (int j = 0; j < 32; ++j) x" << k << "[j] = j < nk ? hct_ld1(" << ptr
+            << " + off0 + j * plane) : 0.0f;\n";
+          break;
+        case Bcast::Scalar: f << "  const float c" << k << " = hct_ld1(" << ptr << ");\n"; break;
+        case Bcast::RowVec: throw Error(HCT_ERR_UNSUPPORTED, "row-vector operand in a convolution epilogue");
+      }
+    }
+    f << "  _Pragma(\"unroll\") for (int j = 0; j < 32; ++j) {\n";
+    for (size_t i = 1; i < grp.nodes.size(); ++i) {
+      const Node& nd = g.nodes[grp.nodes[i]];
+      f << "    const float e" << grp.nodes[i] << " = hct_" << nd.op << "(";
+      for (size_t a = 0; a < nd.args.size(); ++a) f << (a ? ", " : "") << ref(nd.args[a]);
+      f << ");  // " << nd.name << "\n";
+    }
+    for (auto& st : grp.stores) {
+      int pi = ptr_index(st.node, !st.to_output);
+      f << "    if (j < nk) hct_st1((" << ctype(st.dtype) << "*)hct_p.ptr[" << pi << "] + off0 + j * plane, "
+        << (st.node == anchor ? "acc[j]" : "e" + std::to_string(st.node)) << ");\n";
+    }
+    f << "  }\n}\n";
+    return f.str();
+  }
 };
 
 }  // namespace
@@ -258,6 +307,89 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       k.grid[0] = k.max_grid;
       std::ostringstream d;
       d << "gemm tcgen05 tf32x3 128x" << BN << "x32, " << stages << " stages";
+      k.desc = d.str();
+      out->push_back(k);
+      return;
+    }
+  }
+
+  // ---- tensor-core convolution: bf16 inputs, stride 1; layout pre-pass, then implicit GEMM
+  if (grp.kind == GroupKind::Conv && !tun.simt_only) {
+    const auto& xs = a.shape;
+    const auto& ws = b.shape;
+    bool in_bf16 = a.cls == OpClass::Input && b.cls == OpClass::Input && a.dtype == BF16 && b.dtype == BF16;
+    int64_t NB = xs[0], C = xs[1], H = xs[2], W = xs[3], KO = ws[0], FR = ws[2], FS = ws[3];
+    int64_t HO = anchor.shape[2], WO = anchor.shape[3];
+    if (in_bf16 && anchor.stride == 1 && C % 8 == 0 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
+      auto align256 = [](int64_t v) { return (v + 255) / 256 * 256; };
+      const int64_t x_bytes = align256(NB * C * H * W * 2), w_bytes = align256(KO * C * FR * FS * 2);
+      *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(x_bytes + w_bytes));
+      auto scratch = [](int64_t off) {
+        BufRef r;
+        r.kind = BufRef::Scratch;
+        r.scratch_off = off;
+        return r;
+      };
+      auto node_buf = [&](int node) {
+        BufRef r;
+        r.node = node;
+        return r;
+      };
+      {
+        KernelSpec k;
+        k.name = "hct_conv_prep_g" + std::to_string(gi);
+        std::ostringstream src;
+        src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_HW " << H * W << "\n#define HCT_KO " << KO
+            << "\n#define HCT_RS " << FR * FS << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+            << skeleton_source("common") << "\nstruct HctParams { void* ptr[4]; };\n" << skeleton_source("conv_prep");
+        k.source = src.str();
+        k.ptrs = {node_buf(anchor.args[0].node), node_buf(anchor.args[1].node), scratch(0), scratch(x_bytes)};
+        int64_t blocks = NB * ((C + 63) / 64) * ((H * W + 63) / 64) + (KO * C * FR * FS + 255) / 256;
+        k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(blocks, 148 * 16));
+        k.block[0] = 256;
+        k.desc = "conv layout pre-pass: NCHW->NHWC activations, KCRS->RSKC weights";
+        out->push_back(k);
+      }
+      int TW = (int)std::min<int64_t>(WO, 128);
+      int TH = (int)std::max<int64_t>(1, std::min<int64_t>(128 / TW, HO));
+      int BN = KO > 64 ? 128 : KO > 32 ? 64 : 32;
+      int stages = BN == 128 ? 6 : 8;
+      std::string epi = eg.conv_fn(KO, HO, WO);
+      KernelSpec k;
+      k.name = "hct_conv_tc_bf16_g" + std::to_string(gi);
+      std::ostringstream src;
+      src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_H " << H << "\n#define HCT_W " << W
+          << "\n#define HCT_KO " << KO << "\n#define HCT_FR " << FR << "\n#define HCT_FS " << FS << "\n#define HCT_PAD " << anchor.pad
+          << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TW " << TW << "\n#define HCT_TH " << TH
+          << "\n#define HCT_BN " << BN << "\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
+          << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
+      src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[2]; void* ptr["
+          << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source("conv_tc");
+      k.source = src.str();
+      k.ptrs = eg.ptrs;
+      k.wants_status = true;
+      TmaDesc tx, tw;
+      tx.buf = scratch(0);
+      tx.elem_bytes = 2;
+      tx.rank = 4;
+      tx.dims[0] = (uint64_t)C; tx.dims[1] = (uint64_t)W; tx.dims[2] = (uint64_t)H; tx.dims[3] = (uint64_t)NB;
+      tx.strides[1] = (uint64_t)C * 2; tx.strides[2] = (uint64_t)W * C * 2; tx.strides[3] = (uint64_t)H * W * C * 2;
+      tx.box[0] = 64; tx.box[1] = (uint32_t)TW; tx.box[2] = (uint32_t)TH; tx.box[3] = 1;
+      tw.buf = scratch(x_bytes);
+      tw.elem_bytes = 2;
+      tw.rank = 2;
+      tw.dims[0] = (uint64_t)C; tw.dims[1] = (uint64_t)(FR * FS * KO);
+      tw.strides[1] = (uint64_t)C * 2;
+      tw.box[0] = 64; tw.box[1] = (uint32_t)BN;
+      k.tmaps = {tx, tw};
+      int64_t tiles = NB * ((HO + TH - 1) / TH) * ((WO + TW - 1) / TW) * ((KO + BN - 1) / BN);
+      k.block[0] = 192;
+      k.smem_bytes = (unsigned)(stages * (128 * 128 + BN * 128) + 1024);
+      k.persistent = true;
+      k.max_grid = (unsigned)std::min<int64_t>(tiles, 0x7fffffff);
+      k.grid[0] = k.max_grid;
+      std::ostringstream d;
+      d << "conv2d tcgen05 bf16 implicit GEMM, tile " << TH << "x" << TW << " pixels x " << BN << " channels, " << stages << " stages";
       k.desc = d.str();
       out->push_back(k);
       return;

@@ -1,0 +1,44 @@
+// Layout pre-pass for the tensor-core convolution: activations NCHW -> NHWC and weights
+// KCRS -> RSKC (both bf16), so that channels, the contraction axis, are contiguous for TMA.
+// Defined by the generator: HCT_NB_IMG, HCT_C, HCT_HW (H*W), HCT_KO, HCT_RS (R*S), HctParams, HCT_KERNEL_NAME.
+// Pointer slots: 0 = X (NCHW), 1 = Wt (KCRS), 2 = X as NHWC, 3 = Wt as RSKC.
+#define HCT_XT_C ((HCT_C + 63) / 64)
+#define HCT_XT_P ((HCT_HW + 63) / 64)
+#define HCT_X_BLOCKS ((long long)HCT_NB_IMG * HCT_XT_C * HCT_XT_P)
+#define HCT_W_ELEMS ((long long)HCT_KO * HCT_C * HCT_RS)
+#define HCT_W_BLOCKS ((HCT_W_ELEMS + 255) / 256)
+extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {
+  __shared__ hct_bf16_t tile[64][66];
+  const hct_bf16_t* __restrict__ X = (const hct_bf16_t*)hct_p.ptr[0];
+  const hct_bf16_t* __restrict__ Wt = (const hct_bf16_t*)hct_p.ptr[1];
+  hct_bf16_t* __restrict__ Xo = (hct_bf16_t*)hct_p.ptr[2];
+  hct_bf16_t* __restrict__ Wo = (hct_bf16_t*)hct_p.ptr[3];
+  for (long long blk = blockIdx.x; blk < HCT_X_BLOCKS + HCT_W_BLOCKS; blk += gridDim.x) {
+    if (blk < HCT_X_BLOCKS) {
+      const long long n = blk / (HCT_XT_C * HCT_XT_P);
+      const int rem = (int)(blk % (HCT_XT_C * HCT_XT_P));
+      const int c0 = (rem / HCT_XT_P) * 64, p0 = (rem % HCT_XT_P) * 64;
+      const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;  // 64 x 4
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int c = c0 + ty + 4 * i, p = p0 + tx;
+        tile[ty + 4 * i][tx] = (c < HCT_C && p < HCT_HW) ? X[(n * HCT_C + c) * HCT_HW + p] : (hct_bf16_t)0;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int p = p0 + ty + 4 * i, c = c0 + tx;
+        if (p < HCT_HW && c < HCT_C) Xo[(n * HCT_HW + p) * HCT_C + c] = tile[tx][ty + 4 * i];
+      }
+      __syncthreads();
+    } else {
+      const long long i = (blk - HCT_X_BLOCKS) * 256 + threadIdx.x;   // index into RSKC
+      if (i < HCT_W_ELEMS) {
+        const int c = (int)(i % HCT_C);
+        const int k = (int)((i / HCT_C) % HCT_KO);
+        const int rs = (int)(i / ((long long)HCT_C * HCT_KO));
+        Wo[i] = Wt[((long long)k * HCT_C + c) * HCT_RS + rs];
+      }
+    }
+  }
+}
