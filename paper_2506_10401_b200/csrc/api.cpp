@@ -25,6 +25,9 @@ struct LoadedKernel {
   CUmodule_t module = nullptr;
   CUfunction_t func = nullptr;
   unsigned grid[3] = {1, 1, 1};
+  // tensor maps embed the base address: re-encoded only when a buffer moves between runs
+  std::vector<TensorMap> tmaps;
+  std::vector<void*> tmap_base;
 };
 
 std::string cu_error(const Driver& d, CUresult_t rc, const char* what) {
@@ -131,7 +134,7 @@ hct_status_t hct_graph_create(const char* spec, size_t spec_len, int device, hct
         if (rc != 0) throw Error(HCT_ERR_COMPILE, cu_error(*d, rc, "cuModuleLoadData"));
         rc = d->ModuleGetFunction(&lk.func, lk.module, ks.name.c_str());
         if (rc != 0) throw Error(HCT_ERR_COMPILE, cu_error(*d, rc, "cuModuleGetFunction"));
-        if (ks.smem_bytes > 48 * 1024) {
+        if (ks.smem_bytes > 0) {
           rc = d->FuncSetAttribute(lk.func, kFuncAttrMaxDynamicSharedSizeBytes, (int)ks.smem_bytes);
           if (rc != 0) throw Error(HCT_ERR_CUDA, cu_error(*d, rc, "cuFuncSetAttribute(max dynamic shared memory)"));
         }
@@ -195,14 +198,22 @@ hct_status_t hct_graph_run(hct_graph_t* g, const void* const* inputs, int n_inpu
       void* ptrs[32];
       for (size_t i = 0; i < k.spec.ptrs.size(); ++i) ptrs[i] = resolve(g, k.spec.ptrs[i], inputs, outputs, (char*)workspace);
       if (k.spec.wants_status) ptrs[np - 1] = (void*)g->status_word;
+      if (k.tmaps.size() != ntm) {
+        k.tmaps.assign(ntm, TensorMap());
+        k.tmap_base.assign(ntm, nullptr);
+      }
       for (size_t i = 0; i < ntm; ++i) {
         const TmaDesc& t = k.spec.tmaps[i];
         void* base = resolve(g, t.buf, inputs, outputs, (char*)workspace);
-        uint32_t estr[5] = {1, 1, 1, 1, 1};
-        int dtype = t.elem_bytes == 2 ? 9 /* bf16 */ : 7 /* fp32 */;
-        CUresult_t rc = d.TensorMapEncodeTiled(&params.tmap[i], dtype, (unsigned)t.rank, base, t.dims, t.strides + 1, t.box, estr,
-                                               0 /* no interleave */, t.swizzle, 2 /* L2 promotion 128B */, 0 /* zero fill */);
-        if (rc != 0) return set_error(HCT_ERR_CUDA, cu_error(d, rc, "cuTensorMapEncodeTiled"));
+        if (base != k.tmap_base[i]) {
+          uint32_t estr[5] = {1, 1, 1, 1, 1};
+          int dtype = t.elem_bytes == 2 ? 9 /* bf16 */ : 7 /* fp32 */;
+          CUresult_t rc = d.TensorMapEncodeTiled(&k.tmaps[i], dtype, (unsigned)t.rank, base, t.dims, t.strides + 1, t.box, estr,
+                                                 0 /* no interleave */, t.swizzle, 2 /* L2 promotion 128B */, 0 /* zero fill */);
+          if (rc != 0) return set_error(HCT_ERR_CUDA, cu_error(d, rc, "cuTensorMapEncodeTiled"));
+          k.tmap_base[i] = base;
+        }
+        params.tmap[i] = k.tmaps[i];
       }
       // the kernel's single by-value argument is either {ptr[]} or {tmap[], ptr[]}
       alignas(64) char block[sizeof(Params)];

@@ -13,6 +13,8 @@ Tunables Tunables::from_env() {
   if (const char* s = std::getenv("HCT_ROW_NV")) t.row_nv = std::max(1, std::atoi(s));
   if (const char* s = std::getenv("HCT_ROW_CTA")) t.row_cta = std::max(32, std::atoi(s));
   if (const char* s = std::getenv("HCT_SIMT_ONLY")) t.simt_only = std::atoi(s) != 0;
+  if (const char* s = std::getenv("HCT_ROW_NO_STAGE")) t.row_no_stage = std::atoi(s) != 0;
+  if (const char* s = std::getenv("HCT_ROW_RING_BYTES")) t.row_ring_bytes = std::max(1024, std::atoi(s));
   return t;
 }
 
@@ -90,12 +92,29 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   // whole warps only
   while ((G * T) % 32 != 0) ++G;
 
+  // Staging through shared memory: every full-width external input whose rows are 16-byte multiples
+  int64_t stage_bytes = 0;
+  bool staged = T >= 32 && V == 4 && !tun.row_no_stage;
+  for (auto& e : grp.ext)
+    if (e.bcast == Bcast::Full) {
+      int64_t rb = C * (g.nodes[e.node].cls == OpClass::Input && g.nodes[e.node].dtype == BF16 ? 2 : 4);
+      if (rb % 16 != 0) staged = false;
+      stage_bytes += rb;
+    }
+  if (stage_bytes == 0) staged = false;
+  int nstg = 0;
+  if (staged) {
+    nstg = (int)std::min<int64_t>(8, tun.row_ring_bytes / (G * stage_bytes));
+    if (nstg < 2) staged = false;
+  }
+
   RowGen rg{g, p, grp, gi, {}, {}};
   std::ostringstream& b = rg.body;
   std::string name = "hct_row_g" + std::to_string(gi);
 
   // ---- external operands
-  std::ostringstream pre, loads;
+  std::ostringstream pre, loads, issue, other_loads;
+  int64_t staged_off = 0;
   for (size_t k = 0; k < grp.ext.size(); ++k) {
     const ExtOperand& e = grp.ext[k];
     int pi = rg.ptr_index(e.node, rg.ext_is_ws(e.node));
@@ -103,7 +122,13 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
     pre << "    const " << ct << "* __restrict__ q" << k << " = (const " << ct << "*)hct_p.ptr[" << pi << "];\n";
     switch (e.bcast) {
       case Bcast::Full:
-        loads << "      float x" << k << "[HCT_E]; hct_load_row(q" << k << ", hct_row, hct_t, x" << k << ", false);\n";
+        if (staged) {
+          loads << "      float x" << k << "[HCT_E]; hct_read_staged<" << ct << ">(hct_slot + " << staged_off << ", hct_t, x" << k << ");\n";
+          issue << "        HCT_STAGED_ISSUE_ONE(q" << k << ", " << staged_off << ", " << C * (rg.ext_dtype(e.node) == BF16 ? 2 : 4) << ")\n";
+          staged_off += C * (rg.ext_dtype(e.node) == BF16 ? 2 : 4);
+        } else {
+          loads << "      float x" << k << "[HCT_E]; hct_load_row(q" << k << ", hct_row, hct_t, x" << k << ", false);\n";
+        }
         break;
       case Bcast::RowVec:
         loads << "      float x" << k << "[HCT_E]; hct_load_row(q" << k << ", 0, hct_t, x" << k << ", true);\n";
@@ -156,9 +181,10 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         << "        float m_ = -HCT_INF;\n"
         << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) if (HCT_HAS(e)) m_ = fmaxf(m_, " << a << ");\n"
         << "        m_ = HCT_RMAX(m_);\n"
+        << "        const float ml_ = -m_ * HCT_LOG2E;\n"
         << "        float d_ = 0.0f;\n"
-        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) { v" << id << "[e] = HCT_HAS(e) ? hct_exp(" << a
-        << " - m_) : 0.0f; d_ += v" << id << "[e]; }\n"
+        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) { v" << id << "[e] = HCT_HAS(e) ? hct_exp2_fast(fmaf(" << a
+        << ", HCT_LOG2E, ml_)) : 0.0f; d_ += v" << id << "[e]; }\n"
         << "        d_ = HCT_RSUM(d_);\n"
         << "        const float inv_ = 1.0f / d_;\n"
         << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) v" << id << "[e] *= inv_;\n"
@@ -197,13 +223,39 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   }
 
   std::ostringstream src;
+  const size_t nptr = rg.ptrs.size() + (staged ? 1 : 0);
   src << "#define HCT_T " << T << "\n#define HCT_G " << G << "\n#define HCT_V " << V << "\n#define HCT_NV " << NV << "\n"
-      << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "\n#define HCT_NPTR " << std::max<size_t>(1, rg.ptrs.size()) << "\n"
-      << skeleton_source("common") << "\n"
-      << skeleton_source("row") << "\n"
-      << "HCT_ROW_KERNEL_BEGIN(" << name << ")\n"
-      << pre.str() << "  HCT_ROW_LOOP_BEGIN\n"
-      << loads.str() << b.str() << stores.str() << "  HCT_ROW_LOOP_END\nHCT_ROW_KERNEL_END\n";
+      << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "\n#define HCT_NPTR " << std::max<size_t>(1, nptr) << "\n";
+  if (staged)
+    src << "#define HCT_STAGED 1\n#define HCT_NSTG " << nstg << "\n#define HCT_STAGE_BYTES " << stage_bytes << "\n#define HCT_STATUS_SLOT "
+        << rg.ptrs.size() << "\n";
+  src << skeleton_source("common") << "\n" << skeleton_source("row") << "\n";
+  if (!staged) {
+    src << "HCT_ROW_KERNEL_BEGIN(" << name << ")\n"
+        << pre.str() << "  HCT_ROW_LOOP_BEGIN\n"
+        << loads.str() << b.str() << stores.str() << "  HCT_ROW_LOOP_END\nHCT_ROW_KERNEL_END\n";
+  } else {
+    src << "HCT_STAGED_KERNEL_BEGIN(" << name << ")\n"
+        << pre.str()
+        << "    const long long hct_stride = (long long)gridDim.x * HCT_G;\n"
+        << "    if (hct_t == 0) {\n"
+        << "      for (int s_ = 0; s_ < HCT_NSTG; ++s_) {\n"
+        << "        HCT_STAGED_ISSUE_BEGIN((long long)blockIdx.x * HCT_G + hct_cx.g + s_ * hct_stride, s_)\n"
+        << issue.str() << "        HCT_STAGED_ISSUE_END\n      }\n    }\n"
+        << "    int hct_it = 0;\n"
+        << "  HCT_ROW_LOOP_BEGIN\n"
+        << "    if (hct_live) {\n"
+        << "      const int hct_s = hct_it % HCT_NSTG;\n"
+        << "      hct_row_mbar_wait(hct_smem_u32(&hct_full[hct_cx.g][hct_s]), (hct_u32)((hct_it / HCT_NSTG) & 1), &hct_failed, hct_status);\n"
+        << "      const unsigned char* hct_slot = hct_my_ring + (size_t)hct_s * HCT_STAGE_BYTES;\n"
+        << loads.str()
+        << "      HCT_GROUP_SYNC;  // every thread of the row has taken its share: the slot may be refilled\n"
+        << "      if (hct_t == 0) {\n"
+        << "        HCT_STAGED_ISSUE_BEGIN(hct_row + HCT_NSTG * hct_stride, hct_s)\n"
+        << issue.str() << "        HCT_STAGED_ISSUE_END\n      }\n"
+        << b.str() << stores.str() << "    }\n    ++hct_it;\n"
+        << "  HCT_ROW_LOOP_END\nHCT_ROW_KERNEL_END\n";
+  }
 
   KernelSpec k;
   k.name = name;
@@ -213,8 +265,13 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   k.max_grid = (unsigned)std::min<int64_t>((R + G - 1) / G, 0x7fffffff);
   k.grid[0] = k.max_grid;
   k.ptrs = rg.ptrs;
+  if (staged) {
+    k.wants_status = true;
+    k.smem_bytes = (unsigned)(G * nstg * stage_bytes);
+  }
   std::ostringstream d;
   d << "row kernel T=" << T << " G=" << G << " V=" << V << " NV=" << NV;
+  if (staged) d << ", " << nstg << "-row bulk-copy ring";
   k.desc = d.str();
   out->push_back(k);
 }

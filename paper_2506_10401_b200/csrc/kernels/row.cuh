@@ -83,6 +83,112 @@ __device__ __forceinline__ void hct_store_row(T* base, long long row, int hct_t,
   }
 }
 
+// ---- staged variant: full-width inputs are prefetched into a shared-memory ring by bulk
+// asynchronous copies (one per row and input, completion counted on an mbarrier), HCT_NSTG rows
+// ahead of the row being computed, so that loads stay in flight during the arithmetic and the
+// reductions of earlier rows.  The generator defines HCT_STAGED, HCT_NSTG, HCT_STAGE_BYTES
+// (bytes of all staged inputs of one row) and HCT_STATUS_SLOT.
+#ifdef HCT_STAGED
+__device__ __forceinline__ hct_u32 hct_smem_u32(const void* p) { return (hct_u32)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void hct_bulk_load(hct_u32 dst, const void* src, hct_u32 bytes, hct_u32 bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src), "r"(bytes),
+               "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ bool hct_row_mbar_try(hct_u32 bar, hct_u32 parity) {
+  hct_u32 ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: on expiry the status word is set and a CTA-wide flag makes later waits return at once.
+__device__ __forceinline__ void hct_row_mbar_wait(hct_u32 bar, hct_u32 parity, volatile int* failed, unsigned int* status) {
+  if (hct_row_mbar_try(bar, parity)) return;
+  for (unsigned it = 0; it < (1u << 24); ++it) {
+    if (hct_row_mbar_try(bar, parity)) return;
+    if (*failed) return;
+    if (it > 64) __nanosleep(20);
+  }
+  *failed = 1;
+  if (status) { atomicCAS(status, 0u, 1u); status[1] = 100u; }
+}
+// one thread's share of a staged row: the same vectors it would have loaded from global memory
+template <typename T>
+__device__ __forceinline__ void hct_read_staged(const unsigned char* slot, int hct_t, float* v);
+template <>
+__device__ __forceinline__ void hct_read_staged<float>(const unsigned char* slot, int hct_t, float* v) {
+#pragma unroll
+  for (int k = 0; k < HCT_NV; ++k) {
+    const int col = (k * HCT_T + hct_t) * HCT_V;
+    if (HCT_FULL_VECS || col < HCT_C) {
+      const float4 t = *(const float4*)(slot + (size_t)col * 4);
+      v[4 * k] = t.x; v[4 * k + 1] = t.y; v[4 * k + 2] = t.z; v[4 * k + 3] = t.w;
+    } else {
+      v[4 * k] = v[4 * k + 1] = v[4 * k + 2] = v[4 * k + 3] = 0.0f;
+    }
+  }
+}
+template <>
+__device__ __forceinline__ void hct_read_staged<hct_bf16_t>(const unsigned char* slot, int hct_t, float* v) {
+#pragma unroll
+  for (int k = 0; k < HCT_NV; ++k) {
+    const int col = (k * HCT_T + hct_t) * HCT_V;
+    if (HCT_FULL_VECS || col < HCT_C) {
+      const uint2 t = *(const uint2*)(slot + (size_t)col * 2);
+      v[4 * k] = __uint_as_float(t.x << 16); v[4 * k + 1] = __uint_as_float(t.x & 0xffff0000u);
+      v[4 * k + 2] = __uint_as_float(t.y << 16); v[4 * k + 3] = __uint_as_float(t.y & 0xffff0000u);
+    } else {
+      v[4 * k] = v[4 * k + 1] = v[4 * k + 2] = v[4 * k + 3] = 0.0f;
+    }
+  }
+}
+
+#define HCT_STAGED_KERNEL_BEGIN(name)                                                          \
+  extern "C" __global__ void __launch_bounds__(HCT_T * HCT_G) name(const HctParams hct_p) {    \
+    HCT_RED_DECL                                                                               \
+    extern __shared__ __align__(128) unsigned char hct_ring[];                                 \
+    __shared__ unsigned long long hct_full[HCT_G][HCT_NSTG];                                   \
+    __shared__ int hct_failed;                                                                 \
+    HctRowCtx hct_cx;                                                                          \
+    hct_cx.t = threadIdx.x % HCT_T;                                                            \
+    hct_cx.g = threadIdx.x / HCT_T;                                                            \
+    hct_cx.par = 0;                                                                            \
+    const int hct_t = hct_cx.t;                                                                \
+    unsigned int* hct_status = (unsigned int*)hct_p.ptr[HCT_STATUS_SLOT];                      \
+    unsigned char* hct_my_ring = hct_ring + (size_t)hct_cx.g * HCT_NSTG * HCT_STAGE_BYTES;      \
+    if (threadIdx.x == 0) hct_failed = 0;                                                      \
+    if (hct_t == 0) {                                                                          \
+      for (int s_ = 0; s_ < HCT_NSTG; ++s_) {                                                  \
+        hct_u32 b_ = hct_smem_u32(&hct_full[hct_cx.g][s_]);                                    \
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(b_) : "memory");           \
+      }                                                                                        \
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");                       \
+    }                                                                                          \
+    __syncthreads();
+
+// issue the copies of row `r_` (if it exists) into ring slot `s_`; called by thread 0 of the row group
+#define HCT_STAGED_ISSUE_BEGIN(r_, s_)                                                         \
+  if ((r_) < HCT_R) {                                                                          \
+    const long long hct_ir = (r_);                                                             \
+    const hct_u32 hct_ib = hct_smem_u32(&hct_full[hct_cx.g][(s_)]);                            \
+    const hct_u32 hct_id = hct_smem_u32(hct_my_ring + (size_t)(s_) * HCT_STAGE_BYTES);         \
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(hct_ib), "n"(HCT_STAGE_BYTES) : "memory");
+#define HCT_STAGED_ISSUE_ONE(ptr, off, bytes_per_row) \
+    hct_bulk_load(hct_id + (off), (const unsigned char*)(ptr) + hct_ir * (long long)(bytes_per_row), (bytes_per_row), hct_ib);
+#define HCT_STAGED_ISSUE_END }
+
+#if HCT_T > 32
+#define HCT_GROUP_SYNC asm volatile("bar.sync %0, %1;" ::"r"(hct_cx.g + 1), "n"(HCT_T) : "memory")
+#else
+#define HCT_GROUP_SYNC __syncwarp()
+#endif
+#endif  // HCT_STAGED
+
 #define HCT_ROW_KERNEL_BEGIN(name)                                                            \
   extern "C" __global__ void __launch_bounds__(HCT_T * HCT_G) name(const HctParams hct_p) {   \
     HCT_RED_DECL                                                                              \
