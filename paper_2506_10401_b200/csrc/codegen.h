@@ -43,8 +43,9 @@ struct KernelSpec {
 struct Tunables {
   int row_nv = 4;        // vectors per thread in row kernels
   int row_cta = 256;     // threads per CTA in row kernels
+  int row_cta_staged = 1024;       // threads per CTA of a staged row kernel (one CTA per SM)
   bool row_no_stage = false;       // load rows straight from global memory instead of through the shared-memory ring
-  int row_ring_bytes = 96 * 1024;  // shared memory one CTA of a row kernel may spend on its prefetch ring
+  int row_ring_bytes = 200 * 1024; // shared memory a staged row kernel may spend on resident row vectors plus its prefetch ring
   bool simt_only = false;  // keep contractions on the fp32 FMA kernels (for debugging tensor-core paths)
   static Tunables from_env();
 };

@@ -13,6 +13,7 @@ Tunables Tunables::from_env() {
   if (const char* s = std::getenv("HCT_ROW_NV")) t.row_nv = std::max(1, std::atoi(s));
   if (const char* s = std::getenv("HCT_ROW_CTA")) t.row_cta = std::max(32, std::atoi(s));
   if (const char* s = std::getenv("HCT_SIMT_ONLY")) t.simt_only = std::atoi(s) != 0;
+  if (const char* s = std::getenv("HCT_ROW_CTA_STAGED")) t.row_cta_staged = std::max(32, std::atoi(s));
   if (const char* s = std::getenv("HCT_ROW_NO_STAGE")) t.row_no_stage = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_RING_BYTES")) t.row_ring_bytes = std::max(1024, std::atoi(s));
   return t;
@@ -31,6 +32,13 @@ std::string float_lit(double v) {
 const char* ctype(DType d) { return d == BF16 ? "hct_bf16_t" : "float"; }
 
 namespace {
+
+inline bool HCT_T_GT32(int T) { return T > 32; }
+inline std::string strip_marker(std::string s) {
+  size_t m = s.find("@REFILL@");
+  if (m != std::string::npos) s.erase(m, 8);
+  return s;
+}  // rows that span several warps reduce through a barrier
 
 struct RowGen {
   const Graph& g;
@@ -102,19 +110,41 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
       stage_bytes += rb;
     }
   if (stage_bytes == 0) staged = false;
+  // A staged kernel runs one large CTA per SM: its row groups share the row-vector operands, which
+  // are copied to shared memory once (as fp32) instead of being re-read through L1 for every row.
   int nstg = 0;
+  int64_t rowvec_bytes = 0;
+  int n_rowvec = 0;
   if (staged) {
-    nstg = (int)std::min<int64_t>(8, tun.row_ring_bytes / (G * stage_bytes));
-    if (nstg < 2) staged = false;
+    for (auto& e : grp.ext)
+      if (e.bcast == Bcast::RowVec) {
+        rowvec_bytes += C * 4;
+        ++n_rowvec;
+      }
+    if (rowvec_bytes > 80 * 1024) {
+      rowvec_bytes = 0;  // too large to keep resident: read them through the cache instead
+      n_rowvec = 0;
+    }
+    int Gs = std::max(1, std::min<int>(tun.row_cta_staged / T, 15));
+    if ((int64_t)Gs > R) Gs = (int)std::max<int64_t>(1, R);
+    while ((Gs * T) % 32 != 0) ++Gs;
+    int64_t budget = (int64_t)tun.row_ring_bytes - rowvec_bytes;
+    while (Gs > 1 && budget / (Gs * stage_bytes) < 2) --Gs;
+    nstg = (int)std::min<int64_t>(8, budget / (Gs * stage_bytes));
+    if (nstg < 2 || (Gs * T) % 32 != 0)
+      staged = false;
+    else
+      G = Gs;
   }
+  const bool smem_rowvec = staged && n_rowvec > 0;
 
   RowGen rg{g, p, grp, gi, {}, {}};
   std::ostringstream& b = rg.body;
   std::string name = "hct_row_g" + std::to_string(gi);
 
   // ---- external operands
-  std::ostringstream pre, loads, issue, other_loads;
-  int64_t staged_off = 0;
+  std::ostringstream pre, loads, issue, fill;
+  int64_t staged_off = 0, rowvec_off = 0;
   for (size_t k = 0; k < grp.ext.size(); ++k) {
     const ExtOperand& e = grp.ext[k];
     int pi = rg.ptr_index(e.node, rg.ext_is_ws(e.node));
@@ -131,7 +161,15 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         }
         break;
       case Bcast::RowVec:
-        loads << "      float x" << k << "[HCT_E]; hct_load_row(q" << k << ", 0, hct_t, x" << k << ", true);\n";
+        if (smem_rowvec) {
+          fill << "    for (int i_ = threadIdx.x * 4; i_ < HCT_C; i_ += HCT_T * HCT_G * 4) {\n"
+               << "      float t_[4]; hct_vecio<4>::ld_keep(q" << k << " + i_, t_);\n"
+               << "      *(float4*)(hct_ring + " << rowvec_off << " + (size_t)i_ * 4) = make_float4(t_[0], t_[1], t_[2], t_[3]);\n    }\n";
+          loads << "      float x" << k << "[HCT_E]; hct_read_staged<float>(hct_ring + " << rowvec_off << ", hct_t, x" << k << ");\n";
+          rowvec_off += C * 4;
+        } else {
+          loads << "      float x" << k << "[HCT_E]; hct_load_row(q" << k << ", 0, hct_t, x" << k << ", true);\n";
+        }
         break;
       case Bcast::Scalar:
         pre << "    const float c" << k << " = hct_ld1(q" << k << ");\n";
@@ -152,9 +190,11 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   }
 
   // ---- nodes
+  bool refill_placed = false;
   for (int ni : grp.nodes) {
     const Node& nd = g.nodes[ni];
     std::string id = std::to_string(ni);
+    const bool reduces = nd.cls == OpClass::RowReduce || nd.cls == OpClass::RowSoftmax || nd.cls == OpClass::RowLayernorm;
     b << "      // " << nd.name << " = " << nd.op << "\n";
     if (nd.cls == OpClass::Unary || nd.cls == OpClass::Binary) {
       std::string call = "hct_" + nd.op + "(";
@@ -173,6 +213,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         << "      _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) if (HCT_HAS(e)) s" << id << " = "
         << (is_max ? "fmaxf(s" + id + ", " + a + ")" : "s" + id + " + " + a) << ";\n"
         << "      s" << id << " = " << (is_max ? "HCT_RMAX" : "HCT_RSUM") << "(s" << id << ");\n";
+      if (!refill_placed) { b << "@REFILL@"; refill_placed = true; }
       if (nd.op == "row_mean") b << "      s" << id << " = s" << id << " / (float)HCT_C;\n";
     } else if (nd.cls == OpClass::RowSoftmax) {
       std::string a = rg.ref(nd.args[0], true);
@@ -181,6 +222,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         << "        float m_ = -HCT_INF;\n"
         << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) if (HCT_HAS(e)) m_ = fmaxf(m_, " << a << ");\n"
         << "        m_ = HCT_RMAX(m_);\n"
+        << (refill_placed ? "" : "@REFILL@")
         << "        const float ml_ = -m_ * HCT_LOG2E;\n"
         << "        float d_ = 0.0f;\n"
         << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) { v" << id << "[e] = HCT_HAS(e) ? hct_exp2_fast(fmaf(" << a
@@ -197,6 +239,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         << "        float m_ = 0.0f;\n"
         << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) if (HCT_HAS(e)) m_ += " << a << ";\n"
         << "        m_ = HCT_RSUM(m_) / (float)HCT_C;\n"
+        << (refill_placed ? "" : "@REFILL@")
         << "        float q_ = 0.0f;\n"
         << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) { const float d_ = HCT_HAS(e) ? " << a
         << " - m_ : 0.0f; v" << id << "[e] = d_; q_ = fmaf(d_, d_, q_); }\n"
@@ -208,6 +251,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
     } else {
       throw Error(HCT_ERR_UNSUPPORTED, "operator " + nd.op + " cannot be part of a row kernel");
     }
+    if (reduces) refill_placed = true;
   }
 
   // ---- stores
@@ -227,16 +271,16 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   src << "#define HCT_T " << T << "\n#define HCT_G " << G << "\n#define HCT_V " << V << "\n#define HCT_NV " << NV << "\n"
       << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "\n#define HCT_NPTR " << std::max<size_t>(1, nptr) << "\n";
   if (staged)
-    src << "#define HCT_STAGED 1\n#define HCT_NSTG " << nstg << "\n#define HCT_STAGE_BYTES " << stage_bytes << "\n#define HCT_STATUS_SLOT "
+    src << "#define HCT_MINB 1\n#define HCT_RING_OFF " << rowvec_bytes << "\n#define HCT_STAGED 1\n#define HCT_NSTG " << nstg << "\n#define HCT_STAGE_BYTES " << stage_bytes << "\n#define HCT_STATUS_SLOT "
         << rg.ptrs.size() << "\n";
   src << skeleton_source("common") << "\n" << skeleton_source("row") << "\n";
   if (!staged) {
     src << "HCT_ROW_KERNEL_BEGIN(" << name << ")\n"
         << pre.str() << "  HCT_ROW_LOOP_BEGIN\n"
-        << loads.str() << b.str() << stores.str() << "  HCT_ROW_LOOP_END\nHCT_ROW_KERNEL_END\n";
+        << loads.str() << strip_marker(b.str()) << stores.str() << "  HCT_ROW_LOOP_END\nHCT_ROW_KERNEL_END\n";
   } else {
     src << "HCT_STAGED_KERNEL_BEGIN(" << name << ")\n"
-        << pre.str()
+        << pre.str() << fill.str() << (smem_rowvec ? "    __syncthreads();\n" : "")
         << "    const long long hct_stride = (long long)gridDim.x * HCT_G;\n"
         << "    if (hct_t == 0) {\n"
         << "      for (int s_ = 0; s_ < HCT_NSTG; ++s_) {\n"
@@ -248,12 +292,20 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         << "      const int hct_s = hct_it % HCT_NSTG;\n"
         << "      hct_row_mbar_wait(hct_smem_u32(&hct_full[hct_cx.g][hct_s]), (hct_u32)((hct_it / HCT_NSTG) & 1), &hct_failed, hct_status);\n"
         << "      const unsigned char* hct_slot = hct_my_ring + (size_t)hct_s * HCT_STAGE_BYTES;\n"
-        << loads.str()
-        << "      HCT_GROUP_SYNC;  // every thread of the row has taken its share: the slot may be refilled\n"
-        << "      if (hct_t == 0) {\n"
-        << "        HCT_STAGED_ISSUE_BEGIN(hct_row + HCT_NSTG * hct_stride, hct_s)\n"
-        << issue.str() << "        HCT_STAGED_ISSUE_END\n      }\n"
-        << b.str() << stores.str() << "    }\n    ++hct_it;\n"
+        << loads.str();
+    // The slot may be refilled once every thread of the row has taken its share, i.e. after any
+    // barrier of the row group: the first reduction's barrier if the chain has one, else one of its own.
+    std::string refill = "      if (hct_t == 0) {\n        HCT_STAGED_ISSUE_BEGIN(hct_row + HCT_NSTG * hct_stride, hct_s)\n" + issue.str() +
+                         "        HCT_STAGED_ISSUE_END\n      }\n";
+    std::string body = b.str();
+    size_t mark = body.find("@REFILL@");
+    if (mark != std::string::npos && HCT_T_GT32(T))
+      body.replace(mark, 8, refill);
+    else {
+      if (mark != std::string::npos) body.erase(mark, 8);
+      src << "      HCT_GROUP_SYNC;\n" << refill;
+    }
+    src << body << stores.str() << "    }\n    ++hct_it;\n"
         << "  HCT_ROW_LOOP_END\nHCT_ROW_KERNEL_END\n";
   }
 
@@ -267,7 +319,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   k.ptrs = rg.ptrs;
   if (staged) {
     k.wants_status = true;
-    k.smem_bytes = (unsigned)(G * nstg * stage_bytes);
+    k.smem_bytes = (unsigned)(rowvec_bytes + G * nstg * stage_bytes);
   }
   std::ostringstream d;
   d << "row kernel T=" << T << " G=" << G << " V=" << V << " NV=" << NV;

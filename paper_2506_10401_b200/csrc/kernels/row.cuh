@@ -39,13 +39,18 @@ __device__ __forceinline__ float hct_row_reduce(float v, HctRowCtx& cx, float (*
     v = IS_MAX ? fmaxf(v, u) : v + u;
   }
 #if HCT_T > 32
+  // one partial per warp goes through shared memory; every warp then folds the HCT_T/32 partials
+  // with a second, shorter butterfly, so all threads end with the same value
   float* slot = red[cx.g][cx.par];
   cx.par ^= 1u;
   if ((cx.t & 31) == 0) slot[cx.t >> 5] = v;
   asm volatile("bar.sync %0, %1;" ::"r"(cx.g + 1), "n"(HCT_T) : "memory");
-  v = slot[0];
+  v = slot[cx.t & (HCT_T / 32 - 1)];
 #pragma unroll
-  for (int w = 1; w < HCT_T / 32; ++w) v = IS_MAX ? fmaxf(v, slot[w]) : v + slot[w];
+  for (int o = HCT_T / 64; o > 0; o >>= 1) {
+    float u = __shfl_xor_sync(0xffffffffu, v, o);
+    v = IS_MAX ? fmaxf(v, u) : v + u;
+  }
 #endif
   return v;
 }
@@ -87,7 +92,8 @@ __device__ __forceinline__ void hct_store_row(T* base, long long row, int hct_t,
 // asynchronous copies (one per row and input, completion counted on an mbarrier), HCT_NSTG rows
 // ahead of the row being computed, so that loads stay in flight during the arithmetic and the
 // reductions of earlier rows.  The generator defines HCT_STAGED, HCT_NSTG, HCT_STAGE_BYTES
-// (bytes of all staged inputs of one row) and HCT_STATUS_SLOT.
+// (bytes of all staged inputs of one row), HCT_RING_OFF (bytes of resident row vectors placed
+// before the ring) and HCT_STATUS_SLOT.
 #ifdef HCT_STAGED
 __device__ __forceinline__ hct_u32 hct_smem_u32(const void* p) { return (hct_u32)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void hct_bulk_load(hct_u32 dst, const void* src, hct_u32 bytes, hct_u32 bar) {
@@ -149,7 +155,7 @@ __device__ __forceinline__ void hct_read_staged<hct_bf16_t>(const unsigned char*
 }
 
 #define HCT_STAGED_KERNEL_BEGIN(name)                                                          \
-  extern "C" __global__ void __launch_bounds__(HCT_T * HCT_G) name(const HctParams hct_p) {    \
+  extern "C" __global__ void __launch_bounds__(HCT_T * HCT_G, HCT_MINB) name(const HctParams hct_p) {    \
     HCT_RED_DECL                                                                               \
     extern __shared__ __align__(128) unsigned char hct_ring[];                                 \
     __shared__ unsigned long long hct_full[HCT_G][HCT_NSTG];                                   \
@@ -160,7 +166,7 @@ __device__ __forceinline__ void hct_read_staged<hct_bf16_t>(const unsigned char*
     hct_cx.par = 0;                                                                            \
     const int hct_t = hct_cx.t;                                                                \
     unsigned int* hct_status = (unsigned int*)hct_p.ptr[HCT_STATUS_SLOT];                      \
-    unsigned char* hct_my_ring = hct_ring + (size_t)hct_cx.g * HCT_NSTG * HCT_STAGE_BYTES;      \
+    unsigned char* hct_my_ring = hct_ring + HCT_RING_OFF + (size_t)hct_cx.g * HCT_NSTG * HCT_STAGE_BYTES;      \
     if (threadIdx.x == 0) hct_failed = 0;                                                      \
     if (hct_t == 0) {                                                                          \
       for (int s_ = 0; s_ < HCT_NSTG; ++s_) {                                                  \
