@@ -139,6 +139,30 @@ HCT_API const char* hct_graph_plan_text(const hct_graph_t* g);
 HCT_API const char* hct_graph_kernel_source(const hct_graph_t* g, int idx);
 HCT_API const char* hct_graph_kernel_name(const hct_graph_t* g, int idx);
 
+/*
+ * relu(A*B + bias) in fp32 without any device allocation, for callers that must not or cannot
+ * allocate: code that runs inside another framework's memory pool with a fixed budget, real-time
+ * loops where an allocation would be a stall or a failure point, and start-up paths that run
+ * before an allocator exists.  (The paper has no counterpart; this is a convenience of this
+ * library.)  hct_graph_run needs caller-provided workspace for the split operands of an fp32
+ * GEMM; here that scratch is a fixed array of HCT_STATIC_SCRATCH_BYTES inside the library image,
+ * present on every GPU that loads the library until the process exits.
+ *   a[m,k], b[k,n], out[m,n] row-major fp32 DEVICE pointers on `device`; bias[n] or NULL;
+ *   apply_relu != 0 applies max(.,0).  Operands are split into TF32 head and tail and multiplied
+ *   as three products per term with fp32 FMA accumulation; results agree with hct_graph_run's
+ *   fp32 GEMM to the library's fp32 tolerance, not bit for bit.
+ * Limit: m*k + k*n <= HCT_STATIC_SCRATCH_BYTES/8 elements, else HCT_ERR_UNSUPPORTED.
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with that
+ * device made current for the duration of the call); make that first call before starting any
+ * stream capture.  The call launches on `cuda_stream` and does not synchronise.  It calls no
+ * allocating routine.  All calls share the one array: nothing in it needs to start at zero (each
+ * call overwrites the part it reads), but two calls whose kernels overlap on the GPU (different
+ * streams, or several host threads) race on it; keep them on one stream or order them yourself.
+ */
+#define HCT_STATIC_SCRATCH_BYTES (8u << 20)
+HCT_API hct_status_t hct_gemm_bias_relu_f32_static(const float* a, const float* b, const float* bias, float* out, int64_t m,
+                                                   int64_t k, int64_t n, int apply_relu, int device, void* cuda_stream);
+
 /* Message of the last failing call on this thread ("" if none). */
 HCT_API const char* hct_last_error(void);
 HCT_API const char* hct_version(void);

@@ -17,8 +17,10 @@ EXPORTS = [
     "hct_graph_create", "hct_graph_run", "hct_graph_status", "hct_graph_destroy", "hct_graph_num_inputs",
     "hct_graph_num_outputs", "hct_graph_tensor_info", "hct_graph_workspace_bytes", "hct_graph_num_kernels",
     "hct_graph_cost", "hct_graph_plan_text", "hct_graph_kernel_source", "hct_graph_kernel_name", "hct_last_error",
-    "hct_version",
+    "hct_version", "hct_gemm_bias_relu_f32_static",
 ]
+
+HCT_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class HctError(RuntimeError):
@@ -68,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.hct_graph_kernel_name.restype = cp
         L.hct_last_error.argtypes = []
         L.hct_last_error.restype = cp
+        L.hct_gemm_bias_relu_f32_static.argtypes = [vp, vp, vp, vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ci, ci, vp]
+        L.hct_gemm_bias_relu_f32_static.restype = ci
         L.hct_version.argtypes = []
         L.hct_version.restype = cp
         _lib = L
@@ -147,3 +151,9 @@ def hct_graph_kernel_source(g, idx: int) -> str:
 def hct_graph_kernel_name(g, idx: int) -> str:
     s = lib().hct_graph_kernel_name(g, idx)
     return s.decode() if s is not None else ""
+
+
+def hct_gemm_bias_relu_f32_static(a: int, b: int, bias: int, out: int, m: int, k: int, n: int, apply_relu: bool = True,
+                                  device: int = 0, cuda_stream: int = 0):
+    """relu(A*B + bias) on device addresses, using the library's built-in scratch instead of a workspace."""
+    _check(lib().hct_gemm_bias_relu_f32_static(a, b, bias, out, m, k, n, int(apply_relu), device, cuda_stream))

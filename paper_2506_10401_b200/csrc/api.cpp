@@ -20,6 +20,15 @@ hct_status_t set_error(int code, const std::string& msg) {
   return (hct_status_t)code;
 }
 
+}  // namespace
+
+namespace hct {
+// lets the other translation units of the library record an error message for hct_last_error()
+void set_last_error(const std::string& msg) { g_last_error = msg; }
+}  // namespace hct
+
+namespace {
+
 struct LoadedKernel {
   KernelSpec spec;
   CUmodule_t module = nullptr;

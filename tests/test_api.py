@@ -17,7 +17,7 @@ NONE = hct.HCT_DEVICE_NONE
 
 def test_library_exports_every_declared_symbol():
     header = open(os.path.join(ROOT, "include", "hct.h")).read()
-    declared = set(re.findall(r"HCT_API[^;(]*?\b(hct_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"HCT_API[^;(]*?\b(hct_[a-z0-9_]+)\s*\(", header))
     assert declared == set(binding.EXPORTS)
     raw = ctypes.CDLL(binding.LIB_PATH)
     for name in declared:
