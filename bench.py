@@ -89,6 +89,22 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity when not distributed)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def whole_job_value(bound, bytes_per_rank, flops_per_rank, world, slowest_seconds_per_step):
+    """Replicas: every rank processes the same units; the job's rate is all units over the slowest rank's time."""
+    return metric_of(bound, bytes_per_rank * world, flops_per_rank * world, slowest_seconds_per_step)
+
+
 def metric_of(bound, bytes_, flops, seconds):
     if bound == "hbm":
         return bytes_ / seconds / 1e9, "GB/s"
@@ -193,16 +209,80 @@ def run_gpu(name, steps, warmup, rank, world, device):
     barrier()
     e2e_s = a.elapsed_time(b) * 1e-3 / e2e_steps
 
-    if world > 1:
-        t = torch.tensor([dev_s, e2e_s], device=f"cuda:{device}", dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        dev_s, e2e_s = float(t[0]), float(t[1])
-    value, unit = metric_of(info["bound"], bytes_ * world, flops * world, dev_s / steps)
-    e2e_v, _ = metric_of(info["bound"], bytes_ * world, flops * world, e2e_s)
+    dev_s, e2e_s = max_over_ranks([dev_s, e2e_s], f"cuda:{device}")
+    value, unit = whole_job_value(info["bound"], bytes_, flops, world, dev_s / steps)
+    e2e_v, _ = whole_job_value(info["bound"], bytes_, flops, world, e2e_s)
     kern_s = float(np.mean(per_step))
     return dict(value=value, unit=unit, ms_per_step=dev_s / steps * 1e3, bytes=bytes_, flops=flops, kernel_s=kern_s,
                 kernels=g.num_kernels, clocks=clocks.summary(), e2e=dict(value=e2e_v, unit=unit, h2d_bytes_per_step=h2d,
                                                                          d2h_bytes_per_step=d2h), plan=g.plan)
+
+
+def run_sweep(steps, warmup, device, out_path=None):
+    """The 200 random operator DAGs: per-graph time against its own roofline, and class aggregates.
+
+    Inputs are drawn on the device from the same laws (normal / uniform with the recipe's mean and
+    spread, seeded per graph) because host-side generation of ~10^10 elements would dominate the run;
+    parity on these graphs is covered by the tests with the counter-based host generator."""
+    import torch
+    import paper_2506_10401_b200 as hct
+    from workloads import sweep
+    pk = peaks()
+    dev = f"cuda:{device}"
+    flush = torch.empty(192 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(device)
+    records = []
+    launches = 0
+    for e in sweep.entries():
+        spec, laws, meta = sweep.get(e["seed"])
+        g = hct.FusedGraph(spec, device)
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(1000 + e["seed"])
+        ins = []
+        for name, dtype, shape in configs.parse_inputs(spec):
+            law = laws[name]
+            if law["kind"] == "normal":
+                t = torch.randn(shape, device=dev, generator=gen) * law.get("std", 1.0) + law.get("mean", 0.0)
+            else:
+                t = torch.rand(shape, device=dev, generator=gen) * (law["hi"] - law["lo"]) + law["lo"]
+            ins.append(t.to(torch.bfloat16) if dtype == "bf16" else t)
+        outs = g.alloc_outputs()
+        for _ in range(max(1, warmup)):
+            g.run(ins, outs, stream)
+        torch.cuda.synchronize(device)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in ev:
+            flush.zero_()
+            a.record(stream)
+            g.run(ins, outs, stream)
+            b.record(stream)
+        torch.cuda.synchronize(device)
+        g.status()
+        sec = float(np.median([a.elapsed_time(b) for a, b in ev])) * 1e-3
+        bytes_, flops = g.cost()
+        t_mem = bytes_ / (pk["hbm"] * 1e9)
+        t_mma = flops / (pk["tensor"] / 6.0 * 1e12)  # fp32 GEMM = three TF32 products at half the bf16 rate
+        cls = "gemm" if t_mma > t_mem else "memory"
+        records.append(dict(seed=e["seed"], cls=cls, us=sec * 1e6, bytes=bytes_, flops=flops, kernels=g.num_kernels,
+                            frac=max(t_mem, t_mma) / sec))
+        launches += g.num_kernels * (steps + max(1, warmup))
+        g.close()
+        del ins, outs
+    if out_path:
+        with open(out_path, "w") as f:
+            for r in records:
+                f.write(json.dumps(r) + "\n")
+    mem = [r for r in records if r["cls"] == "memory"]
+    mma = [r for r in records if r["cls"] == "gemm"]
+    geo = lambda rs: float(np.exp(np.mean(np.log([r["frac"] for r in rs])))) if rs else None
+    agg = dict(graphs=len(records), memory_graphs=len(mem), gemm_graphs=len(mma),
+               memory_GBps=sum(r["bytes"] for r in mem) / sum(r["us"] for r in mem) / 1e3 if mem else None,
+               gemm_TFLOPps_fp32=sum(r["flops"] for r in mma) / sum(r["us"] for r in mma) / 1e6 if mma else None,
+               memory_frac_geomean=geo(mem), gemm_frac_geomean=geo(mma),
+               memory_share_ge_0p7=float(np.mean([r["frac"] >= 0.7 for r in mem])) if mem else None,
+               gemm_share_ge_0p6=float(np.mean([r["frac"] >= 0.6 for r in mma])) if mma else None,
+               total_ms=sum(r["us"] for r in records) / 1e3)
+    return agg, launches
 
 
 def main():
@@ -211,7 +291,8 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="hct", choices=["hct", "reference"])
-    ap.add_argument("--workload", default=HEADLINE, choices=list(WORKLOADS))
+    ap.add_argument("--workload", default=HEADLINE, choices=list(WORKLOADS) + ["c5_sweep"])
+    ap.add_argument("--out", default=None, help="c5_sweep: write one JSON record per graph to this file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -224,6 +305,8 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return
+        if name == "c5_sweep":
+            name = HEADLINE
         r = oracle_arm(name, max(1, min(args.steps, 5)), min(args.warmup, 1))
         line = dict(impl="reference", metric=metric, value=r["value"], unit=r["unit"], n_gpus=args.gpus, steps=args.steps,
                     warmup=args.warmup, ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
@@ -236,6 +319,21 @@ def main():
     import torch
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the fused chains have no CPU execution path")
+    if name == "c5_sweep":
+        if world > 1:
+            raise SystemExit("the sweep runs on one GPU")
+        with ClockSampler(local) as clocks:
+            agg, launches = run_sweep(max(3, min(args.steps, 10)), args.warmup, local, args.out)
+        pk = peaks()
+        print(json.dumps(dict(metric=metric, value=agg["memory_GBps"], unit="GB/s", n_gpus=1, steps=args.steps, warmup=args.warmup,
+                              ms_per_step=agg["total_ms"], higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
+                              data="synthetic", config={"workload": "c5_sweep: 200 random operator DAGs, seeds 0..199",
+                                                        "l2": "flushed between runs", "value_is": "aggregate over memory-bound graphs"},
+                              clocks=clocks.summary(), gpu_launches=launches, sweep=agg,
+                              roofline=dict(bound="hbm", achieved=agg["memory_GBps"], peak=pk["hbm"], unit="GB/s",
+                                            frac=agg["memory_GBps"] / pk["hbm"], traffic=None, peak_source=pk["source"]),
+                              e2e=None, cpu_baseline=None)))
+        return
     if world > 1:
         torch.cuda.set_device(local)
         torch.distributed.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
