@@ -299,7 +299,7 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     name = args.workload
-    info = WORKLOADS[name]
+    info = WORKLOADS.get(name)
     metric = "fused-chain throughput: GB/s (memory-bound) / TFLOP/s (GEMM,conv) and % of B200 roofline"
 
     if args.impl == "reference":
