@@ -68,12 +68,15 @@ struct EpiGen {
 
   // Run epilogue for the tensor-core GEMM: one thread owns 32 consecutive columns of one row.
   // `ncols` of them exist; vector access is legal when N is a multiple of the vector length.
-  std::string run_fn(int64_t N) {
+  // `N` is the distance between consecutive rows; every run starts at a multiple of `vec_unit`
+  // elements plus a multiple of 32; `rowidx` is the index expression of per-row operands.
+  std::string run_fn(int64_t N, int64_t vec_unit = -1, const std::string& rowidx = "row") {
+    if (vec_unit < 0) vec_unit = N;
     std::ostringstream f;
     f << "__device__ __forceinline__ void hct_epilogue_run(const HctParams& hct_p, float (&acc)[32], long long row, int col0, int ncols) {\n";
     int anchor = grp.nodes[0];
     std::ostringstream loads;
-    auto vec_ok = [&](DType d) { return N % (d == BF16 ? 8 : 4) == 0 ? "true" : "false"; };
+    auto vec_ok = [&](DType d) { return (N % (d == BF16 ? 8 : 4) == 0 && vec_unit % (d == BF16 ? 8 : 4) == 0) ? "true" : "false"; };
     auto ref = [&](const Operand& a) -> std::string {
       if (a.is_literal()) return float_lit(a.literal);
       if (p.group_of[a.node] == gi) return a.node == anchor ? "acc[j]" : "e" + std::to_string(a.node);
@@ -97,7 +100,7 @@ struct EpiGen {
                 << ");\n";
           break;
         case Bcast::Scalar: loads << "  const float c" << k << " = hct_ld1(" << ptr << ");\n"; break;
-        case Bcast::RowIdx: loads << "  const float c" << k << " = hct_ld1(" << ptr << " + row);\n"; break;
+        case Bcast::RowIdx: loads << "  const float c" << k << " = hct_ld1(" << ptr << " + " << rowidx << ");\n"; break;
       }
     }
     f << loads.str();
@@ -320,7 +323,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     bool in_bf16 = a.cls == OpClass::Input && b.cls == OpClass::Input && a.dtype == BF16 && b.dtype == BF16;
     int64_t NB = xs[0], C = xs[1], H = xs[2], W = xs[3], KO = ws[0], FR = ws[2], FS = ws[3];
     int64_t HO = anchor.shape[2], WO = anchor.shape[3];
-    if (in_bf16 && anchor.stride == 1 && C % 8 == 0 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
+    if (in_bf16 && anchor.stride == 1 && C % 8 == 0 && WO <= 256 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
       auto align256 = [](int64_t v) { return (v + 255) / 256 * 256; };
       const int64_t x_bytes = align256(NB * C * H * W * 2), w_bytes = align256(KO * C * FR * FS * 2);
       *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(x_bytes + w_bytes));
@@ -350,46 +353,47 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         k.desc = "conv layout pre-pass: NCHW->NHWC activations, KCRS->RSKC weights";
         out->push_back(k);
       }
-      int TW = (int)std::min<int64_t>(WO, 128);
-      int TH = (int)std::max<int64_t>(1, std::min<int64_t>(128 / TW, HO));
-      int BN = KO > 64 ? 128 : KO > 32 ? 64 : 32;
-      int stages = BN == 128 ? 6 : 8;
-      std::string epi = eg.conv_fn(KO, HO, WO);
+      int TH = (int)std::max<int64_t>(1, std::min<int64_t>(256 / WO, HO));
+      int stages = 4;
+      std::string epi = eg.run_fn(HO * WO, WO, "(row % " + std::to_string(KO) + "LL)");
       KernelSpec k;
       k.name = "hct_conv_tc_bf16_g" + std::to_string(gi);
       std::ostringstream src;
       src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_H " << H << "\n#define HCT_W " << W
           << "\n#define HCT_KO " << KO << "\n#define HCT_FR " << FR << "\n#define HCT_FS " << FS << "\n#define HCT_PAD " << anchor.pad
-          << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TW " << TW << "\n#define HCT_TH " << TH
-          << "\n#define HCT_BN " << BN << "\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
+          << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TH " << TH << "\n#define HCT_TH2 1\n#define HCT_SPLIT "
+          << TH << "\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
           << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
-      src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[2]; void* ptr["
+      src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[3]; void* ptr["
           << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source("conv_tc");
       k.source = src.str();
       k.ptrs = eg.ptrs;
       k.wants_status = true;
-      TmaDesc tx, tw;
-      tx.buf = scratch(0);
-      tx.elem_bytes = 2;
-      tx.rank = 4;
-      tx.dims[0] = (uint64_t)C; tx.dims[1] = (uint64_t)W; tx.dims[2] = (uint64_t)H; tx.dims[3] = (uint64_t)NB;
-      tx.strides[1] = (uint64_t)C * 2; tx.strides[2] = (uint64_t)W * C * 2; tx.strides[3] = (uint64_t)H * W * C * 2;
-      tx.box[0] = 64; tx.box[1] = (uint32_t)TW; tx.box[2] = (uint32_t)TH; tx.box[3] = 1;
+      TmaDesc tw;
       tw.buf = scratch(x_bytes);
       tw.elem_bytes = 2;
       tw.rank = 2;
       tw.dims[0] = (uint64_t)C; tw.dims[1] = (uint64_t)(FR * FS * KO);
       tw.strides[1] = (uint64_t)C * 2;
-      tw.box[0] = 64; tw.box[1] = (uint32_t)BN;
-      k.tmaps = {tx, tw};
-      int64_t tiles = NB * ((HO + TH - 1) / TH) * ((WO + TW - 1) / TW) * ((KO + BN - 1) / BN);
+      tw.box[0] = 64; tw.box[1] = 128;
+      TmaDesc tx;
+      tx.buf = scratch(0);
+      tx.elem_bytes = 2;
+      tx.rank = 4;
+      tx.dims[0] = (uint64_t)C; tx.dims[1] = (uint64_t)W; tx.dims[2] = (uint64_t)H; tx.dims[3] = (uint64_t)NB;
+      tx.strides[1] = (uint64_t)C * 2; tx.strides[2] = (uint64_t)W * C * 2; tx.strides[3] = (uint64_t)H * W * C * 2;
+      tx.box[0] = 64; tx.box[1] = (uint32_t)WO; tx.box[2] = (uint32_t)TH; tx.box[3] = 1;
+      TmaDesc tx2 = tx;
+      tx2.box[2] = 1;
+      k.tmaps = {tw, tx, tx2};
+      int64_t tiles = NB * ((HO + TH - 1) / TH) * ((KO + 127) / 128);
       k.block[0] = 192;
-      k.smem_bytes = (unsigned)(stages * (128 * 128 + BN * 128) + 1024);
+      k.smem_bytes = (unsigned)(stages * (128 * 128 + 32768) + 1024);
       k.persistent = true;
       k.max_grid = (unsigned)std::min<int64_t>(tiles, 0x7fffffff);
       k.grid[0] = k.max_grid;
       std::ostringstream d;
-      d << "conv2d tcgen05 bf16 implicit GEMM, tile " << TH << "x" << TW << " pixels x " << BN << " channels, " << stages << " stages";
+      d << "conv2d tcgen05 bf16 implicit GEMM, tile 128 channels x " << TH << " rows of " << WO << " pixels, " << stages << " stages";
       k.desc = d.str();
       out->push_back(k);
       return;

@@ -1,35 +1,49 @@
 // Persistent tensor-core conv2d (stride 1, zero padding) as an implicit GEMM with fused epilogue.
 //
-// GEMM view: rows = output pixels of one image, columns = output channels, contraction over
-// (filter tap, input channel).  A tile of HCT_TH output rows x HCT_TW output columns (at most 128
-// pixels) is one accumulator of 128 x HCT_BN in tensor memory.  For every filter tap (r,s) and
-// block of 64 input channels the producer warp loads, with one 4-D TMA box from the NHWC copy of
-// the input, the pixels shifted by the tap (coordinates outside the image read zeros, which is
-// the padding) and the tap's [HCT_BN x 64] weight slice; the MMA warp multiplies them into the
-// accumulator; four epilogue warps apply the generated epilogue and write NCHW.
+// GEMM view: rows (M = 128) = output channels, columns (N <= 256) = the pixels of HCT_TH full output
+// rows of one image, contraction over (filter tap, input channel).  For every tap (r,s) and block
+// of 64 input channels the producer warp loads the tap's [128 x 64] weight slice (A operand) and,
+// with one 4-D TMA box from the NHWC copy of the input, the pixels shifted by the tap (B operand;
+// coordinates outside the image read zeros, which is the padding; the channel coordinate is the
+// innermost one and a multiple of 64, so every copy starts 16-byte aligned).  The MMA warp
+// accumulates into one of two tensor-memory accumulators; four epilogue warps (one output channel
+// per thread, 32 consecutive pixels per step, contiguous in NCHW) apply the generated epilogue.
+//
+// Work is split into tiles of HCT_TH output rows; when the last round over the SMs would be
+// nearly empty, its tiles are cut into HCT_TH2-row pieces so that all SMs finish together.
 //
 // Defined by the generator: HCT_NB_IMG, HCT_C, HCT_H, HCT_W, HCT_KO, HCT_FR, HCT_FS, HCT_PAD, HCT_HO, HCT_WO,
-// HCT_TW, HCT_TH, HCT_BN, HCT_STAGES, HCT_STATUS_SLOT, HCT_KERNEL_NAME, HctParams, hct_epilogue_conv().
+// HCT_TH, HCT_TH2, HCT_SPLIT (pieces per cut tile, HCT_TH2 * HCT_SPLIT >= HCT_TH), HCT_STAGES,
+// HCT_STATUS_SLOT, HCT_KERNEL_NAME, HctParams, hct_epilogue_run().
 #define HCT_BM 128
-#define HCT_A_BYTES (HCT_BM * 128)
-#define HCT_A_BOX_BYTES (HCT_TW * HCT_TH * 128)
-#define HCT_B_BYTES (HCT_BN * 128)
+#define HCT_A_BYTES (HCT_BM * 128)                       // weights: 128 channels x 64 inputs, bf16
+#define HCT_B_BYTES 32768                                // pixels: up to 256 x 64 inputs
 #define HCT_STAGE_BYTES (HCT_A_BYTES + HCT_B_BYTES)
 #define HCT_CB ((HCT_C + 63) / 64)
 #define HCT_KB (HCT_FR * HCT_FS * HCT_CB)
 #define HCT_HT ((HCT_HO + HCT_TH - 1) / HCT_TH)
-#define HCT_WT ((HCT_WO + HCT_TW - 1) / HCT_TW)
-#define HCT_NBK ((HCT_KO + HCT_BN - 1) / HCT_BN)
-#define HCT_TILES ((long long)HCT_NB_IMG * HCT_HT * HCT_WT * HCT_NBK)
-#define HCT_TMEM_COLS (2 * HCT_BN < 32 ? 32 : 2 * HCT_BN)
+#define HCT_MBK ((HCT_KO + HCT_BM - 1) / HCT_BM)
+#define HCT_FULL_TILES ((long long)HCT_NB_IMG * HCT_HT * HCT_MBK)
 
-struct HctConvTile { int n, h0, w0, nbk; };
-__device__ __forceinline__ HctConvTile hct_conv_tile(long long t) {
+struct HctConvTile { int n, h0, th, mbk; bool cut; };
+
+// Tile t of the schedule.  Tiles below `t1` are whole; the rest are pieces of the remaining whole tiles.
+__device__ __forceinline__ HctConvTile hct_conv_tile(long long t, long long t1) {
   HctConvTile r;
-  r.nbk = (int)(t % HCT_NBK); t /= HCT_NBK;
-  r.w0 = (int)(t % HCT_WT) * HCT_TW; t /= HCT_WT;
-  r.h0 = (int)(t % HCT_HT) * HCT_TH; t /= HCT_HT;
-  r.n = (int)t;
+  long long whole = t;
+  int sub = 0;
+  r.cut = t >= t1;
+  if (r.cut) {
+    whole = t1 + (t - t1) / HCT_SPLIT;
+    sub = (int)((t - t1) % HCT_SPLIT);
+  }
+  r.mbk = (int)(whole % HCT_MBK); whole /= HCT_MBK;
+  r.h0 = (int)(whole % HCT_HT) * HCT_TH + sub * HCT_TH2;
+  r.n = (int)(whole / HCT_HT);
+  int th = r.cut ? HCT_TH2 : HCT_TH;
+  if (r.cut && sub * HCT_TH2 + th > HCT_TH) th = HCT_TH - sub * HCT_TH2;
+  if (r.h0 + th > HCT_HO) th = HCT_HO - r.h0;
+  r.th = th > 0 ? th : 0;   // 0: nothing to do (identically for every warp role)
   return r;
 }
 
@@ -44,6 +58,16 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
   const hct_u32 full0 = hct_smem_addr(&bars[0]), empty0 = hct_smem_addr(&bars[HCT_STAGES]);
   const hct_u32 tfull0 = hct_smem_addr(&bars[2 * HCT_STAGES]), tempty0 = hct_smem_addr(&bars[2 * HCT_STAGES + 2]);
 
+  // schedule: whole tiles for as many full rounds over the grid as there are, the rest cut in pieces
+  long long t1 = HCT_FULL_TILES, n_tiles = HCT_FULL_TILES;
+  {
+    const long long rest = HCT_FULL_TILES % gridDim.x;
+    if (HCT_SPLIT > 1 && rest > 0 && rest * HCT_SPLIT <= (long long)gridDim.x) {
+      t1 = HCT_FULL_TILES - rest;
+      n_tiles = t1 + rest * HCT_SPLIT;
+    }
+  }
+
   if (threadIdx.x == 0) {
     failed = 0;
     for (int s = 0; s < HCT_STAGES; ++s) {
@@ -57,8 +81,9 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     hct_prefetch_tmap(&hct_p.tmap[0]);
     hct_prefetch_tmap(&hct_p.tmap[1]);
+    hct_prefetch_tmap(&hct_p.tmap[2]);
   }
-  if (warp == 1) hct_tmem_alloc(hct_smem_addr(&tmem_holder), HCT_TMEM_COLS);
+  if (warp == 1) hct_tmem_alloc(hct_smem_addr(&tmem_holder), 512);
   hct_tc_fence_before();
   __syncthreads();
   hct_tc_fence_after();
@@ -68,33 +93,38 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
     if (lane == 0) {
       int stage = 0;
       hct_u32 phase = 0;
-      for (long long tile = blockIdx.x; tile < HCT_TILES; tile += gridDim.x) {
-        const HctConvTile t = hct_conv_tile(tile);
+      for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const HctConvTile t = hct_conv_tile(tile, t1);
+        if (t.th == 0) continue;
+        // whole tiles use the HCT_TH-row box, pieces the HCT_TH2-row box
+        const HctTensorMap* xmap = t.cut ? &hct_p.tmap[2] : &hct_p.tmap[1];
+        const hct_u32 bytes = HCT_A_BYTES + (hct_u32)(t.cut ? HCT_TH2 : HCT_TH) * HCT_WO * 128u;
         for (int kb = 0; kb < HCT_KB; ++kb) {
           const int tap = kb / HCT_CB, cb = kb % HCT_CB;
           const int r = tap / HCT_FS, s = tap % HCT_FS;
           hct_mbar_wait(empty0 + 8 * stage, phase ^ 1u, &failed, status, 1);
           const hct_u32 full = full0 + 8 * stage;
-          hct_mbar_expect_tx(full, HCT_A_BOX_BYTES + HCT_B_BYTES);
+          hct_mbar_expect_tx(full, bytes);
           const hct_u32 dst = smem_base + stage * HCT_STAGE_BYTES;
-          // input pixels of this tap: channel coordinate is a multiple of 64 (16-byte aligned start);
-          // w and h may start outside the image and then read the zero padding
-          hct_tma_load_4d(dst, &hct_p.tmap[0], cb * 64, t.w0 + s - HCT_PAD, t.h0 + r - HCT_PAD, t.n, full);
-          hct_tma_load_2d(dst + HCT_A_BYTES, &hct_p.tmap[1], cb * 64, tap * HCT_KO + t.nbk * HCT_BN, full);
+          hct_tma_load_2d(dst, &hct_p.tmap[0], cb * 64, tap * HCT_KO + t.mbk * HCT_BM, full);
+          hct_tma_load_4d(dst + HCT_A_BYTES, xmap, cb * 64, s - HCT_PAD, t.h0 + r - HCT_PAD, t.n, full);
           if (++stage == HCT_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      // bf16 x bf16 -> fp32, both operands K-major, M = 128, N = HCT_BN
-      const hct_u32 idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((hct_u32)(HCT_BN >> 3) << 17) | ((hct_u32)(HCT_BM >> 4) << 24);
       int stage = 0, acc = 0;
       hct_u32 phase = 0, acc_phase = 0;
-      for (long long tile = blockIdx.x; tile < HCT_TILES; tile += gridDim.x) {
+      for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const HctConvTile t = hct_conv_tile(tile, t1);
+        if (t.th == 0) continue;
+        // bf16 x bf16 -> fp32, both operands K-major, M = 128, N = pixels of this tile rounded up to 16
+        const hct_u32 n_mma = (hct_u32)((t.th * HCT_WO + 15) & ~15);
+        const hct_u32 idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((n_mma >> 3) << 17) | ((hct_u32)(HCT_BM >> 4) << 24);
         hct_mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, &failed, status, 2);
         hct_tc_fence_after();
-        const hct_u32 d_tmem = tmem_base + acc * HCT_BN;
+        const hct_u32 d_tmem = tmem_base + acc * 256;
         for (int kb = 0; kb < HCT_KB; ++kb) {
           hct_mbar_wait(full0 + 8 * stage, phase, &failed, status, 3);
           hct_tc_fence_after();
@@ -117,21 +147,20 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
     const int q = warp & 3;
     int acc = 0;
     hct_u32 acc_phase = 0;
-    const int p = q * 32 + lane;              // pixel of the tile held by this thread's TMEM lane
-    const int hh = p / HCT_TW, ww = p % HCT_TW;
-    for (long long tile = blockIdx.x; tile < HCT_TILES; tile += gridDim.x) {
-      const HctConvTile t = hct_conv_tile(tile);
+    for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+      const HctConvTile t = hct_conv_tile(tile, t1);
+      if (t.th == 0) continue;
       hct_mbar_wait(tfull0 + 8 * acc, acc_phase, &failed, status, 4);
       hct_tc_fence_after();
-      const int h = t.h0 + hh, w = t.w0 + ww;
-      const bool live = p < HCT_TW * HCT_TH && h < HCT_HO && w < HCT_WO;
+      const int k = t.mbk * HCT_BM + q * 32 + lane;      // output channel of this thread's TMEM lane
+      const int npix = t.th * HCT_WO;                    // contiguous in the (n,k) plane from h0*WO on
+      const int chunks = (npix + 31) / 32;
 #pragma unroll 1
-      for (int c = 0; c < HCT_BN / 32; ++c) {
+      for (int c = 0; c < chunks; ++c) {
         float v[32];
-        hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * HCT_BN + c * 32, v);
-        const int k0 = t.nbk * HCT_BN + c * 32;
-        const int nk = HCT_KO - k0 < 32 ? HCT_KO - k0 : 32;
-        if (live && nk > 0) hct_epilogue_conv(hct_p, v, t.n, h, w, k0, nk);
+        hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * 256 + c * 32, v);
+        const int ncols = npix - c * 32 < 32 ? npix - c * 32 : 32;
+        if (k < HCT_KO) hct_epilogue_run(hct_p, v, (long long)t.n * HCT_KO + k, t.h0 * HCT_WO + c * 32, ncols);
       }
       hct_tc_fence_before();
       hct_mbar_arrive(tempty0 + 8 * acc);
@@ -141,5 +170,5 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
   }
   hct_tc_fence_before();
   __syncthreads();
-  if (warp == 1) hct_tmem_dealloc(tmem_base, HCT_TMEM_COLS);
+  if (warp == 1) hct_tmem_dealloc(tmem_base, 512);
 }
