@@ -15,20 +15,42 @@ extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParam
   hct_bf16_t* __restrict__ Wo = (hct_bf16_t*)hct_p.ptr[3];
   for (long long blk = blockIdx.x; blk < HCT_X_BLOCKS + HCT_W_BLOCKS; blk += gridDim.x) {
     if (blk < HCT_X_BLOCKS) {
+      // 64 channels x 64 pixels per tile: 16-byte reads along pixels, 16-byte writes along channels
       const long long n = blk / (HCT_XT_C * HCT_XT_P);
       const int rem = (int)(blk % (HCT_XT_C * HCT_XT_P));
       const int c0 = (rem / HCT_XT_P) * 64, p0 = (rem % HCT_XT_P) * 64;
-      const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;  // 64 x 4
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const int c = c0 + ty + 4 * i, p = p0 + tx;
-        tile[ty + 4 * i][tx] = (c < HCT_C && p < HCT_HW) ? X[(n * HCT_C + c) * HCT_HW + p] : (hct_bf16_t)0;
+      for (int u = 0; u < 2; ++u) {
+        const int id = threadIdx.x + 256 * u;       // 512 chunks of 8 pixels
+        const int c = c0 + (id >> 3), p = p0 + (id & 7) * 8;
+        __align__(16) hct_bf16_t v[8];
+        if (c < HCT_C && p + 7 < HCT_HW && HCT_HW % 8 == 0) {
+          *(uint4*)v = __ldg((const uint4*)(X + (n * HCT_C + c) * HCT_HW + p));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) v[j] = (c < HCT_C && p + j < HCT_HW) ? X[(n * HCT_C + c) * HCT_HW + p + j] : (hct_bf16_t)0;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) tile[id >> 3][(id & 7) * 8 + j] = v[j];
       }
       __syncthreads();
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const int p = p0 + ty + 4 * i, c = c0 + tx;
-        if (p < HCT_HW && c < HCT_C) Xo[(n * HCT_HW + p) * HCT_C + c] = tile[tx][ty + 4 * i];
+      for (int u = 0; u < 2; ++u) {
+        const int id = threadIdx.x + 256 * u;       // 512 chunks of 8 channels
+        const int p = p0 + (id >> 3), cc = (id & 7) * 8;
+        if (p < HCT_HW) {
+          __align__(16) hct_bf16_t v[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) v[j] = tile[cc + j][id >> 3];
+          hct_bf16_t* dst = Xo + (n * HCT_HW + p) * HCT_C + c0 + cc;
+          if (c0 + cc + 7 < HCT_C) {
+            *(uint4*)dst = *(const uint4*)v;       // HCT_C is a multiple of 8: 16-byte aligned
+          } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (c0 + cc + j < HCT_C) dst[j] = v[j];
+          }
+        }
       }
       __syncthreads();
     } else {
