@@ -46,6 +46,7 @@ struct Tunables {
   int row_cta_staged = 1024;       // threads per CTA of a staged row kernel (one CTA per SM)
   bool row_no_stage = false;       // load rows straight from global memory instead of through the shared-memory ring
   int row_ring_bytes = 200 * 1024; // shared memory a staged row kernel may spend on resident row vectors plus its prefetch ring
+  bool conv_no_halo = false;       // load conv pixels once per tap even when the shared-row schedule applies
   bool simt_only = false;  // keep contractions on the fp32 FMA kernels (for debugging tensor-core paths)
   static Tunables from_env();
 };

@@ -353,7 +353,11 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         k.desc = "conv layout pre-pass: NCHW->NHWC activations, KCRS->RSKC weights";
         out->push_back(k);
       }
-      int TH = (int)std::max<int64_t>(1, std::min<int64_t>(256 / WO, HO));
+      // Two schedules.  With a filter wider than one tap and rows that fill most of a 32-column pitch,
+      // pixels are loaded once per filter row and shared by its taps (conv_tc_halo); otherwise once per tap.
+      int64_t pitch = (WO + FS - 1 + 31) / 32 * 32;
+      const bool halo = FS > 1 && pitch <= 256 && WO * 10 >= pitch * 7 && !tun.conv_no_halo;
+      int TH = (int)std::max<int64_t>(1, std::min<int64_t>(256 / (halo ? pitch : WO), HO));
       int stages = 4;
       std::string epi = eg.run_fn(HO * WO, WO, "(row % " + std::to_string(KO) + "LL)");
       KernelSpec k;
@@ -362,10 +366,10 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_H " << H << "\n#define HCT_W " << W
           << "\n#define HCT_KO " << KO << "\n#define HCT_FR " << FR << "\n#define HCT_FS " << FS << "\n#define HCT_PAD " << anchor.pad
           << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TH " << TH << "\n#define HCT_TH2 1\n#define HCT_SPLIT "
-          << TH << "\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
+          << TH << "\n#define HCT_PITCH " << pitch << "\n#define HCT_NA 6\n#define HCT_NBUF 3\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
           << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
       src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[3]; void* ptr["
-          << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source("conv_tc");
+          << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source(halo ? "conv_tc_halo" : "conv_tc");
       k.source = src.str();
       k.ptrs = eg.ptrs;
       k.wants_status = true;
@@ -382,18 +386,22 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       tx.rank = 4;
       tx.dims[0] = (uint64_t)C; tx.dims[1] = (uint64_t)W; tx.dims[2] = (uint64_t)H; tx.dims[3] = (uint64_t)NB;
       tx.strides[1] = (uint64_t)C * 2; tx.strides[2] = (uint64_t)W * C * 2; tx.strides[3] = (uint64_t)H * W * C * 2;
-      tx.box[0] = 64; tx.box[1] = (uint32_t)WO; tx.box[2] = (uint32_t)TH; tx.box[3] = 1;
+      tx.box[0] = 64; tx.box[1] = (uint32_t)(halo ? pitch : WO); tx.box[2] = (uint32_t)TH; tx.box[3] = 1;
       TmaDesc tx2 = tx;
       tx2.box[2] = 1;
       k.tmaps = {tw, tx, tx2};
       int64_t tiles = NB * ((HO + TH - 1) / TH) * ((KO + 127) / 128);
       k.block[0] = 192;
-      k.smem_bytes = (unsigned)(stages * (128 * 128 + 32768) + 1024);
+      k.smem_bytes = halo ? (unsigned)(6 * 16384 + 3 * 33792 + 1024) : (unsigned)(stages * (128 * 128 + 32768) + 1024);
       k.persistent = true;
       k.max_grid = (unsigned)std::min<int64_t>(tiles, 0x7fffffff);
       k.grid[0] = k.max_grid;
       std::ostringstream d;
-      d << "conv2d tcgen05 bf16 implicit GEMM, tile 128 channels x " << TH << " rows of " << WO << " pixels, " << stages << " stages";
+      d << "conv2d tcgen05 bf16 implicit GEMM, tile 128 channels x " << TH << " rows of " << WO << " pixels, ";
+      if (halo)
+        d << "pixels shared by the taps of a filter row (pitch " << pitch << ")";
+      else
+        d << stages << " stages";
       k.desc = d.str();
       out->push_back(k);
       return;

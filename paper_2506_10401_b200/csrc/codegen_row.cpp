@@ -14,6 +14,7 @@ Tunables Tunables::from_env() {
   if (const char* s = std::getenv("HCT_ROW_CTA")) t.row_cta = std::max(32, std::atoi(s));
   if (const char* s = std::getenv("HCT_SIMT_ONLY")) t.simt_only = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_CTA_STAGED")) t.row_cta_staged = std::max(32, std::atoi(s));
+  if (const char* s = std::getenv("HCT_CONV_NO_HALO")) t.conv_no_halo = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_NO_STAGE")) t.row_no_stage = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_RING_BYTES")) t.row_ring_bytes = std::max(1024, std::atoi(s));
   return t;

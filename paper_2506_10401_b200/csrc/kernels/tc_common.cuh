@@ -113,15 +113,15 @@ __device__ __forceinline__ hct_u64 hct_smem_desc(hct_u32 addr, hct_u32 lbo, hct_
   return (hct_u64)((addr & 0x3ffffu) >> 4) | ((hct_u64)(lbo >> 4) << 16) | ((hct_u64)(sbo >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
-// ---- contiguous runs of 32 epilogue elements
+// ---- contiguous runs of up to 32 epilogue elements (16-byte accesses when the run is a whole number of vectors)
 template <typename T>
 __device__ __forceinline__ void hct_ld_run32(const T* p, float* v, int n, bool vec_ok);
 template <>
 __device__ __forceinline__ void hct_ld_run32<float>(const float* p, float* v, int n, bool vec_ok) {
-  if (n == 32 && vec_ok) {
+  if ((n & 3) == 0 && vec_ok) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      float4 t = __ldg((const float4*)p + i);
+      float4 t = 4 * i < n ? __ldg((const float4*)p + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
       v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
     }
   } else {
@@ -131,10 +131,10 @@ __device__ __forceinline__ void hct_ld_run32<float>(const float* p, float* v, in
 }
 template <>
 __device__ __forceinline__ void hct_ld_run32<hct_bf16_t>(const hct_bf16_t* p, float* v, int n, bool vec_ok) {
-  if (n == 32 && vec_ok) {
+  if ((n & 7) == 0 && vec_ok) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      uint4 t = __ldg((const uint4*)p + i);
+      uint4 t = 8 * i < n ? __ldg((const uint4*)p + i) : make_uint4(0u, 0u, 0u, 0u);
       v[8 * i] = __uint_as_float(t.x << 16); v[8 * i + 1] = __uint_as_float(t.x & 0xffff0000u);
       v[8 * i + 2] = __uint_as_float(t.y << 16); v[8 * i + 3] = __uint_as_float(t.y & 0xffff0000u);
       v[8 * i + 4] = __uint_as_float(t.z << 16); v[8 * i + 5] = __uint_as_float(t.z & 0xffff0000u);
@@ -149,9 +149,10 @@ template <typename T>
 __device__ __forceinline__ void hct_st_run32(T* p, const float* v, int n, bool vec_ok);
 template <>
 __device__ __forceinline__ void hct_st_run32<float>(float* p, const float* v, int n, bool vec_ok) {
-  if (n == 32 && vec_ok) {
+  if ((n & 3) == 0 && vec_ok) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) ((float4*)p)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+    for (int i = 0; i < 8; ++i)
+      if (4 * i < n) ((float4*)p)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
   } else {
 #pragma unroll
     for (int i = 0; i < 32; ++i)
@@ -160,10 +161,10 @@ __device__ __forceinline__ void hct_st_run32<float>(float* p, const float* v, in
 }
 template <>
 __device__ __forceinline__ void hct_st_run32<hct_bf16_t>(hct_bf16_t* p, const float* v, int n, bool vec_ok) {
-  if (n == 32 && vec_ok) {
+  if ((n & 7) == 0 && vec_ok) {
 #pragma unroll
     for (int i = 0; i < 4; ++i)
-      ((uint4*)p)[i] = make_uint4(hct_pack_bf16x2(v[8 * i], v[8 * i + 1]), hct_pack_bf16x2(v[8 * i + 2], v[8 * i + 3]),
+      if (8 * i < n) ((uint4*)p)[i] = make_uint4(hct_pack_bf16x2(v[8 * i], v[8 * i + 1]), hct_pack_bf16x2(v[8 * i + 2], v[8 * i + 3]),
                                   hct_pack_bf16x2(v[8 * i + 4], v[8 * i + 5]), hct_pack_bf16x2(v[8 * i + 6], v[8 * i + 7]));
   } else {
 #pragma unroll
