@@ -43,6 +43,9 @@ struct KernelSpec {
 struct Tunables {
   int row_nv = 4;        // vectors per thread in row kernels
   int row_cta = 256;     // threads per CTA in row kernels
+  int row_batch = 1;               // rows a row group of a staged kernel with reductions carries at once
+  int row_cta_batched = 512;       // threads per CTA when rows are batched (twice the registers per thread)
+  int row_cta_elementwise = 512;   // threads per CTA of a staged row kernel without reductions
   int row_cta_staged = 1024;       // threads per CTA of a staged row kernel (one CTA per SM)
   bool row_no_stage = false;       // load rows straight from global memory instead of through the shared-memory ring
   int row_ring_bytes = 200 * 1024; // shared memory a staged row kernel may spend on resident row vectors plus its prefetch ring

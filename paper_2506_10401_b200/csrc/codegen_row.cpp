@@ -13,6 +13,9 @@ Tunables Tunables::from_env() {
   if (const char* s = std::getenv("HCT_ROW_NV")) t.row_nv = std::max(1, std::atoi(s));
   if (const char* s = std::getenv("HCT_ROW_CTA")) t.row_cta = std::max(32, std::atoi(s));
   if (const char* s = std::getenv("HCT_SIMT_ONLY")) t.simt_only = std::atoi(s) != 0;
+  if (const char* s = std::getenv("HCT_ROW_B")) t.row_batch = std::max(1, std::atoi(s));
+  if (const char* s = std::getenv("HCT_ROW_CTA_BATCHED")) t.row_cta_batched = std::max(32, std::atoi(s));
+  if (const char* s = std::getenv("HCT_ROW_CTA_ELEMENTWISE")) t.row_cta_elementwise = std::max(32, std::atoi(s));
   if (const char* s = std::getenv("HCT_ROW_CTA_STAGED")) t.row_cta_staged = std::max(32, std::atoi(s));
   if (const char* s = std::getenv("HCT_CONV_NO_HALO")) t.conv_no_halo = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_NO_STAGE")) t.row_no_stage = std::atoi(s) != 0;
@@ -63,18 +66,19 @@ struct RowGen {
   DType ext_dtype(int node) const { return g.nodes[node].cls == OpClass::Input ? g.nodes[node].dtype : F32; }
   bool ext_is_ws(int node) const { return g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0; }
 
-  // expression for operand `a` at element index variable `e` (full-width context) or as a row scalar
+  // expression for operand `a` inside loops over b (row of the batch) and, in full-width context, e
   std::string ref(const Operand& a, bool full_ctx) {
     if (a.is_literal()) return float_lit(a.literal);
     int n = a.node;
     if (p.group_of[n] == gi) {
-      if (p.is_colv[n]) return "s" + std::to_string(n);
-      return full_ctx ? "v" + std::to_string(n) + "[e]" : "v" + std::to_string(n) + "[0]";
+      if (p.is_colv[n]) return "s" + std::to_string(n) + "[b]";
+      return full_ctx ? "v" + std::to_string(n) + "[b][e]" : "v" + std::to_string(n) + "[b][0]";
     }
     int k = find_ext(grp, n);
     switch (grp.ext[k].bcast) {
-      case Bcast::Full: return "x" + std::to_string(k) + "[e]";
+      case Bcast::Full: return "x" + std::to_string(k) + "[b][e]";
       case Bcast::RowVec: return "x" + std::to_string(k) + "[e]";
+      case Bcast::RowIdx: return "c" + std::to_string(k) + "[b]";
       default: return "c" + std::to_string(k);
     }
   }
@@ -113,7 +117,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   if (stage_bytes == 0) staged = false;
   // A staged kernel runs one large CTA per SM: its row groups share the row-vector operands, which
   // are copied to shared memory once (as fp32) instead of being re-read through L1 for every row.
-  int nstg = 0;
+  int nstg = 0, B = 1;
   int64_t rowvec_bytes = 0;
   int n_rowvec = 0;
   if (staged) {
@@ -126,12 +130,17 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
       rowvec_bytes = 0;  // too large to keep resident: read them through the cache instead
       n_rowvec = 0;
     }
-    int Gs = std::max(1, std::min<int>(tun.row_cta_staged / T, 15));
+    if (grp.has_reduction && tun.row_batch > 1 && R >= 4096) B = tun.row_batch;
+    // chains without reductions have short iterations and want a deep ring (few row groups per CTA);
+    // chains with reductions want many rows in flight to cover the reductions' latency
+    const int cta_threads = B > 1 ? tun.row_cta_batched : grp.has_reduction ? tun.row_cta_staged : tun.row_cta_elementwise;
+    int Gs = std::max(1, std::min<int>(cta_threads / T, 15));
     if ((int64_t)Gs > R) Gs = (int)std::max<int64_t>(1, R);
     while ((Gs * T) % 32 != 0) ++Gs;
     int64_t budget = (int64_t)tun.row_ring_bytes - rowvec_bytes;
-    while (Gs > 1 && budget / (Gs * stage_bytes) < 2) --Gs;
-    nstg = (int)std::min<int64_t>(8, budget / (Gs * stage_bytes));
+    while (Gs > 1 && budget / (Gs * B * stage_bytes) < 2) --Gs;
+    if (budget / (Gs * B * stage_bytes) < 2) B = 1;
+    nstg = (int)std::min<int64_t>(8, budget / (Gs * B * stage_bytes));
     if (nstg < 2 || (Gs * T) % 32 != 0)
       staged = false;
     else
@@ -144,6 +153,8 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   std::string name = "hct_row_g" + std::to_string(gi);
 
   // ---- external operands
+  const std::string FORB = "_Pragma(\"unroll\") for (int b = 0; b < HCT_B; ++b) ";
+  const std::string FORE = "_Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) ";
   std::ostringstream pre, loads, issue, fill;
   int64_t staged_off = 0, rowvec_off = 0;
   for (size_t k = 0; k < grp.ext.size(); ++k) {
@@ -154,11 +165,13 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
     switch (e.bcast) {
       case Bcast::Full:
         if (staged) {
-          loads << "      float x" << k << "[HCT_E]; hct_read_staged<" << ct << ">(hct_slot + " << staged_off << ", hct_t, x" << k << ");\n";
+          loads << "      float x" << k << "[HCT_B][HCT_E];\n      " << FORB << "hct_read_staged<" << ct << ">(hct_slot + " << staged_off
+                << " * HCT_B + b * " << C * (rg.ext_dtype(e.node) == BF16 ? 2 : 4) << ", hct_t, x" << k << "[b]);\n";
           issue << "        HCT_STAGED_ISSUE_ONE(q" << k << ", " << staged_off << ", " << C * (rg.ext_dtype(e.node) == BF16 ? 2 : 4) << ")\n";
           staged_off += C * (rg.ext_dtype(e.node) == BF16 ? 2 : 4);
         } else {
-          loads << "      float x" << k << "[HCT_E]; hct_load_row(q" << k << ", hct_row, hct_t, x" << k << ", false);\n";
+          loads << "      float x" << k << "[HCT_B][HCT_E];\n      " << FORB << "hct_load_row(q" << k << ", HCT_ROWB(b), hct_t, x" << k
+                << "[b], false);\n";
         }
         break;
       case Bcast::RowVec:
@@ -177,14 +190,14 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         break;
       case Bcast::RowIdx: {
         // index from the row's leading coordinates
-        loads << "      float c" << k << ";\n      {\n        long long r_ = hct_row, i_ = 0;\n";
+        loads << "      float c" << k << "[HCT_B];\n      " << FORB << "{\n        long long r_ = HCT_ROWB(b), i_ = 0;\n";
         for (int d = (int)grp.full_shape.size() - 2; d >= 0; --d) {
           int64_t ext = grp.full_shape[d];
           int64_t st = e.lead_stride[d];
           if (st != 0) loads << "        i_ += (r_ % " << ext << "LL) * " << st << "LL;\n";
           loads << "        r_ /= " << ext << "LL;\n";
         }
-        loads << "        c" << k << " = hct_ld1(q" << k << " + i_);\n      }\n";
+        loads << "        c" << k << "[b] = hct_ld1(q" << k << " + i_);\n      }\n";
         break;
       }
     }
@@ -201,53 +214,44 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
       std::string call = "hct_" + nd.op + "(";
       if (p.is_colv[ni]) {
         for (size_t a = 0; a < nd.args.size(); ++a) call += (a ? ", " : "") + rg.ref(nd.args[a], false);
-        b << "      const float s" << id << " = " << call << ");\n";
+        b << "      float s" << id << "[HCT_B];\n      " << FORB << "s" << id << "[b] = " << call << ");\n";
       } else {
         for (size_t a = 0; a < nd.args.size(); ++a) call += (a ? ", " : "") + rg.ref(nd.args[a], true);
-        b << "      float v" << id << "[HCT_E];\n"
-          << "      _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) v" << id << "[e] = " << call << ");\n";
+        b << "      float v" << id << "[HCT_B][HCT_E];\n      " << FORB << FORE << "v" << id << "[b][e] = " << call << ");\n";
       }
     } else if (nd.cls == OpClass::RowReduce) {
       std::string a = rg.ref(nd.args[0], true);
       bool is_max = nd.op == "row_max";
-      b << "      float s" << id << " = " << (is_max ? "-HCT_INF" : "0.0f") << ";\n"
-        << "      _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) if (HCT_HAS(e)) s" << id << " = "
-        << (is_max ? "fmaxf(s" + id + ", " + a + ")" : "s" + id + " + " + a) << ";\n"
-        << "      s" << id << " = " << (is_max ? "HCT_RMAX" : "HCT_RSUM") << "(s" << id << ");\n";
+      b << "      float s" << id << "[HCT_B];\n      " << FORB << "{\n        s" << id << "[b] = " << (is_max ? "-HCT_INF" : "0.0f") << ";\n        "
+        << FORE << "if (HCT_HAS(e)) s" << id << "[b] = " << (is_max ? "fmaxf(s" + id + "[b], " + a + ")" : "s" + id + "[b] + " + a) << ";\n      }\n"
+        << "      " << (is_max ? "HCT_RMAX" : "HCT_RSUM") << "(s" << id << ");\n";
       if (!refill_placed) { b << "@REFILL@"; refill_placed = true; }
-      if (nd.op == "row_mean") b << "      s" << id << " = s" << id << " / (float)HCT_C;\n";
+      if (nd.op == "row_mean") b << "      " << FORB << "s" << id << "[b] = s" << id << "[b] / (float)HCT_C;\n";
     } else if (nd.cls == OpClass::RowSoftmax) {
       std::string a = rg.ref(nd.args[0], true);
-      b << "      float v" << id << "[HCT_E];\n"
+      b << "      float v" << id << "[HCT_B][HCT_E];\n"
         << "      {\n"
-        << "        float m_ = -HCT_INF;\n"
-        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) if (HCT_HAS(e)) m_ = fmaxf(m_, " << a << ");\n"
-        << "        m_ = HCT_RMAX(m_);\n"
+        << "        float m_[HCT_B];\n        " << FORB << "{\n          m_[b] = -HCT_INF;\n          " << FORE << "if (HCT_HAS(e)) m_[b] = fmaxf(m_[b], " << a
+        << ");\n        }\n"
+        << "        HCT_RMAX(m_);\n"
         << (refill_placed ? "" : "@REFILL@")
-        << "        const float ml_ = -m_ * HCT_LOG2E;\n"
-        << "        float d_ = 0.0f;\n"
-        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) { v" << id << "[e] = HCT_HAS(e) ? hct_exp2_fast(fmaf(" << a
-        << ", HCT_LOG2E, ml_)) : 0.0f; d_ += v" << id << "[e]; }\n"
-        << "        d_ = HCT_RSUM(d_);\n"
-        << "        const float inv_ = 1.0f / d_;\n"
-        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) v" << id << "[e] *= inv_;\n"
+        << "        float d_[HCT_B];\n        " << FORB << "{\n          const float ml_ = -m_[b] * HCT_LOG2E;\n          d_[b] = 0.0f;\n          " << FORE
+        << "{ v" << id << "[b][e] = HCT_HAS(e) ? hct_exp2_fast(fmaf(" << a << ", HCT_LOG2E, ml_)) : 0.0f; d_[b] += v" << id << "[b][e]; }\n        }\n"
+        << "        HCT_RSUM(d_);\n        " << FORB << "{\n          const float inv_ = 1.0f / d_[b];\n          " << FORE << "v" << id
+        << "[b][e] *= inv_;\n        }\n"
         << "      }\n";
     } else if (nd.cls == OpClass::RowLayernorm) {
       std::string a = rg.ref(nd.args[0], true);
       std::string ga = rg.ref(nd.args[1], true), be = rg.ref(nd.args[2], true);
-      b << "      float v" << id << "[HCT_E];\n"
+      b << "      float v" << id << "[HCT_B][HCT_E];\n"
         << "      {\n"
-        << "        float m_ = 0.0f;\n"
-        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) if (HCT_HAS(e)) m_ += " << a << ";\n"
-        << "        m_ = HCT_RSUM(m_) / (float)HCT_C;\n"
+        << "        float m_[HCT_B];\n        " << FORB << "{\n          m_[b] = 0.0f;\n          " << FORE << "if (HCT_HAS(e)) m_[b] += " << a << ";\n        }\n"
+        << "        HCT_RSUM(m_);\n"
         << (refill_placed ? "" : "@REFILL@")
-        << "        float q_ = 0.0f;\n"
-        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) { const float d_ = HCT_HAS(e) ? " << a
-        << " - m_ : 0.0f; v" << id << "[e] = d_; q_ = fmaf(d_, d_, q_); }\n"
-        << "        q_ = HCT_RSUM(q_) / (float)HCT_C;\n"
-        << "        const float r_ = 1.0f / sqrtf(q_ + " << float_lit(nd.eps) << ");\n"
-        << "        _Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) v" << id << "[e] = fmaf(v" << id << "[e] * r_, " << ga
-        << ", " << be << ");\n"
+        << "        float q_[HCT_B];\n        " << FORB << "{\n          m_[b] = m_[b] / (float)HCT_C;\n          q_[b] = 0.0f;\n          " << FORE
+        << "{ const float d_ = HCT_HAS(e) ? " << a << " - m_[b] : 0.0f; v" << id << "[b][e] = d_; q_[b] = fmaf(d_, d_, q_[b]); }\n        }\n"
+        << "        HCT_RSUM(q_);\n        " << FORB << "{\n          const float r_ = 1.0f / sqrtf(q_[b] / (float)HCT_C + " << float_lit(nd.eps)
+        << ");\n          " << FORE << "v" << id << "[b][e] = fmaf(v" << id << "[b][e] * r_, " << ga << ", " << be << ");\n        }\n"
         << "      }\n";
     } else {
       throw Error(HCT_ERR_UNSUPPORTED, "operator " + nd.op + " cannot be part of a row kernel");
@@ -262,17 +266,19 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
     const char* ct = ctype(s.dtype);
     std::string id = std::to_string(s.node);
     if (p.is_colv[s.node])
-      stores << "      if (hct_live && hct_t == 0) hct_st1((" << ct << "*)hct_p.ptr[" << pi << "] + hct_row, s" << id << ");\n";
+      stores << "      " << FORB << "if (HCT_LIVEB(b) && hct_t == 0) hct_st1((" << ct << "*)hct_p.ptr[" << pi << "] + hct_row0 + b, s" << id
+             << "[b]);\n";
     else
-      stores << "      if (hct_live) hct_store_row((" << ct << "*)hct_p.ptr[" << pi << "], hct_row, hct_t, v" << id << ");\n";
+      stores << "      " << FORB << "if (HCT_LIVEB(b)) hct_store_row((" << ct << "*)hct_p.ptr[" << pi << "], hct_row0 + b, hct_t, v" << id
+             << "[b]);\n";
   }
 
   std::ostringstream src;
   const size_t nptr = rg.ptrs.size() + (staged ? 1 : 0);
   src << "#define HCT_T " << T << "\n#define HCT_G " << G << "\n#define HCT_V " << V << "\n#define HCT_NV " << NV << "\n"
-      << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "\n#define HCT_NPTR " << std::max<size_t>(1, nptr) << "\n";
+      << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "\n#define HCT_B " << B << "\n#define HCT_NPTR " << std::max<size_t>(1, nptr) << "\n";
   if (staged)
-    src << "#define HCT_MINB 1\n#define HCT_RING_OFF " << rowvec_bytes << "\n#define HCT_STAGED 1\n#define HCT_NSTG " << nstg << "\n#define HCT_STAGE_BYTES " << stage_bytes << "\n#define HCT_STATUS_SLOT "
+    src << "#define HCT_RING_OFF " << rowvec_bytes << "\n#define HCT_STAGED 1\n#define HCT_NSTG " << nstg << "\n#define HCT_STAGE_BYTES " << stage_bytes << "\n#define HCT_STATUS_SLOT "
         << rg.ptrs.size() << "\n";
   src << skeleton_source("common") << "\n" << skeleton_source("row") << "\n";
   if (!staged) {
@@ -282,21 +288,21 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   } else {
     src << "HCT_STAGED_KERNEL_BEGIN(" << name << ")\n"
         << pre.str() << fill.str() << (smem_rowvec ? "    __syncthreads();\n" : "")
-        << "    const long long hct_stride = (long long)gridDim.x * HCT_G;\n"
+        << "    const long long hct_stride = (long long)gridDim.x * (HCT_G * HCT_B);\n"
         << "    if (hct_t == 0) {\n"
         << "      for (int s_ = 0; s_ < HCT_NSTG; ++s_) {\n"
-        << "        HCT_STAGED_ISSUE_BEGIN((long long)blockIdx.x * HCT_G + hct_cx.g + s_ * hct_stride, s_)\n"
+        << "        HCT_STAGED_ISSUE_BEGIN(((long long)blockIdx.x * HCT_G + hct_cx.g) * HCT_B + s_ * hct_stride, s_)\n"
         << issue.str() << "        HCT_STAGED_ISSUE_END\n      }\n    }\n"
         << "    int hct_it = 0;\n"
         << "  HCT_ROW_LOOP_BEGIN\n"
         << "    if (hct_live) {\n"
         << "      const int hct_s = hct_it % HCT_NSTG;\n"
         << "      hct_row_mbar_wait(hct_smem_u32(&hct_full[hct_cx.g][hct_s]), (hct_u32)((hct_it / HCT_NSTG) & 1), &hct_failed, hct_status);\n"
-        << "      const unsigned char* hct_slot = hct_my_ring + (size_t)hct_s * HCT_STAGE_BYTES;\n"
+        << "      const unsigned char* hct_slot = hct_my_ring + (size_t)hct_s * (HCT_STAGE_BYTES * HCT_B);\n"
         << loads.str();
     // The slot may be refilled once every thread of the row has taken its share, i.e. after any
     // barrier of the row group: the first reduction's barrier if the chain has one, else one of its own.
-    std::string refill = "      if (hct_t == 0) {\n        HCT_STAGED_ISSUE_BEGIN(hct_row + HCT_NSTG * hct_stride, hct_s)\n" + issue.str() +
+    std::string refill = "      if (hct_t == 0) {\n        HCT_STAGED_ISSUE_BEGIN(hct_row0 + HCT_NSTG * hct_stride, hct_s)\n" + issue.str() +
                          "        HCT_STAGED_ISSUE_END\n      }\n";
     std::string body = b.str();
     size_t mark = body.find("@REFILL@");
@@ -315,15 +321,16 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   k.source = src.str();
   k.block[0] = (unsigned)(G * T);
   k.persistent = true;
-  k.max_grid = (unsigned)std::min<int64_t>((R + G - 1) / G, 0x7fffffff);
+  k.max_grid = (unsigned)std::min<int64_t>((R + G * B - 1) / (G * B), 0x7fffffff);
   k.grid[0] = k.max_grid;
   k.ptrs = rg.ptrs;
   if (staged) {
     k.wants_status = true;
-    k.smem_bytes = (unsigned)(rowvec_bytes + G * nstg * stage_bytes);
+    k.smem_bytes = (unsigned)(rowvec_bytes + G * nstg * B * stage_bytes);
   }
   std::ostringstream d;
   d << "row kernel T=" << T << " G=" << G << " V=" << V << " NV=" << NV;
+  if (B > 1) d << " B=" << B;
   if (staged) d << ", " << nstg << "-row bulk-copy ring";
   k.desc = d.str();
   out->push_back(k);

@@ -2,6 +2,8 @@
 //   HCT_T   threads that share one row (power of two)      HCT_G  rows handled side by side per CTA
 //   HCT_V   elements per vector access (1, 2 or 4)         HCT_NV vectors per thread
 //   HCT_R   rows                                           HCT_C  columns
+//   HCT_B   consecutive rows each row group carries at once (their reductions travel together,
+//           so the latency of a block reduction is paid once per HCT_B rows)
 //   HCT_NPTR number of pointer arguments
 // and, after it, the kernel body built from HCT_ROW_BEGIN / HCT_ROW_END.
 //
@@ -20,7 +22,7 @@ struct HctParams { void* ptr[HCT_NPTR]; };
 #define HCT_HAS(e) (HCT_FULL_VECS || HCT_COL(e) < HCT_C)
 
 #if HCT_T > 32
-#define HCT_RED_DECL __shared__ float hct_red_smem[HCT_G][2][32];
+#define HCT_RED_DECL __shared__ float hct_red_smem[HCT_G][2][HCT_B][32];
 #else
 #define HCT_RED_DECL
 #endif
@@ -32,27 +34,36 @@ struct HctRowCtx {
 };
 
 template <bool IS_MAX>
-__device__ __forceinline__ float hct_row_reduce(float v, HctRowCtx& cx, float (*red)[2][32]) {
+__device__ __forceinline__ void hct_row_reduce(float (&v)[HCT_B], HctRowCtx& cx, float (*red)[2][HCT_B][32]) {
 #pragma unroll
   for (int o = (HCT_T < 32 ? HCT_T : 32) / 2; o > 0; o >>= 1) {
-    float u = __shfl_xor_sync(0xffffffffu, v, o);
-    v = IS_MAX ? fmaxf(v, u) : v + u;
+#pragma unroll
+    for (int b = 0; b < HCT_B; ++b) {
+      float u = __shfl_xor_sync(0xffffffffu, v[b], o);
+      v[b] = IS_MAX ? fmaxf(v[b], u) : v[b] + u;
+    }
   }
 #if HCT_T > 32
-  // one partial per warp goes through shared memory; every warp then folds the HCT_T/32 partials
-  // with a second, shorter butterfly, so all threads end with the same value
-  float* slot = red[cx.g][cx.par];
+  // one partial per warp and row goes through shared memory; every warp then folds the HCT_T/32
+  // partials with a second, shorter butterfly, so all threads end with the same values
+  float (*slot)[32] = red[cx.g][cx.par];
   cx.par ^= 1u;
-  if ((cx.t & 31) == 0) slot[cx.t >> 5] = v;
+  if ((cx.t & 31) == 0) {
+#pragma unroll
+    for (int b = 0; b < HCT_B; ++b) slot[b][cx.t >> 5] = v[b];
+  }
   asm volatile("bar.sync %0, %1;" ::"r"(cx.g + 1), "n"(HCT_T) : "memory");
-  v = slot[cx.t & (HCT_T / 32 - 1)];
+#pragma unroll
+  for (int b = 0; b < HCT_B; ++b) v[b] = slot[b][cx.t & (HCT_T / 32 - 1)];
 #pragma unroll
   for (int o = HCT_T / 64; o > 0; o >>= 1) {
-    float u = __shfl_xor_sync(0xffffffffu, v, o);
-    v = IS_MAX ? fmaxf(v, u) : v + u;
+#pragma unroll
+    for (int b = 0; b < HCT_B; ++b) {
+      float u = __shfl_xor_sync(0xffffffffu, v[b], o);
+      v[b] = IS_MAX ? fmaxf(v[b], u) : v[b] + u;
+    }
   }
 #endif
-  return v;
 }
 #if HCT_T > 32
 #define HCT_RSUM(v) hct_row_reduce<false>(v, hct_cx, hct_red_smem)
@@ -155,7 +166,7 @@ __device__ __forceinline__ void hct_read_staged<hct_bf16_t>(const unsigned char*
 }
 
 #define HCT_STAGED_KERNEL_BEGIN(name)                                                          \
-  extern "C" __global__ void __launch_bounds__(HCT_T * HCT_G, HCT_MINB) name(const HctParams hct_p) {    \
+  extern "C" __global__ void __launch_bounds__(HCT_T * HCT_G, 1) name(const HctParams hct_p) {    \
     HCT_RED_DECL                                                                               \
     extern __shared__ __align__(128) unsigned char hct_ring[];                                 \
     __shared__ unsigned long long hct_full[HCT_G][HCT_NSTG];                                   \
@@ -166,7 +177,7 @@ __device__ __forceinline__ void hct_read_staged<hct_bf16_t>(const unsigned char*
     hct_cx.par = 0;                                                                            \
     const int hct_t = hct_cx.t;                                                                \
     unsigned int* hct_status = (unsigned int*)hct_p.ptr[HCT_STATUS_SLOT];                      \
-    unsigned char* hct_my_ring = hct_ring + HCT_RING_OFF + (size_t)hct_cx.g * HCT_NSTG * HCT_STAGE_BYTES;      \
+    unsigned char* hct_my_ring = hct_ring + HCT_RING_OFF + (size_t)hct_cx.g * HCT_NSTG * (HCT_STAGE_BYTES * HCT_B);      \
     if (threadIdx.x == 0) hct_failed = 0;                                                      \
     if (hct_t == 0) {                                                                          \
       for (int s_ = 0; s_ < HCT_NSTG; ++s_) {                                                  \
@@ -177,15 +188,17 @@ __device__ __forceinline__ void hct_read_staged<hct_bf16_t>(const unsigned char*
     }                                                                                          \
     __syncthreads();
 
-// issue the copies of row `r_` (if it exists) into ring slot `s_`; called by thread 0 of the row group
+// issue the copies of the HCT_B rows starting at `r_` (those that exist) into ring slot `s_`;
+// called by thread 0 of the row group.  Consecutive rows are contiguous in memory: one copy per input.
 #define HCT_STAGED_ISSUE_BEGIN(r_, s_)                                                         \
   if ((r_) < HCT_R) {                                                                          \
     const long long hct_ir = (r_);                                                             \
+    const hct_u32 hct_in = (hct_u32)(HCT_R - hct_ir < HCT_B ? HCT_R - hct_ir : HCT_B);          \
     const hct_u32 hct_ib = hct_smem_u32(&hct_full[hct_cx.g][(s_)]);                            \
-    const hct_u32 hct_id = hct_smem_u32(hct_my_ring + (size_t)(s_) * HCT_STAGE_BYTES);         \
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(hct_ib), "n"(HCT_STAGE_BYTES) : "memory");
+    const hct_u32 hct_id = hct_smem_u32(hct_my_ring + (size_t)(s_) * (HCT_STAGE_BYTES * HCT_B)); \
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(hct_ib), "r"(hct_in * (hct_u32)HCT_STAGE_BYTES) : "memory");
 #define HCT_STAGED_ISSUE_ONE(ptr, off, bytes_per_row) \
-    hct_bulk_load(hct_id + (off), (const unsigned char*)(ptr) + hct_ir * (long long)(bytes_per_row), (bytes_per_row), hct_ib);
+    hct_bulk_load(hct_id + (off) * HCT_B, (const unsigned char*)(ptr) + hct_ir * (long long)(bytes_per_row), hct_in * (hct_u32)(bytes_per_row), hct_ib);
 #define HCT_STAGED_ISSUE_END }
 
 #if HCT_T > 32
@@ -205,10 +218,14 @@ __device__ __forceinline__ void hct_read_staged<hct_bf16_t>(const unsigned char*
     const int hct_t = hct_cx.t;
 
 #define HCT_ROW_LOOP_BEGIN                                                                    \
-    for (long long hct_base = (long long)blockIdx.x * HCT_G; hct_base < HCT_R;                \
-         hct_base += (long long)gridDim.x * HCT_G) {                                          \
-      const bool hct_live = hct_base + hct_cx.g < HCT_R;                                      \
-      const long long hct_row = hct_live ? hct_base + hct_cx.g : HCT_R - 1;
+    for (long long hct_base = (long long)blockIdx.x * (HCT_G * HCT_B); hct_base < HCT_R;      \
+         hct_base += (long long)gridDim.x * (HCT_G * HCT_B)) {                                \
+      const long long hct_row0 = hct_base + (long long)hct_cx.g * HCT_B;                      \
+      const bool hct_live = hct_row0 < HCT_R;
+
+// row b of this group's batch: clamped for loads, exact for stores (guarded by HCT_LIVEB)
+#define HCT_ROWB(b) (hct_row0 + (b) < HCT_R ? hct_row0 + (b) : HCT_R - 1)
+#define HCT_LIVEB(b) (hct_row0 + (b) < HCT_R)
 
 #define HCT_ROW_LOOP_END }
 #define HCT_ROW_KERNEL_END }
