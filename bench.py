@@ -37,6 +37,26 @@ WORKLOADS = {
 HEADLINE = "c2_softmax_layernorm_chain"
 
 
+def kernel_fingerprint(g):
+    """Hash of the generated source of every kernel of a graph: changes whenever a kernel changes."""
+    import hashlib
+    h = hashlib.sha256()
+    for i in range(g.num_kernels):
+        h.update(g.kernel_source(i).encode())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(name, fingerprint):
+    """DRAM bytes per launch from the committed ncu summary, or None once the kernels have changed since."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return None
+    rec = json.load(open(path)).get(name)
+    if not rec or rec.get("fingerprint") != fingerprint:
+        return None
+    return rec["dram_bytes_per_step"]
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -56,7 +76,7 @@ class ClockSampler:
             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                          "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -214,6 +234,7 @@ def run_gpu(name, steps, warmup, rank, world, device):
     e2e_v, _ = whole_job_value(info["bound"], bytes_, flops, world, e2e_s)
     kern_s = float(np.mean(per_step))
     return dict(value=value, unit=unit, ms_per_step=dev_s / steps * 1e3, bytes=bytes_, flops=flops, kernel_s=kern_s,
+                fingerprint=kernel_fingerprint(g),
                 kernels=g.num_kernels, clocks=clocks.summary(), e2e=dict(value=e2e_v, unit=unit, h2d_bytes_per_step=h2d,
                                                                          d2h_bytes_per_step=d2h), plan=g.plan)
 
@@ -288,7 +309,7 @@ def run_sweep(steps, warmup, device, out_path=None):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="hct", choices=["hct", "reference"])
     ap.add_argument("--workload", default=HEADLINE, choices=list(WORKLOADS) + ["c5_sweep"])
@@ -353,7 +374,8 @@ def main():
                             "parallelism": "replicas" if world > 1 else "single"},
                     clocks=r["clocks"], e2e=r["e2e"], gpu_launches=r["kernels"] * args.steps,
                     roofline=dict(bound=info["bound"], achieved=achieved, peak=peak, unit=("GB/s" if info["bound"] == "hbm" else "TFLOP/s"),
-                                  frac=achieved / peak, traffic=None, peak_source=pk["source"]),
+                                  frac=achieved / peak, traffic=recorded_traffic(name, r["fingerprint"]), peak_source=pk["source"],
+                                  kernel_fingerprint=r["fingerprint"]),
                     cpu_baseline=cpu)
         print(json.dumps(line))
     if world > 1:
