@@ -50,7 +50,11 @@ struct Tunables {
   bool row_no_stage = false;       // load rows straight from global memory instead of through the shared-memory ring
   int row_ring_bytes = 200 * 1024; // shared memory a staged row kernel may spend on resident row vectors plus its prefetch ring
   bool conv_no_halo = false;       // load conv pixels once per tap even when the shared-row schedule applies
-  bool simt_only = false;  // keep contractions on the fp32 FMA kernels (for debugging tensor-core paths)
+  bool simt_only = false;
+  // Failure-path testing: the GEMM producer never issues its loads, so the consumer's bounded wait runs out
+  // (the kernel then reports through the status word and ends normally).  wait_limit shortens the bound.
+  bool fault_never_arrive = false;
+  unsigned wait_limit = 0;  // 0: kernel default  // keep contractions on the fp32 FMA kernels (for debugging tensor-core paths)
   static Tunables from_env();
 };
 

@@ -200,7 +200,9 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       k.name = "hct_gemm_tc_bf16_g" + std::to_string(gi);
       std::ostringstream src;
       src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n#define HCT_BN " << BN
-          << "\n#define HCT_STAGES " << stages << "\n#define HCT_TF32X3 0\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
+          << "\n#define HCT_STAGES " << stages << "\n#define HCT_TF32X3 0\n#define HCT_FAULT_NEVER_ARRIVE " << (tun.fault_never_arrive ? 1 : 0)
+          << (tun.wait_limit ? "\n#define HCT_WAIT_LIMIT " + std::to_string(tun.wait_limit) + "u" : std::string())
+          << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
           << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
       src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[2]; void* ptr["
           << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source("gemm_tc");

@@ -17,6 +17,8 @@ Tunables Tunables::from_env() {
   if (const char* s = std::getenv("HCT_ROW_CTA_BATCHED")) t.row_cta_batched = std::max(32, std::atoi(s));
   if (const char* s = std::getenv("HCT_ROW_CTA_ELEMENTWISE")) t.row_cta_elementwise = std::max(32, std::atoi(s));
   if (const char* s = std::getenv("HCT_ROW_CTA_STAGED")) t.row_cta_staged = std::max(32, std::atoi(s));
+  if (const char* s = std::getenv("HCT_FAULT_NEVER_ARRIVE")) t.fault_never_arrive = std::atoi(s) != 0;
+  if (const char* s = std::getenv("HCT_WAIT_LIMIT")) t.wait_limit = (unsigned)std::max(1, std::atoi(s));
   if (const char* s = std::getenv("HCT_CONV_NO_HALO")) t.conv_no_halo = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_NO_STAGE")) t.row_no_stage = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_RING_BYTES")) t.row_ring_bytes = std::max(1024, std::atoi(s));
@@ -245,10 +247,18 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
       std::string ga = rg.ref(nd.args[1], true), be = rg.ref(nd.args[2], true);
       b << "      float v" << id << "[HCT_B][HCT_E];\n"
         << "      {\n"
-        << "        float m_[HCT_B];\n        " << FORB << "{\n          m_[b] = 0.0f;\n          " << FORE << "if (HCT_HAS(e)) m_[b] += " << a << ";\n        }\n"
-        << "        HCT_RSUM(m_);\n"
-        << (refill_placed ? "" : "@REFILL@")
-        << "        float q_[HCT_B];\n        " << FORB << "{\n          m_[b] = m_[b] / (float)HCT_C;\n          q_[b] = 0.0f;\n          " << FORE
+        << "        float m_[HCT_B];\n";
+      // A softmax row sums to one, so its mean is 1/C: no reduction is needed for it.
+      const Operand& xin = nd.args[0];
+      const bool mean_known = !xin.is_literal() && p.group_of[xin.node] == gi && g.nodes[xin.node].cls == OpClass::RowSoftmax;
+      if (mean_known) {
+        b << "        " << FORB << "m_[b] = 1.0f;\n";
+      } else {
+        b << "        " << FORB << "{\n          m_[b] = 0.0f;\n          " << FORE << "if (HCT_HAS(e)) m_[b] += " << a << ";\n        }\n"
+          << "        HCT_RSUM(m_);\n"
+          << (refill_placed ? "" : "@REFILL@");
+      }
+      b << "        float q_[HCT_B];\n        " << FORB << "{\n          m_[b] = m_[b] / (float)HCT_C;\n          q_[b] = 0.0f;\n          " << FORE
         << "{ const float d_ = HCT_HAS(e) ? " << a << " - m_[b] : 0.0f; v" << id << "[b][e] = d_; q_[b] = fmaf(d_, d_, q_[b]); }\n        }\n"
         << "        HCT_RSUM(q_);\n        " << FORB << "{\n          const float r_ = 1.0f / sqrtf(q_[b] / (float)HCT_C + " << float_lit(nd.eps)
         << ");\n          " << FORE << "v" << id << "[b][e] = fmaf(v" << id << "[b][e] * r_, " << ga << ", " << be << ");\n        }\n"

@@ -85,6 +85,11 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
         const int nb = (int)(tile % HCT_NB), mb = (int)(tile / HCT_NB);
         for (int kb = 0; kb < HCT_KB; ++kb) {
           hct_mbar_wait(empty0 + 8 * stage, phase ^ 1u, &failed, status, 1);
+#if defined(HCT_FAULT_NEVER_ARRIVE) && HCT_FAULT_NEVER_ARRIVE
+          // failure-path test build: nothing ever completes the stage's barrier
+          if (++stage == HCT_STAGES) { stage = 0; phase ^= 1u; }
+          continue;
+#endif
           const hct_u32 full = full0 + 8 * stage;
           hct_mbar_expect_tx(full, HCT_STAGE_BYTES);
           hct_u32 dst = smem_base + stage * HCT_STAGE_BYTES;

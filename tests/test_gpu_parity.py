@@ -201,3 +201,39 @@ def test_bad_pointers_are_rejected_on_the_host():
         hct.hct_graph_run(g.handle, [x.data_ptr()], [])
     with pytest.raises(hct.HctError):
         hct.hct_graph_run(g.handle, [0], [y.data_ptr()])
+
+
+def test_softmax_feeding_layernorm_uses_known_mean_and_matches():
+    spec = """hct 1
+input x f32 [130,1000]
+input g f32 [1000]
+input b f32 [1000]
+node p = row_softmax(x)
+node y = row_layernorm(p, g, b, eps=1e-7)
+node q = add(p, 0.001)
+node z = row_layernorm(q, g, b, eps=1e-7)
+output y
+output z
+"""
+    check_f32(spec, {"x": N_, "g": POS_, "b": N_})
+
+
+def test_expired_device_wait_is_reported_and_the_device_stays_usable(monkeypatch):
+    """A GEMM whose producer never issues its loads: the consumer's bounded wait runs out, the kernel
+    ends normally, hct_graph_status reports the timeout, and the next graph runs as usual."""
+    import torch
+    import paper_2506_10401_b200 as hct
+    spec, laws = configs.get_config("c3_gemm_bf16_gelu_residual", m=128, k=128, n=256)
+    t = configs.draw_inputs(spec, laws, 0)
+    monkeypatch.setenv("HCT_FAULT_NEVER_ARRIVE", "1")
+    monkeypatch.setenv("HCT_WAIT_LIMIT", "2000")
+    g = hct.FusedGraph(spec, 0)
+    monkeypatch.delenv("HCT_FAULT_NEVER_ARRIVE")
+    monkeypatch.delenv("HCT_WAIT_LIMIT")
+    g.run(parity.to_device(spec, t))
+    torch.cuda.synchronize()
+    with pytest.raises(hct.HctError) as e:
+        g.status()
+    assert e.value.code == hct.HCT_ERR_TIMEOUT
+    g.status()  # the word was cleared
+    check_bf16(spec, laws)
