@@ -1,4 +1,5 @@
 // C ABI: graph handle life cycle, launches and queries.
+#include <cstdlib>
 #include <cstring>
 #include <memory>
 #include <sstream>
@@ -55,6 +56,7 @@ struct hct_graph {
   size_t scratch_bytes = 0;     // kernel-private scratch appended after the planner's intermediates
   size_t workspace_bytes = 0;
   int device = HCT_DEVICE_NONE;
+  bool use_pdl = true;
   CUcontext_t ctx = nullptr;
   CUdevice_t cudev = 0;
   CUdeviceptr_t status_word = 0;
@@ -113,6 +115,7 @@ hct_status_t hct_graph_create(const char* spec, size_t spec_len, int device, hct
     for (size_t k = 0; k < specs.size(); ++k) pt << "launch " << k << ": " << specs[k].name << " (" << specs[k].desc << ")\n";
     h->plan_text = pt.str();
     h->device = device;
+    if (const char* e = std::getenv("HCT_NO_PDL")) h->use_pdl = std::atoi(e) == 0;
 
     const Driver* d = nullptr;
     int sms = 148;
@@ -233,8 +236,26 @@ hct_status_t hct_graph_run(hct_graph_t* g, const void* const* inputs, int n_inpu
       }
       std::memcpy(block + off, ptrs, std::max<size_t>(np, 1) * sizeof(void*));
       void* args[] = {block};
-      CUresult_t rc = d.LaunchKernel(k.func, k.grid[0], k.grid[1], k.grid[2], k.spec.block[0], k.spec.block[1], k.spec.block[2],
-                                     k.spec.smem_bytes, (CUstream_t)cuda_stream, args, nullptr);
+      // Kernels after the first may be scheduled while their predecessor drains (programmatic dependent
+      // launch): each kernel waits on the device for the predecessor's completion before it reads memory.
+      CUresult_t rc;
+      if (&k != &g->kernels.front() && g->use_pdl) {
+        LaunchAttr attr;
+        std::memset(&attr, 0, sizeof attr);
+        attr.id = kLaunchAttrProgrammaticStreamSerialization;
+        attr.value.programmatic_stream_serialization_allowed = 1;
+        LaunchConfig cfg;
+        cfg.gridX = k.grid[0]; cfg.gridY = k.grid[1]; cfg.gridZ = k.grid[2];
+        cfg.blockX = k.spec.block[0]; cfg.blockY = k.spec.block[1]; cfg.blockZ = k.spec.block[2];
+        cfg.sharedMemBytes = k.spec.smem_bytes;
+        cfg.stream = (CUstream_t)cuda_stream;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        rc = d.LaunchKernelEx(&cfg, k.func, args, nullptr);
+      } else {
+        rc = d.LaunchKernel(k.func, k.grid[0], k.grid[1], k.grid[2], k.spec.block[0], k.spec.block[1], k.spec.block[2],
+                            k.spec.smem_bytes, (CUstream_t)cuda_stream, args, nullptr);
+      }
       if (rc != 0) return set_error(HCT_ERR_CUDA, cu_error(d, rc, ("launch of " + k.spec.name).c_str()));
     }
   } catch (const Error& e) {

@@ -26,6 +26,23 @@ enum {
   kFuncAttrMaxDynamicSharedSizeBytes = 8,
 };
 
+// cuLaunchKernelEx configuration (layout of CUlaunchConfig / CUlaunchAttribute)
+struct LaunchAttr {
+  int id;
+  char pad[4];
+  union {
+    char pad64[64];
+    int programmatic_stream_serialization_allowed;
+  } value;
+};
+struct LaunchConfig {
+  unsigned gridX, gridY, gridZ, blockX, blockY, blockZ, sharedMemBytes;
+  CUstream_t stream;
+  LaunchAttr* attrs;
+  unsigned numAttrs;
+};
+enum { kLaunchAttrProgrammaticStreamSerialization = 6 };
+
 struct Driver {
   CUresult_t (*Init)(unsigned);
   CUresult_t (*GetErrorString)(CUresult_t, const char**);
@@ -42,6 +59,7 @@ struct Driver {
   CUresult_t (*OccupancyMaxActiveBlocksPerMultiprocessor)(int*, CUfunction_t, int, size_t);
   CUresult_t (*LaunchKernel)(CUfunction_t, unsigned, unsigned, unsigned, unsigned, unsigned, unsigned, unsigned, CUstream_t,
                              void**, void**);
+  CUresult_t (*LaunchKernelEx)(const LaunchConfig*, CUfunction_t, void**, void**);
   CUresult_t (*MemAlloc)(CUdeviceptr_t*, size_t);
   CUresult_t (*MemFree)(CUdeviceptr_t);
   CUresult_t (*MemcpyDtoH)(void*, CUdeviceptr_t, size_t);

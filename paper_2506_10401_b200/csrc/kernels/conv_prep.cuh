@@ -8,6 +8,8 @@
 #define HCT_W_ELEMS ((long long)HCT_KO * HCT_C * HCT_RS)
 #define HCT_W_BLOCKS ((HCT_W_ELEMS + 255) / 256)
 extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {
+  hct_pdl_launch_dependents();
+  hct_pdl_wait();
   __shared__ hct_bf16_t tile[64][66];
   const hct_bf16_t* __restrict__ X = (const hct_bf16_t*)hct_p.ptr[0];
   const hct_bf16_t* __restrict__ Wt = (const hct_bf16_t*)hct_p.ptr[1];

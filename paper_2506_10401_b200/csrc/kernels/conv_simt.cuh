@@ -2,6 +2,8 @@
 // Defined by the generator: HCT_NB, HCT_CI, HCT_H, HCT_W, HCT_KO, HCT_FR, HCT_FS, HCT_STRIDE, HCT_PAD,
 // HCT_HO, HCT_WO, HCT_TA, HCT_TB, HCT_PA, HCT_PB, HctParams, hct_epilogue(), HCT_KERNEL_NAME.
 extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {
+  hct_pdl_launch_dependents();
+  hct_pdl_wait();
   const HCT_TA* __restrict__ X = (const HCT_TA*)hct_p.ptr[HCT_PA];
   const HCT_TB* __restrict__ Wt = (const HCT_TB*)hct_p.ptr[HCT_PB];
   const long long total = (long long)HCT_NB * HCT_KO * HCT_HO * HCT_WO;

@@ -68,6 +68,7 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
     }
   }
 
+  hct_pdl_launch_dependents();
   if (threadIdx.x == 0) {
     failed = 0;
     for (int s = 0; s < HCT_STAGES; ++s) {
@@ -88,6 +89,7 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
   __syncthreads();
   hct_tc_fence_after();
   const hct_u32 tmem_base = *(volatile hct_u32*)&tmem_holder;
+  hct_pdl_wait();   // barriers, tensor memory and descriptors are ready; now the predecessor's data may be read
 
   if (warp == 0) {
     if (lane == 0) {

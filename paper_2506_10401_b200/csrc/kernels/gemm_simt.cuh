@@ -2,6 +2,8 @@
 // Defined by the generator: HCT_M, HCT_N, HCT_K, HCT_TA, HCT_TB (operand element types),
 // HCT_PA, HCT_PB (pointer slots), HctParams, hct_epilogue(), HCT_KERNEL_NAME.
 extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {
+  hct_pdl_launch_dependents();
+  hct_pdl_wait();
   __shared__ float As[16][64 + 4];
   __shared__ float Bs[16][64 + 4];
   const HCT_TA* __restrict__ A = (const HCT_TA*)hct_p.ptr[HCT_PA];

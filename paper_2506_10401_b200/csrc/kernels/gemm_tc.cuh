@@ -56,6 +56,7 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
   const hct_u32 full0 = hct_smem_addr(&bars[0]), empty0 = hct_smem_addr(&bars[HCT_STAGES]);
   const hct_u32 tfull0 = hct_smem_addr(&bars[2 * HCT_STAGES]), tempty0 = hct_smem_addr(&bars[2 * HCT_STAGES + 2]);
 
+  hct_pdl_launch_dependents();
   if (threadIdx.x == 0) {
     failed = 0;
     for (int s = 0; s < HCT_STAGES; ++s) {
@@ -75,6 +76,7 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
   __syncthreads();
   hct_tc_fence_after();
   const hct_u32 tmem_base = *(volatile hct_u32*)&tmem_holder;
+  hct_pdl_wait();   // barriers, tensor memory and descriptors are ready; now the predecessor's data may be read
 
   if (warp == 0) {
     // ---------------- TMA producer

@@ -178,6 +178,7 @@ __device__ __forceinline__ void hct_read_staged<hct_bf16_t>(const unsigned char*
     const int hct_t = hct_cx.t;                                                                \
     unsigned int* hct_status = (unsigned int*)hct_p.ptr[HCT_STATUS_SLOT];                      \
     unsigned char* hct_my_ring = hct_ring + HCT_RING_OFF + (size_t)hct_cx.g * HCT_NSTG * (HCT_STAGE_BYTES * HCT_B);      \
+    hct_pdl_launch_dependents();                                                               \
     if (threadIdx.x == 0) hct_failed = 0;                                                      \
     if (hct_t == 0) {                                                                          \
       for (int s_ = 0; s_ < HCT_NSTG; ++s_) {                                                  \
@@ -186,6 +187,7 @@ __device__ __forceinline__ void hct_read_staged<hct_bf16_t>(const unsigned char*
       }                                                                                        \
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");                       \
     }                                                                                          \
+    hct_pdl_wait();                                                                            \
     __syncthreads();
 
 // issue the copies of the HCT_B rows starting at `r_` (those that exist) into ring slot `s_`;
@@ -215,7 +217,9 @@ __device__ __forceinline__ void hct_read_staged<hct_bf16_t>(const unsigned char*
     hct_cx.t = threadIdx.x % HCT_T;                                                           \
     hct_cx.g = threadIdx.x / HCT_T;                                                           \
     hct_cx.par = 0;                                                                           \
-    const int hct_t = hct_cx.t;
+    const int hct_t = hct_cx.t;                                                               \
+    hct_pdl_launch_dependents();                                                              \
+    hct_pdl_wait();
 
 #define HCT_ROW_LOOP_BEGIN                                                                    \
     for (long long hct_base = (long long)blockIdx.x * (HCT_G * HCT_B); hct_base < HCT_R;      \

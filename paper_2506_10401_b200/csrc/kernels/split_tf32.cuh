@@ -14,6 +14,8 @@ __device__ __forceinline__ float hct_to_tf32(float x) {
 #define HCT_BT_K ((HCT_K + 31) / 32)
 #define HCT_BT_N ((HCT_N + 31) / 32)
 extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {
+  hct_pdl_launch_dependents();
+  hct_pdl_wait();
   __shared__ float tile[32][33];
   for (long long blk = blockIdx.x; blk < HCT_A_BLOCKS + HCT_BT_K * HCT_BT_N; blk += gridDim.x) {
     if (blk < HCT_A_BLOCKS) {

@@ -128,6 +128,7 @@ const Driver& driver() {
     HCT_SYM(FuncSetAttribute, "cuFuncSetAttribute")
     HCT_SYM(OccupancyMaxActiveBlocksPerMultiprocessor, "cuOccupancyMaxActiveBlocksPerMultiprocessor")
     HCT_SYM(LaunchKernel, "cuLaunchKernel")
+    HCT_SYM(LaunchKernelEx, "cuLaunchKernelEx")
     HCT_SYM(MemAlloc, "cuMemAlloc_v2")
     HCT_SYM(MemFree, "cuMemFree_v2")
     HCT_SYM(MemcpyDtoH, "cuMemcpyDtoH_v2")
