@@ -10,6 +10,9 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); runs through the C-ABI library")
+    # the library is built in-tree and kept out of version control: (re)build it when missing or stale
+    from paper_2506_10401_b200 import build as _build
+    _build.build()
 
 
 def pytest_collection_modifyitems(config, items):

@@ -146,3 +146,7 @@ output s
 def test_unsupported_broadcast_is_reported_not_emulated():
     spec = "hct 1\ninput x f32 [4,3,8]\ninput v f32 [4,1,8]\nnode y = add(x, v)\noutput y\n"
     assert _code(spec) == hct.HCT_ERR_UNSUPPORTED
+
+
+def test_row_longer_than_the_limit_is_unsupported():
+    assert _code("hct 1\ninput x f32 [2,131076]\nnode y = row_softmax(x)\noutput y\n") == hct.HCT_ERR_UNSUPPORTED

@@ -27,7 +27,7 @@ def check_bf16(spec, laws, seed=0):
 
 # ------------------------------------------------------------------ memory-bound chains
 
-@pytest.mark.parametrize("r,c", [(300, 4096), (37, 1000), (5, 1023), (64, 130), (1, 4096), (129, 256), (33, 8192), (7, 20000)])
+@pytest.mark.parametrize("r,c", [(300, 4096), (37, 1000), (5, 1023), (64, 130), (1, 4096), (129, 256), (33, 8192), (7, 20000), (3, 65536), (2, 131072)])
 def test_softmax_layernorm_chain_shapes(r, c):
     spec, laws = configs.get_config("c2_softmax_layernorm_chain", r=r, c=c)
     g = check_f32(spec, laws)
@@ -101,7 +101,7 @@ def test_config1_gemm_bias_relu_full_size():
     check_f32(spec, laws)
 
 
-@pytest.mark.parametrize("m,k,n", [(1, 1, 1), (5, 7, 3), (130, 260, 72), (300, 1000, 520), (64, 4096, 128)])
+@pytest.mark.parametrize("m,k,n", [(1, 1, 1), (5, 7, 3), (130, 260, 72), (300, 1000, 520), (64, 4096, 128), (128, 16384, 128), (2, 8, 4100)])
 def test_gemm_f32_shapes(m, k, n):
     spec, laws = configs.get_config("c1_gemm_bias_relu_f32", m=m, k=k, n=n)
     check_f32(spec, laws)
@@ -114,7 +114,7 @@ def test_gemm_f32_integer_inputs_are_exact():
     np.testing.assert_array_equal(got[0], want[0])
 
 
-@pytest.mark.parametrize("m,k,n", [(300, 264, 520), (128, 64, 256), (1, 8, 8), (257, 4096, 136), (2048, 512, 1024)])
+@pytest.mark.parametrize("m,k,n", [(300, 264, 520), (128, 64, 256), (1, 8, 8), (257, 4096, 136), (2048, 512, 1024), (130, 16384, 72)])
 def test_gemm_bf16_chain_shapes(m, k, n):
     spec, laws = configs.get_config("c3_gemm_bf16_gelu_residual", m=m, k=k, n=n)
     check_bf16(spec, laws)
