@@ -131,12 +131,9 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
           hct_mbar_wait(full0 + 8 * stage, phase, &failed, status, 3);
           hct_tc_fence_after();
           const hct_u32 a_addr = smem_base + stage * HCT_STAGE_BYTES, b_addr = a_addr + HCT_A_BYTES;
+          const hct_u64 a_desc0 = hct_smem_desc(a_addr, 16, 1024), b_desc0 = hct_smem_desc(b_addr, 16, 1024);
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
-            const hct_u64 adesc = hct_smem_desc(a_addr + kk * 32, 16, 1024);
-            const hct_u64 bdesc = hct_smem_desc(b_addr + kk * 32, 16, 1024);
-            hct_mma_f16(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0);
-          }
+          for (int kk = 0; kk < 4; ++kk) hct_mma_f16(d_tmem, a_desc0 + kk * 2, b_desc0 + kk * 2, idesc, (kb | kk) != 0);
           hct_mma_commit(empty0 + 8 * stage);
           if (++stage == HCT_STAGES) { stage = 0; phase ^= 1u; }
         }

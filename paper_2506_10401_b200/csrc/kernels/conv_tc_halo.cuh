@@ -141,15 +141,13 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
             hct_mbar_wait(afull0 + 8 * sa, pa, &failed, status, 6);
             hct_tc_fence_after();
             const hct_u32 a_addr = smem_base + sa * HCT_A_BYTES;
+            // tap s reads the pixel buffer s rows (s * 128 bytes) further on.  The 128-byte swizzle is a
+            // function of the absolute shared-memory address (measured: results are exact with the
+            // descriptor's base-offset field left at zero), so a start that is not a multiple of 8 rows
+            // needs nothing else.  Descriptors differ only in the start-address field (16-byte units).
+            const hct_u64 a_desc0 = hct_smem_desc(a_addr, 16, 1024), b_desc0 = hct_smem_desc(b_addr + s * 128, 16, 1024);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              const hct_u64 adesc = hct_smem_desc(a_addr + kk * 32, 16, 1024);
-              // tap s reads the pixel buffer s rows further on.  The 128-byte swizzle is a function of the
-              // absolute shared-memory address (measured: results are exact with the descriptor's
-              // base-offset field left at zero), so a start that is not a multiple of 8 rows needs nothing else
-              const hct_u64 bdesc = hct_smem_desc(b_addr + s * 128 + kk * 32, 16, 1024);
-              hct_mma_f16(d_tmem, adesc, bdesc, idesc, (rb | s | kk) != 0);
-            }
+            for (int kk = 0; kk < 4; ++kk) hct_mma_f16(d_tmem, a_desc0 + kk * 2, b_desc0 + kk * 2, idesc, (rb | s | kk) != 0);
             hct_mma_commit(aempty0 + 8 * sa);
             if (++sa == HCT_NA) { sa = 0; pa ^= 1u; }
           }

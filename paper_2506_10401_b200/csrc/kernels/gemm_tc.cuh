@@ -134,11 +134,13 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
           const hct_u32 a_addr = smem_base + stage * HCT_STAGE_BYTES;
 #if HCT_TF32X3
           const hct_u32 b_addr = a_addr + 2 * HCT_A_BYTES;
+          const hct_u64 a_desc0 = hct_smem_desc(a_addr, 16, 1024), b_desc0 = hct_smem_desc(b_addr, 16, 1024);
 #pragma unroll
           for (int kk = 0; kk < HCT_BK / HCT_UMMA_K; ++kk) {
             // both operands K-major: one MMA step is 32 bytes further along the swizzled rows
-            const hct_u64 a_hi = hct_smem_desc(a_addr + kk * 32, 16, 1024), a_lo = hct_smem_desc(a_addr + HCT_A_BYTES + kk * 32, 16, 1024);
-            const hct_u64 b_hi = hct_smem_desc(b_addr + kk * 32, 16, 1024), b_lo = hct_smem_desc(b_addr + HCT_B_BYTES + kk * 32, 16, 1024);
+            // descriptors differ from the stage's first one only in the start-address field (16-byte units)
+            const hct_u64 a_hi = a_desc0 + kk * 2, a_lo = a_desc0 + (HCT_A_BYTES >> 4) + kk * 2;
+            const hct_u64 b_hi = b_desc0 + kk * 2, b_lo = b_desc0 + (HCT_B_BYTES >> 4) + kk * 2;
             // small cross terms first, then the leading product
             hct_mma_tf32(d_tmem, a_lo, b_hi, idesc, (kb > kb0) || (kk != 0));
             hct_mma_tf32(d_tmem, a_hi, b_lo, idesc, 1);
@@ -146,11 +148,11 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
           }
 #else
           const hct_u32 b_addr = a_addr + HCT_A_BYTES;
+          // descriptors differ from the stage's first one only in the start-address field (16-byte units)
+          const hct_u64 a_desc0 = hct_smem_desc(a_addr, 16, 1024), b_desc0 = hct_smem_desc(b_addr, HCT_BBOX_BYTES, 1024);
 #pragma unroll
           for (int kk = 0; kk < HCT_BK / HCT_UMMA_K; ++kk) {
-            const hct_u64 adesc = hct_smem_desc(a_addr + kk * 32, 16, 1024);
-            const hct_u64 bdesc = hct_smem_desc(b_addr + kk * 2048, HCT_BBOX_BYTES, 1024);
-            hct_mma_f16(d_tmem, adesc, bdesc, idesc, (kb > kb0) || (kk != 0));
+            hct_mma_f16(d_tmem, a_desc0 + kk * 2, b_desc0 + kk * (2048 >> 4), idesc, (kb > kb0) || (kk != 0));
           }
 #endif
           hct_mma_commit(empty0 + 8 * stage);   // frees the stage once these MMAs have read it
