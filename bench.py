@@ -61,8 +61,9 @@ def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         p = json.load(open(path))
-        return {"hbm": p["hbm_gbs"], "tensor": p["bf16_tflops"], "source": "measured"}
-    return {"hbm": 6650.0, "tensor": 1590.0, "source": "fallback"}
+        return {"hbm": p["hbm_gbs"], "tensor": p["bf16_tflops"], "tensor_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm": 6650.0, "tensor": 1590.0, "tensor_sustained": 1400.0, "source": "fallback"}
 
 
 class ClockSampler:
@@ -309,7 +310,7 @@ def run_sweep(steps, warmup, device, out_path=None):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="hct", choices=["hct", "reference"])
     ap.add_argument("--workload", default=HEADLINE, choices=list(WORKLOADS) + ["c5_sweep"])
@@ -369,7 +370,12 @@ def main():
     if rank == 0:
         pk = peaks()
         achieved, unit = metric_of(info["bound"], r["bytes"], r["flops"], r["kernel_s"])
-        peak = pk["hbm"] if info["bound"] == "hbm" else pk["tensor"]
+        # a contraction timed over a long run sits under the power cap: compare with the sustained GEMM
+        # figure then, with the burst figure when the clocks stayed at their maximum
+        clk = r["clocks"]
+        capped = "sw_power_cap" in clk["reasons"] and clk["sm_mhz"] and clk["sm_max_mhz"] and clk["sm_mhz"] < 0.9 * clk["sm_max_mhz"]
+        peak_kind = "copy" if info["bound"] == "hbm" else ("gemm sustained" if capped else "gemm burst")
+        peak = pk["hbm"] if info["bound"] == "hbm" else (pk["tensor_sustained"] if capped else pk["tensor"])
         line = dict(metric=metric, value=r["value"], unit=r["unit"], n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
                     ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
                     dtype="bf16" if "bf16" in name else "f32", data="synthetic",
@@ -378,7 +384,7 @@ def main():
                     clocks=r["clocks"], e2e=r["e2e"], gpu_launches=r["kernels"] * args.steps,
                     roofline=dict(bound=info["bound"], achieved=achieved, peak=peak, unit=("GB/s" if info["bound"] == "hbm" else "TFLOP/s"),
                                   frac=achieved / peak, traffic=recorded_traffic(name, r["fingerprint"]), peak_source=pk["source"],
-                                  kernel_fingerprint=r["fingerprint"]),
+                                  peak_kind=peak_kind, kernel_fingerprint=r["fingerprint"]),
                     cpu_baseline=cpu)
         print(json.dumps(line))
     if world > 1:
