@@ -239,7 +239,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         << (refill_placed ? "" : "@REFILL@")
         << "        float d_[HCT_B];\n        " << FORB << "{\n          const float ml_ = -m_[b] * HCT_LOG2E;\n          d_[b] = 0.0f;\n          " << FORE
         << "{ v" << id << "[b][e] = HCT_HAS(e) ? hct_exp2_fast(fmaf(" << a << ", HCT_LOG2E, ml_)) : 0.0f; d_[b] += v" << id << "[b][e]; }\n        }\n"
-        << "        HCT_RSUM(d_);\n        " << FORB << "{\n          const float inv_ = 1.0f / d_[b];\n          " << FORE << "v" << id
+        << "        HCT_RSUM(d_);\n        " << FORB << "{\n          const float inv_ = hct_rcp_fast(d_[b]);\n          " << FORE << "v" << id
         << "[b][e] *= inv_;\n        }\n"
         << "      }\n";
     } else if (nd.cls == OpClass::RowLayernorm) {
@@ -260,7 +260,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
       }
       b << "        float q_[HCT_B];\n        " << FORB << "{\n          m_[b] = m_[b] / (float)HCT_C;\n          q_[b] = 0.0f;\n          " << FORE
         << "{ const float d_ = HCT_HAS(e) ? " << a << " - m_[b] : 0.0f; v" << id << "[b][e] = d_; q_[b] = fmaf(d_, d_, q_[b]); }\n        }\n"
-        << "        HCT_RSUM(q_);\n        " << FORB << "{\n          const float r_ = 1.0f / sqrtf(q_[b] / (float)HCT_C + " << float_lit(nd.eps)
+        << "        HCT_RSUM(q_);\n        " << FORB << "{\n          const float r_ = hct_rsqrt_fast(q_[b] * (1.0f / (float)HCT_C) + " << float_lit(nd.eps)
         << ");\n          " << FORE << "v" << id << "[b][e] = fmaf(v" << id << "[b][e] * r_, " << ga << ", " << be << ");\n        }\n"
         << "      }\n";
     } else {
