@@ -297,12 +297,14 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         << loads.str() << strip_marker(b.str()) << stores.str() << "  HCT_ROW_LOOP_END\nHCT_ROW_KERNEL_END\n";
   } else {
     src << "HCT_STAGED_KERNEL_BEGIN(" << name << ")\n"
-        << pre.str() << fill.str() << (smem_rowvec ? "    __syncthreads();\n" : "")
+        << pre.str()
         << "    const long long hct_stride = (long long)gridDim.x * (HCT_G * HCT_B);\n"
         << "    if (hct_t == 0) {\n"
         << "      for (int s_ = 0; s_ < HCT_NSTG; ++s_) {\n"
         << "        HCT_STAGED_ISSUE_BEGIN(((long long)blockIdx.x * HCT_G + hct_cx.g) * HCT_B + s_ * hct_stride, s_)\n"
         << issue.str() << "        HCT_STAGED_ISSUE_END\n      }\n    }\n"
+        << "    // row vectors become resident while the first rows are in flight\n"
+        << fill.str() << (smem_rowvec ? "    __syncthreads();\n" : "")
         << "    int hct_it = 0;\n"
         << "  HCT_ROW_LOOP_BEGIN\n"
         << "    if (hct_live) {\n"
