@@ -47,6 +47,11 @@ struct Tunables {
   int row_cta_batched = 512;       // threads per CTA when rows are batched (twice the registers per thread)
   int row_cta_elementwise = 512;   // threads per CTA of a staged row kernel without reductions
   int row_cta_staged = 1024;       // threads per CTA of a staged row kernel (one CTA per SM)
+  int row_min_blocks = 1;          // CTAs per SM the compiler must leave registers for (staged kernels of <= 512 threads)
+  bool row_no_small_ctas = false;  // run reduction chains as one large CTA per SM even when several small ones fit
+  int row_cta_small = 256;         // threads per CTA in the several-small-CTAs shape
+  int row_ring_bytes_small = 48 * 1024;  // ring of one small CTA
+  bool row_no_reg_rowvec = false;  // keep row vectors of reduction-free chains in shared memory instead of registers
   bool row_no_stage = false;       // load rows straight from global memory instead of through the shared-memory ring
   int row_ring_bytes = 200 * 1024; // shared memory a staged row kernel may spend on resident row vectors plus its prefetch ring
   bool conv_no_halo = false;       // load conv pixels once per tap even when the shared-row schedule applies

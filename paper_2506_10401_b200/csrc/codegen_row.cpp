@@ -20,6 +20,11 @@ Tunables Tunables::from_env() {
   if (const char* s = std::getenv("HCT_FAULT_NEVER_ARRIVE")) t.fault_never_arrive = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_WAIT_LIMIT")) t.wait_limit = (unsigned)std::max(1, std::atoi(s));
   if (const char* s = std::getenv("HCT_CONV_NO_HALO")) t.conv_no_halo = std::atoi(s) != 0;
+  if (const char* s = std::getenv("HCT_ROW_MINB")) t.row_min_blocks = std::max(1, std::atoi(s));
+  if (const char* s = std::getenv("HCT_ROW_NO_SMALL_CTAS")) t.row_no_small_ctas = std::atoi(s) != 0;
+  if (const char* s = std::getenv("HCT_ROW_CTA_SMALL")) t.row_cta_small = std::max(32, std::atoi(s));
+  if (const char* s = std::getenv("HCT_ROW_RING_BYTES_SMALL")) t.row_ring_bytes_small = std::max(1024, std::atoi(s));
+  if (const char* s = std::getenv("HCT_ROW_NO_REG_ROWVEC")) t.row_no_reg_rowvec = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_NO_STAGE")) t.row_no_stage = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_RING_BYTES")) t.row_ring_bytes = std::max(1024, std::atoi(s));
   return t;
@@ -120,6 +125,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   // A staged kernel runs one large CTA per SM: its row groups share the row-vector operands, which
   // are copied to shared memory once (as fp32) instead of being re-read through L1 for every row.
   int nstg = 0, B = 1;
+  bool reg_rowvec = false;
   int64_t rowvec_bytes = 0;
   int n_rowvec = 0;
   if (staged) {
@@ -132,14 +138,19 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
       rowvec_bytes = 0;  // too large to keep resident: read them through the cache instead
       n_rowvec = 0;
     }
+    reg_rowvec = n_rowvec > 0 && n_rowvec * NV * V <= 64 && !tun.row_no_reg_rowvec;
+    if (reg_rowvec) rowvec_bytes = 0;
+    // Chains with reductions whose row vectors fit in registers (or that have none) run as several
+    // small CTAs per SM, each with a short ring: measured best on the benchmark chain and the sweep.
+    const bool small_ctas = grp.has_reduction && rowvec_bytes == 0 && !tun.row_no_small_ctas;
     if (grp.has_reduction && tun.row_batch > 1 && R >= 4096) B = tun.row_batch;
     // chains without reductions have short iterations and want a deep ring (few row groups per CTA);
     // chains with reductions want many rows in flight to cover the reductions' latency
-    const int cta_threads = B > 1 ? tun.row_cta_batched : grp.has_reduction ? tun.row_cta_staged : tun.row_cta_elementwise;
+    const int cta_threads = B > 1 ? tun.row_cta_batched : small_ctas ? tun.row_cta_small : grp.has_reduction ? tun.row_cta_staged : tun.row_cta_elementwise;
     int Gs = std::max(1, std::min<int>(cta_threads / T, 15));
     if ((int64_t)Gs > R) Gs = (int)std::max<int64_t>(1, R);
     while ((Gs * T) % 32 != 0) ++Gs;
-    int64_t budget = (int64_t)tun.row_ring_bytes - rowvec_bytes;
+    int64_t budget = (small_ctas ? (int64_t)tun.row_ring_bytes_small : (int64_t)tun.row_ring_bytes) - rowvec_bytes;
     while (Gs > 1 && budget / (Gs * B * stage_bytes) < 2) --Gs;
     if (budget / (Gs * B * stage_bytes) < 2) B = 1;
     nstg = (int)std::min<int64_t>(8, budget / (Gs * B * stage_bytes));
@@ -148,7 +159,10 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
     else
       G = Gs;
   }
-  const bool smem_rowvec = staged && n_rowvec > 0;
+  // Row vectors of a chain with registers to spare stay in registers for the whole kernel (each thread
+  // always meets the same columns); otherwise they are copied to shared memory once per CTA.
+  if (!staged) reg_rowvec = false;
+  const bool smem_rowvec = staged && n_rowvec > 0 && !reg_rowvec;
 
   RowGen rg{g, p, grp, gi, {}, {}};
   std::ostringstream& b = rg.body;
@@ -157,7 +171,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   // ---- external operands
   const std::string FORB = "_Pragma(\"unroll\") for (int b = 0; b < HCT_B; ++b) ";
   const std::string FORE = "_Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) ";
-  std::ostringstream pre, loads, issue, fill;
+  std::ostringstream pre, loads, issue, fill, hoisted;
   int64_t staged_off = 0, rowvec_off = 0;
   for (size_t k = 0; k < grp.ext.size(); ++k) {
     const ExtOperand& e = grp.ext[k];
@@ -177,7 +191,9 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         }
         break;
       case Bcast::RowVec:
-        if (smem_rowvec) {
+        if (reg_rowvec) {
+          hoisted << "    float x" << k << "[HCT_E]; hct_load_row(q" << k << ", 0, hct_t, x" << k << ", true);\n";
+        } else if (smem_rowvec) {
           fill << "    for (int i_ = threadIdx.x * 4; i_ < HCT_C; i_ += HCT_T * HCT_G * 4) {\n"
                << "      float t_[4]; hct_vecio<4>::ld_keep(q" << k << " + i_, t_);\n"
                << "      *(float4*)(hct_ring + " << rowvec_off << " + (size_t)i_ * 4) = make_float4(t_[0], t_[1], t_[2], t_[3]);\n    }\n";
@@ -288,7 +304,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   src << "#define HCT_T " << T << "\n#define HCT_G " << G << "\n#define HCT_V " << V << "\n#define HCT_NV " << NV << "\n"
       << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "\n#define HCT_B " << B << "\n#define HCT_NPTR " << std::max<size_t>(1, nptr) << "\n";
   if (staged)
-    src << "#define HCT_RING_OFF " << rowvec_bytes << "\n#define HCT_STAGED 1\n#define HCT_NSTG " << nstg << "\n#define HCT_STAGE_BYTES " << stage_bytes << "\n#define HCT_STATUS_SLOT "
+    src << "#define HCT_MINB " << (G * T <= 512 ? tun.row_min_blocks : 1) << "\n#define HCT_RING_OFF " << rowvec_bytes << "\n#define HCT_STAGED 1\n#define HCT_NSTG " << nstg << "\n#define HCT_STAGE_BYTES " << stage_bytes << "\n#define HCT_STATUS_SLOT "
         << rg.ptrs.size() << "\n";
   src << skeleton_source("common") << "\n" << skeleton_source("row") << "\n";
   if (!staged) {
@@ -304,7 +320,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         << "        HCT_STAGED_ISSUE_BEGIN(((long long)blockIdx.x * HCT_G + hct_cx.g) * HCT_B + s_ * hct_stride, s_)\n"
         << issue.str() << "        HCT_STAGED_ISSUE_END\n      }\n    }\n"
         << "    // row vectors become resident while the first rows are in flight\n"
-        << fill.str() << (smem_rowvec ? "    __syncthreads();\n" : "")
+        << fill.str() << (smem_rowvec ? "    __syncthreads();\n" : "") << hoisted.str()
         << "    int hct_it = 0;\n"
         << "  HCT_ROW_LOOP_BEGIN\n"
         << "    if (hct_live) {\n"

@@ -166,7 +166,7 @@ __device__ __forceinline__ void hct_read_staged<hct_bf16_t>(const unsigned char*
 }
 
 #define HCT_STAGED_KERNEL_BEGIN(name)                                                          \
-  extern "C" __global__ void __launch_bounds__(HCT_T * HCT_G, 1) name(const HctParams hct_p) {    \
+  extern "C" __global__ void __launch_bounds__(HCT_T * HCT_G, HCT_MINB) name(const HctParams hct_p) {    \
     HCT_RED_DECL                                                                               \
     extern __shared__ __align__(128) unsigned char hct_ring[];                                 \
     __shared__ unsigned long long hct_full[HCT_G][HCT_NSTG];                                   \
