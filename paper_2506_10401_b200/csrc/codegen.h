@@ -55,6 +55,8 @@ struct Tunables {
   bool row_no_stage = false;       // load rows straight from global memory instead of through the shared-memory ring
   int row_ring_bytes = 200 * 1024; // shared memory a staged row kernel may spend on resident row vectors plus its prefetch ring
   bool conv_no_halo = false;       // load conv pixels once per tap even when the shared-row schedule applies
+  bool conv_no_tma_store = false;  // NCHW-reading convolution: store the output with plain vector stores instead of TMA
+  bool conv_no_direct = false;     // always take the NHWC pre-pass, even when the convolution could read NCHW itself
   bool simt_only = false;
   // Failure-path testing: the GEMM producer never issues its loads, so the consumer's bounded wait runs out
   // (the kernel then reports through the status word and ends normally).  wait_limit shortens the bound.

@@ -70,10 +70,16 @@ struct EpiGen {
   // `ncols` of them exist; vector access is legal when N is a multiple of the vector length.
   // `N` is the distance between consecutive rows; every run starts at a multiple of `vec_unit`
   // elements plus a multiple of 32; `rowidx` is the index expression of per-row operands.
-  std::string run_fn(int64_t N, int64_t vec_unit = -1, const std::string& rowidx = "row") {
+  // With `vals_only` (one store only) the function is named hct_epilogue_vals and hands the 32 values to
+  // be stored back in `out` instead of writing them: the caller stores them its own way.
+  std::string run_fn(int64_t N, int64_t vec_unit = -1, const std::string& rowidx = "row", bool vals_only = false) {
     if (vec_unit < 0) vec_unit = N;
     std::ostringstream f;
-    f << "__device__ __forceinline__ void hct_epilogue_run(const HctParams& hct_p, float (&acc)[32], long long row, int col0, int ncols) {\n";
+    if (vals_only)
+      f << "__device__ __forceinline__ void hct_epilogue_vals(const HctParams& hct_p, float (&acc)[32], long long row, int col0, int ncols, "
+           "float (&out)[32]) {\n";
+    else
+      f << "__device__ __forceinline__ void hct_epilogue_run(const HctParams& hct_p, float (&acc)[32], long long row, int col0, int ncols) {\n";
     int anchor = grp.nodes[0];
     std::ostringstream loads;
     auto vec_ok = [&](DType d) { return (N % (d == BF16 ? 8 : 4) == 0 && vec_unit % (d == BF16 ? 8 : 4) == 0) ? "true" : "false"; };
@@ -104,7 +110,8 @@ struct EpiGen {
       }
     }
     f << loads.str();
-    for (auto& st : grp.stores) f << "  float o" << st.node << "_" << (st.to_output ? 1 : 0) << "[32];\n";
+    if (!vals_only)
+      for (auto& st : grp.stores) f << "  float o" << st.node << "_" << (st.to_output ? 1 : 0) << "[32];\n";
     f << "  _Pragma(\"unroll\") for (int j = 0; j < 32; ++j) {\n";
     for (size_t i = 1; i < grp.nodes.size(); ++i) {
       const Node& nd = g.nodes[grp.nodes[i]];
@@ -113,9 +120,13 @@ struct EpiGen {
       f << ");  // " << nd.name << "\n";
     }
     for (auto& st : grp.stores)
-      f << "    o" << st.node << "_" << (st.to_output ? 1 : 0) << "[j] = " << (st.node == anchor ? "acc[j]" : "e" + std::to_string(st.node))
-        << ";\n";
+      f << "    " << (vals_only ? std::string("out") : "o" + std::to_string(st.node) + "_" + (st.to_output ? "1" : "0")) << "[j] = "
+        << (st.node == anchor ? "acc[j]" : "e" + std::to_string(st.node)) << ";\n";
     f << "  }\n";
+    if (vals_only) {
+      f << "}\n";
+      return f.str();
+    }
     for (auto& st : grp.stores) {
       int pi = ptr_index(st.node, !st.to_output);
       f << "  hct_st_run32<" << ctype(st.dtype) << ">((" << ctype(st.dtype) << "*)hct_p.ptr[" << pi << "] + row * " << N << "LL + col0, o"
@@ -326,8 +337,30 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     int64_t NB = xs[0], C = xs[1], H = xs[2], W = xs[3], KO = ws[0], FR = ws[2], FS = ws[3];
     int64_t HO = anchor.shape[2], WO = anchor.shape[3];
     if (in_bf16 && anchor.stride == 1 && C % 8 == 0 && WO <= 256 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
+      // Three schedules.  (1) Rows whose byte length is a multiple of 16 and that fill most of a 32-column
+      // pitch: the kernel reads NCHW itself and re-lays pixels in shared memory (conv_tc_nchw); only the
+      // weights take a pre-pass.  Otherwise a pre-pass writes an NHWC copy and pixels are loaded
+      // (2) once per filter row and shared by its taps (conv_tc_halo) or (3) once per tap (conv_tc).
+      const int64_t pitch = (WO + FS - 1 + 31) / 32 * 32;
+      const bool dense_pitch = pitch <= 256 && WO * 10 >= pitch * 7;
+      const int th_pitch = (int)std::max<int64_t>(1, std::min<int64_t>(256 / std::max<int64_t>(pitch, 1), HO));
+      const int n_stg = 4, n_buf = 2;
+      int n_a = 0;
+      bool direct = false;
+      // The epilogue of the NCHW-reading kernel hands its bf16 output to TMA stores (through 16 KB of
+      // shared memory) when there is a single bf16 graph output whose rows are 16-byte multiples.
+      const bool tma_store = grp.stores.size() == 1 && grp.stores[0].to_output && grp.stores[0].dtype == BF16 && WO % 8 == 0 &&
+                             !tun.conv_no_tma_store;
+      if (dense_pitch && W % 8 == 0 && !tun.conv_no_direct) {
+        // shared memory: operand buffers of TH + FR - 1 rows, staging ring, output staging, and what is left for the weight ring
+        const int64_t fixed = n_buf * ((th_pitch + FR - 1) * pitch * 128 + 1024) + n_stg * pitch * 128 + 1024 + (tma_store ? 16384 : 0);
+        n_a = (int)std::min<int64_t>(6, (232448 - 512 - fixed) / 16384);
+        direct = n_a >= 3;
+      }
+      const bool halo = !direct && FS > 1 && dense_pitch && !tun.conv_no_halo;
+      const int TH = (direct || halo) ? th_pitch : (int)std::max<int64_t>(1, std::min<int64_t>(256 / WO, HO));
       auto align256 = [](int64_t v) { return (v + 255) / 256 * 256; };
-      const int64_t x_bytes = align256(NB * C * H * W * 2), w_bytes = align256(KO * C * FR * FS * 2);
+      const int64_t x_bytes = direct ? 0 : align256(NB * C * H * W * 2), w_bytes = align256(KO * C * FR * FS * 2);
       *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(x_bytes + w_bytes));
       auto scratch = [](int64_t off) {
         BufRef r;
@@ -345,33 +378,30 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         k.name = "hct_conv_prep_g" + std::to_string(gi);
         std::ostringstream src;
         src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_HW " << H * W << "\n#define HCT_KO " << KO
-            << "\n#define HCT_RS " << FR * FS << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+            << "\n#define HCT_RS " << FR * FS << "\n#define HCT_PREP_X " << (direct ? 0 : 1) << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
             << skeleton_source("common") << "\nstruct HctParams { void* ptr[4]; };\n" << skeleton_source("conv_prep");
         k.source = src.str();
         k.ptrs = {node_buf(anchor.args[0].node), node_buf(anchor.args[1].node), scratch(0), scratch(x_bytes)};
-        int64_t blocks = NB * ((C + 63) / 64) * ((H * W + 63) / 64) + (KO * C * FR * FS + 255) / 256;
+        int64_t blocks = (direct ? 0 : NB * ((C + 63) / 64) * ((H * W + 63) / 64)) + (KO * C * FR * FS + 255) / 256;
         k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(blocks, 148 * 16));
         k.block[0] = 256;
-        k.desc = "conv layout pre-pass: NCHW->NHWC activations, KCRS->RSKC weights";
+        k.desc = direct ? "conv weight pre-pass: KCRS->RSKC" : "conv layout pre-pass: NCHW->NHWC activations, KCRS->RSKC weights";
         out->push_back(k);
       }
-      // Two schedules.  With a filter wider than one tap and rows that fill most of a 32-column pitch,
-      // pixels are loaded once per filter row and shared by its taps (conv_tc_halo); otherwise once per tap.
-      int64_t pitch = (WO + FS - 1 + 31) / 32 * 32;
-      const bool halo = FS > 1 && pitch <= 256 && WO * 10 >= pitch * 7 && !tun.conv_no_halo;
-      int TH = (int)std::max<int64_t>(1, std::min<int64_t>(256 / (halo ? pitch : WO), HO));
       int stages = 4;
-      std::string epi = eg.run_fn(HO * WO, WO, "(row % " + std::to_string(KO) + "LL)");
+      const bool use_tma_store = direct && tma_store;
+      std::string epi = eg.run_fn(HO * WO, WO, "(row % " + std::to_string(KO) + "LL)", use_tma_store);
       KernelSpec k;
       k.name = "hct_conv_tc_bf16_g" + std::to_string(gi);
       std::ostringstream src;
       src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_H " << H << "\n#define HCT_W " << W
           << "\n#define HCT_KO " << KO << "\n#define HCT_FR " << FR << "\n#define HCT_FS " << FS << "\n#define HCT_PAD " << anchor.pad
           << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TH " << TH << "\n#define HCT_TH2 1\n#define HCT_SPLIT "
-          << TH << "\n#define HCT_PITCH " << pitch << "\n#define HCT_NA 6\n#define HCT_NBUF 3\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
+          << TH << "\n#define HCT_PITCH " << pitch << "\n#define HCT_NA " << (direct ? n_a : 6) << "\n#define HCT_NBUF " << (direct ? n_buf : 3)
+          << "\n#define HCT_NSTG " << n_stg << "\n#define HCT_TMA_STORE " << (use_tma_store ? 1 : 0) << "\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
           << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
-      src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[3]; void* ptr["
-          << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source(halo ? "conv_tc_halo" : "conv_tc");
+      src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[" << (use_tma_store ? 3 : direct ? 2 : 3)
+          << "]; void* ptr[" << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source(direct ? "conv_tc_nchw" : halo ? "conv_tc_halo" : "conv_tc");
       k.source = src.str();
       k.ptrs = eg.ptrs;
       k.wants_status = true;
@@ -392,15 +422,41 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       TmaDesc tx2 = tx;
       tx2.box[2] = 1;
       k.tmaps = {tw, tx, tx2};
+      if (direct) {  // NCHW input: [64 channels x pitch pixels] of one row, no swizzle (the kernel re-lays it)
+        TmaDesc tn;
+        tn.buf = node_buf(anchor.args[0].node);
+        tn.elem_bytes = 2;
+        tn.rank = 4;
+        tn.dims[0] = (uint64_t)W; tn.dims[1] = (uint64_t)H; tn.dims[2] = (uint64_t)C; tn.dims[3] = (uint64_t)NB;
+        tn.strides[1] = (uint64_t)W * 2; tn.strides[2] = (uint64_t)H * W * 2; tn.strides[3] = (uint64_t)C * H * W * 2;
+        tn.box[0] = (uint32_t)pitch; tn.box[1] = 1; tn.box[2] = 64; tn.box[3] = 1;
+        tn.swizzle = 0;
+        k.tmaps = {tw, tn};
+        if (use_tma_store) {  // NCHW output: [32 channels x 32 pixels] of one row, 64-byte swizzle
+          TmaDesc ty;
+          ty.buf.node = grp.stores[0].node;
+          ty.elem_bytes = 2;
+          ty.rank = 4;
+          ty.dims[0] = (uint64_t)WO; ty.dims[1] = (uint64_t)HO; ty.dims[2] = (uint64_t)KO; ty.dims[3] = (uint64_t)NB;
+          ty.strides[1] = (uint64_t)WO * 2; ty.strides[2] = (uint64_t)HO * WO * 2; ty.strides[3] = (uint64_t)KO * HO * WO * 2;
+          ty.box[0] = 32; ty.box[1] = 1; ty.box[2] = 32; ty.box[3] = 1;
+          ty.swizzle = 2;
+          k.tmaps.push_back(ty);
+        }
+      }
       int64_t tiles = NB * ((HO + TH - 1) / TH) * ((KO + 127) / 128);
-      k.block[0] = 192;
-      k.smem_bytes = halo ? (unsigned)(6 * 16384 + 3 * 33792 + 1024) : (unsigned)(stages * (128 * 128 + 32768) + 1024);
+      k.block[0] = direct ? 480 : 192;
+      k.smem_bytes = direct ? (unsigned)(n_a * 16384 + n_buf * ((TH + FR - 1) * pitch * 128 + 1024) + n_stg * pitch * 128 + 1024 +
+                                         (use_tma_store ? 16384 : 0))
+                     : halo ? (unsigned)(6 * 16384 + 3 * 33792 + 1024) : (unsigned)(stages * (128 * 128 + 32768) + 1024);
       k.persistent = true;
       k.max_grid = (unsigned)std::min<int64_t>(tiles, 0x7fffffff);
       k.grid[0] = k.max_grid;
       std::ostringstream d;
       d << "conv2d tcgen05 bf16 implicit GEMM, tile 128 channels x " << TH << " rows of " << WO << " pixels, ";
-      if (halo)
+      if (direct)
+        d << "NCHW read directly and re-laid in shared memory, every pixel loaded once per tile (pitch " << pitch << ")";
+      else if (halo)
         d << "pixels shared by the taps of a filter row (pitch " << pitch << ")";
       else
         d << stages << " stages";

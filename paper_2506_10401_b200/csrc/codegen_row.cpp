@@ -20,6 +20,8 @@ Tunables Tunables::from_env() {
   if (const char* s = std::getenv("HCT_FAULT_NEVER_ARRIVE")) t.fault_never_arrive = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_WAIT_LIMIT")) t.wait_limit = (unsigned)std::max(1, std::atoi(s));
   if (const char* s = std::getenv("HCT_CONV_NO_HALO")) t.conv_no_halo = std::atoi(s) != 0;
+  if (const char* s = std::getenv("HCT_CONV_NO_TMA_STORE")) t.conv_no_tma_store = std::atoi(s) != 0;
+  if (const char* s = std::getenv("HCT_CONV_NO_DIRECT")) t.conv_no_direct = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_MINB")) t.row_min_blocks = std::max(1, std::atoi(s));
   if (const char* s = std::getenv("HCT_ROW_NO_SMALL_CTAS")) t.row_no_small_ctas = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_CTA_SMALL")) t.row_cta_small = std::max(32, std::atoi(s));

@@ -1,10 +1,11 @@
 // Layout pre-pass for the tensor-core convolution: activations NCHW -> NHWC and weights
 // KCRS -> RSKC (both bf16), so that channels, the contraction axis, are contiguous for TMA.
-// Defined by the generator: HCT_NB_IMG, HCT_C, HCT_HW (H*W), HCT_KO, HCT_RS (R*S), HctParams, HCT_KERNEL_NAME.
+// With HCT_PREP_X = 0 only the weights are rearranged (the convolution then reads NCHW itself).
+// Defined by the generator: HCT_NB_IMG, HCT_C, HCT_HW (H*W), HCT_KO, HCT_RS (R*S), HCT_PREP_X, HctParams, HCT_KERNEL_NAME.
 // Pointer slots: 0 = X (NCHW), 1 = Wt (KCRS), 2 = X as NHWC, 3 = Wt as RSKC.
 #define HCT_XT_C ((HCT_C + 63) / 64)
 #define HCT_XT_P ((HCT_HW + 63) / 64)
-#define HCT_X_BLOCKS ((long long)HCT_NB_IMG * HCT_XT_C * HCT_XT_P)
+#define HCT_X_BLOCKS (HCT_PREP_X ? (long long)HCT_NB_IMG * HCT_XT_C * HCT_XT_P : 0LL)
 #define HCT_W_ELEMS ((long long)HCT_KO * HCT_C * HCT_RS)
 #define HCT_W_BLOCKS ((HCT_W_ELEMS + 255) / 256)
 extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {

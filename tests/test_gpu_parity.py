@@ -134,6 +134,12 @@ def test_gemm_bf16_integer_inputs_are_exact():
     dict(n=2, c=3, h=8, w=8, k=5, ksize=1, pad=0),
     dict(n=1, c=8, h=12, w=10, k=4, stride=2, pad=1),
     dict(n=1, c=4, h=7, w=7, k=4, ksize=3, pad=0),
+    # rows of a multiple of 8 pixels: the kernel reads NCHW itself
+    dict(n=2, c=64, h=20, w=24, k=96),
+    dict(n=1, c=72, h=17, w=40, k=130, ksize=5, pad=2),
+    dict(n=3, c=128, h=6, w=64, k=64, ksize=1, pad=0),
+    dict(n=1, c=16, h=33, w=56, k=128, ksize=3, pad=0),
+    dict(n=2, c=8, h=5, w=120, k=8, ksize=3, pad=2),
 ])
 def test_conv_chain_shapes(kw):
     spec, laws = configs.get_config("c4_conv_bn_relu_bf16", **kw)
@@ -144,6 +150,14 @@ def test_conv_f32_integer_inputs_are_exact():
     spec = "hct 1\ninput x f32 [2,16,10,12]\ninput w f32 [8,16,3,3]\nnode y = conv2d(x, w, stride=1, pad=1)\noutput y\n"
     il = {"kind": "int", "lo": -4, "hi": 4}
     got, want, _ = parity.run_both(spec, {"x": il, "w": il})
+    np.testing.assert_array_equal(got[0], want[0])
+
+
+def test_conv_bf16_nchw_direct_integer_inputs_are_exact():
+    spec = "hct 1\ninput x bf16 [2,80,13,48]\ninput w bf16 [40,80,3,3]\nnode y = conv2d(x, w, stride=1, pad=1)\noutput y f32\n"
+    il = {"kind": "int", "lo": -4, "hi": 4}
+    got, want, g = parity.run_both(spec, {"x": il, "w": il})
+    assert "NCHW read directly" in g.plan
     np.testing.assert_array_equal(got[0], want[0])
 
 
