@@ -344,7 +344,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       const int64_t pitch = (WO + FS - 1 + 31) / 32 * 32;
       const bool dense_pitch = pitch <= 256 && WO * 10 >= pitch * 7;
       const int th_pitch = (int)std::max<int64_t>(1, std::min<int64_t>(256 / std::max<int64_t>(pitch, 1), HO));
-      const int n_stg = 4, n_buf = 2;
+      const int n_stg = 3, n_buf = 2;
       int n_a = 0;
       bool direct = false;
       // The epilogue of the NCHW-reading kernel hands its bf16 output to TMA stores (through 16 KB of
