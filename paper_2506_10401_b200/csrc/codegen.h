@@ -52,6 +52,7 @@ struct Tunables {
   int row_cta_small = 256;         // threads per CTA in the several-small-CTAs shape
   int row_ring_bytes_small = 48 * 1024;  // ring of one small CTA
   bool row_no_reg_rowvec = false;  // keep row vectors of reduction-free chains in shared memory instead of registers
+  bool row_no_softmax_ln_fusion = false;  // layer norm after softmax: take the variance with its own reduction
   bool row_no_stage = false;       // load rows straight from global memory instead of through the shared-memory ring
   int row_ring_bytes = 200 * 1024; // shared memory a staged row kernel may spend on resident row vectors plus its prefetch ring
   bool conv_no_halo = false;       // load conv pixels once per tap even when the shared-row schedule applies

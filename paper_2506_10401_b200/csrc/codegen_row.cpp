@@ -27,6 +27,7 @@ Tunables Tunables::from_env() {
   if (const char* s = std::getenv("HCT_ROW_CTA_SMALL")) t.row_cta_small = std::max(32, std::atoi(s));
   if (const char* s = std::getenv("HCT_ROW_RING_BYTES_SMALL")) t.row_ring_bytes_small = std::max(1024, std::atoi(s));
   if (const char* s = std::getenv("HCT_ROW_NO_REG_ROWVEC")) t.row_no_reg_rowvec = std::atoi(s) != 0;
+  if (const char* s = std::getenv("HCT_ROW_NO_SOFTMAX_LN_FUSION")) t.row_no_softmax_ln_fusion = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_NO_STAGE")) t.row_no_stage = std::atoi(s) != 0;
   if (const char* s = std::getenv("HCT_ROW_RING_BYTES")) t.row_ring_bytes = std::max(1024, std::atoi(s));
   return t;
@@ -224,6 +225,21 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   }
 
   // ---- nodes
+  // A layer normalisation whose input is a softmax of the same group knows its mean (1/C) and may take
+  // its variance from the softmax's sum of squared terms when eps is large enough to absorb the
+  // cancellation in mean(p^2) - 1/C^2 (C * eps >= 1/40: relative error of the result below 1.5e-6).
+  auto ln_var_from_softmax = [&](int ln) {
+    const Node& l = g.nodes[ln];
+    if (l.cls != OpClass::RowLayernorm) return false;
+    const Operand& x = l.args[0];
+    return !x.is_literal() && p.group_of[x.node] == gi && g.nodes[x.node].cls == OpClass::RowSoftmax && (double)C * l.eps >= 0.025 &&
+           !tun.row_no_softmax_ln_fusion;
+  };
+  auto softmax_feeds_fused_ln = [&](int sm) {
+    for (int other : grp.nodes)
+      if (ln_var_from_softmax(other) && g.nodes[other].args[0].node == sm) return true;
+    return false;
+  };
   bool refill_placed = false;
   for (int ni : grp.nodes) {
     const Node& nd = g.nodes[ni];
@@ -248,17 +264,29 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
       if (!refill_placed) { b << "@REFILL@"; refill_placed = true; }
       if (nd.op == "row_mean") b << "      " << FORB << "s" << id << "[b] = s" << id << "[b] / (float)HCT_C;\n";
     } else if (nd.cls == OpClass::RowSoftmax) {
+      // One exchange between the warps of a row: every warp takes its exponentials relative to its own
+      // maximum (found with shuffles alone), and the per-warp (maximum, sum) pairs are folded afterwards.
+      // A layer normalisation that reads this softmax can take its variance from the sum of squared
+      // terms gathered in the same exchange (see below); `sq<id>` then holds sum_j p_j^2 of the row.
       std::string a = rg.ref(nd.args[0], true);
+      const bool with_q = softmax_feeds_fused_ln(ni);
       b << "      float v" << id << "[HCT_B][HCT_E];\n"
+        << "      float sq" << id << "[HCT_B];\n"
         << "      {\n"
         << "        float m_[HCT_B];\n        " << FORB << "{\n          m_[b] = -HCT_INF;\n          " << FORE << "if (HCT_HAS(e)) m_[b] = fmaxf(m_[b], " << a
         << ");\n        }\n"
-        << "        HCT_RMAX(m_);\n"
+        << "        hct_warp_reduce<true>(m_);\n"
+        << "        float d_[HCT_B], q_[HCT_B];\n        " << FORB << "{\n          const float ml_ = -(m_[b] == -HCT_INF ? 0.0f : m_[b]) * HCT_LOG2E;\n"
+        << "          d_[b] = 0.0f;\n          q_[b] = 0.0f;\n          " << FORE
+        << "{ v" << id << "[b][e] = HCT_HAS(e) ? hct_exp2_fast(fmaf(" << a << ", HCT_LOG2E, ml_)) : 0.0f; d_[b] += v" << id << "[b][e];"
+        << (with_q ? " q_[b] = fmaf(v" + id + "[b][e], v" + id + "[b][e], q_[b]);" : "") << " }\n        }\n"
+        << "        hct_warp_reduce<false>(d_);\n"
+        << (with_q ? "        hct_warp_reduce<false>(q_);\n" : "")
+        << "        float f_[HCT_B];\n"
+        << "        hct_softmax_combine<" << (with_q ? "true" : "false") << ">(m_, d_, q_, f_, hct_cx, HCT_SM_SMEM);\n"
         << (refill_placed ? "" : "@REFILL@")
-        << "        float d_[HCT_B];\n        " << FORB << "{\n          const float ml_ = -m_[b] * HCT_LOG2E;\n          d_[b] = 0.0f;\n          " << FORE
-        << "{ v" << id << "[b][e] = HCT_HAS(e) ? hct_exp2_fast(fmaf(" << a << ", HCT_LOG2E, ml_)) : 0.0f; d_[b] += v" << id << "[b][e]; }\n        }\n"
-        << "        HCT_RSUM(d_);\n        " << FORB << "{\n          const float inv_ = hct_rcp_fast(d_[b]);\n          " << FORE << "v" << id
-        << "[b][e] *= inv_;\n        }\n"
+        << "        " << FORB << "{\n          const float inv_ = hct_rcp_fast(d_[b]);\n          const float k_ = f_[b] * inv_;\n          sq" << id
+        << "[b] = q_[b] * inv_ * inv_;\n          " << FORE << "v" << id << "[b][e] *= k_;\n        }\n"
         << "      }\n";
     } else if (nd.cls == OpClass::RowLayernorm) {
       std::string a = rg.ref(nd.args[0], true);
@@ -276,11 +304,23 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
           << "        HCT_RSUM(m_);\n"
           << (refill_placed ? "" : "@REFILL@");
       }
-      b << "        float q_[HCT_B];\n        " << FORB << "{\n          m_[b] = m_[b] / (float)HCT_C;\n          q_[b] = 0.0f;\n          " << FORE
-        << "{ const float d_ = HCT_HAS(e) ? " << a << " - m_[b] : 0.0f; v" << id << "[b][e] = d_; q_[b] = fmaf(d_, d_, q_[b]); }\n        }\n"
-        << "        HCT_RSUM(q_);\n        " << FORB << "{\n          const float r_ = hct_rsqrt_fast(q_[b] * (1.0f / (float)HCT_C) + " << float_lit(nd.eps)
-        << ");\n          " << FORE << "v" << id << "[b][e] = fmaf(v" << id << "[b][e] * r_, " << ga << ", " << be << ");\n        }\n"
-        << "      }\n";
+      if (mean_known && ln_var_from_softmax(ni)) {
+        // variance = mean(p^2) - 1/C^2 with sum p^2 from the softmax's exchange: no reduction at all here.
+        // Rounding of the difference is at most 2^-24 * mean(p^2) <= 2^-24 / C, which the eps under the
+        // root keeps below 2^-24 / (2 C eps) of the result (the rule applies only when C * eps >= 1/40).
+        b << "        " << FORB << "{\n          m_[b] = m_[b] / (float)HCT_C;\n          const float var_ = fmaxf(fmaf(sq" << xin.node
+          << "[b], 1.0f / (float)HCT_C, -m_[b] * m_[b]), 0.0f);\n          const float r_ = hct_rsqrt_fast(var_ + " << float_lit(nd.eps) << ");\n          "
+          << FORE << "{ const float d_ = HCT_HAS(e) ? " << a << " - m_[b] : 0.0f; v" << id << "[b][e] = fmaf(d_ * r_, " << ga << ", " << be
+          << "); }\n        }\n"
+          << "      }\n";
+      } else {
+        b << "        float q_[HCT_B];\n        " << FORB << "{\n          m_[b] = m_[b] / (float)HCT_C;\n          q_[b] = 0.0f;\n          " << FORE
+          << "{ const float d_ = HCT_HAS(e) ? " << a << " - m_[b] : 0.0f; v" << id << "[b][e] = d_; q_[b] = fmaf(d_, d_, q_[b]); }\n        }\n"
+          << "        HCT_RSUM(q_);\n"
+          << "        " << FORB << "{\n          const float r_ = hct_rsqrt_fast(q_[b] * (1.0f / (float)HCT_C) + " << float_lit(nd.eps)
+          << ");\n          " << FORE << "v" << id << "[b][e] = fmaf(v" << id << "[b][e] * r_, " << ga << ", " << be << ");\n        }\n"
+          << "      }\n";
+      }
     } else {
       throw Error(HCT_ERR_UNSUPPORTED, "operator " + nd.op + " cannot be part of a row kernel");
     }

@@ -22,7 +22,7 @@ struct HctParams { void* ptr[HCT_NPTR]; };
 #define HCT_HAS(e) (HCT_FULL_VECS || HCT_COL(e) < HCT_C)
 
 #if HCT_T > 32
-#define HCT_RED_DECL __shared__ float hct_red_smem[HCT_G][2][HCT_B][32];
+#define HCT_RED_DECL __shared__ float hct_red_smem[HCT_G][2][HCT_B][32]; __shared__ float hct_sm_smem[HCT_G][2][HCT_B][3][32];
 #else
 #define HCT_RED_DECL
 #endif
@@ -65,6 +65,74 @@ __device__ __forceinline__ void hct_row_reduce(float (&v)[HCT_B], HctRowCtx& cx,
   }
 #endif
 }
+// Reduction over the lanes of one warp that share a row (no barrier): all of them end with the result.
+template <bool IS_MAX>
+__device__ __forceinline__ void hct_warp_reduce(float (&v)[HCT_B]) {
+#pragma unroll
+  for (int o = (HCT_T < 32 ? HCT_T : 32) / 2; o > 0; o >>= 1) {
+#pragma unroll
+    for (int b = 0; b < HCT_B; ++b) {
+      float u = __shfl_xor_sync(0xffffffffu, v[b], o);
+      v[b] = IS_MAX ? fmaxf(v[b], u) : v[b] + u;
+    }
+  }
+}
+
+// Softmax statistics of a row in ONE exchange between its warps.  Every warp has taken its terms
+// t = 2^((x - m) log2 e) relative to its OWN maximum m (reference 0 when the warp saw no finite
+// value); on entry m, s, q hold the warp's maximum, sum of terms and (WITH_Q) sum of squared terms.
+// The warps' triples meet in shared memory and are folded with weights 2^((m_warp - m_row) log2 e).
+// On exit m is the row maximum, s and q the row's sums relative to it, and f the weight of the calling
+// thread's own terms: term * f / s is the softmax value.
+template <bool WITH_Q>
+__device__ __forceinline__ void hct_softmax_combine(float (&m)[HCT_B], float (&s)[HCT_B], float (&q)[HCT_B], float (&f)[HCT_B], HctRowCtx& cx,
+                                                    float (*red)[2][HCT_B][3][32]) {
+#if HCT_T > 32
+  float (*slot)[3][32] = red[cx.g][cx.par];
+  cx.par ^= 1u;
+  if ((cx.t & 31) == 0) {
+#pragma unroll
+    for (int b = 0; b < HCT_B; ++b) {
+      slot[b][0][cx.t >> 5] = m[b];
+      slot[b][1][cx.t >> 5] = s[b];
+      if (WITH_Q) slot[b][2][cx.t >> 5] = q[b];
+    }
+  }
+  asm volatile("bar.sync %0, %1;" ::"r"(cx.g + 1), "n"(HCT_T) : "memory");
+  const int j = cx.t & (HCT_T / 32 - 1);
+#pragma unroll
+  for (int b = 0; b < HCT_B; ++b) {
+    const float mj = slot[b][0][j];
+    float sj = slot[b][1][j], qj = WITH_Q ? slot[b][2][j] : 0.0f;
+    float mr = mj;
+#pragma unroll
+    for (int o = HCT_T / 64; o > 0; o >>= 1) mr = fmaxf(mr, __shfl_xor_sync(0xffffffffu, mr, o));
+    const float ref = mr == -HCT_INF ? 0.0f : mr;
+    const float fj = hct_exp2_fast(((mj == -HCT_INF ? 0.0f : mj) - ref) * HCT_LOG2E);
+    sj *= fj;
+    qj *= fj * fj;
+#pragma unroll
+    for (int o = HCT_T / 64; o > 0; o >>= 1) {
+      sj += __shfl_xor_sync(0xffffffffu, sj, o);
+      if (WITH_Q) qj += __shfl_xor_sync(0xffffffffu, qj, o);
+    }
+    f[b] = hct_exp2_fast(((m[b] == -HCT_INF ? 0.0f : m[b]) - ref) * HCT_LOG2E);
+    m[b] = mr;
+    s[b] = sj;
+    q[b] = qj;
+  }
+#else
+  (void)cx; (void)red; (void)m; (void)s; (void)q;
+#pragma unroll
+  for (int b = 0; b < HCT_B; ++b) f[b] = 1.0f;
+#endif
+}
+#if HCT_T > 32
+#define HCT_SM_SMEM hct_sm_smem
+#else
+#define HCT_SM_SMEM nullptr
+#endif
+
 #if HCT_T > 32
 #define HCT_RSUM(v) hct_row_reduce<false>(v, hct_cx, hct_red_smem)
 #define HCT_RMAX(v) hct_row_reduce<true>(v, hct_cx, hct_red_smem)

@@ -27,6 +27,17 @@ def check_bf16(spec, laws, seed=0):
 
 # ------------------------------------------------------------------ memory-bound chains
 
+@pytest.mark.parametrize("std,c", [(1e-3, 4096), (30.0, 4096), (1.0, 2560), (1e-3, 8192), (8.0, 16384)])
+def test_layernorm_of_softmax_takes_variance_from_the_softmax_sums(std, c):
+    """Near-uniform rows (variance far below 1/C^2) and nearly one-hot rows are the two ends of the
+    cancellation in mean(p^2) - 1/C^2; both must stay inside the fp32 tolerance."""
+    spec, laws = configs.get_config("c2_softmax_layernorm_chain", r=64, c=c)
+    laws = dict(laws)
+    laws["x"] = {"kind": "normal", "mean": 0.0, "std": std}
+    g = check_f32(spec, laws)
+    assert g.num_kernels == 1
+
+
 @pytest.mark.parametrize("r,c", [(300, 4096), (37, 1000), (5, 1023), (64, 130), (1, 4096), (129, 256), (33, 8192), (7, 20000), (3, 65536), (2, 131072)])
 def test_softmax_layernorm_chain_shapes(r, c):
     spec, laws = configs.get_config("c2_softmax_layernorm_chain", r=r, c=c)
