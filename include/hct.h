@@ -22,10 +22,15 @@
  *     output NAME [DTYPE]                     stored dtype, default f32
  *
  *   unary   relu gelu_tanh gelu_erf sigmoid exp tanh sqrt sin cos neg abs
+ *           dropout(x, p=0.5, seed=0)   inverted dropout with the counter-based mask of the
+ *           paper's first case study (Section 5.4): with i the element's row-major offset,
+ *           h = i + seed; h ^= h >> 17; h ^= h << 31; h ^= h >> 8 (unsigned 64 bit); the
+ *           element is kept and scaled by 1/(1-p) when h mod 1000 >= round(1000 p), else 0
  *   binary  add sub mul div max min   operands broadcast like numpy; supported
  *           patterns: equal shapes, [C] against [..,C], [..,1] against [..,C],
  *           [K,1,1] against [N,K,H,W], a number
  *   row     row_softmax(x)  row_sum(x)  row_mean(x)  row_max(x)   x: [R,C]; sums give [R,1]
+ *           (row_softmax also accepts a single column, where it is identically one)
  *           row_layernorm(x, gamma, beta, eps=1e-5)   biased variance, eps inside the root
  *   gemm(a, b)            a[M,K] · b[K,N], both row-major, both f32 or both bf16 inputs;
  *                         bf16 multiplies on tensor cores with fp32 accumulation, f32

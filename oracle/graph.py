@@ -181,6 +181,19 @@ def _infer(g, name, op, pos, attrs, where):
             if k not in allowed:
                 raise SpecError(f"{where}: unknown attribute {k!r} for {op}")
 
+    if op == "dropout":
+        only_attrs("p", "seed")
+        if len(pos) != 1:
+            raise SpecError(f"{where}: dropout takes one operand")
+        a = _operand(g, pos[0], where, False)
+        try:
+            prob = float(attrs.get("p", "0.5"))
+        except ValueError:
+            raise SpecError(f"{where}: p must be a number") from None
+        seed = _int_attr(attrs, "seed", 0, where)
+        if not (0.0 <= prob < 1.0) or seed < 0 or round(prob * 1000.0) >= 1000:
+            raise SpecError(f"{where}: dropout needs 0 <= p < 1 and a non-negative seed")
+        return Node(name, op, [a], {"p": prob, "seed": seed}, shape_of(a), "f32")
     if op in UNARY:
         only_attrs()
         if len(pos) != 1:
@@ -206,8 +219,8 @@ def _infer(g, name, op, pos, attrs, where):
             raise SpecError(f"{where}: {op} takes one operand")
         a = _operand(g, pos[0], where, False)
         s = shape_of(a)
-        if len(s) != 2 or s[1] < 2:
-            raise SpecError(f"{where}: {op} needs a [R,C] operand with C >= 2")
+        if len(s) != 2 or s[1] < (1 if op == "row_softmax" else 2):
+            raise SpecError(f"{where}: {op} needs a [R,C] operand with enough columns")
         return Node(name, op, [a], {}, s if op in ROW_TO_ROW else (s[0], 1), "f32")
     if op == "row_layernorm":
         only_attrs("eps")

@@ -50,6 +50,28 @@ _BINARY_FN = {
 }
 
 
+def dropout_keep_mask(shape, seed: int, p: float):
+    """Which elements inverted dropout keeps (the paper's first case study, Section 5.4).
+
+    The generator is counter based: the element at row-major offset ``i`` draws
+    ``h = i + seed``, then ``h ^= h >> 17``, ``h ^= h << 31``, ``h ^= h >> 8`` in
+    unsigned 64-bit arithmetic, and its uniform variate is ``(h mod 1000) / 1000``.
+    The case study elides the comparison; the reading taken here keeps the element
+    when the variate is at least ``p``, decided on integers: ``h mod 1000 >= round(1000 p)``.
+    """
+    n = int(np.prod(shape))
+    h = np.arange(n, dtype=np.uint64) + np.uint64(seed)
+    h ^= h >> np.uint64(17)
+    h ^= h << np.uint64(31)      # numpy wraps modulo 2^64, as the unsigned arithmetic does
+    h ^= h >> np.uint64(8)
+    return ((h % np.uint64(1000)) >= np.uint64(round(p * 1000.0))).reshape(shape)
+
+
+def dropout(x, p: float, seed: int):
+    """Kept elements are scaled by 1 / (1 - p), dropped ones are zero."""
+    return np.where(dropout_keep_mask(x.shape, seed, p), x / (1.0 - p), 0.0)
+
+
 # ---- row reductions (Table 1, "Reduction") --------------------------------------------------
 
 def row_sum(x):
@@ -131,7 +153,9 @@ def run_nodes(spec, inputs: dict, dtype=np.float64, gemm_fn=None) -> dict:
             continue
         args = [val[a] if isinstance(a, str) else float(a) for a in node.args]
         op = node.op
-        if op in UNARY:
+        if op == "dropout":
+            out = dropout(args[0], node.attrs["p"], node.attrs["seed"])
+        elif op in UNARY:
             out = _UNARY_FN[op](args[0])
         elif op in BINARY:
             out = _BINARY_FN[op](args[0], args[1])

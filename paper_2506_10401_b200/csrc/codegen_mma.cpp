@@ -54,9 +54,9 @@ struct EpiGen {
     };
     for (size_t i = 1; i < grp.nodes.size(); ++i) {
       const Node& nd = g.nodes[grp.nodes[i]];
-      f << "  const float e" << grp.nodes[i] << " = hct_" << nd.op << "(";
-      for (size_t a = 0; a < nd.args.size(); ++a) f << (a ? ", " : "") << ref(nd.args[a]);
-      f << ");  // " << nd.name << "\n";
+      std::vector<std::string> av;
+      for (auto& a : nd.args) av.push_back(ref(a));
+      f << "  const float e" << grp.nodes[i] << " = " << elementwise_call(nd, av, "off") << ";  // " << nd.name << "\n";
     }
     for (auto& s : grp.stores) {
       int pi = ptr_index(s.node, !s.to_output);
@@ -115,9 +115,10 @@ struct EpiGen {
     f << "  _Pragma(\"unroll\") for (int j = 0; j < 32; ++j) {\n";
     for (size_t i = 1; i < grp.nodes.size(); ++i) {
       const Node& nd = g.nodes[grp.nodes[i]];
-      f << "    const float e" << grp.nodes[i] << " = hct_" << nd.op << "(";
-      for (size_t a = 0; a < nd.args.size(); ++a) f << (a ? ", " : "") << ref(nd.args[a]);
-      f << ");  // " << nd.name << "\n";
+      std::vector<std::string> av;
+      for (auto& a : nd.args) av.push_back(ref(a));
+      f << "    const float e" << grp.nodes[i] << " = " << elementwise_call(nd, av, "row * " + std::to_string(N) + "LL + col0 + j") << ";  // "
+        << nd.name << "\n";
     }
     for (auto& st : grp.stores)
       f << "    " << (vals_only ? std::string("out") : "o" + std::to_string(st.node) + "_" + (st.to_output ? "1" : "0")) << "[j] = "
@@ -172,9 +173,9 @@ struct EpiGen {
     f << "  _Pragma(\"unroll\") for (int j = 0; j < 32; ++j) {\n";
     for (size_t i = 1; i < grp.nodes.size(); ++i) {
       const Node& nd = g.nodes[grp.nodes[i]];
-      f << "    const float e" << grp.nodes[i] << " = hct_" << nd.op << "(";
-      for (size_t a = 0; a < nd.args.size(); ++a) f << (a ? ", " : "") << ref(nd.args[a]);
-      f << ");  // " << nd.name << "\n";
+      std::vector<std::string> av;
+      for (auto& a : nd.args) av.push_back(ref(a));
+      f << "    const float e" << grp.nodes[i] << " = " << elementwise_call(nd, av, "off0 + j * plane") << ";  // " << nd.name << "\n";
     }
     for (auto& st : grp.stores) {
       int pi = ptr_index(st.node, !st.to_output);

@@ -247,13 +247,14 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
     const bool reduces = nd.cls == OpClass::RowReduce || nd.cls == OpClass::RowSoftmax || nd.cls == OpClass::RowLayernorm;
     b << "      // " << nd.name << " = " << nd.op << "\n";
     if (nd.cls == OpClass::Unary || nd.cls == OpClass::Binary) {
-      std::string call = "hct_" + nd.op + "(";
+      std::vector<std::string> av;
       if (p.is_colv[ni]) {
-        for (size_t a = 0; a < nd.args.size(); ++a) call += (a ? ", " : "") + rg.ref(nd.args[a], false);
-        b << "      float s" << id << "[HCT_B];\n      " << FORB << "s" << id << "[b] = " << call << ");\n";
+        for (auto& a : nd.args) av.push_back(rg.ref(a, false));
+        b << "      float s" << id << "[HCT_B];\n      " << FORB << "s" << id << "[b] = " << elementwise_call(nd, av, "hct_row0 + b") << ";\n";
       } else {
-        for (size_t a = 0; a < nd.args.size(); ++a) call += (a ? ", " : "") + rg.ref(nd.args[a], true);
-        b << "      float v" << id << "[HCT_B][HCT_E];\n      " << FORB << FORE << "v" << id << "[b][e] = " << call << ");\n";
+        for (auto& a : nd.args) av.push_back(rg.ref(a, true));
+        b << "      float v" << id << "[HCT_B][HCT_E];\n      " << FORB << FORE << "v" << id << "[b][e] = "
+          << elementwise_call(nd, av, "(hct_row0 + b) * (long long)HCT_C + HCT_COL(e)") << ";\n";
       }
     } else if (nd.cls == OpClass::RowReduce) {
       std::string a = rg.ref(nd.args[0], true);

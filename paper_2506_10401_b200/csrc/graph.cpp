@@ -5,6 +5,8 @@
 
 #include <cctype>
 #include <cstdlib>
+#include <cmath>
+#include <cstdio>
 #include <map>
 #include <sstream>
 
@@ -224,7 +226,24 @@ Graph parse_spec(const std::string& text) {
       n.name = name;
       n.op = op;
       n.dtype = F32;
-      if (is_unary(op)) {
+      if (op == "dropout") {
+        // Inverted dropout with a counter-based mask (the hash generator of the paper's first case study):
+        // h = i + seed; h ^= h >> 17; h ^= h << 31; h ^= h >> 8 in 64-bit arithmetic, i the element's
+        // row-major offset; the element is kept, scaled by 1/(1-p), when h mod 1000 >= round(1000 p).
+        only_attrs({"p", "seed"});
+        if (pos.size() != 1) fail(HCT_ERR_GRAPH, line, "dropout takes one operand");
+        n.cls = OpClass::Unary;
+        n.args = {lookup(pos[0], line, false)};
+        n.shape = g.nodes[n.args[0].node].shape;
+        n.drop_p = 0.5;
+        if (attrs.count("p") && (!parse_number(attrs["p"], &n.drop_p) || !(n.drop_p >= 0.0 && n.drop_p < 1.0)))
+          fail(HCT_ERR_PARSE, line, "p must be a number in [0,1)");
+        int64_t seed = 0;
+        if (attrs.count("seed") && (!parse_int(attrs["seed"], &seed) || seed < 0)) fail(HCT_ERR_PARSE, line, "seed must be a non-negative integer");
+        n.drop_seed = (uint64_t)seed;
+        n.drop_threshold = (unsigned)std::llround(n.drop_p * 1000.0);
+        if (n.drop_threshold >= 1000) fail(HCT_ERR_PARSE, line, "p rounds to 1: nothing would be kept");
+      } else if (is_unary(op)) {
         only_attrs({});
         if (pos.size() != 1) fail(HCT_ERR_GRAPH, line, op + " takes one operand");
         n.cls = OpClass::Unary;
@@ -249,7 +268,9 @@ Graph parse_spec(const std::string& text) {
         n.cls = op == "row_softmax" ? OpClass::RowSoftmax : OpClass::RowReduce;
         n.args = {lookup(pos[0], line, false)};
         auto& s = g.nodes[n.args[0].node].shape;
-        if (s.size() != 2 || s[1] < 2) fail(HCT_ERR_GRAPH, line, op + " needs a [R,C] operand with C >= 2, got " + shape_str(s));
+        // a softmax over a single column is legal (and identically one); the reductions need two columns
+        if (s.size() != 2 || s[1] < (op == "row_softmax" ? 1 : 2))
+          fail(HCT_ERR_GRAPH, line, op + " needs a [R,C] operand with C >= " + (op == "row_softmax" ? "1" : "2") + ", got " + shape_str(s));
         n.shape = s;
         if (n.cls == OpClass::RowReduce) n.shape[1] = 1;
       } else if (op == "row_layernorm") {
@@ -341,6 +362,18 @@ Graph parse_spec(const std::string& text) {
   for (auto& n : g.nodes)
     if (n.numel() == 0) throw Error(HCT_ERR_UNSUPPORTED, "tensor '" + n.name + "' is empty");
   return g;
+}
+
+std::string elementwise_call(const Node& nd, const std::vector<std::string>& args, const std::string& flat_index) {
+  std::string c = "hct_" + nd.op + "(";
+  for (size_t i = 0; i < args.size(); ++i) c += (i ? ", " : "") + args[i];
+  if (nd.op == "dropout") {
+    char scale[32];
+    std::snprintf(scale, sizeof scale, "%.9ef", (double)(float)(1.0 / (1.0 - nd.drop_p)));
+    c += ", (unsigned long long)(" + flat_index + "), " + std::to_string((unsigned long long)nd.drop_seed) + "ULL, " +
+         std::to_string(nd.drop_threshold) + "u, " + scale;
+  }
+  return c + ")";
 }
 
 }  // namespace hct

@@ -31,6 +31,10 @@ struct Node {
   DType dtype = F32;  // storage dtype of an input; computed nodes are fp32 values
   double eps = 1e-5;
   int stride = 1, pad = 0;
+  // dropout: element with flat index i is kept when hash(i + seed) mod 1000 >= drop_threshold (= round(1000 p))
+  double drop_p = 0.0;
+  uint64_t drop_seed = 0;
+  unsigned drop_threshold = 0;
   int input_index = -1;   // position among `input` lines
   int output_index = -1;  // position among `output` lines
   DType out_dtype = F32;  // storage dtype when the node is a graph output
@@ -52,5 +56,9 @@ Graph parse_spec(const std::string& text);
 
 bool is_unary(const std::string& op);
 bool is_binary(const std::string& op);
+
+// Source text of the call that evaluates elementwise node `nd` on the operand expressions `args`;
+// `flat_index` is an expression for the element's row-major offset in the node's tensor (used by dropout).
+std::string elementwise_call(const Node& nd, const std::vector<std::string>& args, const std::string& flat_index);
 
 }  // namespace hct

@@ -49,7 +49,7 @@ def test_error_codes():
     assert _code("hct 1\ninput x f32 [4,8]\ninput u f32 [4,8]\nnode y = relu(x)\noutput y\n") == g
     assert _code("hct 1\ninput x f32 [4,8]\nnode y = frobnicate(x)\noutput y\n") == g
     assert _code("hct 1\ninput x f32 [4,8]\nnode y = relu(x)\nnode y = exp(x)\noutput y\n") == g
-    assert _code("hct 1\ninput x f32 [4,8]\nnode s = row_sum(x)\nnode y = row_softmax(s)\noutput y\n") == g
+    assert _code("hct 1\ninput x f32 [4,8]\nnode s = row_sum(x)\nnode y = row_max(s)\noutput y\n") == g
     assert _code("hct 1\ninput x f32 [4,8]\nnode y = relu(x)\n") == g
     assert _code("hct 1\ninput x f32 [4,8]\noutput x\n") == g
     assert _code("hct 1\ninput x f32 [0,8]\nnode y = relu(x)\noutput y\n") == hct.HCT_ERR_UNSUPPORTED

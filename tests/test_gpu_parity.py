@@ -172,6 +172,54 @@ def test_conv_bf16_nchw_direct_integer_inputs_are_exact():
     np.testing.assert_array_equal(got[0], want[0])
 
 
+# ------------------------------------------------------------------ dropout (counter-based mask)
+
+def _mask_is_exact(got, want):
+    """The mask is integer work: dropped elements are exactly zero on both sides, in the same places."""
+    np.testing.assert_array_equal(got == 0.0, want == 0.0)
+
+
+@pytest.mark.parametrize("r,c,p,seed", [(37, 1000, 0.3, 5), (300, 4096, 0.5, 123456789), (5, 1023, 0.0, 1), (3, 65536, 0.9, (1 << 40) + 7),
+                                        (64, 130, 0.25, 0)])
+def test_dropout_in_row_chain(r, c, p, seed):
+    spec = f"hct 1\ninput x f32 [{r},{c}]\ninput b f32 [{c}]\nnode a = add(x, b)\nnode d = dropout(a, p={p}, seed={seed})\n" \
+           f"node s = row_sum(d)\nnode e = dropout(s, p=0.5, seed={seed + 1})\noutput d\noutput e\n"
+    n = {"kind": "normal", "mean": 0.5, "std": 1.0}
+    got, want, g = parity.run_both(spec, {"x": n, "b": n})
+    _mask_is_exact(got[0], want[0])
+    _mask_is_exact(got[1], want[1])
+    assert max(parity.f32_violation(a, b) for a, b in zip(got, want)) <= 1.0
+    assert g.num_kernels == 1
+
+
+def test_dropout_in_gemm_and_conv_epilogues():
+    spec = "hct 1\ninput x bf16 [300,264]\ninput w bf16 [264,520]\nnode t = gemm(x, w)\nnode d = dropout(t, p=0.4, seed=99)\noutput d f32\n"
+    got, want, g = parity.run_both(spec, {"x": {"kind": "normal", "mean": 0.0, "std": 1.0}, "w": {"kind": "normal", "mean": 0.0, "std": 0.06}})
+    assert "tcgen05" in g.plan and g.num_kernels == 1
+    _mask_is_exact(got[0], want[0])
+    assert parity.bf16_violation(got[0], want[0]) <= 1.0
+    spec = "hct 1\ninput x bf16 [2,64,20,24]\ninput w bf16 [96,64,3,3]\nnode t = conv2d(x, w, stride=1, pad=1)\nnode d = dropout(t, p=0.3, seed=7)\noutput d bf16\n"
+    got, want, g = parity.run_both(spec, {"x": {"kind": "normal", "mean": 0.0, "std": 1.0}, "w": {"kind": "normal", "mean": 0.0, "std": 0.04}})
+    assert "tcgen05" in g.plan
+    _mask_is_exact(got[0], want[0])
+    assert parity.bf16_violation(got[0], want[0]) <= 1.0
+    spec = "hct 1\ninput x f32 [1,8,12,10]\ninput w f32 [4,8,3,3]\nnode t = conv2d(x, w, stride=2, pad=1)\nnode d = dropout(t, p=0.3, seed=7)\noutput d\n"
+    il = {"kind": "int", "lo": -4, "hi": 4}
+    got, want, g = parity.run_both(spec, {"x": il, "w": il})
+    _mask_is_exact(got[0], want[0])
+    assert parity.f32_violation(got[0], want[0]) <= 1.0
+
+
+@pytest.mark.parametrize("m,k,n", [(200, 320, 264), (1024, 512, 1024)])
+def test_case_study_chain_matmul_dropout_mean_softmax(m, k, n):
+    spec, laws = configs.get_config("matmul_dropout_mean_softmax", m=m, k=k, n=n)
+    got, want, g = parity.run_both(spec, laws)
+    np.testing.assert_array_equal(got[0], np.ones((m, 1)))      # softmax of one value per row
+    np.testing.assert_array_equal(want[0], np.ones((m, 1)))
+    assert parity.bf16_violation(got[1], want[1]) <= 1.0
+    assert parity.f32_violation(got[1], want[1], tol=2e-3) <= 1.0  # mean of bf16-input products: far inside the bf16 class
+
+
 # ------------------------------------------------------------------ multi-kernel graphs
 
 def test_gemm_between_row_kernels():

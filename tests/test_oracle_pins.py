@@ -330,7 +330,7 @@ def test_parse_good_and_shapes():
     "hct 1\ninput x f32 [4,8]\ninput u f32 [4,8]\nnode y = relu(x)\noutput y\n",    # unused input
     "hct 1\ninput x f32 [4,8]\nnode y = frobnicate(x)\noutput y\n",
     "hct 1\ninput x f32 [4,8]\nnode y = relu(x)\nnode y = exp(x)\noutput y\n",      # duplicate name
-    "hct 1\ninput x f32 [4,8]\nnode s = row_sum(x)\nnode y = row_softmax(s)\noutput y\n",  # row op on [R,1]
+    "hct 1\ninput x f32 [4,8]\nnode s = row_sum(x)\nnode y = row_max(s)\noutput y\n",  # row op on [R,1]
     "hct 1\ninput x f32 [4,8]\nnode y = relu(x)\n",                                 # no output
     "hct 1\ninput x f32 [4,8]\noutput x\n",
     "hct 1\ninput x f32 [4,8]\nnode y = relu(x, x)\noutput y\n",
@@ -339,6 +339,69 @@ def test_parse_good_and_shapes():
 def test_parse_rejects(bad):
     with pytest.raises(oracle.SpecError):
         oracle.parse(bad)
+
+
+# ---------------------------------------------------------------- dropout (counter-based mask)
+
+_M64 = (1 << 64) - 1
+
+
+def _hash_int(v):
+    """The generator's steps on Python integers (arbitrary precision, masked to 64 bits by hand)."""
+    h = v & _M64
+    h ^= h >> 17
+    h ^= (h << 31) & _M64
+    h ^= h >> 8
+    return h
+
+
+def _golden_hash_rows():
+    rows = []
+    with open(os.path.join(HERE, "golden", "dropout_hash.txt")) as f:
+        for line in f:
+            line = line.split("#", 1)[0].split()
+            if line:
+                rows.append(tuple(int(t) for t in line))
+    return rows
+
+
+def test_dropout_hash_hand_values():
+    # the integer steps reproduce the hand-derived values, and the oracle's mask agrees with them
+    for start, h, r in _golden_hash_rows():
+        assert _hash_int(start) == h and h % 1000 == r
+        for thr in (0, r, r + 1):
+            if thr >= 1000:
+                continue
+            keep = interp.dropout_keep_mask((1,), start, thr / 1000.0)[0]
+            assert bool(keep) == (r >= thr)
+
+
+def test_dropout_mask_bruteforce_including_wraparound():
+    # offsets and seeds beyond 2^31 and up to 2^63: the shift by 31 must wrap modulo 2^64
+    for seed, shape, p in [(0, (5, 7), 0.3), (12345, (3, 4, 5), 0.5), ((1 << 33) + 5, (9,), 0.25), ((1 << 63) - 4, (2, 6), 0.9), (77, (1, 1), 0.0)]:
+        got = interp.dropout_keep_mask(shape, seed, p)
+        want = np.array([_hash_int(i + seed) % 1000 >= round(1000 * p) for i in range(int(np.prod(shape)))]).reshape(shape)
+        np.testing.assert_array_equal(got, want)
+
+
+def test_dropout_closed_forms():
+    x = RNG.normal(size=(200, 500))
+    np.testing.assert_array_equal(interp.dropout(x, 0.0, 9), x)            # p = 0 keeps everything, unscaled
+    y = interp.dropout(x, 0.2, 9)
+    kept = y != 0.0
+    np.testing.assert_allclose(y[kept], x[kept] / 0.8, rtol=1e-15)
+    np.testing.assert_array_equal(kept, interp.dropout_keep_mask(x.shape, 9, 0.2))   # mask does not depend on x
+    assert abs(kept.mean() - 0.8) < 0.01
+    # a row-major reshape moves no element's offset: same mask
+    np.testing.assert_array_equal(interp.dropout_keep_mask((100, 1000), 9, 0.2).ravel(), interp.dropout_keep_mask((100000,), 9, 0.2))
+    # through the interpreter, in the case-study chain: the closing softmax of one value per row is one
+    spec = "hct 1\ninput a f32 [6,8]\ninput b f32 [8,10]\nnode t = gemm(a, b)\nnode d = dropout(t, p=0.3, seed=5)\nnode m = row_mean(d)\nnode s = row_softmax(m)\noutput s\noutput m\n"
+    a, b = RNG.normal(size=(6, 8)), RNG.normal(size=(8, 10))
+    out = oracle.run(spec, {"a": a, "b": b})
+    np.testing.assert_array_equal(out["s"], np.ones((6, 1)))
+    t = a @ b
+    want = np.array([[sum(t[i, j] / 0.7 for j in range(10) if _hash_int(i * 10 + j + 5) % 1000 >= 300) / 10] for i in range(6)])
+    np.testing.assert_allclose(out["m"], want, rtol=1e-13)
 
 
 # ---------------------------------------------------------------- planted mistakes must be caught
@@ -391,6 +454,22 @@ def test_planted_mistakes_are_detected(monkeypatch):
         monkeypatch.setattr(interp, name, wrong)
         assert fails(check), f"planted mistake in {name} ({wrong.__name__}) was not detected"
         monkeypatch.setattr(interp, name, orig[name])
+        check()
+    def mask_32bit(shape, seed, p):   # the shift by 31 truncated to 32 bits
+        n = int(np.prod(shape))
+        h = (np.arange(n, dtype=np.uint64) + np.uint64(seed))
+        h ^= h >> np.uint64(17)
+        h ^= (h << np.uint64(31)) & np.uint64(0xffffffff)
+        h ^= h >> np.uint64(8)
+        return ((h % np.uint64(1000)) >= np.uint64(round(p * 1000.0))).reshape(shape)
+
+    def mask_strict(shape, seed, p):  # keeps only variates strictly above p
+        return orig["dropout_keep_mask"](shape, seed, p) & (orig["dropout_keep_mask"](shape, seed, min(p + 0.001, 0.999)) | (p >= 0.999))
+
+    for wrong, check in [(mask_32bit, test_dropout_hash_hand_values), (mask_strict, test_dropout_closed_forms)]:
+        monkeypatch.setattr(interp, "dropout_keep_mask", wrong)
+        assert fails(check), f"planted mistake {wrong.__name__} was not detected"
+        monkeypatch.setattr(interp, "dropout_keep_mask", orig["dropout_keep_mask"])
         check()
     monkeypatch.setattr(interp, "row_softmax", softmax_no_max)
     with np.errstate(over="ignore", invalid="ignore"):

@@ -85,11 +85,31 @@ output t3 bf16
     return spec, laws
 
 
+def matmul_dropout_mean_softmax(m=8192, k=4096, n=4096, p=0.2, seed=2024):
+    """The fused group of the paper's first case study: matrix product, dropout, mean, softmax.
+
+    The mean leaves one value per row, so the closing softmax is identically one; the mean is a second
+    output so that the chain's arithmetic (product, mask, scaling, reduction) can be compared."""
+    spec = f"""hct 1
+input x bf16 [{m},{k}]
+input w bf16 [{k},{n}]
+node  t0 = gemm(x, w)
+node  t1 = dropout(t0, p={p}, seed={seed})
+node  t2 = row_mean(t1)
+node  t3 = row_softmax(t2)
+output t3 f32
+output t2 f32
+"""
+    laws = {"x": _n(), "w": _n(1.0 / math.sqrt(k))}
+    return spec, laws
+
+
 CONFIGS = {
     "c1_gemm_bias_relu_f32": (gemm_bias_relu, {}),
     "c2_softmax_layernorm_chain": (softmax_layernorm_chain, {}),
     "c3_gemm_bf16_gelu_residual": (gemm_bf16_gelu_residual, {}),
     "c4_conv_bn_relu_bf16": (conv_bn_relu, {}),
+    "matmul_dropout_mean_softmax": (matmul_dropout_mean_softmax, {}),
 }
 
 
