@@ -111,6 +111,35 @@ HCT_API hct_status_t hct_graph_run(hct_graph_t* g, const void* const* inputs, in
                            int n_outputs, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * hct_graph_create with a schedule: `schedule` is NULL (defaults) or text of the form
+ * "knob=integer;knob=integer" that overrides launch-shape knobs of the generated kernels
+ * (threads per row, vectors per thread, CTAs per SM, ring sizes, which convolution schedule;
+ * the knob names are those printed by hct_graph_schedule after a tuning run).  Results do not
+ * depend on the schedule beyond rounding order.  An unknown knob gives HCT_ERR_INVALID_ARG.
+ */
+HCT_API hct_status_t hct_graph_create_scheduled(const char* spec, size_t spec_len, int device, const char* schedule,
+                                                hct_graph_t** out);
+
+/*
+ * Measure-and-pick: builds the graph under up to max_trials candidate schedules, runs each on
+ * the caller's buffers (same arguments as hct_graph_run; all DEVICE pointers, caller-owned,
+ * outputs are overwritten), times it with events on `cuda_stream`, and returns the fastest
+ * handle in *out.  This is the role the measurement trials of the auto-scheduler play in the
+ * paper's pipeline (Section 3.5: every candidate is compiled and executed on the device, the
+ * best one is kept), restricted to this library's own knobs.  The call SYNCHRONISES the stream
+ * repeatedly and is meant for set-up time.  Candidates that need more workspace than
+ * workspace_bytes, do not apply to the graph or fail to build are skipped; the default
+ * schedule is always measured, so a handle is returned whenever hct_graph_create would succeed
+ * and the buffers fit.  Errors as for hct_graph_create / hct_graph_run.
+ */
+HCT_API hct_status_t hct_graph_autotune(const char* spec, size_t spec_len, int device, const void* const* inputs, int n_inputs,
+                                        void* const* outputs, int n_outputs, void* workspace, size_t workspace_bytes,
+                                        void* cuda_stream, int max_trials, hct_graph_t** out);
+
+/* The schedule text a handle was built with ("" for the defaults); owned by the handle. */
+HCT_API const char* hct_graph_schedule(const hct_graph_t* g);
+
+/*
  * After the caller has synchronised the stream: reads the handle's device
  * status word.  HCT_OK, or HCT_ERR_TIMEOUT if a kernel gave up on a bounded
  * wait (its outputs are then undefined).  Clears the word.

@@ -17,7 +17,7 @@ EXPORTS = [
     "hct_graph_create", "hct_graph_run", "hct_graph_status", "hct_graph_destroy", "hct_graph_num_inputs",
     "hct_graph_num_outputs", "hct_graph_tensor_info", "hct_graph_workspace_bytes", "hct_graph_num_kernels",
     "hct_graph_cost", "hct_graph_plan_text", "hct_graph_kernel_source", "hct_graph_kernel_name", "hct_last_error",
-    "hct_version", "hct_gemm_bias_relu_f32_static",
+    "hct_version", "hct_gemm_bias_relu_f32_static", "hct_graph_create_scheduled", "hct_graph_autotune", "hct_graph_schedule",
 ]
 
 HCT_STATIC_SCRATCH_BYTES = 8 << 20
@@ -74,6 +74,12 @@ def lib() -> ctypes.CDLL:
         L.hct_gemm_bias_relu_f32_static.restype = ci
         L.hct_version.argtypes = []
         L.hct_version.restype = cp
+        L.hct_graph_create_scheduled.argtypes = [cp, sz, ci, cp, ctypes.POINTER(vp)]
+        L.hct_graph_create_scheduled.restype = ci
+        L.hct_graph_autotune.argtypes = [cp, sz, ci, ctypes.POINTER(vp), ci, ctypes.POINTER(vp), ci, vp, sz, vp, ci, ctypes.POINTER(vp)]
+        L.hct_graph_autotune.restype = ci
+        L.hct_graph_schedule.argtypes = [vp]
+        L.hct_graph_schedule.restype = cp
         _lib = L
     return _lib
 
@@ -92,6 +98,30 @@ def hct_graph_create(spec: str, device: int = 0) -> ctypes.c_void_p:
     out = ctypes.c_void_p()
     _check(lib().hct_graph_create(raw, len(raw), device, ctypes.byref(out)))
     return out
+
+
+def hct_graph_create_scheduled(spec: str, device: int = 0, schedule: str | None = None) -> ctypes.c_void_p:
+    raw = spec.encode()
+    out = ctypes.c_void_p()
+    _check(lib().hct_graph_create_scheduled(raw, len(raw), device, None if schedule is None else schedule.encode(), ctypes.byref(out)))
+    return out
+
+
+def hct_graph_autotune(spec: str, device: int, inputs, outputs, workspace: int = 0, workspace_bytes: int = 0, cuda_stream: int = 0,
+                       max_trials: int = 16) -> ctypes.c_void_p:
+    """inputs / outputs: device addresses as for hct_graph_run.  Returns the fastest handle."""
+    raw = spec.encode()
+    n_in, n_out = len(inputs), len(outputs)
+    a_in = (ctypes.c_void_p * max(n_in, 1))(*inputs)
+    a_out = (ctypes.c_void_p * max(n_out, 1))(*outputs)
+    out = ctypes.c_void_p()
+    _check(lib().hct_graph_autotune(raw, len(raw), device, a_in, n_in, a_out, n_out, workspace, workspace_bytes, cuda_stream,
+                                    max_trials, ctypes.byref(out)))
+    return out
+
+
+def hct_graph_schedule(g) -> str:
+    return lib().hct_graph_schedule(g).decode()
 
 
 def hct_graph_run(g, inputs, outputs, workspace: int = 0, workspace_bytes: int = 0, cuda_stream: int = 0):

@@ -1,5 +1,6 @@
 // C ABI: graph handle life cycle, launches and queries.
 #include <cstdlib>
+#include <algorithm>
 #include <cstring>
 #include <memory>
 #include <sstream>
@@ -60,6 +61,7 @@ struct hct_graph {
   CUcontext_t ctx = nullptr;
   CUdevice_t cudev = 0;
   CUdeviceptr_t status_word = 0;
+  std::string schedule;  // knob=value;... this handle was built with (empty: defaults)
   std::string plan_text;
 };
 
@@ -91,6 +93,10 @@ const char* hct_last_error(void) { return g_last_error.c_str(); }
 const char* hct_version(void) { return "hct 0.1 (sm_100a)"; }
 
 hct_status_t hct_graph_create(const char* spec, size_t spec_len, int device, hct_graph_t** out) {
+  return hct_graph_create_scheduled(spec, spec_len, device, nullptr, out);
+}
+
+hct_status_t hct_graph_create_scheduled(const char* spec, size_t spec_len, int device, const char* schedule, hct_graph_t** out) {
   if (out) *out = nullptr;
   if (!spec || !out) return set_error(HCT_ERR_INVALID_ARG, "spec and out must not be NULL");
   std::unique_ptr<hct_graph> h(new (std::nothrow) hct_graph);
@@ -99,6 +105,10 @@ hct_status_t hct_graph_create(const char* spec, size_t spec_len, int device, hct
     h->graph = parse_spec(std::string(spec, spec_len));
     h->plan = make_plan(h->graph);
     Tunables tun = Tunables::from_env();
+    if (schedule) {
+      tun.apply_text(schedule);
+      h->schedule = schedule;
+    }
     std::vector<KernelSpec> specs;
     std::vector<int> spec_group;
     for (size_t gi = 0; gi < h->plan.groups.size(); ++gi) {
@@ -284,6 +294,100 @@ hct_status_t hct_graph_status(hct_graph_t* g) {
   }
   return HCT_OK;
 }
+
+// Measure-and-pick over launch shapes: the role the auto-scheduler's measurement trials play in the
+// paper's pipeline (Section 3.5), restricted to the knobs of this library's hand-written kernels.
+hct_status_t hct_graph_autotune(const char* spec, size_t spec_len, int device, const void* const* inputs, int n_inputs,
+                                void* const* outputs, int n_outputs, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                                int max_trials, hct_graph_t** out) {
+  if (out) *out = nullptr;
+  if (!spec || !out) return set_error(HCT_ERR_INVALID_ARG, "spec and out must not be NULL");
+  if (device == HCT_DEVICE_NONE) return set_error(HCT_ERR_INVALID_ARG, "autotuning needs a device");
+  if (max_trials < 1) max_trials = 1;
+  hct_graph_t* best = nullptr;
+  hct_status_t rc = hct_graph_create_scheduled(spec, spec_len, device, "", &best);   // the default shape is always a candidate
+  if (rc != HCT_OK) return rc;
+  bool has_row = false, has_conv = false;
+  for (auto& grp : best->plan.groups) {
+    has_row = has_row || grp.kind == GroupKind::Row;
+    has_conv = has_conv || grp.kind == GroupKind::Conv;
+  }
+  std::vector<std::string> cands;
+  if (has_row)
+    for (const char* c : {"row_cta_small=512", "row_nv=2", "row_cta_small=128", "row_nv=8", "row_minb=2", "row_no_small_ctas=1", "row_b=2",
+                          "row_nv=2;row_cta_small=512", "row_ring_bytes_small=98304", "row_cta_elementwise=256", "row_cta_elementwise=1024",
+                          "row_nv=8;row_cta_small=128", "row_no_stage=1", "row_nv=2;row_minb=2"})
+      cands.push_back(c);
+  if (has_conv)
+    for (const char* c : {"conv_no_tma_store=1", "conv_no_direct=1", "conv_no_direct=1;conv_no_halo=1"}) cands.push_back(c);
+
+  const Driver* d = nullptr;
+  CUevent_t e0 = nullptr, e1 = nullptr;
+  // median time of a few runs, in ms; negative when the candidate cannot run with the caller's buffers
+  auto measure = [&](hct_graph_t* g) -> float {
+    if (g->workspace_bytes > workspace_bytes) return -1.0f;
+    CtxGuard guard(*d, g->ctx);
+    float t[5];
+    for (int i = -2; i < 5; ++i) {
+      if (i >= 0) d->EventRecord(e0, (CUstream_t)cuda_stream);
+      if (hct_graph_run(g, inputs, n_inputs, outputs, n_outputs, workspace, workspace_bytes, cuda_stream) != HCT_OK) return -1.0f;
+      if (i >= 0) {
+        d->EventRecord(e1, (CUstream_t)cuda_stream);
+        if (d->EventSynchronize(e1) != 0 || d->EventElapsedTime(&t[i], e0, e1) != 0) return -1.0f;
+      }
+    }
+    if (hct_graph_status(g) != HCT_OK) return -1.0f;
+    std::sort(t, t + 5);
+    return t[2];
+  };
+  auto drop_events = [&]() {
+    CtxGuard guard(*d, best->ctx);
+    if (e0) d->EventDestroy(e0);
+    if (e1) d->EventDestroy(e1);
+  };
+  try {
+    d = &driver();
+    {
+      CtxGuard guard(*d, best->ctx);
+      if (d->EventCreate(&e0, 0) != 0 || d->EventCreate(&e1, 0) != 0) throw Error(HCT_ERR_CUDA, "cuEventCreate failed");
+    }
+    float best_ms = measure(best);
+    if (best_ms < 0.0f) {
+      std::string why = hct_last_error();
+      drop_events();
+      hct_graph_destroy(best);
+      return set_error(HCT_ERR_INVALID_ARG, "the default schedule cannot run with these buffers: " + why);
+    }
+    int trials = 1;
+    for (size_t c = 0; c < cands.size() && trials < max_trials; ++c) {
+      hct_graph_t* g = nullptr;
+      if (hct_graph_create_scheduled(spec, spec_len, device, cands[c].c_str(), &g) != HCT_OK) continue;   // shape not applicable
+      bool same = g->kernels.size() == best->kernels.size();
+      for (size_t k = 0; same && k < g->kernels.size(); ++k) same = g->kernels[k].spec.source == best->kernels[k].spec.source;
+      if (same) {  // the knob does not touch this graph: nothing to measure
+        hct_graph_destroy(g);
+        continue;
+      }
+      ++trials;
+      float ms = measure(g);
+      if (ms >= 0.0f && ms < best_ms) {
+        hct_graph_destroy(best);
+        best = g;
+        best_ms = ms;
+      } else {
+        hct_graph_destroy(g);
+      }
+    }
+    drop_events();
+  } catch (const Error& e) {
+    hct_graph_destroy(best);
+    return set_error(e.code, e.what());
+  }
+  *out = best;
+  return HCT_OK;
+}
+
+const char* hct_graph_schedule(const hct_graph_t* g) { return g ? g->schedule.c_str() : ""; }
 
 hct_status_t hct_graph_destroy(hct_graph_t* g) {
   if (!g) return HCT_OK;

@@ -64,6 +64,10 @@ struct Tunables {
   bool fault_never_arrive = false;
   unsigned wait_limit = 0;  // 0: kernel default  // keep contractions on the fp32 FMA kernels (for debugging tensor-core paths)
   static Tunables from_env();
+  // Sets one knob by its schedule name; false when the name is unknown or the value is not an integer.
+  bool set(const std::string& key, const std::string& value);
+  // Applies "knob=integer;knob=integer" on top of *this; throws Error(HCT_ERR_INVALID_ARG) on an unknown knob or bad value.
+  void apply_text(const std::string& text);
 };
 
 // Extra workspace a group's kernels need beyond the planner's intermediates is appended to

@@ -1,4 +1,5 @@
 // Generator for fused row kernels: elementwise, broadcast and row-reduction chains over one [R,C] space.
+#include <cctype>
 #include <cstdio>
 #include <cstdlib>
 #include <sstream>
@@ -8,28 +9,82 @@
 
 namespace hct {
 
+namespace {
+struct Knob {
+  const char* key;    // schedule name; the environment variable is HCT_ + upper case
+  int Tunables::*i;   // integer knob (with its lower bound), or
+  int lo;
+  bool Tunables::*b;  // boolean knob
+};
+const Knob kKnobs[] = {
+    {"row_nv", &Tunables::row_nv, 1, nullptr},
+    {"row_cta", &Tunables::row_cta, 32, nullptr},
+    {"row_b", &Tunables::row_batch, 1, nullptr},
+    {"row_cta_batched", &Tunables::row_cta_batched, 32, nullptr},
+    {"row_cta_elementwise", &Tunables::row_cta_elementwise, 32, nullptr},
+    {"row_cta_staged", &Tunables::row_cta_staged, 32, nullptr},
+    {"row_minb", &Tunables::row_min_blocks, 1, nullptr},
+    {"row_cta_small", &Tunables::row_cta_small, 32, nullptr},
+    {"row_ring_bytes_small", &Tunables::row_ring_bytes_small, 1024, nullptr},
+    {"row_ring_bytes", &Tunables::row_ring_bytes, 1024, nullptr},
+    {"simt_only", nullptr, 0, &Tunables::simt_only},
+    {"fault_never_arrive", nullptr, 0, &Tunables::fault_never_arrive},
+    {"conv_no_halo", nullptr, 0, &Tunables::conv_no_halo},
+    {"conv_no_tma_store", nullptr, 0, &Tunables::conv_no_tma_store},
+    {"conv_no_direct", nullptr, 0, &Tunables::conv_no_direct},
+    {"row_no_small_ctas", nullptr, 0, &Tunables::row_no_small_ctas},
+    {"row_no_reg_rowvec", nullptr, 0, &Tunables::row_no_reg_rowvec},
+    {"row_no_softmax_ln_fusion", nullptr, 0, &Tunables::row_no_softmax_ln_fusion},
+    {"row_no_stage", nullptr, 0, &Tunables::row_no_stage},
+};
+}  // namespace
+
+bool Tunables::set(const std::string& key, const std::string& value) {
+  char* end = nullptr;
+  long v = std::strtol(value.c_str(), &end, 10);
+  if (value.empty() || *end != '\0') return false;
+  if (key == "wait_limit") {
+    wait_limit = (unsigned)std::max(1L, v);
+    return true;
+  }
+  for (const Knob& k : kKnobs)
+    if (key == k.key) {
+      if (k.i)
+        this->*(k.i) = (int)std::max<long>(k.lo, v);
+      else
+        this->*(k.b) = v != 0;
+      return true;
+    }
+  return false;
+}
+
+void Tunables::apply_text(const std::string& text) {
+  size_t pos = 0;
+  while (pos < text.size()) {
+    size_t semi = text.find(';', pos);
+    if (semi == std::string::npos) semi = text.size();
+    std::string item = text.substr(pos, semi - pos);
+    pos = semi + 1;
+    std::string packed;
+    for (char c : item)
+      if (c != ' ' && c != '\t' && c != '\n') packed += c;
+    if (packed.empty()) continue;
+    size_t eq = packed.find('=');
+    if (eq == std::string::npos || !set(packed.substr(0, eq), packed.substr(eq + 1)))
+      throw Error(HCT_ERR_INVALID_ARG, "schedule item '" + item + "' is not a known knob=integer");
+  }
+}
+
 Tunables Tunables::from_env() {
   Tunables t;
-  if (const char* s = std::getenv("HCT_ROW_NV")) t.row_nv = std::max(1, std::atoi(s));
-  if (const char* s = std::getenv("HCT_ROW_CTA")) t.row_cta = std::max(32, std::atoi(s));
-  if (const char* s = std::getenv("HCT_SIMT_ONLY")) t.simt_only = std::atoi(s) != 0;
-  if (const char* s = std::getenv("HCT_ROW_B")) t.row_batch = std::max(1, std::atoi(s));
-  if (const char* s = std::getenv("HCT_ROW_CTA_BATCHED")) t.row_cta_batched = std::max(32, std::atoi(s));
-  if (const char* s = std::getenv("HCT_ROW_CTA_ELEMENTWISE")) t.row_cta_elementwise = std::max(32, std::atoi(s));
-  if (const char* s = std::getenv("HCT_ROW_CTA_STAGED")) t.row_cta_staged = std::max(32, std::atoi(s));
-  if (const char* s = std::getenv("HCT_FAULT_NEVER_ARRIVE")) t.fault_never_arrive = std::atoi(s) != 0;
-  if (const char* s = std::getenv("HCT_WAIT_LIMIT")) t.wait_limit = (unsigned)std::max(1, std::atoi(s));
-  if (const char* s = std::getenv("HCT_CONV_NO_HALO")) t.conv_no_halo = std::atoi(s) != 0;
-  if (const char* s = std::getenv("HCT_CONV_NO_TMA_STORE")) t.conv_no_tma_store = std::atoi(s) != 0;
-  if (const char* s = std::getenv("HCT_CONV_NO_DIRECT")) t.conv_no_direct = std::atoi(s) != 0;
-  if (const char* s = std::getenv("HCT_ROW_MINB")) t.row_min_blocks = std::max(1, std::atoi(s));
-  if (const char* s = std::getenv("HCT_ROW_NO_SMALL_CTAS")) t.row_no_small_ctas = std::atoi(s) != 0;
-  if (const char* s = std::getenv("HCT_ROW_CTA_SMALL")) t.row_cta_small = std::max(32, std::atoi(s));
-  if (const char* s = std::getenv("HCT_ROW_RING_BYTES_SMALL")) t.row_ring_bytes_small = std::max(1024, std::atoi(s));
-  if (const char* s = std::getenv("HCT_ROW_NO_REG_ROWVEC")) t.row_no_reg_rowvec = std::atoi(s) != 0;
-  if (const char* s = std::getenv("HCT_ROW_NO_SOFTMAX_LN_FUSION")) t.row_no_softmax_ln_fusion = std::atoi(s) != 0;
-  if (const char* s = std::getenv("HCT_ROW_NO_STAGE")) t.row_no_stage = std::atoi(s) != 0;
-  if (const char* s = std::getenv("HCT_ROW_RING_BYTES")) t.row_ring_bytes = std::max(1024, std::atoi(s));
+  auto env_of = [](const char* key) {
+    std::string name = "HCT_";
+    for (const char* c = key; *c; ++c) name += (char)std::toupper((unsigned char)*c);
+    return std::getenv(name.c_str());
+  };
+  for (const Knob& k : kKnobs)
+    if (const char* s = env_of(k.key)) t.set(k.key, s);
+  if (const char* s = env_of("wait_limit")) t.set("wait_limit", s);
   return t;
 }
 

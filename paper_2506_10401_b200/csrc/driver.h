@@ -12,6 +12,7 @@ typedef struct CUctx_st* CUcontext_t;
 typedef struct CUmod_st* CUmodule_t;
 typedef struct CUfunc_st* CUfunction_t;
 typedef struct CUstream_st* CUstream_t;
+typedef struct CUevent_st* CUevent_t;
 typedef unsigned long long CUdeviceptr_t;
 
 struct alignas(64) TensorMap {
@@ -64,6 +65,11 @@ struct Driver {
   CUresult_t (*MemFree)(CUdeviceptr_t);
   CUresult_t (*MemcpyDtoH)(void*, CUdeviceptr_t, size_t);
   CUresult_t (*MemsetD8)(CUdeviceptr_t, unsigned char, size_t);
+  CUresult_t (*EventCreate)(CUevent_t*, unsigned);
+  CUresult_t (*EventRecord)(CUevent_t, CUstream_t);
+  CUresult_t (*EventSynchronize)(CUevent_t);
+  CUresult_t (*EventElapsedTime)(float*, CUevent_t, CUevent_t);
+  CUresult_t (*EventDestroy)(CUevent_t);
   // CUtensorMap*, dtype, rank, globalAddress, globalDim, globalStrides, boxDim, elementStrides, interleave, swizzle,
   // l2Promotion, oobFill
   CUresult_t (*TensorMapEncodeTiled)(TensorMap*, int, unsigned, void*, const uint64_t*, const uint64_t*, const uint32_t*,

@@ -133,6 +133,11 @@ const Driver& driver() {
     HCT_SYM(MemFree, "cuMemFree_v2")
     HCT_SYM(MemcpyDtoH, "cuMemcpyDtoH_v2")
     HCT_SYM(MemsetD8, "cuMemsetD8_v2")
+    HCT_SYM(EventCreate, "cuEventCreate")
+    HCT_SYM(EventRecord, "cuEventRecord")
+    HCT_SYM(EventSynchronize, "cuEventSynchronize")
+    HCT_SYM(EventElapsedTime, "cuEventElapsedTime")
+    HCT_SYM(EventDestroy, "cuEventDestroy_v2")
     HCT_SYM(TensorMapEncodeTiled, "cuTensorMapEncodeTiled")
 #undef HCT_SYM
     if (err.empty()) {

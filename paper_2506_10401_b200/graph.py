@@ -8,8 +8,8 @@ from . import binding as B
 
 
 class FusedGraph:
-    def __init__(self, spec: str, device: int = 0):
-        self.handle = B.hct_graph_create(spec, device)
+    def __init__(self, spec: str, device: int = 0, schedule: str | None = None, handle=None):
+        self.handle = handle if handle is not None else B.hct_graph_create_scheduled(spec, device, schedule)
         self.device = device
         self.n_in = B.hct_graph_num_inputs(self.handle)
         self.n_out = B.hct_graph_num_outputs(self.handle)
@@ -17,6 +17,26 @@ class FusedGraph:
         self.outputs = [B.hct_graph_tensor_info(self.handle, True, i) for i in range(self.n_out)]
         self.workspace_bytes = B.hct_graph_workspace_bytes(self.handle)
         self._ws = None
+
+    @classmethod
+    def autotuned(cls, spec: str, inputs, device: int = 0, max_trials: int = 16, workspace_bytes: int | None = None):
+        """Measures candidate schedules on `inputs` (torch CUDA tensors in spec order) and keeps the fastest.
+        Scratch outputs and a workspace are allocated here for the measurement (torch memory only)."""
+        import torch
+        probe = cls(spec, device)
+        outs = probe.alloc_outputs()
+        ws_bytes = workspace_bytes if workspace_bytes is not None else 2 * probe.workspace_bytes + (64 << 20)
+        ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device=f"cuda:{device}")
+        ws_ptr = (ws.data_ptr() + 255) // 256 * 256
+        stream = torch.cuda.current_stream(device).cuda_stream
+        probe.close()
+        h = B.hct_graph_autotune(spec, device, [t.data_ptr() for t in inputs], [t.data_ptr() for t in outs], ws_ptr, ws_bytes, stream,
+                                 max_trials)
+        return cls(spec, device, handle=h)
+
+    @property
+    def schedule(self) -> str:
+        return B.hct_graph_schedule(self.handle)
 
     # -- queries
     @property

@@ -150,3 +150,18 @@ def test_unsupported_broadcast_is_reported_not_emulated():
 
 def test_row_longer_than_the_limit_is_unsupported():
     assert _code("hct 1\ninput x f32 [2,131076]\nnode y = row_softmax(x)\noutput y\n") == hct.HCT_ERR_UNSUPPORTED
+
+
+def test_schedule_text_selects_launch_shapes_and_rejects_unknown_knobs():
+    B = binding
+    spec, _ = configs.get_config("c2_softmax_layernorm_chain", r=64, c=4096)
+    a = B.hct_graph_create_scheduled(spec, B.HCT_DEVICE_NONE, None)
+    b = B.hct_graph_create_scheduled(spec, B.HCT_DEVICE_NONE, "row_nv=2; row_cta_small=512")
+    assert B.hct_graph_schedule(a) == "" and B.hct_graph_schedule(b) == "row_nv=2; row_cta_small=512"
+    assert "#define HCT_T 256" in B.hct_graph_kernel_source(a, 0) and "#define HCT_T 512" in B.hct_graph_kernel_source(b, 0)
+    for bad in ("no_such_knob=1", "row_nv", "row_nv=four"):
+        with pytest.raises(B.HctError) as e:
+            B.hct_graph_create_scheduled(spec, B.HCT_DEVICE_NONE, bad)
+        assert e.value.code == B.HCT_ERR_INVALID_ARG
+    B.hct_graph_destroy(a)
+    B.hct_graph_destroy(b)

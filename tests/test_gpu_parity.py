@@ -220,6 +220,36 @@ def test_case_study_chain_matmul_dropout_mean_softmax(m, k, n):
     assert parity.f32_violation(got[1], want[1], tol=2e-3) <= 1.0  # mean of bf16-input products: far inside the bf16 class
 
 
+# ------------------------------------------------------------------ measure-and-pick over schedules
+
+def test_autotune_keeps_results_and_reports_its_choice():
+    import torch
+    import oracle
+    import paper_2506_10401_b200 as hct
+    spec, laws = configs.get_config("c2_softmax_layernorm_chain", r=2048, c=4096)
+    t = configs.draw_inputs(spec, laws, 0)
+    ins = parity.to_device(spec, t)
+    g = hct.FusedGraph.autotuned(spec, ins, max_trials=6)
+    outs = g.run(ins)
+    torch.cuda.synchronize()
+    g.status()
+    ref = oracle.run(spec, parity.oracle_inputs(spec, t))["t4"]
+    assert parity.f32_violation(parity.to_numpy64(outs[0]), ref) <= 1.0
+    # the chosen schedule can be replayed through the plain entry point and gives the same kernels
+    again = hct.FusedGraph(spec, 0, schedule=g.schedule)
+    assert again.kernel_source(0) == g.kernel_source(0)
+    # a convolution graph: the candidates include the other convolution schedules
+    spec, laws = configs.get_config("c4_conv_bn_relu_bf16", n=2, h=24, w=24)
+    t = configs.draw_inputs(spec, laws, 0)
+    ins = parity.to_device(spec, t)
+    g = hct.FusedGraph.autotuned(spec, ins, max_trials=4)
+    outs = g.run(ins)
+    torch.cuda.synchronize()
+    g.status()
+    ref = oracle.run(spec, parity.oracle_inputs(spec, t))["t3"]
+    assert parity.bf16_violation(parity.to_numpy64(outs[0]), ref) <= 1.0
+
+
 # ------------------------------------------------------------------ multi-kernel graphs
 
 def test_gemm_between_row_kernels():
