@@ -29,7 +29,8 @@
  *   binary  add sub mul div max min   operands broadcast like numpy; supported
  *           patterns: equal shapes, [C] against [..,C], [..,1] against [..,C],
  *           [K,1,1] against [N,K,H,W], a number
- *   row     row_softmax(x)  row_sum(x)  row_mean(x)  row_max(x)   x: [R,C]; sums give [R,1]
+ *   row     row_softmax(x)  row_sum(x)  row_mean(x)  row_max(x)  row_min(x)   x: [R,C]; reductions give [R,1]
+ *           row_argmax(x)  row_argmin(x)   column of the extreme element, the first among equals, as an fp32 value
  *           (row_softmax also accepts a single column, where it is identically one)
  *           row_layernorm(x, gamma, beta, eps=1e-5)   biased variance, eps inside the root
  *   gemm(a, b)            a[M,K] · b[K,N], both row-major, both f32 or both bf16 inputs;

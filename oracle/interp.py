@@ -86,6 +86,19 @@ def row_max(x):
     return x.max(axis=1, keepdims=True)
 
 
+def row_min(x):
+    return x.min(axis=1, keepdims=True)
+
+
+def row_argmax(x):
+    # column of the largest element of each row, the first one among equals (Table 1, "argmax"), as a float
+    return np.argmax(x, axis=1).reshape(-1, 1).astype(np.float64)
+
+
+def row_argmin(x):
+    return np.argmin(x, axis=1).reshape(-1, 1).astype(np.float64)
+
+
 def row_softmax(x):
     # y_ij = exp(x_ij - m_i) / sum_j exp(x_ij - m_i), m_i the row maximum
     e = np.exp(x - x.max(axis=1, keepdims=True))
@@ -168,6 +181,12 @@ def run_nodes(spec, inputs: dict, dtype=np.float64, gemm_fn=None) -> dict:
             out = row_mean(args[0])
         elif op == "row_max":
             out = row_max(args[0])
+        elif op == "row_min":
+            out = row_min(args[0])
+        elif op == "row_argmax":
+            out = row_argmax(args[0])
+        elif op == "row_argmin":
+            out = row_argmin(args[0])
         elif op == "row_layernorm":
             out = row_layernorm(args[0], args[1], args[2], node.attrs["eps"])
         elif op == "gemm":

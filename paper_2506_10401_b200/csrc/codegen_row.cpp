@@ -311,6 +311,24 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         b << "      float v" << id << "[HCT_B][HCT_E];\n      " << FORB << FORE << "v" << id << "[b][e] = "
           << elementwise_call(nd, av, "(hct_row0 + b) * (long long)HCT_C + HCT_COL(e)") << ";\n";
       }
+    } else if (nd.cls == OpClass::RowReduce && (nd.op == "row_argmax" || nd.op == "row_argmin")) {
+      // column of the largest / smallest element (the first one among equals), delivered as an fp32 value
+      std::string a = rg.ref(nd.args[0], true);
+      const bool amax = nd.op == "row_argmax";
+      b << "      float s" << id << "[HCT_B];\n      {\n        float bv_[HCT_B]; int bi_[HCT_B];\n        " << FORB << "{\n          bv_[b] = "
+        << (amax ? "-HCT_INF" : "HCT_INF") << ";\n          bi_[b] = 0x7fffffff;\n          " << FORE << "if (HCT_HAS(e) && (" << a
+        << (amax ? " > " : " < ") << "bv_[b] || bi_[b] == 0x7fffffff)) { bv_[b] = " << a << "; bi_[b] = HCT_COL(e); }\n        }\n"
+        << "        hct_row_argreduce<" << (amax ? "true" : "false") << ">(bv_, bi_, hct_cx, HCT_SM_SMEM);\n"
+        << (refill_placed ? "" : "@REFILL@")
+        << "        " << FORB << "s" << id << "[b] = (float)bi_[b];\n      }\n";
+    } else if (nd.cls == OpClass::RowReduce && nd.op == "row_min") {
+      // min(x) = -max(-x): shares the maximum's exchange
+      std::string a = rg.ref(nd.args[0], true);
+      b << "      float s" << id << "[HCT_B];\n      " << FORB << "{\n        s" << id << "[b] = -HCT_INF;\n        "
+        << FORE << "if (HCT_HAS(e)) s" << id << "[b] = fmaxf(s" << id << "[b], -(" << a << "));\n      }\n"
+        << "      HCT_RMAX(s" << id << ");\n";
+      if (!refill_placed) { b << "@REFILL@"; refill_placed = true; }
+      b << "      " << FORB << "s" << id << "[b] = -s" << id << "[b];\n";
     } else if (nd.cls == OpClass::RowReduce) {
       std::string a = rg.ref(nd.args[0], true);
       bool is_max = nd.op == "row_max";

@@ -262,7 +262,8 @@ Graph parse_spec(const std::string& text) {
           n.shape = g.nodes[n.args[0].node].shape;
         else
           n.shape = broadcast(g.nodes[n.args[0].node].shape, g.nodes[n.args[1].node].shape, line);
-      } else if (op == "row_softmax" || op == "row_sum" || op == "row_mean" || op == "row_max") {
+      } else if (op == "row_softmax" || op == "row_sum" || op == "row_mean" || op == "row_max" || op == "row_min" || op == "row_argmax" ||
+                 op == "row_argmin") {
         only_attrs({});
         if (pos.size() != 1) fail(HCT_ERR_GRAPH, line, op + " takes one operand");
         n.cls = op == "row_softmax" ? OpClass::RowSoftmax : OpClass::RowReduce;

@@ -127,6 +127,51 @@ __device__ __forceinline__ void hct_softmax_combine(float (&m)[HCT_B], float (&s
   for (int b = 0; b < HCT_B; ++b) f[b] = 1.0f;
 #endif
 }
+// Arg-reduction over a row: on entry v / ix hold each thread's best value and its column (the first
+// one among equals); on exit every thread holds the row's best value and the smallest column that has it.
+template <bool IS_MAX>
+__device__ __forceinline__ void hct_row_argreduce(float (&v)[HCT_B], int (&ix)[HCT_B], HctRowCtx& cx, float (*red)[2][HCT_B][3][32]) {
+  auto fold = [](float& a, int& ia, float b, int ib) {
+    const bool take = IS_MAX ? (b > a || (b == a && ib < ia)) : (b < a || (b == a && ib < ia));
+    if (take) { a = b; ia = ib; }
+  };
+#pragma unroll
+  for (int o = (HCT_T < 32 ? HCT_T : 32) / 2; o > 0; o >>= 1) {
+#pragma unroll
+    for (int b = 0; b < HCT_B; ++b) {
+      const float u = __shfl_xor_sync(0xffffffffu, v[b], o);
+      const int iu = __shfl_xor_sync(0xffffffffu, ix[b], o);
+      fold(v[b], ix[b], u, iu);
+    }
+  }
+#if HCT_T > 32
+  float (*slot)[3][32] = red[cx.g][cx.par];
+  cx.par ^= 1u;
+  if ((cx.t & 31) == 0) {
+#pragma unroll
+    for (int b = 0; b < HCT_B; ++b) {
+      slot[b][0][cx.t >> 5] = v[b];
+      slot[b][1][cx.t >> 5] = __int_as_float(ix[b]);
+    }
+  }
+  asm volatile("bar.sync %0, %1;" ::"r"(cx.g + 1), "n"(HCT_T) : "memory");
+  const int j = cx.t & (HCT_T / 32 - 1);
+#pragma unroll
+  for (int b = 0; b < HCT_B; ++b) {
+    v[b] = slot[b][0][j];
+    ix[b] = __float_as_int(slot[b][1][j]);
+#pragma unroll
+    for (int o = HCT_T / 64; o > 0; o >>= 1) {
+      const float u = __shfl_xor_sync(0xffffffffu, v[b], o);
+      const int iu = __shfl_xor_sync(0xffffffffu, ix[b], o);
+      fold(v[b], ix[b], u, iu);
+    }
+  }
+#else
+  (void)cx; (void)red;
+#endif
+}
+
 #if HCT_T > 32
 #define HCT_SM_SMEM hct_sm_smem
 #else

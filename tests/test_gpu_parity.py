@@ -172,6 +172,33 @@ def test_conv_bf16_nchw_direct_integer_inputs_are_exact():
     np.testing.assert_array_equal(got[0], want[0])
 
 
+# ------------------------------------------------------------------ arg reductions (indices are exact)
+
+@pytest.mark.parametrize("r,c", [(37, 1000), (300, 4096), (5, 1023), (64, 130), (3, 65536), (129, 24)])
+def test_row_argmax_argmin_min(r, c):
+    # taken on the inputs themselves (and on exact maps of them), so both sides see the same values
+    spec = f"hct 1\ninput x f32 [{r},{c}]\nnode a = row_argmax(x)\nnode n = neg(x)\nnode b = row_argmin(n)\nnode q = relu(x)\n" \
+           f"node c = row_argmin(q)\nnode d = row_min(x)\nnode e = row_argmin(x)\noutput a\noutput b\noutput c\noutput d\noutput e\n"
+    got, want, g = parity.run_both(spec, {"x": {"kind": "normal", "mean": 0.0, "std": 1.0}})
+    for a, b in zip(got, want):
+        np.testing.assert_array_equal(a, b)      # relu makes many equal zeros: the first column must win
+
+
+def test_row_argmax_after_inexact_chain_points_at_a_maximum():
+    # after rounding arithmetic the winner may differ between fp32 and fp64: what is checked is that the
+    # reported column holds a value within the fp32 tolerance of the row maximum
+    import oracle
+    spec = "hct 1\ninput x f32 [200,3000]\ninput w f32 [3000]\nnode t = mul(x, w)\nnode u = gelu_tanh(t)\nnode a = row_argmax(u)\noutput a\noutput u\n"
+    n = {"kind": "normal", "mean": 0.0, "std": 1.0}
+    got, want, g = parity.run_both(spec, {"x": n, "w": n})
+    idx = got[0][:, 0].astype(np.int64)
+    assert np.all((idx >= 0) & (idx < 3000))
+    u = want[1]
+    top = u.max(axis=1)
+    picked = u[np.arange(200), idx]
+    assert np.all(top - picked <= 1e-5 * np.abs(u).max(axis=1))
+
+
 # ------------------------------------------------------------------ dropout (counter-based mask)
 
 def _mask_is_exact(got, want):

@@ -341,6 +341,25 @@ def test_parse_rejects(bad):
         oracle.parse(bad)
 
 
+def test_row_min_and_arg_reductions_bruteforce_and_ties():
+    x = RNG.normal(size=(7, 13))
+    x[2, 4] = x[2, 9] = x[2].max() + 1.0      # a tie for the maximum: the first column wins
+    x[5, 0] = x[5, 12] = x[5].min() - 1.0     # a tie for the minimum
+    spec = "hct 1\ninput x f32 [7,13]\nnode a = row_argmax(x)\nnode b = row_argmin(x)\nnode c = row_min(x)\noutput a\noutput b\noutput c\n"
+    out = oracle.run(spec, {"x": x})
+    for i in range(7):
+        best_hi = max(range(13), key=lambda j: (x[i, j], -j))
+        best_lo = min(range(13), key=lambda j: (x[i, j], j))
+        assert out["a"][i, 0] == best_hi and out["b"][i, 0] == best_lo
+        assert out["c"][i, 0] == min(x[i, j] for j in range(13))
+    assert out["a"][2, 0] == 4 and out["b"][5, 0] == 0
+    t = torch.from_numpy(x)
+    np.testing.assert_array_equal(out["a"][:, 0], torch.argmax(t, dim=1).numpy())
+    # argmax commutes with increasing maps, argmin is the argmax of the negation
+    np.testing.assert_array_equal(interp.row_argmax(np.exp(x)), interp.row_argmax(x))
+    np.testing.assert_array_equal(interp.row_argmin(x), interp.row_argmax(-x))
+
+
 # ---------------------------------------------------------------- dropout (counter-based mask)
 
 _M64 = (1 << 64) - 1
