@@ -33,6 +33,7 @@
  *           row_argmax(x)  row_argmin(x)   column of the extreme element, the first among equals, as an fp32 value
  *           (row_softmax also accepts a single column, where it is identically one)
  *           row_layernorm(x, gamma, beta, eps=1e-5)   biased variance, eps inside the root
+ *   transpose(x)          y[j,i] = x[i,j] for x[R,C]; elementwise consumers are applied at the store
  *   gemm(a, b)            a[M,K] · b[K,N], both row-major, both f32 or both bf16 inputs;
  *                         bf16 multiplies on tensor cores with fp32 accumulation, f32
  *                         uses error-compensated TF32 products (or fp32 FMA for shapes

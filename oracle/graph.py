@@ -222,6 +222,15 @@ def _infer(g, name, op, pos, attrs, where):
         if len(s) != 2 or s[1] < (1 if op == "row_softmax" else 2):
             raise SpecError(f"{where}: {op} needs a [R,C] operand with enough columns")
         return Node(name, op, [a], {}, s if op in ROW_TO_ROW else (s[0], 1), "f32")
+    if op == "transpose":
+        only_attrs()
+        if len(pos) != 1:
+            raise SpecError(f"{where}: transpose takes one operand")
+        a = _operand(g, pos[0], where, False)
+        s = shape_of(a)
+        if len(s) != 2:
+            raise SpecError(f"{where}: transpose needs a [R,C] operand")
+        return Node(name, op, [a], {}, (s[1], s[0]), "f32")
     if op == "row_layernorm":
         only_attrs("eps")
         if len(pos) != 3:

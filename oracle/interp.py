@@ -86,6 +86,17 @@ def row_max(x):
     return x.max(axis=1, keepdims=True)
 
 
+# ---- layout transform (Table 1, "LayoutTransform") ------------------------------------------
+
+def transpose(x):
+    # y[j, i] = x[i, j]
+    r, c = x.shape
+    y = np.empty((c, r), dtype=x.dtype)
+    for i in range(r):
+        y[:, i] = x[i, :]
+    return y
+
+
 def row_min(x):
     return x.min(axis=1, keepdims=True)
 
@@ -173,6 +184,8 @@ def run_nodes(spec, inputs: dict, dtype=np.float64, gemm_fn=None) -> dict:
         elif op in BINARY:
             out = _BINARY_FN[op](args[0], args[1])
             out = np.broadcast_to(out, node.shape)
+        elif op == "transpose":
+            out = transpose(args[0])
         elif op == "row_softmax":
             out = row_softmax(args[0])
         elif op == "row_sum":

@@ -199,6 +199,29 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
   const Node& b = g.nodes[anchor.args[1].node];
   EpiGen eg{g, p, grp, gi, {}};
 
+  // ---- layout transform: tiled transposition through shared memory, consumers applied at the store
+  if (grp.kind == GroupKind::Transpose) {
+    const int src = anchor.args[0].node;
+    const int64_t R = a.shape[0], C = a.shape[1];
+    const int pa = eg.ptr_index(src, g.nodes[src].cls != OpClass::Input && p.ws_offset[src] >= 0);
+    const DType ta = eg.buf_dtype(src);
+    std::string epi = eg.scalar_fn();
+    KernelSpec k;
+    k.name = "hct_transpose_g" + std::to_string(gi);
+    std::ostringstream src_text;
+    src_text << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "LL\n#define HCT_TA " << ctype(ta) << "\n#define HCT_PA " << pa
+             << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+             << skeleton_source("common") << "\nstruct HctParams { void* ptr[" << eg.ptrs.size() << "]; };\n" << epi << skeleton_source("transpose");
+    k.source = src_text.str();
+    k.ptrs = eg.ptrs;
+    const int64_t tiles = ((R + 63) / 64) * ((C + 63) / 64);
+    k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(tiles, 148 * 8));
+    k.block[0] = 256;
+    k.desc = "transpose through 64x64 shared-memory tiles, consumers fused at the store";
+    out->push_back(k);
+    return;
+  }
+
   // ---- tensor-core GEMM: bf16 operands straight from their buffers
   if (grp.kind == GroupKind::Gemm && !tun.simt_only) {
     int64_t M = a.shape[0], K = a.shape[1], N = b.shape[1];

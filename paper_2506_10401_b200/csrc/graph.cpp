@@ -289,6 +289,15 @@ Graph parse_spec(const std::string& text) {
         if (attrs.count("eps") && (!parse_number(attrs["eps"], &n.eps) || !(n.eps >= 0)))
           fail(HCT_ERR_PARSE, line, "eps must be a non-negative number");
         n.shape = s;
+      } else if (op == "transpose") {
+        // layout transform (Table 1): y[j,i] = x[i,j] for a 2-D operand
+        only_attrs({});
+        if (pos.size() != 1) fail(HCT_ERR_GRAPH, line, "transpose takes one operand");
+        n.cls = OpClass::Transpose;
+        n.args = {lookup(pos[0], line, false)};
+        auto& s = g.nodes[n.args[0].node].shape;
+        if (s.size() != 2) fail(HCT_ERR_GRAPH, line, "transpose needs a [R,C] operand, got " + shape_str(s));
+        n.shape = {s[1], s[0]};
       } else if (op == "gemm") {
         only_attrs({"precision"});
         if (pos.size() != 2) fail(HCT_ERR_GRAPH, line, "gemm takes (a, b)");

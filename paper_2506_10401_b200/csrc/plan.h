@@ -3,7 +3,7 @@
 // Two kinds of group exist.  A *row group* is a maximal set of elementwise, broadcast and
 // row-reduction nodes that share one [R,C] iteration space, so a row can stay in registers from
 // the first load to the last store.  A *contraction group* is one gemm or conv2d node together
-// with the elementwise nodes that consume its result (its epilogue).  Values that cross a group
+// with the elementwise nodes that consume its result (its epilogue); a transpose anchors a group the same way.  Values that cross a group
 // boundary are written once to caller-provided workspace (fp32).
 #pragma once
 #include <string>
@@ -13,7 +13,7 @@
 
 namespace hct {
 
-enum class GroupKind { Row, Gemm, Conv };
+enum class GroupKind { Row, Gemm, Conv, Transpose };
 
 // How an operand indexes relative to the group's full shape [.., C].
 enum class Bcast {

@@ -172,6 +172,39 @@ def test_conv_bf16_nchw_direct_integer_inputs_are_exact():
     np.testing.assert_array_equal(got[0], want[0])
 
 
+# ------------------------------------------------------------------ layout transform
+
+@pytest.mark.parametrize("r,c", [(37, 1000), (300, 4096), (5, 1023), (1, 7), (64, 64), (129, 65), (2048, 2048)])
+def test_transpose_is_exact_and_fuses_its_consumers(r, c):
+    spec = f"hct 1\ninput x f32 [{r},{c}]\ninput b f32 [{r}]\ninput y bf16 [{r},{c}]\nnode t = transpose(x)\nnode u = add(t, b)\nnode v = relu(u)\n" \
+           f"node w = transpose(y)\noutput t\noutput v\noutput w bf16\n"
+    n = {"kind": "normal", "mean": 0.0, "std": 1.0}
+    got, want, g = parity.run_both(spec, {"x": n, "b": n, "y": n})
+    np.testing.assert_array_equal(got[0], want[0])     # pure data movement
+    np.testing.assert_array_equal(got[2], want[2])     # bf16 in, bf16 out: exact too
+    assert parity.f32_violation(got[1], want[1]) <= 1.0
+    assert g.num_kernels == 2 and "transpose" in g.plan
+
+
+def test_transpose_between_other_kernels():
+    spec = """hct 1
+input x f32 [96,256]
+input w f32 [96,128]
+input g f32 [128]
+input b f32 [128]
+node a = gelu_tanh(x)
+node t = transpose(a)
+node m = gemm(t, w)
+node n = row_layernorm(m, g, b, eps=1e-5)
+node o = transpose(n)
+output o
+"""
+    n = {"kind": "normal", "mean": 0.0, "std": 1.0}
+    got, want, g = parity.run_both(spec, {"x": n, "w": {"kind": "normal", "mean": 0.0, "std": 0.1}, "g": n, "b": n})
+    assert got[0].shape == (128, 256)
+    assert parity.f32_violation(got[0], want[0]) <= 1.0
+
+
 # ------------------------------------------------------------------ arg reductions (indices are exact)
 
 @pytest.mark.parametrize("r,c", [(37, 1000), (300, 4096), (5, 1023), (64, 130), (3, 65536), (129, 24)])

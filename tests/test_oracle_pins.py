@@ -341,6 +341,24 @@ def test_parse_rejects(bad):
         oracle.parse(bad)
 
 
+def test_transpose_pins():
+    x = RNG.normal(size=(5, 9))
+    spec = "hct 1\ninput x f32 [5,9]\nnode t = transpose(x)\nnode u = transpose(t)\noutput t\noutput u\n"
+    out = oracle.run(spec, {"x": x})
+    assert out["t"].shape == (9, 5)
+    for i in range(5):
+        for j in range(9):
+            assert out["t"][j, i] == x[i, j]
+    np.testing.assert_array_equal(out["u"], x)                           # an involution
+    np.testing.assert_array_equal(out["t"], torch.from_numpy(x).t().numpy())
+    # (A B)^T = B^T A^T ties the layout transform to the matrix product
+    a, b = RNG.integers(-8, 9, size=(4, 6)).astype(float), RNG.integers(-8, 9, size=(6, 3)).astype(float)
+    spec = ("hct 1\ninput a f32 [4,6]\ninput b f32 [6,3]\nnode p = gemm(a, b)\nnode pt = transpose(p)\nnode at = transpose(a)\n"
+            "node bt = transpose(b)\nnode q = gemm(bt, at)\noutput pt\noutput q\n")
+    out = oracle.run(spec, {"a": a, "b": b})
+    np.testing.assert_array_equal(out["pt"], out["q"])
+
+
 def test_row_min_and_arg_reductions_bruteforce_and_ties():
     x = RNG.normal(size=(7, 13))
     x[2, 4] = x[2, 9] = x[2].max() + 1.0      # a tie for the maximum: the first column wins

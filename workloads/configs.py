@@ -104,12 +104,27 @@ output t2 f32
     return spec, laws
 
 
+def transpose_bias_relu(r=16384, c=4096):
+    """A layout transform with fused consumers (Table 1, "LayoutTransform"): y = relu(x^T + bias)."""
+    spec = f"""hct 1
+input x    f32 [{r},{c}]
+input bias f32 [{r}]
+node  t0 = transpose(x)
+node  t1 = add(t0, bias)
+node  t2 = relu(t1)
+output t2 f32
+"""
+    laws = {"x": _n(), "bias": _n()}
+    return spec, laws
+
+
 CONFIGS = {
     "c1_gemm_bias_relu_f32": (gemm_bias_relu, {}),
     "c2_softmax_layernorm_chain": (softmax_layernorm_chain, {}),
     "c3_gemm_bf16_gelu_residual": (gemm_bf16_gelu_residual, {}),
     "c4_conv_bn_relu_bf16": (conv_bn_relu, {}),
     "matmul_dropout_mean_softmax": (matmul_dropout_mean_softmax, {}),
+    "transpose_bias_relu": (transpose_bias_relu, {}),
 }
 
 
