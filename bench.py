@@ -33,6 +33,9 @@ WORKLOADS = {
     "c3_gemm_bf16_gelu_residual": dict(bound="tensor", sample=dict(m=2048)),
     "c4_conv_bn_relu_bf16": dict(bound="tensor", sample=dict(n=8)),
     "c1_gemm_bias_relu_f32": dict(bound="tensor", sample=dict()),
+    # operator classes beyond the five configurations: a layout transform and the case-study chain with dropout
+    "transpose_bias_relu": dict(bound="hbm", sample=dict(r=4096)),
+    "matmul_dropout_mean_softmax": dict(bound="tensor", sample=dict(m=1024)),
 }
 HEADLINE = "c2_softmax_layernorm_chain"
 
@@ -168,7 +171,7 @@ def oracle_arm(name, steps, warmup):
                 ms_per_step=dt * 1e3)
 
 
-def run_gpu(name, steps, warmup, rank, world, device):
+def run_gpu(name, steps, warmup, rank, world, device, tune=0):
     import torch
     import paper_2506_10401_b200 as hct
     from tests import parity
@@ -176,8 +179,9 @@ def run_gpu(name, steps, warmup, rank, world, device):
     info = WORKLOADS[name]
     spec, laws = configs.get_config(name)
     host = configs.draw_inputs(spec, laws, 0)
-    g = hct.FusedGraph(spec, device)
     ins = parity.to_device(spec, host, f"cuda:{device}")
+    # with --tune N the schedule is picked by measurement (set-up, untimed); the default is the fixed rules
+    g = hct.FusedGraph.autotuned(spec, ins, device, max_trials=tune) if tune > 0 else hct.FusedGraph(spec, device)
     outs = g.alloc_outputs()
     bytes_, flops = g.cost()
     stream = torch.cuda.current_stream(device)
@@ -237,10 +241,11 @@ def run_gpu(name, steps, warmup, rank, world, device):
     return dict(value=value, unit=unit, ms_per_step=dev_s / steps * 1e3, bytes=bytes_, flops=flops, kernel_s=kern_s,
                 fingerprint=kernel_fingerprint(g),
                 kernels=g.num_kernels, clocks=clocks.summary(), e2e=dict(value=e2e_v, unit=unit, h2d_bytes_per_step=h2d,
-                                                                         d2h_bytes_per_step=d2h), plan=g.plan)
+                                                                         d2h_bytes_per_step=d2h), plan=g.plan,
+                schedule=g.schedule)
 
 
-def run_sweep(steps, warmup, device, out_path=None):
+def run_sweep(steps, warmup, device, out_path=None, tune=0):
     """The 200 random operator DAGs: per-graph time against its own roofline, and class aggregates.
 
     Inputs are drawn on the device from the same laws (normal / uniform with the recipe's mean and
@@ -257,7 +262,6 @@ def run_sweep(steps, warmup, device, out_path=None):
     launches = 0
     for e in sweep.entries():
         spec, laws, meta = sweep.get(e["seed"])
-        g = hct.FusedGraph(spec, device)
         gen = torch.Generator(device=dev)
         gen.manual_seed(1000 + e["seed"])
         ins = []
@@ -268,6 +272,7 @@ def run_sweep(steps, warmup, device, out_path=None):
             else:
                 t = torch.rand(shape, device=dev, generator=gen) * (law["hi"] - law["lo"]) + law["lo"]
             ins.append(t.to(torch.bfloat16) if dtype == "bf16" else t)
+        g = hct.FusedGraph.autotuned(spec, ins, device, max_trials=tune) if tune > 0 else hct.FusedGraph(spec, device)
         outs = g.alloc_outputs()
         for _ in range(max(1, warmup)):
             g.run(ins, outs, stream)
@@ -285,7 +290,7 @@ def run_sweep(steps, warmup, device, out_path=None):
         t_mem = bytes_ / (pk["hbm"] * 1e9)
         t_mma = flops / (pk["tensor"] / 6.0 * 1e12)  # fp32 GEMM = three TF32 products at half the bf16 rate
         cls = "gemm" if t_mma > t_mem else "memory"
-        records.append(dict(seed=e["seed"], cls=cls, us=sec * 1e6, bytes=bytes_, flops=flops, kernels=g.num_kernels,
+        records.append(dict(seed=e["seed"], cls=cls, us=sec * 1e6, bytes=bytes_, flops=flops, kernels=g.num_kernels, schedule=g.schedule,
                             frac=max(t_mem, t_mma) / sec))
         launches += g.num_kernels * (steps + max(1, warmup))
         g.close()
@@ -316,6 +321,7 @@ def main():
     ap.add_argument("--workload", default=HEADLINE, choices=list(WORKLOADS) + ["c5_sweep"])
     ap.add_argument("--out", default=None, help="c5_sweep: write one JSON record per graph to this file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tune", type=int, default=0, help="pick each graph's schedule by measuring up to N candidates (untimed set-up)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -348,12 +354,13 @@ def main():
         if world > 1:
             raise SystemExit("the sweep runs on one GPU")
         with ClockSampler(local) as clocks:
-            agg, launches = run_sweep(max(3, min(args.steps, 10)), args.warmup, local, args.out)
+            agg, launches = run_sweep(max(3, min(args.steps, 10)), args.warmup, local, args.out, args.tune)
         pk = peaks()
         print(json.dumps(dict(metric=metric, value=agg["memory_GBps"], unit="GB/s", n_gpus=1, steps=args.steps, warmup=args.warmup,
                               ms_per_step=agg["total_ms"], higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
                               data="synthetic", config={"workload": "c5_sweep: 200 random operator DAGs, seeds 0..199",
-                                                        "l2": "flushed between runs", "value_is": "aggregate over memory-bound graphs"},
+                                                        "l2": "flushed between runs", "value_is": "aggregate over memory-bound graphs",
+                                                        "tuned_trials": args.tune},
                               clocks=clocks.summary(), gpu_launches=launches, sweep=agg,
                               roofline=dict(bound="hbm", achieved=agg["memory_GBps"], peak=pk["hbm"], unit="GB/s",
                                             frac=agg["memory_GBps"] / pk["hbm"], traffic=None, peak_source=pk["source"]),
@@ -362,7 +369,7 @@ def main():
     if world > 1:
         torch.cuda.set_device(local)
         torch.distributed.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
-    r = run_gpu(name, args.steps, args.warmup, rank, world, local)
+    r = run_gpu(name, args.steps, args.warmup, rank, world, local, args.tune)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         o = oracle_arm(name, 4, 1)
@@ -378,9 +385,10 @@ def main():
         peak = pk["hbm"] if info["bound"] == "hbm" else (pk["tensor_sustained"] if capped else pk["tensor"])
         line = dict(metric=metric, value=r["value"], unit=r["unit"], n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
                     ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
-                    dtype="bf16" if "bf16" in name else "f32", data="synthetic",
+                    dtype="bf16" if ("bf16" in name or name == "matmul_dropout_mean_softmax") else "f32", data="synthetic",
                     config={"workload": name, "l2": "flushed between steps (192 MB write, untimed)", "kernels_per_step": r["kernels"],
-                            "parallelism": "replicas" if world > 1 else "single"},
+                            "parallelism": "replicas" if world > 1 else "single",
+                            "schedule": r["schedule"] or "default", "tuned_trials": args.tune},
                     clocks=r["clocks"], e2e=r["e2e"], gpu_launches=r["kernels"] * args.steps,
                     roofline=dict(bound=info["bound"], achieved=achieved, peak=peak, unit=("GB/s" if info["bound"] == "hbm" else "TFLOP/s"),
                                   frac=achieved / peak, traffic=recorded_traffic(name, r["fingerprint"]), peak_source=pk["source"],
