@@ -208,31 +208,54 @@ def run_gpu(name, steps, warmup, rank, world, device, tune=0):
     per_step = [a.elapsed_time(b) * 1e-3 for a, b in ev]
     dev_s = float(np.sum(per_step))
 
-    # end to end: pinned host inputs -> device, run, result back to the host, every step
-    pinned = [torch.from_numpy(host[n].view(np.int16) if d == "bf16" else host[n]).pin_memory() for n, d, _ in configs.parse_inputs(spec)]
-    dev_in = [torch.empty_like(t, device=f"cuda:{device}") for t in pinned]
-    run_in = [t.view(torch.bfloat16) if d == "bf16" else t for t, (_, d, _) in zip(dev_in, configs.parse_inputs(spec))]
-    host_out = [torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in outs]
+    # end to end: pinned host inputs -> device, run, result back to the host, every step.  The three
+    # phases of consecutive steps overlap (copy-in, compute and copy-out streams, two sets of device
+    # buffers): PCIe is full duplex, so step i+1's inputs travel while step i's result returns.
+    specs_in = configs.parse_inputs(spec)
+    pinned = [torch.from_numpy(host[n].view(np.int16) if d == "bf16" else host[n]).pin_memory() for n, d, _ in specs_in]
+    dev_in = [[torch.empty_like(t, device=f"cuda:{device}") for t in pinned] for _ in range(2)]
+    run_in = [[t.view(torch.bfloat16) if d == "bf16" else t for t, (_, d, _) in zip(buf, specs_in)] for buf in dev_in]
+    dev_out = [outs, g.alloc_outputs()]
+    host_out = [[torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in outs] for _ in range(2)]
     h2d = sum(t.numel() * t.element_size() for t in pinned)
-    d2h = sum(t.numel() * t.element_size() for t in host_out)
-    e2e_steps = max(2, min(steps, 5))
+    d2h = sum(t.numel() * t.element_size() for t in host_out[0])
+    e2e_steps = max(4, min(steps, 8))
+    s_in, s_run, s_out = (torch.cuda.Stream(device) for _ in range(3))
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_run = [torch.cuda.Event() for _ in range(2)]
+    ev_out = [torch.cuda.Event() for _ in range(2)]
 
-    def e2e_once():
-        for src, dst in zip(pinned, dev_in):
-            dst.copy_(src, non_blocking=True)
-        g.run(run_in, outs, stream)
-        for src, dst in zip(outs, host_out):
-            dst.copy_(src, non_blocking=True)
+    def e2e_loop(n):
+        for i in range(n):
+            b = i % 2
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(ev_run[b])      # the kernels of step i-2 have read this input set
+                for src, dst in zip(pinned, dev_in[b]):
+                    dst.copy_(src, non_blocking=True)
+                ev_in[b].record(s_in)
+            s_run.wait_event(ev_in[b])
+            if i >= 2:
+                s_run.wait_event(ev_out[b])         # step i-2's result has left this output set
+            g.run(run_in[b], dev_out[b], s_run)
+            ev_run[b].record(s_run)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_run[b])
+                for src, dst in zip(dev_out[b], host_out[b]):
+                    dst.copy_(src, non_blocking=True)
+                ev_out[b].record(s_out)
 
-    e2e_once()
+    e2e_loop(2)
     barrier()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(stream)
-    for _ in range(e2e_steps):
-        e2e_once()
-    b.record(stream)
+    a.record(s_in)
+    e2e_loop(e2e_steps)
+    s_out.wait_stream(s_in)
+    s_out.wait_stream(s_run)
+    b.record(s_out)
     barrier()
     e2e_s = a.elapsed_time(b) * 1e-3 / e2e_steps
+    g.status()
 
     dev_s, e2e_s = max_over_ranks([dev_s, e2e_s], f"cuda:{device}")
     value, unit = whole_job_value(info["bound"], bytes_, flops, world, dev_s / steps)

@@ -307,10 +307,11 @@ hct_status_t hct_graph_autotune(const char* spec, size_t spec_len, int device, c
   hct_graph_t* best = nullptr;
   hct_status_t rc = hct_graph_create_scheduled(spec, spec_len, device, "", &best);   // the default shape is always a candidate
   if (rc != HCT_OK) return rc;
-  bool has_row = false, has_conv = false;
+  bool has_row = false, has_conv = false, has_gemm = false;
   for (auto& grp : best->plan.groups) {
     has_row = has_row || grp.kind == GroupKind::Row;
     has_conv = has_conv || grp.kind == GroupKind::Conv;
+    has_gemm = has_gemm || grp.kind == GroupKind::Gemm;
   }
   std::vector<std::string> cands;
   if (has_row)
@@ -318,6 +319,8 @@ hct_status_t hct_graph_autotune(const char* spec, size_t spec_len, int device, c
                           "row_nv=2;row_cta_small=512", "row_ring_bytes_small=98304", "row_cta_elementwise=256", "row_cta_elementwise=1024",
                           "row_nv=8;row_cta_small=128", "row_no_stage=1", "row_nv=2;row_minb=2"})
       cands.push_back(c);
+  if (has_gemm)
+    for (const char* c : {"gemm_bn=64", "gemm_bn=128", "gemm_bn=32"}) cands.insert(cands.begin(), c);
   if (has_conv)
     for (const char* c : {"conv_no_tma_store=1", "conv_no_direct=1", "conv_no_direct=1;conv_no_halo=1"}) cands.push_back(c);
 

@@ -55,6 +55,7 @@ struct Tunables {
   bool row_no_softmax_ln_fusion = false;  // layer norm after softmax: take the variance with its own reduction
   bool row_no_stage = false;       // load rows straight from global memory instead of through the shared-memory ring
   int row_ring_bytes = 200 * 1024; // shared memory a staged row kernel may spend on resident row vectors plus its prefetch ring
+  int gemm_bn = 0;                 // output-tile width of the tensor-core GEMMs (0: by rule; else 32..256, clamped to what the kernel takes)
   bool conv_no_halo = false;       // load conv pixels once per tap even when the shared-row schedule applies
   bool conv_no_tma_store = false;  // NCHW-reading convolution: store the output with plain vector stores instead of TMA
   bool conv_no_direct = false;     // always take the NHWC pre-pass, even when the convolution could read NCHW itself

@@ -191,7 +191,6 @@ struct EpiGen {
 
 void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunables& tun, size_t* scratch_bytes,
                              std::vector<KernelSpec>* out) {
-  (void)tun;
   (void)scratch_bytes;
   const Group& grp = p.groups[gi];
   const Node& anchor = g.nodes[grp.nodes[0]];
@@ -228,7 +227,11 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     DType da = g.nodes[anchor.args[0].node].cls == OpClass::Input ? a.dtype : F32;
     DType db = g.nodes[anchor.args[1].node].cls == OpClass::Input ? b.dtype : F32;
     if (da == BF16 && db == BF16 && K % 8 == 0 && N % 8 == 0 && M <= 0x7fffffff && N <= 0x7fffffff && K <= 0x7fffffff) {
-      int BN = N > 128 ? 256 : N > 64 ? 128 : 64;
+      const int bn_max = N > 128 ? 256 : N > 64 ? 128 : 64;
+      int BN = bn_max;
+      // few tiles leave SMs idle: halve the tile width while that at least doubles the busy SMs
+      while (BN > 64 && ((M + 127) / 128) * ((N + BN - 1) / BN) * 2 <= 148) BN /= 2;
+      if (tun.gemm_bn >= 64) BN = std::min(bn_max, tun.gemm_bn >= 256 ? 256 : tun.gemm_bn >= 128 ? 128 : 64);
       int stages = BN == 256 ? 4 : 6;
       std::string epi = eg.run_fn(N);
       KernelSpec k;
@@ -309,7 +312,10 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         k.desc = "tf32 head/tail split of both gemm operands, B transposed";
         out->push_back(k);
       }
-      int BN = N > 64 ? 128 : N > 32 ? 64 : 32;
+      const int bn_max = N > 64 ? 128 : N > 32 ? 64 : 32;
+      int BN = bn_max;
+      while (BN > 64 && ((M + 127) / 128) * ((N + BN - 1) / BN) * 2 <= 148) BN /= 2;
+      if (tun.gemm_bn >= 32) BN = std::min(bn_max, tun.gemm_bn >= 128 ? 128 : tun.gemm_bn >= 64 ? 64 : 32);
       int stages = BN == 128 ? 3 : BN == 64 ? 4 : 5;
       std::string epi = eg.run_fn(N);
       KernelSpec k;
