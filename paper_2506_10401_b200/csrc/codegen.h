@@ -34,6 +34,7 @@ struct KernelSpec {
   unsigned block[3] = {1, 1, 1};
   unsigned smem_bytes = 0;       // dynamic shared memory
   bool persistent = false;       // grid[0] is scaled to SM count x occupancy at load time
+  unsigned cluster = 1;          // CTAs per cluster (compiled into the kernel); the grid is kept a multiple of it
   unsigned max_grid = 0;         // upper bound for a persistent grid (number of work items)
   std::vector<BufRef> ptrs;      // pointer arguments in order (params.ptr[i])
   std::vector<TmaDesc> tmaps;    // tensor maps in order (params.tmap[i])
@@ -55,6 +56,7 @@ struct Tunables {
   bool row_no_softmax_ln_fusion = false;  // layer norm after softmax: take the variance with its own reduction
   bool row_no_stage = false;       // load rows straight from global memory instead of through the shared-memory ring
   int row_ring_bytes = 200 * 1024; // shared memory a staged row kernel may spend on resident row vectors plus its prefetch ring
+  int gemm_pair = 0;               // bf16 GEMM on CTA pairs (256x256 tiles): 0 by rule (enough tiles for every pair), 1 always, 2 never
   int gemm_bn = 0;                 // output-tile width of the tensor-core GEMMs (0: by rule; else 32..256, clamped to what the kernel takes)
   bool conv_no_halo = false;       // load conv pixels once per tap even when the shared-row schedule applies
   bool conv_no_tma_store = false;  // NCHW-reading convolution: store the output with plain vector stores instead of TMA

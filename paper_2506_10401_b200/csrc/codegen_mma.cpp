@@ -226,6 +226,47 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     int64_t M = a.shape[0], K = a.shape[1], N = b.shape[1];
     DType da = g.nodes[anchor.args[0].node].cls == OpClass::Input ? a.dtype : F32;
     DType db = g.nodes[anchor.args[1].node].cls == OpClass::Input ? b.dtype : F32;
+    // CTA pairs on 256 x 256 tiles when every pair of SMs gets at least one tile
+    const int64_t pair_tiles = ((M + 255) / 256) * ((N + 255) / 256);
+    const bool use_pair = tun.gemm_pair == 1 || (tun.gemm_pair == 0 && pair_tiles >= 74 && !tun.fault_never_arrive && tun.gemm_bn == 0);
+    if (da == BF16 && db == BF16 && K % 8 == 0 && N % 8 == 0 && M <= 0x7fffffff && N <= 0x7fffffff && K <= 0x7fffffff && use_pair) {
+      const int stages = 6;
+      std::string epi = eg.run_fn(N);
+      KernelSpec k;
+      k.name = "hct_gemm_tc2_bf16_g" + std::to_string(gi);
+      std::ostringstream src;
+      src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n#define HCT_STAGES " << stages
+          << (tun.wait_limit ? "\n#define HCT_WAIT_LIMIT " + std::to_string(tun.wait_limit) + "u" : std::string())
+          << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size() << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
+      src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[2]; void* ptr["
+          << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source("gemm_tc2");
+      k.source = src.str();
+      k.ptrs = eg.ptrs;
+      k.wants_status = true;
+      TmaDesc ta, tb;
+      ta.buf.node = anchor.args[0].node;
+      ta.elem_bytes = 2;
+      ta.rank = 2;
+      ta.dims[0] = (uint64_t)K; ta.dims[1] = (uint64_t)M;
+      ta.strides[1] = (uint64_t)K * 2;
+      ta.box[0] = 64; ta.box[1] = 128;
+      tb.buf.node = anchor.args[1].node;
+      tb.elem_bytes = 2;
+      tb.rank = 2;
+      tb.dims[0] = (uint64_t)N; tb.dims[1] = (uint64_t)K;
+      tb.strides[1] = (uint64_t)N * 2;
+      tb.box[0] = 64; tb.box[1] = 64;
+      k.tmaps = {ta, tb};
+      k.block[0] = 192;
+      k.smem_bytes = (unsigned)(stages * 32768 + 1024);
+      k.persistent = true;
+      k.cluster = 2;
+      k.max_grid = (unsigned)std::min<int64_t>(2 * pair_tiles, 0x7ffffffe);
+      k.grid[0] = k.max_grid;
+      k.desc = "gemm tcgen05 bf16 on CTA pairs, 256x256x64 per pair, " + std::to_string(stages) + " stages";
+      out->push_back(k);
+      return;
+    }
     if (da == BF16 && db == BF16 && K % 8 == 0 && N % 8 == 0 && M <= 0x7fffffff && N <= 0x7fffffff && K <= 0x7fffffff) {
       const int bn_max = N > 128 ? 256 : N > 64 ? 128 : 64;
       int BN = bn_max;

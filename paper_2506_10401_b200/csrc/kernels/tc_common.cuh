@@ -113,6 +113,50 @@ __device__ __forceinline__ hct_u64 hct_smem_desc(hct_u32 addr, hct_u32 lbo, hct_
   return (hct_u64)((addr & 0x3ffffu) >> 4) | ((hct_u64)(lbo >> 4) << 16) | ((hct_u64)(sbo >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// ---- CTA pairs (cta_group::2): two CTAs of a cluster share one MMA of 256 rows; the even CTA issues it
+__device__ __forceinline__ hct_u32 hct_cluster_ctarank() {
+  hct_u32 r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of this CTA's shared-memory location `addr` as seen in CTA `rank` of the cluster
+__device__ __forceinline__ hct_u32 hct_mapa(hct_u32 addr, hct_u32 rank) {
+  hct_u32 r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void hct_mbar_arrive_cluster(hct_u32 cluster_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+// TMA tile load into this CTA's shared memory whose completion is counted on a barrier of either CTA of the pair
+__device__ __forceinline__ void hct_tma_load_2d_pair(hct_u32 dst, const HctTensorMap* map, int c0, int c1, hct_u32 cluster_bar) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+               "l"(map), "r"(c0), "r"(c1), "r"(cluster_bar)
+               : "memory");
+}
+__device__ __forceinline__ void hct_mma_f16_pair(hct_u32 d_tmem, hct_u64 adesc, hct_u64 bdesc, hct_u32 idesc, hct_u32 accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// completes `cluster_bar` (a barrier of either CTA) once every MMA issued so far by this thread has finished
+__device__ __forceinline__ void hct_mma_commit_pair(hct_u32 cluster_bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void hct_tmem_alloc_pair(hct_u32 holder_smem, hct_u32 ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void hct_tmem_dealloc_pair(hct_u32 taddr, hct_u32 ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void hct_cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // ---- contiguous runs of up to 32 epilogue elements (16-byte accesses when the run is a whole number of vectors)
 template <typename T>
 __device__ __forceinline__ void hct_ld_run32(const T* p, float* v, int n, bool vec_ok);

@@ -131,6 +131,32 @@ def test_gemm_bf16_chain_shapes(m, k, n):
     check_bf16(spec, laws)
 
 
+@pytest.mark.parametrize("m,k,n", [(300, 264, 520), (257, 4096, 136), (1, 8, 8), (512, 64, 512), (130, 1000, 264), (1000, 320, 776)])
+def test_gemm_bf16_on_cta_pairs(m, k, n):
+    """The CTA-pair kernel (256 x 256 tiles, chosen by rule only for large problems) forced onto small and ragged shapes."""
+    import torch
+    import oracle
+    import paper_2506_10401_b200 as hct
+    spec, laws = configs.get_config("c3_gemm_bf16_gelu_residual", m=m, k=k, n=n)
+    t = configs.draw_inputs(spec, laws, 0)
+    g = hct.FusedGraph(spec, 0, schedule="gemm_pair=1")
+    assert "CTA pairs" in g.plan
+    out = g.run(parity.to_device(spec, t))[0]
+    torch.cuda.synchronize()
+    g.status()
+    ref = oracle.run(spec, parity.oracle_inputs(spec, t))["t3"]
+    assert parity.bf16_violation(parity.to_numpy64(out), ref) <= 1.0
+    # integer-valued operands: every partial sum is exact, so the product must match bit for bit
+    spec = f"hct 1\ninput x bf16 [{m},{k}]\ninput w bf16 [{k},{n}]\nnode y = gemm(x, w)\noutput y f32\n"
+    il = {"kind": "int", "lo": -8, "hi": 8}
+    t = configs.draw_inputs(spec, {"x": il, "w": il}, 1)
+    g = hct.FusedGraph(spec, 0, schedule="gemm_pair=1")
+    out = g.run(parity.to_device(spec, t))[0]
+    torch.cuda.synchronize()
+    g.status()
+    np.testing.assert_array_equal(parity.to_numpy64(out), oracle.run(spec, parity.oracle_inputs(spec, t))["y"])
+
+
 def test_gemm_bf16_integer_inputs_are_exact():
     spec = "hct 1\ninput x bf16 [200,320]\ninput w bf16 [320,264]\nnode y = gemm(x, w)\noutput y f32\n"
     il = {"kind": "int", "lo": -8, "hi": 8}
