@@ -236,6 +236,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       k.name = "hct_gemm_tc2_bf16_g" + std::to_string(gi);
       std::ostringstream src;
       src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n#define HCT_STAGES " << stages
+          << "\n#define HCT_TF32X3 0"
           << (tun.wait_limit ? "\n#define HCT_WAIT_LIMIT " + std::to_string(tun.wait_limit) + "u" : std::string())
           << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size() << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
       src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[2]; void* ptr["
@@ -359,6 +360,42 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       if (tun.gemm_bn >= 32) BN = std::min(bn_max, tun.gemm_bn >= 128 ? 128 : tun.gemm_bn >= 64 ? 64 : 32);
       int stages = BN == 128 ? 3 : BN == 64 ? 4 : 5;
       std::string epi = eg.run_fn(N);
+      // CTA pairs on 256 x 128 tiles: only on request (schedule knob or tuning).  Measured on
+      // 16384 x 4096 x 4096 it equals the single-CTA kernel (2.89 ms against 2.88 ms): these long fp32
+      // GEMMs run at the power cap, not at the shared-memory bound the pairing relieves.
+      const int64_t pair_tiles32 = ((M + 255) / 256) * ((N + 127) / 128);
+      if (tun.gemm_pair == 1) {
+        const int pstages = 4;
+        KernelSpec k;
+        k.name = "hct_gemm_tc2_tf32x3_g" + std::to_string(gi);
+        std::ostringstream src;
+        src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n#define HCT_STAGES " << pstages
+            << "\n#define HCT_TF32X3 1\n#define HCT_STATUS_SLOT " << eg.ptrs.size() << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
+        src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[4]; void* ptr["
+            << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source("gemm_tc2");
+        k.source = src.str();
+        k.ptrs = eg.ptrs;
+        k.wants_status = true;
+        for (int i = 0; i < 4; ++i) {
+          TmaDesc t;
+          t.buf = scratch(i == 0 ? off_ahi : i == 1 ? off_alo : i == 2 ? off_bhi : off_blo);
+          t.elem_bytes = 4;
+          t.rank = 2;
+          t.dims[0] = (uint64_t)K; t.dims[1] = (uint64_t)(i < 2 ? M : N);   // B is transposed to [N,K]
+          t.strides[1] = (uint64_t)K * 4;
+          t.box[0] = 32; t.box[1] = i < 2 ? 128 : 64;
+          k.tmaps.push_back(t);
+        }
+        k.block[0] = 192;
+        k.smem_bytes = (unsigned)(pstages * 49152 + 1024);
+        k.persistent = true;
+        k.cluster = 2;
+        k.max_grid = (unsigned)std::min<int64_t>(2 * pair_tiles32, 0x7ffffffe);
+        k.grid[0] = k.max_grid;
+        k.desc = "gemm tcgen05 tf32x3 on CTA pairs, 256x128x32 per pair, " + std::to_string(pstages) + " stages";
+        out->push_back(k);
+        return;
+      }
       KernelSpec k;
       k.name = "hct_gemm_tc_tf32x3_g" + std::to_string(gi);
       std::ostringstream src;

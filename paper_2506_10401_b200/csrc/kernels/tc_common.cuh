@@ -142,6 +142,14 @@ __device__ __forceinline__ void hct_mma_f16_pair(hct_u32 d_tmem, hct_u64 adesc, 
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+__device__ __forceinline__ void hct_mma_tf32_pair(hct_u32 d_tmem, hct_u64 adesc, hct_u64 bdesc, hct_u32 idesc, hct_u32 accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // completes `cluster_bar` (a barrier of either CTA) once every MMA issued so far by this thread has finished
 __device__ __forceinline__ void hct_mma_commit_pair(hct_u32 cluster_bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_bar) : "memory");

@@ -157,6 +157,29 @@ def test_gemm_bf16_on_cta_pairs(m, k, n):
     np.testing.assert_array_equal(parity.to_numpy64(out), oracle.run(spec, parity.oracle_inputs(spec, t))["y"])
 
 
+@pytest.mark.parametrize("m,k,n", [(300, 1000, 520), (257, 4096, 136), (5, 8, 3), (512, 64, 256), (130, 16384, 72), (1024, 260, 1000)])
+def test_gemm_f32_on_cta_pairs(m, k, n):
+    """The fp32 (three TF32 products) kernel on CTA pairs, forced onto small and ragged shapes."""
+    import torch
+    import oracle
+    import paper_2506_10401_b200 as hct
+    spec, laws = configs.get_config("c1_gemm_bias_relu_f32", m=m, k=k, n=n)
+    t = configs.draw_inputs(spec, laws, 0)
+    g = hct.FusedGraph(spec, 0, schedule="gemm_pair=1")
+    assert "CTA pairs" in g.plan
+    out = g.run(parity.to_device(spec, t))[0]
+    torch.cuda.synchronize()
+    g.status()
+    ref = oracle.run(spec, parity.oracle_inputs(spec, t))["t2"]
+    assert parity.f32_violation(parity.to_numpy64(out), ref) <= 1.0
+    il = {"kind": "int", "lo": -8, "hi": 8}
+    t = configs.draw_inputs(spec, {"a": il, "b": il, "bias": il}, 1)
+    out = g.run(parity.to_device(spec, t))[0]
+    torch.cuda.synchronize()
+    g.status()
+    np.testing.assert_array_equal(parity.to_numpy64(out), oracle.run(spec, parity.oracle_inputs(spec, t))["t2"])
+
+
 def test_gemm_bf16_integer_inputs_are_exact():
     spec = "hct 1\ninput x bf16 [200,320]\ninput w bf16 [320,264]\nnode y = gemm(x, w)\noutput y f32\n"
     il = {"kind": "int", "lo": -8, "hi": 8}
