@@ -321,7 +321,7 @@ hct_status_t hct_graph_autotune(const char* spec, size_t spec_len, int device, c
                           "row_nv=8;row_cta_small=128", "row_no_stage=1", "row_nv=2;row_minb=2"})
       cands.push_back(c);
   if (has_gemm)
-    for (const char* c : {"gemm_bn=64", "gemm_bn=128", "gemm_bn=32", "gemm_pair=1", "gemm_pair=2"}) cands.insert(cands.begin(), c);
+    for (const char* c : {"gemm_bn=64", "gemm_bn=128", "gemm_bn=32", "gemm_pair=1", "gemm_pair=2", "gemm_insplit=1"}) cands.insert(cands.begin(), c);
   if (has_conv)
     for (const char* c : {"conv_no_tma_store=1", "conv_no_direct=1", "conv_no_direct=1;conv_no_halo=1"}) cands.push_back(c);
 

@@ -322,6 +322,59 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     int64_t M = a.shape[0], K = a.shape[1], N = b.shape[1];
     DType da = g.nodes[anchor.args[0].node].cls == OpClass::Input ? a.dtype : F32;
     DType db = g.nodes[anchor.args[1].node].cls == OpClass::Input ? b.dtype : F32;
+    // On request (schedule knob or tuning): one launch that splits the operands inside the kernel, with no
+    // pre-pass and no scratch.  Not the default: measured, it only ties the two-launch path on 256^3
+    // (16 us both) and loses on larger problems (4096x1024x1024: 115 us against 63 us), the split warps
+    // being the slowest stage of its pipeline.
+    const bool insplit = da == F32 && db == F32 && K % 4 == 0 && N % 4 == 0 && tun.gemm_pair != 1 && tun.gemm_insplit == 1;
+    if (insplit && M <= 0x7fffffff && N <= 0x7fffffff && K <= 0x7fffffff) {
+      const int BN = 64;   // 448 threads share the register file: a 128-column running sum per epilogue thread would spill
+      const int rstages = 3, stages = 3;
+      std::string epi = eg.run_fn(N);
+      KernelSpec k;
+      k.name = "hct_gemm_tc_tf32x3_insplit_g" + std::to_string(gi);
+      std::ostringstream src;
+      src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n#define HCT_BN " << BN
+          << "\n#define HCT_RSTAGES " << rstages << "\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
+          << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
+      src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[2]; void* ptr["
+          << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source("gemm_tc_insplit");
+      k.source = src.str();
+      k.ptrs = eg.ptrs;
+      k.wants_status = true;
+      auto operand_ref = [&](int node) {
+        BufRef r;
+        r.node = node;
+        r.ws_copy = g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0;
+        return r;
+      };
+      TmaDesc ta, tb;
+      ta.buf = operand_ref(anchor.args[0].node);
+      ta.elem_bytes = 4;
+      ta.rank = 2;
+      ta.dims[0] = (uint64_t)K; ta.dims[1] = (uint64_t)M;
+      ta.strides[1] = (uint64_t)K * 4;
+      ta.box[0] = 32; ta.box[1] = 128;
+      tb.buf = operand_ref(anchor.args[1].node);
+      tb.elem_bytes = 4;
+      tb.rank = 2;
+      tb.dims[0] = (uint64_t)N; tb.dims[1] = (uint64_t)K;
+      tb.strides[1] = (uint64_t)N * 4;
+      tb.box[0] = 32; tb.box[1] = 32;
+      tb.swizzle = 0;
+      k.tmaps = {ta, tb};
+      int64_t tiles = ((M + 127) / 128) * ((N + BN - 1) / BN);
+      k.block[0] = 448;
+      k.smem_bytes = (unsigned)(rstages * (16384 + BN * 128) + stages * (2 * 16384 + 2 * BN * 128) + 1024);
+      k.persistent = true;
+      k.max_grid = (unsigned)std::min<int64_t>(tiles, 0x7fffffff);
+      k.grid[0] = k.max_grid;
+      std::ostringstream d;
+      d << "gemm tcgen05 tf32x3 128x" << BN << "x32, operands split in the kernel (" << rstages << " raw + " << stages << " operand stages)";
+      k.desc = d.str();
+      out->push_back(k);
+      return;
+    }
     if (da == F32 && db == F32 && K % 4 == 0 && M <= 0x7fffffff && N <= 0x7fffffff && K <= 0x7fffffff) {
       auto align256 = [](int64_t v) { return (v + 255) / 256 * 256; };
       const int64_t a_bytes = align256(M * K * 4), b_bytes = align256(K * N * 4);

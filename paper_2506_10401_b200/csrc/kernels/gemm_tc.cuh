@@ -70,6 +70,10 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     hct_prefetch_tmap(&hct_p.tmap[0]);
     hct_prefetch_tmap(&hct_p.tmap[1]);
+#if HCT_TF32X3
+    hct_prefetch_tmap(&hct_p.tmap[2]);
+    hct_prefetch_tmap(&hct_p.tmap[3]);
+#endif
   }
   if (warp == 1) hct_tmem_alloc(hct_smem_addr(&tmem_holder), HCT_TMEM_COLS);
   hct_tc_fence_before();

@@ -157,6 +157,29 @@ def test_gemm_bf16_on_cta_pairs(m, k, n):
     np.testing.assert_array_equal(parity.to_numpy64(out), oracle.run(spec, parity.oracle_inputs(spec, t))["y"])
 
 
+@pytest.mark.parametrize("m,k,n", [(300, 1000, 520), (257, 4096, 136), (1, 4, 4), (512, 64, 256), (130, 16384, 72), (1024, 260, 1000), (64, 36, 100)])
+def test_gemm_f32_split_inside_the_kernel(m, k, n):
+    """One launch, no scratch: the kernel splits fp32 operands into TF32 head and tail itself (forced here; by rule for small problems)."""
+    import torch
+    import oracle
+    import paper_2506_10401_b200 as hct
+    spec, laws = configs.get_config("c1_gemm_bias_relu_f32", m=m, k=k, n=n)
+    t = configs.draw_inputs(spec, laws, 0)
+    g = hct.FusedGraph(spec, 0, schedule="gemm_insplit=1")
+    assert "split in the kernel" in g.plan and g.num_kernels == 1 and g.workspace_bytes == 0
+    out = g.run(parity.to_device(spec, t))[0]
+    torch.cuda.synchronize()
+    g.status()
+    ref = oracle.run(spec, parity.oracle_inputs(spec, t))["t2"]
+    assert parity.f32_violation(parity.to_numpy64(out), ref) <= 1.0
+    il = {"kind": "int", "lo": -8, "hi": 8}
+    t = configs.draw_inputs(spec, {"a": il, "b": il, "bias": il}, 1)
+    out = g.run(parity.to_device(spec, t))[0]
+    torch.cuda.synchronize()
+    g.status()
+    np.testing.assert_array_equal(parity.to_numpy64(out), oracle.run(spec, parity.oracle_inputs(spec, t))["t2"])
+
+
 @pytest.mark.parametrize("m,k,n", [(300, 1000, 520), (257, 4096, 136), (5, 8, 3), (512, 64, 256), (130, 16384, 72), (1024, 260, 1000)])
 def test_gemm_f32_on_cta_pairs(m, k, n):
     """The fp32 (three TF32 products) kernel on CTA pairs, forced onto small and ragged shapes."""
