@@ -36,6 +36,7 @@ WORKLOADS = {
     # operator classes beyond the five configurations: a layout transform and the case-study chain with dropout
     "transpose_bias_relu": dict(bound="hbm", sample=dict(r=4096)),
     "matmul_dropout_mean_softmax": dict(bound="tensor", sample=dict(m=1024)),
+    "conv_block": dict(bound="tensor", sample=dict(n=4)),
 }
 HEADLINE = "c2_softmax_layernorm_chain"
 
@@ -408,7 +409,7 @@ def main():
         peak = pk["hbm"] if info["bound"] == "hbm" else (pk["tensor_sustained"] if capped else pk["tensor"])
         line = dict(metric=metric, value=r["value"], unit=r["unit"], n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
                     ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
-                    dtype="bf16" if ("bf16" in name or name == "matmul_dropout_mean_softmax") else "f32", data="synthetic",
+                    dtype="bf16" if ("bf16" in name or name in ("matmul_dropout_mean_softmax", "conv_block")) else "f32", data="synthetic",
                     config={"workload": name, "l2": "flushed between steps (192 MB write, untimed)", "kernels_per_step": r["kernels"],
                             "parallelism": "replicas" if world > 1 else "single",
                             "schedule": r["schedule"] or "default", "tuned_trials": args.tune},

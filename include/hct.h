@@ -22,6 +22,8 @@
  *     output NAME [DTYPE]                     stored dtype, default f32
  *
  *   unary   relu gelu_tanh gelu_erf sigmoid exp tanh sqrt sin cos neg abs
+ *           cast_bf16(x)   rounds to bfloat16 (nearest even); the result may be the first operand of a bf16
+ *           gemm / conv2d and is kept as bf16 where it is materialised between kernels
  *           dropout(x, p=0.5, seed=0)   inverted dropout with the counter-based mask of the
  *           paper's first case study (Section 5.4): with i the element's row-major offset,
  *           h = i + seed; h ^= h >> 17; h ^= h << 31; h ^= h >> 8 (unsigned 64 bit); the

@@ -181,6 +181,12 @@ def _infer(g, name, op, pos, attrs, where):
             if k not in allowed:
                 raise SpecError(f"{where}: unknown attribute {k!r} for {op}")
 
+    if op == "cast_bf16":
+        only_attrs()
+        if len(pos) != 1:
+            raise SpecError(f"{where}: cast_bf16 takes one operand")
+        a = _operand(g, pos[0], where, False)
+        return Node(name, op, [a], {}, shape_of(a), "bf16")
     if op == "dropout":
         only_attrs("p", "seed")
         if len(pos) != 1:

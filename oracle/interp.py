@@ -50,6 +50,15 @@ _BINARY_FN = {
 }
 
 
+def cast_bf16(x):
+    """Rounds to bfloat16, nearest even: the value is first taken to float32 (the width every computed
+    value has on the device), then its low 16 bits are rounded away."""
+    u = np.asarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    r = ((u + np.uint64(0x7FFF) + ((u >> np.uint64(16)) & np.uint64(1))) >> np.uint64(16)) << np.uint64(16)
+    y = r.astype(np.uint32).view(np.float32).astype(np.float64)
+    return np.where(np.isfinite(x), y, x)
+
+
 def dropout_keep_mask(shape, seed: int, p: float):
     """Which elements inverted dropout keeps (the paper's first case study, Section 5.4).
 
@@ -177,7 +186,9 @@ def run_nodes(spec, inputs: dict, dtype=np.float64, gemm_fn=None) -> dict:
             continue
         args = [val[a] if isinstance(a, str) else float(a) for a in node.args]
         op = node.op
-        if op == "dropout":
+        if op == "cast_bf16":
+            out = cast_bf16(args[0])
+        elif op == "dropout":
             out = dropout(args[0], node.attrs["p"], node.attrs["seed"])
         elif op in UNARY:
             out = _UNARY_FN[op](args[0])

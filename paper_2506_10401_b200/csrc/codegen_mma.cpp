@@ -27,7 +27,7 @@ struct EpiGen {
     ptrs.push_back(b);
     return (int)ptrs.size() - 1;
   }
-  DType buf_dtype(int node) const { return g.nodes[node].cls == OpClass::Input ? g.nodes[node].dtype : F32; }
+  DType buf_dtype(int node) const { return g.nodes[node].dtype; }   // inputs: as declared; computed values: fp32, or bf16 after a cast
   bool is_ws(int node) const { return g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0; }
 
   // Scalar epilogue: value `acc` of element at linear offset `off`, per-row index `ri`
@@ -224,8 +224,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
   // ---- tensor-core GEMM: bf16 operands straight from their buffers
   if (grp.kind == GroupKind::Gemm && !tun.simt_only) {
     int64_t M = a.shape[0], K = a.shape[1], N = b.shape[1];
-    DType da = g.nodes[anchor.args[0].node].cls == OpClass::Input ? a.dtype : F32;
-    DType db = g.nodes[anchor.args[1].node].cls == OpClass::Input ? b.dtype : F32;
+    DType da = a.dtype, db = b.dtype;
     // CTA pairs on 256 x 256 tiles when every pair of SMs gets at least one tile
     const int64_t pair_tiles = ((M + 255) / 256) * ((N + 255) / 256);
     const bool use_pair = tun.gemm_pair == 1 || (tun.gemm_pair == 0 && pair_tiles >= 74 && !tun.fault_never_arrive && tun.gemm_bn == 0);
@@ -246,12 +245,14 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       k.wants_status = true;
       TmaDesc ta, tb;
       ta.buf.node = anchor.args[0].node;
+      ta.buf.ws_copy = a.cls != OpClass::Input && p.ws_offset[anchor.args[0].node] >= 0;
       ta.elem_bytes = 2;
       ta.rank = 2;
       ta.dims[0] = (uint64_t)K; ta.dims[1] = (uint64_t)M;
       ta.strides[1] = (uint64_t)K * 2;
       ta.box[0] = 64; ta.box[1] = 128;
       tb.buf.node = anchor.args[1].node;
+      tb.buf.ws_copy = b.cls != OpClass::Input && p.ws_offset[anchor.args[1].node] >= 0;
       tb.elem_bytes = 2;
       tb.rank = 2;
       tb.dims[0] = (uint64_t)N; tb.dims[1] = (uint64_t)K;
@@ -291,12 +292,14 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       k.wants_status = true;
       TmaDesc ta, tb;
       ta.buf.node = anchor.args[0].node;
+      ta.buf.ws_copy = a.cls != OpClass::Input && p.ws_offset[anchor.args[0].node] >= 0;
       ta.elem_bytes = 2;
       ta.rank = 2;
       ta.dims[0] = (uint64_t)K; ta.dims[1] = (uint64_t)M;
       ta.strides[1] = (uint64_t)K * 2;
       ta.box[0] = 64; ta.box[1] = 128;
       tb.buf.node = anchor.args[1].node;
+      tb.buf.ws_copy = b.cls != OpClass::Input && p.ws_offset[anchor.args[1].node] >= 0;
       tb.elem_bytes = 2;
       tb.rank = 2;
       tb.dims[0] = (uint64_t)N; tb.dims[1] = (uint64_t)K;
@@ -320,8 +323,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
   // ---- tensor-core GEMM on fp32 operands: split pre-pass, then three TF32 products per k step
   if (grp.kind == GroupKind::Gemm && !tun.simt_only) {
     int64_t M = a.shape[0], K = a.shape[1], N = b.shape[1];
-    DType da = g.nodes[anchor.args[0].node].cls == OpClass::Input ? a.dtype : F32;
-    DType db = g.nodes[anchor.args[1].node].cls == OpClass::Input ? b.dtype : F32;
+    DType da = a.dtype, db = b.dtype;
     // On request (schedule knob or tuning): one launch that splits the operands inside the kernel, with no
     // pre-pass and no scratch.  Not the default: measured, it only ties the two-launch path on 256^3
     // (16 us both) and loses on larger problems (4096x1024x1024: 115 us against 63 us), the split warps
@@ -494,7 +496,8 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
   if (grp.kind == GroupKind::Conv && !tun.simt_only) {
     const auto& xs = a.shape;
     const auto& ws = b.shape;
-    bool in_bf16 = a.cls == OpClass::Input && b.cls == OpClass::Input && a.dtype == BF16 && b.dtype == BF16;
+    // weights must be a graph input (they take a layout pre-pass); the activations may be an earlier kernel's bf16 result
+    bool in_bf16 = b.cls == OpClass::Input && a.dtype == BF16 && b.dtype == BF16;
     int64_t NB = xs[0], C = xs[1], H = xs[2], W = xs[3], KO = ws[0], FR = ws[2], FS = ws[3];
     int64_t HO = anchor.shape[2], WO = anchor.shape[3];
     if (in_bf16 && anchor.stride == 1 && C % 8 == 0 && WO <= 256 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
@@ -509,9 +512,8 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       int n_a = 0;
       bool direct = false;
       // The epilogue of the NCHW-reading kernel hands its bf16 output to TMA stores (through 16 KB of
-      // shared memory) when there is a single bf16 graph output whose rows are 16-byte multiples.
-      const bool tma_store = grp.stores.size() == 1 && grp.stores[0].to_output && grp.stores[0].dtype == BF16 && WO % 8 == 0 &&
-                             !tun.conv_no_tma_store;
+      // shared memory) when it stores a single bf16 tensor (output or intermediate) whose rows are 16-byte multiples.
+      const bool tma_store = grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && WO % 8 == 0 && !tun.conv_no_tma_store;
       if (dense_pitch && W % 8 == 0 && !tun.conv_no_direct) {
         // shared memory: operand buffers of TH + FR - 1 rows, staging ring, output staging, and what is left for the weight ring
         const int64_t fixed = n_buf * ((th_pitch + FR - 1) * pitch * 128 + 1024) + n_stg * pitch * 128 + 1024 + (tma_store ? 16384 : 0);
@@ -532,6 +534,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       auto node_buf = [&](int node) {
         BufRef r;
         r.node = node;
+        r.ws_copy = g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0;
         return r;
       };
       {
@@ -559,7 +562,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
           << "\n#define HCT_KO " << KO << "\n#define HCT_FR " << FR << "\n#define HCT_FS " << FS << "\n#define HCT_PAD " << anchor.pad
           << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TH " << TH << "\n#define HCT_TH2 1\n#define HCT_SPLIT "
           << TH << "\n#define HCT_PITCH " << pitch << "\n#define HCT_NA " << (direct ? n_a : 6) << "\n#define HCT_NBUF " << (direct ? n_buf : 3)
-          << "\n#define HCT_NSTG " << n_stg << "\n#define HCT_TMA_STORE " << (use_tma_store ? 1 : 0) << "\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
+          << "\n#define HCT_NSTG " << n_stg << "\n#define HCT_X_IS_INPUT " << (a.cls == OpClass::Input ? 1 : 0) << "\n#define HCT_TMA_STORE " << (use_tma_store ? 1 : 0) << "\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
           << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
       src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[" << (use_tma_store ? 3 : direct ? 2 : 3)
           << "]; void* ptr[" << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source(direct ? "conv_tc_nchw" : halo ? "conv_tc_halo" : "conv_tc");
@@ -596,6 +599,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         if (use_tma_store) {  // NCHW output: [32 channels x 32 pixels] of one row, 64-byte swizzle
           TmaDesc ty;
           ty.buf.node = grp.stores[0].node;
+          ty.buf.ws_copy = !grp.stores[0].to_output;
           ty.elem_bytes = 2;
           ty.rank = 4;
           ty.dims[0] = (uint64_t)WO; ty.dims[1] = (uint64_t)HO; ty.dims[2] = (uint64_t)KO; ty.dims[3] = (uint64_t)NB;

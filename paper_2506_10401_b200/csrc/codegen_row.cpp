@@ -131,7 +131,7 @@ struct RowGen {
   }
 
   // storage dtype of a buffer this group reads
-  DType ext_dtype(int node) const { return g.nodes[node].cls == OpClass::Input ? g.nodes[node].dtype : F32; }
+  DType ext_dtype(int node) const { return g.nodes[node].dtype; }   // inputs: as declared; computed values: fp32, or bf16 after a cast
   bool ext_is_ws(int node) const { return g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0; }
 
   // expression for operand `a` inside loops over b (row of the batch) and, in full-width context, e

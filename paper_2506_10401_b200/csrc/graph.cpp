@@ -226,7 +226,16 @@ Graph parse_spec(const std::string& text) {
       n.name = name;
       n.op = op;
       n.dtype = F32;
-      if (op == "dropout") {
+      if (op == "cast_bf16") {
+        // rounds to bfloat16 (nearest even); the value may then feed a bf16 gemm / conv2d, and is kept as
+        // bf16 when it has to be materialised between kernels
+        only_attrs({});
+        if (pos.size() != 1) fail(HCT_ERR_GRAPH, line, "cast_bf16 takes one operand");
+        n.cls = OpClass::Unary;
+        n.args = {lookup(pos[0], line, false)};
+        n.shape = g.nodes[n.args[0].node].shape;
+        n.dtype = BF16;
+      } else if (op == "dropout") {
         // Inverted dropout with a counter-based mask (the hash generator of the paper's first case study):
         // h = i + seed; h ^= h >> 17; h ^= h << 31; h ^= h >> 8 in 64-bit arithmetic, i the element's
         // row-major offset; the element is kept, scaled by 1/(1-p), when h mod 1000 >= round(1000 p).

@@ -28,7 +28,7 @@ struct Node {
   OpClass cls = OpClass::Input;
   std::vector<Operand> args;
   std::vector<int64_t> shape;
-  DType dtype = F32;  // storage dtype of an input; computed nodes are fp32 values
+  DType dtype = F32;  // storage dtype of an input; computed nodes are fp32 values (BF16: values rounded to bfloat16 by cast_bf16)
   double eps = 1e-5;
   int stride = 1, pad = 0;
   // dropout: element with flat index i is kept when hash(i + seed) mod 1000 >= drop_threshold (= round(1000 p))

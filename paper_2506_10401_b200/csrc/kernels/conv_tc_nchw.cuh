@@ -20,11 +20,11 @@
 // Columns w >= HCT_WO of each pitch are computed and dropped.
 //
 // Warps: 0 weight producer, 1 MMA issue, 2-5 epilogue, 6 pixel producer, 7-14 transposers.
-// The activations are a graph input, so only the weight producer and the epilogue wait for the
-// preceding kernel (programmatic dependent launch); the pixel pipeline fills meanwhile.
+// When the activations are a graph input (HCT_X_IS_INPUT) only the weight producer and the epilogue
+// wait for the preceding kernel (programmatic dependent launch) and the pixel pipeline fills meanwhile.
 //
 // Defined by the generator: HCT_NB_IMG, HCT_C, HCT_H, HCT_W, HCT_KO, HCT_FR, HCT_FS, HCT_PAD, HCT_HO, HCT_WO,
-// HCT_PITCH, HCT_TH, HCT_TH2 (= 1), HCT_SPLIT, HCT_NA, HCT_NBUF, HCT_NSTG, HCT_TMA_STORE, HCT_STATUS_SLOT,
+// HCT_PITCH, HCT_TH, HCT_TH2 (= 1), HCT_SPLIT, HCT_NA, HCT_NBUF, HCT_NSTG, HCT_X_IS_INPUT, HCT_TMA_STORE, HCT_STATUS_SLOT,
 // HCT_KERNEL_NAME, HctParams, hct_epilogue_run() or (HCT_TMA_STORE) hct_epilogue_vals().
 #define HCT_BM 128
 #define HCT_A_BYTES (HCT_BM * 128)                       // weights: 128 channels x 64 inputs, bf16
@@ -246,6 +246,9 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(co
   } else if (warp == 6) {
     // ---- pixels: one staged box per (channel block, input row)
     if (lane == 0) {
+#if !HCT_X_IS_INPUT
+      hct_pdl_wait();   // the activations are an earlier kernel's result
+#endif
       int ss = 0;
       hct_u32 ps = 0;
       for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {

@@ -189,12 +189,13 @@ Plan make_plan(const Graph& g) {
     Group& grp = p.groups[p.group_of[i]];
     bool out = nd.output_index >= 0;
     // consumers always read fp32; an output stored as bf16 cannot serve them
-    bool need_ws = cross[i] && !(out && nd.out_dtype == F32);
+    bool need_ws = cross[i] && !(out && nd.out_dtype == nd.dtype);   // an output of the value's own width serves its consumers too
     if (out) grp.stores.push_back({i, nd.out_dtype, true});
     if (need_ws) {
+      // intermediates are fp32, except values a cast has rounded to bf16, which keep that width
       p.ws_offset[i] = (int64_t)ws;
-      ws += ((size_t)nd.numel() * 4 + 255) / 256 * 256;
-      grp.stores.push_back({i, F32, false});
+      ws += ((size_t)nd.numel() * (nd.dtype == BF16 ? 2 : 4) + 255) / 256 * 256;
+      grp.stores.push_back({i, nd.dtype, false});
     }
   }
   p.workspace_bytes = ws;
@@ -224,7 +225,7 @@ Plan make_plan(const Graph& g) {
                                 nd.shape.back() > 512;
         unavoidable = unavoidable || into_contraction || from_contraction;
       }
-    if (unavoidable) p.algorithmic_bytes += 8.0 * nd.numel();
+    if (unavoidable) p.algorithmic_bytes += (nd.dtype == BF16 ? 4.0 : 8.0) * nd.numel();
   }
 
   std::ostringstream os;

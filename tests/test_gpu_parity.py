@@ -244,6 +244,38 @@ def test_conv_bf16_nchw_direct_integer_inputs_are_exact():
     np.testing.assert_array_equal(got[0], want[0])
 
 
+# ------------------------------------------------------------------ stacked contractions through bf16 intermediates
+
+@pytest.mark.parametrize("kw", [dict(n=2, c=64, h=20, w=24, k=64), dict(n=1, c=128, h=56, w=56, k=128), dict(n=2, c=16, h=9, w=11, k=32)])
+def test_conv_block_keeps_bf16_activations_on_the_device(kw):
+    spec, laws = configs.get_config("conv_block", **kw)
+    got, want, g = parity.run_both(spec, laws)
+    assert g.plan.count("tcgen05") == 2       # both convolutions on tensor cores
+    assert parity.bf16_violation(got[0], want[0]) <= 1.0
+
+
+def test_gemm_chain_through_cast_bf16():
+    spec = """hct 1
+input x  bf16 [300,264]
+input w1 bf16 [264,520]
+input b1 bf16 [520]
+input w2 bf16 [520,136]
+node h0 = gemm(x, w1)
+node h1 = add(h0, b1)
+node h2 = gelu_tanh(h1)
+node h3 = cast_bf16(h2)
+node y  = gemm(h3, w2)
+output y f32
+output h3 bf16
+"""
+    n = {"kind": "normal", "mean": 0.0, "std": 1.0}
+    got, want, g = parity.run_both(spec, {"x": n, "w1": {"kind": "normal", "mean": 0.0, "std": 0.06}, "b1": n,
+                                          "w2": {"kind": "normal", "mean": 0.0, "std": 0.04}})
+    assert g.plan.count("tcgen05") == 2 and g.num_kernels == 2
+    assert parity.bf16_violation(got[0], want[0]) <= 1.0
+    assert parity.bf16_violation(got[1], want[1]) <= 1.0
+
+
 # ------------------------------------------------------------------ layout transform
 
 @pytest.mark.parametrize("r,c", [(37, 1000), (300, 4096), (5, 1023), (1, 7), (64, 64), (129, 65), (2048, 2048)])

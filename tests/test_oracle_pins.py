@@ -341,6 +341,22 @@ def test_parse_rejects(bad):
         oracle.parse(bad)
 
 
+def test_cast_bf16_pins():
+    # exactly representable values pass through; ties go to the even neighbour; 8 significant bits remain
+    x = np.array([1.0, -2.5, 0.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -7, 3.0e38, -1e-30])
+    y = interp.cast_bf16(x)
+    assert y[0] == 1.0 and y[1] == -2.5 and y[2] == 0.0
+    assert y[3] == 1.0                      # tie between 1 and 1 + 2^-7: even mantissa wins
+    assert y[4] == 1.0 + 2.0 ** -6          # tie between 1 + 2^-7 and 1 + 2^-6: even again
+    assert y[5] == 1.0 + 2.0 ** -7
+    t = torch.tensor(x, dtype=torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    np.testing.assert_array_equal(y, t)
+    z = RNG.normal(size=1000) * 10.0 ** RNG.integers(-5, 5, size=1000)
+    np.testing.assert_array_equal(interp.cast_bf16(z), torch.tensor(z, dtype=torch.float32).to(torch.bfloat16).to(torch.float64).numpy())
+    assert np.all(np.abs(interp.cast_bf16(z) - z) <= np.abs(z) * 2.0 ** -8)
+    np.testing.assert_array_equal(interp.cast_bf16(interp.cast_bf16(z)), interp.cast_bf16(z))   # idempotent
+
+
 def test_transpose_pins():
     x = RNG.normal(size=(5, 9))
     spec = "hct 1\ninput x f32 [5,9]\nnode t = transpose(x)\nnode u = transpose(t)\noutput t\noutput u\n"

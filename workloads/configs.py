@@ -104,6 +104,33 @@ output t2 f32
     return spec, laws
 
 
+def conv_block(n=32, c=128, h=56, w=56, k=128):
+    """Two stacked conv3x3 -> folded batch norm -> ReLU stages (a VGG-style block): the first stage's
+    activations are rounded to bf16 and feed the second convolution without leaving the device."""
+    spec = f"""hct 1
+input x  bf16 [{n},{c},{h},{w}]
+input w1 bf16 [{k},{c},3,3]
+input s1 f32  [{k},1,1]
+input b1 f32  [{k},1,1]
+input w2 bf16 [{k},{k},3,3]
+input s2 f32  [{k},1,1]
+input b2 f32  [{k},1,1]
+node  a0 = conv2d(x, w1, stride=1, pad=1)
+node  a1 = mul(a0, s1)
+node  a2 = add(a1, b1)
+node  a3 = relu(a2)
+node  a4 = cast_bf16(a3)
+node  c0 = conv2d(a4, w2, stride=1, pad=1)
+node  c1 = mul(c0, s2)
+node  c2 = add(c1, b2)
+node  c3 = relu(c2)
+output c3 bf16
+"""
+    laws = {"x": _n(), "w1": _n(math.sqrt(2.0 / (c * 9))), "s1": _u(0.5, 1.5), "b1": _n(0.1),
+            "w2": _n(math.sqrt(2.0 / (k * 9))), "s2": _u(0.5, 1.5), "b2": _n(0.1)}
+    return spec, laws
+
+
 def transpose_bias_relu(r=16384, c=4096):
     """A layout transform with fused consumers (Table 1, "LayoutTransform"): y = relu(x^T + bias)."""
     spec = f"""hct 1
@@ -125,6 +152,7 @@ CONFIGS = {
     "c4_conv_bn_relu_bf16": (conv_bn_relu, {}),
     "matmul_dropout_mean_softmax": (matmul_dropout_mean_softmax, {}),
     "transpose_bias_relu": (transpose_bias_relu, {}),
+    "conv_block": (conv_block, {}),
 }
 
 
