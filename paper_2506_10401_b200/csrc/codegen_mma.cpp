@@ -415,12 +415,12 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       if (tun.gemm_bn >= 32) BN = std::min(bn_max, tun.gemm_bn >= 128 ? 128 : tun.gemm_bn >= 64 ? 64 : 32);
       int stages = BN == 128 ? 3 : BN == 64 ? 4 : 5;
       std::string epi = eg.run_fn(N);
-      // CTA pairs on 256 x 128 tiles: only on request (schedule knob or tuning).  Measured on
-      // 16384 x 4096 x 4096 it equals the single-CTA kernel (2.89 ms against 2.88 ms): these long fp32
-      // GEMMs run at the power cap, not at the shared-memory bound the pairing relieves.
-      const int64_t pair_tiles32 = ((M + 255) / 256) * ((N + 127) / 128);
-      if (tun.gemm_pair == 1) {
-        const int pstages = 4;
+      // CTA pairs on 256 x 256 tiles when every pair of SMs gets at least one tile.  Measured on
+      // 16384 x 4096 x 4096: 2.31 ms against 2.93 ms for 128 x 128 tiles on single CTAs (a TF32 MMA of
+      // 128 columns does not fill the tensor pipe's issue interval; 256 columns per instruction do).
+      const int64_t pair_tiles32 = ((M + 255) / 256) * ((N + 255) / 256);
+      if (tun.gemm_pair == 1 || (tun.gemm_pair == 0 && pair_tiles32 >= 74 && tun.gemm_bn == 0)) {
+        const int pstages = 3;
         KernelSpec k;
         k.name = "hct_gemm_tc2_tf32x3_g" + std::to_string(gi);
         std::ostringstream src;
@@ -438,16 +438,16 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
           t.rank = 2;
           t.dims[0] = (uint64_t)K; t.dims[1] = (uint64_t)(i < 2 ? M : N);   // B is transposed to [N,K]
           t.strides[1] = (uint64_t)K * 4;
-          t.box[0] = 32; t.box[1] = i < 2 ? 128 : 64;
+          t.box[0] = 32; t.box[1] = 128;
           k.tmaps.push_back(t);
         }
-        k.block[0] = 192;
-        k.smem_bytes = (unsigned)(pstages * 49152 + 1024);
+        k.block[0] = 320;
+        k.smem_bytes = (unsigned)(pstages * 65536 + 1024);
         k.persistent = true;
         k.cluster = 2;
         k.max_grid = (unsigned)std::min<int64_t>(2 * pair_tiles32, 0x7ffffffe);
         k.grid[0] = k.max_grid;
-        k.desc = "gemm tcgen05 tf32x3 on CTA pairs, 256x128x32 per pair, " + std::to_string(pstages) + " stages";
+        k.desc = "gemm tcgen05 tf32x3 on CTA pairs, 256x256x32 per pair, " + std::to_string(pstages) + " stages";
         out->push_back(k);
         return;
       }

@@ -14,23 +14,26 @@
 // by two tcgen05.commit (one per CTA) from the issuing thread.  tempty[a] lives in the even CTA and
 // counts the epilogue threads of both.  No load is multicast.  All waits are bounded.
 //
-// The fp32 variant (HCT_TF32X3) works on 256 x 128 tiles per pair from the head/tail operands its
+// The fp32 variant (HCT_TF32X3) works on 256 x 256 tiles per pair from the head/tail operands its
 // split pre-pass wrote (B transposed to [N,K]): three TF32 products per k step, at most 128 elements
 // of K accumulated in tensor memory and those chunks summed in registers, exactly as in the
-// single-CTA kernel; each CTA stages 128 rows of A and 64 rows of B^T (48 KB per 32-deep stage).
+// single-CTA kernel; each CTA stages 128 rows of A and 128 rows of B^T (64 KB per 32-deep stage), and
+// eight epilogue warps share the running sums (128 columns each).
 //
 // Defined by the generator: HCT_M, HCT_N, HCT_K, HCT_STAGES, HCT_TF32X3 (0/1), HCT_STATUS_SLOT,
 // HCT_KERNEL_NAME, HctParams, hct_epilogue_run().
 #if HCT_TF32X3
 #define HCT_BK 32
-#define HCT_BNP 128                             // tile columns per pair
+#define HCT_BNP 256                             // tile columns per pair
 #define HCT_A_BYTES 16384                       // 128 rows x 32 k, fp32 (head; the tail follows)
-#define HCT_B_BYTES 8192                        // 64 rows of B^T x 32 k, fp32
+#define HCT_B_BYTES 16384                       // 128 rows of B^T x 32 k, fp32
+#define HCT_EPI_WARPS 8                         // two warps per lane quarter: 128 columns of the running sum each
 #define HCT_STAGE_BYTES (2 * HCT_A_BYTES + 2 * HCT_B_BYTES)
 #define HCT_KBC 4                               // k blocks accumulated in tensor memory before the chunk is drained
 #else
 #define HCT_BK 64
 #define HCT_BNP 256
+#define HCT_EPI_WARPS 4
 #define HCT_A_BYTES 16384                       // 128 rows x 64 k, bf16
 #define HCT_B_BYTES 16384                       // 64 k x 128 columns, bf16 (two 64-column boxes)
 #define HCT_STAGE_BYTES (HCT_A_BYTES + HCT_B_BYTES)
@@ -43,7 +46,7 @@
 #define HCT_TILES ((long long)HCT_MB * HCT_NB)
 #define HCT_TMEM_COLS (2 * HCT_BNP)
 
-extern "C" __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __grid_constant__ HctParams hct_p) {
+extern "C" __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(64 + 32 * HCT_EPI_WARPS, 1) HCT_KERNEL_NAME(const __grid_constant__ HctParams hct_p) {
   extern __shared__ unsigned char hct_smem_raw[];
   __shared__ unsigned long long bars[2 * HCT_STAGES + 4];
   __shared__ hct_u32 tmem_holder;
@@ -65,7 +68,7 @@ extern "C" __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1) H
     }
     for (int a = 0; a < 2; ++a) {
       hct_mbar_init(tfull0 + 8 * a, 1);
-      hct_mbar_init(tempty0 + 8 * a, 256);   // the epilogue threads of both CTAs
+      hct_mbar_init(tempty0 + 8 * a, 64 * HCT_EPI_WARPS);   // the epilogue threads of both CTAs
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     hct_prefetch_tmap(&hct_p.tmap[0]);
@@ -99,8 +102,8 @@ extern "C" __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1) H
           hct_tma_load_2d_pair(dst, &hct_p.tmap[0], kb * HCT_BK, mb * 256 + (int)rank * 128, full_even);                     // A head
           hct_tma_load_2d_pair(dst + HCT_A_BYTES, &hct_p.tmap[1], kb * HCT_BK, mb * 256 + (int)rank * 128, full_even);       // A tail
           dst += 2 * HCT_A_BYTES;
-          hct_tma_load_2d_pair(dst, &hct_p.tmap[2], kb * HCT_BK, nb * HCT_BNP + (int)rank * 64, full_even);                  // B^T head
-          hct_tma_load_2d_pair(dst + HCT_B_BYTES, &hct_p.tmap[3], kb * HCT_BK, nb * HCT_BNP + (int)rank * 64, full_even);    // B^T tail
+          hct_tma_load_2d_pair(dst, &hct_p.tmap[2], kb * HCT_BK, nb * HCT_BNP + (int)rank * 128, full_even);                  // B^T head
+          hct_tma_load_2d_pair(dst + HCT_B_BYTES, &hct_p.tmap[3], kb * HCT_BK, nb * HCT_BNP + (int)rank * 128, full_even);    // B^T tail
 #else
           hct_tma_load_2d_pair(dst, &hct_p.tmap[0], kb * 64, mb * 256 + (int)rank * 128, full_even);
           dst += HCT_A_BYTES;
@@ -186,17 +189,20 @@ extern "C" __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1) H
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
 #else
-      float sum[HCT_BNP];
+      // this warp's share of the columns: HCT_BNP / (HCT_EPI_WARPS / 4) starting at c0 chunks of 32
+      constexpr int NCW = HCT_BNP / 32 / (HCT_EPI_WARPS / 4);
+      const int c0 = ((warp - 2) >> 2) * NCW;
+      float sum[NCW * 32];
 #pragma unroll
-      for (int j = 0; j < HCT_BNP; ++j) sum[j] = 0.0f;
+      for (int j = 0; j < NCW * 32; ++j) sum[j] = 0.0f;
 #pragma unroll 1
       for (int ch = 0; ch < HCT_NCH; ++ch) {
         hct_mbar_wait(tfull0 + 8 * acc, acc_phase, &failed, status, 4);
         hct_tc_fence_after();
 #pragma unroll
-        for (int c = 0; c < HCT_BNP / 32; ++c) {
+        for (int c = 0; c < NCW; ++c) {
           float v[32];
-          hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * HCT_BNP + c * 32, v);
+          hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * HCT_BNP + (c0 + c) * 32, v);
 #pragma unroll
           for (int j = 0; j < 32; ++j) sum[c * 32 + j] += v[j];
         }
@@ -206,8 +212,8 @@ extern "C" __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1) H
         if (acc == 0) acc_phase ^= 1u;
       }
 #pragma unroll
-      for (int c = 0; c < HCT_BNP / 32; ++c) {
-        const long long col0 = (long long)nb * HCT_BNP + c * 32;
+      for (int c = 0; c < NCW; ++c) {
+        const long long col0 = (long long)nb * HCT_BNP + (c0 + c) * 32;
         const int ncols = (int)(HCT_N - col0 < 32 ? HCT_N - col0 : 32);
         if (row < HCT_M && ncols > 0) hct_epilogue_run(hct_p, *(float(*)[32])(sum + c * 32), row, (int)col0, ncols);
       }
