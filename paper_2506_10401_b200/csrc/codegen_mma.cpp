@@ -419,7 +419,8 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       // 16384 x 4096 x 4096: 2.31 ms against 2.93 ms for 128 x 128 tiles on single CTAs (a TF32 MMA of
       // 128 columns does not fill the tensor pipe's issue interval; 256 columns per instruction do).
       const int64_t pair_tiles32 = ((M + 255) / 256) * ((N + 255) / 256);
-      if (tun.gemm_pair == 1 || (tun.gemm_pair == 0 && pair_tiles32 >= 74 && tun.gemm_bn == 0)) {
+      // (from 56 tiles on, and a contraction deep enough to amortise the pair's set-up: measured break-even)
+      if (tun.gemm_pair == 1 || (tun.gemm_pair == 0 && pair_tiles32 >= 56 && K >= 512 && tun.gemm_bn == 0)) {
         const int pstages = 3;
         KernelSpec k;
         k.name = "hct_gemm_tc2_tf32x3_g" + std::to_string(gi);
