@@ -67,15 +67,15 @@ def bf16_violation(got, ref):
     return float((np.abs(got - ref) / (TOL_BF16_ABS + TOL_BF16_REL * np.abs(ref))).max())
 
 
-def run_both(spec, laws, seed=0, device=0):
-    """Runs the CUDA library and the oracle on the same seeded inputs.
+def run_both(spec, laws, seed=0, device=0, schedule=None):
+    """Runs the CUDA library (optionally under a schedule text) and the oracle on the same seeded inputs.
     Returns (list of GPU outputs as float64 arrays, list of oracle outputs, FusedGraph)."""
     import torch
     import oracle
     import paper_2506_10401_b200 as hct
     t = configs.draw_inputs(spec, laws, seed)
     ref = oracle.run(spec, oracle_inputs(spec, t))
-    g = hct.FusedGraph(spec, device)
+    g = hct.FusedGraph(spec, device, schedule=schedule)
     outs = g.run(to_device(spec, t, f"cuda:{device}"))
     torch.cuda.synchronize(device)
     g.status()
