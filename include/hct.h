@@ -21,7 +21,7 @@
  *     node   NAME = OP(arg, ..., key=value)   args: earlier names or (binary ops) a number
  *     output NAME [DTYPE]                     stored dtype, default f32
  *
- *   unary   relu gelu_tanh gelu_erf sigmoid exp tanh sqrt sin cos neg abs
+ *   unary   relu gelu_tanh gelu_erf sigmoid exp tanh sqrt sin cos neg abs log rsqrt square reciprocal
  *           cast_bf16(x)   rounds to bfloat16 (nearest even); the result may be the first operand of a bf16
  *           gemm / conv2d and is kept as bf16 where it is materialised between kernels
  *           dropout(x, p=0.5, seed=0)   inverted dropout with the counter-based mask of the

@@ -16,7 +16,8 @@ class SpecError(ValueError):
     pass
 
 
-UNARY = ("relu", "gelu_tanh", "gelu_erf", "sigmoid", "exp", "tanh", "sqrt", "sin", "cos", "neg", "abs")
+UNARY = ("relu", "gelu_tanh", "gelu_erf", "sigmoid", "exp", "tanh", "sqrt", "sin", "cos", "neg", "abs", "log", "rsqrt", "square",
+         "reciprocal")
 BINARY = ("add", "sub", "mul", "div", "max", "min")
 ROW_TO_ROW = ("row_softmax",)
 ROW_TO_COL = ("row_sum", "row_mean", "row_max", "row_min", "row_argmax", "row_argmin")

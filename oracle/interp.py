@@ -42,7 +42,8 @@ def gelu_erf(x):
 _UNARY_FN = {
     "relu": relu, "gelu_tanh": gelu_tanh, "gelu_erf": gelu_erf, "sigmoid": sigmoid,
     "exp": np.exp, "tanh": np.tanh, "sqrt": np.sqrt, "sin": np.sin, "cos": np.cos,
-    "neg": np.negative, "abs": np.abs,
+    "neg": np.negative, "abs": np.abs, "log": np.log, "rsqrt": lambda x: 1.0 / np.sqrt(x), "square": lambda x: x * x,
+    "reciprocal": lambda x: 1.0 / x,
 }
 _BINARY_FN = {
     "add": np.add, "sub": np.subtract, "mul": np.multiply, "div": np.divide,

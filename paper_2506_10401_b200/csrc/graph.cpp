@@ -14,7 +14,8 @@
 
 namespace hct {
 
-static const char* kUnary[] = {"relu", "gelu_tanh", "gelu_erf", "sigmoid", "exp", "tanh", "sqrt", "sin", "cos", "neg", "abs"};
+static const char* kUnary[] = {"relu", "gelu_tanh", "gelu_erf", "sigmoid", "exp", "tanh", "sqrt", "sin", "cos", "neg", "abs",
+                               "log", "rsqrt", "square", "reciprocal"};
 static const char* kBinary[] = {"add", "sub", "mul", "div", "max", "min"};
 
 bool is_unary(const std::string& op) {

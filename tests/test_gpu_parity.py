@@ -50,10 +50,11 @@ def test_two_column_rows():
     check_f32(spec, {"x": N_})
 
 
-@pytest.mark.parametrize("op", ["relu", "gelu_tanh", "gelu_erf", "sigmoid", "exp", "tanh", "sqrt", "sin", "cos", "neg", "abs"])
+@pytest.mark.parametrize("op", ["relu", "gelu_tanh", "gelu_erf", "sigmoid", "exp", "tanh", "sqrt", "sin", "cos", "neg", "abs", "log", "rsqrt",
+                                "square", "reciprocal"])
 def test_unary(op):
     spec = f"hct 1\ninput x f32 [67,200]\nnode y = {op}(x)\noutput y\n"
-    check_f32(spec, {"x": POS_ if op == "sqrt" else N_})
+    check_f32(spec, {"x": POS_ if op in ("sqrt", "log", "rsqrt", "reciprocal") else N_})
 
 
 @pytest.mark.parametrize("op", ["add", "sub", "mul", "div", "max", "min"])

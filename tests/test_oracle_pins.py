@@ -89,9 +89,10 @@ def _spec1(op, shape="[3,4]"):
 
 
 @pytest.mark.parametrize("op,fn", [("exp", math.exp), ("tanh", math.tanh), ("sin", math.sin), ("cos", math.cos),
-                                   ("neg", lambda v: -v), ("abs", abs), ("sqrt", lambda v: math.sqrt(v))])
+                                   ("neg", lambda v: -v), ("abs", abs), ("sqrt", lambda v: math.sqrt(v)), ("log", math.log),
+                                   ("rsqrt", lambda v: 1.0 / math.sqrt(v)), ("square", lambda v: v * v), ("reciprocal", lambda v: 1.0 / v)])
 def test_unary_through_interpreter(op, fn):
-    x = np.abs(RNG.normal(size=(3, 4))) + 0.1 if op == "sqrt" else RNG.normal(size=(3, 4))
+    x = np.abs(RNG.normal(size=(3, 4))) + 0.1 if op in ("sqrt", "log", "rsqrt", "reciprocal") else RNG.normal(size=(3, 4))
     y = oracle.run(_spec1(op), {"x": x})["y"]
     want = np.array([[fn(v) for v in row] for row in x])
     np.testing.assert_allclose(y, want, rtol=1e-15, atol=0)
