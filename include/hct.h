@@ -40,7 +40,8 @@
  *                         bf16 multiplies on tensor cores with fp32 accumulation, f32
  *                         uses error-compensated TF32 products (or fp32 FMA for shapes
  *                         the tensor-core path does not take)
- *   conv2d(x, w, stride=1, pad=0)   x[N,C,H,W], w[K,C,R,S]; cross-correlation, zero padding
+ *   conv2d(x, w, stride=1, pad=0, dilation=1)   x[N,C,H,W], w[K,C,R,S]; cross-correlation, zero padding;
+ *                         y[n,k,h,w] = sum x[n,c,h*stride-pad+r*dilation, w*stride-pad+s*dilation] * w[k,c,r,s]
  *
  * Every computed value is fp32; bf16 inputs are widened exactly; an output
  * stored as bf16 is rounded to nearest-even once, at the store.

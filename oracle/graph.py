@@ -268,20 +268,22 @@ def _infer(g, name, op, pos, attrs, where):
             raise SpecError(f"{where}: gemm operands must have one dtype")
         return Node(name, op, [a, b], dict(attrs), (sa[0], sb[1]), "f32")
     if op == "conv2d":
-        only_attrs("stride", "pad")
+        only_attrs("stride", "pad", "dilation")
         if len(pos) != 2:
             raise SpecError(f"{where}: conv2d takes (x, w)")
         a, b = (_operand(g, p, where, False) for p in pos)
         sa, sb = shape_of(a), shape_of(b)
         stride = _int_attr(attrs, "stride", 1, where)
         pad = _int_attr(attrs, "pad", 0, where)
-        if len(sa) != 4 or len(sb) != 4 or sa[1] != sb[1] or stride < 1 or pad < 0:
+        dil = _int_attr(attrs, "dilation", 1, where)
+        if len(sa) != 4 or len(sb) != 4 or sa[1] != sb[1] or stride < 1 or pad < 0 or dil < 1:
             raise SpecError(f"{where}: conv2d operands {sa}, {sb} are inconsistent")
         if g.nodes[a].dtype != g.nodes[b].dtype:
             raise SpecError(f"{where}: conv2d operands must have one dtype")
-        ho = (sa[2] + 2 * pad - sb[2]) // stride + 1
-        wo = (sa[3] + 2 * pad - sb[3]) // stride + 1
-        if ho < 1 or wo < 1:
+        # a filter of R taps spaced `dil` apart spans dil*(R-1)+1 input rows
+        eh, ew = sa[2] + 2 * pad - (dil * (sb[2] - 1) + 1), sa[3] + 2 * pad - (dil * (sb[3] - 1) + 1)
+        if eh < 0 or ew < 0:
             raise SpecError(f"{where}: conv2d output is empty")
-        return Node(name, op, [a, b], {"stride": stride, "pad": pad}, (sa[0], sb[0], ho, wo), "f32")
+        ho, wo = eh // stride + 1, ew // stride + 1
+        return Node(name, op, [a, b], {"stride": stride, "pad": pad, "dilation": dil}, (sa[0], sb[0], ho, wo), "f32")
     raise SpecError(f"{where}: unknown operator {op!r}")

@@ -142,8 +142,8 @@ def gemm(a, b):
     return np.matmul(a, b)
 
 
-def conv2d(x, w, stride, pad):
-    """Y[n,k,h,w] = sum_{c,r,s} X[n,c,h*stride-pad+r, w*stride-pad+s] * Wt[k,c,r,s].
+def conv2d(x, w, stride, pad, dilation=1):
+    """Y[n,k,h,w] = sum_{c,r,s} X[n,c,h*stride-pad+r*dilation, w*stride-pad+s*dilation] * Wt[k,c,r,s].
 
     Cross-correlation over an NCHW input with zeros outside the image, as in
     the paper's convolution case study (input row h - P + kh, column w - P + kw,
@@ -153,14 +153,15 @@ def conv2d(x, w, stride, pad):
     """
     n, c, h, wd = x.shape
     k, _, kr, ks = w.shape
-    ho = (h + 2 * pad - kr) // stride + 1
-    wo = (wd + 2 * pad - ks) // stride + 1
+    ho = (h + 2 * pad - dilation * (kr - 1) - 1) // stride + 1
+    wo = (wd + 2 * pad - dilation * (ks - 1) - 1) // stride + 1
     xp = np.zeros((n, c, h + 2 * pad, wd + 2 * pad), dtype=x.dtype)
     xp[:, :, pad:pad + h, pad:pad + wd] = x
     y = np.zeros((n, k, ho, wo), dtype=x.dtype)
     for r in range(kr):
         for s in range(ks):
-            win = xp[:, :, r:r + (ho - 1) * stride + 1:stride, s:s + (wo - 1) * stride + 1:stride]
+            r0, s0 = r * dilation, s * dilation
+            win = xp[:, :, r0:r0 + (ho - 1) * stride + 1:stride, s0:s0 + (wo - 1) * stride + 1:stride]
             y += np.einsum("nchw,kc->nkhw", win, w[:, :, r, s], optimize=True)
     return y
 
@@ -217,7 +218,7 @@ def run_nodes(spec, inputs: dict, dtype=np.float64, gemm_fn=None) -> dict:
         elif op == "gemm":
             out = (gemm_fn or gemm)(args[0], args[1])
         elif op == "conv2d":
-            out = conv2d(args[0], args[1], node.attrs["stride"], node.attrs["pad"])
+            out = conv2d(args[0], args[1], node.attrs["stride"], node.attrs["pad"], node.attrs["dilation"])
         else:  # pragma: no cover - parse() rejects unknown operators
             raise ValueError(op)
         assert tuple(out.shape) == tuple(node.shape), (name, out.shape, node.shape)

@@ -229,7 +229,7 @@ hct_status_t hct_graph_run(hct_graph_t* g, const void* const* inputs, int n_inpu
         const TmaDesc& t = k.spec.tmaps[i];
         void* base = resolve(g, t.buf, inputs, outputs, (char*)workspace);
         if (base != k.tmap_base[i]) {
-          uint32_t estr[5] = {1, 1, 1, 1, 1};
+          uint32_t estr[5] = {t.estride[0], t.estride[1], t.estride[2], t.estride[3], t.estride[4]};
           int dtype = t.elem_bytes == 2 ? 9 /* bf16 */ : 7 /* fp32 */;
           CUresult_t rc = d.TensorMapEncodeTiled(&k.tmaps[i], dtype, (unsigned)t.rank, base, t.dims, t.strides + 1, t.box, estr,
                                                  0 /* no interleave */, t.swizzle, 2 /* L2 promotion 128B */, 0 /* zero fill */);

@@ -22,7 +22,8 @@ struct TmaDesc {
   int rank = 2;
   uint64_t dims[5] = {1, 1, 1, 1, 1};     // innermost first
   uint64_t strides[5] = {0, 0, 0, 0, 0};  // bytes, for dims[1..]; strides[0] unused
-  uint32_t box[5] = {1, 1, 1, 1, 1};
+  uint32_t box[5] = {1, 1, 1, 1, 1};       // elements traversed; ceil(box / estride) of them are loaded
+  uint32_t estride[5] = {1, 1, 1, 1, 1};   // traversal stride per dimension (estride[0] must stay 1)
   int swizzle = 3;                // 0 none, 1 32B, 2 64B, 3 128B
 };
 

@@ -493,7 +493,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     }
   }
 
-  // ---- tensor-core convolution: bf16 inputs, stride 1; layout pre-pass, then implicit GEMM
+  // ---- tensor-core convolution: bf16 inputs; layout pre-pass, then implicit GEMM
   if (grp.kind == GroupKind::Conv && !tun.simt_only) {
     const auto& xs = a.shape;
     const auto& ws = b.shape;
@@ -501,7 +501,11 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     bool in_bf16 = b.cls == OpClass::Input && a.dtype == BF16 && b.dtype == BF16;
     int64_t NB = xs[0], C = xs[1], H = xs[2], W = xs[3], KO = ws[0], FR = ws[2], FS = ws[3];
     int64_t HO = anchor.shape[2], WO = anchor.shape[3];
-    if (in_bf16 && anchor.stride == 1 && C % 8 == 0 && WO <= 256 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
+    // Stride and dilation other than 1 take the per-tap schedule: the pixel box of a tap is loaded with a
+    // traversal stride (every ST-th pixel of every ST-th row), which the tensor map allows up to 8 and a box of 256.
+    const int64_t ST = anchor.stride, DIL = anchor.dilation;
+    const bool unit = ST == 1 && DIL == 1;
+    if (in_bf16 && ST <= 8 && WO * ST <= 256 && C % 8 == 0 && WO <= 256 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
       // Three schedules.  (1) Rows whose byte length is a multiple of 16 and that fill most of a 32-column
       // pitch: the kernel reads NCHW itself and re-lays pixels in shared memory (conv_tc_nchw); only the
       // weights take a pre-pass.  Otherwise a pre-pass writes an NHWC copy and pixels are loaded
@@ -515,14 +519,14 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       // The epilogue of the NCHW-reading kernel hands its bf16 output to TMA stores (through 16 KB of
       // shared memory) when it stores a single bf16 tensor (output or intermediate) whose rows are 16-byte multiples.
       const bool tma_store = grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && WO % 8 == 0 && !tun.conv_no_tma_store;
-      if (dense_pitch && W % 8 == 0 && !tun.conv_no_direct) {
+      if (unit && dense_pitch && W % 8 == 0 && !tun.conv_no_direct) {
         // shared memory: operand buffers of TH + FR - 1 rows, staging ring, output staging, and what is left for the weight ring
         const int64_t fixed = n_buf * ((th_pitch + FR - 1) * pitch * 128 + 1024) + n_stg * pitch * 128 + 1024 + (tma_store ? 16384 : 0);
         n_a = (int)std::min<int64_t>(6, (232448 - 512 - fixed) / 16384);
         direct = n_a >= 3;
       }
-      const bool halo = !direct && FS > 1 && dense_pitch && !tun.conv_no_halo;
-      const int TH = (direct || halo) ? th_pitch : (int)std::max<int64_t>(1, std::min<int64_t>(256 / WO, HO));
+      const bool halo = unit && !direct && FS > 1 && dense_pitch && !tun.conv_no_halo;
+      const int TH = (direct || halo) ? th_pitch : (int)std::max<int64_t>(1, std::min<int64_t>(256 / WO, std::min<int64_t>(HO, 256 / ST)));
       auto align256 = [](int64_t v) { return (v + 255) / 256 * 256; };
       const int64_t x_bytes = direct ? 0 : align256(NB * C * H * W * 2), w_bytes = align256(KO * C * FR * FS * 2);
       *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(x_bytes + w_bytes));
@@ -561,7 +565,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       std::ostringstream src;
       src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_H " << H << "\n#define HCT_W " << W
           << "\n#define HCT_KO " << KO << "\n#define HCT_FR " << FR << "\n#define HCT_FS " << FS << "\n#define HCT_PAD " << anchor.pad
-          << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TH " << TH << "\n#define HCT_TH2 1\n#define HCT_SPLIT "
+          << "\n#define HCT_STRIDE " << ST << "\n#define HCT_DIL " << DIL << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TH " << TH << "\n#define HCT_TH2 1\n#define HCT_SPLIT "
           << TH << "\n#define HCT_PITCH " << pitch << "\n#define HCT_NA " << (direct ? n_a : 6) << "\n#define HCT_NBUF " << (direct ? n_buf : 3)
           << "\n#define HCT_NSTG " << n_stg << "\n#define HCT_X_IS_INPUT " << (a.cls == OpClass::Input ? 1 : 0) << "\n#define HCT_TMA_STORE " << (use_tma_store ? 1 : 0) << "\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
           << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
@@ -583,9 +587,10 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       tx.rank = 4;
       tx.dims[0] = (uint64_t)C; tx.dims[1] = (uint64_t)W; tx.dims[2] = (uint64_t)H; tx.dims[3] = (uint64_t)NB;
       tx.strides[1] = (uint64_t)C * 2; tx.strides[2] = (uint64_t)W * C * 2; tx.strides[3] = (uint64_t)H * W * C * 2;
-      tx.box[0] = 64; tx.box[1] = (uint32_t)(halo ? pitch : WO); tx.box[2] = (uint32_t)TH; tx.box[3] = 1;
+      tx.box[0] = 64; tx.box[1] = (uint32_t)(halo ? pitch : WO * ST); tx.box[2] = (uint32_t)(TH * ST); tx.box[3] = 1;
+      tx.estride[1] = tx.estride[2] = (uint32_t)ST;
       TmaDesc tx2 = tx;
-      tx2.box[2] = 1;
+      tx2.box[2] = (uint32_t)ST;
       k.tmaps = {tw, tx, tx2};
       if (direct) {  // NCHW input: [64 channels x pitch pixels] of one row, no swizzle (the kernel re-lays it)
         TmaDesc tn;
@@ -625,7 +630,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       else if (halo)
         d << "pixels shared by the taps of a filter row (pitch " << pitch << ")";
       else
-        d << stages << " stages";
+        d << stages << " stages" << (unit ? "" : ", strided pixel boxes");
       k.desc = d.str();
       out->push_back(k);
       return;
@@ -661,8 +666,8 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     k.name = "hct_conv_simt_g" + std::to_string(gi);
     src << "#define HCT_NB " << xs[0] << "\n#define HCT_CI " << xs[1] << "\n#define HCT_H " << xs[2] << "\n#define HCT_W " << xs[3]
         << "\n#define HCT_KO " << ws[0] << "\n#define HCT_FR " << ws[2] << "\n#define HCT_FS " << ws[3] << "\n#define HCT_STRIDE "
-        << anchor.stride << "\n#define HCT_PAD " << anchor.pad << "\n#define HCT_HO " << anchor.shape[2] << "\n#define HCT_WO "
-        << anchor.shape[3] << "\n";
+        << anchor.stride << "\n#define HCT_PAD " << anchor.pad << "\n#define HCT_DIL " << anchor.dilation << "\n#define HCT_HO "
+        << anchor.shape[2] << "\n#define HCT_WO " << anchor.shape[3] << "\n";
     src << "#define HCT_TA " << ctype(ta) << "\n#define HCT_TB " << ctype(tb) << "\n#define HCT_PA " << pa << "\n#define HCT_PB "
         << pb << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
     src << skeleton_source("common") << "\nstruct HctParams { void* ptr[" << eg.ptrs.size() << "]; };\n" << epi

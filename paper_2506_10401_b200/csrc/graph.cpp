@@ -320,7 +320,7 @@ Graph parse_spec(const std::string& text) {
         if (a.dtype != b.dtype) fail(HCT_ERR_GRAPH, line, "gemm operands must have one dtype");
         n.shape = {a.shape[0], b.shape[1]};
       } else if (op == "conv2d") {
-        only_attrs({"stride", "pad"});
+        only_attrs({"stride", "pad", "dilation"});
         if (pos.size() != 2) fail(HCT_ERR_GRAPH, line, "conv2d takes (x, w)");
         n.cls = OpClass::Conv;
         n.args = {lookup(pos[0], line, false), lookup(pos[1], line, false)};
@@ -328,13 +328,15 @@ Graph parse_spec(const std::string& text) {
         auto& b = g.nodes[n.args[1].node];
         n.stride = int_attr("stride", 1);
         n.pad = int_attr("pad", 0);
-        if (a.shape.size() != 4 || b.shape.size() != 4 || a.shape[1] != b.shape[1] || n.stride < 1 || n.pad < 0)
+        n.dilation = int_attr("dilation", 1);
+        if (a.shape.size() != 4 || b.shape.size() != 4 || a.shape[1] != b.shape[1] || n.stride < 1 || n.pad < 0 || n.dilation < 1)
           fail(HCT_ERR_GRAPH, line, "conv2d operands " + shape_str(a.shape) + ", " + shape_str(b.shape) + " are inconsistent");
         if (a.dtype != b.dtype) fail(HCT_ERR_GRAPH, line, "conv2d operands must have one dtype");
-        int64_t ho = (a.shape[2] + 2 * n.pad - b.shape[2]) / n.stride + 1;
-        int64_t wo = (a.shape[3] + 2 * n.pad - b.shape[3]) / n.stride + 1;
-        if (a.shape[2] + 2 * n.pad < b.shape[2] || a.shape[3] + 2 * n.pad < b.shape[3] || ho < 1 || wo < 1)
-          fail(HCT_ERR_GRAPH, line, "conv2d output is empty");
+        // a filter of R taps spaced `dilation` apart spans dilation * (R - 1) + 1 input rows
+        const int64_t eh = a.shape[2] + 2 * n.pad - ((int64_t)n.dilation * (b.shape[2] - 1) + 1);
+        const int64_t ew = a.shape[3] + 2 * n.pad - ((int64_t)n.dilation * (b.shape[3] - 1) + 1);
+        if (eh < 0 || ew < 0) fail(HCT_ERR_GRAPH, line, "conv2d output is empty");
+        int64_t ho = eh / n.stride + 1, wo = ew / n.stride + 1;
         n.shape = {a.shape[0], b.shape[0], ho, wo};
       } else {
         fail(HCT_ERR_GRAPH, line, "unknown operator '" + op + "'");

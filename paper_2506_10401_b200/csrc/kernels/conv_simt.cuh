@@ -1,5 +1,5 @@
 // Direct convolution, one thread per output element, for shapes the tensor-core kernel does not take.
-// Defined by the generator: HCT_NB, HCT_CI, HCT_H, HCT_W, HCT_KO, HCT_FR, HCT_FS, HCT_STRIDE, HCT_PAD,
+// Defined by the generator: HCT_NB, HCT_CI, HCT_H, HCT_W, HCT_KO, HCT_FR, HCT_FS, HCT_STRIDE, HCT_PAD, HCT_DIL,
 // HCT_HO, HCT_WO, HCT_TA, HCT_TB, HCT_PA, HCT_PB, HctParams, hct_epilogue(), HCT_KERNEL_NAME.
 extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {
   hct_pdl_launch_dependents();
@@ -15,10 +15,10 @@ extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParam
     float acc = 0.0f;
     for (int c = 0; c < HCT_CI; ++c)
       for (int r = 0; r < HCT_FR; ++r) {
-        int ih = h * HCT_STRIDE - HCT_PAD + r;
+        int ih = h * HCT_STRIDE - HCT_PAD + r * HCT_DIL;
         if (ih < 0 || ih >= HCT_H) continue;
         for (int s = 0; s < HCT_FS; ++s) {
-          int iw = w * HCT_STRIDE - HCT_PAD + s;
+          int iw = w * HCT_STRIDE - HCT_PAD + s * HCT_DIL;
           if (iw < 0 || iw >= HCT_W) continue;
           acc = fmaf(hct_ld1(X + ((n * HCT_CI + c) * HCT_H + ih) * HCT_W + iw),
                      hct_ld1(Wt + (((long long)k * HCT_CI + c) * HCT_FR + r) * HCT_FS + s), acc);

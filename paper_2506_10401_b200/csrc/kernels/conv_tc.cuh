@@ -1,18 +1,20 @@
-// Persistent tensor-core conv2d (stride 1, zero padding) as an implicit GEMM with fused epilogue.
+// Persistent tensor-core conv2d (zero padding, any stride and dilation the tensor map can traverse)
+// as an implicit GEMM with fused epilogue.
 //
 // GEMM view: rows (M = 128) = output channels, columns (N <= 256) = the pixels of HCT_TH full output
 // rows of one image, contraction over (filter tap, input channel).  For every tap (r,s) and block
 // of 64 input channels the producer warp loads the tap's [128 x 64] weight slice (A operand) and,
 // with one 4-D TMA box from the NHWC copy of the input, the pixels shifted by the tap (B operand;
 // coordinates outside the image read zeros, which is the padding; the channel coordinate is the
-// innermost one and a multiple of 64, so every copy starts 16-byte aligned).  The MMA warp
+// innermost one and a multiple of 64, so every copy starts 16-byte aligned; with a stride the box
+// is traversed in steps of HCT_STRIDE pixels and rows, so it still delivers HCT_WO pixels per row).  The MMA warp
 // accumulates into one of two tensor-memory accumulators; four epilogue warps (one output channel
 // per thread, 32 consecutive pixels per step, contiguous in NCHW) apply the generated epilogue.
 //
 // Work is split into tiles of HCT_TH output rows; when the last round over the SMs would be
 // nearly empty, its tiles are cut into HCT_TH2-row pieces so that all SMs finish together.
 //
-// Defined by the generator: HCT_NB_IMG, HCT_C, HCT_H, HCT_W, HCT_KO, HCT_FR, HCT_FS, HCT_PAD, HCT_HO, HCT_WO,
+// Defined by the generator: HCT_NB_IMG, HCT_C, HCT_H, HCT_W, HCT_KO, HCT_FR, HCT_FS, HCT_PAD, HCT_STRIDE, HCT_DIL, HCT_HO, HCT_WO,
 // HCT_TH, HCT_TH2, HCT_SPLIT (pieces per cut tile, HCT_TH2 * HCT_SPLIT >= HCT_TH), HCT_STAGES,
 // HCT_STATUS_SLOT, HCT_KERNEL_NAME, HctParams, hct_epilogue_run().
 #define HCT_BM 128
@@ -109,7 +111,7 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
           hct_mbar_expect_tx(full, bytes);
           const hct_u32 dst = smem_base + stage * HCT_STAGE_BYTES;
           hct_tma_load_2d(dst, &hct_p.tmap[0], cb * 64, tap * HCT_KO + t.mbk * HCT_BM, full);
-          hct_tma_load_4d(dst + HCT_A_BYTES, xmap, cb * 64, s - HCT_PAD, t.h0 + r - HCT_PAD, t.n, full);
+          hct_tma_load_4d(dst + HCT_A_BYTES, xmap, cb * 64, s * HCT_DIL - HCT_PAD, t.h0 * HCT_STRIDE + r * HCT_DIL - HCT_PAD, t.n, full);
           if (++stage == HCT_STAGES) { stage = 0; phase ^= 1u; }
         }
       }

@@ -245,6 +245,33 @@ def test_conv_bf16_nchw_direct_integer_inputs_are_exact():
     np.testing.assert_array_equal(got[0], want[0])
 
 
+@pytest.mark.parametrize("shape,wshape,attrs", [
+    ((2, 64, 28, 30), (96, 64, 3, 3), "stride=2, pad=1"),
+    ((1, 128, 56, 56), (256, 128, 1, 1), "stride=2, pad=0"),          # downsampling 1x1
+    ((2, 16, 23, 19), (40, 16, 3, 3), "stride=3, pad=1"),
+    ((1, 72, 21, 26), (130, 72, 3, 3), "stride=1, pad=2, dilation=2"),
+    ((2, 8, 25, 31), (8, 8, 3, 2), "stride=2, pad=3, dilation=3"),
+    ((1, 8, 40, 70), (16, 8, 5, 5), "stride=8, pad=2"),
+    ((1, 8, 6, 300), (8, 8, 3, 3), "stride=2, pad=1"),                # too wide for one strided box: fp32-FMA kernel
+])
+def test_conv_bf16_stride_and_dilation_integer_inputs_are_exact(shape, wshape, attrs):
+    dims = lambda t: "[" + ",".join(str(v) for v in t) + "]"
+    spec = f"hct 1\ninput x bf16 {dims(shape)}\ninput w bf16 {dims(wshape)}\nnode y = conv2d(x, w, {attrs})\noutput y f32\n"
+    il = {"kind": "int", "lo": -4, "hi": 4}
+    got, want, g = parity.run_both(spec, {"x": il, "w": il})
+    assert ("strided pixel boxes" in g.plan) == (shape[3] != 300)
+    np.testing.assert_array_equal(got[0], want[0])
+
+
+def test_conv_strided_chain_and_f32_dilation():
+    spec, laws = configs.get_config("c4_conv_bn_relu_bf16", n=2, c=64, h=56, w=56, k=128, stride=2, pad=1)
+    check_bf16(spec, laws)
+    spec = "hct 1\ninput x f32 [2,6,11,12]\ninput w f32 [5,6,3,3]\nnode y = conv2d(x, w, stride=2, pad=2, dilation=2)\noutput y\n"
+    il = {"kind": "int", "lo": -4, "hi": 4}
+    got, want, _ = parity.run_both(spec, {"x": il, "w": il})
+    np.testing.assert_array_equal(got[0], want[0])
+
+
 # ------------------------------------------------------------------ stacked contractions through bf16 intermediates
 
 @pytest.mark.parametrize("kw", [dict(n=2, c=64, h=20, w=24, k=64), dict(n=1, c=128, h=56, w=56, k=128), dict(n=2, c=16, h=9, w=11, k=32)])

@@ -243,12 +243,12 @@ def test_gemm_integer_exact_and_torch():
 
 # ---------------------------------------------------------------- conv2d
 
-def _conv_loops(x, w, stride, pad):
+def _conv_loops(x, w, stride, pad, dil=1):
     """The definition as a seven-deep loop nest (NCHW, zero contribution outside the image)."""
     n_, c_, h_, w_ = x.shape
     k_, _, r_, s_ = w.shape
-    ho = (h_ + 2 * pad - r_) // stride + 1
-    wo = (w_ + 2 * pad - s_) // stride + 1
+    ho = (h_ + 2 * pad - dil * (r_ - 1) - 1) // stride + 1
+    wo = (w_ + 2 * pad - dil * (s_ - 1) - 1) // stride + 1
     y = np.zeros((n_, k_, ho, wo))
     for n in range(n_):
         for k in range(k_):
@@ -258,8 +258,8 @@ def _conv_loops(x, w, stride, pad):
                     for c in range(c_):
                         for r in range(r_):
                             for s in range(s_):
-                                ih = h * stride - pad + r
-                                iw = q * stride - pad + s
+                                ih = h * stride - pad + r * dil
+                                iw = q * stride - pad + s * dil
                                 if 0 <= ih < h_ and 0 <= iw < w_:
                                     acc += x[n, c, ih, iw] * w[k, c, r, s]
                     y[n, k, h, q] = acc
@@ -279,6 +279,24 @@ def test_conv_bruteforce_and_torch(shape, wshape, stride, pad):
     np.testing.assert_allclose(y, _conv_loops(x, w, stride, pad), rtol=1e-13, atol=1e-13)
     t = torch.nn.functional.conv2d(torch.from_numpy(x), torch.from_numpy(w), stride=stride, padding=pad)
     np.testing.assert_allclose(y, t.numpy(), rtol=1e-12, atol=1e-12)
+
+
+@pytest.mark.parametrize("shape,wshape,stride,pad,dil", [
+    ((1, 2, 9, 8), (3, 2, 3, 3), 1, 2, 2),
+    ((2, 1, 11, 10), (2, 1, 3, 2), 2, 1, 3),
+    ((1, 3, 7, 7), (2, 3, 2, 2), 1, 0, 2),
+])
+def test_conv_dilation_bruteforce_and_torch(shape, wshape, stride, pad, dil):
+    x, w = RNG.normal(size=shape), RNG.normal(size=wshape)
+    y = interp.conv2d(x, w, stride, pad, dil)
+    np.testing.assert_allclose(y, _conv_loops(x, w, stride, pad, dil), rtol=1e-13, atol=1e-13)
+    t = torch.nn.functional.conv2d(torch.from_numpy(x), torch.from_numpy(w), stride=stride, padding=pad, dilation=dil)
+    np.testing.assert_allclose(y, t.numpy(), rtol=1e-12, atol=1e-12)
+    # a dilated filter equals the dense filter with zeros between its taps
+    k_, c_, r_, s_ = wshape
+    wz = np.zeros((k_, c_, dil * (r_ - 1) + 1, dil * (s_ - 1) + 1))
+    wz[:, :, ::dil, ::dil] = w
+    np.testing.assert_allclose(y, interp.conv2d(x, wz, stride, pad), rtol=1e-13, atol=1e-13)
 
 
 def test_conv_structure_pins():
@@ -314,6 +332,8 @@ def test_parse_good_and_shapes():
     assert g.inputs == ["x", "b"] and g.outputs == [("y", "f32")]
     g = oracle.parse("hct 1\ninput x bf16 [2,3,8,8]\ninput w bf16 [5,3,3,3]\nnode y = conv2d(x, w, stride=2, pad=1)\noutput y bf16\n")
     assert g.nodes["y"].shape == (2, 5, 4, 4)
+    g = oracle.parse("hct 1\ninput x bf16 [2,3,9,8]\ninput w bf16 [5,3,3,3]\nnode y = conv2d(x, w, pad=1, dilation=2)\noutput y bf16\n")
+    assert g.nodes["y"].shape == (2, 5, 7, 6)
     g = oracle.parse("hct 1\ninput x f32 [4,8]\nnode s = row_sum(x)\nnode y = div(x, s)\noutput y\n")
     assert g.nodes["s"].shape == (4, 1) and g.nodes["y"].shape == (4, 8)
 
