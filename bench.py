@@ -37,6 +37,8 @@ WORKLOADS = {
     "transpose_bias_relu": dict(bound="hbm", sample=dict(r=4096)),
     "matmul_dropout_mean_softmax": dict(bound="tensor", sample=dict(m=1024)),
     "conv_block": dict(bound="tensor", sample=dict(n=4)),
+    "dwconv_bn_relu": dict(bound="hbm", sample=dict(n=8)),
+    "mbconv_block": dict(bound="hbm", sample=dict(n=4)),
 }
 HEADLINE = "c2_softmax_layernorm_chain"
 
@@ -409,7 +411,7 @@ def main():
         peak = pk["hbm"] if info["bound"] == "hbm" else (pk["tensor_sustained"] if capped else pk["tensor"])
         line = dict(metric=metric, value=r["value"], unit=r["unit"], n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
                     ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
-                    dtype="bf16" if ("bf16" in name or name in ("matmul_dropout_mean_softmax", "conv_block")) else "f32", data="synthetic",
+                    dtype="bf16" if ("bf16" in name or name in ("matmul_dropout_mean_softmax", "conv_block", "dwconv_bn_relu", "mbconv_block")) else "f32", data="synthetic",
                     config={"workload": name, "l2": "flushed between steps (192 MB write, untimed)", "kernels_per_step": r["kernels"],
                             "parallelism": "replicas" if world > 1 else "single",
                             "schedule": r["schedule"] or "default", "tuned_trials": args.tune},

@@ -268,7 +268,7 @@ def _infer(g, name, op, pos, attrs, where):
             raise SpecError(f"{where}: gemm operands must have one dtype")
         return Node(name, op, [a, b], dict(attrs), (sa[0], sb[1]), "f32")
     if op == "conv2d":
-        only_attrs("stride", "pad", "dilation")
+        only_attrs("stride", "pad", "dilation", "groups")
         if len(pos) != 2:
             raise SpecError(f"{where}: conv2d takes (x, w)")
         a, b = (_operand(g, p, where, False) for p in pos)
@@ -276,7 +276,10 @@ def _infer(g, name, op, pos, attrs, where):
         stride = _int_attr(attrs, "stride", 1, where)
         pad = _int_attr(attrs, "pad", 0, where)
         dil = _int_attr(attrs, "dilation", 1, where)
-        if len(sa) != 4 or len(sb) != 4 or sa[1] != sb[1] or stride < 1 or pad < 0 or dil < 1:
+        groups = _int_attr(attrs, "groups", 1, where)
+        # channels and filters are cut into `groups` equal parts; filter k of a part sees only that part's channels
+        if (len(sa) != 4 or len(sb) != 4 or stride < 1 or pad < 0 or dil < 1 or groups < 1 or sa[1] != sb[1] * groups
+                or sb[0] % groups != 0):
             raise SpecError(f"{where}: conv2d operands {sa}, {sb} are inconsistent")
         if g.nodes[a].dtype != g.nodes[b].dtype:
             raise SpecError(f"{where}: conv2d operands must have one dtype")
@@ -285,5 +288,5 @@ def _infer(g, name, op, pos, attrs, where):
         if eh < 0 or ew < 0:
             raise SpecError(f"{where}: conv2d output is empty")
         ho, wo = eh // stride + 1, ew // stride + 1
-        return Node(name, op, [a, b], {"stride": stride, "pad": pad, "dilation": dil}, (sa[0], sb[0], ho, wo), "f32")
+        return Node(name, op, [a, b], {"stride": stride, "pad": pad, "dilation": dil, "groups": groups}, (sa[0], sb[0], ho, wo), "f32")
     raise SpecError(f"{where}: unknown operator {op!r}")

@@ -142,7 +142,7 @@ def gemm(a, b):
     return np.matmul(a, b)
 
 
-def conv2d(x, w, stride, pad, dilation=1):
+def conv2d(x, w, stride, pad, dilation=1, groups=1):
     """Y[n,k,h,w] = sum_{c,r,s} X[n,c,h*stride-pad+r*dilation, w*stride-pad+s*dilation] * Wt[k,c,r,s].
 
     Cross-correlation over an NCHW input with zeros outside the image, as in
@@ -150,19 +150,29 @@ def conv2d(x, w, stride, pad, dilation=1):
     taps outside the image contribute nothing; output index ((n*K+k)*H+h)*W+w).
     For each tap (r, s) the strided window of the zero-padded input is
     contracted over channels with the tap's [K,C] weight slice.
+
+    With ``groups`` = G the C input channels and the K filters are cut into G
+    equal consecutive parts, Wt is [K, C/G, R, S], and the filters of part g
+    sum over the channels of part g only (G = C: one filter plane per channel,
+    the depthwise operator class of the paper's model workloads).
     """
     n, c, h, wd = x.shape
-    k, _, kr, ks = w.shape
+    k, cg, kr, ks = w.shape
+    assert c == cg * groups and k % groups == 0
+    kg = k // groups
     ho = (h + 2 * pad - dilation * (kr - 1) - 1) // stride + 1
     wo = (wd + 2 * pad - dilation * (ks - 1) - 1) // stride + 1
     xp = np.zeros((n, c, h + 2 * pad, wd + 2 * pad), dtype=x.dtype)
     xp[:, :, pad:pad + h, pad:pad + wd] = x
     y = np.zeros((n, k, ho, wo), dtype=x.dtype)
-    for r in range(kr):
-        for s in range(ks):
-            r0, s0 = r * dilation, s * dilation
-            win = xp[:, :, r0:r0 + (ho - 1) * stride + 1:stride, s0:s0 + (wo - 1) * stride + 1:stride]
-            y += np.einsum("nchw,kc->nkhw", win, w[:, :, r, s], optimize=True)
+    for g in range(groups):
+        xg = xp[:, g * cg:(g + 1) * cg]
+        wg = w[g * kg:(g + 1) * kg]
+        for r in range(kr):
+            for s in range(ks):
+                r0, s0 = r * dilation, s * dilation
+                win = xg[:, :, r0:r0 + (ho - 1) * stride + 1:stride, s0:s0 + (wo - 1) * stride + 1:stride]
+                y[:, g * kg:(g + 1) * kg] += np.einsum("nchw,kc->nkhw", win, wg[:, :, r, s], optimize=True)
     return y
 
 
@@ -218,7 +228,7 @@ def run_nodes(spec, inputs: dict, dtype=np.float64, gemm_fn=None) -> dict:
         elif op == "gemm":
             out = (gemm_fn or gemm)(args[0], args[1])
         elif op == "conv2d":
-            out = conv2d(args[0], args[1], node.attrs["stride"], node.attrs["pad"], node.attrs["dilation"])
+            out = conv2d(args[0], args[1], node.attrs["stride"], node.attrs["pad"], node.attrs["dilation"], node.attrs["groups"])
         else:  # pragma: no cover - parse() rejects unknown operators
             raise ValueError(op)
         assert tuple(out.shape) == tuple(node.shape), (name, out.shape, node.shape)

@@ -505,7 +505,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     // traversal stride (every ST-th pixel of every ST-th row), which the tensor map allows up to 8 and a box of 256.
     const int64_t ST = anchor.stride, DIL = anchor.dilation;
     const bool unit = ST == 1 && DIL == 1;
-    if (in_bf16 && ST <= 8 && WO * ST <= 256 && C % 8 == 0 && WO <= 256 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
+    if (in_bf16 && anchor.groups == 1 && ST <= 8 && WO * ST <= 256 && C % 8 == 0 && WO <= 256 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
       // Three schedules.  (1) Rows whose byte length is a multiple of 16 and that fill most of a 32-column
       // pitch: the kernel reads NCHW itself and re-lays pixels in shared memory (conv_tc_nchw); only the
       // weights take a pre-pass.  Otherwise a pre-pass writes an NHWC copy and pixels are loaded
@@ -660,11 +660,31 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     if ((M + 63) / 64 > 65535) throw Error(HCT_ERR_UNSUPPORTED, "gemm with more than 4M rows is not supported");
     k.block[0] = 256;
     k.desc = "gemm fp32-FMA 64x64x16";
+  } else if (anchor.groups == a.shape[1] && b.shape[1] == 1 && b.shape[2] * b.shape[3] <= 49 && !tun.simt_only) {
+    // depthwise: memory-bound, one thread per column of P vertically adjacent output pixels
+    const auto& xs = a.shape;
+    const auto& ws = b.shape;
+    int P = 1;
+    for (int cand : {4, 2})
+      if (cand <= anchor.shape[2] && ((cand - 1) * anchor.stride + (ws[2] - 1) * anchor.dilation + 1) * ws[3] <= 160) { P = cand; break; }
+    k.name = "hct_conv_dw_g" + std::to_string(gi);
+    src << "#define HCT_NB " << xs[0] << "\n#define HCT_C " << xs[1] << "\n#define HCT_MULT " << ws[0] / xs[1] << "\n#define HCT_H " << xs[2]
+        << "\n#define HCT_W " << xs[3] << "\n#define HCT_FR " << ws[2] << "\n#define HCT_FS " << ws[3] << "\n#define HCT_STRIDE "
+        << anchor.stride << "\n#define HCT_PAD " << anchor.pad << "\n#define HCT_DIL " << anchor.dilation << "\n#define HCT_HO "
+        << anchor.shape[2] << "\n#define HCT_WO " << anchor.shape[3] << "\n#define HCT_P " << P << "\n";
+    src << "#define HCT_TA " << ctype(ta) << "\n#define HCT_TB " << ctype(tb) << "\n#define HCT_PA " << pa << "\n#define HCT_PB "
+        << pb << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
+    src << skeleton_source("common") << "\nstruct HctParams { void* ptr[" << eg.ptrs.size() << "]; };\n" << epi
+        << skeleton_source("conv_dw");
+    int64_t units = xs[0] * ws[0] * ((anchor.shape[2] + P - 1) / P) * anchor.shape[3];
+    k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>((units + 255) / 256, 148 * 64));
+    k.block[0] = 256;
+    k.desc = "conv2d depthwise fp32-FMA, " + std::to_string(P) + " output rows per thread";
   } else {
     const auto& xs = a.shape;
     const auto& ws = b.shape;
     k.name = "hct_conv_simt_g" + std::to_string(gi);
-    src << "#define HCT_NB " << xs[0] << "\n#define HCT_CI " << xs[1] << "\n#define HCT_H " << xs[2] << "\n#define HCT_W " << xs[3]
+    src << "#define HCT_NB " << xs[0] << "\n#define HCT_CI " << ws[1] << "\n#define HCT_GROUPS " << anchor.groups << "\n#define HCT_H " << xs[2] << "\n#define HCT_W " << xs[3]
         << "\n#define HCT_KO " << ws[0] << "\n#define HCT_FR " << ws[2] << "\n#define HCT_FS " << ws[3] << "\n#define HCT_STRIDE "
         << anchor.stride << "\n#define HCT_PAD " << anchor.pad << "\n#define HCT_DIL " << anchor.dilation << "\n#define HCT_HO "
         << anchor.shape[2] << "\n#define HCT_WO " << anchor.shape[3] << "\n";

@@ -320,7 +320,7 @@ Graph parse_spec(const std::string& text) {
         if (a.dtype != b.dtype) fail(HCT_ERR_GRAPH, line, "gemm operands must have one dtype");
         n.shape = {a.shape[0], b.shape[1]};
       } else if (op == "conv2d") {
-        only_attrs({"stride", "pad", "dilation"});
+        only_attrs({"stride", "pad", "dilation", "groups"});
         if (pos.size() != 2) fail(HCT_ERR_GRAPH, line, "conv2d takes (x, w)");
         n.cls = OpClass::Conv;
         n.args = {lookup(pos[0], line, false), lookup(pos[1], line, false)};
@@ -329,7 +329,10 @@ Graph parse_spec(const std::string& text) {
         n.stride = int_attr("stride", 1);
         n.pad = int_attr("pad", 0);
         n.dilation = int_attr("dilation", 1);
-        if (a.shape.size() != 4 || b.shape.size() != 4 || a.shape[1] != b.shape[1] || n.stride < 1 || n.pad < 0 || n.dilation < 1)
+        n.groups = int_attr("groups", 1);
+        // channels and filters are cut into `groups` equal parts; a filter sees only its part's channels
+        if (a.shape.size() != 4 || b.shape.size() != 4 || n.stride < 1 || n.pad < 0 || n.dilation < 1 || n.groups < 1 ||
+            a.shape[1] != b.shape[1] * n.groups || b.shape[0] % n.groups != 0)
           fail(HCT_ERR_GRAPH, line, "conv2d operands " + shape_str(a.shape) + ", " + shape_str(b.shape) + " are inconsistent");
         if (a.dtype != b.dtype) fail(HCT_ERR_GRAPH, line, "conv2d operands must have one dtype");
         // a filter of R taps spaced `dilation` apart spans dilation * (R - 1) + 1 input rows

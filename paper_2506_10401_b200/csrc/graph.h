@@ -30,7 +30,7 @@ struct Node {
   std::vector<int64_t> shape;
   DType dtype = F32;  // storage dtype of an input; computed nodes are fp32 values (BF16: values rounded to bfloat16 by cast_bf16)
   double eps = 1e-5;
-  int stride = 1, pad = 0, dilation = 1;
+  int stride = 1, pad = 0, dilation = 1, groups = 1;
   // dropout: element with flat index i is kept when hash(i + seed) mod 1000 >= drop_threshold (= round(1000 p))
   double drop_p = 0.0;
   uint64_t drop_seed = 0;

@@ -272,6 +272,40 @@ def test_conv_strided_chain_and_f32_dilation():
     np.testing.assert_array_equal(got[0], want[0])
 
 
+@pytest.mark.parametrize("dtype,shape,wshape,attrs", [
+    ("bf16", (2, 32, 28, 28), (32, 1, 3, 3), "pad=1, groups=32"),
+    ("bf16", (1, 24, 57, 41), (24, 1, 3, 3), "stride=2, pad=1, groups=24"),
+    ("f32", (1, 4, 9, 9), (8, 1, 3, 3), "stride=2, pad=1, groups=4"),                # two filters per channel
+    ("f32", (2, 5, 13, 11), (5, 1, 5, 5), "pad=2, groups=5"),
+    ("bf16", (1, 6, 17, 19), (6, 1, 3, 3), "pad=2, dilation=2, groups=6"),
+    ("f32", (1, 3, 2, 70), (3, 1, 3, 3), "pad=1, groups=3"),                         # fewer output rows than a thread's block
+    ("f32", (1, 2, 30, 9), (2, 1, 7, 7), "stride=3, pad=3, groups=2"),
+    ("bf16", (2, 6, 8, 7), (4, 3, 3, 2), "pad=1, dilation=2, groups=2"),             # grouped, not depthwise
+    ("f32", (1, 8, 6, 6), (12, 2, 1, 1), "groups=4"),
+])
+def test_conv_groups_integer_inputs_are_exact(dtype, shape, wshape, attrs):
+    dims = lambda t: "[" + ",".join(str(v) for v in t) + "]"
+    spec = f"hct 1\ninput x {dtype} {dims(shape)}\ninput w {dtype} {dims(wshape)}\nnode y = conv2d(x, w, {attrs})\noutput y f32\n"
+    il = {"kind": "int", "lo": -4, "hi": 4}
+    got, want, g = parity.run_both(spec, {"x": il, "w": il})
+    assert ("depthwise" in g.plan) == (wshape[1] == 1)
+    np.testing.assert_array_equal(got[0], want[0])
+
+
+@pytest.mark.parametrize("kw", [dict(n=2, c=48, h=28, w=28), dict(n=1, c=16, h=15, w=21, stride=2), dict(n=2, c=192, h=56, w=56)])
+def test_depthwise_chain(kw):
+    spec, laws = configs.get_config("dwconv_bn_relu", **kw)
+    check_bf16(spec, laws)
+
+
+@pytest.mark.parametrize("kw", [dict(n=2, c=32, h=28, w=24), dict(n=1, c=16, h=14, w=14, expand=4), dict(n=2, c=32, h=56, w=56)])
+def test_inverted_residual_block(kw):
+    spec, laws = configs.get_config("mbconv_block", **kw)
+    got, want, g = parity.run_both(spec, laws)
+    assert g.plan.count("tcgen05") == 2 and g.plan.count("depthwise") == 1
+    assert parity.bf16_violation(got[0], want[0]) <= 1.0
+
+
 # ------------------------------------------------------------------ stacked contractions through bf16 intermediates
 
 @pytest.mark.parametrize("kw", [dict(n=2, c=64, h=20, w=24, k=64), dict(n=1, c=128, h=56, w=56, k=128), dict(n=2, c=16, h=9, w=11, k=32)])

@@ -243,10 +243,10 @@ def test_gemm_integer_exact_and_torch():
 
 # ---------------------------------------------------------------- conv2d
 
-def _conv_loops(x, w, stride, pad, dil=1):
+def _conv_loops(x, w, stride, pad, dil=1, groups=1):
     """The definition as a seven-deep loop nest (NCHW, zero contribution outside the image)."""
-    n_, c_, h_, w_ = x.shape
-    k_, _, r_, s_ = w.shape
+    n_, _, h_, w_ = x.shape
+    k_, c_, r_, s_ = w.shape            # c_ channels per group
     ho = (h_ + 2 * pad - dil * (r_ - 1) - 1) // stride + 1
     wo = (w_ + 2 * pad - dil * (s_ - 1) - 1) // stride + 1
     y = np.zeros((n_, k_, ho, wo))
@@ -261,7 +261,7 @@ def _conv_loops(x, w, stride, pad, dil=1):
                                 ih = h * stride - pad + r * dil
                                 iw = q * stride - pad + s * dil
                                 if 0 <= ih < h_ and 0 <= iw < w_:
-                                    acc += x[n, c, ih, iw] * w[k, c, r, s]
+                                    acc += x[n, (k // (k_ // groups)) * c_ + c, ih, iw] * w[k, c, r, s]
                     y[n, k, h, q] = acc
     return y
 
@@ -299,6 +299,27 @@ def test_conv_dilation_bruteforce_and_torch(shape, wshape, stride, pad, dil):
     np.testing.assert_allclose(y, interp.conv2d(x, wz, stride, pad), rtol=1e-13, atol=1e-13)
 
 
+@pytest.mark.parametrize("shape,wshape,stride,pad,dil,groups", [
+    ((2, 6, 7, 8), (6, 1, 3, 3), 1, 1, 1, 6),        # depthwise
+    ((1, 4, 9, 9), (8, 1, 3, 3), 2, 1, 1, 4),        # depthwise, two filters per channel
+    ((1, 6, 8, 7), (4, 3, 3, 2), 1, 1, 2, 2),
+    ((2, 8, 6, 6), (12, 2, 1, 1), 1, 0, 1, 4),
+])
+def test_conv_groups_bruteforce_torch_and_block_diagonal(shape, wshape, stride, pad, dil, groups):
+    x, w = RNG.normal(size=shape), RNG.normal(size=wshape)
+    y = interp.conv2d(x, w, stride, pad, dil, groups)
+    np.testing.assert_allclose(y, _conv_loops(x, w, stride, pad, dil, groups), rtol=1e-13, atol=1e-13)
+    t = torch.nn.functional.conv2d(torch.from_numpy(x), torch.from_numpy(w), stride=stride, padding=pad, dilation=dil, groups=groups)
+    np.testing.assert_allclose(y, t.numpy(), rtol=1e-12, atol=1e-12)
+    # a grouped filter bank is a dense one whose weights vanish outside the diagonal blocks
+    k_, cg, r_, s_ = wshape
+    dense = np.zeros((k_, cg * groups, r_, s_))
+    for k in range(k_):
+        g = k // (k_ // groups)
+        dense[k, g * cg:(g + 1) * cg] = w[k]
+    np.testing.assert_allclose(y, interp.conv2d(x, dense, stride, pad, dil), rtol=1e-13, atol=1e-13)
+
+
 def test_conv_structure_pins():
     n, c, h, w, k = 2, 3, 5, 4, 4
     x = RNG.normal(size=(n, c, h, w))
@@ -334,6 +355,8 @@ def test_parse_good_and_shapes():
     assert g.nodes["y"].shape == (2, 5, 4, 4)
     g = oracle.parse("hct 1\ninput x bf16 [2,3,9,8]\ninput w bf16 [5,3,3,3]\nnode y = conv2d(x, w, pad=1, dilation=2)\noutput y bf16\n")
     assert g.nodes["y"].shape == (2, 5, 7, 6)
+    g = oracle.parse("hct 1\ninput x bf16 [2,6,9,8]\ninput w bf16 [12,2,3,3]\nnode y = conv2d(x, w, pad=1, groups=3)\noutput y bf16\n")
+    assert g.nodes["y"].shape == (2, 12, 9, 8)
     g = oracle.parse("hct 1\ninput x f32 [4,8]\nnode s = row_sum(x)\nnode y = div(x, s)\noutput y\n")
     assert g.nodes["s"].shape == (4, 1) and g.nodes["y"].shape == (4, 8)
 

@@ -131,6 +131,61 @@ output c3 bf16
     return spec, laws
 
 
+def dwconv_bn_relu(n=32, c=192, h=56, w=56, stride=1):
+    """Depthwise conv3x3 -> folded batch norm -> ReLU (the memory-bound stage of a MobileNetV2-style block)."""
+    spec = f"""hct 1
+input x     bf16 [{n},{c},{h},{w}]
+input wt    bf16 [{c},1,3,3]
+input scale f32  [{c},1,1]
+input shift f32  [{c},1,1]
+node  t0 = conv2d(x, wt, stride={stride}, pad=1, groups={c})
+node  t1 = mul(t0, scale)
+node  t2 = add(t1, shift)
+node  t3 = relu(t2)
+output t3 bf16
+"""
+    laws = {"x": _n(), "wt": _n(math.sqrt(2.0 / 9)), "scale": _u(0.5, 1.5), "shift": _n(0.1)}
+    return spec, laws
+
+
+def mbconv_block(n=32, c=32, h=56, w=56, expand=6):
+    """An inverted-residual block in the style of MobileNetV2: pointwise expansion -> BN -> ReLU, depthwise
+    3x3 -> BN -> ReLU, pointwise projection -> BN, plus the block input; activations between the
+    convolutions are rounded to bf16 and stay on the device."""
+    e = c * expand
+    spec = f"""hct 1
+input x  bf16 [{n},{c},{h},{w}]
+input w1 bf16 [{e},{c},1,1]
+input s1 f32  [{e},1,1]
+input b1 f32  [{e},1,1]
+input w2 bf16 [{e},1,3,3]
+input s2 f32  [{e},1,1]
+input b2 f32  [{e},1,1]
+input w3 bf16 [{c},{e},1,1]
+input s3 f32  [{c},1,1]
+input b3 f32  [{c},1,1]
+node  a0 = conv2d(x, w1)
+node  a1 = mul(a0, s1)
+node  a2 = add(a1, b1)
+node  a3 = relu(a2)
+node  a4 = cast_bf16(a3)
+node  d0 = conv2d(a4, w2, pad=1, groups={e})
+node  d1 = mul(d0, s2)
+node  d2 = add(d1, b2)
+node  d3 = relu(d2)
+node  d4 = cast_bf16(d3)
+node  p0 = conv2d(d4, w3)
+node  p1 = mul(p0, s3)
+node  p2 = add(p1, b3)
+node  y  = add(p2, x)
+output y bf16
+"""
+    laws = {"x": _n(), "w1": _n(math.sqrt(2.0 / c)), "s1": _u(0.5, 1.5), "b1": _n(0.1),
+            "w2": _n(math.sqrt(2.0 / 9)), "s2": _u(0.5, 1.5), "b2": _n(0.1),
+            "w3": _n(math.sqrt(1.0 / e)), "s3": _u(0.5, 1.5), "b3": _n(0.1)}
+    return spec, laws
+
+
 def transpose_bias_relu(r=16384, c=4096):
     """A layout transform with fused consumers (Table 1, "LayoutTransform"): y = relu(x^T + bias)."""
     spec = f"""hct 1
@@ -153,6 +208,8 @@ CONFIGS = {
     "matmul_dropout_mean_softmax": (matmul_dropout_mean_softmax, {}),
     "transpose_bias_relu": (transpose_bias_relu, {}),
     "conv_block": (conv_block, {}),
+    "dwconv_bn_relu": (dwconv_bn_relu, {}),
+    "mbconv_block": (mbconv_block, {}),
 }
 
 
