@@ -280,6 +280,12 @@ def test_conv_strided_chain_and_f32_dilation():
     ("bf16", (1, 6, 17, 19), (6, 1, 3, 3), "pad=2, dilation=2, groups=6"),
     ("f32", (1, 3, 2, 70), (3, 1, 3, 3), "pad=1, groups=3"),                         # fewer output rows than a thread's block
     ("f32", (1, 2, 30, 9), (2, 1, 7, 7), "stride=3, pad=3, groups=2"),
+    # rows of whole 16-byte vectors at stride 1: blocks of 8 columns per thread
+    ("bf16", (2, 16, 12, 24), (16, 1, 3, 3), "pad=1, groups=16"),
+    ("f32", (1, 3, 7, 16), (6, 1, 5, 5), "pad=2, groups=3"),
+    ("f32", (1, 4, 5, 40), (4, 1, 1, 1), "groups=4"),
+    ("bf16", (1, 4, 9, 16), (4, 1, 5, 3), "pad=1, groups=4"),                        # 7 output rows: ragged last block
+    ("bf16", (3, 8, 1, 8), (8, 1, 3, 3), "pad=1, groups=8"),                         # a single output row
     ("bf16", (2, 6, 8, 7), (4, 3, 3, 2), "pad=1, dilation=2, groups=2"),             # grouped, not depthwise
     ("f32", (1, 8, 6, 6), (12, 2, 1, 1), "groups=4"),
 ])
@@ -289,6 +295,7 @@ def test_conv_groups_integer_inputs_are_exact(dtype, shape, wshape, attrs):
     il = {"kind": "int", "lo": -4, "hi": 4}
     got, want, g = parity.run_both(spec, {"x": il, "w": il})
     assert ("depthwise" in g.plan) == (wshape[1] == 1)
+    assert ("8 columns" in g.plan) == (wshape[1] == 1 and shape[3] % 8 == 0)
     np.testing.assert_array_equal(got[0], want[0])
 
 
