@@ -40,8 +40,11 @@
  *                         bf16 multiplies on tensor cores with fp32 accumulation, f32
  *                         uses error-compensated TF32 products (or fp32 FMA for shapes
  *                         the tensor-core path does not take)
- *   conv2d(x, w, stride=1, pad=0, dilation=1)   x[N,C,H,W], w[K,C,R,S]; cross-correlation, zero padding;
- *                         y[n,k,h,w] = sum x[n,c,h*stride-pad+r*dilation, w*stride-pad+s*dilation] * w[k,c,r,s]
+ *   conv2d(x, w, stride=1, pad=0, dilation=1, groups=1)   x[N,C,H,W], w[K,C/groups,R,S]; cross-correlation,
+ *                         zero padding; y[n,k,h,w] = sum x[n,c,h*stride-pad+r*dilation, w*stride-pad+s*dilation] * w[k,c',r,s]
+ *                         over the C/groups channels c of filter k's group (groups = C: depthwise).
+ *                         bf16 operands with groups = 1 run on tensor cores (strides up to 8); depthwise
+ *                         and grouped convolutions run on fp32 FMA kernels
  *
  * Every computed value is fp32; bf16 inputs are widened exactly; an output
  * stored as bf16 is rounded to nearest-even once, at the store.

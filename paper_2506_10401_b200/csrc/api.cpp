@@ -323,7 +323,8 @@ hct_status_t hct_graph_autotune(const char* spec, size_t spec_len, int device, c
   if (has_gemm)
     for (const char* c : {"gemm_bn=64", "gemm_bn=128", "gemm_bn=32", "gemm_pair=1", "gemm_pair=2", "gemm_insplit=1"}) cands.insert(cands.begin(), c);
   if (has_conv)
-    for (const char* c : {"conv_no_tma_store=1", "conv_no_direct=1", "conv_no_direct=1;conv_no_halo=1"}) cands.push_back(c);
+    for (const char* c : {"conv_no_tma_store=1", "conv_no_direct=1", "conv_no_direct=1;conv_no_halo=1", "dw_p=4", "dw_p=4;dw_cta=256", "dw_p=8;dw_cta=64"})
+      cands.push_back(c);
 
   const Driver* d = nullptr;
   CUevent_t e0 = nullptr, e1 = nullptr;

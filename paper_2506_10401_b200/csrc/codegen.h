@@ -62,6 +62,8 @@ struct Tunables {
   int gemm_bn = 0;                 // output-tile width of the tensor-core GEMMs (0: by rule; else 32..256, clamped to what the kernel takes)
   bool conv_no_halo = false;       // load conv pixels once per tap even when the shared-row schedule applies
   bool conv_no_tma_store = false;  // NCHW-reading convolution: store the output with plain vector stores instead of TMA
+  int dw_p = 0;                    // depthwise conv: output rows per thread (0: rule; 1, 2, 4 or 8)
+  int dw_cta = 0;                  // depthwise conv: threads per block (0: rule; else a multiple of 32, up to 1024)
   bool conv_no_direct = false;     // always take the NHWC pre-pass, even when the convolution could read NCHW itself
   bool simt_only = false;
   // Failure-path testing: the GEMM producer never issues its loads, so the consumer's bounded wait runs out

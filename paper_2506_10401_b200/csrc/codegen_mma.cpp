@@ -671,10 +671,12 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     const int64_t HOd = anchor.shape[2], WOd = anchor.shape[3];
     const bool vec = anchor.stride == 1 && anchor.dilation == 1 && xs[3] % 8 == 0 && WOd % 8 == 0 && 2 * anchor.pad <= ws[3] - 1 &&
                      ws[3] <= 7 && xs[0] * ws[0] * HOd * (WOd / 8) < 0x7fffffffLL;
-    if (vec) P = HOd >= 4 ? 4 : HOd >= 2 ? 2 : 1;
+    if (vec) P = HOd >= 16 ? 8 : HOd >= 4 ? 4 : HOd >= 2 ? 2 : 1;
+    if (tun.dw_p == 1 || tun.dw_p == 2 || tun.dw_p == 4 || (tun.dw_p == 8 && vec)) P = tun.dw_p;
+    const unsigned cta = (unsigned)std::min(1024, std::max(32, (tun.dw_cta > 0 ? tun.dw_cta : vec ? 128 : 256) / 32 * 32));
     const std::string epi_dw = vec ? eg.run_fn(HOd * WOd, WOd, "(row % " + std::to_string(ws[0]) + "LL)") : epi;
     k.name = "hct_conv_dw_g" + std::to_string(gi);
-    src << "#define HCT_VEC " << (vec ? 1 : 0) << "\n";
+    src << "#define HCT_VEC " << (vec ? 1 : 0) << "\n#define HCT_CTA " << cta << "\n";
     src << "#define HCT_NB " << xs[0] << "\n#define HCT_C " << xs[1] << "\n#define HCT_MULT " << ws[0] / xs[1] << "\n#define HCT_H " << xs[2]
         << "\n#define HCT_W " << xs[3] << "\n#define HCT_FR " << ws[2] << "\n#define HCT_FS " << ws[3] << "\n#define HCT_STRIDE "
         << anchor.stride << "\n#define HCT_PAD " << anchor.pad << "\n#define HCT_DIL " << anchor.dilation << "\n#define HCT_HO "
@@ -684,8 +686,8 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     src << skeleton_source("common") << "\n" << (vec ? skeleton_source("tc_common") : std::string()) << "\nstruct HctParams { void* ptr["
         << eg.ptrs.size() << "]; };\n" << epi_dw << skeleton_source("conv_dw");
     int64_t units = xs[0] * ws[0] * ((anchor.shape[2] + P - 1) / P) * (vec ? WOd / 8 : WOd);
-    k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>((units + 255) / 256, 148 * 64));
-    k.block[0] = 256;
+    k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>((units + cta - 1) / cta, 148 * 64));
+    k.block[0] = cta;
     k.desc = "conv2d depthwise fp32-FMA, " + std::string(vec ? "8 columns x " : "") + std::to_string(P) + " output rows per thread";
   } else {
     const auto& xs = a.shape;

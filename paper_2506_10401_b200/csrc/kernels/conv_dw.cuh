@@ -11,7 +11,7 @@
 // output row one vector store through the generated run epilogue, so that about nine of every
 // thirteen instructions are the multiply-adds themselves.
 //
-// Defined by the generator: HCT_VEC, HCT_NB, HCT_C, HCT_MULT, HCT_H, HCT_W, HCT_FR, HCT_FS, HCT_STRIDE, HCT_PAD, HCT_DIL,
+// Defined by the generator: HCT_VEC, HCT_CTA (threads per block), HCT_NB, HCT_C, HCT_MULT, HCT_H, HCT_W, HCT_FR, HCT_FS, HCT_STRIDE, HCT_PAD, HCT_DIL,
 // HCT_HO, HCT_WO, HCT_P, HCT_TA, HCT_TB, HCT_PA, HCT_PB, HctParams, hct_epilogue(), HCT_KERNEL_NAME.
 #define HCT_KO (HCT_C * HCT_MULT)
 #define HCT_HB ((HCT_HO + HCT_P - 1) / HCT_P)                                  // blocks of HCT_P output rows per plane
@@ -20,13 +20,13 @@
 #if HCT_VEC
 #define HCT_WB (HCT_WO / 8)                 // 8-column blocks per output row
 #define HCT_XW (8 + HCT_FS - 1)             // input columns under one block
-extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {
+extern "C" __global__ void __launch_bounds__(HCT_CTA) HCT_KERNEL_NAME(const HctParams hct_p) {
   hct_pdl_launch_dependents();
   hct_pdl_wait();
   const HCT_TA* __restrict__ X = (const HCT_TA*)hct_p.ptr[HCT_PA];
   const HCT_TB* __restrict__ Wt = (const HCT_TB*)hct_p.ptr[HCT_PB];
   const unsigned units = (unsigned)HCT_NB * HCT_KO * HCT_HB * HCT_WB;   // below 2^31 (checked by the generator)
-  for (unsigned u = blockIdx.x * 256u + threadIdx.x; u < units; u += gridDim.x * 256u) {
+  for (unsigned u = blockIdx.x * (unsigned)HCT_CTA + threadIdx.x; u < units; u += gridDim.x * (unsigned)HCT_CTA) {
     const int w0 = (int)(u % HCT_WB) * 8;
     unsigned t = u / HCT_WB;
     const int h0 = (int)(t % HCT_HB) * HCT_P;
@@ -81,13 +81,13 @@ extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParam
   }
 }
 #else
-extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {
+extern "C" __global__ void __launch_bounds__(HCT_CTA) HCT_KERNEL_NAME(const HctParams hct_p) {
   hct_pdl_launch_dependents();
   hct_pdl_wait();
   const HCT_TA* __restrict__ X = (const HCT_TA*)hct_p.ptr[HCT_PA];
   const HCT_TB* __restrict__ Wt = (const HCT_TB*)hct_p.ptr[HCT_PB];
   const long long units = (long long)HCT_NB * HCT_KO * HCT_HB * HCT_WO;
-  for (long long u = (long long)blockIdx.x * 256 + threadIdx.x; u < units; u += (long long)gridDim.x * 256) {
+  for (long long u = (long long)blockIdx.x * HCT_CTA + threadIdx.x; u < units; u += (long long)gridDim.x * HCT_CTA) {
     const int w = (int)(u % HCT_WO);
     long long t = u / HCT_WO;
     const int hb = (int)(t % HCT_HB);
