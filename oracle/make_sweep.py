@@ -1,4 +1,5 @@
-"""Writes workloads/sweep_specs.json: the 200 random operator DAGs of the graph-augmentation sweep.
+"""Writes workloads/sweep_specs.json: the 200 random operator DAGs of the graph-augmentation sweep,
+and workloads/growth_specs.json: 60 branching multi-output DAGs grown with the whole of Algorithm 1.
 
     python -m oracle.make_sweep
 
@@ -21,10 +22,11 @@ import numpy as np
 
 from oracle import graph as ograph
 from oracle import interp
-from workloads import configs, random_dag, tensors
+from workloads import configs, graph_growth, random_dag, tensors
 
 N_SEEDS = 200
 PROXY_ROWS = 64
+N_GROWN = 60
 OUT = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "workloads", "sweep_specs.json")
 
 
@@ -56,12 +58,14 @@ def well_conditioned(spec: str, laws: dict, seed: int) -> bool:
         v = exact[name]
         if not np.all(np.isfinite(v)) or np.abs(v).max() > 1e30:
             return False
-    out = g.outputs[0][0]
-    a, b = exact[out], single[out].astype(np.float64)
-    if not np.all(np.isfinite(b)):
-        return False
-    rho = column_scale(a)
-    return bool(np.all(np.abs(a - b) <= 2e-6 * np.maximum(np.abs(a), rho)))
+    for out, _ in g.outputs:
+        a, b = exact[out], single[out].astype(np.float64)
+        if not np.all(np.isfinite(b)):
+            return False
+        rho = column_scale(a)
+        if not np.all(np.abs(a - b) <= 2e-6 * np.maximum(np.abs(a), rho)):
+            return False
+    return True
 
 
 def main():
@@ -81,6 +85,22 @@ def main():
         f.write("\n")
     rej = sum(e["attempt"] for e in entries)
     print(f"wrote {OUT}: {len(entries)} graphs, {rej} redraws for conditioning")
+
+    grown = []
+    for seed in range(N_GROWN):
+        attempt = 0
+        while True:
+            proxy_spec, laws, meta = graph_growth.grow_graph(seed, attempt, rows=PROXY_ROWS)
+            if well_conditioned(proxy_spec, laws, seed):
+                break
+            attempt += 1
+            assert attempt < 200, f"grown graph {seed}: no well-conditioned graph in 200 attempts"
+        grown.append(meta)
+    out2 = os.path.join(os.path.dirname(OUT), "growth_specs.json")
+    with open(out2, "w") as f:
+        json.dump({"generator": "workloads.graph_growth.grow_graph(seed, attempt)", "entries": grown}, f, indent=0)
+        f.write("\n")
+    print(f"wrote {out2}: {len(grown)} graphs, {sum(e['attempt'] for e in grown)} redraws for conditioning")
 
 
 if __name__ == "__main__":

@@ -355,10 +355,15 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         << "        float m_[HCT_B];\n        " << FORB << "{\n          m_[b] = -HCT_INF;\n          " << FORE << "if (HCT_HAS(e)) m_[b] = fmaxf(m_[b], " << a
         << ");\n        }\n"
         << "        hct_warp_reduce<true>(m_);\n"
-        << "        float d_[HCT_B], q_[HCT_B];\n        " << FORB << "{\n          const float ml_ = -(m_[b] == -HCT_INF ? 0.0f : m_[b]) * HCT_LOG2E;\n"
-        << "          d_[b] = 0.0f;\n          q_[b] = 0.0f;\n          " << FORE
+        // exp(x - m) as 2^(x*log2e - m*log2e) in one multiply-add: the product m*log2e is rounded on its own,
+        // which scales the warp's terms by up to 2^(|m| * 1.45 * 2^-24).  Below |m| = 16 that is under 1e-6 and
+        // harmless; above, the difference is taken first (exact where it matters, and safe for huge values).
+        << "        float d_[HCT_B], q_[HCT_B];\n        " << FORB << "{\n          const float mr_ = m_[b] == -HCT_INF ? 0.0f : m_[b];\n"
+        << "          d_[b] = 0.0f;\n          q_[b] = 0.0f;\n          if (fabsf(mr_) < 16.0f) {\n            const float ml_ = -mr_ * HCT_LOG2E;\n            " << FORE
         << "{ v" << id << "[b][e] = HCT_HAS(e) ? hct_exp2_fast(fmaf(" << a << ", HCT_LOG2E, ml_)) : 0.0f; d_[b] += v" << id << "[b][e];"
-        << (with_q ? " q_[b] = fmaf(v" + id + "[b][e], v" + id + "[b][e], q_[b]);" : "") << " }\n        }\n"
+        << (with_q ? " q_[b] = fmaf(v" + id + "[b][e], v" + id + "[b][e], q_[b]);" : "") << " }\n          } else {\n            " << FORE
+        << "{ v" << id << "[b][e] = HCT_HAS(e) ? hct_exp2_fast((" << a << " - mr_) * HCT_LOG2E) : 0.0f; d_[b] += v" << id << "[b][e];"
+        << (with_q ? " q_[b] = fmaf(v" + id + "[b][e], v" + id + "[b][e], q_[b]);" : "") << " }\n          }\n        }\n"
         << "        hct_warp_reduce<false>(d_);\n"
         << (with_q ? "        hct_warp_reduce<false>(q_);\n" : "")
         << "        float f_[HCT_B];\n"

@@ -113,6 +113,12 @@ def test_shape_inference_agrees_on_sweep():
         _agree_with_oracle_reader(spec)
 
 
+def test_shape_inference_agrees_on_grown_graphs():
+    for seed in range(0, 60, 6):
+        spec, _, _ = sweep.get_grown(seed, rows=64)
+        _agree_with_oracle_reader(spec)
+
+
 def test_plan_cuts_and_workspace():
     spec = """hct 1
 input x f32 [64,256]

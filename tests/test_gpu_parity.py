@@ -510,6 +510,23 @@ def test_sweep_graphs_reduced_rows(seed):
     check_f32(spec, laws, seed)
 
 
+@pytest.mark.parametrize("mean,std", [(100.0, 30.0), (-5000.0, 3.0), (0.0, 3e9), (2.5e10, 1e10), (15.9, 0.2)])
+@pytest.mark.parametrize("cols", [96, 4096])
+def test_softmax_of_large_magnitudes(mean, std, cols):
+    """Row maxima far from zero: the exponent of every term must be taken relative to the maximum without
+    losing it to the rounding of a large product (also for rows spread over several warps)."""
+    spec = f"hct 1\ninput x f32 [64,{cols}]\nnode p = row_softmax(x)\nnode s = row_sum(p)\noutput p\noutput s\n"
+    check_f32(spec, {"x": {"kind": "normal", "mean": mean, "std": std}})
+
+
+@pytest.mark.parametrize("seed", list(range(60)))
+def test_grown_graphs_reduced_rows(seed):
+    """Branching multi-output graphs grown with the whole of Algorithm 1 (usage caps, random connections,
+    branches, merges), 96 rows each; every output is compared."""
+    spec, laws, _ = sweep.get_grown(seed, rows=96)
+    check_f32(spec, laws, seed)
+
+
 def test_run_twice_is_bitwise_repeatable():
     import torch
     import paper_2506_10401_b200 as hct
