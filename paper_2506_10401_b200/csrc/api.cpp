@@ -213,11 +213,11 @@ hct_status_t hct_graph_run(hct_graph_t* g, const void* const* inputs, int n_inpu
     for (auto& k : g->kernels) {
       // parameter block: tensor maps first (64-byte aligned), then pointers
       struct alignas(64) Params {
-        TensorMap tmap[8];
+        TensorMap tmap[17];   // a strided convolution carries 1 + 2 * stride maps (stride <= 8)
         void* ptr[32];
       } params;
       size_t ntm = k.spec.tmaps.size(), np = k.spec.ptrs.size() + (k.spec.wants_status ? 1 : 0);
-      if (ntm > 8 || np > 32) return set_error(HCT_ERR_UNSUPPORTED, "kernel has too many arguments");
+      if (ntm > 17 || np > 32) return set_error(HCT_ERR_UNSUPPORTED, "kernel has too many arguments");
       void* ptrs[32];
       for (size_t i = 0; i < k.spec.ptrs.size(); ++i) ptrs[i] = resolve(g, k.spec.ptrs[i], inputs, outputs, (char*)workspace);
       if (k.spec.wants_status) ptrs[np - 1] = (void*)g->status_word;
@@ -227,7 +227,7 @@ hct_status_t hct_graph_run(hct_graph_t* g, const void* const* inputs, int n_inpu
       }
       for (size_t i = 0; i < ntm; ++i) {
         const TmaDesc& t = k.spec.tmaps[i];
-        void* base = resolve(g, t.buf, inputs, outputs, (char*)workspace);
+        void* base = (char*)resolve(g, t.buf, inputs, outputs, (char*)workspace) + t.base_offset;
         if (base != k.tmap_base[i]) {
           uint32_t estr[5] = {t.estride[0], t.estride[1], t.estride[2], t.estride[3], t.estride[4]};
           int dtype = t.elem_bytes == 2 ? 9 /* bf16 */ : 7 /* fp32 */;

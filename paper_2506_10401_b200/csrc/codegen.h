@@ -24,6 +24,7 @@ struct TmaDesc {
   uint64_t strides[5] = {0, 0, 0, 0, 0};  // bytes, for dims[1..]; strides[0] unused
   uint32_t box[5] = {1, 1, 1, 1, 1};       // elements traversed; ceil(box / estride) of them are loaded
   uint32_t estride[5] = {1, 1, 1, 1, 1};   // traversal stride per dimension (estride[0] must stay 1)
+  uint64_t base_offset = 0;                // bytes added to the buffer's address (a multiple of 16)
   int swizzle = 3;                // 0 none, 1 32B, 2 64B, 3 128B
 };
 

@@ -83,6 +83,21 @@ struct EpiGen {
     int anchor = grp.nodes[0];
     std::ostringstream loads;
     auto vec_ok = [&](DType d) { return (N % (d == BF16 ? 8 : 4) == 0 && vec_unit % (d == BF16 ? 8 : 4) == 0) ? "true" : "false"; };
+    // Runs whose start is not a whole 16-byte vector but still a multiple of 2 or 4 elements use accesses of
+    // that width (helpers of run_partial.cuh, emitted in front of the function when needed): 0 = not applicable.
+    bool need_partial = false;
+    auto part_w = [&](DType d) -> int {
+      const int64_t full = d == BF16 ? 8 : 4;
+      if (N % full == 0 && vec_unit % full == 0) return 0;
+      for (int64_t w = full / 2; w >= 2; w /= 2)
+        if (N % w == 0 && vec_unit % w == 0) { need_partial = true; return (int)w; }
+      return 0;
+    };
+    auto ld_call = [&](DType d, const std::string& ptr_expr, const std::string& dst) {
+      const int w = part_w(d);
+      if (w) return std::string("hct_ld_run32w<") + std::to_string(w) + ">(" + ptr_expr + ", " + dst + ", ncols);\n";
+      return std::string("hct_ld_run32<") + ctype(d) + ">(" + ptr_expr + ", " + dst + ", ncols, " + vec_ok(d) + ");\n";
+    };
     auto ref = [&](const Operand& a) -> std::string {
       if (a.is_literal()) return float_lit(a.literal);
       if (p.group_of[a.node] == gi) return a.node == anchor ? "acc[j]" : "e" + std::to_string(a.node);
@@ -98,12 +113,10 @@ struct EpiGen {
       std::string ptr = std::string("((const ") + ctype(d) + "*)hct_p.ptr[" + std::to_string(pi) + "])";
       switch (e.bcast) {
         case Bcast::Full:
-          loads << "  float x" << k << "[32]; hct_ld_run32<" << ctype(d) << ">(" << ptr << " + row * " << N << "LL + col0, x" << k
-                << ", ncols, " << vec_ok(d) << ");\n";
+          loads << "  float x" << k << "[32]; " << ld_call(d, ptr + " + row * " + std::to_string(N) + "LL + col0", "x" + std::to_string(k));
           break;
         case Bcast::RowVec:
-          loads << "  float x" << k << "[32]; hct_ld_run32<" << ctype(d) << ">(" << ptr << " + col0, x" << k << ", ncols, " << vec_ok(d)
-                << ");\n";
+          loads << "  float x" << k << "[32]; " << ld_call(d, ptr + " + col0", "x" + std::to_string(k));
           break;
         case Bcast::Scalar: loads << "  const float c" << k << " = hct_ld1(" << ptr << ");\n"; break;
         case Bcast::RowIdx: loads << "  const float c" << k << " = hct_ld1(" << ptr << " + " << rowidx << ");\n"; break;
@@ -126,15 +139,20 @@ struct EpiGen {
     f << "  }\n";
     if (vals_only) {
       f << "}\n";
-      return f.str();
+      return (need_partial ? std::string(skeleton_source("run_partial")) + "\n" : std::string()) + f.str();
     }
     for (auto& st : grp.stores) {
       int pi = ptr_index(st.node, !st.to_output);
-      f << "  hct_st_run32<" << ctype(st.dtype) << ">((" << ctype(st.dtype) << "*)hct_p.ptr[" << pi << "] + row * " << N << "LL + col0, o"
-        << st.node << "_" << (st.to_output ? 1 : 0) << ", ncols, " << vec_ok(st.dtype) << ");\n";
+      const int w = part_w(st.dtype);
+      if (w)
+        f << "  hct_st_run32w<" << w << ">((" << ctype(st.dtype) << "*)hct_p.ptr[" << pi << "] + row * " << N << "LL + col0, o" << st.node << "_"
+          << (st.to_output ? 1 : 0) << ", ncols);\n";
+      else
+        f << "  hct_st_run32<" << ctype(st.dtype) << ">((" << ctype(st.dtype) << "*)hct_p.ptr[" << pi << "] + row * " << N << "LL + col0, o"
+          << st.node << "_" << (st.to_output ? 1 : 0) << ", ncols, " << vec_ok(st.dtype) << ");\n";
     }
     f << "}\n";
-    return f.str();
+    return (need_partial ? std::string(skeleton_source("run_partial")) + "\n" : std::string()) + f.str();
   }
 
   // Epilogue of the tensor-core convolution: one thread owns one output pixel (n,h,w) and 32
@@ -505,7 +523,9 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     // traversal stride (every ST-th pixel of every ST-th row), which the tensor map allows up to 8 and a box of 256.
     const int64_t ST = anchor.stride, DIL = anchor.dilation;
     const bool unit = ST == 1 && DIL == 1;
-    if (in_bf16 && anchor.groups == 1 && ST <= 8 && WO * ST <= 256 && C % 8 == 0 && WO <= 256 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
+    // a stride that divides both image extents: dense boxes of a phase view instead of strided boxes
+    const bool phased = ST > 1 && ST <= 8 && H % ST == 0 && W % ST == 0;
+    if (in_bf16 && anchor.groups == 1 && ST <= 8 && (WO * ST <= 256 || phased) && C % 8 == 0 && WO <= 256 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
       // Three schedules.  (1) Rows whose byte length is a multiple of 16 and that fill most of a 32-column
       // pitch: the kernel reads NCHW itself and re-lays pixels in shared memory (conv_tc_nchw); only the
       // weights take a pre-pass.  Otherwise a pre-pass writes an NHWC copy and pixels are loaded
@@ -526,7 +546,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         direct = n_a >= 3;
       }
       const bool halo = unit && !direct && FS > 1 && dense_pitch && !tun.conv_no_halo;
-      const int TH = (direct || halo) ? th_pitch : (int)std::max<int64_t>(1, std::min<int64_t>(256 / WO, std::min<int64_t>(HO, 256 / ST)));
+      const int TH = (direct || halo) ? th_pitch : (int)std::max<int64_t>(1, std::min<int64_t>(256 / WO, std::min<int64_t>(HO, phased ? 256 : 256 / ST)));
       auto align256 = [](int64_t v) { return (v + 255) / 256 * 256; };
       const int64_t x_bytes = direct ? 0 : align256(NB * C * H * W * 2), w_bytes = align256(KO * C * FR * FS * 2);
       *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(x_bytes + w_bytes));
@@ -565,11 +585,11 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       std::ostringstream src;
       src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_H " << H << "\n#define HCT_W " << W
           << "\n#define HCT_KO " << KO << "\n#define HCT_FR " << FR << "\n#define HCT_FS " << FS << "\n#define HCT_PAD " << anchor.pad
-          << "\n#define HCT_STRIDE " << ST << "\n#define HCT_DIL " << DIL << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TH " << TH << "\n#define HCT_TH2 1\n#define HCT_SPLIT "
+          << "\n#define HCT_STRIDE " << ST << "\n#define HCT_DIL " << DIL << "\n#define HCT_PHASED " << (phased ? 1 : 0) << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TH " << TH << "\n#define HCT_TH2 1\n#define HCT_SPLIT "
           << TH << "\n#define HCT_PITCH " << pitch << "\n#define HCT_NA " << (direct ? n_a : 6) << "\n#define HCT_NBUF " << (direct ? n_buf : 3)
           << "\n#define HCT_NSTG " << n_stg << "\n#define HCT_X_IS_INPUT " << (a.cls == OpClass::Input ? 1 : 0) << "\n#define HCT_TMA_STORE " << (use_tma_store ? 1 : 0) << "\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
           << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
-      src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[" << (use_tma_store ? 3 : direct ? 2 : 3)
+      src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[" << (phased ? 1 + 2 * ST : use_tma_store ? 3 : direct ? 2 : 3)
           << "]; void* ptr[" << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source(direct ? "conv_tc_nchw" : halo ? "conv_tc_halo" : "conv_tc");
       k.source = src.str();
       k.ptrs = eg.ptrs;
@@ -587,11 +607,28 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       tx.rank = 4;
       tx.dims[0] = (uint64_t)C; tx.dims[1] = (uint64_t)W; tx.dims[2] = (uint64_t)H; tx.dims[3] = (uint64_t)NB;
       tx.strides[1] = (uint64_t)C * 2; tx.strides[2] = (uint64_t)W * C * 2; tx.strides[3] = (uint64_t)H * W * C * 2;
-      tx.box[0] = 64; tx.box[1] = (uint32_t)(halo ? pitch : WO * ST); tx.box[2] = (uint32_t)(TH * ST); tx.box[3] = 1;
-      tx.estride[1] = tx.estride[2] = (uint32_t)ST;
+      tx.box[0] = 64; tx.box[1] = (uint32_t)(halo ? pitch : phased ? 1 : WO * ST); tx.box[2] = (uint32_t)(phased ? 1 : TH * ST); tx.box[3] = 1;
+      tx.estride[1] = tx.estride[2] = (uint32_t)(phased ? 1 : ST);   // (with a phase view these two maps are replaced below)
       TmaDesc tx2 = tx;
-      tx2.box[2] = (uint32_t)ST;
+      tx2.box[2] = (uint32_t)(phased ? 1 : ST);
       k.tmaps = {tw, tx, tx2};
+      if (phased) {
+        // view of the NHWC copy for row phase ph: [n][h / ST][w / ST][w mod ST][c], starting ph rows into each image
+        k.tmaps = {tw};
+        for (int piece = 0; piece < 2; ++piece)
+          for (int64_t ph = 0; ph < ST; ++ph) {
+            TmaDesc tp;
+            tp.buf = scratch(0);
+            tp.base_offset = (uint64_t)(ph * W * C * 2);
+            tp.elem_bytes = 2;
+            tp.rank = 5;
+            tp.dims[0] = (uint64_t)C; tp.dims[1] = (uint64_t)ST; tp.dims[2] = (uint64_t)(W / ST); tp.dims[3] = (uint64_t)(H / ST); tp.dims[4] = (uint64_t)NB;
+            tp.strides[1] = (uint64_t)C * 2; tp.strides[2] = (uint64_t)ST * C * 2; tp.strides[3] = (uint64_t)ST * W * C * 2;
+            tp.strides[4] = (uint64_t)H * W * C * 2;
+            tp.box[0] = 64; tp.box[1] = 1; tp.box[2] = (uint32_t)WO; tp.box[3] = (uint32_t)(piece ? 1 : TH); tp.box[4] = 1;
+            k.tmaps.push_back(tp);
+          }
+      }
       if (direct) {  // NCHW input: [64 channels x pitch pixels] of one row, no swizzle (the kernel re-lays it)
         TmaDesc tn;
         tn.buf = node_buf(anchor.args[0].node);
@@ -630,7 +667,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       else if (halo)
         d << "pixels shared by the taps of a filter row (pitch " << pitch << ")";
       else
-        d << stages << " stages" << (unit ? "" : ", strided pixel boxes");
+        d << stages << " stages" << (unit ? "" : phased ? ", dense pixel boxes of a stride-phase view" : ", strided pixel boxes");
       k.desc = d.str();
       out->push_back(k);
       return;

@@ -14,9 +14,16 @@
 // Work is split into tiles of HCT_TH output rows; when the last round over the SMs would be
 // nearly empty, its tiles are cut into HCT_TH2-row pieces so that all SMs finish together.
 //
-// Defined by the generator: HCT_NB_IMG, HCT_C, HCT_H, HCT_W, HCT_KO, HCT_FR, HCT_FS, HCT_PAD, HCT_STRIDE, HCT_DIL, HCT_HO, HCT_WO,
+// Defined by the generator: HCT_NB_IMG, HCT_C, HCT_H, HCT_W, HCT_KO, HCT_FR, HCT_FS, HCT_PAD, HCT_STRIDE, HCT_DIL, HCT_PHASED, HCT_HO, HCT_WO,
 // HCT_TH, HCT_TH2, HCT_SPLIT (pieces per cut tile, HCT_TH2 * HCT_SPLIT >= HCT_TH), HCT_STAGES,
 // HCT_STATUS_SLOT, HCT_KERNEL_NAME, HctParams, hct_epilogue_run().
+//
+// HCT_PHASED (stride > 1 dividing the image's height and width): the NHWC copy is viewed as
+// [n][h / stride][w / stride][w mod stride][c] through one tensor map per row phase h mod stride, so the
+// pixels a tap needs are a dense box of that view (coordinate = tap offset divided by the stride,
+// phase = its remainder) and the copies run at the rate of ordinary tiles; a box with a traversal
+// stride delivers the same pixels but was measured 4x slower.  Maps: [0] weights, [1 + phase] whole
+// tiles, [1 + stride + phase] one-row pieces.
 #define HCT_BM 128
 #define HCT_A_BYTES (HCT_BM * 128)                       // weights: 128 channels x 64 inputs, bf16
 #define HCT_B_BYTES 32768                                // pixels: up to 256 x 64 inputs
@@ -26,6 +33,16 @@
 #define HCT_HT ((HCT_HO + HCT_TH - 1) / HCT_TH)
 #define HCT_MBK ((HCT_KO + HCT_BM - 1) / HCT_BM)
 #define HCT_FULL_TILES ((long long)HCT_NB_IMG * HCT_HT * HCT_MBK)
+
+#if HCT_PHASED
+__device__ __forceinline__ void hct_tma_load_5d(hct_u32 dst, const HctTensorMap* map, int c0, int c1, int c2, int c3, int c4, hct_u32 bar) {
+  asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];" ::"r"(dst),
+               "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
+               : "memory");
+}
+// floor(a / HCT_STRIDE) and the non-negative remainder, for offsets that may be negative (padding)
+__device__ __forceinline__ int hct_floordiv(int a) { return (a >= 0 ? a : a - (HCT_STRIDE - 1)) / HCT_STRIDE; }
+#endif
 
 struct HctConvTile { int n, h0, th, mbk; bool cut; };
 
@@ -83,8 +100,12 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     hct_prefetch_tmap(&hct_p.tmap[0]);
+#if HCT_PHASED
+    for (int i = 1; i < 1 + 2 * HCT_STRIDE; ++i) hct_prefetch_tmap(&hct_p.tmap[i]);
+#else
     hct_prefetch_tmap(&hct_p.tmap[1]);
     hct_prefetch_tmap(&hct_p.tmap[2]);
+#endif
   }
   if (warp == 1) hct_tmem_alloc(hct_smem_addr(&tmem_holder), 512);
   hct_tc_fence_before();
@@ -101,7 +122,9 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
         const HctConvTile t = hct_conv_tile(tile, t1);
         if (t.th == 0) continue;
         // whole tiles use the HCT_TH-row box, pieces the HCT_TH2-row box
+#if !HCT_PHASED
         const HctTensorMap* xmap = t.cut ? &hct_p.tmap[2] : &hct_p.tmap[1];
+#endif
         const hct_u32 bytes = HCT_A_BYTES + (hct_u32)(t.cut ? HCT_TH2 : HCT_TH) * HCT_WO * 128u;
         for (int kb = 0; kb < HCT_KB; ++kb) {
           const int tap = kb / HCT_CB, cb = kb % HCT_CB;
@@ -111,7 +134,16 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
           hct_mbar_expect_tx(full, bytes);
           const hct_u32 dst = smem_base + stage * HCT_STAGE_BYTES;
           hct_tma_load_2d(dst, &hct_p.tmap[0], cb * 64, tap * HCT_KO + t.mbk * HCT_BM, full);
+#if HCT_PHASED
+          {
+            const int a = s * HCT_DIL - HCT_PAD, b = r * HCT_DIL - HCT_PAD;
+            const int wq = hct_floordiv(a), hq = hct_floordiv(b);
+            const int pw = a - wq * HCT_STRIDE, ph = b - hq * HCT_STRIDE;
+            hct_tma_load_5d(dst + HCT_A_BYTES, &hct_p.tmap[1 + (t.cut ? HCT_STRIDE : 0) + ph], cb * 64, pw, wq, t.h0 + hq, t.n, full);
+          }
+#else
           hct_tma_load_4d(dst + HCT_A_BYTES, xmap, cb * 64, s * HCT_DIL - HCT_PAD, t.h0 * HCT_STRIDE + r * HCT_DIL - HCT_PAD, t.n, full);
+#endif
           if (++stage == HCT_STAGES) { stage = 0; phase ^= 1u; }
         }
       }

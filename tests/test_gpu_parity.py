@@ -248,18 +248,25 @@ def test_conv_bf16_nchw_direct_integer_inputs_are_exact():
 @pytest.mark.parametrize("shape,wshape,attrs", [
     ((2, 64, 28, 30), (96, 64, 3, 3), "stride=2, pad=1"),
     ((1, 128, 56, 56), (256, 128, 1, 1), "stride=2, pad=0"),          # downsampling 1x1
-    ((2, 16, 23, 19), (40, 16, 3, 3), "stride=3, pad=1"),
+    ((2, 16, 23, 19), (40, 16, 3, 3), "stride=3, pad=1"),             # extents not divisible by the stride: strided boxes
+    ((2, 16, 24, 18), (40, 16, 3, 3), "stride=3, pad=1"),
+    ((1, 8, 16, 32), (16, 8, 3, 3), "stride=4, pad=1, dilation=3"),
+    ((3, 24, 12, 16), (20, 24, 5, 5), "stride=2, pad=4"),             # padding beyond half the filter
+    ((1, 8, 40, 72), (16, 8, 5, 5), "stride=8, pad=2"),
     ((1, 72, 21, 26), (130, 72, 3, 3), "stride=1, pad=2, dilation=2"),
     ((2, 8, 25, 31), (8, 8, 3, 2), "stride=2, pad=3, dilation=3"),
     ((1, 8, 40, 70), (16, 8, 5, 5), "stride=8, pad=2"),
-    ((1, 8, 6, 300), (8, 8, 3, 3), "stride=2, pad=1"),                # too wide for one strided box: fp32-FMA kernel
+    ((1, 8, 6, 300), (8, 8, 3, 3), "stride=2, pad=1"),
+    ((1, 8, 6, 301), (8, 8, 3, 3), "stride=2, pad=1"),                # too wide for one strided box: fp32-FMA kernel
 ])
 def test_conv_bf16_stride_and_dilation_integer_inputs_are_exact(shape, wshape, attrs):
     dims = lambda t: "[" + ",".join(str(v) for v in t) + "]"
     spec = f"hct 1\ninput x bf16 {dims(shape)}\ninput w bf16 {dims(wshape)}\nnode y = conv2d(x, w, {attrs})\noutput y f32\n"
     il = {"kind": "int", "lo": -4, "hi": 4}
     got, want, g = parity.run_both(spec, {"x": il, "w": il})
-    assert ("strided pixel boxes" in g.plan) == (shape[3] != 300)
+    assert ("pixel boxes" in g.plan) == (shape[3] != 301)
+    divisible = shape[2] % int(attrs[7]) == 0 and shape[3] % int(attrs[7]) == 0
+    assert ("stride-phase view" in g.plan) == (int(attrs[7]) > 1 and divisible)
     np.testing.assert_array_equal(got[0], want[0])
 
 
