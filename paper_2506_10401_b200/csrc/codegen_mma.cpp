@@ -523,8 +523,9 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     // traversal stride (every ST-th pixel of every ST-th row), which the tensor map allows up to 8 and a box of 256.
     const int64_t ST = anchor.stride, DIL = anchor.dilation;
     const bool unit = ST == 1 && DIL == 1;
-    // a stride that divides both image extents: dense boxes of a phase view instead of strided boxes
-    const bool phased = ST > 1 && ST <= 8 && H % ST == 0 && W % ST == 0;
+    // Rows too wide for one strided box (W' * stride > 256) with a stride that divides both image extents:
+    // dense boxes of a stride-phase view.  Both forms were measured at the same speed; `conv_phase=1` prefers the view.
+    const bool phased = ST > 1 && ST <= 8 && H % ST == 0 && W % ST == 0 && (WO * ST > 256 || tun.conv_phase);
     if (in_bf16 && anchor.groups == 1 && ST <= 8 && (WO * ST <= 256 || phased) && C % 8 == 0 && WO <= 256 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
       // Three schedules.  (1) Rows whose byte length is a multiple of 16 and that fill most of a 32-column
       // pitch: the kernel reads NCHW itself and re-lays pixels in shared memory (conv_tc_nchw); only the

@@ -18,12 +18,12 @@
 // HCT_TH, HCT_TH2, HCT_SPLIT (pieces per cut tile, HCT_TH2 * HCT_SPLIT >= HCT_TH), HCT_STAGES,
 // HCT_STATUS_SLOT, HCT_KERNEL_NAME, HctParams, hct_epilogue_run().
 //
-// HCT_PHASED (stride > 1 dividing the image's height and width): the NHWC copy is viewed as
+// HCT_PHASED (stride > 1 dividing the image's height and width; used where a row times the stride
+// exceeds the 256 elements a box may span): the NHWC copy is viewed as
 // [n][h / stride][w / stride][w mod stride][c] through one tensor map per row phase h mod stride, so the
 // pixels a tap needs are a dense box of that view (coordinate = tap offset divided by the stride,
-// phase = its remainder) and the copies run at the rate of ordinary tiles; a box with a traversal
-// stride delivers the same pixels but was measured 4x slower.  Maps: [0] weights, [1 + phase] whole
-// tiles, [1 + stride + phase] one-row pieces.
+// phase = its remainder).  Both forms deliver the same pixels at the same measured speed.
+// Maps: [0] weights, [1 + phase] whole tiles, [1 + stride + phase] one-row pieces.
 #define HCT_BM 128
 #define HCT_A_BYTES (HCT_BM * 128)                       // weights: 128 channels x 64 inputs, bf16
 #define HCT_B_BYTES 32768                                // pixels: up to 256 x 64 inputs

@@ -259,14 +259,16 @@ def test_conv_bf16_nchw_direct_integer_inputs_are_exact():
     ((1, 8, 6, 300), (8, 8, 3, 3), "stride=2, pad=1"),
     ((1, 8, 6, 301), (8, 8, 3, 3), "stride=2, pad=1"),                # too wide for one strided box: fp32-FMA kernel
 ])
-def test_conv_bf16_stride_and_dilation_integer_inputs_are_exact(shape, wshape, attrs):
+@pytest.mark.parametrize("schedule", [None, "conv_phase=1"])
+def test_conv_bf16_stride_and_dilation_integer_inputs_are_exact(shape, wshape, attrs, schedule):
     dims = lambda t: "[" + ",".join(str(v) for v in t) + "]"
     spec = f"hct 1\ninput x bf16 {dims(shape)}\ninput w bf16 {dims(wshape)}\nnode y = conv2d(x, w, {attrs})\noutput y f32\n"
     il = {"kind": "int", "lo": -4, "hi": 4}
-    got, want, g = parity.run_both(spec, {"x": il, "w": il})
+    got, want, g = parity.run_both(spec, {"x": il, "w": il}, schedule=schedule)
     assert ("pixel boxes" in g.plan) == (shape[3] != 301)
-    divisible = shape[2] % int(attrs[7]) == 0 and shape[3] % int(attrs[7]) == 0
-    assert ("stride-phase view" in g.plan) == (int(attrs[7]) > 1 and divisible)
+    stride = int(attrs[7])
+    divisible = stride > 1 and shape[2] % stride == 0 and shape[3] % stride == 0
+    assert ("stride-phase view" in g.plan) == (divisible and (schedule is not None or shape[3] == 300))
     np.testing.assert_array_equal(got[0], want[0])
 
 
