@@ -36,6 +36,10 @@
  *           (row_softmax also accepts a single column, where it is identically one)
  *           row_layernorm(x, gamma, beta, eps=1e-5)   biased variance, eps inside the root
  *   transpose(x)          y[j,i] = x[i,j] for x[R,C]; elementwise consumers are applied at the store
+ *   row_sort(x, descending=0)   the values of every row of x[R,C] in non-decreasing (descending=1:
+ *                         non-increasing) order; row_topk(x, k=K) the K largest values of every row,
+ *                         largest first, as [R,K].  C <= 8192.  Values are moved, never changed;
+ *                         elementwise consumers are applied at the store
  *   gemm(a, b)            a[M,K] · b[K,N], both row-major, both f32 or both bf16 inputs;
  *                         bf16 multiplies on tensor cores with fp32 accumulation, f32
  *                         uses error-compensated TF32 products (or fp32 FMA for shapes

@@ -229,6 +229,20 @@ def _infer(g, name, op, pos, attrs, where):
         if len(s) != 2 or s[1] < (1 if op == "row_softmax" else 2):
             raise SpecError(f"{where}: {op} needs a [R,C] operand with enough columns")
         return Node(name, op, [a], {}, s if op in ROW_TO_ROW else (s[0], 1), "f32")
+    if op in ("row_sort", "row_topk"):
+        only_attrs("k") if op == "row_topk" else only_attrs("descending")
+        if len(pos) != 1:
+            raise SpecError(f"{where}: {op} takes one operand")
+        a = _operand(g, pos[0], where, False)
+        s = shape_of(a)
+        if len(s) != 2:
+            raise SpecError(f"{where}: {op} needs a [R,C] operand")
+        if op == "row_topk":
+            k = _int_attr(attrs, "k", 1, where)
+            if k < 1 or k > s[1]:
+                raise SpecError(f"{where}: row_topk needs 1 <= k <= C")
+            return Node(name, op, [a], {"k": k}, (s[0], k), "f32")
+        return Node(name, op, [a], {"descending": _int_attr(attrs, "descending", 0, where)}, s, "f32")
     if op == "transpose":
         only_attrs()
         if len(pos) != 1:

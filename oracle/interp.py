@@ -96,6 +96,19 @@ def row_max(x):
     return x.max(axis=1, keepdims=True)
 
 
+# ---- logic-intensive operators (Table 1): ordering the values of a row ------------------------
+
+def row_sort(x, descending=False):
+    # y[i, :] holds the values of x[i, :] in non-decreasing (non-increasing) order
+    y = np.sort(x, axis=1, kind="stable")
+    return y[:, ::-1].copy() if descending else y
+
+
+def row_topk(x, k):
+    # the k largest values of every row, largest first
+    return row_sort(x, descending=True)[:, :k].copy()
+
+
 # ---- layout transform (Table 1, "LayoutTransform") ------------------------------------------
 
 def transpose(x):
@@ -207,6 +220,10 @@ def run_nodes(spec, inputs: dict, dtype=np.float64, gemm_fn=None) -> dict:
         elif op in BINARY:
             out = _BINARY_FN[op](args[0], args[1])
             out = np.broadcast_to(out, node.shape)
+        elif op == "row_sort":
+            out = row_sort(args[0], bool(node.attrs["descending"]))
+        elif op == "row_topk":
+            out = row_topk(args[0], node.attrs["k"])
         elif op == "transpose":
             out = transpose(args[0])
         elif op == "row_softmax":

@@ -213,8 +213,36 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
   const Group& grp = p.groups[gi];
   const Node& anchor = g.nodes[grp.nodes[0]];
   const Node& a = g.nodes[anchor.args[0].node];
-  const Node& b = g.nodes[anchor.args[1].node];
+  const Node& b = g.nodes[anchor.args[anchor.args.size() > 1 ? 1 : 0].node];   // transpose and sort have one operand
   EpiGen eg{g, p, grp, gi, {}};
+
+  // ---- row sort / top-k: bitonic network in shared memory, one CTA per row, consumers applied at the store
+  if (grp.kind == GroupKind::Sort) {
+    const int src = anchor.args[0].node;
+    const int64_t R = a.shape[0], C = a.shape[1], KOUT = anchor.shape[1];
+    int64_t NP = 2;
+    while (NP < C) NP *= 2;
+    const int64_t T = std::max<int64_t>(32, std::min<int64_t>(512, NP / 2));
+    const int pa = eg.ptr_index(src, g.nodes[src].cls != OpClass::Input && p.ws_offset[src] >= 0);
+    const DType ta = eg.buf_dtype(src);
+    std::string epi = eg.scalar_fn();
+    KernelSpec k;
+    k.name = "hct_row_sort_g" + std::to_string(gi);
+    std::ostringstream src_text;
+    src_text << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "\n#define HCT_NP " << NP << "\n#define HCT_KOUT " << KOUT
+             << "\n#define HCT_DESC " << (anchor.descending ? 1 : 0) << "\n#define HCT_T " << T << "\n#define HCT_TA " << ctype(ta)
+             << "\n#define HCT_PA " << pa << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+             << skeleton_source("common") << "\nstruct HctParams { void* ptr[" << eg.ptrs.size() << "]; };\n" << epi << skeleton_source("row_sort");
+    k.source = src_text.str();
+    k.ptrs = eg.ptrs;
+    // resident CTAs per SM: limited by threads (2048) and by shared memory (4 * NP bytes each)
+    const int64_t per_sm = std::max<int64_t>(1, std::min<int64_t>(2048 / T, std::min<int64_t>(16, (200 * 1024) / (4 * NP))));
+    k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(R, 148 * per_sm));
+    k.block[0] = (unsigned)T;
+    k.desc = std::string(anchor.sort_k ? "row top-k" : "row sort") + ": bitonic network over " + std::to_string(NP) + " shared-memory slots, one CTA per row";
+    out->push_back(k);
+    return;
+  }
 
   // ---- layout transform: tiled transposition through shared memory, consumers applied at the store
   if (grp.kind == GroupKind::Transpose) {

@@ -308,6 +308,20 @@ Graph parse_spec(const std::string& text) {
         auto& s = g.nodes[n.args[0].node].shape;
         if (s.size() != 2) fail(HCT_ERR_GRAPH, line, "transpose needs a [R,C] operand, got " + shape_str(s));
         n.shape = {s[1], s[0]};
+      } else if (op == "row_sort" || op == "row_topk") {
+        // logic-intensive operators (Table 1): the values of every row in order; row_topk keeps the k largest, largest first
+        const bool topk = op == "row_topk";
+        if (topk) only_attrs({"k"}); else only_attrs({"descending"});
+        if (pos.size() != 1) fail(HCT_ERR_GRAPH, line, op + " takes one operand");
+        n.cls = OpClass::Sort;
+        n.args = {lookup(pos[0], line, false)};
+        auto& s = g.nodes[n.args[0].node].shape;
+        if (s.size() != 2) fail(HCT_ERR_GRAPH, line, op + " needs a [R,C] operand, got " + shape_str(s));
+        if (s[1] > 8192) fail(HCT_ERR_UNSUPPORTED, line, op + " supports rows of up to 8192 elements");
+        n.descending = topk || int_attr("descending", 0) != 0;
+        n.sort_k = topk ? int_attr("k", 1) : 0;
+        if (topk && (n.sort_k < 1 || n.sort_k > s[1])) fail(HCT_ERR_GRAPH, line, "row_topk needs 1 <= k <= C");
+        n.shape = {s[0], topk ? (int64_t)n.sort_k : s[1]};
       } else if (op == "gemm") {
         only_attrs({"precision"});
         if (pos.size() != 2) fail(HCT_ERR_GRAPH, line, "gemm takes (a, b)");

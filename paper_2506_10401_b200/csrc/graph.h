@@ -9,7 +9,7 @@ namespace hct {
 
 enum DType { F32 = 0, BF16 = 1 };
 
-enum class OpClass { Input, Unary, Binary, RowSoftmax, RowLayernorm, RowReduce, Gemm, Conv, Transpose };
+enum class OpClass { Input, Unary, Binary, RowSoftmax, RowLayernorm, RowReduce, Gemm, Conv, Transpose, Sort };
 
 struct Error : std::runtime_error {
   int code;
@@ -31,6 +31,8 @@ struct Node {
   DType dtype = F32;  // storage dtype of an input; computed nodes are fp32 values (BF16: values rounded to bfloat16 by cast_bf16)
   double eps = 1e-5;
   int stride = 1, pad = 0, dilation = 1, groups = 1;
+  int sort_k = 0;            // row_topk: number of leading elements kept (0: the whole sorted row)
+  bool descending = false;   // row_sort / row_topk: largest first
   // dropout: element with flat index i is kept when hash(i + seed) mod 1000 >= drop_threshold (= round(1000 p))
   double drop_p = 0.0;
   uint64_t drop_seed = 0;

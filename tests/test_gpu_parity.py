@@ -519,6 +519,44 @@ def test_sweep_graphs_reduced_rows(seed):
     check_f32(spec, laws, seed)
 
 
+# ------------------------------------------------------------------ logic-intensive operators: row sort and top-k
+
+@pytest.mark.parametrize("rows,cols", [(5, 1), (7, 2), (33, 5), (64, 100), (40, 1024), (9, 3000), (6, 4096), (3, 8192)])
+@pytest.mark.parametrize("descending", [0, 1])
+def test_row_sort_moves_values_exactly(rows, cols, descending):
+    spec = f"hct 1\ninput x f32 [{rows},{cols}]\nnode s = row_sort(x, descending={descending})\noutput s\n"
+    for law in (N_, {"kind": "int", "lo": -6, "hi": 6}):        # distinct values, and many equal ones
+        got, want, g = parity.run_both(spec, {"x": law})
+        assert "bitonic" in g.plan
+        np.testing.assert_array_equal(got[0], want[0])
+
+
+@pytest.mark.parametrize("cols,k", [(7, 1), (100, 8), (1000, 1000), (4096, 50), (300, 299)])
+def test_row_topk_with_fused_consumers(cols, k):
+    spec = (f"hct 1\ninput x bf16 [37,{cols}]\ninput b f32 [{k}]\nnode t = row_topk(x, k={k})\nnode u = add(t, b)\n"
+            "node v = relu(u)\noutput t\noutput v\n")
+    got, want, g = parity.run_both(spec, {"x": N_, "b": N_})
+    assert g.num_kernels == 1
+    np.testing.assert_array_equal(got[0], want[0])               # the selected values are inputs, moved unchanged
+    assert parity.f32_violation(got[1], want[1]) <= 1.0
+
+
+def test_sort_inside_a_chain():
+    spec = """hct 1
+input x f32 [50,777]
+input w f32 [16,40]
+node a = gelu_tanh(x)
+node s = row_sort(a)
+node p = row_softmax(s)
+node t = row_topk(p, k=16)
+node y = gemm(t, w)
+output y
+output s
+"""
+    g = check_f32(spec, {"x": N_, "w": N_})
+    assert g.num_kernels >= 4
+
+
 @pytest.mark.parametrize("mean,std", [(100.0, 30.0), (-5000.0, 3.0), (0.0, 3e9), (2.5e10, 1e10), (15.9, 0.2)])
 @pytest.mark.parametrize("cols", [96, 4096])
 def test_softmax_of_large_magnitudes(mean, std, cols):

@@ -342,6 +342,48 @@ def test_conv_structure_pins():
     np.testing.assert_array_equal(interp.conv2d(xi, wi, 1, 1), _conv_loops(xi, wi, 1, 1))
 
 
+# ---------------------------------------------------------------- row_sort / row_topk
+
+def _insertion_sorted(row):
+    out = []
+    for v in row:
+        i = 0
+        while i < len(out) and out[i] <= v:
+            i += 1
+        out.insert(i, v)
+    return out
+
+
+def test_sort_hand_values_bruteforce_and_invariants():
+    x = np.array([[3.0, 1.0, 2.0, 5.0, 4.0], [0.0, -1.0, 7.0, 7.0, 2.0], [1.0, 1.0, 1.0, 0.0, 9.0]])
+    np.testing.assert_array_equal(interp.row_sort(x), [[1, 2, 3, 4, 5], [-1, 0, 2, 7, 7], [0, 1, 1, 1, 9]])
+    np.testing.assert_array_equal(interp.row_sort(x, descending=True), [[5, 4, 3, 2, 1], [7, 7, 2, 0, -1], [9, 1, 1, 1, 0]])
+    np.testing.assert_array_equal(interp.row_topk(x, 2), [[5, 4], [7, 7], [9, 1]])
+    y = RNG.integers(-5, 6, size=(7, 23)).astype(np.float64)          # many equal values
+    z = RNG.normal(size=(5, 40))
+    for a in (y, z):
+        s = interp.row_sort(a)
+        for i in range(a.shape[0]):
+            assert list(s[i]) == _insertion_sorted(list(a[i]))
+        assert np.all(np.diff(s, axis=1) >= 0)
+        np.testing.assert_array_equal(interp.row_sort(a, descending=True), s[:, ::-1])
+        # sorting is invariant under a permutation of the columns and idempotent
+        np.testing.assert_array_equal(interp.row_sort(a[:, RNG.permutation(a.shape[1])]), s)
+        np.testing.assert_array_equal(interp.row_sort(s), s)
+        # top-k by repeatedly removing the maximum
+        for k in (1, 3, a.shape[1]):
+            t = interp.row_topk(a, k)
+            for i in range(a.shape[0]):
+                rest, want = list(a[i]), []
+                for _ in range(k):
+                    m = max(rest)
+                    want.append(m)
+                    rest.remove(m)
+                assert list(t[i]) == want
+    g = oracle.parse("hct 1\ninput x f32 [4,9]\nnode t = row_topk(x, k=3)\nnode s = row_sort(x, descending=1)\noutput t\noutput s\n")
+    assert g.nodes["t"].shape == (4, 3) and g.nodes["s"].shape == (4, 9)
+
+
 # ---------------------------------------------------------------- graph validity (paper section 3.2)
 
 GOOD = "hct 1\ninput x f32 [4,8]\ninput b f32 [8]\nnode t = add(x, b)\nnode y = row_softmax(t)\noutput y\n"
@@ -540,6 +582,8 @@ def test_planted_mistakes_are_detected(monkeypatch):
         return orig["gelu_erf"](x)
 
     plants = [
+        ("row_sort", lambda x, descending=False: orig["row_sort"](x, not descending), test_sort_hand_values_bruteforce_and_invariants),
+        ("row_topk", lambda x, k: orig["row_sort"](x)[:, :k], test_sort_hand_values_bruteforce_and_invariants),
         ("row_layernorm", unbiased_ln, test_layernorm_closed_forms),
         ("row_layernorm", eps_outside_ln, test_layernorm_bruteforce_and_torch),
         ("conv2d", flipped_conv, test_conv_structure_pins),
