@@ -226,6 +226,27 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     const int pa = eg.ptr_index(src, g.nodes[src].cls != OpClass::Input && p.ws_offset[src] >= 0);
     const DType ta = eg.buf_dtype(src);
     std::string epi = eg.scalar_fn();
+    if (anchor.sort_k > 0 && anchor.sort_k <= 256 && C >= 2 && !tun.topk_no_select) {
+      // small k: radix selection of the k-th largest key, then a sort of the k selected values only
+      int64_t KP = 2;
+      while (KP < KOUT) KP *= 2;
+      KernelSpec k;
+      k.name = "hct_row_topk_g" + std::to_string(gi);
+      std::ostringstream st;
+      st << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "\n#define HCT_K " << KOUT << "\n#define HCT_KP " << KP
+         << "\n#define HCT_T 256\n#define HCT_TA " << ctype(ta) << "\n#define HCT_PA " << pa << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+         << skeleton_source("common") << "\nstruct HctParams { void* ptr[" << eg.ptrs.size() << "]; };\n" << epi << skeleton_source("row_topk");
+      k.source = st.str();
+      k.ptrs = eg.ptrs;
+      const int64_t per_sm = std::max<int64_t>(1, std::min<int64_t>(8, (200 * 1024) / (4 * C + 4 * KP + 1280)));
+      k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(R, 148 * per_sm));
+      k.block[0] = 256;
+      k.desc = std::string("row top-k: ") + (KOUT <= 64 ? "bound from per-thread maxima and a 128-slot bitonic network, else " : "") +
+               "radix selection of the k-th largest key in shared memory, one CTA per row, then a bitonic network over " + std::to_string(KP) +
+               " selected keys";
+      out->push_back(k);
+      return;
+    }
     KernelSpec k;
     k.name = "hct_row_sort_g" + std::to_string(gi);
     std::ostringstream src_text;

@@ -38,6 +38,7 @@ const Knob kKnobs[] = {
     {"conv_no_tma_store", nullptr, 0, &Tunables::conv_no_tma_store},
     {"conv_no_direct", nullptr, 0, &Tunables::conv_no_direct},
     {"conv_phase", nullptr, 0, &Tunables::conv_phase},
+    {"topk_no_select", nullptr, 0, &Tunables::topk_no_select},
     {"row_no_small_ctas", nullptr, 0, &Tunables::row_no_small_ctas},
     {"row_no_reg_rowvec", nullptr, 0, &Tunables::row_no_reg_rowvec},
     {"row_no_softmax_ln_fusion", nullptr, 0, &Tunables::row_no_softmax_ln_fusion},

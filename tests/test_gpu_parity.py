@@ -541,6 +541,37 @@ def test_row_topk_with_fused_consumers(cols, k):
     assert parity.f32_violation(got[1], want[1]) <= 1.0
 
 
+@pytest.mark.parametrize("rows,cols,k", [(3, 2, 1), (16, 64, 64), (40, 777, 5), (9, 8192, 256), (21, 4096, 33), (12, 1000, 128)])
+@pytest.mark.parametrize("law", ["normal", "ties"])
+def test_row_topk_radix_selection_moves_values_exactly(rows, cols, k, law):
+    spec = f"hct 1\ninput x f32 [{rows},{cols}]\nnode t = row_topk(x, k={k})\noutput t\n"
+    got, want, g = parity.run_both(spec, {"x": N_ if law == "normal" else {"kind": "int", "lo": -3, "hi": 3}})
+    assert "radix selection" in g.plan
+    np.testing.assert_array_equal(got[0], want[0])
+    got2, _, g2 = parity.run_both(spec, {"x": N_ if law == "normal" else {"kind": "int", "lo": -3, "hi": 3}}, schedule="topk_no_select=1")
+    assert "bitonic network over" in g2.plan and "radix" not in g2.plan
+    np.testing.assert_array_equal(got2[0], want[0])
+
+
+def test_row_topk_when_one_thread_holds_every_large_value():
+    """Large values 256 columns apart all belong to one thread of the top-k kernel, so the bound taken from the
+    per-thread maxima admits most of the row and the kernel has to fall back to the radix selection."""
+    import torch
+    import oracle
+    import paper_2506_10401_b200 as hct
+    rng = np.random.default_rng(5)
+    x = rng.normal(size=(6, 4096)).astype(np.float32)
+    x[:, ::256] += 100.0
+    x[3, :] = np.sort(x[3, :])[::-1]            # one row already in descending order
+    for k in (8, 16, 64):
+        spec = f"hct 1\ninput x f32 [6,4096]\nnode t = row_topk(x, k={k})\noutput t\n"
+        g = hct.FusedGraph(spec, 0)
+        got = g.run([torch.from_numpy(x).cuda()])[0].cpu().numpy()
+        g.status()
+        want = oracle.run(spec, {"x": x.astype(np.float64)})["t"]
+        np.testing.assert_array_equal(got.astype(np.float64), want)
+
+
 def test_sort_inside_a_chain():
     spec = """hct 1
 input x f32 [50,777]
