@@ -38,6 +38,7 @@ WORKLOADS = {
     "matmul_dropout_mean_softmax": dict(bound="tensor", sample=dict(m=1024)),
     "conv_block": dict(bound="tensor", sample=dict(n=4)),
     "dwconv_bn_relu": dict(bound="hbm", sample=dict(n=8)),
+    "topk_bias_relu": dict(bound="hbm", sample=dict(r=2048)),
     "mbconv_block": dict(bound="hbm", sample=dict(n=4)),
 }
 HEADLINE = "c2_softmax_layernorm_chain"

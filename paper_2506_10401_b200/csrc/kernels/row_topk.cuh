@@ -9,10 +9,10 @@
 // Values are only moved; the elementwise consumers of the result are applied at the store.
 //
 // For k <= 64 a shortcut comes first.  Every thread keeps the largest of its own keys; the k-th
-// largest of these per-thread maxima, found by 32 rounds of bisection with a counting barrier, is a
+// largest of these per-thread maxima, found by the first warp in 32 rounds of bisection over the key bits, is a
 // lower bound of the k-th largest key of the row (k different elements reach it).  The keys that
-// reach the bound, usually little more than k of them, are collected and sorted by a 128-slot bitonic
-// network.  When more than 128 keys reach the bound (many equal values, or a row whose large values
+// reach the bound, usually little more than k of them, are collected and sorted by one warp in a 64- or
+// 128-slot bitonic network (warp barriers only).  When more than 128 keys reach the bound (many equal values, or a row whose large values
 // all sit with one thread) the row takes the radix selection instead.
 // Defined by the generator: HCT_R, HCT_C, HCT_K, HCT_KP (power of two >= HCT_K, <= 2 * HCT_T), HCT_T (threads,
 // 256), HCT_TA, HCT_PA, HctParams, hct_epilogue(), HCT_KERNEL_NAME.
@@ -24,35 +24,68 @@ __device__ __forceinline__ float hct_value_of(unsigned k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
+template <typename T> struct hct_topk_is_f32 { static const bool value = false; };
+template <> struct hct_topk_is_f32<float> { static const bool value = true; };
+
 extern "C" __global__ void __launch_bounds__(HCT_T) HCT_KERNEL_NAME(const HctParams hct_p) {
   hct_pdl_launch_dependents();
   hct_pdl_wait();
-  __shared__ unsigned key[HCT_C];
+  __shared__ __align__(16) unsigned key[HCT_C];
   __shared__ unsigned hist[256];
   __shared__ unsigned sel[HCT_KP];
   __shared__ unsigned pick_bin, pick_need, n_above;
 #if HCT_K <= 64
   __shared__ unsigned few[128];
+  __shared__ unsigned tmax[HCT_T];
+  __shared__ unsigned bound;
 #endif
   const HCT_TA* __restrict__ X = (const HCT_TA*)hct_p.ptr[HCT_PA];
   const int tid = threadIdx.x;
   for (long long row = blockIdx.x; row < HCT_R; row += gridDim.x) {
     unsigned mymax = 0u;
-    for (int i = tid; i < HCT_C; i += HCT_T) {
-      const unsigned u = hct_key_of(hct_ld1(X + row * HCT_C + i));
-      key[i] = u;
-      mymax = u > mymax ? u : mymax;
+    if (hct_topk_is_f32<HCT_TA>::value && HCT_C % 4 == 0) {
+      const float4* __restrict__ x4 = (const float4*)((const float*)X + row * HCT_C);
+      for (int i = tid; i < HCT_C / 4; i += HCT_T) {
+        const float4 v = __ldg(x4 + i);
+        const uint4 u = make_uint4(hct_key_of(v.x), hct_key_of(v.y), hct_key_of(v.z), hct_key_of(v.w));
+        ((uint4*)key)[i] = u;
+        const unsigned a = u.x > u.y ? u.x : u.y, b = u.z > u.w ? u.z : u.w;
+        const unsigned c = a > b ? a : b;
+        mymax = c > mymax ? c : mymax;
+      }
+    } else {
+      for (int i = tid; i < HCT_C; i += HCT_T) {
+        const unsigned u = hct_key_of(hct_ld1(X + row * HCT_C + i));
+        key[i] = u;
+        mymax = u > mymax ? u : mymax;
+      }
     }
 #if HCT_K <= 64
     {
-      unsigned low = 0u;   // becomes the HCT_K-th largest per-thread maximum (at least HCT_K threads hold an element)
-#pragma unroll 1
-      for (int bit = 31; bit >= 0; --bit) {
-        const unsigned cand = low | (1u << bit);
-        if (__syncthreads_count(mymax >= cand) >= HCT_K) low = cand;
-      }
-      if (tid == 0) n_above = 0u;
+      // The first warp finds the HCT_K-th largest per-thread maximum (at least HCT_K threads hold an element)
+      // by bisection over the key bits, eight maxima per lane.
+      tmax[tid] = mymax;
       __syncthreads();
+      if (tid < 32) {
+        unsigned m[HCT_T / 32];
+#pragma unroll
+        for (int q = 0; q < HCT_T / 32; ++q) m[q] = tmax[tid + 32 * q];
+        unsigned low = 0u;
+#pragma unroll 1
+        for (int bit = 31; bit >= 0; --bit) {
+          const unsigned cand = low | (1u << bit);
+          int c = 0;
+#pragma unroll
+          for (int q = 0; q < HCT_T / 32; ++q) c += m[q] >= cand ? 1 : 0;
+          if (__reduce_add_sync(0xffffffffu, c) >= HCT_K) low = cand;
+        }
+        if (tid == 0) {
+          bound = low;
+          n_above = 0u;
+        }
+      }
+      __syncthreads();
+      const unsigned low = bound;
       for (int i = tid; i < HCT_C; i += HCT_T) {
         const unsigned u = key[i];
         if (u >= low) {
@@ -63,22 +96,26 @@ extern "C" __global__ void __launch_bounds__(HCT_T) HCT_KERNEL_NAME(const HctPar
       __syncthreads();
       const unsigned cnt = n_above;     // >= HCT_K; the same for every thread
       if (cnt <= 128u) {
-        for (int i = (int)cnt + tid; i < 128; i += HCT_T) few[i] = 0u;   // 0 sorts last
-        __syncthreads();
-        for (int k = 2; k <= 128; k <<= 1) {
-          for (int j = k >> 1; j > 0; j >>= 1) {
-            if (tid < 64) {
-              const int i = ((tid & ~(j - 1)) << 1) | (tid & (j - 1));
-              const int l = i | j;
-              const unsigned a = few[i], b = few[l];
-              if ((a < b) == ((i & k) == 0)) {
-                few[i] = b;
-                few[l] = a;
+        if (tid < 32) {                 // one warp sorts the collected keys, largest first; 0 sorts last
+          const int np = cnt <= 64u ? 64 : 128;
+          for (int i = (int)cnt + tid; i < np; i += 32) few[i] = 0u;
+          __syncwarp();
+          for (int k = 2; k <= np; k <<= 1) {
+            for (int j = k >> 1; j > 0; j >>= 1) {
+              for (int t = tid; t < np / 2; t += 32) {
+                const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+                const int l = i | j;
+                const unsigned a = few[i], b = few[l];
+                if ((a < b) == ((i & k) == 0)) {
+                  few[i] = b;
+                  few[l] = a;
+                }
               }
+              __syncwarp();
             }
-            __syncthreads();
           }
         }
+        __syncthreads();
         for (int i = tid; i < HCT_K; i += HCT_T) hct_epilogue(hct_p, hct_value_of(few[i]), row * HCT_K + i, row, i);
         __syncthreads();
         continue;

@@ -572,6 +572,12 @@ def test_row_topk_when_one_thread_holds_every_large_value():
         np.testing.assert_array_equal(got.astype(np.float64), want)
 
 
+def test_topk_config_small():
+    spec, laws = configs.get_config("topk_bias_relu", r=96, c=2048, k=32)
+    g = check_f32(spec, laws)
+    assert g.num_kernels == 1
+
+
 def test_sort_inside_a_chain():
     spec = """hct 1
 input x f32 [50,777]

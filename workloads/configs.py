@@ -186,6 +186,20 @@ output y bf16
     return spec, laws
 
 
+def topk_bias_relu(r=8192, c=4096, k=32):
+    """A logic-intensive operator with fused consumers (Table 1): the k largest values of every row, plus a bias, through ReLU."""
+    spec = f"""hct 1
+input x    f32 [{r},{c}]
+input bias f32 [{k}]
+node  t0 = row_topk(x, k={k})
+node  t1 = add(t0, bias)
+node  t2 = relu(t1)
+output t2 f32
+"""
+    laws = {"x": _n(), "bias": _n()}
+    return spec, laws
+
+
 def transpose_bias_relu(r=16384, c=4096):
     """A layout transform with fused consumers (Table 1, "LayoutTransform"): y = relu(x^T + bias)."""
     spec = f"""hct 1
@@ -209,6 +223,7 @@ CONFIGS = {
     "transpose_bias_relu": (transpose_bias_relu, {}),
     "conv_block": (conv_block, {}),
     "dwconv_bn_relu": (dwconv_bn_relu, {}),
+    "topk_bias_relu": (topk_bias_relu, {}),
     "mbconv_block": (mbconv_block, {}),
 }
 
