@@ -36,6 +36,8 @@
  *           (row_softmax also accepts a single column, where it is identically one)
  *           row_layernorm(x, gamma, beta, eps=1e-5)   biased variance, eps inside the root
  *   transpose(x)          y[j,i] = x[i,j] for x[R,C]; elementwise consumers are applied at the store
+ *   reshape(x, rows=R, cols=C)   the elements of x (any rank) in row-major order as [R,C], R*C = numel(x);
+ *                         a bf16 value stays bf16; one copy pass, elementwise consumers applied at the store
  *   row_sort(x, descending=0)   the values of every row of x[R,C] in non-decreasing (descending=1:
  *                         non-increasing) order; row_topk(x, k=K) the K largest values of every row,
  *                         largest first, as [R,K].  C <= 8192.  Values are moved, never changed;

@@ -229,6 +229,21 @@ def _infer(g, name, op, pos, attrs, where):
         if len(s) != 2 or s[1] < (1 if op == "row_softmax" else 2):
             raise SpecError(f"{where}: {op} needs a [R,C] operand with enough columns")
         return Node(name, op, [a], {}, s if op in ROW_TO_ROW else (s[0], 1), "f32")
+    if op == "reshape":
+        only_attrs("rows", "cols")
+        if len(pos) != 1:
+            raise SpecError(f"{where}: reshape takes one operand")
+        a = _operand(g, pos[0], where, False)
+        s = shape_of(a)
+        if "rows" not in attrs or "cols" not in attrs:
+            raise SpecError(f"{where}: reshape needs rows=R, cols=C")
+        rows, cols = _int_attr(attrs, "rows", 0, where), _int_attr(attrs, "cols", 0, where)
+        n = 1
+        for v in s:
+            n *= v
+        if rows < 1 or cols < 1 or rows * cols != n:
+            raise SpecError(f"{where}: reshape of {s} must keep the number of elements")
+        return Node(name, op, [a], {"rows": rows, "cols": cols}, (rows, cols), g.nodes[a].dtype)
     if op in ("row_sort", "row_topk"):
         only_attrs("k") if op == "row_topk" else only_attrs("descending")
         if len(pos) != 1:

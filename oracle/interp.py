@@ -96,6 +96,15 @@ def row_max(x):
     return x.max(axis=1, keepdims=True)
 
 
+def reshape(x, rows, cols):
+    # element number t of x in row-major order becomes y[t // cols, t % cols]
+    flat = np.ascontiguousarray(x).ravel(order="C")
+    y = np.empty((rows, cols), dtype=x.dtype)
+    for i in range(rows):
+        y[i, :] = flat[i * cols:(i + 1) * cols]
+    return y
+
+
 # ---- logic-intensive operators (Table 1): ordering the values of a row ------------------------
 
 def row_sort(x, descending=False):
@@ -220,6 +229,8 @@ def run_nodes(spec, inputs: dict, dtype=np.float64, gemm_fn=None) -> dict:
         elif op in BINARY:
             out = _BINARY_FN[op](args[0], args[1])
             out = np.broadcast_to(out, node.shape)
+        elif op == "reshape":
+            out = reshape(args[0], node.attrs["rows"], node.attrs["cols"])
         elif op == "row_sort":
             out = row_sort(args[0], bool(node.attrs["descending"]))
         elif op == "row_topk":

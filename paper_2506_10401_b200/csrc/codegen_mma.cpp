@@ -216,6 +216,27 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
   const Node& b = g.nodes[anchor.args[anchor.args.size() > 1 ? 1 : 0].node];   // transpose and sort have one operand
   EpiGen eg{g, p, grp, gi, {}};
 
+  // ---- reshape: flat copy through the generated epilogue
+  if (grp.kind == GroupKind::Reshape) {
+    const int src = anchor.args[0].node;
+    const int pa = eg.ptr_index(src, g.nodes[src].cls != OpClass::Input && p.ws_offset[src] >= 0);
+    const DType ta = eg.buf_dtype(src);
+    std::string epi = eg.scalar_fn();
+    KernelSpec k;
+    k.name = "hct_reshape_g" + std::to_string(gi);
+    std::ostringstream st;
+    st << "#define HCT_ROWS " << anchor.shape[0] << "LL\n#define HCT_COLS " << anchor.shape[1] << "LL\n#define HCT_TA " << ctype(ta)
+       << "\n#define HCT_PA " << pa << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+       << skeleton_source("common") << "\nstruct HctParams { void* ptr[" << eg.ptrs.size() << "]; };\n" << epi << skeleton_source("reshape");
+    k.source = st.str();
+    k.ptrs = eg.ptrs;
+    k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>((anchor.numel() + 255) / 256, 148 * 64));
+    k.block[0] = 256;
+    k.desc = "reshape: flat copy, consumers fused at the store";
+    out->push_back(k);
+    return;
+  }
+
   // ---- row sort / top-k: bitonic network in shared memory, one CTA per row, consumers applied at the store
   if (grp.kind == GroupKind::Sort) {
     const int src = anchor.args[0].node;

@@ -308,6 +308,20 @@ Graph parse_spec(const std::string& text) {
         auto& s = g.nodes[n.args[0].node].shape;
         if (s.size() != 2) fail(HCT_ERR_GRAPH, line, "transpose needs a [R,C] operand, got " + shape_str(s));
         n.shape = {s[1], s[0]};
+      } else if (op == "reshape") {
+        // layout transform (Table 1): the same elements in row-major order under a new 2-D shape, e.g. flattening
+        // [N,C,H,W] into [N, C*H*W] in front of a gemm
+        only_attrs({"rows", "cols"});
+        if (pos.size() != 1) fail(HCT_ERR_GRAPH, line, "reshape takes one operand");
+        n.cls = OpClass::Reshape;
+        n.args = {lookup(pos[0], line, false)};
+        const Node& src = g.nodes[n.args[0].node];
+        int64_t rows, cols;
+        if (!attrs.count("rows") || !attrs.count("cols") || !parse_int(attrs["rows"], &rows) || !parse_int(attrs["cols"], &cols) || rows < 1 || cols < 1)
+          fail(HCT_ERR_PARSE, line, "reshape needs rows=R, cols=C (positive integers)");
+        if (rows * cols != src.numel()) fail(HCT_ERR_GRAPH, line, "reshape of " + shape_str(src.shape) + " must keep the number of elements");
+        n.shape = {rows, cols};
+        n.dtype = src.dtype;   // values are moved unchanged, so a bf16 value stays bf16
       } else if (op == "row_sort" || op == "row_topk") {
         // logic-intensive operators (Table 1): the values of every row in order; row_topk keeps the k largest, largest first
         const bool topk = op == "row_topk";

@@ -9,7 +9,7 @@ namespace hct {
 
 enum DType { F32 = 0, BF16 = 1 };
 
-enum class OpClass { Input, Unary, Binary, RowSoftmax, RowLayernorm, RowReduce, Gemm, Conv, Transpose, Sort };
+enum class OpClass { Input, Unary, Binary, RowSoftmax, RowLayernorm, RowReduce, Gemm, Conv, Transpose, Sort, Reshape };
 
 struct Error : std::runtime_error {
   int code;

@@ -128,10 +128,11 @@ Plan make_plan(const Graph& g) {
     const Node& nd = g.nodes[i];
     if (nd.cls == OpClass::Input) continue;
     int gi = -1;
-    if (nd.cls == OpClass::Gemm || nd.cls == OpClass::Conv || nd.cls == OpClass::Transpose || nd.cls == OpClass::Sort) {
+    if (nd.cls == OpClass::Gemm || nd.cls == OpClass::Conv || nd.cls == OpClass::Transpose || nd.cls == OpClass::Sort ||
+        nd.cls == OpClass::Reshape) {
       Group grp;
       grp.kind = nd.cls == OpClass::Gemm ? GroupKind::Gemm : nd.cls == OpClass::Conv ? GroupKind::Conv
-                 : nd.cls == OpClass::Transpose ? GroupKind::Transpose : GroupKind::Sort;
+                 : nd.cls == OpClass::Transpose ? GroupKind::Transpose : nd.cls == OpClass::Sort ? GroupKind::Sort : GroupKind::Reshape;
       grp.full_shape = nd.shape;
       p.groups.push_back(grp);
       gi = (int)p.groups.size() - 1;
@@ -170,7 +171,8 @@ Plan make_plan(const Graph& g) {
     const Node& nd = g.nodes[i];
     if (nd.cls == OpClass::Input) continue;
     Group& grp = p.groups[p.group_of[i]];
-    bool anchor = nd.cls == OpClass::Gemm || nd.cls == OpClass::Conv || nd.cls == OpClass::Transpose || nd.cls == OpClass::Sort;
+    bool anchor = nd.cls == OpClass::Gemm || nd.cls == OpClass::Conv || nd.cls == OpClass::Transpose || nd.cls == OpClass::Sort ||
+                  nd.cls == OpClass::Reshape;
     for (auto& a : nd.args) {
       if (a.is_literal() || p.group_of[a.node] == p.group_of[i]) continue;
       if (anchor) continue;  // contraction operands are bound separately
@@ -222,7 +224,7 @@ Plan make_plan(const Graph& g) {
       for (auto& a : g.nodes[j].args) {
         if (a.is_literal() || a.node != i || p.group_of[j] == p.group_of[i]) continue;
         bool into_contraction = g.nodes[j].cls == OpClass::Gemm || g.nodes[j].cls == OpClass::Conv || g.nodes[j].cls == OpClass::Transpose ||
-                                g.nodes[j].cls == OpClass::Sort;
+                                g.nodes[j].cls == OpClass::Sort || g.nodes[j].cls == OpClass::Reshape;
         bool from_contraction = p.groups[p.group_of[i]].kind != GroupKind::Row && p.groups[p.group_of[j]].has_reduction &&
                                 nd.shape.back() > 512;
         unavoidable = unavoidable || into_contraction || from_contraction;
@@ -233,7 +235,7 @@ Plan make_plan(const Graph& g) {
   std::ostringstream os;
   for (size_t gi = 0; gi < p.groups.size(); ++gi) {
     const Group& grp = p.groups[gi];
-    os << "kernel " << gi << " " << (grp.kind == GroupKind::Row ? "row" : grp.kind == GroupKind::Gemm ? "gemm" : grp.kind == GroupKind::Conv ? "conv" : grp.kind == GroupKind::Transpose ? "transpose" : "sort") << " [";
+    os << "kernel " << gi << " " << (grp.kind == GroupKind::Row ? "row" : grp.kind == GroupKind::Gemm ? "gemm" : grp.kind == GroupKind::Conv ? "conv" : grp.kind == GroupKind::Transpose ? "transpose" : grp.kind == GroupKind::Sort ? "sort" : "reshape") << " [";
     for (size_t d = 0; d < grp.full_shape.size(); ++d) os << (d ? "," : "") << grp.full_shape[d];
     os << "]:";
     for (int i : grp.nodes) os << " " << g.nodes[i].name << "=" << g.nodes[i].op;

@@ -13,7 +13,7 @@
 
 namespace hct {
 
-enum class GroupKind { Row, Gemm, Conv, Transpose, Sort };
+enum class GroupKind { Row, Gemm, Conv, Transpose, Sort, Reshape };
 
 // How an operand indexes relative to the group's full shape [.., C].
 enum class Bcast {

@@ -519,6 +519,43 @@ def test_sweep_graphs_reduced_rows(seed):
     check_f32(spec, laws, seed)
 
 
+# ------------------------------------------------------------------ reshape
+
+@pytest.mark.parametrize("dtype,shape,rows,cols", [("f32", (6, 20), 8, 15), ("bf16", (2, 3, 4, 5), 2, 60), ("f32", (1000,), 8, 125),
+                                                    ("bf16", (37, 129), 129, 37), ("f32", (4, 8, 16, 16), 32, 256)])
+def test_reshape_moves_values_exactly_and_fuses_consumers(dtype, shape, rows, cols):
+    dims = "[" + ",".join(str(v) for v in shape) + "]"
+    spec = (f"hct 1\ninput x {dtype} {dims}\ninput b f32 [{cols}]\ninput s f32 [{rows},1]\nnode f = reshape(x, rows={rows}, cols={cols})\n"
+            "node u = add(f, b)\nnode v = mul(u, s)\noutput f\noutput v\n")
+    got, want, g = parity.run_both(spec, {"x": N_, "b": N_, "s": N_})
+    assert g.num_kernels == 1
+    np.testing.assert_array_equal(got[0], want[0])
+    assert parity.f32_violation(got[1], want[1]) <= 1.0
+
+
+def test_conv_flatten_gemm_head():
+    """conv -> bias -> ReLU -> bf16 -> flatten -> fully connected layer: the flattened activations stay bf16 and feed the tensor-core GEMM."""
+    spec = """hct 1
+input x  bf16 [64,32,8,8]
+input w  bf16 [32,32,3,3]
+input b  f32 [32,1,1]
+input fc bf16 [2048,256]
+input fb f32 [256]
+node c0 = conv2d(x, w, pad=1)
+node c1 = add(c0, b)
+node c2 = relu(c1)
+node c3 = cast_bf16(c2)
+node f  = reshape(c3, rows=64, cols=2048)
+node y0 = gemm(f, fc)
+node y  = add(y0, fb)
+output y
+"""
+    wl = {"kind": "normal", "mean": 0.0, "std": 0.06}
+    got, want, g = parity.run_both(spec, {"x": N_, "w": wl, "b": N_, "fc": {"kind": "normal", "mean": 0.0, "std": 0.02}, "fb": N_})
+    assert "hct_reshape" in g.plan and g.plan.count("tcgen05") == 2
+    assert parity.bf16_violation(got[0], want[0]) <= 1.0
+
+
 # ------------------------------------------------------------------ logic-intensive operators: row sort and top-k
 
 @pytest.mark.parametrize("rows,cols", [(5, 1), (7, 2), (33, 5), (64, 100), (40, 1024), (9, 3000), (6, 4096), (3, 8192)])

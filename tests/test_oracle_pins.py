@@ -342,6 +342,29 @@ def test_conv_structure_pins():
     np.testing.assert_array_equal(interp.conv2d(xi, wi, 1, 1), _conv_loops(xi, wi, 1, 1))
 
 
+# ---------------------------------------------------------------- reshape
+
+def test_reshape_keeps_row_major_order():
+    x = np.arange(2 * 3 * 4 * 5, dtype=np.float64).reshape(2, 3, 4, 5)
+    y = interp.reshape(x, 6, 20)
+    np.testing.assert_array_equal(y.ravel(), np.arange(120))            # element t stays element t
+    assert y[4, 7] == x[1, 1, 1, 2]                                     # 4*20+7 = 87 = ((1*3+1)*4+1)*5+2
+    for (n, c, h, w) in [(2, 3, 4, 5), (1, 7, 2, 2)]:
+        a = RNG.normal(size=(n, c, h, w))
+        f = interp.reshape(a, n, c * h * w)
+        for i in range(n):
+            for j in range(c):
+                for k in range(h):
+                    for m in range(w):
+                        assert f[i, (j * h + k) * w + m] == a[i, j, k, m]
+    a = RNG.normal(size=(6, 8))
+    np.testing.assert_array_equal(interp.reshape(interp.reshape(a, 12, 4), 6, 8), a)
+    g = oracle.parse("hct 1\ninput x bf16 [2,3,4,5]\nnode f = reshape(x, rows=6, cols=20)\noutput f bf16\n")
+    assert g.nodes["f"].shape == (6, 20) and g.nodes["f"].dtype == "bf16"
+    with pytest.raises(oracle.SpecError):
+        oracle.parse("hct 1\ninput x f32 [2,3]\nnode f = reshape(x, rows=4, cols=2)\noutput f\n")
+
+
 # ---------------------------------------------------------------- row_sort / row_topk
 
 def _insertion_sorted(row):
@@ -582,6 +605,7 @@ def test_planted_mistakes_are_detected(monkeypatch):
         return orig["gelu_erf"](x)
 
     plants = [
+        ("reshape", lambda x, rows, cols: np.ascontiguousarray(x).ravel(order="F").reshape(rows, cols), test_reshape_keeps_row_major_order),
         ("row_sort", lambda x, descending=False: orig["row_sort"](x, not descending), test_sort_hand_values_bruteforce_and_invariants),
         ("row_topk", lambda x, k: orig["row_sort"](x)[:, :k], test_sort_hand_values_bruteforce_and_invariants),
         ("row_layernorm", unbiased_ln, test_layernorm_closed_forms),
