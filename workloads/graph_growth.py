@@ -30,7 +30,8 @@ from . import tensors
 UNARY = ("relu", "gelu_tanh", "sigmoid", "tanh", "exp", "abs")
 BINARY = ("add", "sub", "mul", "max")
 ROW = ("row_softmax", "row_layernorm", "row_sum", "row_max")
-POOL = UNARY + BINARY + ("broadcast_bias",) + ROW + ("gemm",)
+ORDER = ("row_sort", "row_topk")          # logic-intensive operators
+POOL = UNARY + BINARY + ("broadcast_bias",) + ROW + ORDER + ("gemm",)
 COLS = (128, 512, 2048)
 GEMM_N = (256, 1024)
 ROWS = (1024, 4096)
@@ -117,7 +118,7 @@ def grow_graph(seed: int, attempt: int = 0, rows: int | None = None, p_op: float
             if not allowed:
                 allowed = list(UNARY)
             op = d.choice(allowed)
-            if op in ROW + ("gemm", "broadcast_bias") and not full:
+            if op in ROW + ORDER + ("gemm", "broadcast_bias") and not full:
                 counters["rollbacks"] += 1      # operator does not fit the operand's shape
                 continue
             usage[op] += 1
@@ -141,6 +142,11 @@ def grow_graph(seed: int, attempt: int = 0, rows: int | None = None, p_op: float
                 return emit(op, [src], shape)
             if op in ("row_sum", "row_max"):
                 return emit(op, [src], (shape[0], 1))
+            if op == "row_sort":
+                return emit(op, [src], shape, ", descending=1" if d.next() < 0.5 else "")
+            if op == "row_topk":
+                k = d.choice([kk for kk in (8, 32, 128) if kk < shape[1]] or [shape[1]])
+                return emit(op, [src], (shape[0], k), f", k={k}")
             n_out = d.choice(GEMM_N)
             w = fresh((shape[1], n_out), {"kind": "normal", "mean": 0.0, "std": 1.0 / math.sqrt(shape[1])})
             return emit("gemm", [src, w], (shape[0], n_out))
