@@ -24,6 +24,8 @@ __device__ __forceinline__ float hct_value_of(unsigned k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
+static_assert(HCT_T == 256, "one thread per histogram bin");
+static_assert(HCT_KP <= 2 * HCT_T && HCT_K <= HCT_KP, "the selected keys are sorted by one pass of the block");
 template <typename T> struct hct_topk_is_f32 { static const bool value = false; };
 template <> struct hct_topk_is_f32<float> { static const bool value = true; };
 
