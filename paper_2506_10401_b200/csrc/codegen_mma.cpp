@@ -241,9 +241,9 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
   if (grp.kind == GroupKind::Sort) {
     const int src = anchor.args[0].node;
     const int64_t R = a.shape[0], C = a.shape[1], KOUT = anchor.shape[1];
-    int64_t NP = 2;
+    int64_t NP = 8;
     while (NP < C) NP *= 2;
-    const int64_t T = std::max<int64_t>(32, std::min<int64_t>(512, NP / 2));
+    const int64_t T = std::max<int64_t>(32, std::min<int64_t>(512, NP / 8));   // a thread owns blocks of 8 slots
     const int pa = eg.ptr_index(src, g.nodes[src].cls != OpClass::Input && p.ws_offset[src] >= 0);
     const DType ta = eg.buf_dtype(src);
     std::string epi = eg.scalar_fn();
