@@ -604,7 +604,11 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       const int64_t pitch = (WO + FS - 1 + 31) / 32 * 32;
       const bool dense_pitch = pitch <= 256 && WO * 10 >= pitch * 7;
       const int th_pitch = (int)std::max<int64_t>(1, std::min<int64_t>(256 / std::max<int64_t>(pitch, 1), HO));
-      const int n_stg = 3, n_buf = 2;
+      // Slots of the pixel staging ring and operand buffers (a deeper ring was measured on 1x1 convolutions,
+      // whose tiles have a single weight stage, and changed nothing: their limit is the epilogue's store rate).
+      int n_stg = 3, n_buf = 2;
+      if (tun.conv_nstg >= 2 && tun.conv_nstg <= 12) n_stg = tun.conv_nstg;
+      if (tun.conv_nbuf >= 2 && tun.conv_nbuf <= 3) n_buf = tun.conv_nbuf;
       int n_a = 0;
       bool direct = false;
       // The epilogue of the NCHW-reading kernel hands its bf16 output to TMA stores (through 16 KB of
