@@ -206,6 +206,9 @@ HCT_API const char* hct_graph_kernel_name(const hct_graph_t* g, int idx);
  * allocating routine.  All calls share the one array: nothing in it needs to start at zero (each
  * call overwrites the part it reads), but two calls whose kernels overlap on the GPU (different
  * streams, or several host threads) race on it; keep them on one stream or order them yourself.
+ * A CUDA error already pending on the calling thread is reported by this call (HCT_ERR_CUDA) and
+ * left pending.  The looked-up address is cached per device for the life of the process: after
+ * cudaDeviceReset on that device it is stale and this entry point must not be used again.
  */
 #define HCT_STATIC_SCRATCH_BYTES (8u << 20)
 HCT_API hct_status_t hct_gemm_bias_relu_f32_static(const float* a, const float* b, const float* bias, float* out, int64_t m,

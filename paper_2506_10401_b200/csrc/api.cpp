@@ -154,11 +154,18 @@ hct_status_t hct_graph_create_scheduled(const char* spec, size_t spec_len, int d
         CtxGuard guard(*d, h->ctx);
         CUresult_t rc = d->ModuleLoadData(&lk.module, cubin.data());
         if (rc != 0) throw Error(HCT_ERR_COMPILE, cu_error(*d, rc, "cuModuleLoadData"));
+        // until the kernel is in h->kernels nothing else owns the module: unload it on the way out of a failure
+        auto fail = [&](hct_status_t code, const char* what) {
+          std::string msg = cu_error(*d, rc, what);
+          d->ModuleUnload(lk.module);
+          lk.module = nullptr;
+          throw Error(code, msg);
+        };
         rc = d->ModuleGetFunction(&lk.func, lk.module, ks.name.c_str());
-        if (rc != 0) throw Error(HCT_ERR_COMPILE, cu_error(*d, rc, "cuModuleGetFunction"));
+        if (rc != 0) fail(HCT_ERR_COMPILE, "cuModuleGetFunction");
         if (ks.smem_bytes > 0) {
           rc = d->FuncSetAttribute(lk.func, kFuncAttrMaxDynamicSharedSizeBytes, (int)ks.smem_bytes);
-          if (rc != 0) throw Error(HCT_ERR_CUDA, cu_error(*d, rc, "cuFuncSetAttribute(max dynamic shared memory)"));
+          if (rc != 0) fail(HCT_ERR_CUDA, "cuFuncSetAttribute(max dynamic shared memory)");
         }
         if (ks.persistent) {
           int per_sm = 1;

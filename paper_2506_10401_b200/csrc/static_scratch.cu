@@ -158,8 +158,9 @@ extern "C" HCT_API hct_status_t hct_gemm_bias_relu_f32_static(const float* a, co
     split_static<<<(unsigned)(blocks < 148 * 16 ? blocks : 148 * 16), 256, 0, stream>>>(a, b, n_a, n_b, hi, lo);
     dim3 grid((unsigned)((n + 63) / 64), (unsigned)((m + 63) / 64));
     gemm_split_static<<<grid, 256, 0, stream>>>(hi, lo, n_a, bias, out, m, k, n, apply_relu);
-    rc = cudaGetLastError();
-    if (rc != cudaSuccess) status = fail(HCT_ERR_CUDA, std::string("kernel launch: ") + cudaGetErrorString(rc));
+    // peek, not get: an error that was already pending on this thread is reported here but left for its owner to clear
+    rc = cudaPeekAtLastError();
+    if (rc != cudaSuccess) status = fail(HCT_ERR_CUDA, std::string("kernel launch (or an earlier pending error): ") + cudaGetErrorString(rc));
   }
   cudaSetDevice(prev);
   return status;

@@ -27,3 +27,20 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _label_parity_records(request):
+    from tests import parity
+    parity.set_label(request.node.name)
+    yield
+
+
+def pytest_terminal_summary(terminalreporter):
+    """Ungraded strict figures of the fp32 comparisons (largest relative error with no allowance for cancellation)."""
+    from tests import parity
+    lines = parity.report_lines()
+    if lines:
+        terminalreporter.write_sep("-", "fp32 parity: strict figures")
+        for line in lines:
+            terminalreporter.write_line(line)

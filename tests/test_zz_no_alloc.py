@@ -1,10 +1,12 @@
-"""The allocation-free GEMM entry point against the regular graph path.  Collected last on purpose:
-a run that stops at the first failure has then already exercised everything else.
+"""The allocation-free GEMM entry point against the CPU oracle and the regular graph path.  Collected
+last on purpose: a run that stops at the first failure has then already exercised everything else.
 
 hct_gemm_bias_relu_f32_static keeps the split operands of an fp32 GEMM in a fixed array inside the
 library instead of caller workspace, for callers that cannot allocate device memory.  Two calls in
 a row (different shapes, so the second overwrites only part of what the first left in the array)
-must each agree with hct_graph_run on the same inputs within the library's fp32 tolerance.
+must each agree with the oracle on the same inputs within the library's fp32 tolerance, and so
+must hct_graph_run; the two device results are two roundings of the same product, so they are
+also compared with each other at twice that tolerance.
 """
 import ctypes
 
@@ -30,14 +32,18 @@ def _both(m, k, n, seed):
                                       torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
     g.status()
-    return parity.to_numpy64(out), parity.to_numpy64(ref)
+    want = parity.oracle_reference(spec, parity.oracle_inputs(spec, t))["t2"]
+    return parity.to_numpy64(out), parity.to_numpy64(ref), want
 
 
-def test_static_scratch_gemm_matches_graph_path_twice():
+def test_static_scratch_gemm_matches_oracle_and_graph_path_twice():
     for (m, k, n, seed) in [(256, 256, 256, 0), (70, 132, 200, 1), (256, 256, 256, 2)]:
-        got, ref = _both(m, k, n, seed)
-        worst = parity.f32_violation(got, ref)
-        assert worst <= 1.0, f"({m},{k},{n}): static-scratch result differs from the graph path by factor {worst:.3g} of tolerance"
+        got, graph, want = _both(m, k, n, seed)
+        worst = parity.f32_violation(got, want)
+        assert worst <= 1.0, f"({m},{k},{n}): static-scratch result differs from the oracle by factor {worst:.3g} of tolerance"
+        assert parity.f32_violation(graph, want) <= 1.0
+        bound, _ = parity.f32_bound(want)
+        assert np.all(np.abs(got - graph) <= 2 * bound)
 
 
 def test_static_scratch_rejects_oversized_and_bad_arguments():
