@@ -25,7 +25,7 @@ import oracle
 from oracle import interp
 
 U = 2.0 ** -24          # unit round-off of float32
-SAFETY = 4.0            # first-order bounds ignore second-order terms and differences in evaluation order
+SAFETY = 2.0            # first-order bounds ignore second-order terms and differences in evaluation order
 
 # own rounding of one operator, in units of u relative to |result|
 C_EXACT = 0.0           # selections and sign changes: relu, neg, abs, max, min, data movement
