@@ -7,6 +7,9 @@ One step = one run of a whole fused chain (every kernel of its plan) on one batc
 synthetic input.  The headline workload is the memory-bound chain (affine, GELU, row softmax,
 row layer normalisation on an fp32 [8192,4096] tensor); throughput is algorithmic bytes per
 second (inputs read once, outputs written once).  Contraction chains report TFLOP/s.
+Without --workload the line also carries, under "configs", the other four benchmark
+configurations (fp32 GEMM chain, bf16 GEMM chain, bf16 convolution chain, the 200-graph sweep),
+each timed the same way in the same process.
 With N > 1 every rank runs an independent replica on its own GPU (the chains do not shard
 across devices); the value is the sum over ranks divided by the slowest rank's time.
 Prints one JSON line.
@@ -29,9 +32,11 @@ import numpy as np  # noqa: E402
 from workloads import configs  # noqa: E402
 
 WORKLOADS = {
-    "c2_softmax_layernorm_chain": dict(bound="hbm", sample=dict(r=8192)),
-    "c3_gemm_bf16_gelu_residual": dict(bound="tensor", sample=dict(m=2048)),
-    "c4_conv_bn_relu_bf16": dict(bound="tensor", sample=dict(n=8)),
+    # sample: what the CPU-baseline leg times (a few steps); ref_sample: one step of the reference arm, which
+    # runs every requested step and warm-up, so its sample is smaller
+    "c2_softmax_layernorm_chain": dict(bound="hbm", sample=dict(r=8192), ref_sample=dict(r=1024)),
+    "c3_gemm_bf16_gelu_residual": dict(bound="tensor", sample=dict(m=2048), ref_sample=dict(m=256)),
+    "c4_conv_bn_relu_bf16": dict(bound="tensor", sample=dict(n=8), ref_sample=dict(n=2)),
     "c1_gemm_bias_relu_f32": dict(bound="tensor", sample=dict()),
     # operator classes beyond the five configurations: a layout transform and the case-study chain with dropout
     "transpose_bias_relu": dict(bound="hbm", sample=dict(r=4096)),
@@ -42,6 +47,15 @@ WORKLOADS = {
     "mbconv_block": dict(bound="hbm", sample=dict(n=4)),
 }
 HEADLINE = "c2_softmax_layernorm_chain"
+SMALL_BYTES = 24 * 1024 * 1024
+# the other configurations reported beside the headline, with the steps they are timed over
+# (at most; --steps caps them) and the GPU test that checks the same launch configuration against the oracle
+ALSO = [("c1_gemm_bias_relu_f32", 200, "tests/test_gpu_parity.py::test_config1_gemm_bias_relu_full_size"),
+        ("c3_gemm_bf16_gelu_residual", 100, "tests/test_gpu_fullsize.py::test_config3_full_size_sampled_rows"),
+        ("c4_conv_bn_relu_bf16", 200, "tests/test_gpu_fullsize.py::test_config4_full_size_all_images")]
+PARITY_TEST = {HEADLINE: "tests/test_gpu_fullsize.py::test_config2_full_size_all_rows",
+               "c5_sweep": "tests/test_gpu_fullsize.py::test_sweep_graph_full_size_sampled_rows (all 200 seeds)"}
+PARITY_TEST.update({n: t for n, _, t in ALSO})
 
 
 def kernel_fingerprint(g):
@@ -139,12 +153,13 @@ def metric_of(bound, bytes_, flops, seconds):
     return flops / seconds / 1e12, "TFLOP/s"
 
 
-def oracle_arm(name, steps, warmup):
+def oracle_arm(name, steps, warmup, sample_key="sample"):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload."""
     import oracle
     from workloads import tensors
     info = WORKLOADS[name]
-    spec, laws = configs.get_config(name, **info["sample"])
+    sample_kw = info.get(sample_key, info["sample"])
+    spec, laws = configs.get_config(name, **sample_kw)
     t = configs.draw_inputs(spec, laws, 0)
     ins = {n: tensors.as_float64(t[n], d) for n, d, _ in configs.parse_inputs(spec)}
     g = oracle.parse(spec)
@@ -165,17 +180,21 @@ def oracle_arm(name, steps, warmup):
         oracle.run(g, ins)
     dt = (time.perf_counter() - t0) / steps
     value, unit = metric_of(info["bound"], in_bytes + out_bytes, flops, dt)
-    try:
-        from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
-    except Exception:
-        cores = os.cpu_count() or 1
-    sample = ", ".join(f"{k}={v}" for k, v in info["sample"].items()) or "full size"
+    # numpy evaluates elementwise operators and reductions on one thread; only the matrix products
+    # of a contraction (matmul, einsum) run on the BLAS pool
+    cores = 1
+    if flops > 0:
+        try:
+            from threadpoolctl import threadpool_info
+            cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        except Exception:
+            cores = os.cpu_count() or 1
+    sample = ", ".join(f"{k}={v}" for k, v in sample_kw.items()) or "full size"
     return dict(value=value, unit=unit, cores=cores, kind="oracle", sample=f"{name} at {sample} ({out_elems} output elements per step)",
                 ms_per_step=dt * 1e3)
 
 
-def run_gpu(name, steps, warmup, rank, world, device, tune=0):
+def run_gpu(name, steps, warmup, rank, world, device, tune=0, with_e2e=True):
     import torch
     import paper_2506_10401_b200 as hct
     from tests import parity
@@ -207,10 +226,23 @@ def run_gpu(name, steps, warmup, rank, world, device, tune=0):
             a.record(stream)
             g.run(ins, outs, stream)
             b.record(stream)
+        # nvidia-smi samples every 50 ms and a short timed region may end before its first sample: the same
+        # steps keep running, untimed, until the sampler has seen about 0.3 s of this load
+        t_end = time.perf_counter() + max(0.0, 0.3 - 1e-3 * steps)
+        while time.perf_counter() < t_end:
+            flush.zero_()
+            g.run(ins, outs, stream)
+            torch.cuda.synchronize(device)
         barrier()
     g.status()
     per_step = [a.elapsed_time(b) * 1e-3 for a, b in ev]
     dev_s = float(np.sum(per_step))
+    if not with_e2e:
+        dev_s = max_over_ranks([dev_s], f"cuda:{device}")[0]
+        value, unit = whole_job_value(info["bound"], bytes_, flops, world, dev_s / steps)
+        return dict(value=value, unit=unit, ms_per_step=dev_s / steps * 1e3, bytes=bytes_, flops=flops, kernel_s=float(np.mean(per_step)),
+                    fingerprint=kernel_fingerprint(g), kernels=g.num_kernels, clocks=clocks.summary(), e2e=None, plan=g.plan,
+                    schedule=g.schedule)
 
     # end to end: pinned host inputs -> device, run, result back to the host, every step.  The three
     # phases of consecutive steps overlap (copy-in, compute and copy-out streams, two sets of device
@@ -223,7 +255,7 @@ def run_gpu(name, steps, warmup, rank, world, device, tune=0):
     host_out = [[torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in outs] for _ in range(2)]
     h2d = sum(t.numel() * t.element_size() for t in pinned)
     d2h = sum(t.numel() * t.element_size() for t in host_out[0])
-    e2e_steps = max(4, min(steps, 8))
+    e2e_steps = max(4, min(steps, 50))
     s_in, s_run, s_out = (torch.cuda.Stream(device) for _ in range(3))
     ev_in = [torch.cuda.Event() for _ in range(2)]
     ev_run = [torch.cuda.Event() for _ in range(2)]
@@ -287,8 +319,22 @@ def run_sweep(steps, warmup, device, out_path=None, tune=0):
     stream = torch.cuda.current_stream(device)
     records = []
     launches = 0
-    for e in sweep.entries():
+    # Graph creation (planning + NVRTC) is untimed set-up and dominates the wall clock of the sweep:
+    # graphs are created a few ahead of use on a thread pool (the compiler runs outside the interpreter lock).
+    from concurrent.futures import ThreadPoolExecutor
+    todo = sweep.entries()
+
+    def make(e):
         spec, laws, meta = sweep.get(e["seed"])
+        return spec, laws, (None if tune > 0 else hct.FusedGraph(spec, device))
+
+    pool = ThreadPoolExecutor(max_workers=6)
+    ahead = [pool.submit(make, e) for e in todo[:12]]
+    for i, e in enumerate(todo):
+        if i + 12 < len(todo):
+            ahead.append(pool.submit(make, todo[i + 12]))
+        spec, laws, made = ahead[i].result()
+        ahead[i] = None
         gen = torch.Generator(device=dev)
         gen.manual_seed(1000 + e["seed"])
         ins = []
@@ -299,7 +345,7 @@ def run_sweep(steps, warmup, device, out_path=None, tune=0):
             else:
                 t = torch.rand(shape, device=dev, generator=gen) * (law["hi"] - law["lo"]) + law["lo"]
             ins.append(t.to(torch.bfloat16) if dtype == "bf16" else t)
-        g = hct.FusedGraph.autotuned(spec, ins, device, max_trials=tune) if tune > 0 else hct.FusedGraph(spec, device)
+        g = hct.FusedGraph.autotuned(spec, ins, device, max_trials=tune) if tune > 0 else made
         outs = g.alloc_outputs()
         for _ in range(max(1, warmup)):
             g.run(ins, outs, stream)
@@ -322,38 +368,86 @@ def run_sweep(steps, warmup, device, out_path=None, tune=0):
         launches += g.num_kernels * (steps + max(1, warmup))
         g.close()
         del ins, outs
+    pool.shutdown()
     if out_path:
         with open(out_path, "w") as f:
             for r in records:
                 f.write(json.dumps(r) + "\n")
-    mem = [r for r in records if r["cls"] == "memory"]
+    # Graphs that move less than SMALL_BYTES are latency-bound (a few microseconds for a tensor that
+    # sits in L2): they are reported as a latency class of their own, not against the HBM roofline.
+    small = [r for r in records if r["cls"] == "memory" and r["bytes"] < SMALL_BYTES]
+    mem = [r for r in records if r["cls"] == "memory" and r["bytes"] >= SMALL_BYTES]
     mma = [r for r in records if r["cls"] == "gemm"]
     geo = lambda rs: float(np.exp(np.mean(np.log([r["frac"] for r in rs])))) if rs else None
-    agg = dict(graphs=len(records), memory_graphs=len(mem), gemm_graphs=len(mma),
+    agg = dict(graphs=len(records), memory_graphs=len(mem), gemm_graphs=len(mma), small_graphs=len(small),
                memory_GBps=sum(r["bytes"] for r in mem) / sum(r["us"] for r in mem) / 1e3 if mem else None,
                gemm_TFLOPps_fp32=sum(r["flops"] for r in mma) / sum(r["us"] for r in mma) / 1e6 if mma else None,
                memory_frac_geomean=geo(mem), gemm_frac_geomean=geo(mma),
                memory_share_ge_0p7=float(np.mean([r["frac"] >= 0.7 for r in mem])) if mem else None,
                gemm_share_ge_0p6=float(np.mean([r["frac"] >= 0.6 for r in mma])) if mma else None,
+               small_us_median=float(np.median([r["us"] for r in small])) if small else None,
+               small_us_max=float(np.max([r["us"] for r in small])) if small else None,
+               small_launches_mean=float(np.mean([r["kernels"] for r in small])) if small else None,
+               small_bytes_below=SMALL_BYTES,
+               all_memory_GBps=sum(r["bytes"] for r in mem + small) / sum(r["us"] for r in mem + small) / 1e3 if mem or small else None,
                total_ms=sum(r["us"] for r in records) / 1e3)
     return agg, launches
+
+
+def roofline_of(name, r, pk):
+    """Roofline record of one timed workload: algorithmic bytes or flops of a step over the mean step time on the device."""
+    info = WORKLOADS[name]
+    achieved, unit = metric_of(info["bound"], r["bytes"], r["flops"], r["kernel_s"])
+    # a contraction timed over a long run sits under the power cap: compare with the sustained GEMM
+    # figure then, with the burst figure when the clocks stayed at their maximum
+    clk = r["clocks"]
+    capped = "sw_power_cap" in clk["reasons"] and clk["sm_mhz"] and clk["sm_max_mhz"] and clk["sm_mhz"] < 0.9 * clk["sm_max_mhz"]
+    peak_kind = "copy" if info["bound"] == "hbm" else ("gemm sustained" if capped else "gemm burst")
+    peak = pk["hbm"] if info["bound"] == "hbm" else (pk["tensor_sustained"] if capped else pk["tensor"])
+    return dict(bound=info["bound"], achieved=achieved, peak=peak, unit=unit, frac=achieved / peak,
+                traffic=recorded_traffic(name, r["fingerprint"]), peak_source=pk["source"], peak_kind=peak_kind,
+                kernel_fingerprint=r["fingerprint"])
+
+
+def dtype_of(name):
+    return "bf16" if ("bf16" in name or name in ("matmul_dropout_mean_softmax", "conv_block", "dwconv_bn_relu", "mbconv_block")) else "f32"
+
+
+def sweep_record(steps, warmup, device, out_path, tune):
+    """The sweep as one entry of the "configs" list (also the body of the line --workload c5_sweep prints)."""
+    with ClockSampler(device) as clocks:
+        agg, launches = run_sweep(steps, warmup, device, out_path, tune)
+    pk = peaks()
+    return dict(workload="c5_sweep: 200 random operator DAGs, seeds 0..199", dtype="f32", steps=steps, warmup=max(1, warmup),
+                ms_per_step=agg["total_ms"], value=agg["memory_GBps"], unit="GB/s",
+                value_is="aggregate bytes / time over the memory-bound graphs of at least %d MB; see sweep for the GEMM-bound and small classes"
+                         % (SMALL_BYTES >> 20),
+                roofline=dict(bound="hbm", achieved=agg["memory_GBps"], peak=pk["hbm"], unit="GB/s", frac=agg["memory_GBps"] / pk["hbm"],
+                              traffic=None, peak_source=pk["source"], peak_kind="copy"),
+                gemm_roofline=dict(bound="tensor", achieved=agg["gemm_TFLOPps_fp32"], peak=pk["tensor"] / 6.0, unit="TFLOP/s",
+                                   frac=agg["gemm_TFLOPps_fp32"] / (pk["tensor"] / 6.0), peak_source=pk["source"],
+                                   peak_kind="gemm burst / 6 (three TF32 products at half the bf16 rate)"),
+                sweep=agg, clocks=clocks.summary(), gpu_launches=launches, l2="flushed between runs", tuned_trials=tune,
+                parity_checked=PARITY_TEST["c5_sweep"])
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="hct", choices=["hct", "reference"])
-    ap.add_argument("--workload", default=HEADLINE, choices=list(WORKLOADS) + ["c5_sweep"])
-    ap.add_argument("--out", default=None, help="c5_sweep: write one JSON record per graph to this file")
+    ap.add_argument("--workload", default=None, choices=list(WORKLOADS) + ["c5_sweep"],
+                    help="time this workload alone (default: the headline chain, with the other four configurations under 'configs')")
+    ap.add_argument("--out", default=None, help="write one JSON record per sweep graph to this file")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tune", type=int, default=0, help="pick each graph's schedule by measuring up to N candidates (untimed set-up)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    name = args.workload
+    all_configs = args.workload is None and world == 1
+    name = args.workload or HEADLINE
     info = WORKLOADS.get(name)
     metric = "fused-chain throughput: GB/s (memory-bound) / TFLOP/s (GEMM,conv) and % of B200 roofline"
 
@@ -362,9 +456,11 @@ def main():
             return
         if name == "c5_sweep":
             name = HEADLINE
-        r = oracle_arm(name, max(1, min(args.steps, 5)), min(args.warmup, 1))
-        line = dict(impl="reference", metric=metric, value=r["value"], unit=r["unit"], n_gpus=args.gpus, steps=args.steps,
-                    warmup=args.warmup, ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
+        # every step is a bounded sample of the workload; all requested steps and warm-ups are run
+        r = oracle_arm(name, max(1, args.steps), max(0, args.warmup), "ref_sample")
+        line = dict(impl="reference", metric=metric, value=r["value"], unit=r["unit"], n_gpus=args.gpus, steps=max(1, args.steps),
+                    warmup=max(0, args.warmup),
+                    ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
                     dtype="f64", data="synthetic", config={"workload": name, "sample": r["sample"]},
                     cpu_baseline=dict(value=r["value"], unit=r["unit"], cores=r["cores"], kind="oracle", sample=r["sample"]),
                     e2e=dict(value=r["value"], unit=r["unit"], h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
@@ -377,21 +473,17 @@ def main():
     if rank == 0:
         from paper_2506_10401_b200 import build as _build
         _build.build()  # in-tree library, rebuilt only when missing or stale
+    sweep_steps = max(3, min(args.steps, 10)) if name == "c5_sweep" else 3
     if name == "c5_sweep":
         if world > 1:
             raise SystemExit("the sweep runs on one GPU")
-        with ClockSampler(local) as clocks:
-            agg, launches = run_sweep(max(3, min(args.steps, 10)), args.warmup, local, args.out, args.tune)
-        pk = peaks()
-        print(json.dumps(dict(metric=metric, value=agg["memory_GBps"], unit="GB/s", n_gpus=1, steps=args.steps, warmup=args.warmup,
-                              ms_per_step=agg["total_ms"], higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
-                              data="synthetic", config={"workload": "c5_sweep: 200 random operator DAGs, seeds 0..199",
-                                                        "l2": "flushed between runs", "value_is": "aggregate over memory-bound graphs",
+        rec = sweep_record(sweep_steps, args.warmup, local, args.out, args.tune)
+        print(json.dumps(dict(metric=metric, value=rec["value"], unit="GB/s", n_gpus=1, steps=sweep_steps, warmup=rec["warmup"],
+                              ms_per_step=rec["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
+                              data="synthetic", config={"workload": rec["workload"], "l2": rec["l2"], "value_is": rec["value_is"],
                                                         "tuned_trials": args.tune},
-                              clocks=clocks.summary(), gpu_launches=launches, sweep=agg,
-                              roofline=dict(bound="hbm", achieved=agg["memory_GBps"], peak=pk["hbm"], unit="GB/s",
-                                            frac=agg["memory_GBps"] / pk["hbm"], traffic=None, peak_source=pk["source"]),
-                              e2e=None, cpu_baseline=None)))
+                              clocks=rec["clocks"], gpu_launches=rec["gpu_launches"], sweep=rec["sweep"], roofline=rec["roofline"],
+                              gemm_roofline=rec["gemm_roofline"], e2e=None, cpu_baseline=None)))
         return
     if world > 1:
         torch.cuda.set_device(local)
@@ -401,26 +493,30 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         o = oracle_arm(name, 4, 1)
         cpu = dict(value=o["value"], unit=o["unit"], cores=o["cores"], kind="oracle", sample=o["sample"])
+    others = []
+    if all_configs:
+        pk = peaks()
+        for other, cap, test in ALSO:
+            k = max(3, min(args.steps, cap))
+            o = run_gpu(other, k, args.warmup, rank, world, local, args.tune, with_e2e=False)
+            others.append(dict(workload=other, dtype=dtype_of(other), steps=k, warmup=max(args.warmup, 3), ms_per_step=o["ms_per_step"],
+                               value=o["value"], unit=o["unit"], roofline=roofline_of(other, o, pk), clocks=o["clocks"],
+                               kernels_per_step=o["kernels"], gpu_launches=o["kernels"] * k, l2="flushed between steps",
+                               parity_checked=test))
+        others.append(sweep_record(sweep_steps, min(args.warmup, 2), local, args.out, args.tune))
     if rank == 0:
         pk = peaks()
-        achieved, unit = metric_of(info["bound"], r["bytes"], r["flops"], r["kernel_s"])
-        # a contraction timed over a long run sits under the power cap: compare with the sustained GEMM
-        # figure then, with the burst figure when the clocks stayed at their maximum
-        clk = r["clocks"]
-        capped = "sw_power_cap" in clk["reasons"] and clk["sm_mhz"] and clk["sm_max_mhz"] and clk["sm_mhz"] < 0.9 * clk["sm_max_mhz"]
-        peak_kind = "copy" if info["bound"] == "hbm" else ("gemm sustained" if capped else "gemm burst")
-        peak = pk["hbm"] if info["bound"] == "hbm" else (pk["tensor_sustained"] if capped else pk["tensor"])
         line = dict(metric=metric, value=r["value"], unit=r["unit"], n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
                     ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
-                    dtype="bf16" if ("bf16" in name or name in ("matmul_dropout_mean_softmax", "conv_block", "dwconv_bn_relu", "mbconv_block")) else "f32", data="synthetic",
+                    dtype=dtype_of(name), data="synthetic",
                     config={"workload": name, "l2": "flushed between steps (192 MB write, untimed)", "kernels_per_step": r["kernels"],
                             "parallelism": "replicas" if world > 1 else "single",
-                            "schedule": r["schedule"] or "default", "tuned_trials": args.tune},
+                            "schedule": r["schedule"] or "default", "tuned_trials": args.tune,
+                            "parity_checked": PARITY_TEST.get(name)},
                     clocks=r["clocks"], e2e=r["e2e"], gpu_launches=r["kernels"] * args.steps,
-                    roofline=dict(bound=info["bound"], achieved=achieved, peak=peak, unit=("GB/s" if info["bound"] == "hbm" else "TFLOP/s"),
-                                  frac=achieved / peak, traffic=recorded_traffic(name, r["fingerprint"]), peak_source=pk["source"],
-                                  peak_kind=peak_kind, kernel_fingerprint=r["fingerprint"]),
-                    cpu_baseline=cpu)
+                    roofline=roofline_of(name, r, pk), cpu_baseline=cpu)
+        if all_configs:
+            line["configs"] = others
         print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()
