@@ -646,8 +646,8 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
             << skeleton_source("common") << "\nstruct HctParams { void* ptr[4]; };\n" << skeleton_source("conv_prep");
         k.source = src.str();
         k.ptrs = {node_buf(anchor.args[0].node), node_buf(anchor.args[1].node), scratch(0), scratch(x_bytes)};
-        int64_t blocks = (direct ? 0 : NB * ((C + 63) / 64) * ((H * W + 63) / 64)) + (KO * C * FR * FS + 255) / 256;
-        k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(blocks, 148 * 16));
+        int64_t blocks = direct ? (KO * C * FR * FS / 8 + 255) / 256 : NB * ((C + 63) / 64) * ((H * W + 63) / 64) + (KO * C * FR * FS + 255) / 256;
+        k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(blocks, direct ? 148 : 148 * 16));
         k.block[0] = 256;
         k.desc = direct ? "conv weight pre-pass: KCRS->RSKC" : "conv layout pre-pass: NCHW->NHWC activations, KCRS->RSKC weights";
         out->push_back(k);

@@ -1,12 +1,34 @@
 // Layout pre-pass for the tensor-core convolution: activations NCHW -> NHWC and weights
 // KCRS -> RSKC (both bf16), so that channels, the contraction axis, are contiguous for TMA.
-// With HCT_PREP_X = 0 only the weights are rearranged (the convolution then reads NCHW itself).
+// With HCT_PREP_X = 0 only the weights are rearranged (the convolution then reads NCHW itself): that
+// variant uses no shared memory and few CTAs, so that the convolution kernel, launched as a programmatic
+// dependent and needing a whole SM's shared memory per CTA, becomes resident beside it at once and
+// fills its pixel pipeline while the weights are being rearranged.
 // Defined by the generator: HCT_NB_IMG, HCT_C, HCT_HW (H*W), HCT_KO, HCT_RS (R*S), HCT_PREP_X, HctParams, HCT_KERNEL_NAME.
 // Pointer slots: 0 = X (NCHW), 1 = Wt (KCRS), 2 = X as NHWC, 3 = Wt as RSKC.
 #define HCT_XT_C ((HCT_C + 63) / 64)
 #define HCT_XT_P ((HCT_HW + 63) / 64)
 #define HCT_X_BLOCKS (HCT_PREP_X ? (long long)HCT_NB_IMG * HCT_XT_C * HCT_XT_P : 0LL)
 #define HCT_W_ELEMS ((long long)HCT_KO * HCT_C * HCT_RS)
+#if !HCT_PREP_X
+// one thread per 16-byte piece of the RSKC copy: 8 consecutive channels of one (tap, filter)
+extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {
+  hct_pdl_launch_dependents();
+  hct_pdl_wait();
+  const hct_bf16_t* __restrict__ Wt = (const hct_bf16_t*)hct_p.ptr[1];
+  hct_bf16_t* __restrict__ Wo = (hct_bf16_t*)hct_p.ptr[3];
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < HCT_W_ELEMS / 8; i += (long long)gridDim.x * 256) {
+    const int c = (int)(i % (HCT_C / 8)) * 8;
+    const int k = (int)((i / (HCT_C / 8)) % HCT_KO);
+    const int rs = (int)(i / ((long long)(HCT_C / 8) * HCT_KO));
+    const hct_bf16_t* src = Wt + ((long long)k * HCT_C + c) * HCT_RS + rs;
+    hct_u32 w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) w[j] = (hct_u32)__ldg(src + (2 * j) * HCT_RS) | ((hct_u32)__ldg(src + (2 * j + 1) * HCT_RS) << 16);
+    *(uint4*)(Wo + i * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+#else
 #define HCT_W_BLOCKS ((HCT_W_ELEMS + 255) / 256)
 extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {
   hct_pdl_launch_dependents();
@@ -67,3 +89,4 @@ extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParam
     }
   }
 }
+#endif
