@@ -67,6 +67,7 @@ struct Tunables {
   int dw_cta = 0;                  // depthwise conv: threads per block (0: rule; else a multiple of 32, up to 1024)
   int conv_nstg = 0;               // NCHW-reading conv: slots of the pixel staging ring (0: rule)
   int conv_nbuf = 0;               // NCHW-reading conv: operand buffers (0: rule)
+  int conv_flat = 0;               // NCHW-reading conv: tiles of 256 consecutive positions instead of whole rows (0: rule, 1: always, 2: never)
   bool topk_no_select = false;     // row_topk: full bitonic sort of the row even for small k
   bool conv_phase = false;         // strided convolutions: a stride-phase view wherever one exists, not only for rows too wide for a strided box
   bool conv_no_direct = false;     // always take the NHWC pre-pass, even when the convolution could read NCHW itself

@@ -610,7 +610,13 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       if (tun.conv_nstg >= 2 && tun.conv_nstg <= 12) n_stg = tun.conv_nstg;
       if (tun.conv_nbuf >= 2 && tun.conv_nbuf <= 3) n_buf = tun.conv_nbuf;
       int n_a = 0;
-      bool direct = false;
+      bool direct = false, flat = false;
+      // Flat tiling of the NCHW-reading kernel: tiles of 256 consecutive positions at the pitch of the padded row.
+      // An MMA takes about the same time whatever its width, so the schedule with fewer K loops on the busiest
+      // CTA wins: whole-row tiles cost one more loop whenever their count is not a multiple of the grid.
+      const int64_t flat_p = W + 2 * anchor.pad, flat_win = 256 + (FR - 1) * flat_p + FS - 1;
+      const int64_t flat_tiles = NB * ((HO * flat_p + 255) / 256) * ((KO + 127) / 128);
+      const int64_t flat_buf = (flat_win * 128 + 1023) / 1024 * 1024;
       // The epilogue of the NCHW-reading kernel hands its bf16 output to TMA stores (through 16 KB of
       // shared memory) when it stores a single bf16 tensor (output or intermediate) whose rows are 16-byte multiples.
       const bool tma_store = grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && WO % 8 == 0 && !tun.conv_no_tma_store;
@@ -619,6 +625,22 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         const int64_t fixed = n_buf * ((th_pitch + FR - 1) * pitch * 128 + 1024) + n_stg * pitch * 128 + 1024 + (tma_store ? 16384 : 0);
         n_a = (int)std::min<int64_t>(6, (232448 - 512 - fixed) / 16384);
         direct = n_a >= 3;
+        if (direct && grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && WO >= 32 && FS - 1 <= 4 && flat_p <= pitch && tun.conv_flat != 2) {
+          const int64_t row_tiles = NB * ((HO + th_pitch - 1) / th_pitch) * ((KO + 127) / 128);
+          const int64_t loops_row = row_tiles / 148 + (row_tiles % 148 ? 1 : 0), loops_flat = (flat_tiles + 147) / 148;
+          const int64_t fixed_flat = n_buf * flat_buf + n_stg * pitch * 128 + 1024 + 16384;
+          const int n_a_flat = (int)std::min<int64_t>(6, (232448 - 512 - fixed_flat) / 16384);
+          (void)loops_row; (void)loops_flat;
+          // measured slower than whole-row tiles on the benchmark convolution (37.9 against 35.8 us: its epilogue cannot use TMA
+          // stores and its tiles need more input rows), so it is taken on request only
+          if (n_a_flat >= 3 && tun.conv_flat == 1) {
+            flat = true;
+            n_a = n_a_flat;
+            // what the weight ring leaves over goes to the pixel staging ring: a flat tile needs more input rows before its first MMA
+            const int64_t left_over = 232448 - 512 - fixed_flat - (int64_t)n_a * 16384;
+            if (tun.conv_nstg == 0) n_stg += (int)std::min<int64_t>(3, left_over / (pitch * 128));
+          }
+        }
       }
       const bool halo = unit && !direct && FS > 1 && dense_pitch && !tun.conv_no_halo;
       const int TH = (direct || halo) ? th_pitch : (int)std::max<int64_t>(1, std::min<int64_t>(256 / WO, std::min<int64_t>(HO, phased ? 256 : 256 / ST)));
@@ -653,15 +675,17 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         out->push_back(k);
       }
       int stages = 4;
-      const bool use_tma_store = direct && tma_store;
-      std::string epi = eg.run_fn(HO * WO, WO, "(row % " + std::to_string(KO) + "LL)", use_tma_store);
+      const bool use_tma_store = direct && tma_store && !flat;
+      std::string epi = eg.run_fn(HO * WO, flat ? 1 : WO, "(row % " + std::to_string(KO) + "LL)", use_tma_store || flat);
+      const int out_slot = flat ? eg.ptr_index(grp.stores[0].node, !grp.stores[0].to_output) : 0;
       KernelSpec k;
       k.name = "hct_conv_tc_bf16_g" + std::to_string(gi);
       std::ostringstream src;
       src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_H " << H << "\n#define HCT_W " << W
           << "\n#define HCT_KO " << KO << "\n#define HCT_FR " << FR << "\n#define HCT_FS " << FS << "\n#define HCT_PAD " << anchor.pad
           << "\n#define HCT_STRIDE " << ST << "\n#define HCT_DIL " << DIL << "\n#define HCT_PHASED " << (phased ? 1 : 0) << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TH " << TH << "\n#define HCT_TH2 1\n#define HCT_SPLIT "
-          << TH << "\n#define HCT_PITCH " << pitch << "\n#define HCT_NA " << (direct ? n_a : 6) << "\n#define HCT_NBUF " << (direct ? n_buf : 3)
+          << (flat ? 1 : TH) << "\n#define HCT_PITCH " << pitch << "\n#define HCT_NA " << (direct ? n_a : 6) << "\n#define HCT_NBUF " << (direct ? n_buf : 3)
+          << "\n#define HCT_FLAT " << (flat ? 1 : 0) << "\n#define HCT_P " << flat_p << "\n#define HCT_OUT_SLOT " << out_slot
           << "\n#define HCT_NSTG " << n_stg << "\n#define HCT_X_IS_INPUT " << (a.cls == OpClass::Input ? 1 : 0) << "\n#define HCT_TMA_STORE " << (use_tma_store ? 1 : 0) << "\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
           << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
       src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[" << (phased ? 1 + 2 * ST : use_tma_store ? 3 : direct ? 2 : 3)
@@ -727,9 +751,10 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
           k.tmaps.push_back(ty);
         }
       }
-      int64_t tiles = NB * ((HO + TH - 1) / TH) * ((KO + 127) / 128);
-      k.block[0] = direct ? 480 : 192;
-      k.smem_bytes = direct ? (unsigned)(n_a * 16384 + n_buf * ((TH + FR - 1) * pitch * 128 + 1024) + n_stg * pitch * 128 + 1024 +
+      int64_t tiles = flat ? flat_tiles : NB * ((HO + TH - 1) / TH) * ((KO + 127) / 128);
+      k.block[0] = flat ? 608 : direct ? 480 : 192;
+      k.smem_bytes = flat   ? (unsigned)(n_a * 16384 + n_buf * flat_buf + n_stg * pitch * 128 + 1024 + 16384)
+                     : direct ? (unsigned)(n_a * 16384 + n_buf * ((TH + FR - 1) * pitch * 128 + 1024) + n_stg * pitch * 128 + 1024 +
                                          (use_tma_store ? 16384 : 0))
                      : halo ? (unsigned)(6 * 16384 + 3 * 33792 + 1024) : (unsigned)(stages * (128 * 128 + 32768) + 1024);
       k.persistent = true;
@@ -737,7 +762,9 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       k.grid[0] = k.max_grid;
       std::ostringstream d;
       d << "conv2d tcgen05 bf16 implicit GEMM, tile 128 channels x " << TH << " rows of " << WO << " pixels, ";
-      if (direct)
+      if (flat)
+        d << "NCHW read directly and re-laid in shared memory, flat tiles of 256 positions at pitch " << flat_p;
+      else if (direct)
         d << "NCHW read directly and re-laid in shared memory, every pixel loaded once per tile (pitch " << pitch << ")";
       else if (halo)
         d << "pixels shared by the taps of a filter row (pitch " << pitch << ")";

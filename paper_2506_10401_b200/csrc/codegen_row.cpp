@@ -32,6 +32,7 @@ const Knob kKnobs[] = {
     {"gemm_insplit", &Tunables::gemm_insplit, 0, nullptr},
     {"conv_nstg", &Tunables::conv_nstg, 0, nullptr},
     {"conv_nbuf", &Tunables::conv_nbuf, 0, nullptr},
+    {"conv_flat", &Tunables::conv_flat, 0, nullptr},
     {"dw_p", &Tunables::dw_p, 0, nullptr},
     {"dw_cta", &Tunables::dw_cta, 0, nullptr},
     {"simt_only", nullptr, 0, &Tunables::simt_only},

@@ -23,13 +23,31 @@
 // When the activations are a graph input (HCT_X_IS_INPUT) only the weight producer and the epilogue
 // wait for the preceding kernel (programmatic dependent launch) and the pixel pipeline fills meanwhile.
 //
+// Flat tiling (HCT_FLAT).  An MMA instruction of this shape takes about the same time whatever its
+// width, so what counts is the number of K loops on the busiest CTA.  With tiles of whole output
+// rows at a pitch that is a multiple of 32, part of every MMA works on padding columns, and a tile
+// count just above a multiple of the grid costs one more K loop.  In flat mode the positions of an
+// image are numbered row after row at a pitch of HCT_P = W + 2 * pad (the padded row, no rounding),
+// a tile is 256 consecutive positions of one image wherever they start, and the operand buffer holds
+// the window of padded input positions under it: tap (r,s) still starts r * HCT_P + s rows later.
+// The HCT_P - HCT_WO positions at the end of every row are computed and dropped; the epilogue closes
+// the gap they leave, so that the values of a 32-column chunk form one contiguous run of the NCHW
+// plane, stages the run in shared memory, and the warp stores it channel by channel (64 contiguous
+// bytes per instruction; the run may start at any element, so no vector or TMA store).
+//
 // Defined by the generator: HCT_NB_IMG, HCT_C, HCT_H, HCT_W, HCT_KO, HCT_FR, HCT_FS, HCT_PAD, HCT_HO, HCT_WO,
 // HCT_PITCH, HCT_TH, HCT_TH2 (= 1), HCT_SPLIT, HCT_NA, HCT_NBUF, HCT_NSTG, HCT_X_IS_INPUT, HCT_TMA_STORE, HCT_STATUS_SLOT,
 // HCT_KERNEL_NAME, HctParams, hct_epilogue_run() or (HCT_TMA_STORE) hct_epilogue_vals().
 #define HCT_BM 128
 #define HCT_A_BYTES (HCT_BM * 128)                       // weights: 128 channels x 64 inputs, bf16
+#if HCT_FLAT
+#define HCT_WIN (256 + (HCT_FR - 1) * HCT_P + HCT_FS - 1)     // padded input positions under a tile of 256 output positions
+#define HCT_B_BYTES ((HCT_WIN * 128 + 1023) / 1024 * 1024)
+#define HCT_TPI ((HCT_HO * HCT_P + 255) / 256)                // tiles per image
+#else
 #define HCT_ROWS_MAX (HCT_TH + HCT_FR - 1)               // input rows under a whole tile
 #define HCT_B_BYTES (HCT_ROWS_MAX * HCT_PITCH * 128 + 1024)   // operand buffer + room for the shifted reads
+#endif
 #define HCT_S_BYTES (HCT_PITCH * 128)                    // staging box: 64 channels x pitch pixels
 #define HCT_RING_B_OFF (HCT_NA * HCT_A_BYTES)
 #define HCT_RING_S_OFF (HCT_RING_B_OFF + HCT_NBUF * HCT_B_BYTES)
@@ -37,15 +55,38 @@
 #define HCT_CB ((HCT_C + 63) / 64)
 #define HCT_HT ((HCT_HO + HCT_TH - 1) / HCT_TH)
 #define HCT_MBK ((HCT_KO + HCT_BM - 1) / HCT_BM)
+#if HCT_FLAT
+#define HCT_FULL_TILES ((long long)HCT_NB_IMG * HCT_TPI * HCT_MBK)
+#else
 #define HCT_FULL_TILES ((long long)HCT_NB_IMG * HCT_HT * HCT_MBK)
+#endif
 #define HCT_NT 256                                       // transposer threads
+#if HCT_FLAT
+#define HCT_EPI2 4                                       // extra epilogue warps (15-18): every lane quarter is drained by two warps
+#else
+#define HCT_EPI2 0
+#endif
 #define HCT_NBAR (2 * HCT_NA + 2 * HCT_NBUF + 2 * HCT_NSTG + 4)
 
-struct HctConvTile { int n, h0, th, mbk; bool cut; };
+struct HctConvTile { int n, h0, th, mbk; bool cut; int o0, lo, nrows; };
 
 // Tile t of the schedule.  Tiles below `t1` are whole; the rest are pieces of the remaining whole tiles.
 __device__ __forceinline__ HctConvTile hct_conv_tile(long long t, long long t1) {
   HctConvTile r;
+#if HCT_FLAT
+  // tile = 256 consecutive positions of one image; `lo` .. `lo + nrows - 1` are the padded input rows its window meets
+  (void)t1;
+  long long w_ = t;
+  r.mbk = (int)(w_ % HCT_MBK); w_ /= HCT_MBK;
+  r.o0 = (int)(w_ % HCT_TPI) * 256;
+  r.n = (int)(w_ / HCT_TPI);
+  r.lo = r.o0 / HCT_P;
+  int hi = (r.o0 + HCT_WIN - 1) / HCT_P;
+  if (hi > HCT_H + 2 * HCT_PAD - 1) hi = HCT_H + 2 * HCT_PAD - 1;
+  r.nrows = hi - r.lo + 1;
+  r.h0 = 0; r.th = 1; r.cut = false;
+  return r;
+#endif
   long long whole = t;
   int sub = 0;
   r.cut = t >= t1;
@@ -63,7 +104,7 @@ __device__ __forceinline__ HctConvTile hct_conv_tile(long long t, long long t1) 
   return r;
 }
 
-extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(const __grid_constant__ HctParams hct_p) {
+extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HCT_KERNEL_NAME(const __grid_constant__ HctParams hct_p) {
   extern __shared__ unsigned char hct_smem_raw[];
   __shared__ unsigned long long bars[HCT_NBAR];
   __shared__ hct_u32 tmem_holder;
@@ -103,7 +144,7 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(co
     }
     for (int a = 0; a < 2; ++a) {
       hct_mbar_init(tfull0 + 8 * a, 1);
-      hct_mbar_init(tempty0 + 8 * a, 128);
+      hct_mbar_init(tempty0 + 8 * a, 128 + 32 * HCT_EPI2);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     hct_prefetch_tmap(&hct_p.tmap[0]);
@@ -145,7 +186,11 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(co
         const HctConvTile t = hct_conv_tile(tile, t1);
         if (t.th == 0) continue;
         // bf16 x bf16 -> fp32, both operands K-major, M = 128, N = rows of this tile times the pitch
+#if HCT_FLAT
+        const hct_u32 n_mma = 256u;
+#else
         const hct_u32 n_mma = (hct_u32)(t.th * HCT_PITCH);
+#endif
         const hct_u32 idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((n_mma >> 3) << 17) | ((hct_u32)(HCT_BM >> 4) << 24);
         hct_mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, &failed, status, 2);
         hct_tc_fence_after();
@@ -161,7 +206,11 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(co
               // tap (r,s) reads the operand buffer r * pitch + s pixel rows (128 bytes each) further on; the
               // 128-byte swizzle follows the absolute shared-memory address, so only the start field changes
               const hct_u64 a_desc0 = hct_smem_desc(smem_base + sa * HCT_A_BYTES, 16, 1024);
+#if HCT_FLAT
+              const hct_u64 b_desc0 = hct_smem_desc(b_addr + (r * HCT_P + s) * 128, 16, 1024);
+#else
               const hct_u64 b_desc0 = hct_smem_desc(b_addr + (r * HCT_PITCH + s) * 128, 16, 1024);
+#endif
 #pragma unroll
               for (int kk = 0; kk < 4; ++kk) hct_mma_f16(d_tmem, a_desc0 + kk * 2, b_desc0 + kk * 2, idesc, (cb | r | s | kk) != 0);
               hct_mma_commit(aempty0 + 8 * sa);
@@ -175,7 +224,7 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(co
         if (acc == 0) acc_phase ^= 1u;
       }
     }
-  } else if (warp < 6) {
+  } else if (warp < 6 || warp >= 15) {
     // ---- epilogue: one output channel per thread, 32 consecutive pixels per step
     const int q = warp & 3;
     int acc = 0;
@@ -190,6 +239,65 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(co
       hct_mbar_wait(tfull0 + 8 * acc, acc_phase, &failed, status, 4);
       hct_tc_fence_after();
       const int k = t.mbk * HCT_BM + q * 32 + lane;      // output channel of this thread's TMEM lane
+#if HCT_FLAT
+#pragma unroll 1
+      for (int c = (warp >= 15 ? 1 : 0); c < 8; c += 2) {
+        // positions oc .. oc + 31 of the image: n1 valid ones up to the end of output row `hrow`, then `skip`
+        // dropped ones (the padding columns of that row), then n2 valid ones of the next row
+        const int oc = t.o0 + c * 32;
+        if (oc >= HCT_HO * HCT_P) break;
+        const int hrow = oc / HCT_P, a = oc - hrow * HCT_P;
+        const int n1 = a < HCT_WO ? (HCT_WO - a < 32 ? HCT_WO - a : 32) : 0;
+        const int jend = HCT_P - a < 32 ? HCT_P - a : 32;
+        const int skip = jend - n1;
+        const int run = n1 + (hrow + 1 < HCT_HO ? 32 - jend : 0);
+        if (run == 0) continue;
+        const int idx0 = hrow * HCT_WO + (a < HCT_WO ? a : HCT_WO);     // index of the run's first element in its plane
+        float v[32], w[32];
+        hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * 256 + c * 32, v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          float x = v[j];
+#pragma unroll
+          for (int g = 1; g <= HCT_P - HCT_WO; ++g)
+            if (j + g < 32) x = (skip == g && j >= n1) ? v[j + g < 32 ? j + g : 31] : x;
+          w[j] = x;
+        }
+        float o[32];
+        if (k < HCT_KO) {
+          hct_epilogue_vals(hct_p, w, (long long)t.n * HCT_KO + k, idx0, run, o);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[j] = 0.0f;
+        }
+        // rows of 64 bytes (one channel each), 16-byte piece j of row i at piece j ^ ((i >> 1) & 3)
+        const hct_u32 o_slot = smem_base + HCT_RING_O_OFF + (hct_u32)((q * 2 + (warp >= 15 ? 1 : 0)) * 2048);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const hct_u32 dst = o_slot + (hct_u32)lane * 64u + (((hct_u32)j ^ (((hct_u32)lane >> 1) & 3u)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(hct_pack_bf16x2(o[8 * j], o[8 * j + 1])),
+                       "r"(hct_pack_bf16x2(o[8 * j + 2], o[8 * j + 3])), "r"(hct_pack_bf16x2(o[8 * j + 4], o[8 * j + 5])),
+                       "r"(hct_pack_bf16x2(o[8 * j + 6], o[8 * j + 7]))
+                       : "memory");
+        }
+        __syncwarp();
+        // the warp stores the run of every channel: lane = element of the run
+        const int kbase = t.mbk * HCT_BM + q * 32;
+        hct_bf16_t* yrow = (hct_bf16_t*)hct_p.ptr[HCT_OUT_SLOT] + ((long long)t.n * HCT_KO + kbase) * (long long)(HCT_HO * HCT_WO) + idx0 + lane;
+        const hct_u32 src0 = o_slot + ((hct_u32)lane & 7u) * 2u;
+        if (lane < run) {
+#pragma unroll 8
+          for (int i = 0; i < 32; ++i) {
+            if (kbase + i < HCT_KO) {
+              unsigned short e_;
+              asm volatile("ld.shared.u16 %0, [%1];" : "=h"(e_) : "r"(src0 + (hct_u32)i * 64u + ((((hct_u32)lane >> 3) ^ (((hct_u32)i >> 1) & 3u)) << 4)) : "memory");
+              yrow[(long long)i * (HCT_HO * HCT_WO)] = e_;
+            }
+          }
+        }
+        __syncwarp();
+      }
+#else
       const int chunks = t.th * (HCT_PITCH / 32);
 #pragma unroll 1
       for (int c = 0; c < chunks; ++c) {
@@ -235,6 +343,7 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(co
         if (k < HCT_KO) hct_epilogue_run(hct_p, v, (long long)t.n * HCT_KO + k, (t.h0 + hh) * HCT_WO + part * 32, ncols);
 #endif
       }
+#endif   // HCT_FLAT
       hct_tc_fence_before();
       hct_mbar_arrive(tempty0 + 8 * acc);
       acc ^= 1;
@@ -254,12 +363,16 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(co
       for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         const HctConvTile t = hct_conv_tile(tile, t1);
         if (t.th == 0) continue;
-        const int nrows = t.th + HCT_FR - 1;
+#if HCT_FLAT
+        const int nrows = t.nrows, row0 = t.lo - HCT_PAD;
+#else
+        const int nrows = t.th + HCT_FR - 1, row0 = t.h0 - HCT_PAD;
+#endif
         for (int cb = 0; cb < HCT_CB; ++cb)
           for (int rr = 0; rr < nrows; ++rr) {
             hct_mbar_wait(sempty0 + 8 * ss, ps ^ 1u, &failed, status, 7);
             hct_mbar_expect_tx(sfull0 + 8 * ss, HCT_S_BYTES);
-            hct_tma_load_4d(smem_base + HCT_RING_S_OFF + ss * HCT_S_BYTES, &hct_p.tmap[1], 0, t.h0 - HCT_PAD + rr, cb * 64, t.n, sfull0 + 8 * ss);
+            hct_tma_load_4d(smem_base + HCT_RING_S_OFF + ss * HCT_S_BYTES, &hct_p.tmap[1], 0, row0 + rr, cb * 64, t.n, sfull0 + 8 * ss);
             if (++ss == HCT_NSTG) { ss = 0; ps ^= 1u; }
           }
       }
@@ -268,6 +381,7 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(co
     // ---- transposers: staged [channel][pixel] box -> operand rows [pixel][channel], shifted by the padding
     const int tt = threadIdx.x - 224;    // 0 .. HCT_NT-1
     const unsigned char* smem_gen = hct_smem_raw + (smem_base - hct_smem_addr(hct_smem_raw));   // generic view of smem_base
+#if !HCT_FLAT
     // the left border (positions below the padding) is never written again: zero it once in every buffer
     for (int i = tt; i < HCT_NBUF * HCT_ROWS_MAX * HCT_PAD * 8; i += HCT_NT) {
       const int unit = i & 7, rest = i >> 3;
@@ -275,18 +389,32 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(co
       const int buf = rowi / HCT_ROWS_MAX, rr = rowi % HCT_ROWS_MAX;
       *(uint4*)(smem_gen + HCT_RING_B_OFF + buf * HCT_B_BYTES + (rr * HCT_PITCH + pos) * 128 + unit * 16) = make_uint4(0u, 0u, 0u, 0u);
     }
+#endif
     int ss = 0, sb = 0;
     hct_u32 ps = 0, pb = 0;
     for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
       const HctConvTile t = hct_conv_tile(tile, t1);
       if (t.th == 0) continue;
+#if HCT_FLAT
+      const int nrows = t.nrows;
+#else
       const int nrows = t.th + HCT_FR - 1;
+#endif
       for (int cb = 0; cb < HCT_CB; ++cb) {
         hct_mbar_wait(bempty0 + 8 * sb, pb ^ 1u, &failed, status, 1);
         unsigned char* b_gen = (unsigned char*)smem_gen + HCT_RING_B_OFF + sb * HCT_B_BYTES;
         for (int rr = 0; rr < nrows; ++rr) {
           hct_mbar_wait(sfull0 + 8 * ss, ps, &failed, status, 8);
           const unsigned char* s_gen = smem_gen + HCT_RING_S_OFF + ss * HCT_S_BYTES;
+#if HCT_FLAT
+          // position of this padded row's first column in the window (may lie before it); the columns left of
+          // the image are zero, the ones right of it arrive as zeros in the staged box
+          const int rowbase = (t.lo + rr) * HCT_P - t.o0;
+          if (tt < 8 * HCT_PAD) {
+            const int q0 = rowbase + (tt >> 3);
+            if (q0 >= 0 && q0 < HCT_WIN) *(uint4*)(b_gen + (hct_u32)q0 * 128u + (((hct_u32)(tt & 7) ^ ((hct_u32)q0 & 7u)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+          }
+#endif
           // work item = (pair of neighbouring pixels, group of 8 channels): eight 4-byte reads along the staged
           // channel rows give both pixels; each pixel's 8 channels leave as one 16-byte write into its row.
           // A warp shares the channel group and covers 32 consecutive pairs; half of every 8 lanes writes its
@@ -296,6 +424,9 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(co
             const int it = i0 + tt;
             if (HCT_PITCH * 4 % HCT_NT != 0 && it >= HCT_PITCH * 4) break;
             const int m = it % (HCT_PITCH / 2), u = it / (HCT_PITCH / 2);
+#if HCT_FLAT
+            if (rowbase + 2 * m + HCT_PAD + 1 < 0 || rowbase + 2 * m + HCT_PAD >= HCT_WIN || 2 * m + HCT_PAD >= HCT_P) continue;
+#endif
             const hct_u32* src = (const hct_u32*)(s_gen + ((u * 8) * HCT_PITCH + 2 * m) * 2);
             hct_u32 e[8];
 #pragma unroll
@@ -307,9 +438,16 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT, 1) HCT_KERNEL_NAME(co
             lo.w = __byte_perm(e[6], e[7], 0x5410); hi.w = __byte_perm(e[6], e[7], 0x7632);
             const bool odd_first = (m & 4) != 0;
             const int pos_a = 2 * m + HCT_PAD + (odd_first ? 1 : 0), pos_b = 2 * m + HCT_PAD + (odd_first ? 0 : 1);
+#if HCT_FLAT
+            const int qa_ = rowbase + pos_a, qb_ = rowbase + pos_b;
+            const hct_u32 qa = (hct_u32)qa_, qb = (hct_u32)qb_;
+            if (pos_a < HCT_P && qa_ >= 0 && qa_ < HCT_WIN) *(uint4*)(b_gen + qa * 128u + (((hct_u32)u ^ (qa & 7u)) << 4)) = odd_first ? hi : lo;
+            if (pos_b < HCT_P && qb_ >= 0 && qb_ < HCT_WIN) *(uint4*)(b_gen + qb * 128u + (((hct_u32)u ^ (qb & 7u)) << 4)) = odd_first ? lo : hi;
+#else
             const hct_u32 qa = (hct_u32)(rr * HCT_PITCH + pos_a), qb = (hct_u32)(rr * HCT_PITCH + pos_b);
             if (pos_a < HCT_PITCH) *(uint4*)(b_gen + qa * 128u + (((hct_u32)u ^ (qa & 7u)) << 4)) = odd_first ? hi : lo;
             if (pos_b < HCT_PITCH) *(uint4*)(b_gen + qb * 128u + (((hct_u32)u ^ (qb & 7u)) << 4)) = odd_first ? lo : hi;
+#endif
           }
           __syncwarp();
           if (lane == 0) hct_mbar_arrive(sempty0 + 8 * ss);

@@ -230,6 +230,30 @@ def test_conv_chain_shapes(kw):
     check_bf16(spec, laws)
 
 
+@pytest.mark.parametrize("kw", [
+    dict(n=2, c=128, h=56, w=56, k=128),                       # tiles start in the middle of rows; 13 tiles per image, the last one short
+    dict(n=1, c=72, h=17, w=48, k=130, ksize=5, pad=2),        # four dropped positions per row, two blocks of output channels
+    dict(n=3, c=128, h=6, w=64, k=64, ksize=1, pad=0),         # no dropped positions at all
+    dict(n=1, c=16, h=33, w=56, k=128, ksize=3, pad=0),        # no padding: the pitch is the image width
+    dict(n=2, c=8, h=5, w=88, k=8, ksize=3, pad=1),            # rows longer than two chunks
+    dict(n=1, c=64, h=9, w=48, k=32, ksize=3, pad=2),          # padding wider than half the filter: output rows longer than input rows
+])
+def test_conv_flat_tiles(kw):
+    """Tiles of 256 consecutive positions (chosen by rule only when they save a K loop), forced onto other shapes:
+    the chain within the bf16 tolerance, and the bare convolution bit for bit on integer-valued inputs."""
+    spec, laws = configs.get_config("c4_conv_bn_relu_bf16", **kw)
+    got, want, g = parity.run_both(spec, laws, schedule="conv_flat=1")
+    assert "flat tiles" in g.plan
+    assert parity.bf16_violation(got[0], want[0]) <= 1.0
+    ks, pad = kw.get("ksize", 3), kw.get("pad", 1)
+    spec = (f"hct 1\ninput x bf16 [{kw['n']},{kw['c']},{kw['h']},{kw['w']}]\ninput w bf16 [{kw['k']},{kw['c']},{ks},{ks}]\n"
+            f"node y = conv2d(x, w, stride=1, pad={pad})\nnode z = cast_bf16(y)\noutput z bf16\n")
+    il = {"kind": "int", "lo": -2, "hi": 2}
+    got, want, g = parity.run_both(spec, {"x": il, "w": il}, schedule="conv_flat=1")
+    assert "flat tiles" in g.plan
+    np.testing.assert_array_equal(got[0], want[0])
+
+
 def test_conv_f32_integer_inputs_are_exact():
     spec = "hct 1\ninput x f32 [2,16,10,12]\ninput w f32 [8,16,3,3]\nnode y = conv2d(x, w, stride=1, pad=1)\noutput y\n"
     il = {"kind": "int", "lo": -4, "hi": 4}
