@@ -304,6 +304,67 @@ def run_gpu(name, steps, warmup, rank, world, device, tune=0, with_e2e=True):
                 schedule=g.schedule)
 
 
+def replay_seconds(g, ins, device, budget_bytes=256 << 20, max_sets=24, target_ms=4.0):
+    """Steady-state time of one run of graph `g`, without a host launch or an event pair per step.
+
+    A step timed between its own pair of events costs about 6 us on top of the kernel (measured with a
+    one-thread kernel in the same place), which buries chains that run for a few microseconds.  Here the
+    inputs, outputs and workspace exist in several copies whose total exceeds L2 twice over (as many as
+    `budget_bytes` needs, at most `max_sets`), one run per copy is captured into a CUDA graph, and the graph
+    is replayed between ONE pair of events: kernels follow each other on the device and every run finds its
+    operands cold in L2 (or, for graphs too small to fill the budget with `max_sets` copies, partly warm:
+    the second value returned says which).  Returns (seconds per run, "cold" | "warm") or None when the
+    capture is not possible."""
+    import torch
+    import paper_2506_10401_b200 as hct
+    dev = f"cuda:{device}"
+    per_set = sum(t.numel() * t.element_size() for t in ins) + g.workspace_bytes
+    outs0 = g.alloc_outputs()
+    per_set += sum(t.numel() * t.element_size() for t in outs0)
+    n_sets = int(max(1, min(max_sets, -(-budget_bytes // per_set))))
+    sets = []
+    for i in range(n_sets):
+        si = ins if i == 0 else [t.clone() for t in ins]
+        so = outs0 if i == 0 else g.alloc_outputs()
+        ws = torch.empty(g.workspace_bytes + 256, dtype=torch.uint8, device=dev) if g.workspace_bytes else None
+        ws_ptr = (ws.data_ptr() + 255) // 256 * 256 if ws is not None else 0
+        sets.append((si, so, ws, [t.data_ptr() for t in si], [t.data_ptr() for t in so], ws_ptr))
+    side = torch.cuda.Stream(device)
+
+    def enqueue(stream):
+        for _, _, _, pi, po, pw in sets:
+            hct.hct_graph_run(g.handle, pi, po, pw, g.workspace_bytes, stream.cuda_stream)
+
+    try:
+        side.wait_stream(torch.cuda.current_stream(device))
+        with torch.cuda.stream(side):
+            enqueue(side)
+        side.synchronize()
+        cg = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(cg, stream=side, capture_error_mode="thread_local"):
+            enqueue(side)
+    except Exception as e:  # noqa: BLE001 - any capture failure falls back to the per-step protocol
+        print(f"replay capture failed: {e}", file=sys.stderr)
+        return None
+    stream = torch.cuda.current_stream(device)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    cg.replay()
+    torch.cuda.synchronize(device)
+    a.record(stream); cg.replay(); b.record(stream)
+    torch.cuda.synchronize(device)
+    once_ms = max(a.elapsed_time(b), 1e-3)
+    reps = int(max(2, min(200, target_ms / once_ms)))
+    a.record(stream)
+    for _ in range(reps):
+        cg.replay()
+    b.record(stream)
+    torch.cuda.synchronize(device)
+    g.status()
+    sec = a.elapsed_time(b) * 1e-3 / (reps * n_sets)
+    del cg
+    return sec, ("cold" if per_set * n_sets >= 192 << 20 else "warm"), n_sets
+
+
 def run_sweep(steps, warmup, device, out_path=None, tune=0):
     """The 200 random operator DAGs: per-graph time against its own roofline, and class aggregates.
 
@@ -358,16 +419,25 @@ def run_sweep(steps, warmup, device, out_path=None, tune=0):
             b.record(stream)
         torch.cuda.synchronize(device)
         g.status()
-        sec = float(np.median([a.elapsed_time(b) for a, b in ev])) * 1e-3
+        # event time stamps on this platform step by about 2 us: the mean over the steps (largest one dropped)
+        # resolves a microsecond-scale run, their median does not
+        ms = sorted(a.elapsed_time(b) for a, b in ev)
+        sec = float(np.mean(ms[:-1] if len(ms) > 3 else ms)) * 1e-3
         bytes_, flops = g.cost()
         t_mem = bytes_ / (pk["hbm"] * 1e9)
         t_mma = flops / (pk["tensor"] / 6.0 * 1e12)  # fp32 GEMM = three TF32 products at half the bf16 rate
         cls = "gemm" if t_mma > t_mem else "memory"
-        records.append(dict(seed=e["seed"], cls=cls, us=sec * 1e6, bytes=bytes_, flops=flops, kernels=g.num_kernels, schedule=g.schedule,
-                            frac=max(t_mem, t_mma) / sec))
+        del outs
+        rp = replay_seconds(g, ins, device)
+        sec_events = sec
+        if rp is not None:
+            sec = rp[0]
+        records.append(dict(seed=e["seed"], cls=cls, us=sec * 1e6, us_events=sec_events * 1e6, l2=(rp[1] if rp else "flushed"),
+                            sets=(rp[2] if rp else 1), bytes=bytes_, flops=flops, kernels=g.num_kernels, schedule=g.schedule,
+                            frac=max(t_mem, t_mma) / sec, frac_events=max(t_mem, t_mma) / sec_events))
         launches += g.num_kernels * (steps + max(1, warmup))
         g.close()
-        del ins, outs
+        del ins
     pool.shutdown()
     if out_path:
         with open(out_path, "w") as f:
@@ -389,6 +459,11 @@ def run_sweep(steps, warmup, device, out_path=None, tune=0):
                small_us_max=float(np.max([r["us"] for r in small])) if small else None,
                small_launches_mean=float(np.mean([r["kernels"] for r in small])) if small else None,
                small_bytes_below=SMALL_BYTES,
+               timing="CUDA-graph replay over rotating copies of every buffer (total above twice L2), one event pair per graph",
+               events_memory_GBps=sum(r["bytes"] for r in mem) / sum(r["us_events"] for r in mem) / 1e3 if mem else None,
+               events_gemm_TFLOPps_fp32=sum(r["flops"] for r in mma) / sum(r["us_events"] for r in mma) / 1e6 if mma else None,
+               events_small_us_median=float(np.median([r["us_events"] for r in small])) if small else None,
+               events_note="same graphs, every step between its own event pair after an L2 flush: about 6 us of launch and event cost per step",
                all_memory_GBps=sum(r["bytes"] for r in mem + small) / sum(r["us"] for r in mem + small) / 1e3 if mem or small else None,
                total_ms=sum(r["us"] for r in records) / 1e3)
     return agg, launches
@@ -427,7 +502,7 @@ def sweep_record(steps, warmup, device, out_path, tune):
                 gemm_roofline=dict(bound="tensor", achieved=agg["gemm_TFLOPps_fp32"], peak=pk["tensor"] / 6.0, unit="TFLOP/s",
                                    frac=agg["gemm_TFLOPps_fp32"] / (pk["tensor"] / 6.0), peak_source=pk["source"],
                                    peak_kind="gemm burst / 6 (three TF32 products at half the bf16 rate)"),
-                sweep=agg, clocks=clocks.summary(), gpu_launches=launches, l2="flushed between runs", tuned_trials=tune,
+                sweep=agg, clocks=clocks.summary(), gpu_launches=launches, l2="cold: rotating buffer copies larger than L2 (graphs under %d MB: warm, reported as latency)" % (SMALL_BYTES >> 20), tuned_trials=tune,
                 parity_checked=PARITY_TEST["c5_sweep"])
 
 
