@@ -497,18 +497,22 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         k.desc = "tf32 head/tail split of both gemm operands, B transposed";
         out->push_back(k);
       }
-      const int bn_max = N > 64 ? 128 : N > 32 ? 64 : 32;
-      int BN = bn_max;
+      // 256-column tiles (`gemm_bn=256`) halve the instruction count but were measured no faster than 128-column ones
+      // (28 against 26 us on 1024 x 256 x 4096): with head and tail of both operands a k step moves 96 KB into shared
+      // memory per 6 MFLOP, and the kernel runs at the rate L2 delivers them.  They are taken on request only.
+      const int bn_max = N > 128 ? 256 : N > 64 ? 128 : N > 32 ? 64 : 32;
+      int BN = std::min(bn_max, 128);
       while (BN > 64 && ((M + 127) / 128) * ((N + BN - 1) / BN) * 2 <= 148) BN /= 2;
-      if (tun.gemm_bn >= 32) BN = std::min(bn_max, tun.gemm_bn >= 128 ? 128 : tun.gemm_bn >= 64 ? 64 : 32);
-      int stages = BN == 128 ? 3 : BN == 64 ? 4 : 5;
+      if (tun.gemm_bn >= 32) BN = std::min(bn_max, tun.gemm_bn >= 256 ? 256 : tun.gemm_bn >= 128 ? 128 : tun.gemm_bn >= 64 ? 64 : 32);
+      int stages = BN == 256 ? 2 : BN == 128 ? 3 : BN == 64 ? 4 : 5;
       std::string epi = eg.run_fn(N);
       // CTA pairs on 256 x 256 tiles when every pair of SMs gets at least one tile.  Measured on
       // 16384 x 4096 x 4096: 2.31 ms against 2.93 ms for 128 x 128 tiles on single CTAs (a TF32 MMA of
       // 128 columns does not fill the tensor pipe's issue interval; 256 columns per instruction do).
       const int64_t pair_tiles32 = ((M + 255) / 256) * ((N + 255) / 256);
       // (from 56 tiles on, and a contraction deep enough to amortise the pair's set-up: measured break-even)
-      if (tun.gemm_pair == 1 || (tun.gemm_pair == 0 && pair_tiles32 >= 56 && K >= 512 && tun.gemm_bn == 0)) {
+      // (a shallow contraction still gains once there are several rounds of tiles: 16384 x 256 x 4096 measured 224 against 254 us)
+      if (tun.gemm_pair == 1 || (tun.gemm_pair == 0 && ((pair_tiles32 >= 56 && K >= 512) || pair_tiles32 >= 512) && tun.gemm_bn == 0)) {
         const int pstages = 3;
         KernelSpec k;
         k.name = "hct_gemm_tc2_tf32x3_g" + std::to_string(gi);
@@ -568,7 +572,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         k.tmaps.push_back(t);
       }
       int64_t tiles = ((M + 127) / 128) * ((N + BN - 1) / BN);
-      k.block[0] = 192;
+      k.block[0] = BN > 128 ? 320 : 192;   // wide tiles: eight epilogue warps
       k.smem_bytes = (unsigned)(stages * (2 * 128 * 128 + 2 * BN * 128) + 1024);
       k.persistent = true;
       k.max_grid = (unsigned)std::min<int64_t>(tiles, 0x7fffffff);

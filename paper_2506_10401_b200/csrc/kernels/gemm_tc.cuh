@@ -44,8 +44,16 @@
 #define HCT_NB ((HCT_N + HCT_BN - 1) / HCT_BN)
 #define HCT_TILES ((long long)HCT_MB * HCT_NB)
 #define HCT_TMEM_COLS (2 * HCT_BN < 32 ? 32 : 2 * HCT_BN)
+// A TF32 instruction covers 8 elements of K and takes about as long at 128 columns as at 256, so wide
+// tiles halve the instruction count.  Their running sums (one register per column) are then shared by
+// two epilogue warps per lane quarter, 128 columns each.
+#if HCT_TF32X3 && HCT_BN > 128
+#define HCT_EPI_WARPS 8
+#else
+#define HCT_EPI_WARPS 4
+#endif
 
-extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __grid_constant__ HctParams hct_p) {
+extern "C" __global__ void __launch_bounds__(64 + 32 * HCT_EPI_WARPS, 1) HCT_KERNEL_NAME(const __grid_constant__ HctParams hct_p) {
   extern __shared__ unsigned char hct_smem_raw[];
   __shared__ unsigned long long bars[2 * HCT_STAGES + 4];
   __shared__ hct_u32 tmem_holder;
@@ -65,7 +73,7 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
     }
     for (int a = 0; a < 2; ++a) {
       hct_mbar_init(tfull0 + 8 * a, 1);
-      hct_mbar_init(tempty0 + 8 * a, 128);
+      hct_mbar_init(tempty0 + 8 * a, 32 * HCT_EPI_WARPS);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     hct_prefetch_tmap(&hct_p.tmap[0]);
@@ -192,17 +200,20 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
 #else
-      float sum[HCT_BN];
+      // this warp's share of the columns: NCW chunks of 32 starting at chunk c0
+      constexpr int NCW = HCT_BN / 32 / (HCT_EPI_WARPS / 4);
+      const int c0 = ((warp - 2) >> 2) * NCW;
+      float sum[NCW * 32];
 #pragma unroll
-      for (int j = 0; j < HCT_BN; ++j) sum[j] = 0.0f;
+      for (int j = 0; j < NCW * 32; ++j) sum[j] = 0.0f;
 #pragma unroll 1
       for (int ch = 0; ch < HCT_NCH; ++ch) {
         hct_mbar_wait(tfull0 + 8 * acc, acc_phase, &failed, status, 4);
         hct_tc_fence_after();
 #pragma unroll
-        for (int c = 0; c < HCT_BN / 32; ++c) {
+        for (int c = 0; c < NCW; ++c) {
           float v[32];
-          hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * HCT_BN + c * 32, v);
+          hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * HCT_BN + (c0 + c) * 32, v);
 #pragma unroll
           for (int j = 0; j < 32; ++j) sum[c * 32 + j] += v[j];
         }
@@ -212,8 +223,8 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
         if (acc == 0) acc_phase ^= 1u;
       }
 #pragma unroll
-      for (int c = 0; c < HCT_BN / 32; ++c) {
-        const long long col0 = (long long)nb * HCT_BN + c * 32;
+      for (int c = 0; c < NCW; ++c) {
+        const long long col0 = (long long)nb * HCT_BN + (c0 + c) * 32;
         const int ncols = (int)(HCT_N - col0 < 32 ? HCT_N - col0 : 32);
         if (row < HCT_M && ncols > 0) hct_epilogue_run(hct_p, *(float(*)[32])(sum + c * 32), row, (int)col0, ncols);
       }

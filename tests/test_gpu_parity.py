@@ -119,6 +119,29 @@ def test_gemm_f32_shapes(m, k, n):
     check_f32(spec, laws)
 
 
+@pytest.mark.parametrize("m,k,n", [(300, 1000, 520), (257, 4096, 136), (130, 264, 1000), (1024, 260, 300), (64, 36, 257)])
+def test_gemm_f32_wide_tiles(m, k, n):
+    """128 x 256 tiles of the fp32 (three TF32 products) kernel, whose running sums are shared by eight epilogue warps,
+    forced onto small and ragged shapes (by rule they are taken when narrower tiles need more than one round)."""
+    import torch
+    import paper_2506_10401_b200 as hct
+    spec, laws = configs.get_config("c1_gemm_bias_relu_f32", m=m, k=k, n=n)
+    t = configs.draw_inputs(spec, laws, 0)
+    g = hct.FusedGraph(spec, 0, schedule="gemm_bn=256;gemm_pair=2")
+    assert "128x256x32" in g.plan
+    out = g.run(parity.to_device(spec, t))[0]
+    torch.cuda.synchronize()
+    g.status()
+    ref = parity.oracle_reference(spec, parity.oracle_inputs(spec, t))["t2"]
+    assert parity.f32_violation(parity.to_numpy64(out), ref) <= 1.0
+    il = {"kind": "int", "lo": -8, "hi": 8}
+    t = configs.draw_inputs(spec, {"a": il, "b": il, "bias": il}, 1)
+    out = g.run(parity.to_device(spec, t))[0]
+    torch.cuda.synchronize()
+    g.status()
+    np.testing.assert_array_equal(parity.to_numpy64(out), parity.oracle_reference(spec, parity.oracle_inputs(spec, t))["t2"])
+
+
 def test_gemm_f32_integer_inputs_are_exact():
     spec, _ = configs.get_config("c1_gemm_bias_relu_f32", m=96, k=160, n=136)
     il = {"kind": "int", "lo": -8, "hi": 8}
