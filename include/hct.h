@@ -138,7 +138,10 @@ HCT_API hct_status_t hct_graph_create_scheduled(const char* spec, size_t spec_le
  * Measure-and-pick: builds the graph under up to max_trials candidate schedules, runs each on
  * the caller's buffers (same arguments as hct_graph_run; all DEVICE pointers, caller-owned,
  * outputs are overwritten), times it with events on `cuda_stream`, and returns the fastest
- * handle in *out.  This is the role the measurement trials of the auto-scheduler play in the
+ * handle in *out.  Trials run with a cold L2 when the workspace has at least 160 MiB to spare
+ * beyond what the candidates need (that part is overwritten before every run; nothing is
+ * allocated), otherwise warm; a trial is the smallest of three batches of ten runs, and a
+ * candidate replaces the incumbent only when it is at least 2 % faster.  This is the role the measurement trials of the auto-scheduler play in the
  * paper's pipeline (Section 3.5: every candidate is compiled and executed on the device, the
  * best one is kept), restricted to this library's own knobs.  The call SYNCHRONISES the stream
  * repeatedly and is meant for set-up time.  Candidates that need more workspace than
@@ -176,8 +179,11 @@ HCT_API int hct_graph_num_kernels(const hct_graph_t* g);
 /*
  * Work accounting for roofline figures.  algorithmic_bytes: every graph input
  * read once and every output written once, plus one write and one read for
- * each intermediate that no single pass can keep on chip (an edge from a
- * contraction into a row reduction, or from any node into a contraction).
+ * each intermediate that no single pass can keep on chip: a value that
+ * depends on a reduction (row reduction or contraction) and feeds a
+ * contraction or transposition, and a contraction's result that feeds a row
+ * reduction over rows wider than 512 columns.  Elementwise producers of a
+ * contraction, sorts and reshapes are free.
  * flops: 2·M·N·K summed over the contractions.
  */
 HCT_API hct_status_t hct_graph_cost(const hct_graph_t* g, double* algorithmic_bytes, double* flops);

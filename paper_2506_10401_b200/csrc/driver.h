@@ -65,6 +65,7 @@ struct Driver {
   CUresult_t (*MemFree)(CUdeviceptr_t);
   CUresult_t (*MemcpyDtoH)(void*, CUdeviceptr_t, size_t);
   CUresult_t (*MemsetD8)(CUdeviceptr_t, unsigned char, size_t);
+  CUresult_t (*MemsetD8Async)(CUdeviceptr_t, unsigned char, size_t, CUstream_t);
   CUresult_t (*EventCreate)(CUevent_t*, unsigned);
   CUresult_t (*EventRecord)(CUevent_t, CUstream_t);
   CUresult_t (*EventSynchronize)(CUevent_t);

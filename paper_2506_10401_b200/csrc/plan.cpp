@@ -217,15 +217,21 @@ Plan make_plan(const Graph& g) {
       p.flops += 2.0 * nd.numel() * w[1] * w[2] * w[3];
     }
     if (p.ws_offset[i] < 0) continue;
-    // an intermediate no single pass could keep on chip: contraction -> row group (row wider than one
-    // accumulator tile), or anything -> contraction operand
+    // An intermediate counts (one write, one read) only where no single pass could keep it on chip:
+    //  * a value that depends on a reduction (a row reduction of its group, or a contraction) and feeds a
+    //    contraction or a transposition: every element of the operand needs the whole reduction first;
+    //  * a contraction's result that feeds a row reduction over rows wider than one accumulator tile (512 columns).
+    // Elementwise producers of a contraction could be applied while the operand is loaded, a sort is local to
+    // its row, and a reshape moves no data: those edges are free.
     bool unavoidable = false;
+    const Group& pg = p.groups[p.group_of[i]];
+    const bool after_reduction = pg.kind == GroupKind::Gemm || pg.kind == GroupKind::Conv || (pg.kind == GroupKind::Row && pg.has_reduction);
     for (int j = 0; j < n; ++j)
       for (auto& a : g.nodes[j].args) {
         if (a.is_literal() || a.node != i || p.group_of[j] == p.group_of[i]) continue;
-        bool into_contraction = g.nodes[j].cls == OpClass::Gemm || g.nodes[j].cls == OpClass::Conv || g.nodes[j].cls == OpClass::Transpose ||
-                                g.nodes[j].cls == OpClass::Sort || g.nodes[j].cls == OpClass::Reshape;
-        bool from_contraction = p.groups[p.group_of[i]].kind != GroupKind::Row && p.groups[p.group_of[j]].has_reduction &&
+        bool into_contraction = (g.nodes[j].cls == OpClass::Gemm || g.nodes[j].cls == OpClass::Conv || g.nodes[j].cls == OpClass::Transpose) &&
+                                after_reduction;
+        bool from_contraction = (pg.kind == GroupKind::Gemm || pg.kind == GroupKind::Conv) && p.groups[p.group_of[j]].has_reduction &&
                                 nd.shape.back() > 512;
         unavoidable = unavoidable || into_contraction || from_contraction;
       }

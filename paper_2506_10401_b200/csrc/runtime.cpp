@@ -133,6 +133,7 @@ const Driver& driver() {
     HCT_SYM(MemFree, "cuMemFree_v2")
     HCT_SYM(MemcpyDtoH, "cuMemcpyDtoH_v2")
     HCT_SYM(MemsetD8, "cuMemsetD8_v2")
+    HCT_SYM(MemsetD8Async, "cuMemsetD8Async")
     HCT_SYM(EventCreate, "cuEventCreate")
     HCT_SYM(EventRecord, "cuEventRecord")
     HCT_SYM(EventSynchronize, "cuEventSynchronize")

@@ -25,7 +25,8 @@ class FusedGraph:
         import torch
         probe = cls(spec, device)
         outs = probe.alloc_outputs()
-        ws_bytes = workspace_bytes if workspace_bytes is not None else 2 * probe.workspace_bytes + (64 << 20)
+        # room for every candidate's scratch plus the 160 MB the trials overwrite between runs to evict L2
+        ws_bytes = workspace_bytes if workspace_bytes is not None else 2 * probe.workspace_bytes + (64 << 20) + (160 << 20)
         ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device=f"cuda:{device}")
         ws_ptr = (ws.data_ptr() + 255) // 256 * 256
         stream = torch.cuda.current_stream(device).cuda_stream
