@@ -25,7 +25,7 @@
  *           cast_bf16(x)   rounds to bfloat16 (nearest even); the result may be the first operand of a bf16
  *           gemm / conv2d and is kept as bf16 where it is materialised between kernels
  *           dropout(x, p=0.5, seed=0)   inverted dropout with the counter-based mask of the
- *           paper's first case study (Section 5.4): with i the element's row-major offset,
+ *           paper's first case study (Section 5.3, "Detailed Case Study"): with i the element's row-major offset,
  *           h = i + seed; h ^= h >> 17; h ^= h << 31; h ^= h >> 8 (unsigned 64 bit); the
  *           element is kept and scaled by 1/(1-p) when h mod 1000 >= round(1000 p), else 0
  *   binary  add sub mul div max min   operands broadcast like numpy; supported
@@ -111,8 +111,9 @@ HCT_API hct_status_t hct_graph_create(const char* spec, size_t spec_len, int dev
 
 /*
  * Launch the graph's kernels, in dependency order, on `cuda_stream`
- * (a cudaStream_t / CUstream; NULL is the default stream).  Does not
- * synchronise.
+ * (a cudaStream_t / CUstream; NULL is the default stream).  This is the step
+ * the paper's pipeline repeats for every candidate (Section 3.5: compile, then
+ * execute on the device and time).  Does not synchronise.
  *   inputs[i]   device pointer to the i-th `input` line's tensor (read only)
  *   outputs[i]  device pointer to the i-th `output` line's tensor (written)
  *   workspace   device scratch of at least hct_graph_workspace_bytes() bytes,
@@ -157,16 +158,19 @@ HCT_API hct_status_t hct_graph_autotune(const char* spec, size_t spec_len, int d
 HCT_API const char* hct_graph_schedule(const hct_graph_t* g);
 
 /*
- * After the caller has synchronised the stream: reads the handle's device
+ * The "execute" phase's error report (paper Section 3.6: a candidate that loads and compiles may
+ * still fail when it runs).  After the caller has synchronised the stream: reads the handle's device
  * status word.  HCT_OK, or HCT_ERR_TIMEOUT if a kernel gave up on a bounded
  * wait (its outputs are then undefined).  Clears the word.
  */
 HCT_API hct_status_t hct_graph_status(hct_graph_t* g);
 
-/* Release the handle and everything it owns.  NULL is accepted. */
+/* Release the handle and everything it owns: modules, the status word, host state (Section 3.5: a compiled
+ * candidate is discarded after its measurement).  NULL is accepted. */
 HCT_API hct_status_t hct_graph_destroy(hct_graph_t* g);
 
-/* ---- queries (host only) ---- */
+/* ---- queries (host only): what shape and type inference (Section 3.2: operator types must agree with the
+ * shapes and dtypes of their operands) and the fusion plan (Section 3.5: one schedule per fused graph) decided ---- */
 HCT_API int hct_graph_num_inputs(const hct_graph_t* g);
 HCT_API int hct_graph_num_outputs(const hct_graph_t* g);
 /* Name (owned by g), dtype (HCT_F32/HCT_BF16), rank and extents of an input (is_output = 0)

@@ -61,7 +61,7 @@ def cast_bf16(x):
 
 
 def dropout_keep_mask(shape, seed: int, p: float):
-    """Which elements inverted dropout keeps (the paper's first case study, Section 5.4).
+    """Which elements inverted dropout keeps (the paper's first case study, Section 5.3 "Detailed Case Study").
 
     The generator is counter based: the element at row-major offset ``i`` draws
     ``h = i + seed``, then ``h ^= h >> 17``, ``h ^= h << 31``, ``h ^= h >> 8`` in

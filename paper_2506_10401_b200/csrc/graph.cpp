@@ -4,6 +4,7 @@
 #include "graph.h"
 
 #include <cctype>
+#include <cerrno>
 #include <cstdlib>
 #include <cmath>
 #include <cstdio>
@@ -30,6 +31,7 @@ bool is_binary(const std::string& op) {
 }
 
 namespace {
+constexpr int64_t kMaxElements = (int64_t)1 << 40;
 
 std::string trim(const std::string& s) {
   size_t a = 0, b = s.size();
@@ -71,8 +73,9 @@ bool parse_number(const std::string& s, double* out) {
 bool parse_int(const std::string& s, int64_t* out) {
   if (s.empty()) return false;
   char* end = nullptr;
+  errno = 0;
   long long v = std::strtoll(s.c_str(), &end, 10);
-  if (end != s.c_str() + s.size()) return false;
+  if (end != s.c_str() + s.size() || errno == ERANGE) return false;   // not a number, or not representable
   *out = v;
   return true;
 }
@@ -176,6 +179,13 @@ Graph parse_spec(const std::string& text) {
         n.shape.push_back(d);
       }
       if (n.shape.empty() || n.shape.size() > 4) fail(HCT_ERR_PARSE, line, "rank must be 1..4");
+      {  // tensors are capped at 2^40 elements, so that element counts, byte counts and workspace offsets stay far inside int64
+        int64_t count = 1;
+        for (int64_t d : n.shape) {
+          if (d > kMaxElements || (d > 0 && count > kMaxElements / d)) fail(HCT_ERR_UNSUPPORTED, line, "tensors of more than 2^40 elements are not supported");
+          count *= d;
+        }
+      }
       n.input_index = (int)g.inputs.size();
       index[name] = (int)g.nodes.size();
       g.inputs.push_back((int)g.nodes.size());

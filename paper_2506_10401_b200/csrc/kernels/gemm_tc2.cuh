@@ -12,7 +12,7 @@
 // Hand-offs.  full[s] lives in the even CTA: its producer announces the bytes of BOTH CTAs' loads,
 // and both CTAs' TMA copies count on it.  empty[s] and tfull[a] exist in both CTAs and are completed
 // by two tcgen05.commit (one per CTA) from the issuing thread.  tempty[a] lives in the even CTA and
-// counts the epilogue threads of both.  No load is multicast.  All waits are bounded.
+// counts the epilogue threads of both.  Every CTA issues its own loads.  All waits are bounded.
 //
 // The fp32 variant (HCT_TF32X3) works on 256 x 256 tiles per pair from the head/tail operands its
 // split pre-pass wrote (B transposed to [N,K]): three TF32 products per k step, at most 128 elements

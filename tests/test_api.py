@@ -171,3 +171,17 @@ def test_schedule_text_selects_launch_shapes_and_rejects_unknown_knobs():
         assert e.value.code == B.HCT_ERR_INVALID_ARG
     B.hct_graph_destroy(a)
     B.hct_graph_destroy(b)
+
+
+def test_extents_out_of_range_are_rejected_not_wrapped():
+    """An extent that does not fit a 64-bit integer, and shapes whose element count would overflow, are errors of
+    the spec (the parser must not wrap them into small numbers and plan a kernel)."""
+    import paper_2506_10401_b200 as hct
+    for dims in ("[99999999999999999999,4]", "[4294967296,4294967296]", "[1099511627777]", "[2097152,1048576,2]"):
+        spec = f"hct 1\ninput x f32 {dims}\nnode y = relu(x)\noutput y\n"
+        with pytest.raises(hct.HctError) as e:
+            hct.hct_graph_create(spec, hct.HCT_DEVICE_NONE)
+        assert e.value.code in (hct.HCT_ERR_PARSE, hct.HCT_ERR_UNSUPPORTED), dims
+    spec = "hct 1\ninput x f32 [8,64]\nnode y = dropout(x, p=0.5, seed=99999999999999999999)\noutput y\n"
+    with pytest.raises(hct.HctError):
+        hct.hct_graph_create(spec, hct.HCT_DEVICE_NONE)
