@@ -42,6 +42,8 @@ WORKLOADS = {
     "transpose_bias_relu": dict(bound="hbm", sample=dict(r=4096)),
     "matmul_dropout_mean_softmax": dict(bound="tensor", sample=dict(m=1024)),
     "conv_block": dict(bound="tensor", sample=dict(n=4)),
+    "conv_s2_bn_relu": dict(bound="tensor", sample=dict(n=4)),
+    "conv_s2_bn_relu_nhwc": dict(bound="tensor", sample=dict(n=4)),
     "dwconv_bn_relu": dict(bound="hbm", sample=dict(n=8)),
     "topk_bias_relu": dict(bound="hbm", sample=dict(r=2048)),
     "mbconv_block": dict(bound="hbm", sample=dict(n=4)),
@@ -248,7 +250,11 @@ def run_gpu(name, steps, warmup, rank, world, device, tune=0, with_e2e=True):
     # phases of consecutive steps overlap (copy-in, compute and copy-out streams, two sets of device
     # buffers): PCIe is full duplex, so step i+1's inputs travel while step i's result returns.
     specs_in = configs.parse_inputs(spec)
-    pinned = [torch.from_numpy(host[n].view(np.int16) if d == "bf16" else host[n]).pin_memory() for n, d, _ in specs_in]
+    layouts = configs.input_layouts(spec)
+    as_host = lambda n, d: torch.from_numpy(host[n].view(np.int16) if d == "bf16" else host[n])
+    # an input declared channels-last is channels-last on the host as well: the copy moves bytes, it does not permute them
+    pinned = [(as_host(n, d).contiguous(memory_format=torch.channels_last) if layouts.get(n) == "nhwc" else as_host(n, d)).pin_memory()
+              for n, d, _ in specs_in]
     dev_in = [[torch.empty_like(t, device=f"cuda:{device}") for t in pinned] for _ in range(2)]
     run_in = [[t.view(torch.bfloat16) if d == "bf16" else t for t, (_, d, _) in zip(buf, specs_in)] for buf in dev_in]
     dev_out = [outs, g.alloc_outputs()]
@@ -485,7 +491,7 @@ def roofline_of(name, r, pk):
 
 
 def dtype_of(name):
-    return "bf16" if ("bf16" in name or name in ("matmul_dropout_mean_softmax", "conv_block", "dwconv_bn_relu", "mbconv_block")) else "f32"
+    return "bf16" if ("bf16" in name or name in ("matmul_dropout_mean_softmax", "conv_block", "dwconv_bn_relu", "mbconv_block", "conv_s2_bn_relu", "conv_s2_bn_relu_nhwc")) else "f32"
 
 
 def sweep_record(steps, warmup, device, out_path, tune):

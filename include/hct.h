@@ -17,7 +17,9 @@
  * Spec text (line oriented, '#' starts a comment):
  *
  *     hct 1
- *     input  NAME DTYPE [d0,d1,...]           DTYPE: f32 | bf16, rank 1..4
+ *     input  NAME DTYPE [d0,d1,...] [nhwc]    DTYPE: f32 | bf16, rank 1..4; `nhwc` after a bf16 [N,C,H,W] shape says
+ *                                             the buffer is channels-last, x[n][h][w][c] (only as conv2d's first
+ *                                             operand: such a convolution needs no layout pass over its activations)
  *     node   NAME = OP(arg, ..., key=value)   args: earlier names or (binary ops) a number
  *     output NAME [DTYPE]                     stored dtype, default f32
  *
@@ -180,6 +182,9 @@ HCT_API hct_status_t hct_graph_tensor_info(const hct_graph_t* g, int is_output, 
 HCT_API size_t hct_graph_workspace_bytes(const hct_graph_t* g);
 /* Number of kernel launches one hct_graph_run issues. */
 HCT_API int hct_graph_num_kernels(const hct_graph_t* g);
+/* Memory layout of input `idx`: 0 = row-major in the declared order of extents (NCHW for rank 4),
+ * 1 = declared `nhwc`: extents are still reported as [N,C,H,W], the buffer holds x[n][h][w][c].  -1: bad index. */
+HCT_API int hct_graph_input_layout(const hct_graph_t* g, int idx);
 /*
  * Work accounting for roofline figures.  algorithmic_bytes: every graph input
  * read once and every output written once, plus one write and one read for

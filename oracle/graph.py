@@ -91,10 +91,12 @@ def parse(text: str) -> Graph:
             continue
         kw = line.split(None, 1)[0]
         if kw == "input":
-            m = re.match(r"^input\s+(\S+)\s+(\S+)\s*\[([^\]]*)\]$", line)
+            m = re.match(r"^input\s+(\S+)\s+(\S+)\s*\[([^\]]*)\]\s*(\S*)$", line)
             if not m:
                 raise SpecError(f"{where}: malformed input")
-            name, dtype, dims = m.groups()
+            name, dtype, dims, layout = m.groups()
+            if layout not in ("", "nchw", "nhwc"):
+                raise SpecError(f"{where}: unknown layout {layout!r}")
             if not _NAME.match(name) or name in g.nodes:
                 raise SpecError(f"{where}: bad or duplicate name {name!r}")
             if dtype not in ("f32", "bf16"):
@@ -105,7 +107,10 @@ def parse(text: str) -> Graph:
                 raise SpecError(f"{where}: malformed shape") from None
             if not 1 <= len(shape) <= 4 or any(d < 0 for d in shape):
                 raise SpecError(f"{where}: rank must be 1..4 and extents non-negative")
-            g.nodes[name] = Node(name, "input", [], {}, shape, dtype)
+            if layout == "nhwc" and (len(shape) != 4 or dtype != "bf16"):
+                raise SpecError(f"{where}: nhwc needs a bf16 input of rank 4")
+            # the layout word only says how the device buffer is ordered; values are always handed over as [N,C,H,W]
+            g.nodes[name] = Node(name, "input", [], {"layout": layout or "nchw"}, shape, dtype)
             g.inputs.append(name)
         elif kw == "node":
             m = re.match(r"^node\s+(\S+)\s*=\s*([A-Za-z_0-9]+)\s*\((.*)\)$", line)
@@ -137,6 +142,11 @@ def parse(text: str) -> Graph:
         raise SpecError("empty spec")
     if not g.outputs:
         raise SpecError("no output")
+    # a channels-last input may only be the activation operand of a convolution
+    for node in g.nodes.values():
+        for pos, a in enumerate(node.args):
+            if isinstance(a, str) and g.nodes[a].attrs.get("layout") == "nhwc" and not (node.op == "conv2d" and pos == 0):
+                raise SpecError(f"input {a!r} is declared nhwc and may only be the first operand of conv2d")
     # every node and every input must reach an output (no dangling nodes)
     live = set()
     stack = [o for o, _ in g.outputs]

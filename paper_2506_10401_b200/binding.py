@@ -18,6 +18,7 @@ EXPORTS = [
     "hct_graph_num_outputs", "hct_graph_tensor_info", "hct_graph_workspace_bytes", "hct_graph_num_kernels",
     "hct_graph_cost", "hct_graph_plan_text", "hct_graph_kernel_source", "hct_graph_kernel_name", "hct_last_error",
     "hct_version", "hct_gemm_bias_relu_f32_static", "hct_graph_create_scheduled", "hct_graph_autotune", "hct_graph_schedule",
+    "hct_graph_input_layout",
 ]
 
 HCT_STATIC_SCRATCH_BYTES = 8 << 20
@@ -58,6 +59,8 @@ def lib() -> ctypes.CDLL:
         L.hct_graph_tensor_info.restype = ci
         L.hct_graph_workspace_bytes.argtypes = [vp]
         L.hct_graph_workspace_bytes.restype = sz
+        L.hct_graph_input_layout.argtypes = [vp, ci]
+        L.hct_graph_input_layout.restype = ci
         L.hct_graph_num_kernels.argtypes = [vp]
         L.hct_graph_num_kernels.restype = ci
         L.hct_graph_cost.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
@@ -157,6 +160,10 @@ def hct_graph_tensor_info(g, is_output: bool, idx: int):
 
 def hct_graph_workspace_bytes(g) -> int:
     return lib().hct_graph_workspace_bytes(g)
+
+
+def hct_graph_input_layout(g, idx: int) -> int:
+    return lib().hct_graph_input_layout(g, idx)
 
 
 def hct_graph_num_kernels(g) -> int:

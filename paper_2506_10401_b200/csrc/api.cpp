@@ -459,6 +459,10 @@ hct_status_t hct_graph_tensor_info(const hct_graph_t* g, int is_output, int idx,
 
 size_t hct_graph_workspace_bytes(const hct_graph_t* g) { return g ? g->workspace_bytes : 0; }
 int hct_graph_num_kernels(const hct_graph_t* g) { return g ? (int)g->kernels.size() : -1; }
+int hct_graph_input_layout(const hct_graph_t* g, int idx) {
+  if (!g || idx < 0 || idx >= (int)g->graph.inputs.size()) return -1;
+  return g->graph.nodes[g->graph.inputs[idx]].nhwc ? 1 : 0;
+}
 
 hct_status_t hct_graph_cost(const hct_graph_t* g, double* algorithmic_bytes, double* flops) {
   if (!g) return set_error(HCT_ERR_INVALID_ARG, "graph is NULL");

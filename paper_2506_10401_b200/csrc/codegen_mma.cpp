@@ -624,7 +624,8 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       // The epilogue of the NCHW-reading kernel hands its bf16 output to TMA stores (through 16 KB of
       // shared memory) when it stores a single bf16 tensor (output or intermediate) whose rows are 16-byte multiples.
       const bool tma_store = grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && WO % 8 == 0 && !tun.conv_no_tma_store;
-      if (unit && dense_pitch && W % 8 == 0 && !tun.conv_no_direct) {
+      const bool x_nhwc = a.nhwc;   // the activations already are channels-last: no layout pass, and no NCHW-reading schedule
+      if (unit && dense_pitch && W % 8 == 0 && !tun.conv_no_direct && !x_nhwc) {
         // shared memory: operand buffers of TH + FR - 1 rows, staging ring, output staging, and what is left for the weight ring
         const int64_t fixed = n_buf * ((th_pitch + FR - 1) * pitch * 128 + 1024) + n_stg * pitch * 128 + 1024 + (tma_store ? 16384 : 0);
         n_a = (int)std::min<int64_t>(6, (232448 - 512 - fixed) / 16384);
@@ -649,7 +650,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       const bool halo = unit && !direct && FS > 1 && dense_pitch && !tun.conv_no_halo;
       const int TH = (direct || halo) ? th_pitch : (int)std::max<int64_t>(1, std::min<int64_t>(256 / WO, std::min<int64_t>(HO, phased ? 256 : 256 / ST)));
       auto align256 = [](int64_t v) { return (v + 255) / 256 * 256; };
-      const int64_t x_bytes = direct ? 0 : align256(NB * C * H * W * 2), w_bytes = align256(KO * C * FR * FS * 2);
+      const int64_t x_bytes = (direct || x_nhwc) ? 0 : align256(NB * C * H * W * 2), w_bytes = align256(KO * C * FR * FS * 2);
       *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(x_bytes + w_bytes));
       auto scratch = [](int64_t off) {
         BufRef r;
@@ -668,14 +669,15 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         k.name = "hct_conv_prep_g" + std::to_string(gi);
         std::ostringstream src;
         src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_HW " << H * W << "\n#define HCT_KO " << KO
-            << "\n#define HCT_RS " << FR * FS << "\n#define HCT_PREP_X " << (direct ? 0 : 1) << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+            << "\n#define HCT_RS " << FR * FS << "\n#define HCT_PREP_X " << ((direct || x_nhwc) ? 0 : 1) << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
             << skeleton_source("common") << "\nstruct HctParams { void* ptr[4]; };\n" << skeleton_source("conv_prep");
         k.source = src.str();
         k.ptrs = {node_buf(anchor.args[0].node), node_buf(anchor.args[1].node), scratch(0), scratch(x_bytes)};
-        int64_t blocks = direct ? (KO * C * FR * FS / 8 + 255) / 256 : NB * ((C + 63) / 64) * ((H * W + 63) / 64) + (KO * C * FR * FS + 255) / 256;
-        k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(blocks, direct ? 148 : 148 * 16));
+        const bool w_only = direct || x_nhwc;
+        int64_t blocks = w_only ? (KO * C * FR * FS / 8 + 255) / 256 : NB * ((C + 63) / 64) * ((H * W + 63) / 64) + (KO * C * FR * FS + 255) / 256;
+        k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(blocks, w_only ? 148 : 148 * 16));
         k.block[0] = 256;
-        k.desc = direct ? "conv weight pre-pass: KCRS->RSKC" : "conv layout pre-pass: NCHW->NHWC activations, KCRS->RSKC weights";
+        k.desc = w_only ? "conv weight pre-pass: KCRS->RSKC" : "conv layout pre-pass: NCHW->NHWC activations, KCRS->RSKC weights";
         out->push_back(k);
       }
       int stages = 4;
@@ -705,7 +707,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       tw.strides[1] = (uint64_t)C * 2;
       tw.box[0] = 64; tw.box[1] = 128;
       TmaDesc tx;
-      tx.buf = scratch(0);
+      tx.buf = x_nhwc ? node_buf(anchor.args[0].node) : scratch(0);
       tx.elem_bytes = 2;
       tx.rank = 4;
       tx.dims[0] = (uint64_t)C; tx.dims[1] = (uint64_t)W; tx.dims[2] = (uint64_t)H; tx.dims[3] = (uint64_t)NB;
@@ -721,7 +723,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         for (int piece = 0; piece < 2; ++piece)
           for (int64_t ph = 0; ph < ST; ++ph) {
             TmaDesc tp;
-            tp.buf = scratch(0);
+            tp.buf = x_nhwc ? node_buf(anchor.args[0].node) : scratch(0);
             tp.base_offset = (uint64_t)(ph * W * C * 2);
             tp.elem_bytes = 2;
             tp.rank = 5;
@@ -771,15 +773,18 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       else if (direct)
         d << "NCHW read directly and re-laid in shared memory, every pixel loaded once per tile (pitch " << pitch << ")";
       else if (halo)
-        d << "pixels shared by the taps of a filter row (pitch " << pitch << ")";
+        d << "pixels shared by the taps of a filter row (pitch " << pitch << ")" << (x_nhwc ? ", channels-last input read in place" : "");
       else
-        d << stages << " stages" << (unit ? "" : phased ? ", dense pixel boxes of a stride-phase view" : ", strided pixel boxes");
+        d << stages << " stages" << (unit ? "" : phased ? ", dense pixel boxes of a stride-phase view" : ", strided pixel boxes")
+          << (x_nhwc ? ", channels-last input read in place" : "");
       k.desc = d.str();
       out->push_back(k);
       return;
     }
   }
 
+  if (grp.kind == GroupKind::Conv && a.nhwc)
+    throw Error(HCT_ERR_UNSUPPORTED, "a channels-last (nhwc) input needs the tensor-core convolution: bf16 operands, groups = 1, channels a multiple of 8, stride <= 8");
   auto operand_buf = [&](int node) {
     return eg.ptr_index(node, g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0);
   };

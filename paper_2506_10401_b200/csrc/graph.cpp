@@ -172,6 +172,17 @@ Graph parse_spec(const std::string& text) {
         n.dtype = BF16;
       else
         fail(HCT_ERR_PARSE, line, "unknown dtype '" + dtype + "'");
+      {  // optional layout word after the shape
+        size_t rb = rest.find(']');
+        if (rb != std::string::npos && rb + 1 < rest.size()) {
+          std::string layout = trim(rest.substr(rb + 1));
+          rest = rest.substr(0, rb + 1);
+          if (layout == "nhwc")
+            n.nhwc = true;
+          else if (layout != "nchw")
+            fail(HCT_ERR_PARSE, line, "unknown layout '" + layout + "' (nchw or nhwc)");
+        }
+      }
       if (rest.size() < 2 || rest.front() != '[' || rest.back() != ']') fail(HCT_ERR_PARSE, line, "malformed shape");
       for (auto& t : split(rest.substr(1, rest.size() - 2), ',')) {
         int64_t d;
@@ -179,6 +190,7 @@ Graph parse_spec(const std::string& text) {
         n.shape.push_back(d);
       }
       if (n.shape.empty() || n.shape.size() > 4) fail(HCT_ERR_PARSE, line, "rank must be 1..4");
+      if (n.nhwc && (n.shape.size() != 4 || n.dtype != BF16)) fail(HCT_ERR_UNSUPPORTED, line, "the nhwc layout is supported for bf16 inputs of rank 4");
       {  // tensors are capped at 2^40 elements, so that element counts, byte counts and workspace offsets stay far inside int64
         int64_t count = 1;
         for (int64_t d : n.shape) {
@@ -408,6 +420,14 @@ Graph parse_spec(const std::string& text) {
   }
   if (!header) throw Error(HCT_ERR_PARSE, "empty spec");
   if (g.outputs.empty()) throw Error(HCT_ERR_GRAPH, "the graph has no output");
+  // a channels-last input is an activation tensor for convolutions: nothing else reads that layout
+  for (const Node& nd : g.nodes)
+    for (size_t ai = 0; ai < nd.args.size(); ++ai) {
+      const Operand& a = nd.args[ai];
+      if (a.is_literal() || !g.nodes[a.node].nhwc) continue;
+      if (!(nd.cls == OpClass::Conv && ai == 0))
+        throw Error(HCT_ERR_UNSUPPORTED, "input '" + g.nodes[a.node].name + "' is declared nhwc and may only be the first operand of conv2d");
+    }
 
   // No dangling nodes: everything must reach an output.
   std::vector<char> live(g.nodes.size(), 0);

@@ -15,6 +15,7 @@ class FusedGraph:
         self.n_out = B.hct_graph_num_outputs(self.handle)
         self.inputs = [B.hct_graph_tensor_info(self.handle, False, i) for i in range(self.n_in)]
         self.outputs = [B.hct_graph_tensor_info(self.handle, True, i) for i in range(self.n_out)]
+        self.input_nhwc = [B.hct_graph_input_layout(self.handle, i) == 1 for i in range(self.n_in)]
         self.workspace_bytes = B.hct_graph_workspace_bytes(self.handle)
         self._ws = None
 
@@ -73,10 +74,12 @@ class FusedGraph:
         import torch
         if outputs is None:
             outputs = self.alloc_outputs()
-        for t, (name, dtype, shape) in zip(inputs, self.inputs):
+        for t, (name, dtype, shape), nhwc in zip(inputs, self.inputs, self.input_nhwc):
             want = torch.bfloat16 if dtype == B.HCT_BF16 else torch.float32
-            if tuple(t.shape) != tuple(shape) or t.dtype != want or not t.is_contiguous() or not t.is_cuda:
-                raise ValueError(f"input {name}: expected contiguous CUDA {want} tensor of shape {shape}")
+            # an input declared nhwc is passed as a [N,C,H,W] tensor in torch's channels-last memory format
+            dense = t.is_contiguous(memory_format=torch.channels_last) if nhwc else t.is_contiguous()
+            if tuple(t.shape) != tuple(shape) or t.dtype != want or not dense or not t.is_cuda:
+                raise ValueError(f"input {name}: expected {'channels-last' if nhwc else 'contiguous'} CUDA {want} tensor of shape {shape}")
         ws = self.workspace()
         ws_ptr = 0
         if ws is not None:

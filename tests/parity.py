@@ -61,12 +61,16 @@ def oracle_reference(spec, inputs64):
 def to_device(spec, tensors_by_name, device="cuda:0"):
     import torch
     out = []
+    layouts = configs.input_layouts(spec)
     for n, d, _ in configs.parse_inputs(spec):
         a = tensors_by_name[n]
         if d == "bf16":
-            out.append(torch.from_numpy(a.view(np.int16)).to(device).view(torch.bfloat16))
+            t = torch.from_numpy(a.view(np.int16)).to(device).view(torch.bfloat16)
         else:
-            out.append(torch.from_numpy(a).to(device))
+            t = torch.from_numpy(a).to(device)
+        if layouts.get(n) == "nhwc":      # same values, channels-last in memory
+            t = t.contiguous(memory_format=torch.channels_last)
+        out.append(t)
     return out
 
 

@@ -277,6 +277,32 @@ def test_conv_flat_tiles(kw):
     np.testing.assert_array_equal(got[0], want[0])
 
 
+@pytest.mark.parametrize("shape,wshape,attrs", [
+    ((2, 64, 28, 30), (96, 64, 3, 3), "stride=2, pad=1"),             # strided pixel boxes straight from the caller's buffer
+    ((1, 128, 56, 56), (256, 128, 1, 1), "stride=2, pad=0"),
+    ((2, 64, 20, 24), (96, 64, 3, 3), "stride=1, pad=1"),             # stride 1: pixels shared by the taps of a filter row
+    ((1, 72, 17, 40), (130, 72, 5, 5), "stride=1, pad=2"),
+    ((3, 8, 9, 11), (32, 8, 3, 3), "stride=1, pad=1"),                # small image: one box per tap
+    ((1, 8, 6, 300), (8, 8, 3, 3), "stride=2, pad=1"),                # stride-phase view of the caller's buffer
+    ((1, 8, 16, 32), (16, 8, 3, 3), "stride=4, pad=1, dilation=3"),
+])
+def test_conv_channels_last_input_is_read_in_place(shape, wshape, attrs):
+    """An input declared nhwc: same values as the NCHW graph, channels-last in memory; the convolution reads the
+    caller's buffer through its tensor maps and the only pre-pass left is the one over the weights."""
+    dims = lambda t: "[" + ",".join(str(v) for v in t) + "]"
+    spec = f"hct 1\ninput x bf16 {dims(shape)} nhwc\ninput w bf16 {dims(wshape)}\nnode y = conv2d(x, w, {attrs})\noutput y f32\n"
+    il = {"kind": "int", "lo": -4, "hi": 4}
+    got, want, g = parity.run_both(spec, {"x": il, "w": il})
+    assert "channels-last input read in place" in g.plan and "weight pre-pass" in g.plan and "NHWC activations" not in g.plan
+    assert g.workspace_bytes <= 256 + 2 * int(np.prod(wshape))
+    np.testing.assert_array_equal(got[0], want[0])
+
+
+def test_conv_channels_last_chain():
+    spec, laws = configs.get_config("c4_conv_bn_relu_bf16", n=2, c=64, h=56, w=56, k=128, stride=2, pad=1, nhwc=True)
+    check_bf16(spec, laws)
+
+
 def test_conv_f32_integer_inputs_are_exact():
     spec = "hct 1\ninput x f32 [2,16,10,12]\ninput w f32 [8,16,3,3]\nnode y = conv2d(x, w, stride=1, pad=1)\noutput y\n"
     il = {"kind": "int", "lo": -4, "hi": 4}

@@ -69,9 +69,9 @@ output t3 bf16
     return spec, laws
 
 
-def conv_bn_relu(n=32, c=128, h=56, w=56, k=128, ksize=3, stride=1, pad=1):
+def conv_bn_relu(n=32, c=128, h=56, w=56, k=128, ksize=3, stride=1, pad=1, nhwc=False):
     spec = f"""hct 1
-input x     bf16 [{n},{c},{h},{w}]
+input x     bf16 [{n},{c},{h},{w}]{" nhwc" if nhwc else ""}
 input wt    bf16 [{k},{c},{ksize},{ksize}]
 input scale f32  [{k},1,1]
 input shift f32  [{k},1,1]
@@ -219,6 +219,9 @@ CONFIGS = {
     "c2_softmax_layernorm_chain": (softmax_layernorm_chain, {}),
     "c3_gemm_bf16_gelu_residual": (gemm_bf16_gelu_residual, {}),
     "c4_conv_bn_relu_bf16": (conv_bn_relu, {}),
+    # a ResNet-style downsampling convolution, [32,128,56,56] -> 256 channels at stride 2, activations NCHW / channels-last
+    "conv_s2_bn_relu": (conv_bn_relu, dict(k=256, stride=2)),
+    "conv_s2_bn_relu_nhwc": (conv_bn_relu, dict(k=256, stride=2, nhwc=True)),
     "matmul_dropout_mean_softmax": (matmul_dropout_mean_softmax, {}),
     "transpose_bias_relu": (transpose_bias_relu, {}),
     "conv_block": (conv_block, {}),
@@ -235,8 +238,19 @@ def parse_inputs(spec: str):
         line = line.split("#", 1)[0].strip()
         if line.startswith("input"):
             _, name, dtype, shape = line.split(None, 3)
+            shape = shape[:shape.index("]") + 1]
             dims = tuple(int(t) for t in shape.strip()[1:-1].split(",") if t.strip())
             out.append((name, dtype, dims))
+    return out
+
+
+def input_layouts(spec: str):
+    """name -> "nhwc" for the inputs declared channels-last.  Text handling only."""
+    out = {}
+    for line in spec.splitlines():
+        line = line.split("#", 1)[0].strip()
+        if line.startswith("input") and line.endswith("nhwc"):
+            out[line.split()[1]] = "nhwc"
     return out
 
 
