@@ -37,6 +37,8 @@
  *           row_argmax(x)  row_argmin(x)   column of the extreme element, the first among equals, as an fp32 value
  *           (row_softmax also accepts a single column, where it is identically one)
  *           row_layernorm(x, gamma, beta, eps=1e-5)   biased variance, eps inside the root
+ *   row_argsort(x, descending=0)  row_topk_indices(x, k=K)   the columns the values of row_sort / row_topk came
+ *                         from, as fp32 values; among equal values (-0 and +0 are equal) the smaller column first
  *   transpose(x)          y[j,i] = x[i,j] for x[R,C]; elementwise consumers are applied at the store
  *   reshape(x, rows=R, cols=C)   the elements of x (any rank) in row-major order as [R,C], R*C = numel(x);
  *                         a bf16 value stays bf16; one copy pass, elementwise consumers applied at the store

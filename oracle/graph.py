@@ -254,18 +254,18 @@ def _infer(g, name, op, pos, attrs, where):
         if rows < 1 or cols < 1 or rows * cols != n:
             raise SpecError(f"{where}: reshape of {s} must keep the number of elements")
         return Node(name, op, [a], {"rows": rows, "cols": cols}, (rows, cols), g.nodes[a].dtype)
-    if op in ("row_sort", "row_topk"):
-        only_attrs("k") if op == "row_topk" else only_attrs("descending")
+    if op in ("row_sort", "row_topk", "row_argsort", "row_topk_indices"):
+        only_attrs("k") if op.startswith("row_topk") else only_attrs("descending")
         if len(pos) != 1:
             raise SpecError(f"{where}: {op} takes one operand")
         a = _operand(g, pos[0], where, False)
         s = shape_of(a)
         if len(s) != 2:
             raise SpecError(f"{where}: {op} needs a [R,C] operand")
-        if op == "row_topk":
+        if op.startswith("row_topk"):
             k = _int_attr(attrs, "k", 1, where)
             if k < 1 or k > s[1]:
-                raise SpecError(f"{where}: row_topk needs 1 <= k <= C")
+                raise SpecError(f"{where}: {op} needs 1 <= k <= C")
             return Node(name, op, [a], {"k": k}, (s[0], k), "f32")
         return Node(name, op, [a], {"descending": _int_attr(attrs, "descending", 0, where)}, s, "f32")
     if op == "transpose":

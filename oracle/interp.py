@@ -118,6 +118,22 @@ def row_topk(x, k):
     return row_sort(x, descending=True)[:, :k].copy()
 
 
+def row_argsort(x, descending=False):
+    # y[i, j] = column of the j-th value of row i in non-decreasing (non-increasing) order; among equal
+    # values the smaller column comes first in both directions (-0 and +0 are equal).  Returned as floats.
+    r, c = x.shape
+    y = np.empty((r, c), dtype=np.float64)
+    for i in range(r):
+        cols = sorted(range(c), key=lambda j: ((-x[i, j] if descending else x[i, j]) + 0.0, j))
+        y[i, :] = cols
+    return y
+
+
+def row_topk_indices(x, k):
+    # columns of the k largest values of every row, largest first, smaller column first among equal values
+    return row_argsort(x, descending=True)[:, :k].copy()
+
+
 # ---- layout transform (Table 1, "LayoutTransform") ------------------------------------------
 
 def transpose(x):
@@ -235,6 +251,10 @@ def run_nodes(spec, inputs: dict, dtype=np.float64, gemm_fn=None) -> dict:
             out = row_sort(args[0], bool(node.attrs["descending"]))
         elif op == "row_topk":
             out = row_topk(args[0], node.attrs["k"])
+        elif op == "row_argsort":
+            out = row_argsort(args[0], bool(node.attrs["descending"]))
+        elif op == "row_topk_indices":
+            out = row_topk_indices(args[0], node.attrs["k"])
         elif op == "transpose":
             out = transpose(args[0])
         elif op == "row_softmax":

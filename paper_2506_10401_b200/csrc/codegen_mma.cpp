@@ -247,6 +247,26 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     const int pa = eg.ptr_index(src, g.nodes[src].cls != OpClass::Input && p.ws_offset[src] >= 0);
     const DType ta = eg.buf_dtype(src);
     std::string epi = eg.scalar_fn();
+    if (anchor.sort_indices) {
+      // columns instead of values: 64-bit (value, column) keys through the same network, 8 bytes of shared memory per slot
+      KernelSpec k;
+      k.name = "hct_row_argsort_g" + std::to_string(gi);
+      std::ostringstream st;
+      st << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "\n#define HCT_NP " << NP << "\n#define HCT_KOUT " << KOUT
+         << "\n#define HCT_DESC " << (anchor.descending ? 1 : 0) << "\n#define HCT_T " << T << "\n#define HCT_TA " << ctype(ta)
+         << "\n#define HCT_PA " << pa << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+         << skeleton_source("common") << "\nstruct HctParams { void* ptr[" << eg.ptrs.size() << "]; };\n" << epi << skeleton_source("row_argsort");
+      k.source = st.str();
+      k.ptrs = eg.ptrs;
+      k.smem_bytes = (unsigned)(8 * NP);
+      const int64_t per_sm = std::max<int64_t>(1, std::min<int64_t>(2048 / T, std::min<int64_t>(16, (200 * 1024) / (8 * NP))));
+      k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(R, 148 * per_sm));
+      k.block[0] = (unsigned)T;
+      k.desc = std::string(anchor.sort_k ? "row top-k indices" : "row argsort") + ": bitonic network over " + std::to_string(NP) +
+               " 64-bit (value, column) keys in shared memory, one CTA per row";
+      out->push_back(k);
+      return;
+    }
     if (anchor.sort_k > 0 && anchor.sort_k <= 256 && C >= 2 && !tun.topk_no_select) {
       // small k: radix selection of the k-th largest key, then a sort of the k selected values only
       int64_t KP = 2;

@@ -344,9 +344,11 @@ Graph parse_spec(const std::string& text) {
         if (rows * cols != src.numel()) fail(HCT_ERR_GRAPH, line, "reshape of " + shape_str(src.shape) + " must keep the number of elements");
         n.shape = {rows, cols};
         n.dtype = src.dtype;   // values are moved unchanged, so a bf16 value stays bf16
-      } else if (op == "row_sort" || op == "row_topk") {
-        // logic-intensive operators (Table 1): the values of every row in order; row_topk keeps the k largest, largest first
-        const bool topk = op == "row_topk";
+      } else if (op == "row_sort" || op == "row_topk" || op == "row_argsort" || op == "row_topk_indices") {
+        // logic-intensive operators (Table 1): the values of every row in order; row_topk keeps the k largest, largest first;
+        // row_argsort / row_topk_indices deliver the columns those values came from (the smaller column first among equals)
+        const bool topk = op == "row_topk" || op == "row_topk_indices";
+        n.sort_indices = op == "row_argsort" || op == "row_topk_indices";
         if (topk) only_attrs({"k"}); else only_attrs({"descending"});
         if (pos.size() != 1) fail(HCT_ERR_GRAPH, line, op + " takes one operand");
         n.cls = OpClass::Sort;
@@ -356,7 +358,7 @@ Graph parse_spec(const std::string& text) {
         if (s[1] > 8192) fail(HCT_ERR_UNSUPPORTED, line, op + " supports rows of up to 8192 elements");
         n.descending = topk || int_attr("descending", 0) != 0;
         n.sort_k = topk ? int_attr("k", 1) : 0;
-        if (topk && (n.sort_k < 1 || n.sort_k > s[1])) fail(HCT_ERR_GRAPH, line, "row_topk needs 1 <= k <= C");
+        if (topk && (n.sort_k < 1 || n.sort_k > s[1])) fail(HCT_ERR_GRAPH, line, op + " needs 1 <= k <= C");
         n.shape = {s[0], topk ? (int64_t)n.sort_k : s[1]};
       } else if (op == "gemm") {
         only_attrs({"precision"});

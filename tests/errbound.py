@@ -175,7 +175,7 @@ def bound(spec, inputs, values=None):
             e = _sum_rows(av[0], ae[0]) / av[0].shape[1] + U * np.abs(y)
         elif op in ("row_max", "row_min"):
             e = _row_extreme(av[0], ae[0], op == "row_max")
-        elif op in ("row_argmax", "row_argmin"):
+        elif op in ("row_argmax", "row_argmin", "row_argsort", "row_topk_indices"):
             e = np.zeros_like(y)      # an index: compared exactly (tests give these operators exact operands)
         elif op == "row_layernorm":
             e = _layernorm(av[0], av[1], av[2], node.attrs["eps"], y, ae[0], ae[1], ae[2])

@@ -701,6 +701,33 @@ def test_row_topk_radix_selection_moves_values_exactly(rows, cols, k, law):
     np.testing.assert_array_equal(got2[0], want[0])
 
 
+@pytest.mark.parametrize("rows,cols,k", [(5, 1, 1), (7, 2, 2), (33, 5, 3), (64, 100, 100), (40, 1024, 50), (9, 3000, 7), (6, 4096, 4096), (3, 8192, 256)])
+@pytest.mark.parametrize("law", ["normal", "ties"])
+def test_row_argsort_and_topk_indices_are_exact(rows, cols, k, law):
+    """Columns of the ordered values: index work, compared bit for bit; with many equal values (and both zeros) the
+    smaller column must come first in both directions."""
+    spec = (f"hct 1\ninput x f32 [{rows},{cols}]\ninput y bf16 [{rows},{cols}]\nnode a = row_argsort(x)\nnode d = row_argsort(y, descending=1)\n"
+            f"node t = row_topk_indices(x, k={k})\nnode u = add(t, 0.5)\noutput a\noutput d\noutput t\noutput u\n")
+    lw = N_ if law == "normal" else {"kind": "int", "lo": -2, "hi": 2}
+    got, want, g = parity.run_both(spec, {"x": lw, "y": lw})
+    assert g.plan.count("64-bit (value, column) keys") == 3
+    for a, b in zip(got, want):
+        np.testing.assert_array_equal(a, b)
+
+
+def test_row_argsort_treats_both_zeros_as_equal():
+    import torch
+    import oracle
+    import paper_2506_10401_b200 as hct
+    x = np.array([[0.0, -0.0, 1.0, -0.0, 0.0, -1.0, 0.0, -0.0]] * 3, dtype=np.float32)
+    for desc in (0, 1):
+        spec = f"hct 1\ninput x f32 [3,8]\nnode a = row_argsort(x, descending={desc})\noutput a\n"
+        g = hct.FusedGraph(spec, 0)
+        got = g.run([torch.from_numpy(x).cuda()])[0].cpu().numpy().astype(np.float64)
+        g.status()
+        np.testing.assert_array_equal(got, oracle.run(spec, {"x": x.astype(np.float64)})["a"])
+
+
 def test_row_topk_when_one_thread_holds_every_large_value():
     """Large values 256 columns apart all belong to one thread of the top-k kernel, so the bound taken from the
     per-thread maxima admits most of the row and the kernel has to fall back to the radix selection."""

@@ -407,6 +407,36 @@ def test_sort_hand_values_bruteforce_and_invariants():
     assert g.nodes["t"].shape == (4, 3) and g.nodes["s"].shape == (4, 9)
 
 
+def test_argsort_hand_values_bruteforce_and_ties():
+    x = np.array([[3.0, 1.0, 2.0, 5.0, 4.0], [0.0, -1.0, 7.0, 7.0, 2.0], [1.0, 1.0, 1.0, -0.0, 0.0]])
+    # hand values: equal values keep their column order in BOTH directions
+    np.testing.assert_array_equal(interp.row_argsort(x), [[1, 2, 0, 4, 3], [1, 0, 4, 2, 3], [3, 4, 0, 1, 2]])
+    np.testing.assert_array_equal(interp.row_argsort(x, descending=True), [[3, 4, 0, 2, 1], [2, 3, 4, 0, 1], [0, 1, 2, 3, 4]])
+    np.testing.assert_array_equal(interp.row_topk_indices(x, 2), [[3, 4], [2, 3], [0, 1]])
+    y = RNG.integers(-3, 4, size=(6, 29)).astype(np.float64)          # many equal values
+    z = RNG.normal(size=(4, 33))
+    for a in (y, z):
+        for desc in (False, True):
+            idx = interp.row_argsort(a, descending=desc).astype(np.int64)
+            # a permutation of the columns that puts the values in order ...
+            assert all(sorted(idx[i]) == list(range(a.shape[1])) for i in range(a.shape[0]))
+            np.testing.assert_array_equal(np.take_along_axis(a, idx, axis=1), interp.row_sort(a, descending=desc))
+            # ... and, by brute force, each slot takes the first not yet used column holding the wanted value
+            for i in range(a.shape[0]):
+                used, want = set(), []
+                for v in interp.row_sort(a, descending=desc)[i]:
+                    j = next(j for j in range(a.shape[1]) if j not in used and a[i, j] == v)
+                    used.add(j)
+                    want.append(j)
+                assert list(idx[i]) == want
+        np.testing.assert_array_equal(interp.row_argsort(a), np.argsort(a + 0.0, axis=1, kind="stable"))   # library routine
+        for k in (1, 5, a.shape[1]):
+            np.testing.assert_array_equal(interp.row_topk_indices(a, k), interp.row_argsort(a, descending=True)[:, :k])
+            np.testing.assert_array_equal(np.take_along_axis(a, interp.row_topk_indices(a, k).astype(np.int64), axis=1), interp.row_topk(a, k))
+    g = oracle.parse("hct 1\ninput x f32 [4,9]\nnode t = row_topk_indices(x, k=3)\nnode s = row_argsort(x, descending=1)\noutput t\noutput s\n")
+    assert g.nodes["t"].shape == (4, 3) and g.nodes["s"].shape == (4, 9)
+
+
 # ---------------------------------------------------------------- graph validity (paper section 3.2)
 
 GOOD = "hct 1\ninput x f32 [4,8]\ninput b f32 [8]\nnode t = add(x, b)\nnode y = row_softmax(t)\noutput y\n"
@@ -608,6 +638,8 @@ def test_planted_mistakes_are_detected(monkeypatch):
         ("reshape", lambda x, rows, cols: np.ascontiguousarray(x).ravel(order="F").reshape(rows, cols), test_reshape_keeps_row_major_order),
         ("row_sort", lambda x, descending=False: orig["row_sort"](x, not descending), test_sort_hand_values_bruteforce_and_invariants),
         ("row_topk", lambda x, k: orig["row_sort"](x)[:, :k], test_sort_hand_values_bruteforce_and_invariants),
+        ("row_argsort", lambda x, descending=False: np.argsort(-x if descending else x, axis=1).astype(np.float64)[:, ::1] if not descending
+         else np.argsort(x, axis=1, kind="stable")[:, ::-1].astype(np.float64), test_argsort_hand_values_bruteforce_and_ties),
         ("row_layernorm", unbiased_ln, test_layernorm_closed_forms),
         ("row_layernorm", eps_outside_ln, test_layernorm_bruteforce_and_torch),
         ("conv2d", flipped_conv, test_conv_structure_pins),
