@@ -124,7 +124,12 @@ struct EpiGen {
     }
     f << loads.str();
     if (!vals_only)
-      for (auto& st : grp.stores) f << "  float o" << st.node << "_" << (st.to_output ? 1 : 0) << "[32];\n";
+      for (auto& st : grp.stores) {
+        if (p.partial_cols[st.node] > 0 && !st.to_output)
+          f << "  float ps" << st.node << " = 0.0f;\n";   // row sum of this 32-column chunk
+        else
+          f << "  float o" << st.node << "_" << (st.to_output ? 1 : 0) << "[32];\n";
+      }
     f << "  _Pragma(\"unroll\") for (int j = 0; j < 32; ++j) {\n";
     for (size_t i = 1; i < grp.nodes.size(); ++i) {
       const Node& nd = g.nodes[grp.nodes[i]];
@@ -133,9 +138,13 @@ struct EpiGen {
       f << "    const float e" << grp.nodes[i] << " = " << elementwise_call(nd, av, "row * " + std::to_string(N) + "LL + col0 + j") << ";  // "
         << nd.name << "\n";
     }
-    for (auto& st : grp.stores)
-      f << "    " << (vals_only ? std::string("out") : "o" + std::to_string(st.node) + "_" + (st.to_output ? "1" : "0")) << "[j] = "
-        << (st.node == anchor ? "acc[j]" : "e" + std::to_string(st.node)) << ";\n";
+    for (auto& st : grp.stores) {
+      const std::string val = st.node == anchor ? "acc[j]" : "e" + std::to_string(st.node);
+      if (!vals_only && p.partial_cols[st.node] > 0 && !st.to_output)
+        f << "    if (j < ncols) ps" << st.node << " += " << val << ";\n";
+      else
+        f << "    " << (vals_only ? std::string("out") : "o" + std::to_string(st.node) + "_" + (st.to_output ? "1" : "0")) << "[j] = " << val << ";\n";
+    }
     f << "  }\n";
     if (vals_only) {
       f << "}\n";
@@ -143,6 +152,10 @@ struct EpiGen {
     }
     for (auto& st : grp.stores) {
       int pi = ptr_index(st.node, !st.to_output);
+      if (p.partial_cols[st.node] > 0 && !st.to_output) {   // one value per row and chunk; every chunk starts at a multiple of 32 columns
+        f << "  ((float*)hct_p.ptr[" << pi << "])[row * " << p.partial_cols[st.node] << "LL + (col0 >> 5)] = ps" << st.node << ";\n";
+        continue;
+      }
       const int w = part_w(st.dtype);
       if (w)
         f << "  hct_st_run32w<" << w << ">((" << ctype(st.dtype) << "*)hct_p.ptr[" << pi << "] + row * " << N << "LL + col0, o" << st.node << "_"
@@ -805,6 +818,9 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
 
   if (grp.kind == GroupKind::Conv && a.nhwc)
     throw Error(HCT_ERR_UNSUPPORTED, "a channels-last (nhwc) input needs the tensor-core convolution: bf16 operands, groups = 1, channels a multiple of 8, stride <= 8");
+  for (auto& st : grp.stores)
+    if (p.partial_cols[st.node] > 0)
+      throw Error(HCT_ERR_UNSUPPORTED, "row sums folded into a GEMM epilogue need the tensor-core kernel (not available with simt_only)");
   auto operand_buf = [&](int node) {
     return eg.ptr_index(node, g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0);
   };

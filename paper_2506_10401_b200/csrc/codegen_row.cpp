@@ -346,7 +346,8 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         << FORE << "if (HCT_HAS(e)) s" << id << "[b] = " << (is_max ? "fmaxf(s" + id + "[b], " + a + ")" : "s" + id + "[b] + " + a) << ";\n      }\n"
         << "      " << (is_max ? "HCT_RMAX" : "HCT_RSUM") << "(s" << id << ");\n";
       if (!refill_placed) { b << "@REFILL@"; refill_placed = true; }
-      if (nd.op == "row_mean") b << "      " << FORB << "s" << id << "[b] = s" << id << "[b] / (float)HCT_C;\n";
+      if (nd.op == "row_mean")
+        b << "      " << FORB << "s" << id << "[b] = s" << id << "[b] / (float)" << (p.reduce_count[ni] > 0 ? std::to_string(p.reduce_count[ni]) : std::string("HCT_C")) << ";\n";
     } else if (nd.cls == OpClass::RowSoftmax) {
       // One exchange between the warps of a row: every warp takes its exponentials relative to its own
       // maximum (found with shuffles alone), and the per-warp (maximum, sum) pairs are folded afterwards.

@@ -72,11 +72,18 @@ Plan make_plan(const Graph& g) {
   p.group_of.assign(n, -1);
   p.ws_offset.assign(n, -1);
   p.is_colv.assign(n, 0);
+  p.partial_cols.assign(n, 0);
+  p.reduce_count.assign(n, 0);
 
   auto add_ext = [&](Group& grp, int node, int consumer) {
     if (find_ext(grp, node) >= 0) return;
     ExtOperand e;
     e.node = node;
+    if (p.partial_cols[node] > 0) {   // arrives as [R, chunks] partial sums: a full-width operand of the rewritten group
+      e.bcast = Bcast::Full;
+      grp.ext.push_back(e);
+      return;
+    }
     if (!classify(g.nodes[node].shape, grp.full_shape, &e.bcast, &e.lead_stride))
       throw Error(HCT_ERR_UNSUPPORTED, "node '" + g.nodes[consumer].name + "': broadcast pattern of operand '" +
                                            g.nodes[node].name + "' is not supported");
@@ -161,6 +168,47 @@ Plan make_plan(const Graph& g) {
       grp.has_reduction = true;
   }
 
+  // Row sums folded into a contraction's epilogue (the paper's first case study: matrix product, dropout, mean,
+  // softmax in one fused group).  When a value of a bf16 GEMM group is read only by row_sum / row_mean nodes
+  // whose row group holds nothing but per-row values, the epilogue emits one partial sum per row and 32-column
+  // chunk instead of the value, and that row group runs over [R, chunks].
+  for (int v = 0; v < n; ++v) {
+    const Node& nv = g.nodes[v];
+    if (nv.cls == OpClass::Input || nv.output_index >= 0 || nv.dtype != F32) continue;
+    const int gv = p.group_of[v];
+    if (p.groups[gv].kind != GroupKind::Gemm) continue;
+    const Node& an = g.nodes[p.groups[gv].nodes[0]];
+    const Node& opa = g.nodes[an.args[0].node];
+    const Node& opb = g.nodes[an.args[1].node];
+    if (opa.dtype != BF16 || opb.dtype != BF16 || opa.shape[1] % 8 != 0 || an.shape[1] % 32 != 0) continue;
+    int target = -1;
+    bool ok = true, any = false;
+    for (int u = 0; u < n && ok; ++u)
+      for (auto& a : g.nodes[u].args) {
+        if (a.is_literal() || a.node != v) continue;
+        if (p.group_of[u] == gv) { ok = false; break; }   // also used inside the epilogue: stays an ordinary value
+        const Node& nu = g.nodes[u];
+        if (!(nu.cls == OpClass::RowReduce && (nu.op == "row_sum" || nu.op == "row_mean"))) { ok = false; break; }
+        if (target >= 0 && p.group_of[u] != target) { ok = false; break; }
+        target = p.group_of[u];
+        any = true;
+      }
+    if (!ok || !any) continue;
+    Group& tg = p.groups[target];
+    if (tg.kind != GroupKind::Row) continue;
+    for (int u : tg.nodes) {
+      if (!p.is_colv[u]) ok = false;
+      for (auto& a : g.nodes[u].args)   // no other full-width operand in that group
+        if (!a.is_literal() && a.node != v && p.group_of[a.node] != target && g.nodes[a.node].shape == tg.full_shape) ok = false;
+    }
+    if (!ok) continue;
+    p.partial_cols[v] = nv.shape[1] / 32;
+    for (int u : tg.nodes)
+      for (auto& a : g.nodes[u].args)
+        if (!a.is_literal() && a.node == v) p.reduce_count[u] = nv.shape[1];
+    tg.full_shape = {nv.shape[0], p.partial_cols[v]};
+  }
+
   // Iteration spaces, external operands.
   for (auto& grp : p.groups) {
     grp.C = grp.full_shape.back();
@@ -197,8 +245,11 @@ Plan make_plan(const Graph& g) {
     if (need_ws) {
       // intermediates are fp32, except values a cast has rounded to bf16, which keep that width
       p.ws_offset[i] = (int64_t)ws;
-      ws += ((size_t)nd.numel() * (nd.dtype == BF16 ? 2 : 4) + 255) / 256 * 256;
-      grp.stores.push_back({i, nd.dtype, false});
+      if (p.partial_cols[i] > 0)
+        ws += ((size_t)nd.shape[0] * p.partial_cols[i] * 4 + 255) / 256 * 256;   // fp32 partial row sums
+      else
+        ws += ((size_t)nd.numel() * (nd.dtype == BF16 ? 2 : 4) + 255) / 256 * 256;
+      grp.stores.push_back({i, p.partial_cols[i] > 0 ? F32 : nd.dtype, false});
     }
   }
   p.workspace_bytes = ws;
@@ -246,7 +297,8 @@ Plan make_plan(const Graph& g) {
     os << "]:";
     for (int i : grp.nodes) os << " " << g.nodes[i].name << "=" << g.nodes[i].op;
     os << " | stores:";
-    for (auto& s : grp.stores) os << " " << g.nodes[s.node].name << (s.to_output ? "" : "(ws)");
+    for (auto& s : grp.stores)
+      os << " " << g.nodes[s.node].name << (s.to_output ? "" : p.partial_cols[s.node] > 0 ? "(ws: row sums of 32-column chunks, folded into the epilogue)" : "(ws)");
     os << "\n";
   }
   p.text = os.str();

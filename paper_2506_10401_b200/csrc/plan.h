@@ -51,6 +51,10 @@ struct Plan {
   std::vector<int> group_of;           // per node (-1 for inputs)
   std::vector<int64_t> ws_offset;      // per node, -1 if not in workspace
   std::vector<char> is_colv;           // per node: value is one scalar per row of its group
+  // A contraction result that only feeds row sums is not materialised: the epilogue writes one partial sum per
+  // row and 32-column chunk, and the row group sums those.  partial_cols[node] = chunks per row (0: stored whole);
+  // reduce_count[node] = number of elements a row_mean divides by when its operand arrives as partial sums (0: its width).
+  std::vector<int64_t> partial_cols, reduce_count;
   size_t workspace_bytes = 0;
   double algorithmic_bytes = 0, flops = 0;
   std::string text;
