@@ -169,7 +169,7 @@ Plan make_plan(const Graph& g) {
   }
 
   // Row sums folded into a contraction's epilogue (the paper's first case study: matrix product, dropout, mean,
-  // softmax in one fused group).  When a value of a bf16 GEMM group is read only by row_sum / row_mean nodes
+  // softmax in one fused group).  When a value of a tensor-core GEMM group is read only by row_sum / row_mean nodes
   // whose row group holds nothing but per-row values, the epilogue emits one partial sum per row and 32-column
   // chunk instead of the value, and that row group runs over [R, chunks].
   for (int v = 0; v < n; ++v) {
@@ -180,7 +180,10 @@ Plan make_plan(const Graph& g) {
     const Node& an = g.nodes[p.groups[gv].nodes[0]];
     const Node& opa = g.nodes[an.args[0].node];
     const Node& opb = g.nodes[an.args[1].node];
-    if (opa.dtype != BF16 || opb.dtype != BF16 || opa.shape[1] % 8 != 0 || an.shape[1] % 32 != 0) continue;
+    // (the operand types and extents for which the tensor-core kernels, whose epilogue works on 32-column chunks, are taken)
+    const bool tc_bf16 = opa.dtype == BF16 && opb.dtype == BF16 && opa.shape[1] % 8 == 0;
+    const bool tc_f32 = opa.dtype == F32 && opb.dtype == F32 && opa.shape[1] % 4 == 0;
+    if (!(tc_bf16 || tc_f32) || an.shape[1] % 32 != 0) continue;
     int target = -1;
     bool ok = true, any = false;
     for (int u = 0; u < n && ok; ++u)
