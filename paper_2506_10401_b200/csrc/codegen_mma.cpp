@@ -449,7 +449,8 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     // pre-pass and no scratch.  Not the default: measured, it only ties the two-launch path on 256^3
     // (16 us both) and loses on larger problems (4096x1024x1024: 115 us against 63 us), the split warps
     // being the slowest stage of its pipeline.
-    const bool insplit = da == F32 && db == F32 && K % 4 == 0 && N % 4 == 0 && tun.gemm_pair != 1 && tun.gemm_insplit == 1;
+    const bool a_presplit = p.split_store[anchor.args[0].node] != 0;   // A arrives as TF32 head and tail written by its producer
+    const bool insplit = da == F32 && db == F32 && K % 4 == 0 && N % 4 == 0 && tun.gemm_pair != 1 && tun.gemm_insplit == 1 && !a_presplit;
     if (insplit && M <= 0x7fffffff && N <= 0x7fffffff && K <= 0x7fffffff) {
       const int BN = 64;   // 448 threads share the register file: a 128-column running sum per epilogue thread would spill
       const int rstages = 3, stages = 3;
@@ -500,7 +501,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     }
     if (da == F32 && db == F32 && K % 4 == 0 && M <= 0x7fffffff && N <= 0x7fffffff && K <= 0x7fffffff) {
       auto align256 = [](int64_t v) { return (v + 255) / 256 * 256; };
-      const int64_t a_bytes = align256(M * K * 4), b_bytes = align256(K * N * 4);
+      const int64_t a_bytes = a_presplit ? 0 : align256(M * K * 4), b_bytes = align256(K * N * 4);
       const int64_t off_ahi = 0, off_alo = a_bytes, off_bhi = 2 * a_bytes, off_blo = 2 * a_bytes + b_bytes;
       *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(2 * a_bytes + 2 * b_bytes));
       auto scratch = [](int64_t off) {
@@ -519,15 +520,17 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         KernelSpec k;
         k.name = "hct_split_tf32_g" + std::to_string(gi);
         std::ostringstream src;
-        src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n#define HCT_KERNEL_NAME " << k.name << "\n"
+        src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n#define HCT_SPLIT_A " << (a_presplit ? 0 : 1)
+            << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
             << skeleton_source("common") << "\nstruct HctParams { void* ptr[6]; };\n" << skeleton_source("split_tf32");
         k.source = src.str();
         k.ptrs = {node_buf(anchor.args[0].node), node_buf(anchor.args[1].node), scratch(off_ahi), scratch(off_alo), scratch(off_bhi),
                   scratch(off_blo)};
-        int64_t blocks = (M * K / 4 + 1023) / 1024 + ((K + 31) / 32) * ((N + 31) / 32);
+        int64_t blocks = (a_presplit ? 0 : (M * K / 4 + 1023) / 1024) + ((K + 31) / 32) * ((N + 31) / 32);
         k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(blocks, 148 * 16));
         k.block[0] = 256;
-        k.desc = "tf32 head/tail split of both gemm operands, B transposed";
+        k.desc = a_presplit ? "tf32 head/tail split of the second gemm operand, transposed (the first arrives split)"
+                            : "tf32 head/tail split of both gemm operands, B transposed";
         out->push_back(k);
       }
       // 256-column tiles (`gemm_bn=256`) halve the instruction count but were measured no faster than 128-column ones
@@ -560,6 +563,10 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         for (int i = 0; i < 4; ++i) {
           TmaDesc t;
           t.buf = scratch(i == 0 ? off_ahi : i == 1 ? off_alo : i == 2 ? off_bhi : off_blo);
+          if (a_presplit && i < 2) {
+            t.buf = node_buf(anchor.args[0].node);
+            t.base_offset = i == 0 ? 0 : (uint64_t)p.split_lo_offset[anchor.args[0].node];
+          }
           t.elem_bytes = 4;
           t.rank = 2;
           t.dims[0] = (uint64_t)K; t.dims[1] = (uint64_t)(i < 2 ? M : N);   // B is transposed to [N,K]
@@ -591,6 +598,10 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       for (int i = 0; i < 4; ++i) {
         TmaDesc t;
         t.buf = scratch(i == 0 ? off_ahi : i == 1 ? off_alo : i == 2 ? off_bhi : off_blo);
+        if (a_presplit && i < 2) {
+          t.buf = node_buf(anchor.args[0].node);
+          t.base_offset = i == 0 ? 0 : (uint64_t)p.split_lo_offset[anchor.args[0].node];
+        }
         t.elem_bytes = 4;
         t.rank = 2;
         if (i < 2) {
@@ -821,6 +832,8 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
   for (auto& st : grp.stores)
     if (p.partial_cols[st.node] > 0)
       throw Error(HCT_ERR_UNSUPPORTED, "row sums folded into a GEMM epilogue need the tensor-core kernel (not available with simt_only)");
+  if (grp.kind == GroupKind::Gemm && p.split_store[anchor.args[0].node])
+    throw Error(HCT_ERR_UNSUPPORTED, "an operand stored as TF32 head and tail needs the tensor-core GEMM (not available with simt_only)");
   auto operand_buf = [&](int node) {
     return eg.ptr_index(node, g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0);
   };

@@ -426,6 +426,9 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
     if (p.is_colv[s.node])
       stores << "      " << FORB << "if (HCT_LIVEB(b) && hct_t == 0) hct_st1((" << ct << "*)hct_p.ptr[" << pi << "] + hct_row0 + b, s" << id
              << "[b]);\n";
+    else if (!s.to_output && p.split_store[s.node])
+      stores << "      " << FORB << "if (HCT_LIVEB(b)) hct_store_row_split((float*)hct_p.ptr[" << pi << "], (float*)((char*)hct_p.ptr[" << pi << "] + "
+             << p.split_lo_offset[s.node] << "LL), hct_row0 + b, hct_t, v" << id << "[b]);\n";
     else
       stores << "      " << FORB << "if (HCT_LIVEB(b)) hct_store_row((" << ct << "*)hct_p.ptr[" << pi << "], hct_row0 + b, hct_t, v" << id
              << "[b]);\n";

@@ -34,11 +34,6 @@
 #define HCT_TILES ((long long)HCT_MB * HCT_NB)
 #define HCT_TMEM_COLS (2 * HCT_BN)
 
-__device__ __forceinline__ float hct_to_tf32(float x) {
-  hct_u32 u;
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
-  return __uint_as_float(u);
-}
 
 extern "C" __global__ void __launch_bounds__(192 + HCT_NS, 1) HCT_KERNEL_NAME(const __grid_constant__ HctParams hct_p) {
   extern __shared__ unsigned char hct_smem_raw[];

@@ -212,6 +212,26 @@ __device__ __forceinline__ void hct_store_row(T* base, long long row, int hct_t,
   }
 }
 
+// Store of a value that only fp32 tensor-core GEMMs read as their first operand: its TF32 head and tail.
+__device__ __forceinline__ void hct_store_row_split(float* hi_base, float* lo_base, long long row, int hct_t, const float* v) {
+  float* ph = hi_base + row * (long long)HCT_C;
+  float* pl = lo_base + row * (long long)HCT_C;
+#pragma unroll
+  for (int k = 0; k < HCT_NV; ++k) {
+    int col = (k * HCT_T + hct_t) * HCT_V;
+    if (HCT_FULL_VECS || col < HCT_C) {
+      float h[HCT_V], l[HCT_V];
+#pragma unroll
+      for (int i = 0; i < HCT_V; ++i) {
+        h[i] = hct_to_tf32(v[k * HCT_V + i]);
+        l[i] = hct_to_tf32(v[k * HCT_V + i] - h[i]);
+      }
+      hct_vecio<HCT_V>::st(ph + col, h);
+      hct_vecio<HCT_V>::st(pl + col, l);
+    }
+  }
+}
+
 // ---- staged variant: full-width inputs are prefetched into a shared-memory ring by bulk
 // asynchronous copies (one per row and input, completion counted on an mbarrier), HCT_NSTG rows
 // ahead of the row being computed, so that loads stay in flight during the arithmetic and the

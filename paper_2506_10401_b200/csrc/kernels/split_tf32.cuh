@@ -3,14 +3,10 @@
 // a*b ~ a_lo*b_hi + a_hi*b_lo + a_hi*b_hi with every factor exactly representable in TF32.
 // A[M,K] keeps its layout; B[K,N] is written transposed ([N,K]) so that both tensor-core
 // operands are K-major.
-// Defined by the generator: HCT_M, HCT_N, HCT_K (K a multiple of 4), HctParams, HCT_KERNEL_NAME.
+// With HCT_SPLIT_A = 0 only B is handled: A's head and tail were written by the kernel that produced A.
+// Defined by the generator: HCT_M, HCT_N, HCT_K (K a multiple of 4), HCT_SPLIT_A, HctParams, HCT_KERNEL_NAME.
 // Pointer slots: 0 = A, 1 = B, 2 = A_hi, 3 = A_lo, 4 = Bt_hi, 5 = Bt_lo.
-__device__ __forceinline__ float hct_to_tf32(float x) {
-  hct_u32 u;
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
-  return __uint_as_float(u);
-}
-#define HCT_A_BLOCKS ((HCT_M * HCT_K / 4 + 1023) / 1024)          // 256 threads x 4 vectors
+#define HCT_A_BLOCKS (HCT_SPLIT_A ? (HCT_M * HCT_K / 4 + 1023) / 1024 : 0LL)          // 256 threads x 4 vectors
 #define HCT_BT_K ((HCT_K + 31) / 32)
 #define HCT_BT_N ((HCT_N + 31) / 32)
 extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {

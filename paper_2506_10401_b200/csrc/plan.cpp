@@ -74,6 +74,8 @@ Plan make_plan(const Graph& g) {
   p.is_colv.assign(n, 0);
   p.partial_cols.assign(n, 0);
   p.reduce_count.assign(n, 0);
+  p.split_store.assign(n, 0);
+  p.split_lo_offset.assign(n, 0);
 
   auto add_ext = [&](Group& grp, int node, int consumer) {
     if (find_ext(grp, node) >= 0) return;
@@ -212,6 +214,25 @@ Plan make_plan(const Graph& g) {
     tg.full_shape = {nv.shape[0], p.partial_cols[v]};
   }
 
+  // TF32 head and tail written by the producing row kernel's store.
+  for (int v = 0; v < n; ++v) {
+    const Node& nv = g.nodes[v];
+    if (nv.cls == OpClass::Input || nv.output_index >= 0 || nv.dtype != F32 || nv.shape.size() != 2) continue;
+    const Group& gv = p.groups[p.group_of[v]];
+    if (gv.kind != GroupKind::Row || p.is_colv[v] || nv.shape != gv.full_shape) continue;
+    bool ok = true, any = false;
+    for (int u = 0; u < n && ok; ++u)
+      for (size_t ai = 0; ai < g.nodes[u].args.size(); ++ai) {
+        const Operand& a = g.nodes[u].args[ai];
+        if (a.is_literal() || a.node != v || p.group_of[u] == p.group_of[v]) continue;
+        const Node& nu = g.nodes[u];
+        const bool gemm_a = nu.cls == OpClass::Gemm && ai == 0 && g.nodes[nu.args[1].node].dtype == F32 && nv.shape[1] % 4 == 0;
+        if (!gemm_a) ok = false;
+        any = true;
+      }
+    if (ok && any) p.split_store[v] = 1;
+  }
+
   // Iteration spaces, external operands.
   for (auto& grp : p.groups) {
     grp.C = grp.full_shape.back();
@@ -248,7 +269,10 @@ Plan make_plan(const Graph& g) {
     if (need_ws) {
       // intermediates are fp32, except values a cast has rounded to bf16, which keep that width
       p.ws_offset[i] = (int64_t)ws;
-      if (p.partial_cols[i] > 0)
+      if (p.split_store[i]) {
+        p.split_lo_offset[i] = (int64_t)(((size_t)nd.numel() * 4 + 255) / 256 * 256);   // head, then tail
+        ws += 2 * (size_t)p.split_lo_offset[i];
+      } else if (p.partial_cols[i] > 0)
         ws += ((size_t)nd.shape[0] * p.partial_cols[i] * 4 + 255) / 256 * 256;   // fp32 partial row sums
       else
         ws += ((size_t)nd.numel() * (nd.dtype == BF16 ? 2 : 4) + 255) / 256 * 256;
@@ -301,7 +325,9 @@ Plan make_plan(const Graph& g) {
     for (int i : grp.nodes) os << " " << g.nodes[i].name << "=" << g.nodes[i].op;
     os << " | stores:";
     for (auto& s : grp.stores)
-      os << " " << g.nodes[s.node].name << (s.to_output ? "" : p.partial_cols[s.node] > 0 ? "(ws: row sums of 32-column chunks, folded into the epilogue)" : "(ws)");
+      os << " " << g.nodes[s.node].name
+         << (s.to_output ? "" : p.partial_cols[s.node] > 0 ? "(ws: row sums of 32-column chunks, folded into the epilogue)"
+             : p.split_store[s.node] ? "(ws: TF32 head and tail for the GEMM that reads it)" : "(ws)");
     os << "\n";
   }
   p.text = os.str();

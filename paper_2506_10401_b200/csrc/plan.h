@@ -55,6 +55,11 @@ struct Plan {
   // row and 32-column chunk, and the row group sums those.  partial_cols[node] = chunks per row (0: stored whole);
   // reduce_count[node] = number of elements a row_mean divides by when its operand arrives as partial sums (0: its width).
   std::vector<int64_t> partial_cols, reduce_count;
+  // A full-width fp32 value of a row group whose only readers are fp32 tensor-core GEMMs taking it as their first
+  // operand is stored as the TF32 head and tail those GEMMs multiply (two arrays in its workspace slot, the tail
+  // split_lo_offset bytes after the head) instead of as the value itself: the GEMM's split pre-pass skips it.
+  std::vector<char> split_store;
+  std::vector<int64_t> split_lo_offset;
   size_t workspace_bytes = 0;
   double algorithmic_bytes = 0, flops = 0;
   std::string text;
