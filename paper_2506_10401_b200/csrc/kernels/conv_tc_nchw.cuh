@@ -104,6 +104,84 @@ __device__ __forceinline__ HctConvTile hct_conv_tile(long long t, long long t1) 
   return r;
 }
 
+#if HCT_FLAT
+// Epilogue of one 32-column chunk of a flat tile (columns 32 c .. 32 c + 31 of the accumulator at `taddr`), by one
+// warp whose lanes own output channels q * 32 + lane.  Positions oc .. oc + 31 of the image hold n1 valid ones up
+// to the end of output row `hrow`, then `skip` dropped ones (the padding columns of that row), then valid ones of
+// the next row: the gap is closed, the run staged in `o_slot` (2 KB of shared memory), and stored channel by channel.
+__device__ __forceinline__ void hct_flat_chunk(const HctParams& hct_p, const HctConvTile& t, hct_u32 taddr, int c, int q, int lane, hct_u32 o_slot) {
+  const int oc = t.o0 + c * 32;
+  if (oc >= HCT_HO * HCT_P) return;
+  const int hrow = oc / HCT_P, a = oc - hrow * HCT_P;
+  const int n1 = a < HCT_WO ? (HCT_WO - a < 32 ? HCT_WO - a : 32) : 0;
+  const int jend = HCT_P - a < 32 ? HCT_P - a : 32;
+  const int skip = jend - n1;
+  const int run = n1 + (hrow + 1 < HCT_HO ? 32 - jend : 0);
+  if (run == 0) return;
+  const int idx0 = hrow * HCT_WO + (a < HCT_WO ? a : HCT_WO);     // index of the run's first element in its plane
+  const int k = t.mbk * HCT_BM + q * 32 + lane;                    // output channel of this thread's TMEM lane
+  float v[32], w[32];
+  hct_tmem_ld32(taddr + c * 32, v);
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    float x = v[j];
+#pragma unroll
+    for (int g = 1; g <= HCT_P - HCT_WO; ++g)
+      if (j + g < 32) x = (skip == g && j >= n1) ? v[j + g < 32 ? j + g : 31] : x;
+    w[j] = x;
+  }
+  float o[32];
+  if (k < HCT_KO) {
+    hct_epilogue_vals(hct_p, w, (long long)t.n * HCT_KO + k, idx0, run, o);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) o[j] = 0.0f;
+  }
+  // rows of 64 bytes (one channel each), 16-byte piece j of row i at piece j ^ ((i >> 1) & 3)
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const hct_u32 dst = o_slot + (hct_u32)lane * 64u + (((hct_u32)j ^ (((hct_u32)lane >> 1) & 3u)) << 4);
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(hct_pack_bf16x2(o[8 * j], o[8 * j + 1])),
+                 "r"(hct_pack_bf16x2(o[8 * j + 2], o[8 * j + 3])), "r"(hct_pack_bf16x2(o[8 * j + 4], o[8 * j + 5])),
+                 "r"(hct_pack_bf16x2(o[8 * j + 6], o[8 * j + 7]))
+                 : "memory");
+  }
+  __syncwarp();
+  const int kbase = t.mbk * HCT_BM + q * 32;
+  hct_bf16_t* ybase = (hct_bf16_t*)hct_p.ptr[HCT_OUT_SLOT] + ((long long)t.n * HCT_KO + kbase) * (long long)(HCT_HO * HCT_WO) + idx0;
+#if HCT_P % 2 == 0 && HCT_WO % 2 == 0
+  // every run starts at an even element and has an even length: two elements per lane, two channels per instruction
+  {
+    const int pp = lane & 15, ro = lane >> 4;
+    if (2 * pp < run) {
+#pragma unroll 8
+      for (int i = 0; i < 16; ++i) {
+        const int ch = 2 * i + ro;
+        if (kbase + ch < HCT_KO) {
+          hct_u32 e_;
+          asm volatile("ld.shared.b32 %0, [%1];" : "=r"(e_) : "r"(o_slot + (hct_u32)ch * 64u + ((((hct_u32)pp >> 2) ^ (((hct_u32)ch >> 1) & 3u)) << 4) + ((hct_u32)pp & 3u) * 4u) : "memory");
+          *(hct_u32*)(ybase + (long long)ch * (HCT_HO * HCT_WO) + 2 * pp) = e_;
+        }
+      }
+    }
+  }
+#else
+  if (lane < run) {   // lane = element of the run
+    const hct_u32 src0 = o_slot + ((hct_u32)lane & 7u) * 2u;
+#pragma unroll 8
+    for (int i = 0; i < 32; ++i) {
+      if (kbase + i < HCT_KO) {
+        unsigned short e_;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(e_) : "r"(src0 + (hct_u32)i * 64u + ((((hct_u32)lane >> 3) ^ (((hct_u32)i >> 1) & 3u)) << 4)) : "memory");
+        ybase[(long long)i * (HCT_HO * HCT_WO) + lane] = e_;
+      }
+    }
+  }
+#endif
+  __syncwarp();
+}
+#endif
+
 extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HCT_KERNEL_NAME(const __grid_constant__ HctParams hct_p) {
   extern __shared__ unsigned char hct_smem_raw[];
   __shared__ unsigned long long bars[HCT_NBAR];
@@ -240,63 +318,13 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
       hct_tc_fence_after();
       const int k = t.mbk * HCT_BM + q * 32 + lane;      // output channel of this thread's TMEM lane
 #if HCT_FLAT
+      // chunks of this lane quarter are shared by its two epilogue warps; on the CTA's last tile, whose epilogue
+      // nothing overlaps, the two transposer warps of the quarter (idle by then) take a share as well
+      const bool last_tile = tile + gridDim.x >= n_tiles;
+      const int part = warp >= 15 ? 1 : 0;
 #pragma unroll 1
-      for (int c = (warp >= 15 ? 1 : 0); c < 8; c += 2) {
-        // positions oc .. oc + 31 of the image: n1 valid ones up to the end of output row `hrow`, then `skip`
-        // dropped ones (the padding columns of that row), then n2 valid ones of the next row
-        const int oc = t.o0 + c * 32;
-        if (oc >= HCT_HO * HCT_P) break;
-        const int hrow = oc / HCT_P, a = oc - hrow * HCT_P;
-        const int n1 = a < HCT_WO ? (HCT_WO - a < 32 ? HCT_WO - a : 32) : 0;
-        const int jend = HCT_P - a < 32 ? HCT_P - a : 32;
-        const int skip = jend - n1;
-        const int run = n1 + (hrow + 1 < HCT_HO ? 32 - jend : 0);
-        if (run == 0) continue;
-        const int idx0 = hrow * HCT_WO + (a < HCT_WO ? a : HCT_WO);     // index of the run's first element in its plane
-        float v[32], w[32];
-        hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * 256 + c * 32, v);
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          float x = v[j];
-#pragma unroll
-          for (int g = 1; g <= HCT_P - HCT_WO; ++g)
-            if (j + g < 32) x = (skip == g && j >= n1) ? v[j + g < 32 ? j + g : 31] : x;
-          w[j] = x;
-        }
-        float o[32];
-        if (k < HCT_KO) {
-          hct_epilogue_vals(hct_p, w, (long long)t.n * HCT_KO + k, idx0, run, o);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) o[j] = 0.0f;
-        }
-        // rows of 64 bytes (one channel each), 16-byte piece j of row i at piece j ^ ((i >> 1) & 3)
-        const hct_u32 o_slot = smem_base + HCT_RING_O_OFF + (hct_u32)((q * 2 + (warp >= 15 ? 1 : 0)) * 2048);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const hct_u32 dst = o_slot + (hct_u32)lane * 64u + (((hct_u32)j ^ (((hct_u32)lane >> 1) & 3u)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(hct_pack_bf16x2(o[8 * j], o[8 * j + 1])),
-                       "r"(hct_pack_bf16x2(o[8 * j + 2], o[8 * j + 3])), "r"(hct_pack_bf16x2(o[8 * j + 4], o[8 * j + 5])),
-                       "r"(hct_pack_bf16x2(o[8 * j + 6], o[8 * j + 7]))
-                       : "memory");
-        }
-        __syncwarp();
-        // the warp stores the run of every channel: lane = element of the run
-        const int kbase = t.mbk * HCT_BM + q * 32;
-        hct_bf16_t* yrow = (hct_bf16_t*)hct_p.ptr[HCT_OUT_SLOT] + ((long long)t.n * HCT_KO + kbase) * (long long)(HCT_HO * HCT_WO) + idx0 + lane;
-        const hct_u32 src0 = o_slot + ((hct_u32)lane & 7u) * 2u;
-        if (lane < run) {
-#pragma unroll 8
-          for (int i = 0; i < 32; ++i) {
-            if (kbase + i < HCT_KO) {
-              unsigned short e_;
-              asm volatile("ld.shared.u16 %0, [%1];" : "=h"(e_) : "r"(src0 + (hct_u32)i * 64u + ((((hct_u32)lane >> 3) ^ (((hct_u32)i >> 1) & 3u)) << 4)) : "memory");
-              yrow[(long long)i * (HCT_HO * HCT_WO)] = e_;
-            }
-          }
-        }
-        __syncwarp();
-      }
+      for (int c = part; c < 8; c += last_tile ? 4 : 2)
+        hct_flat_chunk(hct_p, t, tmem_base + ((hct_u32)(q * 32) << 16) + acc * 256, c, q, lane, smem_base + HCT_RING_O_OFF + (hct_u32)((q * 2 + part) * 2048));
 #else
       const int chunks = t.th * (HCT_PITCH / 32);
 #pragma unroll 1
@@ -459,6 +487,23 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
         if (++sb == HCT_NBUF) { sb = 0; pb ^= 1u; }
       }
     }
+#if HCT_FLAT
+    // Nothing is left to transpose: take a share of the last tile's epilogue (chunks 2 and 6, or 3 and 7, of this
+    // warp's lane quarter), staged in the idle pixel ring.  The tile's accumulator and the phase of its barrier
+    // follow from how many tiles this CTA has worked on.
+    if ((long long)blockIdx.x < n_tiles) {
+      const long long ntl = (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x;
+      const HctConvTile t = hct_conv_tile(blockIdx.x + (ntl - 1) * gridDim.x, t1);
+      const int acc_l = (int)((ntl - 1) & 1);
+      const hct_u32 phase_l = (hct_u32)(((ntl - 1) >> 1) & 1);
+      const int q = warp & 3, part = 2 + ((warp - 7) >> 2);
+      hct_mbar_wait(tfull0 + 8 * acc_l, phase_l, &failed, status, 9);
+      hct_tc_fence_after();
+#pragma unroll 1
+      for (int c = part; c < 8; c += 4)
+        hct_flat_chunk(hct_p, t, tmem_base + ((hct_u32)(q * 32) << 16) + acc_l * 256, c, q, lane, smem_base + HCT_RING_S_OFF + (hct_u32)((q * 2 + part - 2) * 2048));
+    }
+#endif
   }
   hct_tc_fence_before();
   __syncthreads();
