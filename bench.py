@@ -230,7 +230,7 @@ def run_gpu(name, steps, warmup, rank, world, device, tune=0, with_e2e=True):
             b.record(stream)
         # nvidia-smi samples every 50 ms and a short timed region may end before its first sample: the same
         # steps keep running, untimed, until the sampler has seen about 0.3 s of this load
-        t_end = time.perf_counter() + max(0.0, 0.3 - 1e-3 * steps)
+        t_end = time.perf_counter() + (max(0.0, 0.3 - 1e-3 * steps) if steps >= 10 else 0.0)   # (short profiling runs stay short)
         while time.perf_counter() < t_end:
             flush.zero_()
             g.run(ins, outs, stream)

@@ -58,6 +58,7 @@ struct hct_graph {
   size_t workspace_bytes = 0;
   int device = HCT_DEVICE_NONE;
   bool use_pdl = true;
+  bool pdl_first = true;   // the first kernel of a run is launched as a programmatic dependent too
   CUcontext_t ctx = nullptr;
   CUdevice_t cudev = 0;
   CUdeviceptr_t status_word = 0;
@@ -126,6 +127,7 @@ hct_status_t hct_graph_create_scheduled(const char* spec, size_t spec_len, int d
     h->plan_text = pt.str();
     h->device = device;
     if (const char* e = std::getenv("HCT_NO_PDL")) h->use_pdl = std::atoi(e) == 0;
+    if (const char* e = std::getenv("HCT_FIRST_NO_PDL")) h->pdl_first = std::atoi(e) == 0;
 
     const Driver* d = nullptr;
     int sms = 148;
@@ -254,10 +256,14 @@ hct_status_t hct_graph_run(hct_graph_t* g, const void* const* inputs, int n_inpu
       }
       std::memcpy(block + off, ptrs, std::max<size_t>(np, 1) * sizeof(void*));
       void* args[] = {block};
-      // Kernels after the first may be scheduled while their predecessor drains (programmatic dependent
-      // launch): each kernel waits on the device for the predecessor's completion before it reads memory.
+      // Every kernel may be scheduled while its predecessor in the stream drains (programmatic dependent
+      // launch): it waits on the device for the predecessor's completion before it touches global memory.
+      // That holds for the first kernel of a run as well, so runs issued back to back overlap their launch
+      // and prologue with the previous run's tail; behind a kernel that never signals its dependents (any
+      // kernel that is not this library's) the launch simply takes place at that kernel's end, as usual.
+      // HCT_FIRST_NO_PDL=1 restores a plain launch for the first kernel.
       CUresult_t rc;
-      if (&k != &g->kernels.front() && g->use_pdl) {
+      if ((&k != &g->kernels.front() || g->pdl_first) && g->use_pdl) {
         LaunchAttr attr;
         std::memset(&attr, 0, sizeof attr);
         attr.id = kLaunchAttrProgrammaticStreamSerialization;
