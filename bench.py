@@ -4,7 +4,10 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
 One step = one run of a whole fused chain (every kernel of its plan) on one batch of seeded
-synthetic input.  The headline workload is the memory-bound chain (affine, GELU, row softmax,
+synthetic input.  The K timed steps run back to back between one pair of CUDA events, rotating over
+copies of every buffer whose total exceeds L2 twice over (a step that moves more than L2 needs one
+copy), each copy's step captured in a CUDA graph; the time of the same steps taken one by one, each
+between its own event pair after an L2 flush, is reported beside it.  The headline workload is the memory-bound chain (affine, GELU, row softmax,
 row layer normalisation on an fp32 [8192,4096] tensor); throughput is algorithmic bytes per
 second (inputs read once, outputs written once).  Contraction chains report TFLOP/s.
 Without --workload the line also carries, under "configs", the other four benchmark
@@ -217,12 +220,31 @@ def run_gpu(name, steps, warmup, rank, world, device, tune=0, with_e2e=True):
             torch.distributed.barrier()
         torch.cuda.synchronize(device)
 
+    # Timed region: exactly `steps` steps, back to back, between one pair of events.  The steps rotate over copies of
+    # every buffer (see RotatingSets), so no step finds its operands in L2 and none waits for a host launch.
+    try:
+        rot = RotatingSets(g, ins, device)
+    except Exception as e:  # noqa: BLE001 - without capture the steps are timed one by one, each after an L2 flush
+        print(f"CUDA-graph capture failed, timing step by step: {e}", file=sys.stderr)
+        rot = None
     for _ in range(max(warmup, 3)):
         flush.zero_()
         g.run(ins, outs, stream)
+    if rot is not None:
+        for _ in range(max(warmup, 3) * rot.n_sets):
+            rot.step()
     barrier()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(device) as clocks:
+        if rot is not None:
+            t0.record(stream)
+            for _ in range(steps):
+                rot.step()
+            t1.record(stream)
+            barrier()
+        # second figure: the same number of steps, each between its own pair of events after an L2 flush (about 6 us of
+        # launch and event cost per step on top of the kernels)
         for a, b in ev:
             flush.zero_()           # evict the previous step's data from L2; not timed
             a.record(stream)
@@ -232,19 +254,28 @@ def run_gpu(name, steps, warmup, rank, world, device, tune=0, with_e2e=True):
         # steps keep running, untimed, until the sampler has seen about 0.3 s of this load
         t_end = time.perf_counter() + (max(0.0, 0.3 - 1e-3 * steps) if steps >= 10 else 0.0)   # (short profiling runs stay short)
         while time.perf_counter() < t_end:
-            flush.zero_()
-            g.run(ins, outs, stream)
+            if rot is not None:
+                for _ in range(8):
+                    rot.step()
+            else:
+                flush.zero_()
+                g.run(ins, outs, stream)
             torch.cuda.synchronize(device)
         barrier()
     g.status()
     per_step = [a.elapsed_time(b) * 1e-3 for a, b in ev]
-    dev_s = float(np.sum(per_step))
+    events_s = float(np.sum(per_step))
+    dev_s = t0.elapsed_time(t1) * 1e-3 if rot is not None else events_s
+    timing = dict(protocol=("steps back to back between one event pair, rotating over %d copies of every buffer (L2 %s)" % (rot.n_sets, rot.l2))
+                  if rot is not None else "each step between its own event pair after an L2 flush",
+                  events_ms_per_step=events_s / steps * 1e3)
     if not with_e2e:
         dev_s = max_over_ranks([dev_s], f"cuda:{device}")[0]
         value, unit = whole_job_value(info["bound"], bytes_, flops, world, dev_s / steps)
-        return dict(value=value, unit=unit, ms_per_step=dev_s / steps * 1e3, bytes=bytes_, flops=flops, kernel_s=float(np.mean(per_step)),
+        return dict(value=value, unit=unit, ms_per_step=dev_s / steps * 1e3, bytes=bytes_, flops=flops, kernel_s=dev_s / steps,
                     fingerprint=kernel_fingerprint(g), kernels=g.num_kernels, clocks=clocks.summary(), e2e=None, plan=g.plan,
-                    schedule=g.schedule)
+                    schedule=g.schedule, timing=timing)
+    del rot
 
     # end to end: pinned host inputs -> device, run, result back to the host, every step.  The three
     # phases of consecutive steps overlap (copy-in, compute and copy-out streams, two sets of device
@@ -302,12 +333,56 @@ def run_gpu(name, steps, warmup, rank, world, device, tune=0, with_e2e=True):
     dev_s, e2e_s = max_over_ranks([dev_s, e2e_s], f"cuda:{device}")
     value, unit = whole_job_value(info["bound"], bytes_, flops, world, dev_s / steps)
     e2e_v, _ = whole_job_value(info["bound"], bytes_, flops, world, e2e_s)
-    kern_s = float(np.mean(per_step))
-    return dict(value=value, unit=unit, ms_per_step=dev_s / steps * 1e3, bytes=bytes_, flops=flops, kernel_s=kern_s,
+    kern_s = dev_s / steps
+    return dict(value=value, unit=unit, ms_per_step=dev_s / steps * 1e3, bytes=bytes_, flops=flops, kernel_s=kern_s, timing=timing,
                 fingerprint=kernel_fingerprint(g),
                 kernels=g.num_kernels, clocks=clocks.summary(), e2e=dict(value=e2e_v, unit=unit, h2d_bytes_per_step=h2d,
                                                                          d2h_bytes_per_step=d2h), plan=g.plan,
                 schedule=g.schedule)
+
+
+class RotatingSets:
+    """Copies of a graph's inputs, outputs and workspace whose total exceeds L2 twice over, and one CUDA graph per
+    copy that runs the fused chain on it.  Steps issued round robin over the copies follow each other on the device
+    without a host launch or an L2 flush in between, and every step finds its operands cold (a workload that moves
+    more than L2 per step needs a single copy; one too small to reach the budget with `max_sets` copies runs partly
+    warm: `l2` says which)."""
+
+    def __init__(self, g, ins, device, budget_bytes=256 << 20, max_sets=24):
+        import torch
+        import paper_2506_10401_b200 as hct
+        self.g, self.device = g, device
+        dev = f"cuda:{device}"
+        outs0 = g.alloc_outputs()
+        per_set = sum(t.numel() * t.element_size() for t in ins) + g.workspace_bytes + sum(t.numel() * t.element_size() for t in outs0)
+        self.n_sets = int(max(1, min(max_sets, -(-budget_bytes // per_set))))
+        self.l2 = "cold" if per_set * self.n_sets >= 192 << 20 else "warm"
+        self.sets = []
+        for i in range(self.n_sets):
+            si = ins if i == 0 else [t.clone() for t in ins]
+            so = outs0 if i == 0 else g.alloc_outputs()
+            ws = torch.empty(g.workspace_bytes + 256, dtype=torch.uint8, device=dev) if g.workspace_bytes else None
+            ws_ptr = (ws.data_ptr() + 255) // 256 * 256 if ws is not None else 0
+            self.sets.append((si, so, ws, [t.data_ptr() for t in si], [t.data_ptr() for t in so], ws_ptr))
+        side = torch.cuda.Stream(device)
+        side.wait_stream(torch.cuda.current_stream(device))
+        self.graphs = []
+        for _, _, _, pi, po, pw in self.sets:
+            with torch.cuda.stream(side):
+                hct.hct_graph_run(g.handle, pi, po, pw, g.workspace_bytes, side.cuda_stream)
+            side.synchronize()
+            cg = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(cg, stream=side, capture_error_mode="thread_local"):
+                hct.hct_graph_run(g.handle, pi, po, pw, g.workspace_bytes, side.cuda_stream)
+            self.graphs.append(cg)
+        self.next = 0
+
+    def step(self):
+        self.graphs[self.next].replay()
+        self.next = (self.next + 1) % self.n_sets
+
+    def outputs_of_last_step(self):
+        return self.sets[(self.next - 1) % self.n_sets][1]
 
 
 def replay_seconds(g, ins, device, budget_bytes=256 << 20, max_sets=24, target_ms=4.0):
@@ -582,7 +657,7 @@ def main():
             o = run_gpu(other, k, args.warmup, rank, world, local, args.tune, with_e2e=False)
             others.append(dict(workload=other, dtype=dtype_of(other), steps=k, warmup=max(args.warmup, 3), ms_per_step=o["ms_per_step"],
                                value=o["value"], unit=o["unit"], roofline=roofline_of(other, o, pk), clocks=o["clocks"],
-                               kernels_per_step=o["kernels"], gpu_launches=o["kernels"] * k, l2="flushed between steps",
+                               kernels_per_step=o["kernels"], gpu_launches=o["kernels"] * k, timing=o["timing"],
                                parity_checked=test))
         others.append(sweep_record(sweep_steps, min(args.warmup, 2), local, args.out, args.tune))
     if rank == 0:
@@ -590,7 +665,8 @@ def main():
         line = dict(metric=metric, value=r["value"], unit=r["unit"], n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
                     ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
                     dtype=dtype_of(name), data="synthetic",
-                    config={"workload": name, "l2": "flushed between steps (192 MB write, untimed)", "kernels_per_step": r["kernels"],
+                    config={"workload": name, "l2": r["timing"]["protocol"], "events_ms_per_step": r["timing"]["events_ms_per_step"],
+                            "kernels_per_step": r["kernels"],
                             "parallelism": "replicas" if world > 1 else "single",
                             "schedule": r["schedule"] or "default", "tuned_trials": args.tune,
                             "parity_checked": PARITY_TEST.get(name)},
