@@ -40,6 +40,9 @@
  *   row_argsort(x, descending=0)  row_topk_indices(x, k=K)   the columns the values of row_sort / row_topk came
  *                         from, as fp32 values; among equal values (-0 and +0 are equal) the smaller column first
  *   transpose(x)          y[j,i] = x[i,j] for x[R,C]; elementwise consumers are applied at the store
+ *   permute(x, axes=DIGITS)  the axes of x (rank 2..4) in another order: output axis d is input axis DIGITS[d]
+ *                         (axes=0231 turns [N,C,H,W] into [N,H,W,C]); a bf16 value stays bf16; one pass, elementwise
+ *                         consumers applied at the store
  *   reshape(x, rows=R, cols=C)   the elements of x (any rank) in row-major order as [R,C], R*C = numel(x);
  *                         a bf16 value stays bf16; one copy pass, elementwise consumers applied at the store
  *   row_sort(x, descending=0)   the values of every row of x[R,C] in non-decreasing (descending=1:

@@ -268,6 +268,17 @@ def _infer(g, name, op, pos, attrs, where):
                 raise SpecError(f"{where}: {op} needs 1 <= k <= C")
             return Node(name, op, [a], {"k": k}, (s[0], k), "f32")
         return Node(name, op, [a], {"descending": _int_attr(attrs, "descending", 0, where)}, s, "f32")
+    if op == "permute":
+        only_attrs("axes")
+        if len(pos) != 1:
+            raise SpecError(f"{where}: permute takes one operand")
+        a = _operand(g, pos[0], where, False)
+        s = shape_of(a)
+        ax = attrs.get("axes", "")
+        if not 2 <= len(s) <= 4 or len(ax) != len(s) or sorted(ax) != [str(d) for d in range(len(s))]:
+            raise SpecError(f"{where}: permute needs rank 2..4 and axes=<a permutation, one digit per axis>")
+        axes = tuple(int(c) for c in ax)
+        return Node(name, op, [a], {"axes": axes}, tuple(s[d] for d in axes), g.nodes[a].dtype)
     if op == "transpose":
         only_attrs()
         if len(pos) != 1:

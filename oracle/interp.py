@@ -145,6 +145,17 @@ def transpose(x):
     return y
 
 
+def permute(x, axes):
+    # y[o] = x[i] with i[axes[d]] = o[d]: output axis d is input axis axes[d]
+    y = np.empty(tuple(x.shape[a] for a in axes), dtype=x.dtype)
+    for o in np.ndindex(*y.shape):
+        i = [0] * x.ndim
+        for d, a in enumerate(axes):
+            i[a] = o[d]
+        y[o] = x[tuple(i)]
+    return y
+
+
 def row_min(x):
     return x.min(axis=1, keepdims=True)
 
@@ -257,6 +268,8 @@ def run_nodes(spec, inputs: dict, dtype=np.float64, gemm_fn=None) -> dict:
             out = row_topk_indices(args[0], node.attrs["k"])
         elif op == "transpose":
             out = transpose(args[0])
+        elif op == "permute":
+            out = permute(args[0], node.attrs["axes"])
         elif op == "row_softmax":
             out = row_softmax(args[0])
         elif op == "row_sum":

@@ -319,6 +319,33 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     return;
   }
 
+  // ---- layout transform: permutation of up to four axes, consumers applied at the store
+  if (grp.kind == GroupKind::Permute) {
+    const int src = anchor.args[0].node;
+    const int pa = eg.ptr_index(src, g.nodes[src].cls != OpClass::Input && p.ws_offset[src] >= 0);
+    const DType ta = eg.buf_dtype(src);
+    std::string epi = eg.scalar_fn();
+    int64_t S[4] = {1, 1, 1, 1};
+    for (size_t d = 0; d < a.shape.size(); ++d) S[4 - a.shape.size() + d] = a.shape[d];
+    KernelSpec k;
+    k.name = "hct_permute_g" + std::to_string(gi);
+    std::ostringstream st;
+    for (int d = 0; d < 4; ++d) st << "#define HCT_S" << d << " " << S[d] << "LL\n#define HCT_P" << d << " " << anchor.perm[d] << "\n";
+    st << "#define HCT_TA " << ctype(ta) << "\n#define HCT_PA " << pa << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+       << skeleton_source("common") << "\nstruct HctParams { void* ptr[" << eg.ptrs.size() << "]; };\n" << epi << skeleton_source("permute");
+    k.source = st.str();
+    k.ptrs = eg.ptrs;
+    const bool inner_kept = anchor.perm[3] == 3;
+    const int64_t work = inner_kept ? (anchor.numel() + 255) / 256
+                                    : (anchor.numel() / std::max<int64_t>(1, S[3] * S[anchor.perm[3]])) * ((S[3] + 63) / 64) * ((S[anchor.perm[3]] + 63) / 64);
+    k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(work, 148 * (inner_kept ? 32 : 8)));
+    k.block[0] = 256;
+    k.desc = inner_kept ? "permute: rows of the innermost axis copied whole, consumers fused at the store"
+                        : "permute: the plane of the old and the new innermost axis transposed through 64x64 shared-memory tiles, consumers fused at the store";
+    out->push_back(k);
+    return;
+  }
+
   // ---- layout transform: tiled transposition through shared memory, consumers applied at the store
   if (grp.kind == GroupKind::Transpose) {
     const int src = anchor.args[0].node;

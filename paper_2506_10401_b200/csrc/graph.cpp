@@ -330,6 +330,27 @@ Graph parse_spec(const std::string& text) {
         auto& s = g.nodes[n.args[0].node].shape;
         if (s.size() != 2) fail(HCT_ERR_GRAPH, line, "transpose needs a [R,C] operand, got " + shape_str(s));
         n.shape = {s[1], s[0]};
+      } else if (op == "permute") {
+        // layout transform (Table 1): the axes of a tensor of rank 2..4 in another order; axes=0231 means
+        // output axis d is input axis digit d (NCHW -> NHWC)
+        only_attrs({"axes"});
+        if (pos.size() != 1) fail(HCT_ERR_GRAPH, line, "permute takes one operand");
+        n.cls = OpClass::Permute;
+        n.args = {lookup(pos[0], line, false)};
+        const Node& src = g.nodes[n.args[0].node];
+        const size_t rank = src.shape.size();
+        const std::string ax = attrs.count("axes") ? attrs["axes"] : "";
+        if (rank < 2 || ax.size() != rank) fail(HCT_ERR_GRAPH, line, "permute needs a tensor of rank 2..4 and axes=<one digit per axis>");
+        bool seen[4] = {false, false, false, false};
+        n.shape.clear();
+        for (size_t d = 0; d < rank; ++d) {
+          const int a = ax[d] - '0';
+          if (a < 0 || a >= (int)rank || seen[a]) fail(HCT_ERR_GRAPH, line, "axes must be a permutation of 0.." + std::to_string(rank - 1));
+          seen[a] = true;
+          n.shape.push_back(src.shape[a]);
+          n.perm[4 - rank + d] = a + (int)(4 - rank);   // in the padded four-axis numbering
+        }
+        n.dtype = src.dtype;   // values are moved unchanged
       } else if (op == "reshape") {
         // layout transform (Table 1): the same elements in row-major order under a new 2-D shape, e.g. flattening
         // [N,C,H,W] into [N, C*H*W] in front of a gemm

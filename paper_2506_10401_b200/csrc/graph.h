@@ -9,7 +9,7 @@ namespace hct {
 
 enum DType { F32 = 0, BF16 = 1 };
 
-enum class OpClass { Input, Unary, Binary, RowSoftmax, RowLayernorm, RowReduce, Gemm, Conv, Transpose, Sort, Reshape };
+enum class OpClass { Input, Unary, Binary, RowSoftmax, RowLayernorm, RowReduce, Gemm, Conv, Transpose, Sort, Reshape, Permute };
 
 struct Error : std::runtime_error {
   int code;
@@ -33,6 +33,7 @@ struct Node {
   int stride = 1, pad = 0, dilation = 1, groups = 1;
   int sort_k = 0;            // row_topk: number of leading elements kept (0: the whole sorted row)
   bool descending = false;   // row_sort / row_topk: largest first
+  int perm[4] = {0, 1, 2, 3}; // permute: output axis d is input axis perm[d] (both padded to four axes with leading ones)
   bool sort_indices = false; // row_argsort / row_topk_indices: the columns of the ordered values instead of the values
   // dropout: element with flat index i is kept when hash(i + seed) mod 1000 >= drop_threshold (= round(1000 p))
   double drop_p = 0.0;

@@ -116,6 +116,7 @@ Plan make_plan(const Graph& g) {
           }
         }
         if (b == Bcast::RowVec && grp.kind == GroupKind::Conv) return false;
+        if (b == Bcast::RowIdx && grp.kind == GroupKind::Permute && grp.full_shape.size() > 2) return false;
       }
       return true;
     }
@@ -138,10 +139,11 @@ Plan make_plan(const Graph& g) {
     if (nd.cls == OpClass::Input) continue;
     int gi = -1;
     if (nd.cls == OpClass::Gemm || nd.cls == OpClass::Conv || nd.cls == OpClass::Transpose || nd.cls == OpClass::Sort ||
-        nd.cls == OpClass::Reshape) {
+        nd.cls == OpClass::Reshape || nd.cls == OpClass::Permute) {
       Group grp;
       grp.kind = nd.cls == OpClass::Gemm ? GroupKind::Gemm : nd.cls == OpClass::Conv ? GroupKind::Conv
-                 : nd.cls == OpClass::Transpose ? GroupKind::Transpose : nd.cls == OpClass::Sort ? GroupKind::Sort : GroupKind::Reshape;
+                 : nd.cls == OpClass::Transpose ? GroupKind::Transpose : nd.cls == OpClass::Sort ? GroupKind::Sort
+                 : nd.cls == OpClass::Permute ? GroupKind::Permute : GroupKind::Reshape;
       grp.full_shape = nd.shape;
       p.groups.push_back(grp);
       gi = (int)p.groups.size() - 1;
@@ -244,7 +246,7 @@ Plan make_plan(const Graph& g) {
     if (nd.cls == OpClass::Input) continue;
     Group& grp = p.groups[p.group_of[i]];
     bool anchor = nd.cls == OpClass::Gemm || nd.cls == OpClass::Conv || nd.cls == OpClass::Transpose || nd.cls == OpClass::Sort ||
-                  nd.cls == OpClass::Reshape;
+                  nd.cls == OpClass::Reshape || nd.cls == OpClass::Permute;
     for (auto& a : nd.args) {
       if (a.is_literal() || p.group_of[a.node] == p.group_of[i]) continue;
       if (anchor) continue;  // contraction operands are bound separately
@@ -307,7 +309,8 @@ Plan make_plan(const Graph& g) {
     for (int j = 0; j < n; ++j)
       for (auto& a : g.nodes[j].args) {
         if (a.is_literal() || a.node != i || p.group_of[j] == p.group_of[i]) continue;
-        bool into_contraction = (g.nodes[j].cls == OpClass::Gemm || g.nodes[j].cls == OpClass::Conv || g.nodes[j].cls == OpClass::Transpose) &&
+        bool into_contraction = (g.nodes[j].cls == OpClass::Gemm || g.nodes[j].cls == OpClass::Conv || g.nodes[j].cls == OpClass::Transpose ||
+                                 g.nodes[j].cls == OpClass::Permute) &&
                                 after_reduction;
         bool from_contraction = (pg.kind == GroupKind::Gemm || pg.kind == GroupKind::Conv) && p.groups[p.group_of[j]].has_reduction &&
                                 nd.shape.back() > 512;
@@ -319,7 +322,7 @@ Plan make_plan(const Graph& g) {
   std::ostringstream os;
   for (size_t gi = 0; gi < p.groups.size(); ++gi) {
     const Group& grp = p.groups[gi];
-    os << "kernel " << gi << " " << (grp.kind == GroupKind::Row ? "row" : grp.kind == GroupKind::Gemm ? "gemm" : grp.kind == GroupKind::Conv ? "conv" : grp.kind == GroupKind::Transpose ? "transpose" : grp.kind == GroupKind::Sort ? "sort" : "reshape") << " [";
+    os << "kernel " << gi << " " << (grp.kind == GroupKind::Row ? "row" : grp.kind == GroupKind::Gemm ? "gemm" : grp.kind == GroupKind::Conv ? "conv" : grp.kind == GroupKind::Transpose ? "transpose" : grp.kind == GroupKind::Sort ? "sort" : grp.kind == GroupKind::Permute ? "permute" : "reshape") << " [";
     for (size_t d = 0; d < grp.full_shape.size(); ++d) os << (d ? "," : "") << grp.full_shape[d];
     os << "]:";
     for (int i : grp.nodes) os << " " << g.nodes[i].name << "=" << g.nodes[i].op;

@@ -13,7 +13,7 @@
 
 namespace hct {
 
-enum class GroupKind { Row, Gemm, Conv, Transpose, Sort, Reshape };
+enum class GroupKind { Row, Gemm, Conv, Transpose, Sort, Reshape, Permute };
 
 // How an operand indexes relative to the group's full shape [.., C].
 enum class Bcast {

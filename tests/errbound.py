@@ -164,6 +164,8 @@ def bound(spec, inputs, values=None):
             e = ae[0].reshape(y.shape)
         elif op == "transpose":
             e = ae[0].T
+        elif op == "permute":
+            e = np.transpose(ae[0], node.attrs["axes"])
         elif op in ("row_sort", "row_topk"):
             # values are moved, not changed; an uncertain key may land in a neighbouring slot
             e = np.broadcast_to(ae[0].max(axis=1, keepdims=True), y.shape)

@@ -441,6 +441,35 @@ def test_transpose_is_exact_and_fuses_its_consumers(r, c):
     assert g.num_kernels == 2 and "transpose" in g.plan
 
 
+@pytest.mark.parametrize("shape,axes", [((2, 6, 5, 7), "0231"), ((2, 6, 5, 7), "0312"), ((3, 70, 9, 66), "0231"), ((2, 3, 4, 5), "3210"),
+                                        ((4, 5, 6), "102"), ((4, 5, 6), "210"), ((130, 67), "10"), ((2, 3, 65, 130), "1032"),
+                                        ((2, 6, 5, 7), "1023"), ((5, 3, 2, 64), "2103"), ((1, 128, 28, 28), "0231")])
+def test_permute_is_exact_and_fuses_its_consumers(shape, axes):
+    """Pure data movement (bit for bit, fp32 and bf16), with elementwise consumers applied at the store."""
+    dims = "[" + ",".join(str(v) for v in shape) + "]"
+    last = shape[int(axes[-1])]
+    spec = (f"hct 1\ninput x f32 {dims}\ninput y bf16 {dims}\ninput b f32 [{last}]\nnode p = permute(x, axes={axes})\nnode q = add(p, b)\n"
+            f"node r = relu(q)\nnode s = permute(y, axes={axes})\noutput p\noutput r\noutput s bf16\n")
+    got, want, g = parity.run_both(spec, {"x": N_, "y": N_, "b": N_})
+    assert g.num_kernels == 2 and g.plan.count("permute") >= 2
+    np.testing.assert_array_equal(got[0], want[0])
+    np.testing.assert_array_equal(got[2], want[2])
+    assert parity.f32_violation(got[1], want[1]) <= 1.0
+
+
+def test_permute_to_channels_last_and_back_around_a_row_kernel():
+    spec = """hct 1
+input x f32 [2,16,6,8]
+input g f32 [16]
+input b f32 [16]
+node a = permute(x, axes=0231)
+node f = reshape(a, rows=96, cols=16)
+node n = row_layernorm(f, g, b, eps=1e-5)
+output n
+"""
+    check_f32(spec, {"x": N_, "g": POS_, "b": N_})
+
+
 def test_transpose_between_other_kernels():
     spec = """hct 1
 input x f32 [96,256]

@@ -407,6 +407,30 @@ def test_sort_hand_values_bruteforce_and_invariants():
     assert g.nodes["t"].shape == (4, 3) and g.nodes["s"].shape == (4, 9)
 
 
+def test_permute_hand_values_inverse_and_library():
+    x = np.arange(24, dtype=np.float64).reshape(2, 3, 4)
+    y = interp.permute(x, (2, 0, 1))                       # y[k, i, j] = x[i, j, k]
+    assert y.shape == (4, 2, 3)
+    assert y[3, 1, 2] == x[1, 2, 3] == 23 and y[1, 0, 2] == x[0, 2, 1] == 9 and y[0, 1, 0] == x[1, 0, 0] == 12
+    z = RNG.normal(size=(3, 4, 5, 6))
+    import itertools
+    for axes in itertools.permutations(range(4)):
+        p = interp.permute(z, axes)
+        np.testing.assert_array_equal(p, np.transpose(z, axes))                      # library routine
+        inv = tuple(int(np.argsort(axes)[d]) for d in range(4))
+        np.testing.assert_array_equal(interp.permute(p, inv), z)                     # the inverse permutation undoes it
+        assert sorted(p.ravel()) == sorted(z.ravel())
+    # two axes: the transposition
+    m = RNG.normal(size=(5, 7))
+    np.testing.assert_array_equal(interp.permute(m, (1, 0)), interp.transpose(m))
+    np.testing.assert_array_equal(interp.permute(m, (0, 1)), m)
+    g = oracle.parse("hct 1\ninput x f32 [2,3,4,5]\nnode p = permute(x, axes=0231)\noutput p\n")
+    assert g.nodes["p"].shape == (2, 4, 5, 3)
+    for bad in ("axes=0221", "axes=012", "axes=0234"):
+        with pytest.raises(oracle.SpecError):
+            oracle.parse(f"hct 1\ninput x f32 [2,3,4,5]\nnode p = permute(x, {bad})\noutput p\n")
+
+
 def test_argsort_hand_values_bruteforce_and_ties():
     x = np.array([[3.0, 1.0, 2.0, 5.0, 4.0], [0.0, -1.0, 7.0, 7.0, 2.0], [1.0, 1.0, 1.0, -0.0, 0.0]])
     # hand values: equal values keep their column order in BOTH directions
@@ -640,6 +664,7 @@ def test_planted_mistakes_are_detected(monkeypatch):
         ("row_topk", lambda x, k: orig["row_sort"](x)[:, :k], test_sort_hand_values_bruteforce_and_invariants),
         ("row_argsort", lambda x, descending=False: np.argsort(-x if descending else x, axis=1).astype(np.float64)[:, ::1] if not descending
          else np.argsort(x, axis=1, kind="stable")[:, ::-1].astype(np.float64), test_argsort_hand_values_bruteforce_and_ties),
+        ("permute", lambda x, axes: np.transpose(x, tuple(int(v) for v in np.argsort(axes))), test_permute_hand_values_inverse_and_library),
         ("row_layernorm", unbiased_ln, test_layernorm_closed_forms),
         ("row_layernorm", eps_outside_ln, test_layernorm_bruteforce_and_torch),
         ("conv2d", flipped_conv, test_conv_structure_pins),
