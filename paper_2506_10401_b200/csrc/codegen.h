@@ -64,6 +64,7 @@ struct Tunables {
   bool conv_no_halo = false;       // load conv pixels once per tap even when the shared-row schedule applies
   bool conv_no_tma_store = false;  // NCHW-reading convolution: store the output with plain vector stores instead of TMA
   int dw_p = 0;                    // depthwise conv: output rows per thread (0: rule; 1, 2, 4 or 8)
+  int dw_pair = 0;                 // depthwise conv: 1 = two filters per thread on packed multiply-adds (needs an even number of filters)
   int dw_cta = 0;                  // depthwise conv: threads per block (0: rule; else a multiple of 32, up to 1024)
   int conv_nstg = 0;               // NCHW-reading conv: slots of the pixel staging ring (0: rule)
   int conv_nbuf = 0;               // NCHW-reading conv: operand buffers (0: rule)
@@ -71,6 +72,8 @@ struct Tunables {
   bool topk_no_select = false;     // row_topk: full bitonic sort of the row even for small k
   bool conv_phase = false;         // strided convolutions: a stride-phase view wherever one exists, not only for rows too wide for a strided box
   bool conv_no_direct = false;     // always take the NHWC pre-pass, even when the convolution could read NCHW itself
+  int conv_pw_warps = 0;           // 1x1 convolution as a per-image GEMM: epilogue warps (0: rule, 16; or 8)
+  bool conv_no_pointwise = false;  // 1x1 convolutions take the general schedules instead of the per-image GEMM
   bool simt_only = false;
   // Failure-path testing: the GEMM producer never issues its loads, so the consumer's bounded wait runs out
   // (the kernel then reports through the status word and ends normally).  wait_limit shortens the bound.

@@ -671,7 +671,83 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     // Rows too wide for one strided box (W' * stride > 256) with a stride that divides both image extents:
     // dense boxes of a stride-phase view.  Both forms were measured at the same speed; `conv_phase=1` prefers the view.
     const bool phased = ST > 1 && ST <= 8 && H % ST == 0 && W % ST == 0 && (WO * ST > 256 || tun.conv_phase);
-    if (in_bf16 && anchor.groups == 1 && ST <= 8 && (WO * ST <= 256 || phased) && C % 8 == 0 && WO <= 256 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
+    // Pointwise convolution on NCHW data: per image the product W[KO,C] * X_n[C,HW], both operands usable as they lie
+    // in memory (weights K-major, pixels N-major): no layout pass at all.
+    if (in_bf16 && anchor.groups == 1 && FR == 1 && FS == 1 && ST == 1 && anchor.pad == 0 && !a.nhwc && (H * W) % 8 == 0 && C % 8 == 0 &&
+        NB <= 0x7fffffff && KO <= 0x7fffffff && H * W <= 0x7fffffff && !tun.conv_no_pointwise) {
+      const int64_t HW = H * W;
+      const bool tma_store = grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && !tun.conv_no_tma_store;
+      const int epw = tun.conv_pw_warps == 8 ? 8 : 16;
+      const int stages = tma_store && epw == 16 ? 3 : 4;
+      std::string epi = eg.run_fn(HW, 32, "(row % " + std::to_string(KO) + "LL)", tma_store);
+      KernelSpec k;
+      k.name = "hct_conv_pw_bf16_g" + std::to_string(gi);
+      std::ostringstream src;
+      src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_KO " << KO << "\n#define HCT_HW " << HW
+          << "\n#define HCT_STAGES " << stages << "\n#define HCT_EPW " << epw << "\n#define HCT_TMA_STORE " << (tma_store ? 1 : 0) << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
+          << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
+      src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[" << (tma_store ? 3 : 2)
+          << "]; void* ptr[" << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source("conv_pw_tc");
+      k.source = src.str();
+      k.ptrs = eg.ptrs;
+      k.wants_status = true;
+      auto node_buf = [&](int node) {
+        BufRef r;
+        r.node = node;
+        r.ws_copy = g.nodes[node].cls != OpClass::Input && p.ws_offset[node] >= 0;
+        return r;
+      };
+      TmaDesc tw;   // weights [KO, C]
+      tw.buf = node_buf(anchor.args[1].node);
+      tw.elem_bytes = 2;
+      tw.rank = 2;
+      tw.dims[0] = (uint64_t)C; tw.dims[1] = (uint64_t)KO;
+      tw.strides[1] = (uint64_t)C * 2;
+      tw.box[0] = 64; tw.box[1] = 128;
+      TmaDesc tx;   // pixels [image][C][HW]
+      tx.buf = node_buf(anchor.args[0].node);
+      tx.elem_bytes = 2;
+      tx.rank = 3;
+      tx.dims[0] = (uint64_t)HW; tx.dims[1] = (uint64_t)C; tx.dims[2] = (uint64_t)NB;
+      tx.strides[1] = (uint64_t)HW * 2; tx.strides[2] = (uint64_t)C * HW * 2;
+      tx.box[0] = 64; tx.box[1] = 64; tx.box[2] = 1;
+      k.tmaps = {tw, tx};
+      if (tma_store) {   // result [image][KO][HW]: 32 channels x 32 pixels, 64-byte swizzle
+        TmaDesc ty;
+        ty.buf.node = grp.stores[0].node;
+        ty.buf.ws_copy = !grp.stores[0].to_output;
+        ty.elem_bytes = 2;
+        ty.rank = 3;
+        ty.dims[0] = (uint64_t)HW; ty.dims[1] = (uint64_t)KO; ty.dims[2] = (uint64_t)NB;
+        ty.strides[1] = (uint64_t)HW * 2; ty.strides[2] = (uint64_t)KO * HW * 2;
+        ty.box[0] = 32; ty.box[1] = 32; ty.box[2] = 1;
+        ty.swizzle = 2;
+        k.tmaps.push_back(ty);
+      }
+      const int64_t tiles = NB * ((HW + 255) / 256) * ((KO + 127) / 128);
+      k.block[0] = (unsigned)(64 + 32 * epw);
+      k.smem_bytes = (unsigned)(stages * (128 * 128 + 32768) + (tma_store ? epw * 4096 : 0) + 1024);
+      k.persistent = true;
+      k.max_grid = (unsigned)std::min<int64_t>(tiles, 0x7fffffff);
+      k.grid[0] = k.max_grid;
+      k.desc = "conv2d 1x1 tcgen05 bf16 as a per-image GEMM on NCHW data (weights and pixels read in place), tile 128 channels x 256 pixels";
+      out->push_back(k);
+      return;
+    }
+    // Groups (other than depthwise, which has a kernel of its own): every block of 128 filters contracts the dense
+    // window of input channels that its groups span, against weights that are zero outside each filter's own group.
+    // The window must start on a 16-byte boundary of the channels-last pixel rows for every block.
+    const int64_t G = anchor.groups, CPG = C / G, KPG = KO / G;
+    int64_t cbw = 0;    // 64-channel blocks of the widest window
+    bool grouped_ok = G > 1 && CPG > 1;
+    if (grouped_ok)
+      for (int64_t k0 = 0; k0 < KO; k0 += 128) {
+        const int64_t g_lo = k0 / KPG, g_hi = (std::min<int64_t>(k0 + 127, KO - 1)) / KPG;
+        if ((g_lo * CPG) % 8 != 0) grouped_ok = false;
+        cbw = std::max<int64_t>(cbw, ((g_hi - g_lo + 1) * CPG + 63) / 64);
+      }
+    const int64_t CWP = cbw * 64;
+    if (in_bf16 && (G == 1 || grouped_ok) && ST <= 8 && (WO * ST <= 256 || phased) && C % 8 == 0 && WO <= 256 && NB <= 0x7fffffff && FR * FS * KO <= 0x7fffffff && H <= 0x7fffff && W <= 0x7fffff) {
       // Three schedules.  (1) Rows whose byte length is a multiple of 16 and that fill most of a 32-column
       // pitch: the kernel reads NCHW itself and re-lays pixels in shared memory (conv_tc_nchw); only the
       // weights take a pre-pass.  Otherwise a pre-pass writes an NHWC copy and pixels are loaded
@@ -696,7 +772,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       // shared memory) when it stores a single bf16 tensor (output or intermediate) whose rows are 16-byte multiples.
       const bool tma_store = grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && WO % 8 == 0 && !tun.conv_no_tma_store;
       const bool x_nhwc = a.nhwc;   // the activations already are channels-last: no layout pass, and no NCHW-reading schedule
-      if (unit && dense_pitch && W % 8 == 0 && !tun.conv_no_direct && !x_nhwc) {
+      if (unit && dense_pitch && W % 8 == 0 && !tun.conv_no_direct && !x_nhwc && G == 1) {
         // shared memory: operand buffers of TH + FR - 1 rows, staging ring, output staging, and what is left for the weight ring
         const int64_t fixed = n_buf * ((th_pitch + FR - 1) * pitch * 128 + 1024) + n_stg * pitch * 128 + 1024 + (tma_store ? 16384 : 0);
         n_a = (int)std::min<int64_t>(6, (232448 - 512 - fixed) / 16384);
@@ -721,7 +797,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       const bool halo = unit && !direct && FS > 1 && dense_pitch && !tun.conv_no_halo;
       const int TH = (direct || halo) ? th_pitch : (int)std::max<int64_t>(1, std::min<int64_t>(256 / WO, std::min<int64_t>(HO, phased ? 256 : 256 / ST)));
       auto align256 = [](int64_t v) { return (v + 255) / 256 * 256; };
-      const int64_t x_bytes = (direct || x_nhwc) ? 0 : align256(NB * C * H * W * 2), w_bytes = align256(KO * C * FR * FS * 2);
+      const int64_t x_bytes = (direct || x_nhwc) ? 0 : align256(NB * C * H * W * 2), w_bytes = align256(KO * (G > 1 ? CWP : C) * FR * FS * 2);
       *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(x_bytes + w_bytes));
       auto scratch = [](int64_t off) {
         BufRef r;
@@ -740,15 +816,18 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         k.name = "hct_conv_prep_g" + std::to_string(gi);
         std::ostringstream src;
         src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_HW " << H * W << "\n#define HCT_KO " << KO
-            << "\n#define HCT_RS " << FR * FS << "\n#define HCT_PREP_X " << ((direct || x_nhwc) ? 0 : 1) << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+            << "\n#define HCT_RS " << FR * FS << "\n#define HCT_PREP_X " << ((direct || x_nhwc) ? 0 : 1) << "\n#define HCT_GROUPS " << G << "\n#define HCT_CWP " << CWP
+            << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
             << skeleton_source("common") << "\nstruct HctParams { void* ptr[4]; };\n" << skeleton_source("conv_prep");
         k.source = src.str();
         k.ptrs = {node_buf(anchor.args[0].node), node_buf(anchor.args[1].node), scratch(0), scratch(x_bytes)};
         const bool w_only = direct || x_nhwc;
-        int64_t blocks = w_only ? (KO * C * FR * FS / 8 + 255) / 256 : NB * ((C + 63) / 64) * ((H * W + 63) / 64) + (KO * C * FR * FS + 255) / 256;
+        const int64_t w_elems = KO * (G > 1 ? CWP : C) * FR * FS;
+        int64_t blocks = w_only ? (w_elems / (G > 1 ? 1 : 8) + 255) / 256 : NB * ((C + 63) / 64) * ((H * W + 63) / 64) + (w_elems + 255) / 256;
         k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(blocks, w_only ? 148 : 148 * 16));
         k.block[0] = 256;
         k.desc = w_only ? "conv weight pre-pass: KCRS->RSKC" : "conv layout pre-pass: NCHW->NHWC activations, KCRS->RSKC weights";
+        if (G > 1) k.desc += " (per filter a window of " + std::to_string(CWP) + " channels, zero outside its group)";
         out->push_back(k);
       }
       int stages = 4;
@@ -759,6 +838,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       k.name = "hct_conv_tc_bf16_g" + std::to_string(gi);
       std::ostringstream src;
       src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_H " << H << "\n#define HCT_W " << W
+          << "\n#define HCT_GROUPS " << G << "\n#define HCT_CBW " << cbw
           << "\n#define HCT_KO " << KO << "\n#define HCT_FR " << FR << "\n#define HCT_FS " << FS << "\n#define HCT_PAD " << anchor.pad
           << "\n#define HCT_STRIDE " << ST << "\n#define HCT_DIL " << DIL << "\n#define HCT_PHASED " << (phased ? 1 : 0) << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TH " << TH << "\n#define HCT_TH2 1\n#define HCT_SPLIT "
           << (flat ? 1 : TH) << "\n#define HCT_PITCH " << pitch << "\n#define HCT_NA " << (direct ? n_a : 6) << "\n#define HCT_NBUF " << (direct ? n_buf : 3)
@@ -774,8 +854,8 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       tw.buf = scratch(x_bytes);
       tw.elem_bytes = 2;
       tw.rank = 2;
-      tw.dims[0] = (uint64_t)C; tw.dims[1] = (uint64_t)(FR * FS * KO);
-      tw.strides[1] = (uint64_t)C * 2;
+      tw.dims[0] = (uint64_t)(G > 1 ? CWP : C); tw.dims[1] = (uint64_t)(FR * FS * KO);
+      tw.strides[1] = (uint64_t)(G > 1 ? CWP : C) * 2;
       tw.box[0] = 64; tw.box[1] = 128;
       TmaDesc tx;
       tx.buf = x_nhwc ? node_buf(anchor.args[0].node) : scratch(0);
@@ -839,6 +919,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       k.grid[0] = k.max_grid;
       std::ostringstream d;
       d << "conv2d tcgen05 bf16 implicit GEMM, tile 128 channels x " << TH << " rows of " << WO << " pixels, ";
+      if (G > 1) d << G << " groups as dense windows of " << CWP << " input channels per block of filters, ";
       if (flat)
         d << "NCHW read directly and re-laid in shared memory, flat tiles of 256 positions at pitch " << flat_p;
       else if (direct)
@@ -855,7 +936,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
   }
 
   if (grp.kind == GroupKind::Conv && a.nhwc)
-    throw Error(HCT_ERR_UNSUPPORTED, "a channels-last (nhwc) input needs the tensor-core convolution: bf16 operands, groups = 1, channels a multiple of 8, stride <= 8");
+    throw Error(HCT_ERR_UNSUPPORTED, "a channels-last (nhwc) input needs the tensor-core convolution: bf16 operands, channels a multiple of 8 (per group too), stride <= 8");
   for (auto& st : grp.stores)
     if (p.partial_cols[st.node] > 0)
       throw Error(HCT_ERR_UNSUPPORTED, "row sums folded into a GEMM epilogue need the tensor-core kernel (not available with simt_only)");
@@ -895,12 +976,16 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     const int64_t HOd = anchor.shape[2], WOd = anchor.shape[3];
     const bool vec = anchor.stride == 1 && anchor.dilation == 1 && xs[3] % 8 == 0 && WOd % 8 == 0 && 2 * anchor.pad <= ws[3] - 1 &&
                      ws[3] <= 7 && xs[0] * ws[0] * HOd * (WOd / 8) < 0x7fffffffLL;
-    if (vec) P = HOd >= 16 ? 8 : HOd >= 4 ? 4 : HOd >= 2 ? 2 : 1;
+    // Two filters per thread on packed multiply-adds (half the rows, so the accumulators need the same registers).
+    // Measured slower than one filter per thread (24.5 against 22.6 us on 32 x 192 x 56 x 56: 128 registers instead
+    // of 74 halve the resident warps, which costs more than the saved issue slots), so it is taken on request only.
+    const bool pair = vec && ws[0] % 2 == 0 && tun.dw_pair == 1;
+    if (vec) P = HOd >= 16 ? (pair ? 4 : 8) : HOd >= 4 ? 4 : HOd >= 2 ? 2 : 1;
     if (tun.dw_p == 1 || tun.dw_p == 2 || tun.dw_p == 4 || (tun.dw_p == 8 && vec)) P = tun.dw_p;
     const unsigned cta = (unsigned)std::min(1024, std::max(32, (tun.dw_cta > 0 ? tun.dw_cta : vec ? 128 : 256) / 32 * 32));
     const std::string epi_dw = vec ? eg.run_fn(HOd * WOd, WOd, "(row % " + std::to_string(ws[0]) + "LL)") : epi;
     k.name = "hct_conv_dw_g" + std::to_string(gi);
-    src << "#define HCT_VEC " << (vec ? 1 : 0) << "\n#define HCT_CTA " << cta << "\n";
+    src << "#define HCT_VEC " << (vec ? 1 : 0) << "\n#define HCT_PAIR " << (pair ? 1 : 0) << "\n#define HCT_CTA " << cta << "\n";
     src << "#define HCT_NB " << xs[0] << "\n#define HCT_C " << xs[1] << "\n#define HCT_MULT " << ws[0] / xs[1] << "\n#define HCT_H " << xs[2]
         << "\n#define HCT_W " << xs[3] << "\n#define HCT_FR " << ws[2] << "\n#define HCT_FS " << ws[3] << "\n#define HCT_STRIDE "
         << anchor.stride << "\n#define HCT_PAD " << anchor.pad << "\n#define HCT_DIL " << anchor.dilation << "\n#define HCT_HO "
@@ -909,10 +994,11 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         << pb << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
     src << skeleton_source("common") << "\n" << (vec ? skeleton_source("tc_common") : std::string()) << "\nstruct HctParams { void* ptr["
         << eg.ptrs.size() << "]; };\n" << epi_dw << skeleton_source("conv_dw");
-    int64_t units = xs[0] * ws[0] * ((anchor.shape[2] + P - 1) / P) * (vec ? WOd / 8 : WOd);
+    int64_t units = xs[0] * (pair ? ws[0] / 2 : ws[0]) * ((anchor.shape[2] + P - 1) / P) * (vec ? WOd / 8 : WOd);
     k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>((units + cta - 1) / cta, 148 * 64));
     k.block[0] = cta;
-    k.desc = "conv2d depthwise fp32-FMA, " + std::string(vec ? "8 columns x " : "") + std::to_string(P) + " output rows per thread";
+    k.desc = "conv2d depthwise fp32-FMA, " + std::string(vec ? "8 columns x " : "") + std::to_string(P) + " output rows" +
+             (pair ? " of two filters per thread (packed multiply-adds)" : " per thread");
   } else {
     const auto& xs = a.shape;
     const auto& ws = b.shape;

@@ -35,11 +35,14 @@ const Knob kKnobs[] = {
     {"conv_flat", &Tunables::conv_flat, 0, nullptr},
     {"dw_p", &Tunables::dw_p, 0, nullptr},
     {"dw_cta", &Tunables::dw_cta, 0, nullptr},
+    {"dw_pair", &Tunables::dw_pair, 0, nullptr},
     {"simt_only", nullptr, 0, &Tunables::simt_only},
     {"fault_never_arrive", nullptr, 0, &Tunables::fault_never_arrive},
     {"conv_no_halo", nullptr, 0, &Tunables::conv_no_halo},
     {"conv_no_tma_store", nullptr, 0, &Tunables::conv_no_tma_store},
     {"conv_no_direct", nullptr, 0, &Tunables::conv_no_direct},
+    {"conv_no_pointwise", nullptr, 0, &Tunables::conv_no_pointwise},
+    {"conv_pw_warps", &Tunables::conv_pw_warps, 0, nullptr},
     {"conv_phase", nullptr, 0, &Tunables::conv_phase},
     {"topk_no_select", nullptr, 0, &Tunables::topk_no_select},
     {"row_no_small_ctas", nullptr, 0, &Tunables::row_no_small_ctas},

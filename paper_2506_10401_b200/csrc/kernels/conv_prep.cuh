@@ -4,12 +4,39 @@
 // variant uses no shared memory and few CTAs, so that the convolution kernel, launched as a programmatic
 // dependent and needing a whole SM's shared memory per CTA, becomes resident beside it at once and
 // fills its pixel pipeline while the weights are being rearranged.
-// Defined by the generator: HCT_NB_IMG, HCT_C, HCT_HW (H*W), HCT_KO, HCT_RS (R*S), HCT_PREP_X, HctParams, HCT_KERNEL_NAME.
+// Defined by the generator: HCT_NB_IMG, HCT_C, HCT_HW (H*W), HCT_KO, HCT_RS (R*S), HCT_PREP_X, HCT_GROUPS, HCT_CWP (grouped only),
+// HctParams, HCT_KERNEL_NAME.
 // Pointer slots: 0 = X (NCHW), 1 = Wt (KCRS), 2 = X as NHWC, 3 = Wt as RSKC.
 #define HCT_XT_C ((HCT_C + 63) / 64)
 #define HCT_XT_P ((HCT_HW + 63) / 64)
 #define HCT_X_BLOCKS (HCT_PREP_X ? (long long)HCT_NB_IMG * HCT_XT_C * HCT_XT_P : 0LL)
-#define HCT_W_ELEMS ((long long)HCT_KO * HCT_C * HCT_RS)
+// Grouped convolution (HCT_GROUPS > 1, filters [KO, C / groups, R, S]): per filter the copy holds HCT_CWP channels
+// (a multiple of 64) starting at the first channel of the first group that the filter's block of 128 filters
+// spans; channels of other groups (and past C) are written as zeros, so the convolution kernel contracts a dense
+// window of input channels and the zeros cancel what does not belong to the filter's group.
+#ifndef HCT_GROUPS
+#define HCT_GROUPS 1
+#endif
+#if HCT_GROUPS > 1
+#define HCT_WC HCT_CWP
+#else
+#define HCT_WC HCT_C
+#endif
+#define HCT_W_ELEMS ((long long)HCT_KO * HCT_WC * HCT_RS)
+// element i of the copy, laid out [tap][filter][channel of the window]
+__device__ __forceinline__ hct_bf16_t hct_w_elem(const hct_bf16_t* __restrict__ Wt, long long i) {
+  const int j = (int)(i % HCT_WC);
+  const int k = (int)((i / HCT_WC) % HCT_KO);
+  const int rs = (int)(i / ((long long)HCT_WC * HCT_KO));
+#if HCT_GROUPS > 1
+  const int cpg = HCT_C / HCT_GROUPS, kpg = HCT_KO / HCT_GROUPS;
+  const int c = ((k / 128) * 128 / kpg) * cpg + j, g = k / kpg;
+  if (c >= HCT_C || c / cpg != g) return (hct_bf16_t)0;
+  return Wt[((long long)k * cpg + (c - g * cpg)) * HCT_RS + rs];
+#else
+  return Wt[((long long)k * HCT_C + j) * HCT_RS + rs];
+#endif
+}
 #if !HCT_PREP_X
 // one thread per 16-byte piece of the RSKC copy: 8 consecutive channels of one (tap, filter)
 extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParams hct_p) {
@@ -17,6 +44,10 @@ extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParam
   hct_pdl_wait();
   const hct_bf16_t* __restrict__ Wt = (const hct_bf16_t*)hct_p.ptr[1];
   hct_bf16_t* __restrict__ Wo = (hct_bf16_t*)hct_p.ptr[3];
+#if HCT_GROUPS > 1
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < HCT_W_ELEMS; i += (long long)gridDim.x * 256) Wo[i] = hct_w_elem(Wt, i);
+  return;
+#endif
   for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < HCT_W_ELEMS / 8; i += (long long)gridDim.x * 256) {
     const int c = (int)(i % (HCT_C / 8)) * 8;
     const int k = (int)((i / (HCT_C / 8)) % HCT_KO);
@@ -80,12 +111,7 @@ extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParam
       __syncthreads();
     } else {
       const long long i = (blk - HCT_X_BLOCKS) * 256 + threadIdx.x;   // index into RSKC
-      if (i < HCT_W_ELEMS) {
-        const int c = (int)(i % HCT_C);
-        const int k = (int)((i / HCT_C) % HCT_KO);
-        const int rs = (int)(i / ((long long)HCT_C * HCT_KO));
-        Wo[i] = Wt[((long long)k * HCT_C + c) * HCT_RS + rs];
-      }
+      if (i < HCT_W_ELEMS) Wo[i] = hct_w_elem(Wt, i);
     }
   }
 }

@@ -28,7 +28,16 @@
 #define HCT_A_BYTES (HCT_BM * 128)                       // weights: 128 channels x 64 inputs, bf16
 #define HCT_B_BYTES 32768                                // pixels: up to 256 x 64 inputs
 #define HCT_STAGE_BYTES (HCT_A_BYTES + HCT_B_BYTES)
+// Grouped convolution (HCT_GROUPS > 1): a block of 128 filters reads only the input channels of the groups it
+// spans.  The weight copy holds, per filter, HCT_CBW blocks of 64 channels starting at the first channel of the
+// block's first group (HCT_C_LO), zero wherever a channel is not of the filter's own group.
+#if HCT_GROUPS > 1
+#define HCT_CB HCT_CBW
+#define HCT_C_LO(mbk) ((((mbk) * HCT_BM) / (HCT_KO / HCT_GROUPS)) * (HCT_C / HCT_GROUPS))
+#else
 #define HCT_CB ((HCT_C + 63) / 64)
+#define HCT_C_LO(mbk) 0
+#endif
 #define HCT_KB (HCT_FR * HCT_FS * HCT_CB)
 #define HCT_HT ((HCT_HO + HCT_TH - 1) / HCT_TH)
 #define HCT_MBK ((HCT_KO + HCT_BM - 1) / HCT_BM)
@@ -139,10 +148,10 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
             const int a = s * HCT_DIL - HCT_PAD, b = r * HCT_DIL - HCT_PAD;
             const int wq = hct_floordiv(a), hq = hct_floordiv(b);
             const int pw = a - wq * HCT_STRIDE, ph = b - hq * HCT_STRIDE;
-            hct_tma_load_5d(dst + HCT_A_BYTES, &hct_p.tmap[1 + (t.cut ? HCT_STRIDE : 0) + ph], cb * 64, pw, wq, t.h0 + hq, t.n, full);
+            hct_tma_load_5d(dst + HCT_A_BYTES, &hct_p.tmap[1 + (t.cut ? HCT_STRIDE : 0) + ph], HCT_C_LO(t.mbk) + cb * 64, pw, wq, t.h0 + hq, t.n, full);
           }
 #else
-          hct_tma_load_4d(dst + HCT_A_BYTES, xmap, cb * 64, s * HCT_DIL - HCT_PAD, t.h0 * HCT_STRIDE + r * HCT_DIL - HCT_PAD, t.n, full);
+          hct_tma_load_4d(dst + HCT_A_BYTES, xmap, HCT_C_LO(t.mbk) + cb * 64, s * HCT_DIL - HCT_PAD, t.h0 * HCT_STRIDE + r * HCT_DIL - HCT_PAD, t.n, full);
 #endif
           if (++stage == HCT_STAGES) { stage = 0; phase ^= 1u; }
         }

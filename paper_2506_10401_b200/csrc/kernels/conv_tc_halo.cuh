@@ -19,7 +19,16 @@
 #define HCT_A_BYTES (HCT_BM * 128)                       // weights: 128 channels x 64 inputs, bf16
 #define HCT_B_BYTES 33792                                // pixels: 256 rows of 128 bytes + room for the shifted reads
 #define HCT_RING_B_OFF (HCT_NA * HCT_A_BYTES)
+// Grouped convolution (HCT_GROUPS > 1): a block of 128 filters reads only the input channels of the groups it
+// spans.  The weight copy holds, per filter, HCT_CBW blocks of 64 channels starting at the first channel of the
+// block's first group (HCT_C_LO), zero wherever a channel is not of the filter's own group.
+#if HCT_GROUPS > 1
+#define HCT_CB HCT_CBW
+#define HCT_C_LO(mbk) ((((mbk) * HCT_BM) / (HCT_KO / HCT_GROUPS)) * (HCT_C / HCT_GROUPS))
+#else
 #define HCT_CB ((HCT_C + 63) / 64)
+#define HCT_C_LO(mbk) 0
+#endif
 #define HCT_RB (HCT_FR * HCT_CB)                          // pixel buffers per tile
 #define HCT_HT ((HCT_HO + HCT_TH - 1) / HCT_TH)
 #define HCT_MBK ((HCT_KO + HCT_BM - 1) / HCT_BM)
@@ -110,7 +119,7 @@ extern "C" __global__ void __launch_bounds__(192, 1) HCT_KERNEL_NAME(const __gri
           const int r = rb / HCT_CB, cb = rb % HCT_CB;
           hct_mbar_wait(bempty0 + 8 * sb, pb ^ 1u, &failed, status, 1);
           hct_mbar_expect_tx(bfull0 + 8 * sb, bbytes);
-          hct_tma_load_4d(smem_base + HCT_RING_B_OFF + sb * HCT_B_BYTES, xmap, cb * 64, -HCT_PAD, t.h0 + r - HCT_PAD, t.n, bfull0 + 8 * sb);
+          hct_tma_load_4d(smem_base + HCT_RING_B_OFF + sb * HCT_B_BYTES, xmap, HCT_C_LO(t.mbk) + cb * 64, -HCT_PAD, t.h0 + r - HCT_PAD, t.n, bfull0 + 8 * sb);
           if (++sb == HCT_NBUF) { sb = 0; pb ^= 1u; }
           for (int s = 0; s < HCT_FS; ++s) {
             hct_mbar_wait(aempty0 + 8 * sa, pa ^ 1u, &failed, status, 5);

@@ -265,14 +265,15 @@ def test_conv_flat_tiles(kw):
     """Tiles of 256 consecutive positions (chosen by rule only when they save a K loop), forced onto other shapes:
     the chain within the bf16 tolerance, and the bare convolution bit for bit on integer-valued inputs."""
     spec, laws = configs.get_config("c4_conv_bn_relu_bf16", **kw)
-    got, want, g = parity.run_both(spec, laws, schedule="conv_flat=1")
+    ks, pad = kw.get("ksize", 3), kw.get("pad", 1)
+    schedule = "conv_flat=1" + (";conv_no_pointwise=1" if ks == 1 else "")
+    got, want, g = parity.run_both(spec, laws, schedule=schedule)
     assert "flat tiles" in g.plan
     assert parity.bf16_violation(got[0], want[0]) <= 1.0
-    ks, pad = kw.get("ksize", 3), kw.get("pad", 1)
     spec = (f"hct 1\ninput x bf16 [{kw['n']},{kw['c']},{kw['h']},{kw['w']}]\ninput w bf16 [{kw['k']},{kw['c']},{ks},{ks}]\n"
             f"node y = conv2d(x, w, stride=1, pad={pad})\nnode z = cast_bf16(y)\noutput z bf16\n")
     il = {"kind": "int", "lo": -2, "hi": 2}
-    got, want, g = parity.run_both(spec, {"x": il, "w": il}, schedule="conv_flat=1")
+    got, want, g = parity.run_both(spec, {"x": il, "w": il}, schedule=schedule)
     assert "flat tiles" in g.plan
     np.testing.assert_array_equal(got[0], want[0])
 
@@ -379,6 +380,96 @@ def test_conv_groups_integer_inputs_are_exact(dtype, shape, wshape, attrs):
     assert ("depthwise" in g.plan) == (wshape[1] == 1)
     assert ("8 columns" in g.plan) == (wshape[1] == 1 and shape[3] % 8 == 0)
     np.testing.assert_array_equal(got[0], want[0])
+
+
+@pytest.mark.parametrize("shape,ko", [
+    ((2, 32, 56, 56), 192),      # expansion of an inverted-residual block: two channel blocks, 13 pixel blocks, the last one short
+    ((3, 192, 14, 28), 32),      # projection: three blocks of input channels, a quarter of the MMA rows used
+    ((1, 72, 6, 12), 130),       # 72 pixels, channels not a multiple of 64, two filters in the second channel block
+    ((2, 8, 2, 4), 8),           # one 16-byte row per channel
+    ((1, 200, 33, 24), 40),      # 792 pixels: three full blocks and 24 pixels
+    ((5, 64, 16, 16), 256),      # whole tiles only
+])
+def test_conv_pointwise_is_a_per_image_gemm(shape, ko):
+    """1x1 convolution, stride 1, no padding, on NCHW data: weights and pixels are read where they lie.  Bare result
+    bit for bit on integer-valued inputs through both store paths (fp32: the generated epilogue's own stores;
+    bf16: shared memory and TMA stores), then a chain with per-channel operands and a residual within the bf16 tolerance."""
+    n, c, h, w = shape
+    il = {"kind": "int", "lo": -4, "hi": 4}
+    head = f"hct 1\ninput x bf16 [{n},{c},{h},{w}]\ninput w bf16 [{ko},{c},1,1]\n"
+    got, want, g = parity.run_both(head + "node y = conv2d(x, w)\noutput y f32\n", {"x": il, "w": il})
+    assert "per-image GEMM" in g.plan and g.num_kernels == 1 and g.workspace_bytes <= 256
+    np.testing.assert_array_equal(got[0], want[0])
+    got, want, g = parity.run_both(head + "node y = conv2d(x, w)\nnode z = cast_bf16(y)\noutput z bf16\n", {"x": il, "w": il})
+    assert "per-image GEMM" in g.plan and g.num_kernels == 1
+    np.testing.assert_array_equal(got[0], want[0])
+    spec = (head + f"input s f32 [{ko},1,1]\ninput b f32 [{ko},1,1]\ninput r bf16 [{n},{ko},{h},{w}]\n"
+            "node y = conv2d(x, w)\nnode a = mul(y, s)\nnode c = add(a, b)\nnode d = relu(c)\nnode e = add(d, r)\noutput e bf16\n")
+    nrm = {"kind": "normal", "mean": 0.0, "std": 1.0}
+    got, want, g = parity.run_both(spec, {"x": nrm, "w": {"kind": "normal", "mean": 0.0, "std": c ** -0.5}, "s": {"kind": "uniform", "lo": 0.5, "hi": 1.5},
+                                          "b": nrm, "r": nrm})
+    assert "per-image GEMM" in g.plan
+    assert parity.bf16_violation(got[0], want[0]) <= 1.0
+    # the general schedules stay available and agree
+    got2, _, g2 = parity.run_both(spec, {"x": nrm, "w": {"kind": "normal", "mean": 0.0, "std": c ** -0.5}, "s": {"kind": "uniform", "lo": 0.5, "hi": 1.5},
+                                         "b": nrm, "r": nrm}, schedule="conv_no_pointwise=1")
+    assert "per-image GEMM" not in g2.plan
+    assert parity.bf16_violation(got2[0], want[0]) <= 1.0
+
+
+@pytest.mark.parametrize("shape,wshape,attrs,nhwc,window", [
+    ((2, 64, 14, 16), (64, 32, 3, 3), "pad=1, groups=2", False, 64),                 # one block of filters spans both groups
+    ((1, 256, 12, 12), (256, 64, 3, 3), "pad=1, groups=4", False, 128),              # two blocks of filters, two groups each
+    ((1, 72, 9, 20), (192, 24, 3, 3), "pad=1, groups=3", False, 64),                 # windows start at channels 0 and 48; both run past their groups
+    ((1, 64, 16, 16), (96, 16, 3, 3), "stride=2, pad=1, groups=4", False, 64),       # strided pixel boxes
+    ((2, 256, 10, 10), (512, 128, 1, 1), "groups=2", False, 128),                    # a block of filters lies inside one group: nothing wasted
+    ((1, 128, 9, 20), (128, 4, 3, 3), "pad=1, groups=32", False, 128),               # four channels per group
+    ((1, 128, 20, 56), (128, 32, 3, 3), "pad=1, groups=4", False, 128),              # pixels shared by the taps of a filter row
+    ((2, 64, 14, 16), (64, 32, 3, 3), "pad=1, groups=2", True, 64),                  # channels-last input read in place
+    ((1, 128, 20, 56), (256, 32, 3, 3), "pad=1, groups=4", True, 64),
+])
+def test_conv_grouped_on_tensor_cores(shape, wshape, attrs, nhwc, window):
+    """1 < groups < channels: each block of 128 filters contracts the dense window of input channels its groups span,
+    against a weight copy that is zero outside every filter's own group.  Bit for bit on integer-valued inputs."""
+    dims = lambda t: "[" + ",".join(str(v) for v in t) + "]"
+    spec = (f"hct 1\ninput x bf16 {dims(shape)}{' nhwc' if nhwc else ''}\ninput w bf16 {dims(wshape)}\n"
+            f"node y = conv2d(x, w, {attrs})\noutput y f32\n")
+    il = {"kind": "int", "lo": -4, "hi": 4}
+    got, want, g = parity.run_both(spec, {"x": il, "w": il})
+    assert "tcgen05" in g.plan and f"dense windows of {window} input channels" in g.plan
+    np.testing.assert_array_equal(got[0], want[0])
+
+
+def test_conv_grouped_window_off_a_16_byte_boundary_takes_the_fma_kernel():
+    spec = "hct 1\ninput x bf16 [1,24,8,8]\ninput w bf16 [256,12,3,3]\nnode y = conv2d(x, w, pad=1, groups=2)\noutput y f32\n"
+    il = {"kind": "int", "lo": -4, "hi": 4}
+    got, want, g = parity.run_both(spec, {"x": il, "w": il})
+    assert "fp32-FMA" in g.plan
+    np.testing.assert_array_equal(got[0], want[0])
+
+
+@pytest.mark.parametrize("dtype,shape,wshape,attrs", [
+    ("bf16", (2, 16, 12, 24), (16, 1, 3, 3), "pad=1, groups=16"),
+    ("f32", (1, 3, 7, 16), (6, 1, 5, 5), "pad=2, groups=3"),                         # two filters per channel: a pair shares its input plane
+    ("f32", (1, 4, 5, 40), (4, 1, 1, 1), "groups=4"),
+    ("bf16", (1, 4, 9, 16), (4, 1, 5, 3), "pad=1, groups=4"),
+    ("bf16", (3, 8, 1, 8), (8, 1, 3, 3), "pad=1, groups=8"),
+    ("bf16", (2, 32, 56, 56), (32, 1, 3, 3), "pad=1, groups=32"),
+])
+def test_depthwise_two_filters_per_thread(dtype, shape, wshape, attrs):
+    """The opt-in schedule with packed multiply-adds (filters k and k+1 in the two halves): same results bit for bit."""
+    dims = lambda t: "[" + ",".join(str(v) for v in t) + "]"
+    spec = f"hct 1\ninput x {dtype} {dims(shape)}\ninput w {dtype} {dims(wshape)}\nnode y = conv2d(x, w, {attrs})\noutput y f32\n"
+    il = {"kind": "int", "lo": -4, "hi": 4}
+    got, want, g = parity.run_both(spec, {"x": il, "w": il}, schedule="dw_pair=1")
+    assert "two filters per thread" in g.plan
+    np.testing.assert_array_equal(got[0], want[0])
+    spec, laws = configs.get_config("dwconv_bn_relu", n=2, c=48, h=28, w=24)
+    got, want, g = parity.run_both(spec, laws, schedule="dw_pair=1")
+    assert "two filters per thread" in g.plan
+    got1, _, _ = parity.run_both(spec, laws)
+    np.testing.assert_array_equal(got[0], got1[0])      # each half is an ordinary fused multiply-add
+    assert parity.bf16_violation(got[0], want[0]) <= 1.0
 
 
 @pytest.mark.parametrize("kw", [dict(n=2, c=48, h=28, w=28), dict(n=1, c=16, h=15, w=21, stride=2), dict(n=2, c=192, h=56, w=56)])
