@@ -21,7 +21,11 @@
  *                                             the buffer is channels-last, x[n][h][w][c] (only as conv2d's first
  *                                             operand: such a convolution needs no layout pass over its activations)
  *     node   NAME = OP(arg, ..., key=value)   args: earlier names or (binary ops) a number
- *     output NAME [DTYPE]                     stored dtype, default f32
+ *     output NAME [DTYPE [nhwc]]              stored dtype, default f32; `nhwc` after the dtype of a rank-4 value says the
+ *                                             output buffer is channels-last, y[n][h][w][c] (extents stay [N,C,H,W]); only
+ *                                             for values stored by a convolution kernel (the convolution or the elementwise
+ *                                             nodes fused behind it), otherwise HCT_ERR_UNSUPPORTED.  With an nhwc input
+ *                                             and an nhwc output a chain of graphs stays channels-last with no layout pass
  *
  *   unary   relu gelu_tanh gelu_erf sigmoid exp tanh sqrt sin cos neg abs log rsqrt square reciprocal
  *           cast_bf16(x)   rounds to bfloat16 (nearest even); the result may be the first operand of a bf16
@@ -56,8 +60,13 @@
  *   conv2d(x, w, stride=1, pad=0, dilation=1, groups=1)   x[N,C,H,W], w[K,C/groups,R,S]; cross-correlation,
  *                         zero padding; y[n,k,h,w] = sum x[n,c,h*stride-pad+r*dilation, w*stride-pad+s*dilation] * w[k,c',r,s]
  *                         over the C/groups channels c of filter k's group (groups = C: depthwise).
- *                         bf16 operands with groups = 1 run on tensor cores (strides up to 8); depthwise
- *                         and grouped convolutions run on fp32 FMA kernels
+ *                         bf16 operands run on tensor cores (strides up to 8): 1x1 at stride 1 on NCHW data as one
+ *                         GEMM per image with no layout pass at all; groups between 1 and C by contracting, per
+ *                         block of 128 filters, the dense window of input channels its groups span against weights
+ *                         that are zero outside each filter's own group (so a non-finite activation in one group
+ *                         makes NaN in the results of the other groups of its window, where the definition gives a
+ *                         finite value).  Depthwise convolutions, fp32 operands and grouped shapes whose windows do
+ *                         not start on 16-byte boundaries run on fp32 FMA kernels
  *
  * Every computed value is fp32; bf16 inputs are widened exactly; an output
  * stored as bf16 is rounded to nearest-even once, at the store.
@@ -190,6 +199,8 @@ HCT_API int hct_graph_num_kernels(const hct_graph_t* g);
 /* Memory layout of input `idx`: 0 = row-major in the declared order of extents (NCHW for rank 4),
  * 1 = declared `nhwc`: extents are still reported as [N,C,H,W], the buffer holds x[n][h][w][c].  -1: bad index. */
 HCT_API int hct_graph_input_layout(const hct_graph_t* g, int idx);
+/* Memory layout of output `idx`, same codes: 1 = declared `output NAME DTYPE nhwc`. */
+HCT_API int hct_graph_output_layout(const hct_graph_t* g, int idx);
 /*
  * Work accounting for roofline figures.  algorithmic_bytes: every graph input
  * read once and every output written once, plus one write and one read for

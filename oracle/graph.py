@@ -38,6 +38,7 @@ class Graph:
     nodes: dict = field(default_factory=dict)   # name -> Node, insertion order = evaluation order
     inputs: list = field(default_factory=list)
     outputs: list = field(default_factory=list)  # (name, dtype)
+    output_layouts: dict = field(default_factory=dict)  # name -> "nhwc" for outputs declared channels-last
 
 
 _NAME = re.compile(r"^[A-Za-z_][A-Za-z0-9_]*$")
@@ -123,10 +124,13 @@ def parse(text: str) -> Graph:
             g.nodes[name] = _infer(g, name, op, pos, attrs, where)
         elif kw == "output":
             toks = line.split()
-            if len(toks) not in (2, 3):
+            if len(toks) not in (2, 3, 4):
                 raise SpecError(f"{where}: malformed output")
             name = toks[1]
-            dtype = toks[2] if len(toks) == 3 else "f32"
+            dtype = toks[2] if len(toks) >= 3 else "f32"
+            layout = toks[3] if len(toks) == 4 else "nchw"
+            if layout not in ("nchw", "nhwc"):
+                raise SpecError(f"{where}: unknown layout {layout!r}")
             if name not in g.nodes:
                 raise SpecError(f"{where}: output {name!r} is not defined")
             if dtype not in ("f32", "bf16"):
@@ -135,6 +139,10 @@ def parse(text: str) -> Graph:
                 raise SpecError(f"{where}: an input cannot be an output")
             if name in [o for o, _ in g.outputs]:
                 raise SpecError(f"{where}: duplicate output")
+            if layout == "nhwc":
+                if len(g.nodes[name].shape) != 4:
+                    raise SpecError(f"{where}: nhwc needs an output of rank 4")
+                g.output_layouts[name] = "nhwc"    # a matter of the caller's buffer only: values and extents stay [N,C,H,W]
             g.outputs.append((name, dtype))
         else:
             raise SpecError(f"{where}: unknown statement {kw!r}")

@@ -19,6 +19,7 @@ EXPORTS = [
     "hct_graph_cost", "hct_graph_plan_text", "hct_graph_kernel_source", "hct_graph_kernel_name", "hct_last_error",
     "hct_version", "hct_gemm_bias_relu_f32_static", "hct_graph_create_scheduled", "hct_graph_autotune", "hct_graph_schedule",
     "hct_graph_input_layout",
+    "hct_graph_output_layout",
 ]
 
 HCT_STATIC_SCRATCH_BYTES = 8 << 20
@@ -61,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.hct_graph_workspace_bytes.restype = sz
         L.hct_graph_input_layout.argtypes = [vp, ci]
         L.hct_graph_input_layout.restype = ci
+        L.hct_graph_output_layout.argtypes = [vp, ci]
+        L.hct_graph_output_layout.restype = ci
         L.hct_graph_num_kernels.argtypes = [vp]
         L.hct_graph_num_kernels.restype = ci
         L.hct_graph_cost.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
@@ -164,6 +167,10 @@ def hct_graph_workspace_bytes(g) -> int:
 
 def hct_graph_input_layout(g, idx: int) -> int:
     return lib().hct_graph_input_layout(g, idx)
+
+
+def hct_graph_output_layout(g, idx: int) -> int:
+    return lib().hct_graph_output_layout(g, idx)
 
 
 def hct_graph_num_kernels(g) -> int:

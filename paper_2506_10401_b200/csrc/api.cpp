@@ -470,6 +470,11 @@ int hct_graph_input_layout(const hct_graph_t* g, int idx) {
   return g->graph.nodes[g->graph.inputs[idx]].nhwc ? 1 : 0;
 }
 
+int hct_graph_output_layout(const hct_graph_t* g, int idx) {
+  if (!g || idx < 0 || idx >= (int)g->graph.outputs.size()) return -1;
+  return g->graph.nodes[g->graph.outputs[idx]].out_nhwc ? 1 : 0;
+}
+
 hct_status_t hct_graph_cost(const hct_graph_t* g, double* algorithmic_bytes, double* flops) {
   if (!g) return set_error(HCT_ERR_INVALID_ARG, "graph is NULL");
   if (algorithmic_bytes) *algorithmic_bytes = g->plan.algorithmic_bytes;

@@ -17,6 +17,10 @@ struct EpiGen {
   const Group& grp;
   int gi;
   std::vector<BufRef> ptrs;
+  int64_t conv_ko = 0, conv_hw = 0;   // output channels and pixels per plane of a convolution group (for channels-last stores)
+
+  // A graph output declared nhwc: element (n, k, pixel) of the [N,K,H,W] value goes to ((n * HW + pixel) * K + k).
+  bool nhwc_store(const Store& st) const { return st.to_output && g.nodes[st.node].out_nhwc; }
 
   int ptr_index(int node, bool ws_copy) {
     for (size_t i = 0; i < ptrs.size(); ++i)
@@ -60,6 +64,12 @@ struct EpiGen {
     }
     for (auto& s : grp.stores) {
       int pi = ptr_index(s.node, !s.to_output);
+      if (nhwc_store(s)) {
+        if (conv_ko <= 0) throw Error(HCT_ERR_UNSUPPORTED, "an nhwc output must be produced by a convolution kernel");
+        f << "  hct_st1((" << ctype(s.dtype) << "*)hct_p.ptr[" << pi << "] + ((ri / " << conv_ko << "LL) * " << conv_hw << "LL + off % " << conv_hw
+          << "LL) * " << conv_ko << "LL + ci, e" << s.node << ");\n";
+        continue;
+      }
       f << "  hct_st1((" << ctype(s.dtype) << "*)hct_p.ptr[" << pi << "] + off, e" << s.node << ");\n";
     }
     f << "}\n";
@@ -156,6 +166,13 @@ struct EpiGen {
         f << "  ((float*)hct_p.ptr[" << pi << "])[row * " << p.partial_cols[st.node] << "LL + (col0 >> 5)] = ps" << st.node << ";\n";
         continue;
       }
+      if (nhwc_store(st)) {   // consecutive lanes hold consecutive channels: every store of a warp covers 32 neighbouring elements
+        if (conv_ko <= 0 || N != conv_hw) throw Error(HCT_ERR_UNSUPPORTED, "an nhwc output must be produced by a convolution kernel");
+        f << "  {\n    " << ctype(st.dtype) << "* q = (" << ctype(st.dtype) << "*)hct_p.ptr[" << pi << "] + ((row / " << conv_ko << "LL) * " << N
+          << "LL + col0) * " << conv_ko << "LL + row % " << conv_ko << "LL;\n    _Pragma(\"unroll\") for (int j = 0; j < 32; ++j) if (j < ncols) hct_st1(q + j * "
+          << conv_ko << "LL, o" << st.node << "_1[j]);\n  }\n";
+        continue;
+      }
       const int w = part_w(st.dtype);
       if (w)
         f << "  hct_st_run32w<" << w << ">((" << ctype(st.dtype) << "*)hct_p.ptr[" << pi << "] + row * " << N << "LL + col0, o" << st.node << "_"
@@ -228,6 +245,14 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
   const Node& a = g.nodes[anchor.args[0].node];
   const Node& b = g.nodes[anchor.args[anchor.args.size() > 1 ? 1 : 0].node];   // transpose and sort have one operand
   EpiGen eg{g, p, grp, gi, {}};
+  bool nhwc_out = false;   // some graph output of this group is declared channels-last
+  for (auto& st : grp.stores) nhwc_out = nhwc_out || eg.nhwc_store(st);
+  if (grp.kind == GroupKind::Conv) {
+    eg.conv_ko = anchor.shape[1];
+    eg.conv_hw = anchor.shape[2] * anchor.shape[3];
+  } else if (nhwc_out) {
+    throw Error(HCT_ERR_UNSUPPORTED, "an nhwc output must be produced by a convolution kernel");
+  }
 
   // ---- reshape: flat copy through the generated epilogue
   if (grp.kind == GroupKind::Reshape) {
@@ -676,7 +701,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     if (in_bf16 && anchor.groups == 1 && FR == 1 && FS == 1 && ST == 1 && anchor.pad == 0 && !a.nhwc && (H * W) % 8 == 0 && C % 8 == 0 &&
         NB <= 0x7fffffff && KO <= 0x7fffffff && H * W <= 0x7fffffff && !tun.conv_no_pointwise) {
       const int64_t HW = H * W;
-      const bool tma_store = grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && !tun.conv_no_tma_store;
+      const bool tma_store = grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && !tun.conv_no_tma_store && !nhwc_out;
       const int epw = tun.conv_pw_warps == 8 ? 8 : 16;
       const int stages = tma_store && epw == 16 ? 3 : 4;
       std::string epi = eg.run_fn(HW, 32, "(row % " + std::to_string(KO) + "LL)", tma_store);
@@ -770,14 +795,14 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       const int64_t flat_buf = (flat_win * 128 + 1023) / 1024 * 1024;
       // The epilogue of the NCHW-reading kernel hands its bf16 output to TMA stores (through 16 KB of
       // shared memory) when it stores a single bf16 tensor (output or intermediate) whose rows are 16-byte multiples.
-      const bool tma_store = grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && WO % 8 == 0 && !tun.conv_no_tma_store;
+      const bool tma_store = grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && WO % 8 == 0 && !tun.conv_no_tma_store && !nhwc_out;
       const bool x_nhwc = a.nhwc;   // the activations already are channels-last: no layout pass, and no NCHW-reading schedule
       if (unit && dense_pitch && W % 8 == 0 && !tun.conv_no_direct && !x_nhwc && G == 1) {
         // shared memory: operand buffers of TH + FR - 1 rows, staging ring, output staging, and what is left for the weight ring
         const int64_t fixed = n_buf * ((th_pitch + FR - 1) * pitch * 128 + 1024) + n_stg * pitch * 128 + 1024 + (tma_store ? 16384 : 0);
         n_a = (int)std::min<int64_t>(6, (232448 - 512 - fixed) / 16384);
         direct = n_a >= 3;
-        if (direct && grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && WO >= 32 && FS - 1 <= 4 && flat_p <= pitch && tun.conv_flat != 2) {
+        if (direct && grp.stores.size() == 1 && grp.stores[0].dtype == BF16 && WO >= 32 && FS - 1 <= 4 && flat_p <= pitch && tun.conv_flat != 2 && !nhwc_out) {
           const int64_t row_tiles = NB * ((HO + th_pitch - 1) / th_pitch) * ((KO + 127) / 128);
           const int64_t loops_row = row_tiles / 148 + (row_tiles % 148 ? 1 : 0), loops_flat = (flat_tiles + 147) / 148;
           const int64_t fixed_flat = n_buf * flat_buf + n_stg * pitch * 128 + 1024 + 16384;

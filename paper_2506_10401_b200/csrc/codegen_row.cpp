@@ -168,6 +168,8 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   const Group& grp = p.groups[gi];
   const int64_t R = grp.R, C = grp.C;
   if (C > (1 << 17)) throw Error(HCT_ERR_UNSUPPORTED, "rows longer than 131072 elements are not supported");
+  for (auto& st : grp.stores)
+    if (st.to_output && g.nodes[st.node].out_nhwc) throw Error(HCT_ERR_UNSUPPORTED, "an nhwc output must be produced by a convolution kernel");
 
   // vector width from alignment of every full-width buffer: rows start at multiples of C elements
   int V = (C % 4 == 0) ? 4 : (C % 2 == 0) ? 2 : 1;

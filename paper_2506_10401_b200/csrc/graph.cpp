@@ -420,10 +420,11 @@ Graph parse_spec(const std::string& text) {
       index[name] = (int)g.nodes.size();
       g.nodes.push_back(n);
     } else if (kw == "output") {
-      std::string name, dtype, extra;
+      std::string name, dtype, layout, extra;
       ls >> name;
       bool has_dtype = (bool)(ls >> dtype);
-      if (name.empty() || (ls >> extra)) fail(HCT_ERR_PARSE, line, "malformed output, expected: output NAME [DTYPE]");
+      bool has_layout = (bool)(ls >> layout);
+      if (name.empty() || (ls >> extra)) fail(HCT_ERR_PARSE, line, "malformed output, expected: output NAME [DTYPE [LAYOUT]]");
       auto it = index.find(name);
       if (it == index.end()) fail(HCT_ERR_GRAPH, line, "output '" + name + "' is not defined");
       Node& n = g.nodes[it->second];
@@ -435,6 +436,13 @@ Graph parse_spec(const std::string& text) {
         n.out_dtype = BF16;
       else
         fail(HCT_ERR_PARSE, line, "unknown dtype '" + dtype + "'");
+      if (has_layout) {
+        if (layout == "nhwc")
+          n.out_nhwc = true;
+        else if (layout != "nchw")
+          fail(HCT_ERR_PARSE, line, "unknown layout '" + layout + "' (nchw or nhwc)");
+        if (n.out_nhwc && n.shape.size() != 4) fail(HCT_ERR_UNSUPPORTED, line, "the nhwc layout is supported for outputs of rank 4");
+      }
       n.output_index = (int)g.outputs.size();
       g.outputs.push_back(it->second);
     } else {

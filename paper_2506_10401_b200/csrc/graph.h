@@ -40,6 +40,7 @@ struct Node {
   uint64_t drop_seed = 0;
   unsigned drop_threshold = 0;
   int input_index = -1;   // position among `input` lines
+  bool out_nhwc = false;  // output only: the output buffer of this rank-4 value is laid out [N,H,W,C]
   bool nhwc = false;      // input only: a rank-4 tensor [N,C,H,W] whose buffer is laid out [N,H,W,C] (channels contiguous)
   int output_index = -1;  // position among `output` lines
   DType out_dtype = F32;  // storage dtype when the node is a graph output

@@ -16,6 +16,7 @@ class FusedGraph:
         self.inputs = [B.hct_graph_tensor_info(self.handle, False, i) for i in range(self.n_in)]
         self.outputs = [B.hct_graph_tensor_info(self.handle, True, i) for i in range(self.n_out)]
         self.input_nhwc = [B.hct_graph_input_layout(self.handle, i) == 1 for i in range(self.n_in)]
+        self.output_nhwc = [B.hct_graph_output_layout(self.handle, i) == 1 for i in range(self.n_out)]
         self.workspace_bytes = B.hct_graph_workspace_bytes(self.handle)
         self._ws = None
 
@@ -59,8 +60,10 @@ class FusedGraph:
     def alloc_outputs(self):
         import torch
         outs = []
-        for _, dtype, shape in self.outputs:
-            outs.append(torch.empty(shape, dtype=torch.bfloat16 if dtype == B.HCT_BF16 else torch.float32, device=f"cuda:{self.device}"))
+        for (_, dtype, shape), nhwc in zip(self.outputs, self.output_nhwc):
+            # an output declared nhwc is a [N,C,H,W] tensor in torch's channels-last memory format
+            outs.append(torch.empty(shape, dtype=torch.bfloat16 if dtype == B.HCT_BF16 else torch.float32, device=f"cuda:{self.device}",
+                                    memory_format=torch.channels_last if nhwc else torch.contiguous_format))
         return outs
 
     def workspace(self):

@@ -185,3 +185,32 @@ def test_extents_out_of_range_are_rejected_not_wrapped():
     spec = "hct 1\ninput x f32 [8,64]\nnode y = dropout(x, p=0.5, seed=99999999999999999999)\noutput y\n"
     with pytest.raises(hct.HctError):
         hct.hct_graph_create(spec, hct.HCT_DEVICE_NONE)
+
+
+def test_layout_words_on_inputs_and_outputs():
+    """`nhwc` on an input or an output is a statement about the caller's buffer: extents stay [N,C,H,W].  Both readers
+    accept and reject the same specs; an nhwc output must come out of a convolution kernel."""
+    conv = "hct 1\ninput x bf16 [2,16,8,8] nhwc\ninput w bf16 [8,16,3,3]\nnode y = conv2d(x, w, pad=1)\nnode z = relu(y)\n"
+    h = hct.hct_graph_create(conv + "output z bf16 nhwc\n", NONE)
+    assert binding.hct_graph_input_layout(h, 0) == 1 and binding.hct_graph_input_layout(h, 1) == 0
+    assert binding.hct_graph_output_layout(h, 0) == 1 and binding.hct_graph_output_layout(h, 1) == -1
+    assert binding.hct_graph_tensor_info(h, True, 0)[2] == (2, 8, 8, 8)
+    hct.hct_graph_destroy(h)
+    g = oracle.parse(conv + "output z bf16 nhwc\n")
+    assert g.output_layouts == {"z": "nhwc"} and g.nodes["z"].shape == (2, 8, 8, 8)
+    h = hct.hct_graph_create(conv + "output z bf16 nchw\n", NONE)
+    assert binding.hct_graph_output_layout(h, 0) == 0
+    hct.hct_graph_destroy(h)
+    assert oracle.parse(conv + "output z bf16 nchw\n").output_layouts == {}
+    for tail, code in (("output z bf16 nwhc\n", hct.HCT_ERR_PARSE), ("output z bf16 nhwc extra\n", hct.HCT_ERR_PARSE)):
+        assert _code(conv + tail) == code
+        with pytest.raises(oracle.SpecError):
+            oracle.parse(conv + tail)
+    flat = "hct 1\ninput x f32 [4,8]\nnode y = relu(x)\noutput y f32 nhwc\n"          # rank 2
+    assert _code(flat) == hct.HCT_ERR_UNSUPPORTED
+    with pytest.raises(oracle.SpecError):
+        oracle.parse(flat)
+    # a rank-4 value that no convolution kernel stores: valid spec, not supported by this library
+    rows = "hct 1\ninput x f32 [2,3,4,8]\nnode y = relu(x)\noutput y f32 nhwc\n"
+    oracle.parse(rows)
+    assert _code(rows) == hct.HCT_ERR_UNSUPPORTED

@@ -299,6 +299,65 @@ def test_conv_channels_last_input_is_read_in_place(shape, wshape, attrs):
     np.testing.assert_array_equal(got[0], want[0])
 
 
+@pytest.mark.parametrize("body", [
+    "input x bf16 [2,64,14,16]\ninput w bf16 [96,64,3,3]\nnode y = conv2d(x, w, pad=1)\noutput y bf16 nhwc\n",               # one box per tap
+    "input x bf16 [2,64,14,16] nhwc\ninput w bf16 [96,64,3,3]\nnode y = conv2d(x, w, stride=2, pad=1)\noutput y f32 nhwc\n",   # channels-last in and out
+    "input x bf16 [2,32,56,56]\ninput w bf16 [72,32,1,1]\nnode y = conv2d(x, w)\noutput y bf16 nhwc\n",                        # per-image GEMM
+    "input x bf16 [2,128,20,56]\ninput w bf16 [130,128,3,3]\nnode y = conv2d(x, w, pad=1)\noutput y f32 nhwc\n",               # NCHW read directly
+    "input x bf16 [1,72,17,40] nhwc\ninput w bf16 [40,72,5,5]\nnode y = conv2d(x, w, pad=2)\noutput y bf16 nhwc\n",             # pixels shared by a filter row
+    "input x bf16 [2,16,12,24]\ninput w bf16 [16,1,3,3]\nnode y = conv2d(x, w, pad=1, groups=16)\noutput y bf16 nhwc\n",        # depthwise, 8 columns per thread
+    "input x bf16 [1,6,9,7]\ninput w bf16 [6,1,3,3]\nnode y = conv2d(x, w, pad=1, groups=6)\noutput y f32 nhwc\n",              # depthwise, one column per thread
+    "input x f32 [2,6,8,8]\ninput w f32 [4,6,3,3]\nnode y = conv2d(x, w, pad=1)\noutput y f32 nhwc\n",                          # fp32-FMA kernel
+    "input x bf16 [2,64,14,16]\ninput w bf16 [64,32,3,3]\nnode y = conv2d(x, w, pad=1, groups=2)\noutput y bf16 nhwc\n",        # grouped
+])
+def test_conv_channels_last_output(body):
+    """An output declared nhwc: same values as the NCHW graph, written channels-last into the caller's buffer."""
+    import torch
+    # a bf16 output is rounded: state the rounding as a node, so that the oracle's value is the rounded one
+    spec = "hct 1\n" + body.replace("output y bf16 nhwc", "node z = cast_bf16(y)\noutput z bf16 nhwc")
+    il = {"kind": "int", "lo": -4, "hi": 4}
+    t = configs.draw_inputs(spec, {"x": il, "w": il}, 0)
+    ref = list(parity.oracle_reference(spec, parity.oracle_inputs(spec, t)).values())[0]
+    g = hct_graph(spec)
+    assert g.output_nhwc == [True]
+    out = g.run(parity.to_device(spec, t))[0]
+    torch.cuda.synchronize()
+    g.status()
+    assert out.is_contiguous(memory_format=torch.channels_last) and tuple(out.shape) == ref.shape
+    np.testing.assert_array_equal(parity.to_numpy64(out), ref)
+    # the buffer itself, read as [N,H,W,C]
+    raw = torch.as_strided(out, (out.shape[0], out.shape[2], out.shape[3], out.shape[1]),
+                           (out.shape[1] * out.shape[2] * out.shape[3], out.shape[3] * out.shape[1], out.shape[1], 1))
+    np.testing.assert_array_equal(parity.to_numpy64(raw), np.transpose(np.asarray(ref), (0, 2, 3, 1)))
+
+
+def test_conv_channels_last_between_two_graphs():
+    """A channels-last pipeline across graphs: the first graph's nhwc output is the second graph's nhwc input, with no
+    layout pass over the activations in either; compared with the oracle's run of the two convolutions as one graph."""
+    import torch
+    one = ("hct 1\ninput x bf16 [2,64,28,28] nhwc\ninput w1 bf16 [128,64,3,3]\ninput s f32 [128,1,1]\nnode a = conv2d(x, w1, stride=2, pad=1)\n"
+           "node b = mul(a, s)\nnode c = relu(b)\noutput c bf16 nhwc\n")
+    two = "hct 1\ninput c bf16 [2,128,14,14] nhwc\ninput w2 bf16 [64,128,3,3]\nnode y = conv2d(c, w2, pad=1)\noutput y f32 nhwc\n"
+    both = ("hct 1\ninput x bf16 [2,64,28,28]\ninput w1 bf16 [128,64,3,3]\ninput s f32 [128,1,1]\ninput w2 bf16 [64,128,3,3]\n"
+            "node a = conv2d(x, w1, stride=2, pad=1)\nnode b = mul(a, s)\nnode c0 = relu(b)\nnode c = cast_bf16(c0)\nnode y = conv2d(c, w2, pad=1)\noutput y f32\n")
+    il = {"kind": "int", "lo": -2, "hi": 2}
+    t = configs.draw_inputs(both, {"x": il, "w1": il, "w2": il, "s": {"kind": "int", "lo": 1, "hi": 2}}, 0)
+    ref = parity.oracle_reference(both, parity.oracle_inputs(both, t))["y"]
+    dev = dict(zip(["x", "w1", "s", "w2"], parity.to_device(both, t)))
+    g1, g2 = hct_graph(one), hct_graph(two)
+    assert "NHWC activations" not in g1.plan and "NHWC activations" not in g2.plan
+    c = g1.run([dev["x"].contiguous(memory_format=torch.channels_last), dev["w1"], dev["s"]])[0]
+    y = g2.run([c, dev["w2"]])[0]
+    torch.cuda.synchronize()
+    g1.status(); g2.status()
+    np.testing.assert_array_equal(parity.to_numpy64(y), ref)
+
+
+def hct_graph(spec, schedule=None):
+    import paper_2506_10401_b200 as hct
+    return hct.FusedGraph(spec, 0, schedule=schedule)
+
+
 def test_conv_channels_last_chain():
     spec, laws = configs.get_config("c4_conv_bn_relu_bf16", n=2, c=64, h=56, w=56, k=128, stride=2, pad=1, nhwc=True)
     check_bf16(spec, laws)
