@@ -50,6 +50,9 @@ WORKLOADS = {
     "dwconv_bn_relu": dict(bound="hbm", sample=dict(n=8)),
     "topk_bias_relu": dict(bound="hbm", sample=dict(r=2048)),
     "mbconv_block": dict(bound="hbm", sample=dict(n=4)),
+    # more than one block: three inverted-residual blocks with a stride-2 transition, and a bottleneck with a grouped 3x3
+    "mobilenet_stage": dict(bound="hbm", sample=dict(n=2)),
+    "resnext_block": dict(bound="hbm", sample=dict(n=4)),
 }
 HEADLINE = "c2_softmax_layernorm_chain"
 SMALL_BYTES = 24 * 1024 * 1024
@@ -566,7 +569,7 @@ def roofline_of(name, r, pk):
 
 
 def dtype_of(name):
-    return "bf16" if ("bf16" in name or name in ("matmul_dropout_mean_softmax", "conv_block", "dwconv_bn_relu", "mbconv_block", "conv_s2_bn_relu", "conv_s2_bn_relu_nhwc")) else "f32"
+    return "bf16" if ("bf16" in name or name in ("matmul_dropout_mean_softmax", "conv_block", "dwconv_bn_relu", "mbconv_block", "conv_s2_bn_relu", "conv_s2_bn_relu_nhwc", "mobilenet_stage", "resnext_block")) else "f32"
 
 
 def sweep_record(steps, warmup, device, out_path, tune):

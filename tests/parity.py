@@ -13,6 +13,7 @@ Tolerances (written here once, used by every GPU test):
     The strict figure (largest |g - r| / |r|, no allowance for cancellation) is recorded for every
     comparison and printed at the end of the run, ungraded.
   * bf16-input, fp32-accumulate contractions with bf16 output: |g - r| <= 1e-2 + 2e-2 * |r|.
+  * graphs of several blocks (six or more contractions in a row, bf16 between them): see bf16_deep_chain_check.
 """
 from __future__ import annotations
 
@@ -124,6 +125,23 @@ def bf16_violation(got, ref):
         return float("inf")
     ref = np.asarray(ref)
     return float((np.abs(got - ref) / (TOL_BF16_ABS + TOL_BF16_REL * np.abs(ref))).max())
+
+
+def bf16_deep_chain_check(got, ref):
+    """Several contractions in a row with bf16 roundings between them.  The oracle rounds fp64 values at every
+    cast_bf16, the kernels fp32 ones: where the two straddle a rounding boundary the intermediate differs by one bf16
+    unit (2^-8 relative), later sums amplify that wherever they cancel, and later roundings can flip in turn.  So the
+    single-contraction rule is asked of all but one element in a thousand, and of every element with |r| replaced by
+    the larger of |r| and the largest magnitude of its (n,k) plane (the scale of the terms that cancel).
+    Returns (share of elements outside the plain rule, largest violation of the plane-scale rule)."""
+    assert got.shape == ref.shape, (got.shape, ref.shape)
+    if not np.all(np.isfinite(got)):
+        return 1.0, float("inf")
+    ref = np.asarray(ref)
+    diff = np.abs(got - ref)
+    plain = diff / (TOL_BF16_ABS + TOL_BF16_REL * np.abs(ref))
+    scaled = diff / (TOL_BF16_ABS + TOL_BF16_REL * np.maximum(np.abs(ref), row_scale(ref)))
+    return float(np.mean(plain > 1.0)), float(scaled.max())
 
 
 def run_both(spec, laws, seed=0, device=0, schedule=None):

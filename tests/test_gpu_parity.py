@@ -545,6 +545,27 @@ def test_inverted_residual_block(kw):
     assert parity.bf16_violation(got[0], want[0]) <= 1.0
 
 
+@pytest.mark.parametrize("kw", [dict(n=1, c=8, h=8, w=8, expand=2, blocks=3, c_out=16), dict(n=2, c=32, h=28, w=24, blocks=3, c_out=64),
+                                dict(n=2, c=16, h=56, w=56, expand=6, blocks=2, c_out=24)])
+def test_mobilenet_stage(kw):
+    """Several inverted-residual blocks and a stride-2 transition as ONE graph: nine convolution kernels, every
+    activation between them kept as bf16 on the device."""
+    spec, laws = configs.get_config("mobilenet_stage", **kw)
+    got, want, g = parity.run_both(spec, laws)
+    assert g.plan.count("depthwise") == kw["blocks"] and g.num_kernels >= 3 * kw["blocks"]
+    outside, worst = parity.bf16_deep_chain_check(got[0], want[0])
+    assert outside <= 1e-3 and worst <= 1.0, (outside, worst)
+
+
+@pytest.mark.parametrize("kw", [dict(n=1, c=32, h=6, w=8, width=16, groups=2), dict(n=2, c=256, h=28, w=28), dict(n=1, c=64, h=14, w=14, width=64, groups=4)])
+def test_resnext_block(kw):
+    """A bottleneck whose 3x3 convolution is grouped: all three convolutions on tensor cores."""
+    spec, laws = configs.get_config("resnext_block", **kw)
+    got, want, g = parity.run_both(spec, laws)
+    assert g.plan.count("tcgen05") == 3 and "dense windows" in g.plan
+    assert parity.bf16_violation(got[0], want[0]) <= 1.0
+
+
 # ------------------------------------------------------------------ stacked contractions through bf16 intermediates
 
 @pytest.mark.parametrize("kw", [dict(n=2, c=64, h=20, w=24, k=64), dict(n=1, c=128, h=56, w=56, k=128), dict(n=2, c=16, h=9, w=11, k=32)])

@@ -186,6 +186,74 @@ output y bf16
     return spec, laws
 
 
+def mobilenet_stage(n=32, c=32, h=56, w=56, expand=6, blocks=3, c_out=64):
+    """Several inverted-residual blocks in a row, as one graph (MobileNetV2 repeats its block within a stage and changes
+    resolution and width between stages): `blocks` - 1 blocks of `c` channels at stride 1 with their residuals, then a
+    block whose depthwise convolution has stride 2 and whose projection gives `c_out` channels, without a residual.
+    Every activation between two convolutions is rounded to bf16 and stays on the device."""
+    e = c * expand
+    lines = ["hct 1", f"input x bf16 [{n},{c},{h},{w}]"]
+    laws = {"x": _n()}
+    nodes = []
+    cur = "x"
+    for i in range(blocks):
+        last = i == blocks - 1
+        co = c_out if last else c
+        for nm, shp, law in ((f"w1_{i}", f"[{e},{c},1,1]", _n(math.sqrt(2.0 / c))), (f"s1_{i}", f"[{e},1,1]", _u(0.5, 1.5)), (f"b1_{i}", f"[{e},1,1]", _n(0.1)),
+                             (f"w2_{i}", f"[{e},1,3,3]", _n(math.sqrt(2.0 / 9))), (f"s2_{i}", f"[{e},1,1]", _u(0.5, 1.5)), (f"b2_{i}", f"[{e},1,1]", _n(0.1)),
+                             (f"w3_{i}", f"[{co},{e},1,1]", _n(math.sqrt(1.0 / e))), (f"s3_{i}", f"[{co},1,1]", _u(0.5, 1.5)), (f"b3_{i}", f"[{co},1,1]", _n(0.1))):
+            lines.append(f"input {nm} {'bf16' if nm[0] == 'w' else 'f32'} {shp}")
+            laws[nm] = law
+        nodes += [f"node a0_{i} = conv2d({cur}, w1_{i})", f"node a1_{i} = mul(a0_{i}, s1_{i})", f"node a2_{i} = add(a1_{i}, b1_{i})",
+                  f"node a3_{i} = relu(a2_{i})", f"node a4_{i} = cast_bf16(a3_{i})",
+                  f"node d0_{i} = conv2d(a4_{i}, w2_{i}, stride={2 if last else 1}, pad=1, groups={e})", f"node d1_{i} = mul(d0_{i}, s2_{i})",
+                  f"node d2_{i} = add(d1_{i}, b2_{i})", f"node d3_{i} = relu(d2_{i})", f"node d4_{i} = cast_bf16(d3_{i})",
+                  f"node p0_{i} = conv2d(d4_{i}, w3_{i})", f"node p1_{i} = mul(p0_{i}, s3_{i})", f"node p2_{i} = add(p1_{i}, b3_{i})"]
+        if last:
+            nodes.append(f"node y = cast_bf16(p2_{i})")
+        else:
+            nodes += [f"node r_{i} = add(p2_{i}, {cur})", f"node o_{i} = cast_bf16(r_{i})"]
+            cur = f"o_{i}"
+    return "\n".join(lines + nodes + ["output y bf16"]) + "\n", laws
+
+
+def resnext_block(n=32, c=256, h=28, w=28, width=128, groups=32):
+    """A bottleneck block with a grouped 3x3 convolution in the style of ResNeXt: 1x1 to `width` channels -> BN -> ReLU,
+    3x3 with `groups` groups -> BN -> ReLU, 1x1 back to `c` channels -> BN, plus the block input, ReLU."""
+    spec = f"""hct 1
+input x  bf16 [{n},{c},{h},{w}]
+input w1 bf16 [{width},{c},1,1]
+input s1 f32  [{width},1,1]
+input b1 f32  [{width},1,1]
+input w2 bf16 [{width},{width // groups},3,3]
+input s2 f32  [{width},1,1]
+input b2 f32  [{width},1,1]
+input w3 bf16 [{c},{width},1,1]
+input s3 f32  [{c},1,1]
+input b3 f32  [{c},1,1]
+node  a0 = conv2d(x, w1)
+node  a1 = mul(a0, s1)
+node  a2 = add(a1, b1)
+node  a3 = relu(a2)
+node  a4 = cast_bf16(a3)
+node  g0 = conv2d(a4, w2, pad=1, groups={groups})
+node  g1 = mul(g0, s2)
+node  g2 = add(g1, b2)
+node  g3 = relu(g2)
+node  g4 = cast_bf16(g3)
+node  p0 = conv2d(g4, w3)
+node  p1 = mul(p0, s3)
+node  p2 = add(p1, b3)
+node  p3 = add(p2, x)
+node  y  = relu(p3)
+output y bf16
+"""
+    laws = {"x": _n(), "w1": _n(math.sqrt(2.0 / c)), "s1": _u(0.5, 1.5), "b1": _n(0.1),
+            "w2": _n(math.sqrt(2.0 / (9 * (width // groups)))), "s2": _u(0.5, 1.5), "b2": _n(0.1),
+            "w3": _n(math.sqrt(1.0 / width)), "s3": _u(0.5, 1.5), "b3": _n(0.1)}
+    return spec, laws
+
+
 def topk_bias_relu(r=8192, c=4096, k=32):
     """A logic-intensive operator with fused consumers (Table 1): the k largest values of every row, plus a bias, through ReLU."""
     spec = f"""hct 1
@@ -228,6 +296,8 @@ CONFIGS = {
     "dwconv_bn_relu": (dwconv_bn_relu, {}),
     "topk_bias_relu": (topk_bias_relu, {}),
     "mbconv_block": (mbconv_block, {}),
+    "mobilenet_stage": (mobilenet_stage, {}),
+    "resnext_block": (resnext_block, {}),
 }
 
 
