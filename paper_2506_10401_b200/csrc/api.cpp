@@ -338,7 +338,7 @@ hct_status_t hct_graph_autotune(const char* spec, size_t spec_len, int device, c
       cands.insert(cands.begin(), c);
   if (has_conv)
     for (const char* c : {"conv_flat=1", "conv_nstg=4", "conv_nstg=5", "conv_no_tma_store=1", "conv_no_direct=1", "conv_no_direct=1;conv_no_halo=1", "dw_p=4",
-                          "dw_p=4;dw_cta=256", "dw_p=8;dw_cta=64", "dw_pair=1", "conv_nbuf=3", "conv_pw_warps=8", "conv_no_pointwise=1"})
+                          "dw_p=4;dw_cta=256", "dw_p=8;dw_cta=64", "dw_pair=1", "conv_nbuf=3", "conv_pw_warps=8", "conv_pw_warps=16", "conv_no_pointwise=1"})
       cands.push_back(c);
 
   const Driver* d = nullptr;

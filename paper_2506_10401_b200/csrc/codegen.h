@@ -72,7 +72,7 @@ struct Tunables {
   bool topk_no_select = false;     // row_topk: full bitonic sort of the row even for small k
   bool conv_phase = false;         // strided convolutions: a stride-phase view wherever one exists, not only for rows too wide for a strided box
   bool conv_no_direct = false;     // always take the NHWC pre-pass, even when the convolution could read NCHW itself
-  int conv_pw_warps = 0;           // 1x1 convolution as a per-image GEMM: epilogue warps (0: rule, 16; or 8)
+  int conv_pw_warps = 0;           // 1x1 convolution as a per-image GEMM: epilogue warps (0: by rule; 8 or 16)
   bool conv_no_pointwise = false;  // 1x1 convolutions take the general schedules instead of the per-image GEMM
   bool simt_only = false;
   // Failure-path testing: the GEMM producer never issues its loads, so the consumer's bounded wait runs out

@@ -7,9 +7,9 @@
 // together and find them in L2).  Warp 0 loads a stage per block of 64 input channels (one weight box,
 // four pixel boxes of 64 pixels x 64 channels; channels past C and pixels past HW read zeros), warp 1
 // issues tcgen05.mma into one of two accumulators in tensor memory, HCT_EPW epilogue warps (8 or 16: two or
-// four per lane quarter, 128 or 64 pixels each) drain the other; a tile has little MMA work, so the step time
-// is the latency of an epilogue chunk times the chunks a warp takes.  A single bf16 result leaves through shared memory and TMA
-// stores of 32 channels x 32 pixels; anything else is stored by the generated epilogue itself.
+// four per lane quarter, 128 or 64 pixels each) drain the other; a tile has little MMA work, so the step time is
+// set by the epilogue.  A single bf16 result leaves through shared memory and TMA stores of 32 channels x 64
+// pixels; anything else is stored by the generated epilogue itself.
 //
 // Defined by the generator: HCT_NB_IMG, HCT_C, HCT_KO, HCT_HW, HCT_STAGES, HCT_EPW, HCT_TMA_STORE, HCT_STATUS_SLOT,
 // HCT_KERNEL_NAME, HctParams, hct_epilogue_run() or (HCT_TMA_STORE) hct_epilogue_vals().
@@ -127,44 +127,47 @@ extern "C" __global__ void __launch_bounds__(64 + 32 * HCT_EPW, 1) HCT_KERNEL_NA
     const int q = warp & 3, part = (warp - 2) >> 2;
     int acc = 0;
     hct_u32 acc_phase = 0;
-#if HCT_TMA_STORE
-    unsigned ostep = 0;
-#endif
     for (long long tile = blockIdx.x; tile < HCT_TILES; tile += gridDim.x) {
       const HctPwTile t = hct_pw_tile(tile);
       hct_mbar_wait(tfull0 + 8 * acc, acc_phase, &failed, status, 4);
       hct_tc_fence_after();
       const int k = t.mbk * HCT_BM + q * 32 + lane;
       const bool live = t.mbk * HCT_BM + q * 32 < HCT_KO;   // this warp's 32 channels exist (warp-uniform)
-#pragma unroll 1
-      for (int c = part * HCT_CPW; c < (part + 1) * HCT_CPW; ++c) {
-        const int pix0 = t.nb * HCT_BN + c * 32;
-        const int ncols = HCT_HW - pix0 < 32 ? HCT_HW - pix0 : 32;
-        if (ncols <= 0 || !live) break;
-        float v[32];
-        hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * HCT_BN + c * 32, v);
 #if HCT_TMA_STORE
-        // 32 channels x 32 pixels leave through shared memory and one TMA store (pixels past HW and channels
-        // past KO are clipped by the copy).  Row = channel (64 bytes), 64-byte swizzle: 16-byte piece j of
-        // row i sits at piece j ^ ((i >> 1) & 3).  Two slots per warp: a slot is rewritten only after the
-        // store issued from it two steps ago has read it.
-        float o[32];
-        if (k < HCT_KO) {
-          hct_epilogue_vals(hct_p, v, (long long)t.n * HCT_KO + k, pix0, ncols, o);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) o[j] = 0.0f;
-        }
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+      // 32 channels x 64 pixels (two chunks) leave through shared memory and one TMA store; pixels past HW and
+      // channels past KO are clipped by the copy.  Row = channel (128 bytes), 128-byte swizzle: 16-byte piece p of
+      // row i sits at piece p ^ (i & 7), which also keeps the writes of neighbouring lanes in different banks.
+      // Rows of 128 bytes matter: the copy engine spends its time per row, and with 64-byte rows the stores of a
+      // tile took longer than everything else in it.  One slot per warp, rewritten once the store issued from
+      // it (a tile ago) has read it.
+      const hct_u32 o_slot = smem_base + HCT_RING_O_OFF + (hct_u32)((warp - 2) * 4096);
+#pragma unroll 1
+      for (int cp = 0; cp < HCT_CPW / 2; ++cp) {
+        const int c0 = part * HCT_CPW + cp * 2;
+        const int pix0 = t.nb * HCT_BN + c0 * 32;
+        if (HCT_HW - pix0 <= 0 || !live) break;
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         __syncwarp();
-        const hct_u32 o_slot = smem_base + HCT_RING_O_OFF + (hct_u32)(((warp - 2) * 2 + (ostep & 1)) * 2048);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const hct_u32 dst = o_slot + (hct_u32)lane * 64u + (((hct_u32)j ^ (((hct_u32)lane >> 1) & 3u)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(hct_pack_bf16x2(o[8 * j], o[8 * j + 1])),
-                       "r"(hct_pack_bf16x2(o[8 * j + 2], o[8 * j + 3])), "r"(hct_pack_bf16x2(o[8 * j + 4], o[8 * j + 5])),
-                       "r"(hct_pack_bf16x2(o[8 * j + 6], o[8 * j + 7]))
-                       : "memory");
+        for (int cc = 0; cc < 2; ++cc) {
+          const int ncols = HCT_HW - (pix0 + cc * 32) < 32 ? HCT_HW - (pix0 + cc * 32) : 32;
+          if (ncols <= 0) break;
+          float v[32], o[32];
+          hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * HCT_BN + (c0 + cc) * 32, v);
+          if (k < HCT_KO) {
+            hct_epilogue_vals(hct_p, v, (long long)t.n * HCT_KO + k, pix0 + cc * 32, ncols, o);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = 0.0f;
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const hct_u32 dst = o_slot + (hct_u32)lane * 128u + (((hct_u32)(cc * 4 + j) ^ ((hct_u32)lane & 7u)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(hct_pack_bf16x2(o[8 * j], o[8 * j + 1])),
+                         "r"(hct_pack_bf16x2(o[8 * j + 2], o[8 * j + 3])), "r"(hct_pack_bf16x2(o[8 * j + 4], o[8 * j + 5])),
+                         "r"(hct_pack_bf16x2(o[8 * j + 6], o[8 * j + 7]))
+                         : "memory");
+          }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
@@ -174,11 +177,18 @@ extern "C" __global__ void __launch_bounds__(64 + 32 * HCT_EPW, 1) HCT_KERNEL_NA
                        : "memory");
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
-        ++ostep;
-#else
-        if (k < HCT_KO) hct_epilogue_run(hct_p, v, (long long)t.n * HCT_KO + k, pix0, ncols);
-#endif
       }
+#else
+#pragma unroll 1
+      for (int c = part * HCT_CPW; c < (part + 1) * HCT_CPW; ++c) {
+        const int pix0 = t.nb * HCT_BN + c * 32;
+        const int ncols = HCT_HW - pix0 < 32 ? HCT_HW - pix0 : 32;
+        if (ncols <= 0 || !live) break;
+        float v[32];
+        hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * HCT_BN + c * 32, v);
+        if (k < HCT_KO) hct_epilogue_run(hct_p, v, (long long)t.n * HCT_KO + k, pix0, ncols);
+      }
+#endif
       hct_tc_fence_before();
       hct_mbar_arrive(tempty0 + 8 * acc);
       acc ^= 1;
