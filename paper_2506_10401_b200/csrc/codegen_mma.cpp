@@ -149,7 +149,12 @@ struct EpiGen {
         << nd.name << "\n";
     }
     for (auto& st : grp.stores) {
-      const std::string val = st.node == anchor ? "acc[j]" : "e" + std::to_string(st.node);
+      std::string val = st.node == anchor ? "acc[j]" : "e" + std::to_string(st.node);
+      // A cast_bf16 stored as bf16: the store rounds (to nearest even, once), so the node's own rounding and the
+      // widening back to fp32 are skipped for the stored copy.
+      const Node& sn = g.nodes[st.node];
+      if (st.dtype == BF16 && sn.op == "cast_bf16" && st.node != anchor && !sn.args[0].is_literal() && p.group_of[sn.args[0].node] == gi)
+        val = sn.args[0].node == anchor ? "acc[j]" : "e" + std::to_string(sn.args[0].node);
       if (!vals_only && p.partial_cols[st.node] > 0 && !st.to_output)
         f << "    if (j < ncols) ps" << st.node << " += " << val << ";\n";
       else
