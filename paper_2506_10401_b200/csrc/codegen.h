@@ -71,6 +71,7 @@ struct Tunables {
   int conv_flat = 0;               // NCHW-reading conv: tiles of 256 consecutive positions instead of whole rows (0: rule, 1: always, 2: never)
   bool topk_no_select = false;     // row_topk: full bitonic sort of the row even for small k
   bool conv_phase = false;         // strided convolutions: a stride-phase view wherever one exists, not only for rows too wide for a strided box
+  bool conv_ksplit = false;        // NCHW-reading conv: a short last round is cut by output row and by part of the contraction (partial sums meet in scratch); measured slower than the cut by rows alone, so on request only
   bool conv_no_direct = false;     // always take the NHWC pre-pass, even when the convolution could read NCHW itself
   int conv_pw_warps = 0;           // 1x1 convolution as a per-image GEMM: epilogue warps (0: by rule; 8 or 16)
   bool conv_no_pointwise = false;  // 1x1 convolutions take the general schedules instead of the per-image GEMM

@@ -831,7 +831,14 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       const int TH = (direct || halo) ? th_pitch : (int)std::max<int64_t>(1, std::min<int64_t>(256 / WO, std::min<int64_t>(HO, phased ? 256 : 256 / ST)));
       auto align256 = [](int64_t v) { return (v + 255) / 256 * 256; };
       const int64_t x_bytes = (direct || x_nhwc) ? 0 : align256(NB * C * H * W * 2), w_bytes = align256(KO * (G > 1 ? CWP : C) * FR * FS * 2);
-      *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(x_bytes + w_bytes));
+      // On request (conv_ksplit=1; measured slower than the cut by rows alone, whose pieces overlap the other
+      // CTAs' last tiles) a short last round of the NCHW-reading kernel is split by output row and by (channel
+      // block, filter row) part of the contraction: 256 arrival counters (zeroed by the pre-pass) and one fp32 slice of
+      // [128 channels][pitch] per piece follow the weight copy in scratch.
+      const int ks_ctrs = 256, ks_max = 160;
+      const bool ksplit = direct && !flat && tun.conv_ksplit && ((C + 63) / 64) * FR > 1;
+      const int64_t ks_bytes = ksplit ? align256(ks_ctrs * 4 + (int64_t)ks_max * 128 * pitch * 4) : 0;
+      *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(x_bytes + w_bytes + ks_bytes));
       auto scratch = [](int64_t off) {
         BufRef r;
         r.kind = BufRef::Scratch;
@@ -850,10 +857,10 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         std::ostringstream src;
         src << "#define HCT_NB_IMG " << NB << "\n#define HCT_C " << C << "\n#define HCT_HW " << H * W << "\n#define HCT_KO " << KO
             << "\n#define HCT_RS " << FR * FS << "\n#define HCT_PREP_X " << ((direct || x_nhwc) ? 0 : 1) << "\n#define HCT_GROUPS " << G << "\n#define HCT_CWP " << CWP
-            << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
-            << skeleton_source("common") << "\nstruct HctParams { void* ptr[4]; };\n" << skeleton_source("conv_prep");
+            << "\n#define HCT_ZERO_WORDS " << (ksplit ? ks_ctrs : 0) << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+            << skeleton_source("common") << "\nstruct HctParams { void* ptr[5]; };\n" << skeleton_source("conv_prep");
         k.source = src.str();
-        k.ptrs = {node_buf(anchor.args[0].node), node_buf(anchor.args[1].node), scratch(0), scratch(x_bytes)};
+        k.ptrs = {node_buf(anchor.args[0].node), node_buf(anchor.args[1].node), scratch(0), scratch(x_bytes), scratch(x_bytes + w_bytes)};
         const bool w_only = direct || x_nhwc;
         const int64_t w_elems = KO * (G > 1 ? CWP : C) * FR * FS;
         int64_t blocks = w_only ? (w_elems / (G > 1 ? 1 : 8) + 255) / 256 : NB * ((C + 63) / 64) * ((H * W + 63) / 64) + (w_elems + 255) / 256;
@@ -876,12 +883,15 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
           << "\n#define HCT_STRIDE " << ST << "\n#define HCT_DIL " << DIL << "\n#define HCT_PHASED " << (phased ? 1 : 0) << "\n#define HCT_HO " << HO << "\n#define HCT_WO " << WO << "\n#define HCT_TH " << TH << "\n#define HCT_TH2 1\n#define HCT_SPLIT "
           << (flat ? 1 : TH) << "\n#define HCT_PITCH " << pitch << "\n#define HCT_NA " << (direct ? n_a : 6) << "\n#define HCT_NBUF " << (direct ? n_buf : 3)
           << "\n#define HCT_FLAT " << (flat ? 1 : 0) << "\n#define HCT_P " << flat_p << "\n#define HCT_OUT_SLOT " << out_slot
-          << "\n#define HCT_NSTG " << n_stg << "\n#define HCT_X_IS_INPUT " << (a.cls == OpClass::Input ? 1 : 0) << "\n#define HCT_TMA_STORE " << (use_tma_store ? 1 : 0) << "\n#define HCT_STAGES " << stages << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
+          << "\n#define HCT_NSTG " << n_stg << "\n#define HCT_X_IS_INPUT " << (a.cls == OpClass::Input ? 1 : 0) << "\n#define HCT_TMA_STORE " << (use_tma_store ? 1 : 0) << "\n#define HCT_STAGES " << stages
+          << "\n#define HCT_KSPLIT " << (ksplit ? 1 : 0) << "\n#define HCT_KS_SLOT " << eg.ptrs.size() << "\n#define HCT_KS_CTRS " << ks_ctrs << "\n#define HCT_KS_MAX " << ks_max
+          << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size() + (ksplit ? 1 : 0)
           << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
       src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[" << (phased ? 1 + 2 * ST : use_tma_store ? 3 : direct ? 2 : 3)
-          << "]; void* ptr[" << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source(direct ? "conv_tc_nchw" : halo ? "conv_tc_halo" : "conv_tc");
+          << "]; void* ptr[" << eg.ptrs.size() + (ksplit ? 2 : 1) << "]; };\n" << epi << skeleton_source(direct ? "conv_tc_nchw" : halo ? "conv_tc_halo" : "conv_tc");
       k.source = src.str();
       k.ptrs = eg.ptrs;
+      if (ksplit) k.ptrs.push_back(scratch(x_bytes + w_bytes));
       k.wants_status = true;
       TmaDesc tw;
       tw.buf = scratch(x_bytes);

@@ -41,6 +41,7 @@ const Knob kKnobs[] = {
     {"conv_no_halo", nullptr, 0, &Tunables::conv_no_halo},
     {"conv_no_tma_store", nullptr, 0, &Tunables::conv_no_tma_store},
     {"conv_no_direct", nullptr, 0, &Tunables::conv_no_direct},
+    {"conv_ksplit", nullptr, 0, &Tunables::conv_ksplit},
     {"conv_no_pointwise", nullptr, 0, &Tunables::conv_no_pointwise},
     {"conv_pw_warps", &Tunables::conv_pw_warps, 0, nullptr},
     {"conv_phase", nullptr, 0, &Tunables::conv_phase},

@@ -6,7 +6,11 @@
 // fills its pixel pipeline while the weights are being rearranged.
 // Defined by the generator: HCT_NB_IMG, HCT_C, HCT_HW (H*W), HCT_KO, HCT_RS (R*S), HCT_PREP_X, HCT_GROUPS, HCT_CWP (grouped only),
 // HctParams, HCT_KERNEL_NAME.
-// Pointer slots: 0 = X (NCHW), 1 = Wt (KCRS), 2 = X as NHWC, 3 = Wt as RSKC.
+// Pointer slots: 0 = X (NCHW), 1 = Wt (KCRS), 2 = X as NHWC, 3 = Wt as RSKC, 4 = HCT_ZERO_WORDS 32-bit words
+// to clear (the arrival counters of a convolution that splits the contraction of its last round; 0: none).
+#ifndef HCT_ZERO_WORDS
+#define HCT_ZERO_WORDS 0
+#endif
 #define HCT_XT_C ((HCT_C + 63) / 64)
 #define HCT_XT_P ((HCT_HW + 63) / 64)
 #define HCT_X_BLOCKS (HCT_PREP_X ? (long long)HCT_NB_IMG * HCT_XT_C * HCT_XT_P : 0LL)
@@ -44,6 +48,8 @@ extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParam
   hct_pdl_wait();
   const hct_bf16_t* __restrict__ Wt = (const hct_bf16_t*)hct_p.ptr[1];
   hct_bf16_t* __restrict__ Wo = (hct_bf16_t*)hct_p.ptr[3];
+  if (blockIdx.x == 0)
+    for (int i = threadIdx.x; i < HCT_ZERO_WORDS; i += 256) ((unsigned*)hct_p.ptr[4])[i] = 0u;
 #if HCT_GROUPS > 1
   for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < HCT_W_ELEMS; i += (long long)gridDim.x * 256) Wo[i] = hct_w_elem(Wt, i);
   return;

@@ -68,14 +68,26 @@
 #endif
 #define HCT_NBAR (2 * HCT_NA + 2 * HCT_NBUF + 2 * HCT_NSTG + 4)
 
-struct HctConvTile { int n, h0, th, mbk; bool cut; int o0, lo, nrows; };
+#ifndef HCT_KSPLIT
+#define HCT_KSPLIT 0
+#endif
+#if HCT_KSPLIT && HCT_FLAT
+#error "the split of the contraction is built for whole-row tiles only"
+#endif
+#define HCT_KP (HCT_CB * HCT_FR)                         // parts of a contraction split by (channel block, filter row)
+
+// A work item: output rows h0 .. h0 + th - 1 of image n (filters of block mbk), contracted over channel blocks
+// cb_lo .. cb_hi - 1 and filter rows r_lo .. r_hi - 1 (a whole tile: all of them).  `ks`: the item is one part of
+// a split contraction, piece number q; its partial sums go to scratch and the last part to arrive finishes the row.
+struct HctConvTile { int n, h0, th, mbk; bool cut; int o0, lo, nrows; int cb_lo, cb_hi, r_lo, r_hi; bool ks; int q; };
 
 // Tile t of the schedule.  Tiles below `t1` are whole; the rest are pieces of the remaining whole tiles.
-__device__ __forceinline__ HctConvTile hct_conv_tile(long long t, long long t1) {
+__device__ __forceinline__ HctConvTile hct_conv_tile(long long t, long long t1, int ksplit) {
   HctConvTile r;
+  r.cb_lo = 0; r.cb_hi = HCT_CB; r.r_lo = 0; r.r_hi = HCT_FR; r.ks = false; r.q = 0;
 #if HCT_FLAT
   // tile = 256 consecutive positions of one image; `lo` .. `lo + nrows - 1` are the padded input rows its window meets
-  (void)t1;
+  (void)t1; (void)ksplit;
   long long w_ = t;
   r.mbk = (int)(w_ % HCT_MBK); w_ /= HCT_MBK;
   r.o0 = (int)(w_ % HCT_TPI) * 256;
@@ -90,7 +102,17 @@ __device__ __forceinline__ HctConvTile hct_conv_tile(long long t, long long t1) 
   long long whole = t;
   int sub = 0;
   r.cut = t >= t1;
-  if (r.cut) {
+  if (r.cut && ksplit) {
+    // one output row, one (channel block, filter row) part of its contraction
+    const long long q = t - t1;
+    whole = t1 + q / (HCT_SPLIT * HCT_KP);
+    const int rem = (int)(q % (HCT_SPLIT * HCT_KP));
+    sub = rem / HCT_KP;
+    const int part = rem % HCT_KP;
+    r.cb_lo = part / HCT_FR; r.cb_hi = r.cb_lo + 1;
+    r.r_lo = part % HCT_FR; r.r_hi = r.r_lo + 1;
+    r.ks = true; r.q = (int)q;
+  } else if (r.cut) {
     whole = t1 + (t - t1) / HCT_SPLIT;
     sub = (int)((t - t1) % HCT_SPLIT);
   }
@@ -187,6 +209,9 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
   __shared__ unsigned long long bars[HCT_NBAR];
   __shared__ hct_u32 tmem_holder;
   __shared__ int failed;
+#if HCT_KSPLIT
+  __shared__ int ks_last;
+#endif
   const hct_u32 smem_base = (hct_smem_addr(hct_smem_raw) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   unsigned int* status = (unsigned int*)hct_p.ptr[HCT_STATUS_SLOT];
@@ -196,9 +221,21 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
   const hct_u32 tfull0 = sempty0 + 8 * HCT_NSTG, tempty0 = tfull0 + 16;
 
   // schedule: whole tiles for as many full rounds over the grid as there are, the rest cut in pieces
+  // A short last round is spread over the grid by output row; with HCT_KSPLIT also by part of the
+  // contraction, when the pieces fit the grid and the scratch slices (a piece then costs a few MMA
+  // instructions instead of a whole K loop, but its partial sums travel through scratch).
   long long t1 = HCT_FULL_TILES, n_tiles = HCT_FULL_TILES;
+  int ksplit = 0;
   {
     const long long rest = HCT_FULL_TILES % gridDim.x;
+#if HCT_KSPLIT
+    const long long pieces = rest * HCT_SPLIT * HCT_KP;
+    if (rest > 0 && HCT_KP > 1 && pieces <= (long long)gridDim.x && pieces <= HCT_KS_MAX) {
+      t1 = HCT_FULL_TILES - rest;
+      n_tiles = t1 + pieces;
+      ksplit = 1;
+    } else
+#endif
     if (HCT_SPLIT > 1 && rest > 0 && rest * HCT_SPLIT <= (long long)gridDim.x) {
       t1 = HCT_FULL_TILES - rest;
       n_tiles = t1 + rest * HCT_SPLIT;
@@ -244,10 +281,10 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
       int sa = 0;
       hct_u32 pa = 0;
       for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-        const HctConvTile t = hct_conv_tile(tile, t1);
+        const HctConvTile t = hct_conv_tile(tile, t1, ksplit);
         if (t.th == 0) continue;
-        for (int cb = 0; cb < HCT_CB; ++cb)
-          for (int tap = 0; tap < HCT_FR * HCT_FS; ++tap) {
+        for (int cb = t.cb_lo; cb < t.cb_hi; ++cb)
+          for (int tap = t.r_lo * HCT_FS; tap < t.r_hi * HCT_FS; ++tap) {
             hct_mbar_wait(aempty0 + 8 * sa, pa ^ 1u, &failed, status, 5);
             hct_mbar_expect_tx(afull0 + 8 * sa, HCT_A_BYTES);
             hct_tma_load_2d(smem_base + sa * HCT_A_BYTES, &hct_p.tmap[0], cb * 64, tap * HCT_KO + t.mbk * HCT_BM, afull0 + 8 * sa);
@@ -261,7 +298,7 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
       int sa = 0, sb = 0, acc = 0;
       hct_u32 pa = 0, pb = 0, acc_phase = 0;
       for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-        const HctConvTile t = hct_conv_tile(tile, t1);
+        const HctConvTile t = hct_conv_tile(tile, t1, ksplit);
         if (t.th == 0) continue;
         // bf16 x bf16 -> fp32, both operands K-major, M = 128, N = rows of this tile times the pitch
 #if HCT_FLAT
@@ -273,11 +310,11 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
         hct_mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, &failed, status, 2);
         hct_tc_fence_after();
         const hct_u32 d_tmem = tmem_base + acc * 256;
-        for (int cb = 0; cb < HCT_CB; ++cb) {
+        for (int cb = t.cb_lo; cb < t.cb_hi; ++cb) {
           hct_mbar_wait(bfull0 + 8 * sb, pb, &failed, status, 3);
           hct_tc_fence_after();
           const hct_u32 b_addr = smem_base + HCT_RING_B_OFF + sb * HCT_B_BYTES;
-          for (int r = 0; r < HCT_FR; ++r)
+          for (int r = t.r_lo; r < t.r_hi; ++r)
             for (int s = 0; s < HCT_FS; ++s) {
               hct_mbar_wait(afull0 + 8 * sa, pa, &failed, status, 6);
               hct_tc_fence_after();
@@ -287,10 +324,10 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
 #if HCT_FLAT
               const hct_u64 b_desc0 = hct_smem_desc(b_addr + (r * HCT_P + s) * 128, 16, 1024);
 #else
-              const hct_u64 b_desc0 = hct_smem_desc(b_addr + (r * HCT_PITCH + s) * 128, 16, 1024);
+              const hct_u64 b_desc0 = hct_smem_desc(b_addr + ((r - t.r_lo) * HCT_PITCH + s) * 128, 16, 1024);   // the buffer starts at input row h0 - pad + r_lo
 #endif
 #pragma unroll
-              for (int kk = 0; kk < 4; ++kk) hct_mma_f16(d_tmem, a_desc0 + kk * 2, b_desc0 + kk * 2, idesc, (cb | r | s | kk) != 0);
+              for (int kk = 0; kk < 4; ++kk) hct_mma_f16(d_tmem, a_desc0 + kk * 2, b_desc0 + kk * 2, idesc, ((cb - t.cb_lo) | (r - t.r_lo) | s | kk) != 0);
               hct_mma_commit(aempty0 + 8 * sa);
               if (++sa == HCT_NA) { sa = 0; pa ^= 1u; }
             }
@@ -312,7 +349,7 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
 #endif
     hct_pdl_wait();   // epilogue operands may come from earlier kernels of the graph
     for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-      const HctConvTile t = hct_conv_tile(tile, t1);
+      const HctConvTile t = hct_conv_tile(tile, t1, ksplit);
       if (t.th == 0) continue;
       hct_mbar_wait(tfull0 + 8 * acc, acc_phase, &failed, status, 4);
       hct_tc_fence_after();
@@ -326,14 +363,8 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
       for (int c = part; c < 8; c += last_tile ? 4 : 2)
         hct_flat_chunk(hct_p, t, tmem_base + ((hct_u32)(q * 32) << 16) + acc * 256, c, q, lane, smem_base + HCT_RING_O_OFF + (hct_u32)((q * 2 + part) * 2048));
 #else
-      const int chunks = t.th * (HCT_PITCH / 32);
-#pragma unroll 1
-      for (int c = 0; c < chunks; ++c) {
-        const int hh = c / (HCT_PITCH / 32), part = c % (HCT_PITCH / 32);
-        const int ncols = HCT_WO - part * 32 < 32 ? HCT_WO - part * 32 : 32;   // columns past WO are padding
-        if (ncols <= 0) continue;
-        float v[32];
-        hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * 256 + c * 32, v);
+      // values of one 32-column chunk (row h0 + hh, columns part * 32 ..) -> elementwise consumers -> store
+      auto finish = [&](float (&v)[32], int hh, int part, int ncols) {
 #if HCT_TMA_STORE
         // The 32 channels x 32 pixels of this warp leave through shared memory and one TMA store (columns
         // past WO and channels past KO are clipped by the copy).  Row = channel (64 bytes), 64-byte swizzle:
@@ -370,6 +401,72 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
 #else
         if (k < HCT_KO) hct_epilogue_run(hct_p, v, (long long)t.n * HCT_KO + k, (t.h0 + hh) * HCT_WO + part * 32, ncols);
 #endif
+      };
+#if HCT_KSPLIT
+      if (t.ks) {
+        // Part of a split contraction (one output row).  The partial sums go to this piece's scratch slice
+        // (128 channels x pitch fp32); a counter per row tells the last part to arrive, whose CTA adds the
+        // slices in part order (so the result does not depend on the order of arrival) and finishes the row.
+        unsigned* ctr = (unsigned*)hct_p.ptr[HCT_KS_SLOT];
+        float* slices = (float*)(ctr + HCT_KS_CTRS);
+        const int m = q * 32 + lane;
+#pragma unroll 1
+        for (int part = 0; part < HCT_PITCH / 32; ++part) {
+          if (HCT_WO - part * 32 <= 0) continue;
+          float v[32];
+          hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * 256 + part * 32, v);
+          // slice layout [chunk][group of 4 columns][channel][4]: a warp's 16-byte accesses are 512 contiguous bytes
+          float4* dst = (float4*)(slices + (long long)t.q * (HCT_BM * HCT_PITCH)) + (part * 8) * HCT_BM + m;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) __stcg(dst + j * HCT_BM, make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]));
+        }
+        hct_tc_fence_before();
+        hct_mbar_arrive(tempty0 + 8 * acc);
+        // the four warps' stores are ordered before the counter update by the barrier and one thread's fence
+        // (fences are cumulative); the last part's reads follow the update in the same way
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (warp == 2 && lane == 0) {
+          __threadfence();
+          ks_last = atomicAdd(ctr + t.q / HCT_KP, 1u) == (unsigned)(HCT_KP - 1) ? 1 : 0;
+          __threadfence();
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (*(volatile int*)&ks_last) {
+          const int q0 = t.q - t.q % HCT_KP;
+#pragma unroll 1
+          for (int part = 0; part < HCT_PITCH / 32; ++part) {
+            const int ncols = HCT_WO - part * 32 < 32 ? HCT_WO - part * 32 : 32;
+            if (ncols <= 0) continue;
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = 0.0f;
+#pragma unroll 1
+            for (int pp = 0; pp < HCT_KP; ++pp) {
+              const float4* src = (const float4*)(slices + (long long)(q0 + pp) * (HCT_BM * HCT_PITCH)) + (part * 8) * HCT_BM + m;
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const float4 a = __ldcg(src + j * HCT_BM);
+                v[4 * j] += a.x; v[4 * j + 1] += a.y; v[4 * j + 2] += a.z; v[4 * j + 3] += a.w;
+              }
+            }
+            finish(v, 0, part, ncols);
+          }
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");   // ks_last may be written again
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+        continue;
+      }
+#endif
+      const int chunks = t.th * (HCT_PITCH / 32);
+#pragma unroll 1
+      for (int c = 0; c < chunks; ++c) {
+        const int hh = c / (HCT_PITCH / 32), part = c % (HCT_PITCH / 32);
+        const int ncols = HCT_WO - part * 32 < 32 ? HCT_WO - part * 32 : 32;   // columns past WO are padding
+        if (ncols <= 0) continue;
+        float v[32];
+        hct_tmem_ld32(tmem_base + ((hct_u32)(q * 32) << 16) + acc * 256 + c * 32, v);
+        finish(v, hh, part, ncols);
       }
 #endif   // HCT_FLAT
       hct_tc_fence_before();
@@ -389,14 +486,14 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
       int ss = 0;
       hct_u32 ps = 0;
       for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-        const HctConvTile t = hct_conv_tile(tile, t1);
+        const HctConvTile t = hct_conv_tile(tile, t1, ksplit);
         if (t.th == 0) continue;
 #if HCT_FLAT
         const int nrows = t.nrows, row0 = t.lo - HCT_PAD;
 #else
-        const int nrows = t.th + HCT_FR - 1, row0 = t.h0 - HCT_PAD;
+        const int nrows = t.th + (t.r_hi - t.r_lo) - 1, row0 = t.h0 - HCT_PAD + t.r_lo;
 #endif
-        for (int cb = 0; cb < HCT_CB; ++cb)
+        for (int cb = t.cb_lo; cb < t.cb_hi; ++cb)
           for (int rr = 0; rr < nrows; ++rr) {
             hct_mbar_wait(sempty0 + 8 * ss, ps ^ 1u, &failed, status, 7);
             hct_mbar_expect_tx(sfull0 + 8 * ss, HCT_S_BYTES);
@@ -421,14 +518,14 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
     int ss = 0, sb = 0;
     hct_u32 ps = 0, pb = 0;
     for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-      const HctConvTile t = hct_conv_tile(tile, t1);
+      const HctConvTile t = hct_conv_tile(tile, t1, ksplit);
       if (t.th == 0) continue;
 #if HCT_FLAT
       const int nrows = t.nrows;
 #else
-      const int nrows = t.th + HCT_FR - 1;
+      const int nrows = t.th + (t.r_hi - t.r_lo) - 1;
 #endif
-      for (int cb = 0; cb < HCT_CB; ++cb) {
+      for (int cb = t.cb_lo; cb < t.cb_hi; ++cb) {
         hct_mbar_wait(bempty0 + 8 * sb, pb ^ 1u, &failed, status, 1);
         unsigned char* b_gen = (unsigned char*)smem_gen + HCT_RING_B_OFF + sb * HCT_B_BYTES;
         for (int rr = 0; rr < nrows; ++rr) {
@@ -493,7 +590,7 @@ extern "C" __global__ void __launch_bounds__(224 + HCT_NT + 32 * HCT_EPI2, 1) HC
     // follow from how many tiles this CTA has worked on.
     if ((long long)blockIdx.x < n_tiles) {
       const long long ntl = (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x;
-      const HctConvTile t = hct_conv_tile(blockIdx.x + (ntl - 1) * gridDim.x, t1);
+      const HctConvTile t = hct_conv_tile(blockIdx.x + (ntl - 1) * gridDim.x, t1, ksplit);
       const int acc_l = (int)((ntl - 1) & 1);
       const hct_u32 phase_l = (hct_u32)(((ntl - 1) >> 1) & 1);
       const int q = warp & 3, part = 2 + ((warp - 7) >> 2);

@@ -144,15 +144,18 @@ def bf16_deep_chain_check(got, ref):
     return float(np.mean(plain > 1.0)), float(scaled.max())
 
 
-def run_both(spec, laws, seed=0, device=0, schedule=None):
-    """Runs the CUDA library (optionally under a schedule text) and the oracle on the same seeded inputs.
+def run_both(spec, laws, seed=0, device=0, schedule=None, runs=1):
+    """Runs the CUDA library (optionally under a schedule text; `runs` times in a row on the same workspace, keeping
+    the last result) and the oracle on the same seeded inputs.
     Returns (list of GPU outputs as float64 arrays, list of oracle outputs with their error bounds, FusedGraph)."""
     import torch
     import paper_2506_10401_b200 as hct
     t = configs.draw_inputs(spec, laws, seed)
     ref = oracle_reference(spec, oracle_inputs(spec, t))
     g = hct.FusedGraph(spec, device, schedule=schedule)
-    outs = g.run(to_device(spec, t, f"cuda:{device}"))
+    dev_inputs = to_device(spec, t, f"cuda:{device}")
+    for _ in range(runs):
+        outs = g.run(dev_inputs)
     torch.cuda.synchronize(device)
     g.status()
     got = [to_numpy64(o) for o in outs]

@@ -278,6 +278,35 @@ def test_conv_flat_tiles(kw):
     np.testing.assert_array_equal(got[0], want[0])
 
 
+@pytest.mark.parametrize("kw,out", [
+    (dict(n=11, c=128, h=56, w=56, k=128), "bf16"),                    # 154 tiles: 6 left over, 6 parts per row
+    (dict(n=11, c=64, h=56, w=56, k=128), "f32"),                      # one channel block: 3 parts; fp32 result without TMA stores
+    (dict(n=15, c=192, h=40, w=56, k=128), "bf16"),                    # three channel blocks: 9 parts
+    (dict(n=19, c=64, h=30, w=56, k=256), "bf16"),                     # two filter blocks, last tile of an image two rows high
+    (dict(n=15, c=72, h=17, w=48, k=130, ksize=5, pad=2), "bf16"),     # 5x5 filter, ragged channel and filter blocks: 10 parts
+])
+def test_conv_last_round_split_by_part_of_the_contraction(kw, out):
+    """Schedule conv_ksplit=1: with a few tiles more than a multiple of the grid, the left-over rows are cut by (channel
+    block, filter row) part; partial sums meet in scratch and the last part to arrive finishes the row.  Shapes chosen for a grid of 148
+    CTAs; the chain within the bf16 tolerance and the bare convolution bit for bit on integer inputs, twice in a row
+    on one workspace (every run clears the arrival counters), and the same under the default schedule."""
+    import torch
+    if torch.cuda.get_device_properties(0).multi_processor_count != 148:
+        pytest.skip("tile counts chosen for 148 SMs")
+    spec, laws = configs.get_config("c4_conv_bn_relu_bf16", **kw)
+    got, want, g = parity.run_both(spec, laws, schedule="conv_ksplit=1")
+    assert "NCHW read directly" in g.plan
+    assert parity.bf16_violation(got[0], want[0]) <= 1.0
+    ks, pad = kw.get("ksize", 3), kw.get("pad", 1)
+    tail = "node z = cast_bf16(y)\noutput z bf16\n" if out == "bf16" else "output y f32\n"
+    spec = (f"hct 1\ninput x bf16 [{kw['n']},{kw['c']},{kw['h']},{kw['w']}]\ninput w bf16 [{kw['k']},{kw['c']},{ks},{ks}]\n"
+            f"node y = conv2d(x, w, stride=1, pad={pad})\n" + tail)
+    il = {"kind": "int", "lo": -2, "hi": 2}
+    for schedule in ("conv_ksplit=1", None):
+        got, want, g = parity.run_both(spec, {"x": il, "w": il}, schedule=schedule, runs=2 if schedule else 1)
+        np.testing.assert_array_equal(got[0], want[0])
+
+
 @pytest.mark.parametrize("shape,wshape,attrs", [
     ((2, 64, 28, 30), (96, 64, 3, 3), "stride=2, pad=1"),             # strided pixel boxes straight from the caller's buffer
     ((1, 128, 56, 56), (256, 128, 1, 1), "stride=2, pad=0"),
