@@ -56,6 +56,7 @@ struct Tunables {
   int row_ring_bytes_small = 48 * 1024;  // ring of one small CTA
   bool row_no_reg_rowvec = false;  // keep row vectors of reduction-free chains in shared memory instead of registers
   bool row_no_softmax_ln_fusion = false;  // layer norm after softmax: take the variance with its own reduction
+  bool row_no_packed = false;      // row kernels: one-value arithmetic everywhere (no .f32x2 pairs, no multiply-add folding, special-function reciprocal in sigmoid)
   bool row_no_stage = false;       // load rows straight from global memory instead of through the shared-memory ring
   int row_ring_bytes = 200 * 1024; // shared memory a staged row kernel may spend on resident row vectors plus its prefetch ring
   int gemm_insplit = 0;            // fp32 GEMM splits its operands inside the kernel (one launch, no scratch) when 1; otherwise a split pre-pass runs first

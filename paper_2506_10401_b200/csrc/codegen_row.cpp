@@ -50,6 +50,7 @@ const Knob kKnobs[] = {
     {"row_no_reg_rowvec", nullptr, 0, &Tunables::row_no_reg_rowvec},
     {"row_no_softmax_ln_fusion", nullptr, 0, &Tunables::row_no_softmax_ln_fusion},
     {"row_no_stage", nullptr, 0, &Tunables::row_no_stage},
+    {"row_no_packed", nullptr, 0, &Tunables::row_no_packed},
 };
 }  // namespace
 
@@ -245,6 +246,60 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
   // ---- external operands
   const std::string FORB = "_Pragma(\"unroll\") for (int b = 0; b < HCT_B; ++b) ";
   const std::string FORE = "_Pragma(\"unroll\") for (int e = 0; e < HCT_E; ++e) ";
+  // Packed arithmetic: neighbouring elements 2p and 2p + 1 of a thread (same vector) go through .f32x2
+  // instructions, which halves the issue slots of multiply-adds.  Reductions that mask the ragged end of a row
+  // (HCT_HAS) keep the one-value form unless every vector of the row is whole.
+  const std::string FORP = "_Pragma(\"unroll\") for (int p_ = 0; p_ < HCT_E / 2; ++p_) ";
+  const bool packed = V % 2 == 0 && !tun.row_no_packed;
+  const bool packed_full = packed && C % ((int64_t)T * V * NV) == 0;
+  auto half = [](std::string e, bool hi) {
+    const std::string from = "[e]", to = hi ? "[2 * p_ + 1]" : "[2 * p_]";
+    for (size_t at = e.find(from); at != std::string::npos; at = e.find(from, at + to.size())) e.replace(at, from.size(), to);
+    return e;
+  };
+  auto pk = [&](const std::string& e) { return "hct_pk(" + half(e, false) + ", " + half(e, true) + ")"; };
+  auto upk_into = [&](const std::string& value2, const std::string& arr) {
+    return "hct_upk(" + value2 + ", " + arr + "[b][2 * p_], " + arr + "[b][2 * p_ + 1]);";
+  };
+  // uses of every node of this group (arguments anywhere in the graph); a product with a single use that is not
+  // stored can be folded into the sum that consumes it
+  std::vector<int> uses(g.nodes.size(), 0);
+  for (auto& n : g.nodes)
+    for (auto& a : n.args)
+      if (!a.is_literal()) ++uses[a.node];
+  auto stored = [&](int node) {
+    for (auto& st : grp.stores)
+      if (st.node == node) return true;
+    return g.nodes[node].output_index >= 0;
+  };
+  auto foldable_mul = [&](const Operand& a) {
+    return packed && !a.is_literal() && p.group_of[a.node] == gi && !p.is_colv[a.node] && g.nodes[a.node].cls == OpClass::Binary &&
+           g.nodes[a.node].op == "mul" && uses[a.node] == 1 && !stored(a.node);
+  };
+  // Where the special-function unit would be busier than DRAM (16 results per clock and SM against the bytes the
+  // chain moves per element, both at their measured rates), sigmoid takes its reciprocal on the multiply-add
+  // pipe (three Newton steps); elsewhere the extra instructions would only cost issue slots.
+  double xu_ops = 0, bytes_per_elem = 0;
+  for (int ni : grp.nodes) {
+    const Node& nd = g.nodes[ni];
+    if (p.is_colv[ni]) continue;
+    if (nd.op == "sigmoid" || nd.op == "gelu_tanh" || nd.op == "tanh" || nd.op == "div" || nd.op == "sin" || nd.op == "cos") xu_ops += 2;
+    else if (nd.op == "exp" || nd.op == "log" || nd.op == "sqrt" || nd.op == "rsqrt" || nd.op == "reciprocal" || nd.op == "gelu_erf" || nd.cls == OpClass::RowSoftmax) xu_ops += 1;
+  }
+  for (auto& e : grp.ext)
+    if (e.bcast == Bcast::Full) bytes_per_elem += (g.nodes[e.node].cls == OpClass::Input && g.nodes[e.node].dtype == BF16) ? 2 : 4;
+  for (auto& st : grp.stores)
+    if (!p.is_colv[st.node]) bytes_per_elem += st.dtype == BF16 ? 2 : 4;
+  const bool xu_bound = xu_ops * 6.5 >= bytes_per_elem * 4.5;
+  std::vector<char> folded(g.nodes.size(), 0);
+  if (packed)
+    for (int ni : grp.nodes) {
+      const Node& nd = g.nodes[ni];
+      if (nd.cls == OpClass::Binary && !p.is_colv[ni] && (nd.op == "add" || nd.op == "sub")) {
+        if (foldable_mul(nd.args[0])) folded[nd.args[0].node] = 1;
+        else if (foldable_mul(nd.args[1])) folded[nd.args[1].node] = 1;
+      }
+    }
   std::ostringstream pre, loads, issue, fill, hoisted;
   int64_t staged_off = 0, rowvec_off = 0;
   for (size_t k = 0; k < grp.ext.size(); ++k) {
@@ -322,6 +377,25 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
       if (p.is_colv[ni]) {
         for (auto& a : nd.args) av.push_back(rg.ref(a, false));
         b << "      float s" << id << "[HCT_B];\n      " << FORB << "s" << id << "[b] = " << elementwise_call(nd, av, "hct_row0 + b") << ";\n";
+      } else if (folded[ni]) {
+        b << "      // (folded into the sum that consumes it)\n";
+      } else if (packed && nd.cls == OpClass::Binary && (nd.op == "add" || nd.op == "sub" || nd.op == "mul")) {
+        std::string e2;
+        const int fa = nd.op == "mul" ? -1 : (!nd.args[0].is_literal() && folded[nd.args[0].node]) ? 0 : (!nd.args[1].is_literal() && folded[nd.args[1].node]) ? 1 : -1;
+        if (fa >= 0) {
+          // a * b + c, a * b - c, c - a * b as one packed multiply-add
+          const Node& m = g.nodes[nd.args[fa].node];
+          std::string ma = rg.ref(m.args[0], true), mb = rg.ref(m.args[1], true), c = rg.ref(nd.args[1 - fa], true);
+          if (nd.op == "sub" && fa == 0) c = "-(" + c + ")";
+          if (nd.op == "sub" && fa == 1) ma = "-(" + ma + ")";
+          e2 = "hct_fma2(" + pk(ma) + ", " + pk(mb) + ", " + pk(c) + ")";
+        } else {
+          e2 = "hct_" + nd.op + "2(" + pk(rg.ref(nd.args[0], true)) + ", " + pk(rg.ref(nd.args[1], true)) + ")";
+        }
+        b << "      float v" << id << "[HCT_B][HCT_E];\n      " << FORB << FORP << upk_into(e2, "v" + id) << "\n";
+      } else if (packed && nd.cls == OpClass::Unary && (nd.op == "sigmoid" || nd.op == "gelu_tanh")) {
+        b << "      float v" << id << "[HCT_B][HCT_E];\n      " << FORB << FORP
+          << upk_into("hct_" + nd.op + (nd.op == "sigmoid" && !xu_bound ? "2m(" : "2(") + pk(rg.ref(nd.args[0], true)) + ")", "v" + id) << "\n";
       } else {
         for (auto& a : nd.args) av.push_back(rg.ref(a, true));
         b << "      float v" << id << "[HCT_B][HCT_E];\n      " << FORB << FORE << "v" << id << "[b][e] = "
@@ -362,7 +436,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
       std::string a = rg.ref(nd.args[0], true);
       const bool with_q = softmax_feeds_fused_ln(ni);
       b << "      float v" << id << "[HCT_B][HCT_E];\n"
-        << "      float sq" << id << "[HCT_B];\n"
+        << "      float sq" << id << "[HCT_B], kk" << id << "[HCT_B];\n"
         << "      {\n"
         << "        float m_[HCT_B];\n        " << FORB << "{\n          m_[b] = -HCT_INF;\n          " << FORE << "if (HCT_HAS(e)) m_[b] = fmaxf(m_[b], " << a
         << ");\n        }\n"
@@ -371,9 +445,17 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         // which scales the warp's terms by up to 2^(|m| * 1.45 * 2^-24).  Below |m| = 16 that is under 1e-6 and
         // harmless; above, the difference is taken first (exact where it matters, and safe for huge values).
         << "        float d_[HCT_B], q_[HCT_B];\n        " << FORB << "{\n          const float mr_ = m_[b] == -HCT_INF ? 0.0f : m_[b];\n"
-        << "          d_[b] = 0.0f;\n          q_[b] = 0.0f;\n          if (fabsf(mr_) < 16.0f) {\n            const float ml_ = -mr_ * HCT_LOG2E;\n            " << FORE
-        << "{ v" << id << "[b][e] = HCT_HAS(e) ? hct_exp2_fast(fmaf(" << a << ", HCT_LOG2E, ml_)) : 0.0f; d_[b] += v" << id << "[b][e];"
-        << (with_q ? " q_[b] = fmaf(v" + id + "[b][e], v" + id + "[b][e], q_[b]);" : "") << " }\n          } else {\n            " << FORE
+        << "          d_[b] = 0.0f;\n          q_[b] = 0.0f;\n          if (fabsf(mr_) < 16.0f) {\n            const float ml_ = -mr_ * HCT_LOG2E;\n            ";
+      if (packed_full) {
+        // exponent, running sum and running sum of squares on pairs; the two partial sums are added at the end
+        b << "hct_f2 d2_ = hct_pk(0.0f, 0.0f), q2_ = d2_;\n            " << FORP << "{ const hct_f2 t_ = hct_exp2_fast2(hct_fma2(" << pk(a)
+          << ", hct_pk(HCT_LOG2E, HCT_LOG2E), hct_pk(ml_, ml_))); " << "hct_upk(t_, v" << id << "[b][2 * p_], v" << id << "[b][2 * p_ + 1]); d2_ = hct_add2(d2_, t_);"
+          << (with_q ? " q2_ = hct_fma2(t_, t_, q2_);" : "") << " }\n            { float lo_, hi_; hct_upk(d2_, lo_, hi_); d_[b] = lo_ + hi_; hct_upk(q2_, lo_, hi_); q_[b] = lo_ + hi_; }\n";
+      } else {
+        b << FORE << "{ v" << id << "[b][e] = HCT_HAS(e) ? hct_exp2_fast(fmaf(" << a << ", HCT_LOG2E, ml_)) : 0.0f; d_[b] += v" << id << "[b][e];"
+          << (with_q ? " q_[b] = fmaf(v" + id + "[b][e], v" + id + "[b][e], q_[b]);" : "") << " }\n";
+      }
+      b << "          } else {\n            " << FORE
         << "{ v" << id << "[b][e] = HCT_HAS(e) ? hct_exp2_fast((" << a << " - mr_) * HCT_LOG2E) : 0.0f; d_[b] += v" << id << "[b][e];"
         << (with_q ? " q_[b] = fmaf(v" + id + "[b][e], v" + id + "[b][e], q_[b]);" : "") << " }\n          }\n        }\n"
         << "        hct_warp_reduce<false>(d_);\n"
@@ -382,7 +464,16 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         << "        hct_softmax_combine<" << (with_q ? "true" : "false") << ">(m_, d_, q_, f_, hct_cx, HCT_SM_SMEM);\n"
         << (refill_placed ? "" : "@REFILL@")
         << "        " << FORB << "{\n          const float inv_ = hct_rcp_fast(d_[b]);\n          const float k_ = f_[b] * inv_;\n          sq" << id
-        << "[b] = q_[b] * inv_ * inv_;\n          " << FORE << "v" << id << "[b][e] *= k_;\n        }\n"
+        << "[b] = q_[b] * inv_ * inv_;\n          ";
+      // The factor that turns the terms into probabilities is left to a layer normalisation that is the only
+      // reader of this softmax and folds it into its own scaling (one multiply-add per element for both).
+      if (with_q && uses[ni] == 1 && !stored(ni))
+        b << "kk" << id << "[b] = k_;\n";
+      else if (packed)
+        b << FORP << upk_into("hct_mul2(" + pk("v" + id + "[b][e]") + ", hct_pk(k_, k_))", "v" + id) << "\n";
+      else
+        b << FORE << "v" << id << "[b][e] *= k_;\n";
+      b << "        }\n"
         << "      }\n";
     } else if (nd.cls == OpClass::RowLayernorm) {
       std::string a = rg.ref(nd.args[0], true);
@@ -406,9 +497,18 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         // root keeps below 2^-24 / (2 C eps) of the result (the rule applies only when C * eps >= 1/40).
         b << "        " << FORB << "{\n          m_[b] = m_[b] / (float)HCT_C;\n          const float var_ = fmaxf(fmaf(sq" << xin.node
           << "[b], 1.0f / (float)HCT_C, -m_[b] * m_[b]), 0.0f);\n          const float r_ = hct_rsqrt_fast(var_ + " << float_lit(nd.eps) << ");\n          "
-          << FORE << "{ const float d_ = HCT_HAS(e) ? " << a << " - m_[b] : 0.0f; v" << id << "[b][e] = fmaf(d_ * r_, " << ga << ", " << be
-          << "); }\n        }\n"
-          << "      }\n";
+          ;
+        const bool deferred = uses[xin.node] == 1 && !stored(xin.node);   // the softmax left its terms unscaled: kk holds the factor
+        if (deferred && packed_full)
+          b << "const float ka_ = kk" << xin.node << "[b] * r_, kb_ = -m_[b] * r_;\n          " << FORP
+            << upk_into("hct_fma2(hct_fma2(" + pk(a) + ", hct_pk(ka_, ka_), hct_pk(kb_, kb_)), " + pk(ga) + ", " + pk(be) + ")", "v" + id) << "\n        }\n";
+        else if (deferred)
+          b << "const float ka_ = kk" << xin.node << "[b] * r_, kb_ = -m_[b] * r_;\n          " << FORE << "v" << id << "[b][e] = fmaf(fmaf(" << a
+            << ", ka_, kb_), " << ga << ", " << be << ");\n        }\n";
+        else
+          b << FORE << "{ const float d_ = HCT_HAS(e) ? " << a << " - m_[b] : 0.0f; v" << id << "[b][e] = fmaf(d_ * r_, " << ga << ", " << be
+            << "); }\n        }\n";
+        b << "      }\n";
       } else {
         b << "        float q_[HCT_B];\n        " << FORB << "{\n          m_[b] = m_[b] / (float)HCT_C;\n          q_[b] = 0.0f;\n          " << FORE
           << "{ const float d_ = HCT_HAS(e) ? " << a << " - m_[b] : 0.0f; v" << id << "[b][e] = d_; q_[b] = fmaf(d_, d_, q_[b]); }\n        }\n"

@@ -27,17 +27,7 @@
 // fma.rn.f32x2 whose low half belongs to filter k and whose high half to filter k + 1, so pixel, weight and
 // accumulator pairs are formed where the values are produced and nothing has to be shuffled between halves.
 // Each half is an ordinary round-to-nearest fused multiply-add: results equal those of the one-plane form.
-__device__ __forceinline__ unsigned long long hct_pack2(float lo, float hi) {
-  unsigned long long r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void hct_unpack2(unsigned long long v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
-__device__ __forceinline__ unsigned long long hct_fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
-  unsigned long long d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
+// (pair helpers hct_pk, hct_upk, hct_fma2: common.cuh)
 extern "C" __global__ void __launch_bounds__(HCT_CTA) HCT_KERNEL_NAME(const HctParams hct_p) {
   hct_pdl_launch_dependents();
   hct_pdl_wait();
@@ -56,7 +46,7 @@ extern "C" __global__ void __launch_bounds__(HCT_CTA) HCT_KERNEL_NAME(const HctP
     unsigned long long wt[HCT_FR * HCT_FS];
 #pragma unroll
     for (int i = 0; i < HCT_FR * HCT_FS; ++i)
-      wt[i] = hct_pack2(hct_ld1(Wt + (long long)k * (HCT_FR * HCT_FS) + i), hct_ld1(Wt + (long long)(k + 1) * (HCT_FR * HCT_FS) + i));
+      wt[i] = hct_pk(hct_ld1(Wt + (long long)k * (HCT_FR * HCT_FS) + i), hct_ld1(Wt + (long long)(k + 1) * (HCT_FR * HCT_FS) + i));
     unsigned long long acc[HCT_P][8];
 #pragma unroll
     for (int p = 0; p < HCT_P; ++p)
@@ -74,17 +64,17 @@ extern "C" __global__ void __launch_bounds__(HCT_CTA) HCT_KERNEL_NAME(const HctP
         hct_ld_run32<HCT_TA>(xr0 + w0, v0, row_ok ? 8 : 0, true);
         hct_ld_run32<HCT_TA>(xr1 + w0, v1, row_ok ? 8 : 0, true);
 #pragma unroll
-        for (int c = 0; c < 8; ++c) xw[HCT_PAD + c] = hct_pack2(v0[c], v1[c]);
+        for (int c = 0; c < 8; ++c) xw[HCT_PAD + c] = hct_pk(v0[c], v1[c]);
       }
 #pragma unroll
       for (int i = 0; i < HCT_PAD; ++i) {
         const bool ok = row_ok && w0 - HCT_PAD + i >= 0;
-        xw[i] = hct_pack2(ok ? hct_ld1(xr0 + w0 - HCT_PAD + i) : 0.0f, ok ? hct_ld1(xr1 + w0 - HCT_PAD + i) : 0.0f);
+        xw[i] = hct_pk(ok ? hct_ld1(xr0 + w0 - HCT_PAD + i) : 0.0f, ok ? hct_ld1(xr1 + w0 - HCT_PAD + i) : 0.0f);
       }
 #pragma unroll
       for (int i = HCT_PAD + 8; i < HCT_XW; ++i) {
         const bool ok = row_ok && w0 - HCT_PAD + i < HCT_W;
-        xw[i] = hct_pack2(ok ? hct_ld1(xr0 + w0 - HCT_PAD + i) : 0.0f, ok ? hct_ld1(xr1 + w0 - HCT_PAD + i) : 0.0f);
+        xw[i] = hct_pk(ok ? hct_ld1(xr0 + w0 - HCT_PAD + i) : 0.0f, ok ? hct_ld1(xr1 + w0 - HCT_PAD + i) : 0.0f);
       }
 #pragma unroll
       for (int p = 0; p < HCT_P; ++p)
@@ -104,7 +94,7 @@ extern "C" __global__ void __launch_bounds__(HCT_CTA) HCT_KERNEL_NAME(const HctP
 #pragma unroll
         for (int c = 0; c < 32; ++c) a0[c] = a1[c] = 0.0f;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) hct_unpack2(acc[p][c], a0[c], a1[c]);
+        for (int c = 0; c < 8; ++c) hct_upk(acc[p][c], a0[c], a1[c]);
         hct_epilogue_run(hct_p, a0, (long long)plane, (h0 + p) * HCT_WO + w0, 8);
         hct_epilogue_run(hct_p, a1, (long long)plane + 1, (h0 + p) * HCT_WO + w0, 8);
       }

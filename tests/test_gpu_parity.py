@@ -45,6 +45,34 @@ def test_softmax_layernorm_chain_shapes(r, c):
     assert g.num_kernels == 1
 
 
+@pytest.mark.parametrize("schedule", [None, "row_no_packed=1"])
+@pytest.mark.parametrize("body,cols", [
+    # three sigmoids and a softmax on few bytes: the reciprocals run as Newton steps on the multiply-add pipe
+    ("node a = sigmoid(x)\nnode b = sigmoid(a)\nnode c = add(b, v)\nnode d = sigmoid(c)\nnode e = row_softmax(d)\noutput e\noutput d\n", 4096),
+    # products folded into sums in every operand order, and a softmax whose scaling is NOT left to the layer norm (two readers)
+    ("node a = mul(x, v)\nnode b = sub(a, x)\nnode m = mul(b, v)\nnode c = sub(x, m)\nnode p = row_softmax(c)\n"
+     "node l = row_layernorm(p, v, v, eps=1e-5)\nnode o = add(l, p)\noutput o\n", 4096),
+    # ragged rows: pairs for the elementwise part, one-value reductions
+    ("node a = mul(x, v)\nnode b = add(a, v)\nnode g = gelu_tanh(b)\nnode p = row_softmax(g)\nnode l = row_layernorm(p, v, v, eps=1e-5)\noutput l\n", 1000),
+    ("node a = sigmoid(x)\nnode b = mul(a, 3.0)\nnode c = add(b, v)\nnode s = row_sum(c)\noutput c\noutput s\n", 4094),
+])
+def test_packed_pairs_and_one_value_arithmetic_agree_with_the_oracle(body, cols, schedule):
+    spec = f"hct 1\ninput x f32 [70,{cols}]\ninput v f32 [{cols}]\n" + body
+    got, want, g = parity.run_both(spec, {"x": {"kind": "normal", "mean": 0.0, "std": 3.0}, "v": N_}, schedule=schedule)
+    for a, b in zip(got, want):
+        assert parity.f32_violation(a, b) <= 1.0, g.plan
+
+
+def test_sigmoid_far_out_in_both_tails():
+    """Arguments up to +-200: beyond -87.3 the exponential's argument is kept at 126 and the result is below the
+    smallest normal number, as the exact value is; +200 gives exactly one."""
+    spec = "hct 1\ninput x f32 [8,4096]\nnode a = sigmoid(x)\nnode b = sigmoid(a)\nnode c = sigmoid(b)\nnode d = sigmoid(c)\nnode e = sigmoid(d)\noutput a\noutput e\n"
+    got, want, g = parity.run_both(spec, {"x": {"kind": "uniform", "lo": -200.0, "hi": 200.0}})
+    assert "hct_sigmoid2(hct_pk(" in g.kernel_source(0)   # the variant with Newton steps
+    for a, b in zip(got, want):
+        assert parity.f32_violation(a, b) <= 1.0, g.plan
+
+
 def test_two_column_rows():
     spec = "hct 1\ninput x f32 [3,2]\nnode y = row_softmax(x)\nnode s = row_sum(y)\noutput y\noutput s\n"
     check_f32(spec, {"x": N_})
