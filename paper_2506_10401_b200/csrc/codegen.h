@@ -70,6 +70,8 @@ struct Tunables {
   int conv_nstg = 0;               // NCHW-reading conv: slots of the pixel staging ring (0: rule)
   int conv_nbuf = 0;               // NCHW-reading conv: operand buffers (0: rule)
   int conv_flat = 0;               // NCHW-reading conv: tiles of 256 consecutive positions instead of whole rows (0: rule, 1: always, 2: never)
+  bool sort_no_reg = false;        // row_sort: the shared-memory network for every row length (no register / shuffle kernel)
+  bool topk_no_reg = false;        // row_topk for small k: keys in shared memory and a bound found by one warp's bisection (the earlier form)
   bool topk_no_select = false;     // row_topk: full bitonic sort of the row even for small k
   bool conv_phase = false;         // strided convolutions: a stride-phase view wherever one exists, not only for rows too wide for a strided box
   bool conv_ksplit = false;        // NCHW-reading conv: a short last round is cut by output row and by part of the contraction (partial sums meet in scratch); measured slower than the cut by rows alone, so on request only

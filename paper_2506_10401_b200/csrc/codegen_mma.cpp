@@ -314,11 +314,14 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       // small k: radix selection of the k-th largest key, then a sort of the k selected values only
       int64_t KP = 2;
       while (KP < KOUT) KP *= 2;
+      // fp32 rows of up to 8192 values in whole 16-byte vectors, k <= 64: keys stay in registers (see row_topk.cuh)
+      const bool topk_reg = KOUT <= 64 && ta == F32 && C % 4 == 0 && C <= 8192 && !tun.topk_no_reg;
       KernelSpec k;
       k.name = "hct_row_topk_g" + std::to_string(gi);
       std::ostringstream st;
       st << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "\n#define HCT_K " << KOUT << "\n#define HCT_KP " << KP
-         << "\n#define HCT_T 256\n#define HCT_TA " << ctype(ta) << "\n#define HCT_PA " << pa << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+         << "\n#define HCT_T 256\n#define HCT_TA " << ctype(ta) << "\n#define HCT_PA " << pa << "\n#define HCT_TOPK_REG " << (topk_reg ? 1 : 0)
+         << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
          << skeleton_source("common") << "\nstruct HctParams { void* ptr[" << eg.ptrs.size() << "]; };\n" << epi << skeleton_source("row_topk");
       k.source = st.str();
       k.ptrs = eg.ptrs;
@@ -328,6 +331,27 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       k.desc = std::string("row top-k: ") + (KOUT <= 64 ? "bound from per-thread maxima and a 128-slot bitonic network, else " : "") +
                "radix selection of the k-th largest key in shared memory, one CTA per row, then a bitonic network over " + std::to_string(KP) +
                " selected keys";
+      out->push_back(k);
+      return;
+    }
+    if (NP >= 512 && NP <= 16384 && !tun.sort_no_reg) {
+      // rows of 512 to 16384 slots: 16 slots per thread in registers, partners met by shuffles, and by shared-memory
+      // exchanges only across warps (row_sort_reg.cuh)
+      const int64_t TR = NP / 16;
+      KernelSpec k;
+      k.name = "hct_row_sort_g" + std::to_string(gi);
+      std::ostringstream st;
+      st << "#define HCT_R " << R << "LL\n#define HCT_C " << C << "\n#define HCT_NP " << NP << "\n#define HCT_KOUT " << KOUT
+         << "\n#define HCT_DESC " << (anchor.descending ? 1 : 0) << "\n#define HCT_T " << TR << "\n#define HCT_TA " << ctype(ta)
+         << "\n#define HCT_PA " << pa << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
+         << skeleton_source("common") << "\nstruct HctParams { void* ptr[" << eg.ptrs.size() << "]; };\n" << epi << skeleton_source("row_sort_reg");
+      k.source = st.str();
+      k.ptrs = eg.ptrs;
+      const int64_t per_sm = std::max<int64_t>(1, std::min<int64_t>(2048 / TR, 16));
+      k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(R, 148 * per_sm));
+      k.block[0] = (unsigned)TR;
+      k.desc = std::string(anchor.sort_k ? "row top-k" : "row sort") + ": bitonic network over " + std::to_string(NP) +
+               " slots, 16 per thread in registers, shuffles within a warp, shared-memory exchanges across warps, one CTA per row";
       out->push_back(k);
       return;
     }

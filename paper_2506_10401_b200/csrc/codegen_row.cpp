@@ -46,6 +46,8 @@ const Knob kKnobs[] = {
     {"conv_pw_warps", &Tunables::conv_pw_warps, 0, nullptr},
     {"conv_phase", nullptr, 0, &Tunables::conv_phase},
     {"topk_no_select", nullptr, 0, &Tunables::topk_no_select},
+    {"topk_no_reg", nullptr, 0, &Tunables::topk_no_reg},
+    {"sort_no_reg", nullptr, 0, &Tunables::sort_no_reg},
     {"row_no_small_ctas", nullptr, 0, &Tunables::row_no_small_ctas},
     {"row_no_reg_rowvec", nullptr, 0, &Tunables::row_no_reg_rowvec},
     {"row_no_softmax_ln_fusion", nullptr, 0, &Tunables::row_no_softmax_ln_fusion},
