@@ -279,8 +279,8 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
            g.nodes[a.node].op == "mul" && uses[a.node] == 1 && !stored(a.node);
   };
   // Where the special-function unit would be busier than DRAM (16 results per clock and SM against the bytes the
-  // chain moves per element, both at their measured rates), sigmoid and the tanh-form GELU take their reciprocal
-  // on the multiply-add pipe (three Newton steps); elsewhere the extra instructions would only cost issue slots.
+  // chain moves per element, both at their measured rates), sigmoid takes its reciprocal on the multiply-add
+  // pipe (three Newton steps); elsewhere the extra instructions would only cost issue slots.
   double xu_ops = 0, bytes_per_elem = 0;
   for (int ni : grp.nodes) {
     const Node& nd = g.nodes[ni];
@@ -397,7 +397,7 @@ void gen_row_kernel(const Graph& g, const Plan& p, int gi, const Tunables& tun, 
         b << "      float v" << id << "[HCT_B][HCT_E];\n      " << FORB << FORP << upk_into(e2, "v" + id) << "\n";
       } else if (packed && nd.cls == OpClass::Unary && (nd.op == "sigmoid" || nd.op == "gelu_tanh")) {
         b << "      float v" << id << "[HCT_B][HCT_E];\n      " << FORB << FORP
-          << upk_into("hct_" + nd.op + (nd.op == "sigmoid" ? (xu_bound ? "2(" : "2m(") : (xu_bound ? "2n(" : "2(")) + pk(rg.ref(nd.args[0], true)) + ")", "v" + id) << "\n";
+          << upk_into("hct_" + nd.op + (nd.op == "sigmoid" && !xu_bound ? "2m(" : "2(") + pk(rg.ref(nd.args[0], true)) + ")", "v" + id) << "\n";
       } else {
         for (auto& a : nd.args) av.push_back(rg.ref(a, true));
         b << "      float v" << id << "[HCT_B][HCT_E];\n      " << FORB << FORE << "v" << id << "[b][e] = "
