@@ -49,6 +49,7 @@ WORKLOADS = {
     "conv_s2_bn_relu_nhwc": dict(bound="tensor", sample=dict(n=4)),
     "dwconv_bn_relu": dict(bound="hbm", sample=dict(n=8)),
     "topk_bias_relu": dict(bound="hbm", sample=dict(r=2048)),
+    "sort_bias_relu": dict(bound="hbm", sample=dict(r=2048)),
     "mbconv_block": dict(bound="hbm", sample=dict(n=4)),
     # more than one block: three inverted-residual blocks with a stride-2 transition, and a bottleneck with a grouped 3x3
     "mobilenet_stage": dict(bound="hbm", sample=dict(n=2)),

@@ -1004,6 +1004,13 @@ def test_row_topk_when_one_thread_holds_every_large_value():
         np.testing.assert_array_equal(got.astype(np.float64), want)
 
 
+@pytest.mark.parametrize("kw", [dict(r=70, c=4096), dict(r=33, c=1000), dict(r=5, c=8192), dict(r=9, c=300)])
+def test_sort_config_small(kw):
+    """Sort with fused consumers; 512 to 16384 slots take the register kernel, shorter rows the shared-memory one."""
+    spec, laws = configs.get_config("sort_bias_relu", **kw)
+    check_f32(spec, laws)
+
+
 def test_topk_config_small():
     spec, laws = configs.get_config("topk_bias_relu", r=96, c=2048, k=32)
     g = check_f32(spec, laws)

@@ -268,6 +268,20 @@ output t2 f32
     return spec, laws
 
 
+def sort_bias_relu(r=8192, c=4096):
+    """The other logic-intensive operator of Table 1 with fused consumers: every row sorted in ascending order, plus a bias, through ReLU."""
+    spec = f"""hct 1
+input x    f32 [{r},{c}]
+input bias f32 [{c}]
+node  t0 = row_sort(x)
+node  t1 = add(t0, bias)
+node  t2 = relu(t1)
+output t2 f32
+"""
+    laws = {"x": _n(), "bias": _n()}
+    return spec, laws
+
+
 def transpose_bias_relu(r=16384, c=4096):
     """A layout transform with fused consumers (Table 1, "LayoutTransform"): y = relu(x^T + bias)."""
     spec = f"""hct 1
@@ -295,6 +309,7 @@ CONFIGS = {
     "conv_block": (conv_block, {}),
     "dwconv_bn_relu": (dwconv_bn_relu, {}),
     "topk_bias_relu": (topk_bias_relu, {}),
+    "sort_bias_relu": (sort_bias_relu, {}),
     "mbconv_block": (mbconv_block, {}),
     "mobilenet_stage": (mobilenet_stage, {}),
     "resnext_block": (resnext_block, {}),
