@@ -60,6 +60,7 @@ struct Tunables {
   bool row_no_stage = false;       // load rows straight from global memory instead of through the shared-memory ring
   int row_ring_bytes = 200 * 1024; // shared memory a staged row kernel may spend on resident row vectors plus its prefetch ring
   int gemm_insplit = 0;            // fp32 GEMM splits its operands inside the kernel (one launch, no scratch) when 1; otherwise a split pre-pass runs first
+  bool gemm_no_ksplit = false;     // fp32 GEMM with few tiles: never split the contraction over idle SMs
   int gemm_pair = 0;               // bf16 GEMM on CTA pairs (256x256 tiles): 0 by rule (enough tiles for every pair), 1 always, 2 never
   int gemm_bn = 0;                 // output-tile width of the tensor-core GEMMs (0: by rule; else 32..256, clamped to what the kernel takes)
   bool conv_no_halo = false;       // load conv pixels once per tap even when the shared-row schedule applies

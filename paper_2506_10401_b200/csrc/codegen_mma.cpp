@@ -583,8 +583,24 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
     if (da == F32 && db == F32 && K % 4 == 0 && M <= 0x7fffffff && N <= 0x7fffffff && K <= 0x7fffffff) {
       auto align256 = [](int64_t v) { return (v + 255) / 256 * 256; };
       const int64_t a_bytes = a_presplit ? 0 : align256(M * K * 4), b_bytes = align256(K * N * 4);
-      const int64_t off_ahi = 0, off_alo = a_bytes, off_bhi = 2 * a_bytes, off_blo = 2 * a_bytes + b_bytes;
-      *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(2 * a_bytes + 2 * b_bytes));
+      const int64_t off_ahi = 0, off_alo = a_bytes, off_bhi = 2 * a_bytes, off_blo = 2 * a_bytes + b_bytes, off_acc = 2 * a_bytes + 2 * b_bytes;
+      // Problems with far fewer 128 x 128 tiles than SMs split the contraction over the idle SMs (single-CTA kernel
+      // only): an MMA instruction takes about 90 ns whatever its width, so the time of a small product is the
+      // number of k steps of one tile, and narrower tiles do not shorten it.  ks parts of whole 128-element chunks,
+      // none empty; partial tiles meet in an fp32 accumulation tile that the pre-pass clears.
+      int ks = 1;
+      const bool will_pair = tun.gemm_pair == 1 || (tun.gemm_pair == 0 && ((((M + 255) / 256) * ((N + 255) / 256) >= 56 && K >= 512) || ((M + 255) / 256) * ((N + 255) / 256) >= 512) && tun.gemm_bn == 0);
+      {
+        const int64_t tiles128 = ((M + 127) / 128) * ((N + 127) / 128), nch = ((K + 31) / 32 + 3) / 4;
+        if (!will_pair && !tun.gemm_no_ksplit && tun.gemm_bn == 0 && N > 64 && tiles128 * 2 <= 148 && nch >= 8) {   // K >= 1024: measured 1024^3 chains 31.7 -> 29.9 us, 1024 x 4096 x 1024 95 -> 70 us; at K = 256 the clearing, the atomics and the read-back cost more than the shorter loop saves (13.5 -> 16.8 us)
+          const int64_t want = std::min<int64_t>(148 / tiles128, nch);
+          const int64_t cpp = (nch + want - 1) / want;
+          ks = (int)((nch + cpp - 1) / cpp);
+        }
+      }
+      const int64_t ks_tiles = ((M + 127) / 128) * ((N + 127) / 128);
+      const int64_t acc_bytes = ks > 1 ? align256(ks_tiles * 128 * 128 * 4 + ks_tiles * 4) : 0;
+      *scratch_bytes = std::max<size_t>(*scratch_bytes, (size_t)(2 * a_bytes + 2 * b_bytes + acc_bytes));
       auto scratch = [](int64_t off) {
         BufRef r;
         r.kind = BufRef::Scratch;
@@ -602,11 +618,11 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         k.name = "hct_split_tf32_g" + std::to_string(gi);
         std::ostringstream src;
         src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n#define HCT_SPLIT_A " << (a_presplit ? 0 : 1)
-            << "\n#define HCT_KERNEL_NAME " << k.name << "\n"
-            << skeleton_source("common") << "\nstruct HctParams { void* ptr[6]; };\n" << skeleton_source("split_tf32");
+            << "\n#define HCT_ZERO_VEC4 " << acc_bytes / 16 << "LL\n#define HCT_KERNEL_NAME " << k.name << "\n"
+            << skeleton_source("common") << "\nstruct HctParams { void* ptr[7]; };\n" << skeleton_source("split_tf32");
         k.source = src.str();
         k.ptrs = {node_buf(anchor.args[0].node), node_buf(anchor.args[1].node), scratch(off_ahi), scratch(off_alo), scratch(off_bhi),
-                  scratch(off_blo)};
+                  scratch(off_blo), scratch(off_acc)};
         int64_t blocks = (a_presplit ? 0 : (M * K / 4 + 1023) / 1024) + ((K + 31) / 32) * ((N + 31) / 32);
         k.grid[0] = (unsigned)std::max<int64_t>(1, std::min<int64_t>(blocks, 148 * 16));
         k.block[0] = 256;
@@ -619,7 +635,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       // memory per 6 MFLOP, and the kernel runs at the rate L2 delivers them.  They are taken on request only.
       const int bn_max = N > 128 ? 256 : N > 64 ? 128 : N > 32 ? 64 : 32;
       int BN = std::min(bn_max, 128);
-      while (BN > 64 && ((M + 127) / 128) * ((N + BN - 1) / BN) * 2 <= 148) BN /= 2;
+      while (ks == 1 && BN > 64 && ((M + 127) / 128) * ((N + BN - 1) / BN) * 2 <= 148) BN /= 2;
       if (tun.gemm_bn >= 32) BN = std::min(bn_max, tun.gemm_bn >= 256 ? 256 : tun.gemm_bn >= 128 ? 128 : tun.gemm_bn >= 64 ? 64 : 32);
       int stages = BN == 256 ? 2 : BN == 128 ? 3 : BN == 64 ? 4 : 5;
       std::string epi = eg.run_fn(N);
@@ -669,12 +685,14 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       k.name = "hct_gemm_tc_tf32x3_g" + std::to_string(gi);
       std::ostringstream src;
       src << "#define HCT_M " << M << "LL\n#define HCT_N " << N << "LL\n#define HCT_K " << K << "LL\n#define HCT_BN " << BN
-          << "\n#define HCT_STAGES " << stages << "\n#define HCT_TF32X3 1\n#define HCT_STATUS_SLOT " << eg.ptrs.size()
+          << "\n#define HCT_STAGES " << stages << "\n#define HCT_TF32X3 1\n#define HCT_KSPLIT " << ks << "\n#define HCT_KS_SLOT " << eg.ptrs.size()
+          << "\n#define HCT_STATUS_SLOT " << eg.ptrs.size() + (ks > 1 ? 1 : 0)
           << "\n#define HCT_KERNEL_NAME " << k.name << "\n";
       src << skeleton_source("common") << "\n" << skeleton_source("tc_common") << "\nstruct HctParams { HctTensorMap tmap[4]; void* ptr["
-          << eg.ptrs.size() + 1 << "]; };\n" << epi << skeleton_source("gemm_tc");
+          << eg.ptrs.size() + (ks > 1 ? 2 : 1) << "]; };\n" << epi << skeleton_source("gemm_tc");
       k.source = src.str();
       k.ptrs = eg.ptrs;
+      if (ks > 1) k.ptrs.push_back(scratch(off_acc));
       k.wants_status = true;
       for (int i = 0; i < 4; ++i) {
         TmaDesc t;
@@ -696,7 +714,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
         }
         k.tmaps.push_back(t);
       }
-      int64_t tiles = ((M + 127) / 128) * ((N + BN - 1) / BN);
+      int64_t tiles = ((M + 127) / 128) * ((N + BN - 1) / BN) * ks;
       k.block[0] = BN > 128 ? 320 : 192;   // wide tiles: eight epilogue warps
       k.smem_bytes = (unsigned)(stages * (2 * 128 * 128 + 2 * BN * 128) + 1024);
       k.persistent = true;
@@ -704,6 +722,7 @@ void gen_contraction_kernels(const Graph& g, const Plan& p, int gi, const Tunabl
       k.grid[0] = k.max_grid;
       std::ostringstream d;
       d << "gemm tcgen05 tf32x3 128x" << BN << "x32, " << stages << " stages";
+      if (ks > 1) d << ", contraction split " << ks << " ways over idle SMs";
       k.desc = d.str();
       out->push_back(k);
       return;

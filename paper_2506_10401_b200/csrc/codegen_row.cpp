@@ -30,6 +30,7 @@ const Knob kKnobs[] = {
     {"gemm_bn", &Tunables::gemm_bn, 0, nullptr},
     {"gemm_pair", &Tunables::gemm_pair, 0, nullptr},
     {"gemm_insplit", &Tunables::gemm_insplit, 0, nullptr},
+    {"gemm_no_ksplit", nullptr, 0, &Tunables::gemm_no_ksplit},
     {"conv_nstg", &Tunables::conv_nstg, 0, nullptr},
     {"conv_nbuf", &Tunables::conv_nbuf, 0, nullptr},
     {"conv_flat", &Tunables::conv_flat, 0, nullptr},

@@ -39,6 +39,16 @@
 #define HCT_KBC HCT_KB
 #endif
 #define HCT_NCH ((HCT_KB + HCT_KBC - 1) / HCT_KBC)
+// Split of the contraction (TF32 variant, problems with far fewer tiles than SMs): a work item is one of
+// HCT_KSPLIT parts of a tile's K extent, HCT_CPP chunks each (the generator picks HCT_KSPLIT so that no part is
+// empty).  Every part adds its partial tile into an fp32 accumulation tile in scratch (vector atomics, cleared
+// by the split pre-pass) and counts its arrival; the last part to arrive reads the sums back and runs the epilogue.
+// The order of the additions is the order of arrival, so the last bits of a result may differ between runs.
+#ifndef HCT_KSPLIT
+#define HCT_KSPLIT 1
+#endif
+#define HCT_CPP ((HCT_NCH + HCT_KSPLIT - 1) / HCT_KSPLIT)
+#define HCT_ITEMS (HCT_TILES * HCT_KSPLIT)
 #define HCT_NCH_IS_ONE (!HCT_TF32X3)
 #define HCT_MB ((HCT_M + HCT_BM - 1) / HCT_BM)
 #define HCT_NB ((HCT_N + HCT_BN - 1) / HCT_BN)
@@ -58,6 +68,9 @@ extern "C" __global__ void __launch_bounds__(64 + 32 * HCT_EPI_WARPS, 1) HCT_KER
   __shared__ unsigned long long bars[2 * HCT_STAGES + 4];
   __shared__ hct_u32 tmem_holder;
   __shared__ int failed;
+#if HCT_KSPLIT > 1
+  __shared__ int ks_last;
+#endif
   const hct_u32 smem_base = (hct_smem_addr(hct_smem_raw) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   unsigned int* status = (unsigned int*)hct_p.ptr[HCT_STATUS_SLOT];
@@ -95,9 +108,12 @@ extern "C" __global__ void __launch_bounds__(64 + 32 * HCT_EPI_WARPS, 1) HCT_KER
     if (lane == 0) {
       int stage = 0;
       hct_u32 phase = 0;
-      for (long long tile = blockIdx.x; tile < HCT_TILES; tile += gridDim.x) {
+      for (long long item = blockIdx.x; item < HCT_ITEMS; item += gridDim.x) {
+        const long long tile = item / HCT_KSPLIT;
+        const int part = (int)(item % HCT_KSPLIT);
         const int nb = (int)(tile % HCT_NB), mb = (int)(tile / HCT_NB);
-        for (int kb = 0; kb < HCT_KB; ++kb) {
+        const int kb_lo = part * HCT_CPP * HCT_KBC, kb_hi = kb_lo + HCT_CPP * HCT_KBC < HCT_KB ? kb_lo + HCT_CPP * HCT_KBC : HCT_KB;
+        for (int kb = kb_lo; kb < kb_hi; ++kb) {
           hct_mbar_wait(empty0 + 8 * stage, phase ^ 1u, &failed, status, 1);
 #if defined(HCT_FAULT_NEVER_ARRIVE) && HCT_FAULT_NEVER_ARRIVE
           // failure-path test build: nothing ever completes the stage's barrier
@@ -134,8 +150,9 @@ extern "C" __global__ void __launch_bounds__(64 + 32 * HCT_EPI_WARPS, 1) HCT_KER
 #endif
       int stage = 0, acc = 0;
       hct_u32 phase = 0, acc_phase = 0;
-      for (long long tile = blockIdx.x; tile < HCT_TILES; tile += gridDim.x) {
-       for (int ch = 0; ch < HCT_NCH; ++ch) {
+      for (long long item = blockIdx.x; item < HCT_ITEMS; item += gridDim.x) {
+       const int ch_lo = (int)(item % HCT_KSPLIT) * HCT_CPP, ch_hi = ch_lo + HCT_CPP < HCT_NCH ? ch_lo + HCT_CPP : HCT_NCH;
+       for (int ch = ch_lo; ch < ch_hi; ++ch) {
         hct_mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, &failed, status, 2);
         hct_tc_fence_after();
         const hct_u32 d_tmem = tmem_base + acc * HCT_BN;
@@ -181,7 +198,8 @@ extern "C" __global__ void __launch_bounds__(64 + 32 * HCT_EPI_WARPS, 1) HCT_KER
     const int q = warp & 3;
     int acc = 0;
     hct_u32 acc_phase = 0;
-    for (long long tile = blockIdx.x; tile < HCT_TILES; tile += gridDim.x) {
+    for (long long item = blockIdx.x; item < HCT_ITEMS; item += gridDim.x) {
+      const long long tile = item / HCT_KSPLIT;
       const int nb = (int)(tile % HCT_NB), mb = (int)(tile / HCT_NB);
       const long long row = (long long)mb * HCT_BM + q * 32 + lane;
 #if HCT_NCH_IS_ONE
@@ -206,8 +224,9 @@ extern "C" __global__ void __launch_bounds__(64 + 32 * HCT_EPI_WARPS, 1) HCT_KER
       float sum[NCW * 32];
 #pragma unroll
       for (int j = 0; j < NCW * 32; ++j) sum[j] = 0.0f;
+      const int ch_lo = (int)(item % HCT_KSPLIT) * HCT_CPP, ch_hi = ch_lo + HCT_CPP < HCT_NCH ? ch_lo + HCT_CPP : HCT_NCH;
 #pragma unroll 1
-      for (int ch = 0; ch < HCT_NCH; ++ch) {
+      for (int ch = ch_lo; ch < ch_hi; ++ch) {
         hct_mbar_wait(tfull0 + 8 * acc, acc_phase, &failed, status, 4);
         hct_tc_fence_after();
 #pragma unroll
@@ -222,6 +241,40 @@ extern "C" __global__ void __launch_bounds__(64 + 32 * HCT_EPI_WARPS, 1) HCT_KER
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
+#if HCT_KSPLIT > 1
+      {
+        // accumulation tile: 16-byte vector j of chunk c of row r at ((tile * chunks + c) * 8 + j) * 128 + r, so that a
+        // warp's access is 512 contiguous bytes; arrival counters follow the tiles
+        float4* accbuf = (float4*)hct_p.ptr[HCT_KS_SLOT];
+        unsigned* ctr = (unsigned*)(accbuf + HCT_TILES * (HCT_BN / 32) * 8 * HCT_BM);
+        float4* mine = accbuf + (tile * (HCT_BN / 32) + c0) * 8 * HCT_BM + q * 32 + lane;
+#pragma unroll
+        for (int c = 0; c < NCW; ++c)
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            atomicAdd(mine + (c * 8 + j) * HCT_BM, make_float4(sum[c * 32 + 4 * j], sum[c * 32 + 4 * j + 1], sum[c * 32 + 4 * j + 2], sum[c * 32 + 4 * j + 3]));
+        // the epilogue warps' additions are ordered before the count by the barrier and one thread's fence
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * HCT_EPI_WARPS) : "memory");
+        if (warp == 2 && lane == 0) {
+          __threadfence();
+          ks_last = atomicAdd(ctr + tile, 1u) == (unsigned)(HCT_KSPLIT - 1) ? 1 : 0;
+          __threadfence();
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * HCT_EPI_WARPS) : "memory");
+        const bool last = *(volatile int*)&ks_last != 0;
+        if (last) {
+#pragma unroll
+          for (int c = 0; c < NCW; ++c)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float4 a = __ldcg(mine + (c * 8 + j) * HCT_BM);
+              sum[c * 32 + 4 * j] = a.x; sum[c * 32 + 4 * j + 1] = a.y; sum[c * 32 + 4 * j + 2] = a.z; sum[c * 32 + 4 * j + 3] = a.w;
+            }
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * HCT_EPI_WARPS) : "memory");   // ks_last may be written again
+        if (!last) continue;
+      }
+#endif
 #pragma unroll
       for (int c = 0; c < NCW; ++c) {
         const long long col0 = (long long)nb * HCT_BN + (c0 + c) * 32;

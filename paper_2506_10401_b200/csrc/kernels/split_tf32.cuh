@@ -5,7 +5,11 @@
 // operands are K-major.
 // With HCT_SPLIT_A = 0 only B is handled: A's head and tail were written by the kernel that produced A.
 // Defined by the generator: HCT_M, HCT_N, HCT_K (K a multiple of 4), HCT_SPLIT_A, HctParams, HCT_KERNEL_NAME.
-// Pointer slots: 0 = A, 1 = B, 2 = A_hi, 3 = A_lo, 4 = Bt_hi, 5 = Bt_lo.
+// Pointer slots: 0 = A, 1 = B, 2 = A_hi, 3 = A_lo, 4 = Bt_hi, 5 = Bt_lo, 6 = HCT_ZERO_VEC4 16-byte vectors to
+// clear (accumulation tiles and arrival counters of a GEMM that splits its contraction; 0: none).
+#ifndef HCT_ZERO_VEC4
+#define HCT_ZERO_VEC4 0LL
+#endif
 #define HCT_A_BLOCKS (HCT_SPLIT_A ? (HCT_M * HCT_K / 4 + 1023) / 1024 : 0LL)          // 256 threads x 4 vectors
 #define HCT_BT_K ((HCT_K + 31) / 32)
 #define HCT_BT_N ((HCT_N + 31) / 32)
@@ -13,6 +17,8 @@ extern "C" __global__ void __launch_bounds__(256) HCT_KERNEL_NAME(const HctParam
   hct_pdl_launch_dependents();
   hct_pdl_wait();
   __shared__ float tile[32][33];
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < HCT_ZERO_VEC4; i += (long long)gridDim.x * 256)
+    ((float4*)hct_p.ptr[6])[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
   for (long long blk = blockIdx.x; blk < HCT_A_BLOCKS + HCT_BT_K * HCT_BT_N; blk += gridDim.x) {
     if (blk < HCT_A_BLOCKS) {
       const long long nva = HCT_M * HCT_K / 4;

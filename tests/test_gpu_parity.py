@@ -170,6 +170,22 @@ def test_gemm_f32_wide_tiles(m, k, n):
     np.testing.assert_array_equal(parity.to_numpy64(out), parity.oracle_reference(spec, parity.oracle_inputs(spec, t))["t2"])
 
 
+@pytest.mark.parametrize("m,k,n", [(300, 1000, 520), (1024, 1024, 1024), (130, 4096, 136), (257, 1028, 264), (70, 16384, 72)])
+def test_gemm_f32_contraction_split_over_idle_sms(m, k, n):
+    """Few tiles and a deep contraction: the K extent is cut into parts that meet in an accumulation tile in scratch
+    (cleared by the pre-pass on every run).  The chain within the fp32 tolerance, twice in a row on one workspace,
+    and bit for bit on integer inputs (exact in any order of addition); the same shapes without the split."""
+    spec, laws = configs.get_config("c1_gemm_bias_relu_f32", m=m, k=k, n=n)
+    got, want, g = parity.run_both(spec, laws, runs=2)
+    assert "contraction split" in g.plan
+    assert parity.f32_violation(got[0], want[0]) <= 1.0
+    il = {"kind": "int", "lo": -8, "hi": 8}
+    for schedule in (None, "gemm_no_ksplit=1"):
+        got, want, g = parity.run_both(spec, {"a": il, "b": il, "bias": il}, schedule=schedule, runs=2)
+        assert ("contraction split" in g.plan) == (schedule is None)
+        np.testing.assert_array_equal(got[0], want[0])
+
+
 def test_gemm_f32_integer_inputs_are_exact():
     spec, _ = configs.get_config("c1_gemm_bias_relu_f32", m=96, k=160, n=136)
     il = {"kind": "int", "lo": -8, "hi": 8}
